@@ -1,0 +1,299 @@
+/*
+ * hccl.h - C ABI of the B200 collective executor.
+ *
+ * The library follows the paper's "compiled communication" model (Sec. I,
+ * Sec. III-B.2): the host compiles a collective into a complete description
+ * (a work packet made of subgraphs of work-queue elements, WQEs, with their
+ * dependencies) and a small, fixed set of execution units runs it on their
+ * own. Here the execution units are the thread blocks of one persistent
+ * sm_100a kernel launched on a caller-chosen number of SMs (the analogue of the
+ * message engines, Sec. II-A.2), and the per-WQE work is what the near-memory
+ * compute unit does: copies and FP32-internal sums on FP32/BF16/FP16 buffers.
+ *
+ * All ranks are virtual: R send buffers and R receive buffers live in the
+ * memory of ONE GPU. There is no network, no second GPU.
+ *
+ * Conventions
+ *  - Every call returns hccl_status_t; out-parameters are written only on
+ *    HCCL_OK. No exceptions cross this boundary.
+ *  - Pointers named host_* / plain arrays of counts are HOST memory. Pointers
+ *    named dev_*, the entries of sendbufs/recvbufs and the workspace are DEVICE
+ *    memory owned by the caller. The library allocates no device memory and
+ *    creates no streams.
+ *  - A plan owns its host tables. hccl_plan_destroy frees them; it never
+ *    touches device memory.
+ *  - hccl_execute is asynchronous on the given stream. A plan must not be in
+ *    flight twice at once. Device-side failures (timeout, malformed table) never
+ *    trap: they are recorded in the workspace and read back with
+ *    hccl_plan_status after the stream has been synchronised. After a
+ *    device-side failure the plan must be bound again before reuse.
+ *  - Only sum reductions exist (Sec. II-A.2). Element types: FP32, BF16, FP16.
+ */
+#ifndef HCCL_B200_H
+#define HCCL_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HCCL_MAX_RANKS 256 /* the paper's largest job is 256 ranks (Sec. V-A) */
+
+typedef enum {
+    HCCL_OK = 0,
+    HCCL_ERR_INVALID_ARG = 1,
+    HCCL_ERR_DTYPE = 2,
+    HCCL_ERR_COUNT_MISMATCH = 3, /* recvcounts[d][s] != sendcounts[s][d], or shard sizes do not add up */
+    HCCL_ERR_OVERLAP = 4,        /* receive ranges of one rank overlap, or a send buffer aliases a receive buffer */
+    HCCL_ERR_ALIGNMENT = 5,      /* a buffer is not aligned to its element size / workspace not 256-B aligned */
+    HCCL_ERR_WORKSPACE = 6,      /* workspace too small */
+    HCCL_ERR_BUSY = 7,
+    HCCL_ERR_CUDA = 8,           /* a CUDA runtime call failed; see hccl_last_cuda_error() */
+    HCCL_ERR_TIMEOUT = 9,        /* device side: a dependency or WAIT did not come true within timeout_ns */
+    HCCL_ERR_BAD_DESCRIPTOR = 10,/* device side: a table entry failed its checks */
+    HCCL_ERR_NOT_BOUND = 11,     /* execute before bind */
+    HCCL_ERR_HAZARD = 12         /* compile-time check: two conflicting WQEs are not ordered by a dependency */
+} hccl_status_t;
+
+typedef enum { HCCL_FP32 = 0, HCCL_BF16 = 1, HCCL_FP16 = 2 } hccl_dtype_t; /* the NMC's three types, Sec. II-A.2 */
+
+typedef enum {
+    HCCL_ALGO_RING = 0,      /* unidirectional ring, reduce-scatter then all-gather (Sec. III-B.2, Fig. 5) */
+    HCCL_ALGO_ONESHOT = 1,   /* "all-to-all style": every rank reads every peer once (Sec. V-F, PE kernels) */
+    HCCL_ALGO_RING_FUSED = 2 /* the ring's sums in the ring's order, but each chunk's chain collapsed into
+                                one multi-input reduction (cf. NOOP-joined tree reductions, Sec. III-B.2).
+                                Reported as its own algorithm, never as "ring". */
+} hccl_algo_t;
+
+/* Which data mover the executor uses for aligned bulk work. */
+typedef enum {
+    HCCL_ENGINE_AUTO = 0,
+    HCCL_ENGINE_LSU = 1,  /* 128-bit vector loads/stores through registers */
+    HCCL_ENGINE_BULK = 2  /* cp.async.bulk (TMA) global->shared->global with mbarrier pipelining */
+} hccl_engine_t;
+
+/* Ticket order of a reduction plan. */
+#define HCCL_FLAG_LEVEL_MAJOR 1u /* all chains' step t before any chain's step t+1 (max parallelism);
+                                    default is chain-group-major so partials stay in L2 */
+#define HCCL_FLAG_CHECK_HAZARDS 2u /* run the host hazard checker at compile time, fail with HCCL_ERR_HAZARD */
+#define HCCL_FLAG_STAGED_RING 4u /* keep the paper's separate transfer and compute WQEs: COPY the peer's
+                                    partial into this rank's staging slot, then REDUCE (A=A+B). Default fuses
+                                    the pair into one REDUCE that reads the peer's buffer directly. */
+
+/* Options. A zero field means "default". */
+typedef struct {
+    int32_t sm_budget;      /* thread blocks of the persistent executor = "message engines" (default 148) */
+    int32_t engine;         /* hccl_engine_t */
+    uint64_t chunk_bytes;   /* ring pipelining granule inside a shard/chunk, in bytes of the data type (default 2 MiB) */
+    uint64_t tile_bytes;    /* work-item size, bytes of the widest operand (default: chosen from size and sm_budget) */
+    uint64_t timeout_ns;    /* bound on every device-side wait (default 2e9) */
+    uint32_t flags;         /* HCCL_FLAG_* */
+    int32_t chain_group;    /* chains scheduled together in chain-group-major order (default 8) */
+    int32_t threads;        /* threads per block, multiple of 32 (default 512) */
+    int32_t reserved[5];
+} hccl_opts_t;
+
+typedef struct hccl_plan hccl_plan_t;   /* opaque, host-owned: a compiled, cacheable work packet (Sec. V-B) */
+typedef struct hccl_graph hccl_graph_t; /* opaque, host-owned: a work packet under construction */
+
+/* ------------------------------------------------------------------------
+ * Collective planners (Sec. III-B.2 "Data Path"; collectives named in Sec. V-A, V-D).
+ * Each validates its arguments, builds the WQE graph of the chosen schedule and
+ * compiles it. Counts are int64. Nothing here touches the GPU.
+ * ------------------------------------------------------------------------ */
+
+/* AllReduce(sum): every rank r ends with Y_r[i] = round(sum_q X_q[i]), i < count.
+ * RING: chunk c = elements [floor(c*count/R), floor((c+1)*count/R)); reduce-scatter step t has rank
+ * (c+t+2) mod R add its own chunk c to its predecessor's partial, so chunk c is summed as
+ * ((X_{c+1}+X_{c+2})+...)+X_c in FP32 and ends on rank c; all-gather step u copies it to rank c+u+1.
+ * FP32 data keeps partials in the receive buffers; 16-bit data keeps FP32 partials in workspace
+ * scratch and is rounded once, on the last reduce step. ONESHOT: R independent R-input sums in rank
+ * order 0..R-1. Send and receive buffers: count elements each. */
+hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_algo_t algo,
+                                  const hccl_opts_t* opts, hccl_plan_t** out);
+
+/* ReduceScatter(sum): rank r ends with Y_r[j] = round(sum_q X_q[o_r + j]), j < recvcounts[r],
+ * o_r = sum of recvcounts below r. count = elements in every send buffer; recvcounts == NULL means
+ * the floor split of count over R ranks; otherwise sum(recvcounts) must equal count
+ * (HCCL_ERR_COUNT_MISMATCH). Ring only: each shard is cut into granules of opts->chunk_bytes and each
+ * granule is an independent chain of R-1 reductions with FP32 partials in scratch. */
+hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t count, hccl_dtype_t dt,
+                                      hccl_algo_t algo, const hccl_opts_t* opts, hccl_plan_t** out);
+
+/* AllGather(v): Y_r[o_q + j] = X_q[j] for all r, q; sendcounts[q] elements from rank q (NULL: count each).
+ * algo RING copies hop by hop (rank r receives chunk (r-u-1) mod R from rank r-1 at step u);
+ * ONESHOT has every rank read every peer directly. */
+hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t count, hccl_dtype_t dt,
+                                  hccl_algo_t algo, const hccl_opts_t* opts, hccl_plan_t** out);
+
+/* AllToAllv (the collective that dominates recommendation training, Sec. I; its per-peer sizes and
+ * offsets are the metadata of Sec. IV-B.2). All matrices are R x R row-major, in units of rows of
+ * row_elems elements: sendcounts[s*R+d], sdispls[s*R+d] describe X_s; recvcounts[d*R+s], rdispls[d*R+s]
+ * describe Y_d. For every (s,d), k < sendcounts[s][d]:
+ *     row rdispls[d][s]+k of Y_d  =  row sdispls[s][d]+k of X_s      (byte for byte)
+ * and no other byte of any Y is written. sdispls == NULL / rdispls == NULL mean packed (exclusive
+ * prefix sums of the counts). recvcounts == NULL means the transpose of sendcounts; otherwise it must
+ * equal it (HCCL_ERR_COUNT_MISMATCH). Send ranges may overlap or leave gaps; receive ranges of one
+ * rank must not overlap (HCCL_ERR_OVERLAP). Zero counts are legal and cost nothing. */
+hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_t* sdispls,
+                                  const int64_t* recvcounts, const int64_t* rdispls, hccl_dtype_t dt,
+                                  int64_t row_elems, const hccl_opts_t* opts, hccl_plan_t** out);
+
+/* ------------------------------------------------------------------------
+ * Work-packet builder: the paper's own vocabulary (Sec. III-B.2). A work packet is a set of
+ * subgraphs that run in parallel; a subgraph is a list of WQEs issued in order; a WQE is a copy or
+ * sum (the NMC forms S=A+B, A=A+B, B=A+B, A=B), a WAIT/SET on a memory location, or a NOOP that only
+ * carries dependencies. The planners above are built on this; it is public so that schedules and
+ * dependency kinds can be tested directly.
+ * ------------------------------------------------------------------------ */
+typedef enum {
+    HCCL_OP_COPY = 0,     /* dst[0:count) = a[0:count)   count in BYTES, any alignment            (A=B) */
+    HCCL_OP_REDUCE = 1,   /* dst[i] = round(f32(a[i]) + f32(b[i])), count in ELEMENTS; dst may alias a or b
+                             exactly (A=A+B, B=A+B) or be separate (S=A+B) */
+    HCCL_OP_REDUCE_N = 2, /* dst[i] = round(((f32(a_0[i]) + f32(a_1[i])) + ...) + f32(a_{nsrc-1}[i])) where a_k is
+                             buffer a.kind of rank (a.rank + k) mod R at byte offset a.offset */
+    HCCL_OP_WAIT = 3,     /* block until signal slot a.offset compares true against value (+ epoch*value_per_epoch) */
+    HCCL_OP_SET = 4,      /* store value (+ epoch*value_per_epoch) to signal slot dst.offset */
+    HCCL_OP_NOOP = 5      /* nothing; exists to carry dependencies */
+} hccl_op_t;
+
+typedef enum {
+    HCCL_BUF_SEND = 0,    /* X_rank: read-only for the library */
+    HCCL_BUF_RECV = 1,    /* Y_rank */
+    HCCL_BUF_SCRATCH = 2, /* library scratch inside the bound workspace (rank ignored) */
+    HCCL_BUF_SIGNAL = 3,  /* 64-bit signal slots inside the workspace; offset = slot index. They persist across
+                             executions, hence the paper's "monotonic increasing values" */
+    HCCL_BUF_USER_SIGNAL = 4 /* a caller-supplied device uint64 array (hccl_plan_set_user_signals); offset = index */
+} hccl_buf_t;
+
+typedef struct {
+    int32_t kind;   /* hccl_buf_t */
+    int32_t rank;
+    int64_t offset; /* bytes (data buffers) or slot index (signals) */
+} hccl_ref_t;
+
+/* Dependency kinds of Sec. III-B.2, as bit flags on a WQE. */
+#define HCCL_DEP_FENCE 1u     /* the NEXT WQE of this subgraph does not start until this one has completed */
+#define HCCL_DEP_SYNC 2u      /* wait for ALL previous WQEs of this subgraph */
+#define HCCL_DEP_WQE_SYNC 4u  /* wait for the WQE whose id is dep_wqe (any subgraph, must be older) */
+#define HCCL_DEP_RECV_SYNC 8u /* wait for all earlier WQEs of this subgraph that bring data INTO the subgraph's rank */
+#define HCCL_DEP_SEND_SYNC 16u/* wait for all earlier WQEs of this subgraph that read data OUT OF the subgraph's rank
+                                 into another rank (its buffers are released) */
+/* Refinement of WQE_SYNC for pipelining (not a sixth kind): element k of this WQE needs only element k of
+ * dep_wqe, so tile k may start as soon as tile k of dep_wqe is done. Honoured only when both WQEs are cut
+ * into the same number of tiles; otherwise the whole of dep_wqe is waited for. The schedule's author is
+ * responsible for the claim; hccl_plan_check_hazards verifies it tile by tile. */
+#define HCCL_DEP_ELEMENTWISE 32u
+
+typedef enum { HCCL_CMP_EQ = 0, HCCL_CMP_NE = 1, HCCL_CMP_GE = 2, HCCL_CMP_GT = 3, HCCL_CMP_LE = 4, HCCL_CMP_LT = 5 } hccl_cmp_t;
+
+typedef struct {
+    int32_t op;                       /* hccl_op_t */
+    int32_t dtype_dst, dtype_a, dtype_b; /* hccl_dtype_t; ignored by COPY/WAIT/SET/NOOP */
+    hccl_ref_t dst, a, b;
+    int64_t count;                    /* bytes (COPY) or elements (REDUCE, REDUCE_N) */
+    int32_t nsrc;                     /* REDUCE_N only: 1..R */
+    uint32_t dep_flags;               /* HCCL_DEP_* */
+    int64_t dep_wqe;                  /* with HCCL_DEP_WQE_SYNC */
+    int64_t dep_wqe2;                 /* optional second WQE_SYNC target, -1 if unused */
+    int32_t cmp;                      /* WAIT: hccl_cmp_t */
+    int32_t reserved;
+    int64_t tile_count;               /* tile size in units of count; 0 = derived from opts.tile_bytes */
+    uint64_t value, value_per_epoch;  /* WAIT/SET: effective value = value + epoch*value_per_epoch, epoch = 1,2,.. per execute */
+} hccl_wqe_t;
+
+/* R ranks; send_bytes[r] / recv_bytes[r] = declared extent of X_r / Y_r (every WQE is bounds-checked
+ * against them at add time), scratch_bytes = library scratch wanted, n_signals = signal slots. */
+hccl_status_t hccl_graph_create(int R, const int64_t* send_bytes, const int64_t* recv_bytes,
+                                int64_t scratch_bytes, int32_t n_signals, hccl_graph_t** out);
+/* A new subgraph acting for virtual rank `rank` (used by RECV_SYNC/SEND_SYNC). Returns its index. */
+hccl_status_t hccl_graph_add_subgraph(hccl_graph_t*, int rank, int32_t* subgraph);
+/* Append a WQE to a subgraph. Issue order across the packet = order of these calls. *wqe_id gets its id. */
+hccl_status_t hccl_graph_add_wqe(hccl_graph_t*, int32_t subgraph, const hccl_wqe_t* wqe, int64_t* wqe_id);
+/* Lower to descriptors, tiles and synchronisation objects. The graph can be destroyed afterwards. */
+hccl_status_t hccl_graph_compile(const hccl_graph_t*, const hccl_opts_t* opts, hccl_plan_t** out);
+void hccl_graph_destroy(hccl_graph_t*);
+
+/* ------------------------------------------------------------------------
+ * Binding, execution, status (work-packet upload and cached re-enqueue, Sec. V-B, V-C).
+ * ------------------------------------------------------------------------ */
+
+/* Bytes of device workspace the plan needs: tables + counters + signals + FP32 scratch. */
+hccl_status_t hccl_plan_workspace_bytes(const hccl_plan_t*, size_t* bytes);
+
+/* Upload the tables into dev_workspace (256-B aligned, >= workspace bytes) with one host-to-device copy
+ * on `stream` (a cudaStream_t passed as void*), zero the counters, reset the epoch. The workspace must
+ * stay valid and untouched by others while the plan is used. Synchronises the stream before returning. */
+hccl_status_t hccl_plan_bind(hccl_plan_t*, void* dev_workspace, size_t bytes, void* stream);
+
+/* Enqueue one execution: a single kernel launch on `stream`. sendbufs/recvbufs are HOST arrays of R
+ * DEVICE pointers (element-size aligned; 16-B alignment enables the fast paths; misaligned buffers are
+ * handled correctly on a slow path). Send buffers are only read. Receive buffers are written only in
+ * the declared ranges. Returns HCCL_ERR_OVERLAP if any send extent intersects any receive extent
+ * (in-place operation is not supported). */
+hccl_status_t hccl_execute(hccl_plan_t*, const void* const* sendbufs, void* const* recvbufs, void* stream);
+
+/* The same through HOST data: copies each host_send[r] (send extent of rank r) into dev_send[r], executes,
+ * and copies each receive extent back into host_recv[r]; all asynchronous on `stream` (use pinned host
+ * memory for true asynchrony). Device staging buffers are the caller's. */
+hccl_status_t hccl_execute_host(hccl_plan_t*, const void* const* host_send, void* const* host_recv,
+                                void* const* dev_send, void* const* dev_recv, void* stream);
+
+/* Device-triggered execution (Sec. IV-B.3): give the plan a caller-owned device array of uint64 that
+ * HCCL_BUF_USER_SIGNAL refs index; hccl_plan_set_trigger makes every execution (a) hold all work until
+ * user signal slot wait_slot satisfies cmp against wait_value + epoch*wait_per_epoch, and (b) store
+ * set_value + epoch*set_per_epoch into slot set_slot once everything has completed. Pass a negative
+ * slot to disable either half. Must be called before hccl_plan_bind. */
+hccl_status_t hccl_plan_set_user_signals(hccl_plan_t*, void* dev_signals, int64_t n_slots);
+hccl_status_t hccl_plan_set_trigger(hccl_plan_t*, int64_t wait_slot, int32_t cmp, uint64_t wait_value,
+                                    uint64_t wait_per_epoch, int64_t set_slot, uint64_t set_value,
+                                    uint64_t set_per_epoch);
+
+/* After the stream has been synchronised: the device-side verdict of the LAST execution.
+ * *device_status is HCCL_OK, HCCL_ERR_TIMEOUT or HCCL_ERR_BAD_DESCRIPTOR; *detail the tile index involved. */
+hccl_status_t hccl_plan_status(hccl_plan_t*, hccl_status_t* device_status, int64_t* detail);
+
+typedef struct {
+    int64_t n_wqe;            /* WQEs in the packet */
+    int64_t n_tiles;          /* work items the executor dispatches */
+    int64_t n_syncs;          /* device-side dependency counters */
+    int64_t chain_depth;      /* longest dependency chain, in WQEs */
+    int64_t schedule_bytes;   /* sum over WQEs of bytes read + bytes written (what the schedule moves) */
+    int64_t compulsory_bytes; /* every input byte read once + every output byte written once */
+    int64_t scratch_bytes;
+    int64_t send_bytes_total, recv_bytes_total; /* declared extents */
+    int32_t R, sm_budget, threads, engine;
+    int64_t tile_bytes;
+    int64_t epoch;            /* executions enqueued since the last bind */
+} hccl_plan_info_t;
+hccl_status_t hccl_plan_info(const hccl_plan_t*, hccl_plan_info_t* out);
+
+/* Declared extent, in bytes, of rank r's send / receive buffer. */
+hccl_status_t hccl_plan_extents(const hccl_plan_t*, int rank, int64_t* send_bytes, int64_t* recv_bytes);
+
+void hccl_plan_destroy(hccl_plan_t*);
+const char* hccl_status_string(hccl_status_t);
+const char* hccl_last_cuda_error(void); /* text of the last CUDA failure seen by this thread, "" if none */
+int hccl_version(void);
+
+/* ------------------------------------------------------------------------
+ * Plan verification on the host (debugging aids for schedules; never part of hccl_execute).
+ * ------------------------------------------------------------------------ */
+
+/* Hazard check: every pair of work items whose byte ranges intersect with at least one writer must be
+ * ordered by a dependency path. *n_violations = pairs found unordered (0 = clean). Cost grows with the
+ * number of conflicting pairs; meant for small and medium plans. */
+hccl_status_t hccl_plan_check_hazards(const hccl_plan_t*, int64_t* n_violations);
+
+/* Run the compiled tables on HOST buffers in a random dependency-respecting order drawn from `seed`
+ * (seed 0 = ticket order). A schedule debugging aid only: it validates what the planner emitted
+ * without a GPU. host_scratch must hold scratch_bytes (see hccl_plan_info); may be NULL if zero. */
+hccl_status_t hccl_plan_interpret_host(const hccl_plan_t*, const void* const* host_send, void* const* host_recv,
+                                       void* host_scratch, uint64_t* host_signals, uint64_t seed);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HCCL_B200_H */

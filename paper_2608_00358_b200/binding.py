@@ -1,0 +1,283 @@
+"""Thin ctypes binding of the C ABI in include/hccl.h: same names, argument marshalling only.
+
+Every step of a collective runs inside the CUDA library; nothing here computes. Device memory and
+streams come from the caller (torch tensors' ``data_ptr()`` and ``torch.cuda.Stream.cuda_stream``
+work, as do raw integers). Importing this module fails loudly if the library cannot be built/loaded.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from typing import Optional, Sequence
+
+from . import _build
+
+# ---- enums (mirrors of hccl.h)
+OK, ERR_INVALID_ARG, ERR_DTYPE, ERR_COUNT_MISMATCH, ERR_OVERLAP, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_BUSY, \
+    ERR_CUDA, ERR_TIMEOUT, ERR_BAD_DESCRIPTOR, ERR_NOT_BOUND, ERR_HAZARD = range(13)
+FP32, BF16, FP16 = 0, 1, 2
+ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED = 0, 1, 2
+ENGINE_AUTO, ENGINE_LSU, ENGINE_BULK = 0, 1, 2
+FLAG_LEVEL_MAJOR, FLAG_CHECK_HAZARDS, FLAG_STAGED_RING = 1, 2, 4
+OP_COPY, OP_REDUCE, OP_REDUCE_N, OP_WAIT, OP_SET, OP_NOOP = range(6)
+BUF_SEND, BUF_RECV, BUF_SCRATCH, BUF_SIGNAL, BUF_USER_SIGNAL = range(5)
+DEP_FENCE, DEP_SYNC, DEP_WQE_SYNC, DEP_RECV_SYNC, DEP_SEND_SYNC, DEP_ELEMENTWISE = 1, 2, 4, 8, 16, 32
+CMP_EQ, CMP_NE, CMP_GE, CMP_GT, CMP_LE, CMP_LT = range(6)
+MAX_RANKS = 256
+ELEM_BYTES = {FP32: 4, BF16: 2, FP16: 2}
+
+
+class Opts(C.Structure):
+    _fields_ = [("sm_budget", C.c_int32), ("engine", C.c_int32), ("chunk_bytes", C.c_uint64),
+                ("tile_bytes", C.c_uint64), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
+                ("chain_group", C.c_int32), ("threads", C.c_int32), ("reserved", C.c_int32 * 5)]
+
+
+class Ref(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("rank", C.c_int32), ("offset", C.c_int64)]
+
+
+class Wqe(C.Structure):
+    _fields_ = [("op", C.c_int32), ("dtype_dst", C.c_int32), ("dtype_a", C.c_int32), ("dtype_b", C.c_int32),
+                ("dst", Ref), ("a", Ref), ("b", Ref), ("count", C.c_int64), ("nsrc", C.c_int32),
+                ("dep_flags", C.c_uint32), ("dep_wqe", C.c_int64), ("dep_wqe2", C.c_int64), ("cmp", C.c_int32),
+                ("reserved", C.c_int32), ("tile_count", C.c_int64), ("value", C.c_uint64),
+                ("value_per_epoch", C.c_uint64)]
+
+
+class PlanInfo(C.Structure):
+    _fields_ = [("n_wqe", C.c_int64), ("n_tiles", C.c_int64), ("n_syncs", C.c_int64), ("chain_depth", C.c_int64),
+                ("schedule_bytes", C.c_int64), ("compulsory_bytes", C.c_int64), ("scratch_bytes", C.c_int64),
+                ("send_bytes_total", C.c_int64), ("recv_bytes_total", C.c_int64), ("R", C.c_int32),
+                ("sm_budget", C.c_int32), ("threads", C.c_int32), ("engine", C.c_int32), ("tile_bytes", C.c_int64),
+                ("epoch", C.c_int64)]
+
+
+class HcclError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        msg = "%s: %s" % (what, status_string(status))
+        if status == ERR_CUDA:
+            msg += " (%s)" % _lib.hccl_last_cuda_error().decode()
+        super().__init__(msg)
+
+
+def _load() -> C.CDLL:
+    path = _build.build()
+    lib = C.CDLL(path)
+    P, I64P = C.c_void_p, C.POINTER(C.c_int64)
+    sigs = {
+        "hccl_plan_allreduce": [C.c_int, C.c_int64, C.c_int, C.c_int, C.POINTER(Opts), C.POINTER(P)],
+        "hccl_plan_reducescatter": [C.c_int, I64P, C.c_int64, C.c_int, C.c_int, C.POINTER(Opts), C.POINTER(P)],
+        "hccl_plan_allgather": [C.c_int, I64P, C.c_int64, C.c_int, C.c_int, C.POINTER(Opts), C.POINTER(P)],
+        "hccl_plan_alltoallv": [C.c_int, I64P, I64P, I64P, I64P, C.c_int, C.c_int64, C.POINTER(Opts), C.POINTER(P)],
+        "hccl_graph_create": [C.c_int, I64P, I64P, C.c_int64, C.c_int32, C.POINTER(P)],
+        "hccl_graph_add_subgraph": [P, C.c_int, C.POINTER(C.c_int32)],
+        "hccl_graph_add_wqe": [P, C.c_int32, C.POINTER(Wqe), I64P],
+        "hccl_graph_compile": [P, C.POINTER(Opts), C.POINTER(P)],
+        "hccl_plan_workspace_bytes": [P, C.POINTER(C.c_size_t)],
+        "hccl_plan_bind": [P, P, C.c_size_t, P],
+        "hccl_execute": [P, C.POINTER(P), C.POINTER(P), P],
+        "hccl_execute_host": [P, C.POINTER(P), C.POINTER(P), C.POINTER(P), C.POINTER(P), P],
+        "hccl_plan_set_user_signals": [P, P, C.c_int64],
+        "hccl_plan_set_trigger": [P, C.c_int64, C.c_int32, C.c_uint64, C.c_uint64, C.c_int64, C.c_uint64, C.c_uint64],
+        "hccl_plan_status": [P, C.POINTER(C.c_int), I64P],
+        "hccl_plan_info": [P, C.POINTER(PlanInfo)],
+        "hccl_plan_extents": [P, C.c_int, I64P, I64P],
+        "hccl_plan_check_hazards": [P, I64P],
+        "hccl_plan_interpret_host": [P, C.POINTER(P), C.POINTER(P), P, C.POINTER(C.c_uint64), C.c_uint64],
+    }
+    for name, args in sigs.items():
+        fn = getattr(lib, name)
+        fn.argtypes = args
+        fn.restype = C.c_int
+    lib.hccl_graph_destroy.argtypes = [P]
+    lib.hccl_graph_destroy.restype = None
+    lib.hccl_plan_destroy.argtypes = [P]
+    lib.hccl_plan_destroy.restype = None
+    lib.hccl_status_string.argtypes = [C.c_int]
+    lib.hccl_status_string.restype = C.c_char_p
+    lib.hccl_last_cuda_error.argtypes = []
+    lib.hccl_last_cuda_error.restype = C.c_char_p
+    lib.hccl_version.argtypes = []
+    lib.hccl_version.restype = C.c_int
+    return lib
+
+
+_lib = _load()
+LIBRARY_PATH = _build.LIB
+EXPORTS = ["hccl_plan_allreduce", "hccl_plan_reducescatter", "hccl_plan_allgather", "hccl_plan_alltoallv",
+           "hccl_graph_create", "hccl_graph_add_subgraph", "hccl_graph_add_wqe", "hccl_graph_compile",
+           "hccl_graph_destroy", "hccl_plan_workspace_bytes", "hccl_plan_bind", "hccl_execute", "hccl_execute_host",
+           "hccl_plan_set_user_signals", "hccl_plan_set_trigger", "hccl_plan_status", "hccl_plan_info",
+           "hccl_plan_extents", "hccl_plan_destroy", "hccl_status_string", "hccl_last_cuda_error", "hccl_version",
+           "hccl_plan_check_hazards", "hccl_plan_interpret_host"]
+
+
+def status_string(status: int) -> str:
+    return _lib.hccl_status_string(status).decode()
+
+
+def _chk(rc: int, what: str):
+    if rc != OK:
+        raise HcclError(rc, what)
+
+
+def _i64(a) -> Optional[C.Array]:
+    if a is None:
+        return None
+    flat = [int(v) for row in a for v in (row if hasattr(row, "__len__") else [row])]
+    return (C.c_int64 * len(flat))(*flat)
+
+
+def _ptr_array(ptrs: Sequence[int]):
+    return (C.c_void_p * len(ptrs))(*[int(p) if p else None for p in ptrs])
+
+
+def make_opts(opts=None, **kw) -> Opts:
+    o = Opts()
+    if isinstance(opts, Opts):
+        C.memmove(C.byref(o), C.byref(opts), C.sizeof(Opts))
+    elif isinstance(opts, dict):
+        kw = {**opts, **kw}
+    for k, v in kw.items():
+        setattr(o, k, v)
+    return o
+
+
+class Plan:
+    """Owner of one hccl_plan_t*. Methods carry the names of the C calls they wrap."""
+
+    def __init__(self, handle: int):
+        self._h = C.c_void_p(handle)
+
+    def __del__(self):
+        self.destroy()
+
+    def destroy(self):
+        if getattr(self, "_h", None):
+            _lib.hccl_plan_destroy(self._h)
+            self._h = None
+
+    def workspace_bytes(self) -> int:
+        n = C.c_size_t()
+        _chk(_lib.hccl_plan_workspace_bytes(self._h, C.byref(n)), "hccl_plan_workspace_bytes")
+        return n.value
+
+    def info(self) -> PlanInfo:
+        i = PlanInfo()
+        _chk(_lib.hccl_plan_info(self._h, C.byref(i)), "hccl_plan_info")
+        return i
+
+    def extents(self, rank: int):
+        s, r = C.c_int64(), C.c_int64()
+        _chk(_lib.hccl_plan_extents(self._h, rank, C.byref(s), C.byref(r)), "hccl_plan_extents")
+        return s.value, r.value
+
+    def bind(self, dev_workspace: int, nbytes: int, stream: int = 0):
+        _chk(_lib.hccl_plan_bind(self._h, C.c_void_p(dev_workspace), nbytes, C.c_void_p(stream)), "hccl_plan_bind")
+
+    def execute(self, sendbufs: Sequence[int], recvbufs: Sequence[int], stream: int = 0):
+        _chk(_lib.hccl_execute(self._h, _ptr_array(sendbufs), _ptr_array(recvbufs), C.c_void_p(stream)), "hccl_execute")
+
+    def execute_ptrs(self, send_arr, recv_arr, stream: int = 0) -> int:
+        """Same as execute() with pre-marshalled pointer arrays; returns the status instead of raising."""
+        return _lib.hccl_execute(self._h, send_arr, recv_arr, C.c_void_p(stream))
+
+    def execute_host(self, host_send, host_recv, dev_send, dev_recv, stream: int = 0):
+        _chk(_lib.hccl_execute_host(self._h, _ptr_array(host_send), _ptr_array(host_recv), _ptr_array(dev_send),
+                                    _ptr_array(dev_recv), C.c_void_p(stream)), "hccl_execute_host")
+
+    def set_user_signals(self, dev_signals: int, n_slots: int):
+        _chk(_lib.hccl_plan_set_user_signals(self._h, C.c_void_p(dev_signals), n_slots), "hccl_plan_set_user_signals")
+
+    def set_trigger(self, wait_slot=-1, cmp=CMP_GE, wait_value=0, wait_per_epoch=0, set_slot=-1, set_value=0,
+                    set_per_epoch=0):
+        _chk(_lib.hccl_plan_set_trigger(self._h, wait_slot, cmp, wait_value, wait_per_epoch, set_slot, set_value,
+                                        set_per_epoch), "hccl_plan_set_trigger")
+
+    def status(self):
+        st, detail = C.c_int(), C.c_int64()
+        _chk(_lib.hccl_plan_status(self._h, C.byref(st), C.byref(detail)), "hccl_plan_status")
+        return st.value, detail.value
+
+    def check_hazards(self) -> int:
+        n = C.c_int64()
+        _chk(_lib.hccl_plan_check_hazards(self._h, C.byref(n)), "hccl_plan_check_hazards")
+        return n.value
+
+    def interpret_host(self, host_send: Sequence[int], host_recv: Sequence[int], host_scratch: int = 0,
+                       host_signals: int = 0, seed: int = 0) -> int:
+        return _lib.hccl_plan_interpret_host(self._h, _ptr_array(host_send), _ptr_array(host_recv),
+                                             C.c_void_p(host_scratch),
+                                             C.cast(C.c_void_p(host_signals), C.POINTER(C.c_uint64)), seed)
+
+
+def _new_plan(rc: int, h: C.c_void_p, what: str) -> Plan:
+    _chk(rc, what)
+    return Plan(h.value)
+
+
+def hccl_plan_allreduce(R: int, count: int, dt: int, algo: int = ALGO_RING, opts=None) -> Plan:
+    h = C.c_void_p()
+    return _new_plan(_lib.hccl_plan_allreduce(R, count, dt, algo, C.byref(make_opts(opts)), C.byref(h)), h,
+                     "hccl_plan_allreduce")
+
+
+def hccl_plan_reducescatter(R: int, recvcounts, count: int, dt: int, algo: int = ALGO_RING, opts=None) -> Plan:
+    h = C.c_void_p()
+    return _new_plan(_lib.hccl_plan_reducescatter(R, _i64(recvcounts), count, dt, algo, C.byref(make_opts(opts)),
+                                                  C.byref(h)), h, "hccl_plan_reducescatter")
+
+
+def hccl_plan_allgather(R: int, sendcounts, count: int, dt: int, algo: int = ALGO_RING, opts=None) -> Plan:
+    h = C.c_void_p()
+    return _new_plan(_lib.hccl_plan_allgather(R, _i64(sendcounts), count, dt, algo, C.byref(make_opts(opts)),
+                                              C.byref(h)), h, "hccl_plan_allgather")
+
+
+def hccl_plan_alltoallv(R: int, sendcounts, sdispls=None, recvcounts=None, rdispls=None, dt: int = BF16,
+                        row_elems: int = 1, opts=None) -> Plan:
+    h = C.c_void_p()
+    return _new_plan(_lib.hccl_plan_alltoallv(R, _i64(sendcounts), _i64(sdispls), _i64(recvcounts), _i64(rdispls), dt,
+                                              row_elems, C.byref(make_opts(opts)), C.byref(h)), h,
+                     "hccl_plan_alltoallv")
+
+
+class Graph:
+    """Owner of one hccl_graph_t* (a work packet under construction)."""
+
+    def __init__(self, R: int, send_bytes, recv_bytes, scratch_bytes: int = 0, n_signals: int = 0):
+        h = C.c_void_p()
+        _chk(_lib.hccl_graph_create(R, _i64(send_bytes), _i64(recv_bytes), scratch_bytes, n_signals, C.byref(h)),
+             "hccl_graph_create")
+        self._h = h
+
+    def __del__(self):
+        if getattr(self, "_h", None):
+            _lib.hccl_graph_destroy(self._h)
+            self._h = None
+
+    def add_subgraph(self, rank: int = 0) -> int:
+        sg = C.c_int32()
+        _chk(_lib.hccl_graph_add_subgraph(self._h, rank, C.byref(sg)), "hccl_graph_add_subgraph")
+        return sg.value
+
+    def add_wqe(self, subgraph: int, op: int, dst=None, a=None, b=None, count: int = 0, dtypes=(FP32, FP32, FP32),
+                nsrc: int = 0, dep_flags: int = 0, dep_wqe: int = -1, dep_wqe2: int = -1, cmp: int = 0,
+                value: int = 0, value_per_epoch: int = 0, tile_count: int = 0) -> int:
+        w = Wqe()
+        w.op = op
+        w.dtype_dst, w.dtype_a, w.dtype_b = dtypes
+        for name, r in (("dst", dst), ("a", a), ("b", b)):
+            if r is not None:
+                setattr(w, name, Ref(*r))
+        w.count, w.nsrc, w.dep_flags, w.dep_wqe, w.dep_wqe2 = count, nsrc, dep_flags, dep_wqe, dep_wqe2
+        w.cmp, w.value, w.value_per_epoch, w.tile_count = cmp, value, value_per_epoch, tile_count
+        wid = C.c_int64()
+        _chk(_lib.hccl_graph_add_wqe(self._h, subgraph, C.byref(w), C.byref(wid)), "hccl_graph_add_wqe")
+        return wid.value
+
+    def compile(self, opts=None) -> Plan:
+        h = C.c_void_p()
+        return _new_plan(_lib.hccl_graph_compile(self._h, C.byref(make_opts(opts)), C.byref(h)), h,
+                         "hccl_graph_compile")

@@ -1,0 +1,72 @@
+// Host-side objects behind the opaque handles of hccl.h.
+#pragma once
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "../../include/hccl.h"
+#include "tables.h"
+
+namespace hccl {
+
+inline int elem_bytes(int dt) { return dt == HCCL_FP32 ? 4 : 2; }
+inline bool valid_dtype(int dt) { return dt == HCCL_FP32 || dt == HCCL_BF16 || dt == HCCL_FP16; }
+inline uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+struct Wqe {
+    hccl_wqe_t w;
+    int32_t subgraph;
+    std::vector<int64_t> preds_full;  // WQE ids this one waits for entirely
+    std::vector<int64_t> preds_elem;  // WQE ids waited for tile by tile
+};
+
+struct Subgraph {
+    int rank;
+    std::vector<int64_t> wqes;        // ids in issue order
+    int64_t last_sync = -1;           // last WQE that carried HCCL_DEP_SYNC
+    bool fence_pending = false;       // previous WQE carried HCCL_DEP_FENCE
+};
+
+}  // namespace hccl
+
+struct hccl_graph {
+    int R = 0;
+    std::vector<int64_t> send_bytes, recv_bytes;
+    int64_t scratch_bytes = 0;
+    int32_t n_signals = 0;
+    std::vector<hccl::Subgraph> subgraphs;
+    std::vector<hccl::Wqe> wqes;
+    int64_t compulsory_bytes = -1;    // planners may state it; -1: derive from extents
+};
+
+struct hccl_plan {
+    int R = 0;
+    hccl_opts_t opts{};
+    std::vector<int64_t> send_bytes, recv_bytes;
+    int64_t scratch_bytes = 0;
+    int32_t n_signals = 0;
+    std::vector<hccl::Desc> descs;
+    std::vector<hccl::Tile> tiles;
+    std::vector<hccl::Wait> waits;
+    std::vector<uint32_t> sync_per_epoch;  // bumps each sync object receives per execution
+    hccl::Layout layout{};
+    hccl_plan_info_t info{};
+    // device-triggered execution (Sec. IV-B.3)
+    void* user_signals = nullptr;
+    int64_t n_user_signals = 0;
+    int64_t trig_wait_slot = -1, trig_set_slot = -1;
+    int32_t trig_cmp = 0;
+    uint64_t trig_wait_value = 0, trig_wait_per_epoch = 0, trig_set_value = 0, trig_set_per_epoch = 0;
+    // binding
+    void* workspace = nullptr;
+    size_t workspace_bytes = 0;
+    uint32_t epoch = 0;
+    // last pointer set that passed the aliasing check
+    std::vector<const void*> checked_send;
+    std::vector<void*> checked_recv;
+};
+
+namespace hccl {
+hccl_status_t compile_graph(const hccl_graph* g, const hccl_opts_t* opts, hccl_plan** out);
+void fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in);
+}  // namespace hccl

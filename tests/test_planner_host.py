@@ -1,0 +1,200 @@
+"""Planner checked on the CPU: the compiled tables, run by the library's host interpreter in random
+dependency-respecting orders, must reproduce the oracle; the hazard checker must find every pair of
+conflicting work items ordered. No GPU needed."""
+import numpy as np
+import pytest
+
+from helpers import assert_reduction_close, interpret, np_dtype
+from oracle import oracle as orc
+from paper_2608_00358_b200 import binding as hb
+from paper_2608_00358_b200 import synth
+
+DTYPES = [hb.FP32, hb.BF16, hb.FP16]
+SMALL = dict(tile_bytes=256, chunk_bytes=1024, chain_group=2, sm_budget=4)
+
+
+def test_library_exports_every_declared_symbol():
+    import ctypes
+    import os
+    import re
+    lib = ctypes.CDLL(hb.LIBRARY_PATH)
+    header = open(os.path.join(os.path.dirname(__file__), "..", "include", "hccl.h")).read()
+    declared = set(re.findall(r"\b(hccl_[a-z_0-9]+)\s*\(", header))
+    assert len(declared) >= 20
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert set(hb.EXPORTS) == declared
+    assert lib.hccl_version() >= 100
+
+
+def test_config1_plan_shape():
+    p = hb.hccl_plan_allreduce(4, 1 << 20, hb.FP32, hb.ALGO_RING)
+    i = p.info()
+    assert (i.n_wqe, i.chain_depth) == (24, 6)
+    assert i.schedule_bytes == 60 << 20 and i.compulsory_bytes == 32 << 20
+    assert i.scratch_bytes == 0
+    assert p.check_hazards() == 0
+
+
+def test_config3_and_5_byte_accounting():
+    # ReduceScatter R=16 bf16, 2 MiB granules: 146 bytes of schedule traffic per output position
+    n = 1 << 22
+    p = hb.hccl_plan_reducescatter(16, None, n, hb.BF16)
+    i = p.info()
+    assert i.schedule_bytes == 146 * n and i.compulsory_bytes == 34 * n
+    assert i.n_wqe == 16 * 15 * ((n // 16 * 2 + (2 << 20) - 1) // (2 << 20))
+    # AllReduce R=8 bf16, m bytes per rank: ring 47 m, one-shot 72 m
+    for m in (4096, 1 << 20):
+        assert hb.hccl_plan_allreduce(8, m // 2, hb.BF16, hb.ALGO_RING).info().schedule_bytes == 47 * m
+        assert hb.hccl_plan_allreduce(8, m // 2, hb.BF16, hb.ALGO_ONESHOT).info().schedule_bytes == 72 * m
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED])
+@pytest.mark.parametrize("R,n", [(1, 5), (2, 9), (3, 2), (4, 257), (5, 1000), (8, 4099), (4, 0), (4, 3)])
+def test_allreduce_plans_match_oracle(R, n, dt, algo):
+    X = synth.normal_ranks(R, n, dt, seed=R * 100 + n)
+    p = hb.hccl_plan_allreduce(R, n, dt, algo, SMALL)
+    assert p.check_hazards() == 0
+    exact = orc.sum_f64(dt, X)
+    want = orc.allreduce(dt, X)
+    if algo == hb.ALGO_ONESHOT:
+        bitwise = orc.allreduce_oneshot_f32(dt, X)
+    else:
+        bitwise = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    for seed in (0, 1, 2):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            got = Y[r].view(np_dtype(dt))
+            assert_reduction_close(dt, got, exact, want[r], "rank %d" % r)
+            # same FP32 adds in the same order as the schedule-ordered oracle: identical bits
+            assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8))
+
+
+@pytest.mark.parametrize("flags", [0, hb.FLAG_LEVEL_MAJOR, hb.FLAG_STAGED_RING])
+@pytest.mark.parametrize("dt", DTYPES)
+def test_ring_variants_same_bits(dt, flags):
+    R, n = 6, 3001
+    X = synth.normal_ranks(R, n, dt, seed=77)
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, dict(SMALL, flags=flags))
+    assert p.check_hazards() == 0
+    want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    for seed in (0, 5):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            assert np.array_equal(Y[r].view(np_dtype(dt)).view(np.uint8), want[r].view(np.uint8))
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_RING_FUSED])
+@pytest.mark.parametrize("R,counts", [(2, [3, 4]), (4, None), (5, [0, 7, 1000, 1, 300]), (16, None), (3, [0, 0, 11])])
+def test_reducescatter_plans_match_oracle(R, counts, dt, algo):
+    n = 4099 if counts is None else sum(counts)
+    rc = np.diff(orc.floor_chunk_offsets(n, R)) if counts is None else np.array(counts)
+    X = synth.normal_ranks(R, n, dt, seed=R + n, std=0.02)
+    p = hb.hccl_plan_reducescatter(R, counts, n, dt, algo, SMALL)
+    assert p.check_hazards() == 0
+    want = orc.reducescatter(dt, X, rc)
+    bitwise = orc.reducescatter_ring_f32(dt, X, rc)
+    exact = orc.sum_f64(dt, X)
+    offs = np.concatenate([[0], np.cumsum(rc)])
+    for seed in (0, 3):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            got = Y[r].view(np_dtype(dt))
+            assert got.size == rc[r]
+            assert_reduction_close(dt, got, exact[offs[r]:offs[r + 1]], want[r])
+            assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8))
+
+
+def test_reducescatter_rejects_bad_counts():
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_reducescatter(4, [1, 2, 3, 4], 11, hb.BF16)
+    assert e.value.status == hb.ERR_COUNT_MISMATCH
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_allreduce(4, 10, 7)
+    assert e.value.status == hb.ERR_DTYPE
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_allreduce(0, 10, hb.FP32)
+    assert e.value.status == hb.ERR_INVALID_ARG
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_allreduce(hb.MAX_RANKS + 1, 10, hb.FP32)
+    assert e.value.status == hb.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT])
+@pytest.mark.parametrize("R,counts", [(1, [5]), (4, [3, 0, 1000, 17]), (8, None)])
+def test_allgather_plans_match_oracle(R, counts, algo):
+    dt = hb.BF16
+    cs = counts if counts is not None else [321] * R
+    rng = np.random.default_rng(R)
+    X = [rng.integers(0, 65536, size=c, dtype=np.uint16) for c in cs]
+    p = hb.hccl_plan_allgather(R, counts, 321, dt, algo, SMALL)
+    assert p.check_hazards() == 0
+    want = orc.allgatherv(X)
+    for seed in (0, 9):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            assert np.array_equal(Y[r].view(np.uint16), want[r])
+
+
+def _a2a_case(R, seed, row_elems, dt, hi=9, packed=True):
+    rng = np.random.default_rng(seed)
+    C = synth.uniform_counts(R, seed, hi=hi)
+    C[rng.integers(0, R), rng.integers(0, R)] = 0
+    rb = row_elems * hb.ELEM_BYTES[dt]
+    if packed:
+        SD, RD = orc.packed_displs(C)
+        send_rows = C.sum(axis=1)
+    else:
+        send_rows = np.full(R, int(C.sum(axis=1).max()) + 2)
+        SD = rng.integers(0, int(send_rows[0]) - int(C.max()) + 1, size=(R, R))
+        RD = np.zeros((R, R), dtype=np.int64)
+        for d in range(R):
+            o = int(rng.integers(0, 3))
+            for s in rng.permutation(R):
+                RD[d, s] = o
+                o += int(C[s, d]) + int(rng.integers(0, 3))
+    X = [rng.integers(0, 256, size=int(send_rows[s]) * rb, dtype=np.uint8) for s in range(R)]
+    return C, SD, RD, X, rb
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 5, 8])
+@pytest.mark.parametrize("packed", [True, False])
+def test_alltoallv_plans_match_oracle(R, packed):
+    dt, row_elems = hb.BF16, 7            # 14-byte rows: nothing is 16-byte aligned
+    C, SD, RD, X, rb = _a2a_case(R, 100 + R, row_elems, dt, packed=packed)
+    p = hb.hccl_plan_alltoallv(R, C, None if packed else SD, C.T.copy(), None if packed else RD, dt, row_elems,
+                               dict(SMALL, tile_bytes=256))
+    assert p.check_hazards() == 0
+    Yw = [np.full(p.extents(r)[1], 0xA5, dtype=np.uint8) for r in range(R)]
+    orc.alltoallv(X, Yw, C, SD, RD, rb)
+    for seed in (0, 4):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            assert np.array_equal(Y[r], Yw[r])        # gaps keep the sentinel
+    i = p.info()
+    assert i.schedule_bytes == 2 * int(C.sum()) * rb == i.compulsory_bytes
+    assert i.n_wqe == int((C > 0).sum())              # zero-length segments cost nothing
+
+
+def test_alltoallv_validation():
+    C = np.array([[1, 2], [3, 4]])
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_alltoallv(2, C, None, C, None, hb.FP16, 4)        # recvcounts must be the transpose
+    assert e.value.status == hb.ERR_COUNT_MISMATCH
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_alltoallv(2, C, None, None, [[0, 2], [0, 1]], hb.FP16, 4)   # rank 0: rows [0,1) and [2,5) fine; rank 1: [0,2) and [1,5) overlap
+    assert e.value.status == hb.ERR_OVERLAP
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_alltoallv(2, [[1, -1], [0, 0]], None, None, None, hb.FP16, 4)
+    assert e.value.status == hb.ERR_INVALID_ARG
+    # overlapping sends are legal
+    p = hb.hccl_plan_alltoallv(2, C, [[0, 0], [0, 0]], None, None, hb.FP16, 4)
+    assert p.info().n_wqe == 4
+
+
+def test_all_zero_counts_is_an_empty_plan():
+    p = hb.hccl_plan_alltoallv(3, np.zeros((3, 3), dtype=np.int64), None, None, None, hb.BF16, 128)
+    assert p.info().n_tiles == 0 and p.info().schedule_bytes == 0
+    assert interpret(p, [np.zeros(1, dtype=np.uint8)] * 3) is not None
