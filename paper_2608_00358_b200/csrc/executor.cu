@@ -601,7 +601,7 @@ static hccl_status_t check_buffers(hccl_plan_t* p, const void* const* sendbufs, 
     if (same) return HCCL_OK;
     for (int r = 0; r < R; ++r) {
         if ((p->send_bytes[r] > 0 && !sendbufs[r]) || (p->recv_bytes[r] > 0 && !recvbufs[r])) return HCCL_ERR_INVALID_ARG;
-        if (((uintptr_t)sendbufs[r] | (uintptr_t)recvbufs[r]) & 1u) return HCCL_ERR_ALIGNMENT;
+        if (((uintptr_t)sendbufs[r] | (uintptr_t)recvbufs[r]) & (uintptr_t)(p->buf_align - 1)) return HCCL_ERR_ALIGNMENT;
     }
     // out-of-place only: no receive extent may intersect a send extent or another receive extent
     for (int d = 0; d < R; ++d) {

@@ -293,6 +293,14 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         if (w.op == HCCL_OP_REDUCE) schedule += w.count * (elem_bytes(w.dtype_a) + elem_bytes(w.dtype_b) + elem_bytes(w.dtype_dst));
         if (w.op == HCCL_OP_REDUCE_N) schedule += w.count * ((int64_t)w.nsrc * elem_bytes(w.dtype_a) + elem_bytes(w.dtype_dst));
         weight += w.count * widest(w);
+        if (w.op == HCCL_OP_REDUCE || w.op == HCCL_OP_REDUCE_N) {
+            auto need = [&](const hccl_ref_t& r, int dt) {
+                if (r.kind == HCCL_BUF_SEND || r.kind == HCCL_BUF_RECV) p->buf_align = std::max(p->buf_align, elem_bytes(dt));
+            };
+            need(w.dst, w.dtype_dst);
+            need(w.a, w.dtype_a);
+            if (w.op == HCCL_OP_REDUCE) need(w.b, w.dtype_b);
+        }
     }
     uint64_t tile_bytes = p->opts.tile_bytes;
     if (tile_bytes == 0) {

@@ -50,6 +50,7 @@ struct hccl_plan {
     std::vector<hccl::Wait> waits;
     std::vector<uint32_t> sync_per_epoch;  // bumps each sync object receives per execution
     hccl::Layout layout{};
+    int buf_align = 1;                     // alignment every send/receive pointer must have (largest element read or written)
     hccl_plan_info_t info{};
     // device-triggered execution (Sec. IV-B.3)
     void* user_signals = nullptr;

@@ -1,0 +1,176 @@
+"""Parity of the CUDA executor against the CPU oracle, through the C ABI. Needs a GPU."""
+import numpy as np
+import pytest
+
+from gpu_helpers import run_plan
+from helpers import assert_reduction_close, np_dtype
+from oracle import oracle as orc
+from paper_2608_00358_b200 import binding as hb
+from paper_2608_00358_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DTYPES = [hb.FP32, hb.BF16, hb.FP16]
+
+
+def _check_allreduce(R, n, dt, algo, opts, X=None, iters=1, misalign=0):
+    X = X if X is not None else synth.normal_ranks(R, n, dt, seed=R * 131 + n)
+    p = hb.hccl_plan_allreduce(R, n, dt, algo, opts)
+    Y = run_plan(p, X, iters=iters, misalign=misalign)
+    exact, want = orc.sum_f64(dt, X), orc.allreduce(dt, X)
+    bitwise = orc.allreduce_oneshot_f32(dt, X) if algo == hb.ALGO_ONESHOT else \
+        orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    for r in range(R):
+        got = Y[r].view(np_dtype(dt))
+        assert_reduction_close(dt, got, exact, want[r], "rank %d" % r)
+        assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8)), "rank %d differs from the schedule-ordered FP32 sums" % r
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED])
+@pytest.mark.parametrize("R,n", [(1, 5), (2, 9), (3, 2), (4, 257), (5, 1000), (8, 4099), (4, 0), (4, 3), (8, 100003)])
+def test_allreduce_small(R, n, dt, algo):
+    _check_allreduce(R, n, dt, algo, dict(tile_bytes=1024, chunk_bytes=4096, chain_group=2, sm_budget=8), iters=2)
+
+
+@pytest.mark.parametrize("budget", [1, 2, 3, 8, 148, 296])
+@pytest.mark.parametrize("dt", [hb.FP32, hb.BF16])
+def test_allreduce_any_sm_budget_same_bits(budget, dt):
+    _check_allreduce(6, 50021, dt, hb.ALGO_RING, dict(tile_bytes=2048, chunk_bytes=16384, sm_budget=budget), iters=3)
+
+
+@pytest.mark.parametrize("misalign", [2, 4, 6, 10])
+@pytest.mark.parametrize("dt", DTYPES)
+def test_allreduce_misaligned_buffers(misalign, dt):
+    if dt == hb.FP32 and misalign % 4:
+        pytest.skip("buffers must be aligned to the element size")
+    _check_allreduce(4, 10007, dt, hb.ALGO_RING, dict(tile_bytes=4096, sm_budget=16), misalign=misalign)
+    _check_allreduce(4, 10007, dt, hb.ALGO_ONESHOT, dict(tile_bytes=4096, sm_budget=16), misalign=misalign)
+
+
+def test_config1_allreduce_ring_r4_fp32():
+    X = synth.uniform_ranks(4, 1 << 20, hb.FP32, seed=0)
+    _check_allreduce(4, 1 << 20, hb.FP32, hb.ALGO_RING, None, X=X, iters=3)
+
+
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT])
+@pytest.mark.parametrize("m", [4096, 65536, 262144, 1 << 20])
+def test_config5_allreduce_r8_bf16(m, algo):
+    X = synth.normal_ranks(8, m // 2, hb.BF16, seed=m)
+    _check_allreduce(8, m // 2, hb.BF16, algo, None, X=X, iters=3)
+
+
+def test_closed_form_on_device():
+    for dt in DTYPES:
+        for R in (2, 4, 8, 16):
+            n = 3000
+            X = [synth.to_bits(np.full(n, r + 1, dtype=np.float32), dt) for r in range(R)]
+            for algo in (hb.ALGO_RING, hb.ALGO_ONESHOT):
+                Y = run_plan(hb.hccl_plan_allreduce(R, n, dt, algo, dict(tile_bytes=1024)), X)
+                for r in range(R):
+                    assert np.all(synth.from_bits(Y[r].view(np_dtype(dt)), dt) == R * (R + 1) / 2)
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_RING_FUSED])
+@pytest.mark.parametrize("R,counts", [(2, [3, 4]), (4, None), (5, [0, 7, 1000, 1, 300]), (16, None), (3, [0, 0, 11])])
+def test_reducescatter_small(R, counts, dt, algo):
+    n = 40099 if counts is None else sum(counts)
+    rc = np.diff(orc.floor_chunk_offsets(n, R)) if counts is None else np.array(counts)
+    X = synth.normal_ranks(R, n, dt, seed=R + n, std=0.02)
+    p = hb.hccl_plan_reducescatter(R, counts, n, dt, algo, dict(tile_bytes=1024, chunk_bytes=2048, chain_group=3, sm_budget=16))
+    Y = run_plan(p, X, iters=2)
+    want, bitwise, exact = orc.reducescatter(dt, X, rc), orc.reducescatter_ring_f32(dt, X, rc), orc.sum_f64(dt, X)
+    offs = np.concatenate([[0], np.cumsum(rc)])
+    for r in range(R):
+        got = Y[r].view(np_dtype(dt))
+        assert_reduction_close(dt, got, exact[offs[r]:offs[r + 1]], want[r])
+        assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8))
+
+
+def test_config3_shape_reducescatter_r16_bf16_reduced_size():
+    # config 3 at 1/16 of its size (4 Mi elements per rank, 2 MiB granules -> still several granules per shard? no:
+    # shards of 256 Ki elements = 512 KiB, so use 128 KiB granules to keep 4 granules per shard)
+    R, n = 16, 1 << 22
+    X = synth.normal_ranks(R, n, hb.BF16, seed=3, std=0.02)
+    p = hb.hccl_plan_reducescatter(R, None, n, hb.BF16, hb.ALGO_RING, dict(chunk_bytes=128 << 10))
+    Y = run_plan(p, X, iters=2)
+    rc = np.full(R, n // R)
+    want, bitwise = orc.reducescatter(hb.BF16, X, rc), orc.reducescatter_ring_f32(hb.BF16, X, rc)
+    for r in range(R):
+        got = Y[r].view(np.uint16)
+        assert orc.ulp_distance(hb.BF16, got, want[r]).max() <= 1
+        assert np.array_equal(got, bitwise[r])
+
+
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT])
+@pytest.mark.parametrize("R,counts", [(1, [5]), (4, [3, 0, 1000, 17]), (8, None)])
+def test_allgather(R, counts, algo):
+    cs = counts if counts is not None else [32100] * R
+    rng = np.random.default_rng(R)
+    X = [rng.integers(0, 65536, size=c, dtype=np.uint16) for c in cs]
+    p = hb.hccl_plan_allgather(R, counts, 32100, hb.BF16, algo, dict(tile_bytes=4096, sm_budget=32))
+    Y = run_plan(p, X, iters=2)
+    want = orc.allgatherv(X)
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np.uint16), want[r])
+
+
+def _a2a(R, C, SD, RD, X, dt, row_elems, opts, packed, iters=1, misalign=0):
+    rb = row_elems * hb.ELEM_BYTES[dt]
+    p = hb.hccl_plan_alltoallv(R, C, None if packed else SD, C.T.copy(), None if packed else RD, dt, row_elems, opts)
+    Y = run_plan(p, X, iters=iters, misalign=misalign)
+    Yw = [np.full(p.extents(r)[1], 0xA5, dtype=np.uint8) for r in range(R)]
+    orc.alltoallv(X, Yw, C, SD, RD, rb)
+    for r in range(R):
+        assert np.array_equal(Y[r], Yw[r]), "rank %d" % r
+    return Y
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 5, 8])
+@pytest.mark.parametrize("packed", [True, False])
+@pytest.mark.parametrize("row_elems", [7, 128])
+def test_alltoallv_small(R, packed, row_elems):
+    from test_planner_host import _a2a_case
+    C, SD, RD, X, rb = _a2a_case(R, 100 + R, row_elems, hb.BF16, hi=40, packed=packed)
+    _a2a(R, C, SD, RD, X, hb.BF16, row_elems, dict(tile_bytes=1024, sm_budget=16), packed, iters=2)
+
+
+@pytest.mark.parametrize("misalign", [1, 3, 8])
+def test_alltoallv_misaligned(misalign):
+    from test_planner_host import _a2a_case
+    C, SD, RD, X, rb = _a2a_case(4, 7, 5, hb.FP16, hi=300, packed=True)
+    _a2a(4, C, SD, RD, X, hb.FP16, 5, dict(tile_bytes=4096), True, misalign=misalign)
+
+
+def test_config2_alltoallv_r8_bf16_rows128():
+    R, row_elems = 8, 128
+    C = synth.uniform_counts(R, 0, hi=4096)
+    assert int(C.sum()) == 133647                       # the seed-0 draw this config is quoted on
+    SD, RD = orc.packed_displs(C)
+    X = [synth.normal_ranks(1, int(C[s].sum()) * row_elems, hb.BF16, seed=1000 + s)[0].view(np.uint8) for s in range(R)]
+    Y = _a2a(R, C, SD, RD, X, hb.BF16, row_elems, None, True, iters=3)
+    # identity invariant: exchanging back with the transposed counts restores every send buffer
+    CT = C.T.copy()
+    SD2, RD2 = orc.packed_displs(CT)
+    p2 = hb.hccl_plan_alltoallv(R, CT, None, None, None, hb.BF16, row_elems)
+    Z = run_plan(p2, Y)
+    for s in range(R):
+        assert np.array_equal(Z[s], X[s])
+
+
+def test_alltoallv_zero_everything():
+    p = hb.hccl_plan_alltoallv(3, np.zeros((3, 3), dtype=np.int64), None, None, None, hb.BF16, 128)
+    run_plan(p, [np.zeros(16, dtype=np.uint8)] * 3, iters=2)
+
+
+def test_overlapping_send_and_receive_is_rejected():
+    import torch
+    p = hb.hccl_plan_allreduce(2, 1024, hb.FP32, hb.ALGO_ONESHOT)
+    from paper_2608_00358_b200.runtime import DeviceCollective
+    dc = DeviceCollective(p)
+    buf = torch.zeros(4 * 4096, dtype=torch.uint8, device="cuda")
+    b = buf.data_ptr()
+    dc.set_buffers([b, b + 4096], [b + 2048, b + 8192])
+    with pytest.raises(hb.HcclError) as e:
+        dc.execute()
+    assert e.value.status == hb.ERR_OVERLAP
