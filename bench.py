@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the collective hot path on B200.
+
+A step is one execution of the rack-scale AllToAllv configuration (R = 64 virtual ranks, rows of 256 fp16,
+Zipf(1.1) per-peer row counts clamped at 32768; ~25.8 GB moved, ~51.6 GB resident), the largest
+single-GPU configuration and the one the HBM-bandwidth target is stated on. The metric is data-path GB/s
+counting bytes read + bytes written. The same JSON line also carries the other configurations (ring
+AllReduce, small AllToAllv, ring ReduceScatter, latency sweep), the GEMM-interference figure, the roofline
+fraction of the executor kernel, an end-to-end figure through host buffers and the CPU oracle's baseline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--quick]
+
+With N > 1 (launched by torchrun) every rank runs an independent replica on its own GPU: the path has no
+exchange between GPUs, so there is no data-path collective; time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "data-path GB/s (bytes read + written), AllToAllv R=64 virtual ranks"
+UNIT = "GB/s"
+# dram bytes (read + write) per algorithmic byte of the executor kernel on this workload, from the ncu
+# capture summarised under profiles/ (captured on a smaller cap of the same workload, traffic scales with
+# the bytes moved). None until measured.
+DRAM_BYTES_PER_ALGORITHMIC_BYTE = None
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while a timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.1):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                 nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                 nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap"}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        import statistics
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ----------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_alltoallv_sample(counts, row_bytes: int, dst_ranks, repeat: int = 1):
+    """Times the oracle's AllToAllv, as it stands, for the given destination ranks of the workload.
+    Host send buffers are virtual-size arrays of which only the rows those destinations read are filled."""
+    import numpy as np
+    from oracle import oracle as orc
+    R = counts.shape[0]
+    sd, rd = orc.packed_displs(counts)
+    X = [np.empty(int(counts[s].sum()) * row_bytes, dtype=np.uint8) for s in range(R)]
+    rng = np.random.default_rng(0)
+    block = rng.integers(0, 256, size=1 << 20, dtype=np.uint8)
+    moved = 0
+    for d in dst_ranks:
+        for s in range(R):
+            lo, n = int(sd[s, d]) * row_bytes, int(counts[s, d]) * row_bytes
+            seg = X[s][lo:lo + n]
+            for o in range(0, n, block.size):
+                k = min(block.size, n - o)
+                seg[o:o + k] = block[:k]
+            moved += n
+    Y = [np.empty(int(counts[:, d].sum()) * row_bytes if d in dst_ranks else 1, dtype=np.uint8) for d in range(R)]
+    times = []
+    for _ in range(repeat):
+        t0 = time.perf_counter()
+        for d in dst_ranks:
+            orc.alltoallv(X, Y, counts, sd, rd, row_bytes, dst_only=d)
+        times.append(time.perf_counter() - t0)
+    return moved, times
+
+
+def run_reference(args, rank: int):
+    """The reference arm: the CPU oracle, unmodified, on a bounded sample of the same workload."""
+    if rank != 0:
+        return
+    from paper_2608_00358_b200 import synth
+    C = synth.zipf_counts(64, 0, 1.1, args.cap)
+    dst = list(range(args.oracle_dst))
+    moved, times = oracle_alltoallv_sample(C, 512, dst, repeat=args.warmup + args.steps)
+    timed = times[args.warmup:]
+    sec = sum(timed) / len(timed)
+    gbs = 2 * moved / sec / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8", "data": "synthetic",
+            "config": {"workload": "alltoallv_r64_fp16_dim256_zipf1.1_cap%d" % args.cap, "sample": "destination ranks 0..%d" % (args.oracle_dst - 1)},
+            "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle",
+                             "sample": "destination ranks 0..%d of 64 (%.2f GB moved per step)" % (args.oracle_dst - 1, moved / 1e9)},
+            "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------------------- GPU legs
+def side_configs(quick: bool):
+    """Configurations 1, 2, 3 and 5: reported next to the headline, never as the headline."""
+    import numpy as np
+    import torch
+    from paper_2608_00358_b200 import binding as hb
+    from paper_2608_00358_b200 import workloads as wk
+    out = {}
+    it, warm = (200, 20) if quick else (1000, 100)
+
+    def latency(wl, key):
+        ms = wk.time_each(wl, it, warm)
+        i = wl.info
+        out[key] = {"p50_us": float(np.percentile(ms, 50) * 1e3), "p99_us": float(np.percentile(ms, 99) * 1e3),
+                    "back_to_back_us": float(wk.time_back_to_back(wl, it, warm) * 1e3),
+                    "schedule_bytes": int(i.schedule_bytes), "compulsory_bytes": int(i.compulsory_bytes),
+                    "tiles": int(i.n_tiles), "chain_depth": int(i.chain_depth), "note": "L2-resident, latency-bound"}
+        out[key]["schedule_gbs_back_to_back"] = i.schedule_bytes / out[key]["back_to_back_us"] / 1e3
+
+    latency(wk.config1(), "1_allreduce_ring_r4_fp32_1Mi")
+    latency(wk.config2(), "2_alltoallv_r8_bf16_dim128")
+    for m in (4096, 65536, 262144, 1 << 20):
+        for algo, nm in ((hb.ALGO_ONESHOT, "oneshot"), (hb.ALGO_RING, "ring")):
+            latency(wk.config5(m, algo), "5_allreduce_r8_bf16_%dB_%s" % (m, nm))
+    torch.cuda.empty_cache()
+    for algo, nm in ((hb.ALGO_RING, "ring"), (hb.ALGO_RING_FUSED, "ring_fused")):
+        wl = wk.config3(algo=algo)
+        ms = wk.time_back_to_back(wl, 10 if quick else 50, 5)
+        i = wl.info
+        out["3_reducescatter_r16_bf16_64Mi_" + nm] = {
+            "ms": float(ms), "schedule_bytes": int(i.schedule_bytes), "compulsory_bytes": int(i.compulsory_bytes),
+            "schedule_gbs": i.schedule_bytes / ms / 1e6, "compulsory_gbs": i.compulsory_bytes / ms / 1e6,
+            "tiles": int(i.n_tiles), "inputs": "2 GiB, larger than L2"}
+        del wl
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_ours(args, rank: int, world: int, local_rank: int):
+    import numpy as np
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2608_00358_b200 import binding as hb
+    from paper_2608_00358_b200 import interference
+    from paper_2608_00358_b200 import workloads as wk
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    opts = dict(sm_budget=args.sm_budget) if args.sm_budget else None
+    wl = wk.config4(opts, seed=0, cap=args.cap)
+    info = wl.info
+    payload = wl.meta["payload_bytes"]
+    stream = torch.cuda.current_stream()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+
+    # ---- device-resident timing: W warm-ups, then exactly K steps, one kernel launch each
+    for _ in range(max(args.warmup, 3)):
+        wl.dc.execute(stream)
+    barrier()
+    sampler.start()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    evs[0].record(stream)
+    for k in range(args.steps):
+        wl.dc.execute(stream)
+        evs[k + 1].record(stream)
+    barrier()
+    clocks = sampler.stop()
+    wl.dc.check()
+    total_ms = evs[0].elapsed_time(evs[-1])
+    per_launch = np.array([evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)])
+    t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t.item())
+    value = world * info.schedule_bytes * args.steps / (total_ms_max * 1e-3) / 1e9
+
+    # ---- end to end through host buffers (rank-local; reported by rank 0)
+    e2e = None
+    if rank == 0 and not args.no_e2e:
+        import psutil
+        need = 2 * payload + (8 << 30)
+        if psutil.virtual_memory().available > need:
+            hs = [torch.empty(t_.numel(), dtype=t_.dtype, pin_memory=True) for t_ in wl.send]
+            hr = [torch.empty(t_.numel(), dtype=t_.dtype, pin_memory=True) for t_ in wl.recv]
+            for h, d_ in zip(hs, wl.send):
+                h.copy_(d_)
+            torch.cuda.synchronize()
+            hp = ([h.data_ptr() for h in hs], [h.data_ptr() for h in hr])
+            dp = ([d_.data_ptr() for d_ in wl.send], [d_.data_ptr() for d_ in wl.recv])
+            wl.plan.execute_host(hp[0], hp[1], dp[0], dp[1], stream.cuda_stream)   # warm-up
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ksteps = args.e2e_steps
+            e0.record(stream)
+            for _ in range(ksteps):
+                wl.plan.execute_host(hp[0], hp[1], dp[0], dp[1], stream.cuda_stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            wl.dc.check()
+            ms = e0.elapsed_time(e1) / ksteps
+            e2e = {"value": info.schedule_bytes / ms / 1e6, "unit": UNIT, "h2d_bytes_per_step": int(payload),
+                   "d2h_bytes_per_step": int(payload), "ms_per_step": ms, "steps": ksteps,
+                   "api": "hccl_execute_host (pinned host buffers -> device -> pinned host buffers)"}
+            del hs, hr
+        else:
+            e2e = {"value": None, "unit": UNIT, "skipped": "host memory too small to pin 2 x %.1f GB" % (payload / 1e9)}
+
+    line = None
+    if rank == 0:
+        peak, which = peaks()
+        launch_ms = float(per_launch.mean())
+        achieved = info.schedule_bytes / launch_ms / 1e6
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "ms_per_step": total_ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8", "data": "synthetic",
+            "config": {"workload": wl.name, "virtual_ranks": 64, "row_bytes": 512, "rows_moved": int(wl.meta["counts"].sum()),
+                       "payload_bytes": int(payload), "resident_bytes": int(2 * payload), "sm_budget": int(info.sm_budget),
+                       "threads": int(info.threads), "tile_bytes": int(info.tile_bytes), "tiles": int(info.n_tiles),
+                       "engine": {1: "lsu", 2: "bulk"}.get(int(info.engine), str(info.engine)),
+                       "cache": "inputs larger than L2 (no flush needed)", "multi_gpu": "replicas only"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "peak_source": which + " copy bandwidth (burst)", "kernel": "hccl_executor",
+                         "algorithmic_bytes_per_launch": int(info.schedule_bytes), "launch_ms": launch_ms,
+                         "traffic": (DRAM_BYTES_PER_ALGORITHMIC_BYTE * info.schedule_bytes) if DRAM_BYTES_PER_ALGORITHMIC_BYTE else None,
+                         "frac_of_nominal_8TBs": achieved / 8000.0},
+            "gpu_launches": args.steps, "clocks": clocks, "e2e": e2e,
+        }
+
+    # ---- interference, other configs, CPU baseline: rank 0 at N = 1 only
+    if rank == 0 and world == 1:
+        if not args.no_gemm:
+            line["interference"] = interference.measure(wl, seconds=2.0 if args.quick else 3.0)
+        del wl
+        torch.cuda.empty_cache()
+        if not args.no_side:
+            line["configs"] = side_configs(args.quick)
+        if not args.no_cpu:
+            from paper_2608_00358_b200 import synth
+            C = synth.zipf_counts(64, 0, 1.1, args.cap)
+            dst = list(range(args.oracle_dst))
+            moved, times = oracle_alltoallv_sample(C, 512, dst, repeat=2)
+            line["cpu_baseline"] = {"value": 2 * moved / min(times) / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                    "sample": "destination ranks 0..%d of 64 (%.2f GB moved), best of 2" % (args.oracle_dst - 1, moved / 1e9),
+                                    "host_cores_available": os.cpu_count()}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cap", type=int, default=32768, help="clamp of the Zipf row counts (32768 = the named config)")
+    ap.add_argument("--sm-budget", type=int, default=0)
+    ap.add_argument("--oracle-dst", type=int, default=8, help="destination ranks in the CPU oracle's sample")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-gemm", action="store_true")
+    ap.add_argument("--no-side", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

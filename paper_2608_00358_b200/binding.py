@@ -154,9 +154,9 @@ class Plan:
         self.destroy()
 
     def destroy(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:
             _lib.hccl_plan_destroy(self._h)
-            self._h = None
+        self._h = None
 
     def workspace_bytes(self) -> int:
         n = C.c_size_t()
@@ -253,9 +253,9 @@ class Graph:
         self._h = h
 
     def __del__(self):
-        if getattr(self, "_h", None):
+        if getattr(self, "_h", None) and _lib is not None:
             _lib.hccl_graph_destroy(self._h)
-            self._h = None
+        self._h = None
 
     def add_subgraph(self, rank: int = 0) -> int:
         sg = C.c_int32()

@@ -1,0 +1,143 @@
+"""Interference harness: a saturating bf16 GEMM on one stream, back-to-back collectives on a second one.
+
+The paper's overlap experiment (Sec. V-E) runs a large GEMM that fills the compute grid while 100
+collectives of one size run back to back on a parallel stream, and reports the GEMM's loss (about 0.5 %
+on its hardware, attributed to HBM contention). Here the GEMM is cuBLAS through torch.matmul and the
+collective is one bound plan re-enqueued on a high-priority stream; the benchmark suite the paper used
+is not available and is not reproduced.
+
+Run as a module for the SM-budget sweep:
+    python -m paper_2608_00358_b200.interference --budgets 4,8,16,32,64,148 --cap 32768
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import time
+from typing import Optional
+
+import numpy as np
+import torch
+
+from . import workloads as wk
+
+
+class Gemm:
+    def __init__(self, n: int = 8192):
+        self.n = n
+        g = torch.Generator(device="cuda")
+        g.manual_seed(1)
+        self.a = torch.randn(n, n, device="cuda", dtype=torch.float32, generator=g).to(torch.bfloat16)
+        self.b = torch.randn(n, n, device="cuda", dtype=torch.float32, generator=g).to(torch.bfloat16)
+        self.c = torch.empty(n, n, device="cuda", dtype=torch.bfloat16)
+        self.flops = 2.0 * n ** 3
+
+    def run(self):
+        torch.matmul(self.a, self.b, out=self.c)
+
+
+def gemm_alone(gemm: Gemm, seconds: float = 3.0, discard: float = 1.0, batch: int = 10) -> dict:
+    """Sustained TFLOP/s of the GEMM with nothing else on the GPU; the first `discard` seconds are dropped."""
+    s = torch.cuda.Stream()
+    base = torch.cuda.Event(enable_timing=True)
+    evs = []
+    with torch.cuda.stream(s):
+        for _ in range(3):
+            gemm.run()
+        s.synchronize()
+        base.record(s)
+        t0 = time.time()
+        while time.time() - t0 < seconds:
+            for _ in range(batch):
+                gemm.run()
+            e = torch.cuda.Event(enable_timing=True)
+            e.record(s)
+            evs.append(e)
+            if len(evs) > 20:
+                evs[-20].synchronize()       # keep the queue bounded
+        s.synchronize()
+    ts = np.array([base.elapsed_time(e) for e in evs])     # ms at the end of each batch
+    keep = ts >= discard * 1e3
+    if keep.sum() < 3:
+        keep[:] = True
+    tk = ts[keep]
+    tf = gemm.flops * batch * (len(tk) - 1) / ((tk[-1] - tk[0]) * 1e-3) / 1e12
+    return dict(tflops=float(tf), batches=int(len(tk) - 1), seconds=float((tk[-1] - tk[0]) * 1e-3))
+
+
+def overlap(gemm: Gemm, wl: wk.Workload, seconds: float = 3.0, discard: float = 1.0, gemm_batch: int = 10) -> dict:
+    """GEMM loop on one stream, collective loop on a high-priority stream; rates are computed only inside
+    the window in which events show both loops running."""
+    sg = torch.cuda.Stream()
+    sc = torch.cuda.Stream(priority=-1)
+    base = torch.cuda.Event(enable_timing=True)
+    eg, ec = [], []
+    torch.cuda.synchronize()
+    base.record(torch.cuda.current_stream())
+    sg.wait_event(base)
+    sc.wait_event(base)
+    t0 = time.time()
+    while time.time() - t0 < seconds:
+        with torch.cuda.stream(sg):
+            for _ in range(gemm_batch):
+                gemm.run()
+            e = torch.cuda.Event(enable_timing=True)
+            e.record(sg)
+            eg.append(e)
+        wl.dc.execute(sc)
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(sc)
+        ec.append(e)
+        if len(eg) > 20:
+            eg[-20].synchronize()
+        if len(ec) > 20:
+            ec[-20].synchronize()
+    torch.cuda.synchronize()
+    wl.dc.check()
+    tg = np.array([base.elapsed_time(e) for e in eg])
+    tc = np.array([base.elapsed_time(e) for e in ec])
+    lo = max(discard * 1e3, min(tg[0], tc[0]))
+    hi = min(tg[-1], tc[-1])
+    kg = tg[(tg >= lo) & (tg <= hi)]
+    kc = tc[(tc >= lo) & (tc <= hi)]
+    out = dict(window_s=float((hi - lo) * 1e-3), gemm_batches=int(max(len(kg) - 1, 0)), collectives=int(max(len(kc) - 1, 0)))
+    if len(kg) >= 2:
+        out["gemm_tflops"] = float(gemm.flops * gemm_batch * (len(kg) - 1) / ((kg[-1] - kg[0]) * 1e-3) / 1e12)
+    if len(kc) >= 2:
+        ms = (kc[-1] - kc[0]) / (len(kc) - 1)
+        out["collective_ms"] = float(ms)
+        out["collective_gbs"] = float(wl.info.schedule_bytes / ms / 1e6)
+    return out
+
+
+def measure(wl: wk.Workload, seconds: float = 3.0, gemm: Optional[Gemm] = None) -> dict:
+    gemm = gemm or Gemm()
+    alone = gemm_alone(gemm, seconds)
+    coll_alone_ms = wk.time_back_to_back(wl, 5, 2)
+    both = overlap(gemm, wl, seconds)
+    res = dict(gemm_alone_tflops=alone["tflops"], collective_alone_ms=float(coll_alone_ms),
+               collective_alone_gbs=float(wl.info.schedule_bytes / coll_alone_ms / 1e6), overlap=both,
+               sm_budget=int(wl.info.sm_budget))
+    if "gemm_tflops" in both:
+        res["gemm_slowdown"] = float(1.0 - both["gemm_tflops"] / alone["tflops"])
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--budgets", default="2,4,8,16,32,64,128,148")
+    ap.add_argument("--cap", type=int, default=32768)
+    ap.add_argument("--seconds", type=float, default=3.0)
+    ap.add_argument("--engine", type=int, default=0)
+    args = ap.parse_args()
+    gemm = Gemm()
+    base = wk.config4(dict(sm_budget=148, engine=args.engine), cap=args.cap)
+    for b in [int(x) for x in args.budgets.split(",")]:
+        plan = wk.hb.hccl_plan_alltoallv(base.meta["R"], base.meta["counts"], None, None, None, wk.hb.FP16,
+                                         base.meta["row_elems"], dict(sm_budget=b, engine=args.engine))
+        wl = wk._bind(base.name, plan, base.send, base.recv, base.meta)
+        print(json.dumps(measure(wl, args.seconds, gemm)), flush=True)
+
+
+if __name__ == "__main__":
+    main()
