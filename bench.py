@@ -31,7 +31,7 @@ UNIT = "GB/s"
 # dram bytes (read + write) per algorithmic byte of the executor kernel on this workload, from the ncu
 # capture summarised under profiles/ (captured on a smaller cap of the same workload, traffic scales with
 # the bytes moved). None until measured.
-DRAM_BYTES_PER_ALGORITHMIC_BYTE = None
+DRAM_BYTES_PER_ALGORITHMIC_BYTE = 0.979
 
 
 def peaks():
@@ -46,7 +46,7 @@ def peaks():
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML (read-only) while a timed region runs."""
 
-    def __init__(self, index: int, period: float = 0.1):
+    def __init__(self, index: int, period: float = 0.02):
         super().__init__(daemon=True)
         self.index, self.period = index, period
         self.samples, self.reasons, self.max_mhz = [], set(), None
