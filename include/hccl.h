@@ -92,7 +92,8 @@ typedef struct {
     uint32_t flags;         /* HCCL_FLAG_* */
     int32_t chain_group;    /* chains scheduled together in chain-group-major order (default 8) */
     int32_t threads;        /* threads per block, multiple of 32 (default 512) */
-    int32_t reserved[5];
+    int32_t stages;         /* bulk engine: shared-memory stages of 32 KiB per block, 2..8 (default 6) */
+    int32_t reserved[4];
 } hccl_opts_t;
 
 typedef struct hccl_plan hccl_plan_t;   /* opaque, host-owned: a compiled, cacheable work packet (Sec. V-B) */

@@ -29,7 +29,7 @@ ELEM_BYTES = {FP32: 4, BF16: 2, FP16: 2}
 class Opts(C.Structure):
     _fields_ = [("sm_budget", C.c_int32), ("engine", C.c_int32), ("chunk_bytes", C.c_uint64),
                 ("tile_bytes", C.c_uint64), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
-                ("chain_group", C.c_int32), ("threads", C.c_int32), ("reserved", C.c_int32 * 5)]
+                ("chain_group", C.c_int32), ("threads", C.c_int32), ("stages", C.c_int32), ("reserved", C.c_int32 * 4)]
 
 
 class Ref(C.Structure):

@@ -76,22 +76,32 @@ def overlap(gemm: Gemm, wl: wk.Workload, seconds: float = 3.0, discard: float = 
     base.record(torch.cuda.current_stream())
     sg.wait_event(base)
     sc.wait_event(base)
+    # Both queues are kept a few batches deep independently of each other, so neither loop is ever
+    # starved by the other's enqueue rate.
+    depth, done_g, done_c = 3, 0, 0
     t0 = time.time()
     while time.time() - t0 < seconds:
-        with torch.cuda.stream(sg):
-            for _ in range(gemm_batch):
-                gemm.run()
+        while done_g < len(eg) and eg[done_g].query():
+            done_g += 1
+        while done_c < len(ec) and ec[done_c].query():
+            done_c += 1
+        busy = True
+        if len(eg) - done_g < depth:
+            with torch.cuda.stream(sg):
+                for _ in range(gemm_batch):
+                    gemm.run()
+                e = torch.cuda.Event(enable_timing=True)
+                e.record(sg)
+                eg.append(e)
+            busy = False
+        if len(ec) - done_c < depth:
+            wl.dc.execute(sc)
             e = torch.cuda.Event(enable_timing=True)
-            e.record(sg)
-            eg.append(e)
-        wl.dc.execute(sc)
-        e = torch.cuda.Event(enable_timing=True)
-        e.record(sc)
-        ec.append(e)
-        if len(eg) > 20:
-            eg[-20].synchronize()
-        if len(ec) > 20:
-            ec[-20].synchronize()
+            e.record(sc)
+            ec.append(e)
+            busy = False
+        if busy:
+            time.sleep(0.0002)
     torch.cuda.synchronize()
     wl.dc.check()
     tg = np.array([base.elapsed_time(e) for e in eg])

@@ -10,6 +10,16 @@ from paper_2608_00358_b200 import synth
 
 pytestmark = pytest.mark.gpu
 DTYPES = [hb.FP32, hb.BF16, hb.FP16]
+ENGINES = [hb.ENGINE_LSU, hb.ENGINE_BULK]
+
+
+@pytest.fixture(params=ENGINES, ids=["lsu", "bulk"])
+def engine(request):
+    return request.param
+
+
+def _with(opts, engine):
+    return dict(opts or {}, engine=engine)
 
 
 def _check_allreduce(R, n, dt, algo, opts, X=None, iters=1, misalign=0):
@@ -28,44 +38,44 @@ def _check_allreduce(R, n, dt, algo, opts, X=None, iters=1, misalign=0):
 @pytest.mark.parametrize("dt", DTYPES)
 @pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED])
 @pytest.mark.parametrize("R,n", [(1, 5), (2, 9), (3, 2), (4, 257), (5, 1000), (8, 4099), (4, 0), (4, 3), (8, 100003)])
-def test_allreduce_small(R, n, dt, algo):
-    _check_allreduce(R, n, dt, algo, dict(tile_bytes=1024, chunk_bytes=4096, chain_group=2, sm_budget=8), iters=2)
+def test_allreduce_small(R, n, dt, algo, engine):
+    _check_allreduce(R, n, dt, algo, _with(dict(tile_bytes=1024, chunk_bytes=4096, chain_group=2, sm_budget=8), engine), iters=2)
 
 
 @pytest.mark.parametrize("budget", [1, 2, 3, 8, 148, 296])
 @pytest.mark.parametrize("dt", [hb.FP32, hb.BF16])
-def test_allreduce_any_sm_budget_same_bits(budget, dt):
-    _check_allreduce(6, 50021, dt, hb.ALGO_RING, dict(tile_bytes=2048, chunk_bytes=16384, sm_budget=budget), iters=3)
+def test_allreduce_any_sm_budget_same_bits(budget, dt, engine):
+    _check_allreduce(6, 50021, dt, hb.ALGO_RING, _with(dict(tile_bytes=2048, chunk_bytes=16384, sm_budget=budget), engine), iters=3)
 
 
 @pytest.mark.parametrize("misalign", [2, 4, 6, 10])
 @pytest.mark.parametrize("dt", DTYPES)
-def test_allreduce_misaligned_buffers(misalign, dt):
+def test_allreduce_misaligned_buffers(misalign, dt, engine):
     if dt == hb.FP32 and misalign % 4:
         pytest.skip("buffers must be aligned to the element size")
-    _check_allreduce(4, 10007, dt, hb.ALGO_RING, dict(tile_bytes=4096, sm_budget=16), misalign=misalign)
-    _check_allreduce(4, 10007, dt, hb.ALGO_ONESHOT, dict(tile_bytes=4096, sm_budget=16), misalign=misalign)
+    _check_allreduce(4, 10007, dt, hb.ALGO_RING, _with(dict(tile_bytes=4096, sm_budget=16), engine), misalign=misalign)
+    _check_allreduce(4, 10007, dt, hb.ALGO_ONESHOT, _with(dict(tile_bytes=4096, sm_budget=16), engine), misalign=misalign)
 
 
-def test_config1_allreduce_ring_r4_fp32():
+def test_config1_allreduce_ring_r4_fp32(engine):
     X = synth.uniform_ranks(4, 1 << 20, hb.FP32, seed=0)
-    _check_allreduce(4, 1 << 20, hb.FP32, hb.ALGO_RING, None, X=X, iters=3)
+    _check_allreduce(4, 1 << 20, hb.FP32, hb.ALGO_RING, _with(None, engine), X=X, iters=3)
 
 
 @pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT])
 @pytest.mark.parametrize("m", [4096, 65536, 262144, 1 << 20])
-def test_config5_allreduce_r8_bf16(m, algo):
+def test_config5_allreduce_r8_bf16(m, algo, engine):
     X = synth.normal_ranks(8, m // 2, hb.BF16, seed=m)
-    _check_allreduce(8, m // 2, hb.BF16, algo, None, X=X, iters=3)
+    _check_allreduce(8, m // 2, hb.BF16, algo, _with(None, engine), X=X, iters=3)
 
 
-def test_closed_form_on_device():
+def test_closed_form_on_device(engine):
     for dt in DTYPES:
         for R in (2, 4, 8, 16):
             n = 3000
             X = [synth.to_bits(np.full(n, r + 1, dtype=np.float32), dt) for r in range(R)]
             for algo in (hb.ALGO_RING, hb.ALGO_ONESHOT):
-                Y = run_plan(hb.hccl_plan_allreduce(R, n, dt, algo, dict(tile_bytes=1024)), X)
+                Y = run_plan(hb.hccl_plan_allreduce(R, n, dt, algo, _with(dict(tile_bytes=1024), engine)), X)
                 for r in range(R):
                     assert np.all(synth.from_bits(Y[r].view(np_dtype(dt)), dt) == R * (R + 1) / 2)
 
@@ -73,11 +83,11 @@ def test_closed_form_on_device():
 @pytest.mark.parametrize("dt", DTYPES)
 @pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_RING_FUSED])
 @pytest.mark.parametrize("R,counts", [(2, [3, 4]), (4, None), (5, [0, 7, 1000, 1, 300]), (16, None), (3, [0, 0, 11])])
-def test_reducescatter_small(R, counts, dt, algo):
+def test_reducescatter_small(R, counts, dt, algo, engine):
     n = 40099 if counts is None else sum(counts)
     rc = np.diff(orc.floor_chunk_offsets(n, R)) if counts is None else np.array(counts)
     X = synth.normal_ranks(R, n, dt, seed=R + n, std=0.02)
-    p = hb.hccl_plan_reducescatter(R, counts, n, dt, algo, dict(tile_bytes=1024, chunk_bytes=2048, chain_group=3, sm_budget=16))
+    p = hb.hccl_plan_reducescatter(R, counts, n, dt, algo, _with(dict(tile_bytes=1024, chunk_bytes=2048, chain_group=3, sm_budget=16), engine))
     Y = run_plan(p, X, iters=2)
     want, bitwise, exact = orc.reducescatter(dt, X, rc), orc.reducescatter_ring_f32(dt, X, rc), orc.sum_f64(dt, X)
     offs = np.concatenate([[0], np.cumsum(rc)])
@@ -87,12 +97,12 @@ def test_reducescatter_small(R, counts, dt, algo):
         assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8))
 
 
-def test_config3_shape_reducescatter_r16_bf16_reduced_size():
+def test_config3_shape_reducescatter_r16_bf16_reduced_size(engine):
     # config 3 at 1/16 of its size (4 Mi elements per rank, 2 MiB granules -> still several granules per shard? no:
     # shards of 256 Ki elements = 512 KiB, so use 128 KiB granules to keep 4 granules per shard)
     R, n = 16, 1 << 22
     X = synth.normal_ranks(R, n, hb.BF16, seed=3, std=0.02)
-    p = hb.hccl_plan_reducescatter(R, None, n, hb.BF16, hb.ALGO_RING, dict(chunk_bytes=128 << 10))
+    p = hb.hccl_plan_reducescatter(R, None, n, hb.BF16, hb.ALGO_RING, _with(dict(chunk_bytes=128 << 10), engine))
     Y = run_plan(p, X, iters=2)
     rc = np.full(R, n // R)
     want, bitwise = orc.reducescatter(hb.BF16, X, rc), orc.reducescatter_ring_f32(hb.BF16, X, rc)
@@ -104,11 +114,11 @@ def test_config3_shape_reducescatter_r16_bf16_reduced_size():
 
 @pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT])
 @pytest.mark.parametrize("R,counts", [(1, [5]), (4, [3, 0, 1000, 17]), (8, None)])
-def test_allgather(R, counts, algo):
+def test_allgather(R, counts, algo, engine):
     cs = counts if counts is not None else [32100] * R
     rng = np.random.default_rng(R)
     X = [rng.integers(0, 65536, size=c, dtype=np.uint16) for c in cs]
-    p = hb.hccl_plan_allgather(R, counts, 32100, hb.BF16, algo, dict(tile_bytes=4096, sm_budget=32))
+    p = hb.hccl_plan_allgather(R, counts, 32100, hb.BF16, algo, _with(dict(tile_bytes=4096, sm_budget=32), engine))
     Y = run_plan(p, X, iters=2)
     want = orc.allgatherv(X)
     for r in range(R):
@@ -129,37 +139,37 @@ def _a2a(R, C, SD, RD, X, dt, row_elems, opts, packed, iters=1, misalign=0):
 @pytest.mark.parametrize("R", [1, 2, 3, 5, 8])
 @pytest.mark.parametrize("packed", [True, False])
 @pytest.mark.parametrize("row_elems", [7, 128])
-def test_alltoallv_small(R, packed, row_elems):
+def test_alltoallv_small(R, packed, row_elems, engine):
     from test_planner_host import _a2a_case
     C, SD, RD, X, rb = _a2a_case(R, 100 + R, row_elems, hb.BF16, hi=40, packed=packed)
-    _a2a(R, C, SD, RD, X, hb.BF16, row_elems, dict(tile_bytes=1024, sm_budget=16), packed, iters=2)
+    _a2a(R, C, SD, RD, X, hb.BF16, row_elems, _with(dict(tile_bytes=1024, sm_budget=16), engine), packed, iters=2)
 
 
 @pytest.mark.parametrize("misalign", [1, 3, 8])
-def test_alltoallv_misaligned(misalign):
+def test_alltoallv_misaligned(misalign, engine):
     from test_planner_host import _a2a_case
     C, SD, RD, X, rb = _a2a_case(4, 7, 5, hb.FP16, hi=300, packed=True)
-    _a2a(4, C, SD, RD, X, hb.FP16, 5, dict(tile_bytes=4096), True, misalign=misalign)
+    _a2a(4, C, SD, RD, X, hb.FP16, 5, _with(dict(tile_bytes=4096), engine), True, misalign=misalign)
 
 
-def test_config2_alltoallv_r8_bf16_rows128():
+def test_config2_alltoallv_r8_bf16_rows128(engine):
     R, row_elems = 8, 128
     C = synth.uniform_counts(R, 0, hi=4096)
     assert int(C.sum()) == 133647                       # the seed-0 draw this config is quoted on
     SD, RD = orc.packed_displs(C)
     X = [synth.normal_ranks(1, int(C[s].sum()) * row_elems, hb.BF16, seed=1000 + s)[0].view(np.uint8) for s in range(R)]
-    Y = _a2a(R, C, SD, RD, X, hb.BF16, row_elems, None, True, iters=3)
+    Y = _a2a(R, C, SD, RD, X, hb.BF16, row_elems, _with(None, engine), True, iters=3)
     # identity invariant: exchanging back with the transposed counts restores every send buffer
     CT = C.T.copy()
     SD2, RD2 = orc.packed_displs(CT)
-    p2 = hb.hccl_plan_alltoallv(R, CT, None, None, None, hb.BF16, row_elems)
+    p2 = hb.hccl_plan_alltoallv(R, CT, None, None, None, hb.BF16, row_elems, _with(None, engine))
     Z = run_plan(p2, Y)
     for s in range(R):
         assert np.array_equal(Z[s], X[s])
 
 
-def test_alltoallv_zero_everything():
-    p = hb.hccl_plan_alltoallv(3, np.zeros((3, 3), dtype=np.int64), None, None, None, hb.BF16, 128)
+def test_alltoallv_zero_everything(engine):
+    p = hb.hccl_plan_alltoallv(3, np.zeros((3, 3), dtype=np.int64), None, None, None, hb.BF16, 128, _with(None, engine))
     run_plan(p, [np.zeros(16, dtype=np.uint8)] * 3, iters=2)
 
 

@@ -163,12 +163,13 @@ def test_wqe_validation():
 @pytest.mark.gpu
 @pytest.mark.parametrize("name", sorted(CASES) + ["signal_pair"])
 @pytest.mark.parametrize("budget", [1, 2, 8])
-def test_dependency_kind_on_gpu(name, budget):
+@pytest.mark.parametrize("engine", [hb.ENGINE_LSU, hb.ENGINE_BULK], ids=["lsu", "bulk"])
+def test_dependency_kind_on_gpu(name, budget, engine):
     from gpu_helpers import run_plan
     g, want = (g_signal_pair() if name == "signal_pair" else CASES[name](True))
     R = len(want(_x(3)))
     X = _x(R, seed=3)
-    p = g.compile(dict(OPTS, sm_budget=budget))
+    p = g.compile(dict(OPTS, sm_budget=budget, engine=engine))
     Y = run_plan(p, X, iters=5)
     for r, w in enumerate(want(X)):
         assert np.array_equal(Y[r].view(np.float32), w), (name, r)
