@@ -236,6 +236,34 @@ hccl_status_t hccl_plan_bind(hccl_plan_t*, void* dev_workspace, size_t bytes, vo
  * (in-place operation is not supported). */
 hccl_status_t hccl_execute(hccl_plan_t*, const void* const* sendbufs, void* const* recvbufs, void* stream);
 
+/* Execution for callers that cannot allocate device memory. (The paper has no counterpart to this call;
+ * it exists for the library's users.) Some callers must not call cudaMalloc at the point where they need a
+ * collective: code that runs under a framework allocator's lock or inside its out-of-memory and
+ * garbage-collection hooks, where asking for memory again would deadlock; processes that have already
+ * handed every free byte of the GPU to another pool, so that cudaMalloc simply fails; and latency-critical
+ * sections that cannot take the device-wide synchronisation cudaMalloc may imply. For them the library
+ * carries its own workspace: a fixed array of HCCL_NOALLOC_WORKSPACE_BYTES = 8 MiB in the library's device
+ * image, which every GPU that loads the library holds until the process exits.
+ *
+ * Runs `plan` once with that array in place of a bound workspace (the plan need not be bound; a bound
+ * plan's own workspace and epoch are not touched). The register-path executor is used whatever
+ * opts.engine says. sendbufs/recvbufs as in hccl_execute. Plans whose hccl_plan_workspace_bytes exceed
+ * 8 MiB are refused with HCCL_ERR_WORKSPACE (for reductions on 16-bit data choose a small opts.chunk_bytes:
+ * the FP32 scratch is 2 * chain_group granules); plans with a trigger are refused with
+ * HCCL_ERR_INVALID_ARG. The call allocates nothing on the device: it calls no cudaMalloc/cudaFree and no
+ * allocating library routine.
+ *
+ * All calls share the one array, and it keeps the previous call's contents: each call rewrites the
+ * tables, control words, dependency counters and signal slots before launching, and leaves the FP32
+ * scratch as it is (every execution writes a scratch slot before reading it). Two calls that overlap on
+ * the GPU would race on the array; within one process the library serialises them, and the call therefore
+ * BLOCKS: it waits for `stream` and returns the device-side verdict (HCCL_OK, HCCL_ERR_TIMEOUT,
+ * HCCL_ERR_BAD_DESCRIPTOR) directly. Calls from different processes use different copies of the array.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current); make that first call outside any stream capture. */
+#define HCCL_NOALLOC_WORKSPACE_BYTES (8u << 20)
+hccl_status_t hccl_execute_noalloc(hccl_plan_t*, const void* const* sendbufs, void* const* recvbufs, void* stream);
+
 /* The same through HOST data: copies each host_send[r] (send extent of rank r) into dev_send[r], executes,
  * and copies each receive extent back into host_recv[r]; all asynchronous on `stream` (use pinned host
  * memory for true asynchrony). Device staging buffers are the caller's. */

@@ -23,6 +23,7 @@ BUF_SEND, BUF_RECV, BUF_SCRATCH, BUF_SIGNAL, BUF_USER_SIGNAL = range(5)
 DEP_FENCE, DEP_SYNC, DEP_WQE_SYNC, DEP_RECV_SYNC, DEP_SEND_SYNC, DEP_ELEMENTWISE = 1, 2, 4, 8, 16, 32
 CMP_EQ, CMP_NE, CMP_GE, CMP_GT, CMP_LE, CMP_LT = range(6)
 MAX_RANKS = 256
+NOALLOC_WORKSPACE_BYTES = 8 << 20
 ELEM_BYTES = {FP32: 4, BF16: 2, FP16: 2}
 
 
@@ -78,6 +79,7 @@ def _load() -> C.CDLL:
         "hccl_plan_bind": [P, P, C.c_size_t, P],
         "hccl_execute": [P, C.POINTER(P), C.POINTER(P), P],
         "hccl_execute_host": [P, C.POINTER(P), C.POINTER(P), C.POINTER(P), C.POINTER(P), P],
+        "hccl_execute_noalloc": [P, C.POINTER(P), C.POINTER(P), P],
         "hccl_plan_set_user_signals": [P, P, C.c_int64],
         "hccl_plan_set_trigger": [P, C.c_int64, C.c_int32, C.c_uint64, C.c_uint64, C.c_int64, C.c_uint64, C.c_uint64],
         "hccl_plan_status": [P, C.POINTER(C.c_int), I64P],
@@ -108,6 +110,7 @@ LIBRARY_PATH = _build.LIB
 EXPORTS = ["hccl_plan_allreduce", "hccl_plan_reducescatter", "hccl_plan_allgather", "hccl_plan_alltoallv",
            "hccl_graph_create", "hccl_graph_add_subgraph", "hccl_graph_add_wqe", "hccl_graph_compile",
            "hccl_graph_destroy", "hccl_plan_workspace_bytes", "hccl_plan_bind", "hccl_execute", "hccl_execute_host",
+           "hccl_execute_noalloc",
            "hccl_plan_set_user_signals", "hccl_plan_set_trigger", "hccl_plan_status", "hccl_plan_info",
            "hccl_plan_extents", "hccl_plan_destroy", "hccl_status_string", "hccl_last_cuda_error", "hccl_version",
            "hccl_plan_check_hazards", "hccl_plan_interpret_host"]
@@ -186,6 +189,12 @@ class Plan:
     def execute_host(self, host_send, host_recv, dev_send, dev_recv, stream: int = 0):
         _chk(_lib.hccl_execute_host(self._h, _ptr_array(host_send), _ptr_array(host_recv), _ptr_array(dev_send),
                                     _ptr_array(dev_recv), C.c_void_p(stream)), "hccl_execute_host")
+
+    def execute_noalloc(self, sendbufs: Sequence[int], recvbufs: Sequence[int], stream: int = 0):
+        """One blocking execution on the library's built-in 8 MiB workspace (for callers that cannot
+        allocate device memory). Raises HcclError with the device-side verdict if it failed."""
+        _chk(_lib.hccl_execute_noalloc(self._h, _ptr_array(sendbufs), _ptr_array(recvbufs), C.c_void_p(stream)),
+             "hccl_execute_noalloc")
 
     def set_user_signals(self, dev_signals: int, n_slots: int):
         _chk(_lib.hccl_plan_set_user_signals(self._h, C.c_void_p(dev_signals), n_slots), "hccl_plan_set_user_signals")

@@ -17,6 +17,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <vector>
 
 #include "plan.hpp"
@@ -1181,3 +1182,104 @@ hccl_status_t hccl_plan_status(hccl_plan_t* p, hccl_status_t* device_status, int
 }
 
 }  // extern "C"
+
+// ====================================================================== execution without any allocation
+// Workspace for callers that cannot obtain device memory of their own: one array that lives in the
+// library's device image for the life of the process (every GPU that loads the library holds it).
+#define HCCL_NOALLOC_WORKSPACE_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_workspace[HCCL_NOALLOC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_noalloc_addr[kMaxDevices] = {};  // device address of g_noalloc_workspace, per device ordinal
+std::mutex g_noalloc_mu;
+}  // namespace
+
+extern "C" hccl_status_t hccl_execute_noalloc(hccl_plan_t* p, const void* const* sendbufs, void* const* recvbufs, void* stream) {
+    if (!p || !sendbufs || !recvbufs) return HCCL_ERR_INVALID_ARG;
+    if (p->layout.total > HCCL_NOALLOC_WORKSPACE_BYTES) {
+        snprintf(g_cuda_err, sizeof(g_cuda_err), "plan needs %llu workspace bytes; the built-in workspace holds %u",
+                 (unsigned long long)p->layout.total, HCCL_NOALLOC_WORKSPACE_BYTES);
+        return HCCL_ERR_WORKSPACE;
+    }
+    if (p->trig_wait_slot >= 0 || p->trig_set_slot >= 0) return HCCL_ERR_INVALID_ARG;  // triggers belong to bound plans
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return HCCL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);  // one user of the array at a time from this process
+    if (!g_noalloc_addr[dev]) {
+        // In host code the array's name is only a handle; its device address on the current device is
+        // looked up once here and that address is what the kernel receives.
+        void* ptr = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_workspace));
+        if (!ptr || ((uintptr_t)ptr % 256) != 0) return HCCL_ERR_ALIGNMENT;
+        g_noalloc_addr[dev] = ptr;
+    }
+    char* ws = (char*)g_noalloc_addr[dev];
+    // same aliasing rules as hccl_execute, checked on every call (nothing is cached for this path)
+    const int R = p->R;
+    for (int r = 0; r < R; ++r) {
+        if ((p->send_bytes[r] > 0 && !sendbufs[r]) || (p->recv_bytes[r] > 0 && !recvbufs[r])) return HCCL_ERR_INVALID_ARG;
+        if (((uintptr_t)sendbufs[r] | (uintptr_t)recvbufs[r]) & (uintptr_t)(p->buf_align - 1)) return HCCL_ERR_ALIGNMENT;
+    }
+    for (int d = 0; d < R; ++d) {
+        const uintptr_t lo = (uintptr_t)recvbufs[d], hi = lo + (uintptr_t)p->recv_bytes[d];
+        if (lo == hi) continue;
+        for (int s = 0; s < R; ++s) {
+            const uintptr_t slo = (uintptr_t)sendbufs[s], shi = slo + (uintptr_t)p->send_bytes[s];
+            if (slo != shi && lo < shi && slo < hi) return HCCL_ERR_OVERLAP;
+            const uintptr_t rlo = (uintptr_t)recvbufs[s], rhi = rlo + (uintptr_t)p->recv_bytes[s];
+            if (s > d && rlo != rhi && lo < rhi && rlo < hi) return HCCL_ERR_OVERLAP;
+        }
+    }
+    // The array keeps whatever the previous call left. Everything that must start at zero (control words,
+    // dependency counters, signal slots) is rewritten together with this plan's tables; the FP32 scratch
+    // behind them is always written before it is read within one execution, so it is left as it is.
+    const Layout& L = p->layout;
+    static thread_local std::vector<char> img;
+    img.assign((size_t)L.scratch, 0);
+    if (!p->descs.empty()) std::memcpy(img.data() + L.descs, p->descs.data(), p->descs.size() * sizeof(Desc));
+    if (!p->tiles.empty()) std::memcpy(img.data() + L.tiles, p->tiles.data(), p->tiles.size() * sizeof(Tile));
+    if (!p->waits.empty()) std::memcpy(img.data() + L.waits, p->waits.data(), p->waits.size() * sizeof(Wait));
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_TRY(cudaMemcpyAsync(ws, img.data(), img.size(), cudaMemcpyHostToDevice, st));
+    static thread_local ExecParams prm;
+    prm.descs = (const Desc*)(ws + L.descs);
+    prm.tiles = (const Tile*)(ws + L.tiles);
+    prm.waits = (const Wait*)(ws + L.waits);
+    prm.counters = (uint32_t*)(ws + L.counters);
+    prm.signals = (unsigned long long*)(ws + L.signals);
+    prm.ctl = (Control*)(ws + L.control);
+    prm.scratch = ws + L.scratch;
+    prm.user_signals = nullptr;
+    prm.n_tiles = (uint32_t)p->tiles.size();
+    prm.n_descs = (uint32_t)p->descs.size();
+    prm.n_syncs = (uint32_t)p->sync_per_epoch.size();
+    prm.n_waits = (uint32_t)p->waits.size();
+    prm.n_signals = (uint32_t)p->n_signals;
+    prm.R = (uint32_t)R;
+    prm.epoch = 1;  // the tables were just reset, so every call is a first execution
+    prm.timeout_ns = p->opts.timeout_ns;
+    prm.n_user_signals = 0;
+    prm.trig_wait_slot = -1;
+    prm.trig_set_slot = -1;
+    prm.trig_cmp = 0;
+    prm.trig_wait_value = prm.trig_set_value = 0;
+    for (int r = 0; r < R; ++r) {
+        prm.send[r] = sendbufs[r];
+        prm.recv[r] = recvbufs[r];
+    }
+    int blocks = p->opts.sm_budget;
+    if ((uint32_t)blocks > prm.n_tiles) blocks = (int)std::max<uint32_t>(prm.n_tiles, 1u);
+    prm.nblocks = (uint32_t)blocks;
+    hccl_executor_lsu<<<blocks, p->opts.threads, 0, st>>>(prm);
+    CUDA_TRY(cudaGetLastError());
+    // This call owns the shared array until its kernel is done, so it waits here and hands back the
+    // device-side verdict itself.
+    CUDA_TRY(cudaStreamSynchronize(st));
+    Control c;
+    CUDA_TRY(cudaMemcpy(&c, ws + L.control, sizeof(c), cudaMemcpyDeviceToHost));
+    if (c.fail_epoch == 1) return (hccl_status_t)c.status;
+    if (c.done_epoch != 1) return HCCL_ERR_BUSY;
+    return HCCL_OK;
+}
