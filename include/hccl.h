@@ -93,7 +93,11 @@ typedef struct {
     int32_t chain_group;    /* chains scheduled together in chain-group-major order (default 8) */
     int32_t threads;        /* threads per block, multiple of 32 (default 512) */
     int32_t stages;         /* bulk engine: shared-memory stages of 32 KiB per block, 2..8 (default 6) */
-    int32_t reserved[4];
+    int32_t cluster;        /* register engine: launch blocks in clusters of this size (2, 4, 8) so that they sit on
+                               neighbouring SMs; 0/1 = no clusters. Ignored unless it divides the block count. */
+    int32_t light;          /* register engine: nonzero = the 64-register build (several blocks per SM) */
+    int32_t copy_by_warps;  /* bulk engine: nonzero = COPY pieces are loaded by the bulk unit but stored by the compute warps */
+    int32_t reserved[1];
 } hccl_opts_t;
 
 typedef struct hccl_plan hccl_plan_t;   /* opaque, host-owned: a compiled, cacheable work packet (Sec. V-B) */
@@ -188,6 +192,10 @@ typedef struct {
  * responsible for the claim; hccl_plan_check_hazards verifies it tile by tile. */
 #define HCCL_DEP_ELEMENTWISE 32u
 
+/* Cache hints on data WQEs. READ_ONCE: no source byte of this WQE is read by any other WQE of the packet
+ * (it is streamed through the L2 with an evict-first policy). */
+#define HCCL_HINT_READ_ONCE 1
+
 typedef enum { HCCL_CMP_EQ = 0, HCCL_CMP_NE = 1, HCCL_CMP_GE = 2, HCCL_CMP_GT = 3, HCCL_CMP_LE = 4, HCCL_CMP_LT = 5 } hccl_cmp_t;
 
 typedef struct {
@@ -200,7 +208,7 @@ typedef struct {
     int64_t dep_wqe;                  /* with HCCL_DEP_WQE_SYNC */
     int64_t dep_wqe2;                 /* optional second WQE_SYNC target, -1 if unused */
     int32_t cmp;                      /* WAIT: hccl_cmp_t */
-    int32_t reserved;
+    int32_t hints;                    /* data WQEs: HCCL_HINT_* */
     int64_t tile_count;               /* tile size in units of count; 0 = derived from opts.tile_bytes */
     uint64_t value, value_per_epoch;  /* WAIT/SET: effective value = value + epoch*value_per_epoch, epoch = 1,2,.. per execute */
 } hccl_wqe_t;

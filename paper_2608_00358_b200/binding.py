@@ -22,6 +22,7 @@ OP_COPY, OP_REDUCE, OP_REDUCE_N, OP_WAIT, OP_SET, OP_NOOP = range(6)
 BUF_SEND, BUF_RECV, BUF_SCRATCH, BUF_SIGNAL, BUF_USER_SIGNAL = range(5)
 DEP_FENCE, DEP_SYNC, DEP_WQE_SYNC, DEP_RECV_SYNC, DEP_SEND_SYNC, DEP_ELEMENTWISE = 1, 2, 4, 8, 16, 32
 CMP_EQ, CMP_NE, CMP_GE, CMP_GT, CMP_LE, CMP_LT = range(6)
+HINT_READ_ONCE = 1
 MAX_RANKS = 256
 NOALLOC_WORKSPACE_BYTES = 8 << 20
 ELEM_BYTES = {FP32: 4, BF16: 2, FP16: 2}
@@ -30,7 +31,8 @@ ELEM_BYTES = {FP32: 4, BF16: 2, FP16: 2}
 class Opts(C.Structure):
     _fields_ = [("sm_budget", C.c_int32), ("engine", C.c_int32), ("chunk_bytes", C.c_uint64),
                 ("tile_bytes", C.c_uint64), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
-                ("chain_group", C.c_int32), ("threads", C.c_int32), ("stages", C.c_int32), ("reserved", C.c_int32 * 4)]
+                ("chain_group", C.c_int32), ("threads", C.c_int32), ("stages", C.c_int32), ("cluster", C.c_int32), ("light", C.c_int32),
+                ("copy_by_warps", C.c_int32), ("reserved", C.c_int32 * 1)]
 
 
 class Ref(C.Structure):
@@ -41,7 +43,7 @@ class Wqe(C.Structure):
     _fields_ = [("op", C.c_int32), ("dtype_dst", C.c_int32), ("dtype_a", C.c_int32), ("dtype_b", C.c_int32),
                 ("dst", Ref), ("a", Ref), ("b", Ref), ("count", C.c_int64), ("nsrc", C.c_int32),
                 ("dep_flags", C.c_uint32), ("dep_wqe", C.c_int64), ("dep_wqe2", C.c_int64), ("cmp", C.c_int32),
-                ("reserved", C.c_int32), ("tile_count", C.c_int64), ("value", C.c_uint64),
+                ("hints", C.c_int32), ("tile_count", C.c_int64), ("value", C.c_uint64),
                 ("value_per_epoch", C.c_uint64)]
 
 
@@ -273,7 +275,7 @@ class Graph:
 
     def add_wqe(self, subgraph: int, op: int, dst=None, a=None, b=None, count: int = 0, dtypes=(FP32, FP32, FP32),
                 nsrc: int = 0, dep_flags: int = 0, dep_wqe: int = -1, dep_wqe2: int = -1, cmp: int = 0,
-                value: int = 0, value_per_epoch: int = 0, tile_count: int = 0) -> int:
+                value: int = 0, value_per_epoch: int = 0, tile_count: int = 0, hints: int = 0) -> int:
         w = Wqe()
         w.op = op
         w.dtype_dst, w.dtype_a, w.dtype_b = dtypes
@@ -281,7 +283,7 @@ class Graph:
             if r is not None:
                 setattr(w, name, Ref(*r))
         w.count, w.nsrc, w.dep_flags, w.dep_wqe, w.dep_wqe2 = count, nsrc, dep_flags, dep_wqe, dep_wqe2
-        w.cmp, w.value, w.value_per_epoch, w.tile_count = cmp, value, value_per_epoch, tile_count
+        w.cmp, w.value, w.value_per_epoch, w.tile_count, w.hints = cmp, value, value_per_epoch, tile_count, hints
         wid = C.c_int64()
         _chk(_lib.hccl_graph_add_wqe(self._h, subgraph, C.byref(w), C.byref(wid)), "hccl_graph_add_wqe")
         return wid.value

@@ -79,6 +79,7 @@ hccl_status_t emit_ring(hccl_graph* g, int R, int dt, const std::vector<Chain>& 
                 if (is_rs && fused) {
                     // the whole chain as one multi-input sum, same order: X_{c+1}, X_{c+2}, ..., X_c
                     w.op = HCCL_OP_REDUCE_N;
+                    w.hints = HCCL_HINT_READ_ONCE;
                     w.dtype_dst = w.dtype_a = dt;
                     w.nsrc = R;
                     w.a = ref(HCCL_BUF_SEND, (c + 1) % R, ch.e0 * es);
@@ -148,15 +149,25 @@ hccl_status_t emit_ring(hccl_graph* g, int R, int dt, const std::vector<Chain>& 
     return HCCL_OK;
 }
 
-int64_t pick_tile_elems(int64_t weight_bytes, const hccl_opts_t& o, int widest) {
-    uint64_t tb = o.tile_bytes;
-    if (tb == 0) {
-        uint64_t per = (uint64_t)weight_bytes / (8ull * (uint64_t)o.sm_budget);
-        uint64_t p2 = 1;
-        while (p2 * 2 <= per) p2 *= 2;
-        tb = std::min<uint64_t>(256u << 10, std::max<uint64_t>(16u << 10, p2));
-    }
-    return std::max<int64_t>(64, (int64_t)(tb / (uint64_t)widest));
+// Tile size in elements for a schedule whose widest operand has `widest` bytes per element. With
+// opts.tile_bytes unset the size follows the total work (about 8 tiles per block, 16..256 KiB) and is
+// rounded to whole passes of the block's threads for operation `op`.
+int64_t pick_tile_elems(int64_t weight_bytes, const hccl_opts_t& o, int widest, int op) {
+    if (o.tile_bytes) return std::max<int64_t>(64, (int64_t)(o.tile_bytes / (uint64_t)widest));
+    uint64_t per = (uint64_t)weight_bytes / (8ull * (uint64_t)o.sm_budget);
+    uint64_t p2 = 1;
+    while (p2 * 2 <= per) p2 *= 2;
+    const uint64_t tb = std::min<uint64_t>(256u << 10, std::max<uint64_t>(16u << 10, p2));
+    return round_tile((int64_t)(tb / (uint64_t)widest), sweep_of(o, op));
+}
+
+// Copy-only schedules: with the engine left to the library, the bulk copy unit moves the bytes
+// (measured a few percent ahead of the register path at full budget, and no thread touches the data).
+void fill_copy_opts(hccl_opts_t* o, const hccl_opts_t* in) {
+    hccl_opts_t tmp;
+    if (in) tmp = *in; else std::memset(&tmp, 0, sizeof(tmp));
+    if (tmp.engine == HCCL_ENGINE_AUTO) tmp.engine = HCCL_ENGINE_BULK;
+    fill_default_opts(o, &tmp);
 }
 
 std::vector<Chain> make_chains(int R, const std::vector<int64_t>& offs, bool scatter, int64_t granule_elems) {
@@ -233,7 +244,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     const int64_t slot_elems = (int64_t)align_up((uint64_t)maxlen, 64);
     const int64_t scratch = need_scratch ? (int64_t)n_slots * slot_elems * 4 * (staged ? 2 : 1) : 0;
     const int64_t weight = count * 4 * (R - 1) + (int64_t)count * es * (R - 1);
-    const int64_t tile_elems = pick_tile_elems(weight, o, in_recv || fused ? es : 4);
+    const int64_t tile_elems = fused ? pick_tile_elems((int64_t)count * es * R, o, es * R / 4, HCCL_OP_REDUCE_N) : pick_tile_elems(weight, o, in_recv ? es : 4, HCCL_OP_REDUCE);
 
     hccl_graph* graw = nullptr;
     CHECK(hccl_graph_create(R, ext.data(), ext.data(), scratch, 0, &graw));
@@ -292,7 +303,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     const int n_slots = need_scratch ? (int)std::min<size_t>(chains.size(), slots_wanted) : 0;
     const int64_t slot_elems = (int64_t)align_up((uint64_t)maxlen, 64);
     const int64_t scratch = need_scratch ? (int64_t)n_slots * slot_elems * 4 * (staged ? 2 : 1) : 0;
-    const int64_t tile_elems = pick_tile_elems(count * 4 * (R - 1), o, fused ? es : 4);
+    const int64_t tile_elems = fused ? pick_tile_elems((int64_t)count * es * R, o, es * R / 4, HCCL_OP_REDUCE_N) : pick_tile_elems(count * 4 * (R - 1), o, 4, HCCL_OP_REDUCE);
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), scratch, 0, &graw));
     GraphPtr g(graw);
     g->compulsory_bytes = compulsory;
@@ -306,7 +317,7 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
     if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
-    fill_default_opts(&o, opts);
+    fill_copy_opts(&o, opts);
     const int es = elem_bytes(dt);
     std::vector<int64_t> offs(R + 1, 0), sext(R), rext(R);
     for (int r = 0; r < R; ++r) {
@@ -320,7 +331,7 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw));
     GraphPtr g(graw);
     g->compulsory_bytes = offs[R] * es + (int64_t)R * offs[R] * es;
-    const int64_t tile = pick_tile_elems(offs[R] * es * R, o, 1);
+    const int64_t tile = pick_tile_elems(offs[R] * es * R, o, 1, HCCL_OP_COPY);
     // one subgraph per chunk q: it first lands in its owner's receive buffer, then goes round (ring)
     // or is read by everyone directly (one-shot)
     std::vector<int32_t> sg(R);
@@ -356,7 +367,7 @@ hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_
     if (!out || !sendcounts || R < 1 || R > HCCL_MAX_RANKS || row_elems < 1) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
     hccl_opts_t o;
-    fill_default_opts(&o, opts);
+    fill_copy_opts(&o, opts);
     const int64_t row_bytes = row_elems * elem_bytes(dt);
     const size_t RR = (size_t)R * R;
     for (size_t i = 0; i < RR; ++i) {

@@ -18,6 +18,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <type_traits>
 #include <vector>
 
 #include "plan.hpp"
@@ -371,26 +372,63 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
     if (tid < head) scalar(tid);
     for (uint32_t i = head + (nv << 3) + tid; i < n; i += nth) scalar(i);
     const size_t hs = (size_t)head * Elem<DS>::BYTES;
-    for (uint32_t i = tid; i < nv; i += nth) {
-        float acc[8];
-        load8<DS, false>(src(0) + hs + (size_t)i * 8 * Elem<DS>::BYTES, acc);
-        int k = 1;
-        for (; k + 4 <= nsrc; k += 4) {
-            float x[4][8];
+    // Vector body: the loads of a group of sources are all issued before the first add, so a thread has G
+    // 16-byte (or 32-byte) requests in flight; the adds then run in source order.
+    constexpr int G = (DS == HCCL_FP32) ? 4 : 8;   // sources fetched together
+    constexpr int W = (DS == HCCL_FP32) ? 2 : 1;   // 16-byte words per 8 elements
+    const bool stream = (d.cmp & 1u) != 0;         // planner's hint: every source byte is read exactly once
+    auto widen = [](const uint4 (&raw)[W], float (&x)[8]) {
+        if constexpr (DS == HCCL_FP32) {
+            x[0] = __uint_as_float(raw[0].x); x[1] = __uint_as_float(raw[0].y);
+            x[2] = __uint_as_float(raw[0].z); x[3] = __uint_as_float(raw[0].w);
+            x[4] = __uint_as_float(raw[W - 1].x); x[5] = __uint_as_float(raw[W - 1].y);
+            x[6] = __uint_as_float(raw[W - 1].z); x[7] = __uint_as_float(raw[W - 1].w);
+        } else {
+            const uint32_t wv[4] = {raw[0].x, raw[0].y, raw[0].z, raw[0].w};
 #pragma unroll
-            for (int j = 0; j < 4; ++j) load8<DS, false>(src(k + j) + hs + (size_t)i * 8 * Elem<DS>::BYTES, x[j]);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e] = acc[e] + x[j][e];
+            for (int h = 0; h < 4; ++h) {
+                if constexpr (DS == HCCL_BF16) {
+                    x[2 * h] = __uint_as_float(wv[h] << 16);
+                    x[2 * h + 1] = __uint_as_float(wv[h] & 0xffff0000u);
+                } else {
+                    const float2 t2 = __half22float2(*reinterpret_cast<const __half2*>(&wv[h]));
+                    x[2 * h] = t2.x;
+                    x[2 * h + 1] = t2.y;
+                }
             }
         }
-        for (; k < nsrc; ++k) {
-            float x[8];
-            load8<DS, false>(src(k) + hs + (size_t)i * 8 * Elem<DS>::BYTES, x);
+    };
+    auto fetch = [&](int k, size_t off, uint4 (&raw)[W]) {
+        const uint4* q = reinterpret_cast<const uint4*>(src(k) + off);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] = acc[e] + x[e];
+        for (int w = 0; w < W; ++w) raw[w] = stream ? __ldcs(q + w) : __ldcg(q + w);
+    };
+    // A group of N consecutive sources starting at k0: N loads in flight, then N adds in source order.
+    // INIT: the group's first source starts the sum (x + 0 would turn -0 into +0).
+    auto group = [&](auto n_tag, auto init_tag, int k0, size_t off, float (&acc)[8]) {
+        constexpr int N = decltype(n_tag)::value;
+        constexpr bool INIT = decltype(init_tag)::value;
+        uint4 raw[N][W];
+#pragma unroll
+        for (int j = 0; j < N; ++j) fetch(k0 + j, off, raw[j]);
+#pragma unroll
+        for (int j = 0; j < N; ++j) {
+            float x[8];
+            widen(raw[j], x);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] = (INIT && j == 0) ? x[e] : acc[e] + x[e];
         }
+    };
+    using T = std::true_type;
+    using F = std::false_type;
+    for (uint32_t i = tid; i < nv; i += nth) {
+        const size_t off = hs + (size_t)i * 8 * Elem<DS>::BYTES;
+        float acc[8];
+        int k;
+        if (nsrc >= G) { group(std::integral_constant<int, G>{}, T{}, 0, off, acc); k = G; }
+        else { group(std::integral_constant<int, 1>{}, T{}, 0, off, acc); k = 1; }
+        for (; k + G <= nsrc; k += G) group(std::integral_constant<int, G>{}, F{}, k, off, acc);
+        for (; k < nsrc; ++k) group(std::integral_constant<int, 1>{}, F{}, k, off, acc);
         store8<DD, false>(dst + (size_t)head * Elem<DD>::BYTES + (size_t)i * 8 * Elem<DD>::BYTES, acc);
     }
 }
@@ -518,38 +556,152 @@ __device__ void leave(const ExecParams& p) {
     }
 }
 
-__global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p) {
-    __shared__ Tile s_tile;
-    __shared__ Desc s_desc;
-    __shared__ int s_go;
-    const uint32_t tid = threadIdx.x;
+// Named barriers of the register engine (id 0 is left to __syncthreads).
+__device__ __forceinline__ void named_sync(uint32_t id, uint32_t nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Loads and checks the records of work item `cur`. No waiting here.
+__device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d) {
+    t = p.tiles[cur];
+    if (!tile_ok(p, t)) {
+        fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
+        return false;
+    }
+    d = p.descs[t.desc];
+    if (!desc_ok(p, d)) {
+        fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
+        return false;
+    }
+    return true;
+}
+// One non-blocking look at every dependency counter of the item.
+__device__ bool deps_ready(const ExecParams& p, const Tile& t) {
+    for (uint32_t w = 0; w < t.wait_cnt; ++w) {
+        const Wait x = p.waits[t.wait_off + w];
+        if (x.sync >= p.n_syncs) return false;
+        if ((int32_t)(ld_acquire_u32(p.counters + x.sync) - p.epoch * x.per_epoch) < 0) return false;
+    }
+    return true;
+}
+// Blocking (bounded) part: dependency counters, then a WAIT's condition; a SET is performed here.
+__device__ bool wait_deps(const ExecParams& p, uint32_t cur, const Tile& t, const Desc& d, bool counters_done) {
+    if (!counters_done) {
+        for (uint32_t w = 0; w < t.wait_cnt; ++w) {
+            const Wait x = p.waits[t.wait_off + w];
+            if (x.sync >= p.n_syncs) {
+                fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
+                return false;
+            }
+            if (!wait_counter(p, x.sync, x.per_epoch, cur)) return false;
+        }
+    }
+    if (d.op == HCCL_OP_WAIT) {
+        const unsigned long long* addr = (d.kind_a == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + d.off_a;
+        if (!wait_signal(p, addr, d.cmp, d.value + (unsigned long long)p.epoch * d.value_per_epoch, cur)) return false;
+    } else if (d.op == HCCL_OP_SET) {
+        unsigned long long* addr = (d.kind_dst == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + d.off_dst;
+        __threadfence();
+        st_release_u64(addr, d.value + (unsigned long long)p.epoch * d.value_per_epoch);
+    }
+    return true;
+}
+
+// Register engine. Warp 0 is the control warp: its first lane claims tickets, fetches the next item's
+// records and looks at its dependency counters while the worker warps are still moving the current item,
+// and publishes an item's completion while the workers are already on the next one. Two shared-memory
+// buffers hold the current and the next item; named barriers FULL[b] (item in buffer b may start) and
+// DONE[b] (workers have stored all of it) pair the two sides.
+__device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
+    __shared__ Tile s_tile[2];
+    __shared__ Desc s_desc[2];
+    __shared__ int s_go[2];
+    const uint32_t tid = threadIdx.x, nth = blockDim.x;
+    constexpr uint32_t FULL = 1, DONE = 3;  // barrier ids FULL+b, DONE+b
+    if (tid >= 32) {
+        const uint32_t wtid = tid - 32, nwork = nth - 32;
+        for (uint32_t k = 0;; ++k) {
+            const uint32_t b = k & 1;
+            named_sync(FULL + b, nth);
+            if (!s_go[b]) break;
+            run_tile_lsu(p, s_desc[b], s_tile[b], wtid, nwork);
+            named_sync(DONE + b, nth);
+        }
+        return;
+    }
+    // ---- control warp; every lane executes the barriers, lane 0 does the rest
     uint32_t next = 0;
-    bool live = true;
+    bool live = true, have = false, ready = false;
     if (tid == 0) {
         if (p.trig_wait_slot >= 0)
             live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value, 0xffffffffu);
         next = atomicAdd(&p.ctl->ticket, 1);
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
     }
-    for (;;) {
+    uint32_t cur = 0;
+    for (uint32_t k = 0;; ++k) {
+        const uint32_t b = k & 1;
+        int32_t sig0 = -1, sig1 = -1;
+        bool prev = false;
         if (tid == 0) {
-            const uint32_t cur = next;
-            int go = 0;
-            if (live && cur < p.n_tiles && !aborted(p)) {
-                next = atomicAdd(&p.ctl->ticket, 1);  // claim ahead: its latency hides behind this item
-                go = prepare_tile(p, cur, s_tile, s_desc) ? 1 : 0;
+            // item k: its records were fetched during item k-1 (or are fetched now for the first one)
+            if (k == 0) {
+                cur = next;
+                have = live && cur < p.n_tiles && !aborted(p);
+                if (have) {
+                    next = atomicAdd(&p.ctl->ticket, 1);
+                    have = fetch_tile(p, cur, s_tile[0], s_desc[0]);
+                    ready = have && deps_ready(p, s_tile[0]);
+                }
             }
-            s_go = go;
+            prev = k > 0;
+            if (prev) {
+                sig0 = s_tile[b ^ 1].signal[0];
+                sig1 = s_tile[b ^ 1].signal[1];
+            }
         }
-        __syncthreads();
-        if (!s_go) break;
-        run_tile_lsu(p, s_desc, s_tile, tid, blockDim.x);
-        __syncthreads();
-        if (tid == 0) publish_tile(p, s_tile);
+        if (k > 0) named_sync(DONE + (b ^ 1), nth);  // the workers have stored all of item k-1
+        if (tid == 0) {
+            const bool simple = have && ready && s_desc[b].op != HCCL_OP_WAIT && s_desc[b].op != HCCL_OP_SET;
+            if (!simple && prev && (sig0 >= 0 || sig1 >= 0)) {
+                // item k may have to wait (perhaps for item k-1 itself): publish k-1 first
+                __threadfence();
+                if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
+                if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
+                sig0 = sig1 = -1;
+            }
+            bool go = have && !aborted(p);
+            if (go && !simple) go = wait_deps(p, cur, s_tile[b], s_desc[b], ready);
+            s_go[b] = go ? 1 : 0;
+        }
+        named_sync(FULL + b, nth);  // workers start item k (or leave)
+        const int go = s_go[b];
+        if (tid == 0) {
+            if (sig0 >= 0 || sig1 >= 0) {  // publish item k-1 while the workers run item k
+                __threadfence();
+                if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
+                if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
+            }
+            if (go) {
+                // look ahead: claim, fetch and poll item k+1 behind the workers' back
+                cur = next;
+                have = cur < p.n_tiles && !aborted(p);
+                if (have) {
+                    next = atomicAdd(&p.ctl->ticket, 1);
+                    have = fetch_tile(p, cur, s_tile[b ^ 1], s_desc[b ^ 1]);
+                    ready = have && deps_ready(p, s_tile[b ^ 1]);
+                }
+            }
+        }
+        if (!go) break;
     }
     if (tid == 0) leave(p);
 }
 
+__global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p) { executor_lsu_body(p); }
+// Same program compiled to at most 64 registers per thread: two 512-thread blocks (or four of 256) fit one
+// SM, and a block of 256 threads leaves three quarters of the register file to whatever else runs there.
+__global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p) { executor_lsu_body(p); }
 
 // ====================================================================== bulk (TMA) engine
 // The same dispatch and dependency protocol, but the data mover is the bulk asynchronous copy unit:
@@ -567,7 +719,10 @@ constexpr uint32_t REGION = 16384;            // bytes per operand region of a s
 constexpr uint32_t STAGE_BYTES = 2 * REGION;  // region A + region B; a COPY piece uses both as one buffer
 constexpr uint32_t PIECE_ELEMS = 4096;        // elements per REDUCE piece (fp32 fills a region exactly)
 
-enum : uint32_t { PIECE_COPY = 0, PIECE_REDUCE = 1, PIECE_TILE = 2, PIECE_EXIT = 3 };
+// PIECE_COPY: loaded and stored by the bulk unit. PIECE_COPYW: loaded by the bulk unit, stored by the compute
+// warps from shared memory (the stage is free as soon as the warps have read it, without waiting for a
+// bulk store to drain, so more of the stage ring is loads in flight).
+enum : uint32_t { PIECE_COPY = 0, PIECE_REDUCE = 1, PIECE_TILE = 2, PIECE_EXIT = 3, PIECE_COPYW = 4 };
 
 struct alignas(16) PieceInfo {  // one per stage, in shared memory; written by the DMA thread
     uint32_t kind;
@@ -734,6 +889,7 @@ struct Dma {
     unsigned long long head, tail, groups;
     unsigned long long pol;
     bool ok;
+    bool copy_by_warps;
 };
 
 // Retire the oldest outstanding piece. A COPY piece is drained to global memory here; REDUCE and TILE
@@ -867,7 +1023,7 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
                 if (!acquire_slot(p, d, k, cur)) return false;
                 const uint32_t slot = (uint32_t)(k % d.ns);
                 PieceInfo& pi = d.info[slot];
-                pi.kind = PIECE_COPY;
+                pi.kind = d.copy_by_warps ? PIECE_COPYW : PIECE_COPY;
                 pi.n = nb;
                 pi.last = (off + nb == body) ? 1u : 0u;
                 pi.tile_index = cur;
@@ -923,7 +1079,7 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
 
 }  // namespace bulk
 
-__global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns) {
+__global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t copy_by_warps) {
     using namespace bulk;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     char* stages_ptr = reinterpret_cast<char*>(smem_raw);
@@ -946,7 +1102,8 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         if (tid != 0) return;  // one elected thread drives the DMA warp
         Dma d;
         d.ns = ns;
-        d.lag = ns > 2 ? ns - 2 : 1;
+        d.lag = copy_by_warps ? ns : (ns > 2 ? ns - 2 : 1);
+        d.copy_by_warps = copy_by_warps != 0;
         d.stages = smem_u32(stages_ptr);
         d.stages_ptr = stages_ptr;
         d.full = full;
@@ -979,7 +1136,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             // stop path: no load may still be writing into this block's shared memory when it exits
             for (unsigned long long j = d.tail; j < d.head; ++j) {
                 const uint32_t slot = (uint32_t)(j % ns);
-                if (info[slot].kind == PIECE_COPY || info[slot].kind == PIECE_REDUCE)
+                if (info[slot].kind == PIECE_COPY || info[slot].kind == PIECE_REDUCE || info[slot].kind == PIECE_COPYW)
                     mbar_wait(p, full + 8 * slot, (uint32_t)((j / ns) & 1), 1000000000ull, 0xfffffffeu);
             }
         }
@@ -1004,6 +1161,14 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         if (kind == PIECE_REDUCE) {
             reduce_piece_dispatch(pi.dt_a, pi.dt_b, pi.dt_d, stages_ptr + (size_t)slot * STAGE_BYTES,
                                   stages_ptr + (size_t)slot * STAGE_BYTES + REGION, pi.dst, pi.n, ctid, cnth);
+        } else if (kind == PIECE_COPYW) {
+            const uint4* src = reinterpret_cast<const uint4*>(stages_ptr + (size_t)slot * STAGE_BYTES);
+            uint4* dst = reinterpret_cast<uint4*>(pi.dst);
+            const uint32_t nv = pi.n >> 4;
+            const bool stream = pi.evict_first != 0;
+            for (uint32_t i = ctid; i < nv; i += cnth) {
+                if (stream) __stcs(dst + i, src[i]); else __stcg(dst + i, src[i]);
+            }
         } else if (kind == PIECE_TILE) {
             run_tile_lsu(p, pi.desc, pi.tile, ctid, cnth);
         }
@@ -1138,9 +1303,30 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
             smem_set = smem;
         }
         const int threads = std::max(64, p->opts.threads);
-        hccl_executor_bulk<<<blocks, threads, smem, (cudaStream_t)stream>>>(prm, ns);
+        hccl_executor_bulk<<<blocks, threads, smem, (cudaStream_t)stream>>>(prm, ns, (uint32_t)(p->opts.copy_by_warps != 0));
     } else {
-        hccl_executor_lsu<<<blocks, p->opts.threads, 0, (cudaStream_t)stream>>>(prm);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks);
+        cfg.blockDim = dim3((unsigned)p->opts.threads);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = (cudaStream_t)stream;
+        cudaLaunchAttribute attr[1];
+        int nattr = 0;
+        if (p->opts.cluster > 1 && blocks % p->opts.cluster == 0) {
+            // blocks of one cluster are placed on SMs of one GPC next to each other: a budget of B blocks then
+            // takes B / cluster neighbourhoods away from a concurrent kernel instead of B scattered SMs
+            attr[nattr].id = cudaLaunchAttributeClusterDimension;
+            attr[nattr].val.clusterDim.x = (unsigned)p->opts.cluster;
+            attr[nattr].val.clusterDim.y = 1;
+            attr[nattr].val.clusterDim.z = 1;
+            ++nattr;
+        }
+        cfg.attrs = attr;
+        cfg.numAttrs = (unsigned)nattr;
+        if (p->opts.light)
+            CUDA_TRY(cudaLaunchKernelEx(&cfg, hccl_executor_lsu_light, prm));
+        else
+            CUDA_TRY(cudaLaunchKernelEx(&cfg, hccl_executor_lsu, prm));
     }
     CUDA_TRY(cudaGetLastError());
     p->epoch = epoch;

@@ -79,8 +79,8 @@ void hccl::fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in) {
     if (o->chunk_bytes == 0) o->chunk_bytes = 2u << 20;
     if (o->timeout_ns == 0) o->timeout_ns = 2000000000ull;
     if (o->chain_group <= 0) o->chain_group = 8;
-    if (o->threads <= 0) o->threads = 512;
-    o->threads = std::min(512, std::max(32, (o->threads + 31) / 32 * 32));
+    if (o->threads <= 0) o->threads = o->engine == HCCL_ENGINE_BULK ? 288 : 512;  // bulk: DMA warp + 8 compute warps; register: control warp + 15 workers
+    o->threads = std::min(512, std::max(64, (o->threads + 31) / 32 * 32));  // one control warp + at least one worker warp
 }
 
 extern "C" {
@@ -319,7 +319,14 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
             ntiles[i] = 1;  // a dependency-only work item
             continue;
         }
-        int64_t tc = w.tile_count > 0 ? w.tile_count : (int64_t)(tile_bytes / (uint64_t)widest(w));
+        int64_t tc = w.tile_count;
+        if (tc <= 0) {
+            // default: tile_bytes of the widest operand (multi-input sums: four times that, spread over the
+            // sources), rounded to whole passes of the block's threads unless the caller fixed tile_bytes
+            const int64_t target = w.op == HCCL_OP_REDUCE_N ? (int64_t)(4 * tile_bytes / (uint64_t)(widest(w) * std::max<int>(w.nsrc, 1)))
+                                                             : (int64_t)(tile_bytes / (uint64_t)widest(w));
+            tc = opts_in && opts_in->tile_bytes ? std::max<int64_t>(target, 1) : round_tile(target, sweep_of(p->opts, w.op));
+        }
         tc = std::min<int64_t>(std::max<int64_t>(tc, 1), 0x7fffffff);
         tcount[i] = tc;
         ntiles[i] = (w.count + tc - 1) / tc;
@@ -363,7 +370,7 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         d.op = (uint8_t)((is_data_op(w.op) && w.count == 0) ? HCCL_OP_NOOP : w.op);
         d.dt_dst = (uint8_t)w.dtype_dst; d.dt_a = (uint8_t)w.dtype_a; d.dt_b = (uint8_t)w.dtype_b;
         d.kind_dst = (uint8_t)w.dst.kind; d.kind_a = (uint8_t)w.a.kind; d.kind_b = (uint8_t)w.b.kind;
-        d.cmp = (uint8_t)w.cmp;
+        d.cmp = (uint8_t)((w.op == HCCL_OP_WAIT) ? w.cmp : w.hints);  // data ops carry their cache hints here
         d.rank_dst = (uint16_t)w.dst.rank; d.rank_a = (uint16_t)w.a.rank; d.rank_b = (uint16_t)w.b.rank;
         d.nsrc = (uint16_t)w.nsrc;
         d.off_dst = w.dst.offset; d.off_a = w.a.offset; d.off_b = w.b.offset;

@@ -1,5 +1,6 @@
 // Host-side objects behind the opaque handles of hccl.h.
 #pragma once
+#include <algorithm>
 #include <cstdint>
 #include <string>
 #include <vector>
@@ -68,6 +69,23 @@ struct hccl_plan {
 };
 
 namespace hccl {
+// Elements (bytes for COPY) that one pass of all data-moving threads of a block covers, per operation.
+// Tiles that are whole multiples of it leave no partly idle pass at the end of a tile.
+inline int64_t sweep_of(const hccl_opts_t& o, int op) {
+    if (o.engine == HCCL_ENGINE_BULK) {
+        if (op == HCCL_OP_COPY) return 32768;                 // one stage
+        if (op == HCCL_OP_REDUCE) return 4096;                // one piece
+        return (int64_t)(o.threads - 32) * 8;                 // multi-input sums run on the compute warps
+    }
+    const int64_t workers = o.threads - 32;
+    if (op == HCCL_OP_COPY) return workers * 128;             // 8 x 16 bytes per thread
+    if (op == HCCL_OP_REDUCE) return workers * 32;            // 4 x 8 elements per thread
+    return workers * 8;                                       // REDUCE_N: 8 elements per thread
+}
+inline int64_t round_tile(int64_t target, int64_t sweep) {
+    if (target >= sweep) return target / sweep * sweep;
+    return std::max<int64_t>(64, (target + 63) / 64 * 64);
+}
 hccl_status_t compile_graph(const hccl_graph* g, const hccl_opts_t* opts, hccl_plan** out);
 void fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in);
 }  // namespace hccl

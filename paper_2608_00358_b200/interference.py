@@ -65,7 +65,7 @@ def gemm_alone(gemm: Gemm, seconds: float = 3.0, discard: float = 1.0, batch: in
     return dict(tflops=float(tf), batches=int(len(tk) - 1), seconds=float((tk[-1] - tk[0]) * 1e-3))
 
 
-def overlap(gemm: Gemm, wl: wk.Workload, seconds: float = 3.0, discard: float = 1.0, gemm_batch: int = 10) -> dict:
+def overlap(gemm: Gemm, wl: Optional[wk.Workload], seconds: float = 3.0, discard: float = 1.0, gemm_batch: int = 10) -> dict:
     """GEMM loop on one stream, collective loop on a high-priority stream; rates are computed only inside
     the window in which events show both loops running."""
     sg = torch.cuda.Stream()
@@ -94,7 +94,7 @@ def overlap(gemm: Gemm, wl: wk.Workload, seconds: float = 3.0, discard: float = 
                 e.record(sg)
                 eg.append(e)
             busy = False
-        if len(ec) - done_c < depth:
+        if wl is not None and len(ec) - done_c < depth:
             wl.dc.execute(sc)
             e = torch.cuda.Event(enable_timing=True)
             e.record(sc)
@@ -103,8 +103,12 @@ def overlap(gemm: Gemm, wl: wk.Workload, seconds: float = 3.0, discard: float = 
         if busy:
             time.sleep(0.0002)
     torch.cuda.synchronize()
-    wl.dc.check()
     tg = np.array([base.elapsed_time(e) for e in eg])
+    if wl is None:      # same enqueue loop with no collective: the GEMM-alone figure, measured the same way
+        kg = tg[tg >= discard * 1e3]
+        return dict(window_s=float((kg[-1] - kg[0]) * 1e-3), gemm_batches=int(len(kg) - 1),
+                    gemm_tflops=float(gemm.flops * gemm_batch * (len(kg) - 1) / ((kg[-1] - kg[0]) * 1e-3) / 1e12))
+    wl.dc.check()
     tc = np.array([base.elapsed_time(e) for e in ec])
     lo = max(discard * 1e3, min(tg[0], tc[0]))
     hi = min(tg[-1], tc[-1])
@@ -122,7 +126,8 @@ def overlap(gemm: Gemm, wl: wk.Workload, seconds: float = 3.0, discard: float = 
 
 def measure(wl: wk.Workload, seconds: float = 3.0, gemm: Optional[Gemm] = None) -> dict:
     gemm = gemm or Gemm()
-    alone = gemm_alone(gemm, seconds)
+    alone = overlap(gemm, None, seconds)      # identical loop, no collective
+    alone = dict(tflops=alone["gemm_tflops"])
     coll_alone_ms = wk.time_back_to_back(wl, 5, 2)
     both = overlap(gemm, wl, seconds)
     res = dict(gemm_alone_tflops=alone["tflops"], collective_alone_ms=float(coll_alone_ms),
@@ -139,14 +144,18 @@ def main():
     ap.add_argument("--cap", type=int, default=32768)
     ap.add_argument("--seconds", type=float, default=3.0)
     ap.add_argument("--engine", type=int, default=0)
+    ap.add_argument("--opts", default="", help="extra plan options, e.g. threads=256,light=1,cluster=2")
     args = ap.parse_args()
+    extra = {k: int(v) for k, v in (kv.split("=") for kv in args.opts.split(",") if kv)}
     gemm = Gemm()
     base = wk.config4(dict(sm_budget=148, engine=args.engine), cap=args.cap)
     for b in [int(x) for x in args.budgets.split(",")]:
         plan = wk.hb.hccl_plan_alltoallv(base.meta["R"], base.meta["counts"], None, None, None, wk.hb.FP16,
-                                         base.meta["row_elems"], dict(sm_budget=b, engine=args.engine))
+                                         base.meta["row_elems"], dict(sm_budget=b, engine=args.engine, **extra))
         wl = wk._bind(base.name, plan, base.send, base.recv, base.meta)
-        print(json.dumps(measure(wl, args.seconds, gemm)), flush=True)
+        res = measure(wl, args.seconds, gemm)
+        res["opts"] = extra
+        print(json.dumps(res), flush=True)
 
 
 if __name__ == "__main__":

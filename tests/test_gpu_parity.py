@@ -10,16 +10,17 @@ from paper_2608_00358_b200 import synth
 
 pytestmark = pytest.mark.gpu
 DTYPES = [hb.FP32, hb.BF16, hb.FP16]
-ENGINES = [hb.ENGINE_LSU, hb.ENGINE_BULK]
+ENGINES = {"lsu": dict(engine=hb.ENGINE_LSU), "lsu_light": dict(engine=hb.ENGINE_LSU, light=1, threads=256),
+           "bulk": dict(engine=hb.ENGINE_BULK), "bulk_warpstore": dict(engine=hb.ENGINE_BULK, copy_by_warps=1, threads=288)}
 
 
-@pytest.fixture(params=ENGINES, ids=["lsu", "bulk"])
+@pytest.fixture(params=sorted(ENGINES), ids=sorted(ENGINES))
 def engine(request):
-    return request.param
+    return ENGINES[request.param]
 
 
 def _with(opts, engine):
-    return dict(opts or {}, engine=engine)
+    return dict(opts or {}, **engine)
 
 
 def _check_allreduce(R, n, dt, algo, opts, X=None, iters=1, misalign=0):
