@@ -188,6 +188,21 @@ def side_configs(quick: bool):
     return out
 
 
+def run_profile_case(args):
+    """A small, single-kernel case for ncu captures (few launches, a few hundred MB on the device):
+    config 3's shape at 1/8 of its size (R = 16, 8 Mi bf16 per rank, 2 MiB granules)."""
+    import torch
+    from paper_2608_00358_b200 import binding as hb
+    from paper_2608_00358_b200 import workloads as wk
+    algo = {"c3ring": hb.ALGO_RING, "c3fused": hb.ALGO_RING_FUSED}[args.profile_case]
+    wl = wk.config3(algo=algo, n=1 << 23)
+    ms = wk.time_back_to_back(wl, args.steps, max(args.warmup, 3))
+    i = wl.info
+    print(json.dumps({"case": args.profile_case, "workload": wl.name, "ms": ms, "schedule_bytes": int(i.schedule_bytes),
+                      "compulsory_bytes": int(i.compulsory_bytes), "schedule_gbs": i.schedule_bytes / ms / 1e6,
+                      "compulsory_gbs": i.compulsory_bytes / ms / 1e6, "tiles": int(i.n_tiles)}), flush=True)
+
+
 def run_ours(args, rank: int, world: int, local_rank: int):
     import numpy as np
     import torch
@@ -292,7 +307,21 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     # ---- interference, other configs, CPU baseline: rank 0 at N = 1 only
     if rank == 0 and world == 1:
         if not args.no_gemm:
-            line["interference"] = interference.measure(wl, seconds=2.0 if args.quick else 3.0)
+            # the GEMM-interference trade-off at a few SM budgets (the full sweep is `python -m
+            # paper_2608_00358_b200.interference`); a budget is a number of thread blocks = SMs taken
+            gemm = interference.Gemm()
+            sweep = []
+            for b in ([8, 148] if args.quick else [4, 16, 64, 148]):
+                plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(sm_budget=b))
+                w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
+                r = interference.measure(w2, seconds=2.0, gemm=gemm)
+                sweep.append({"sm_budget": b, "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
+                              "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_alone_gbs": r["collective_alone_gbs"],
+                              "collective_overlap_gbs": r["overlap"].get("collective_gbs")})
+                del w2, plan
+            line["interference"] = {"gemm": "bf16 8192^3 (cuBLAS via torch.matmul), back to back", "collective": wl.name,
+                                    "protocol": "both loops kept 3 batches deep; rates taken inside the window where both run", "sweep": sweep}
+            del gemm
         del wl
         torch.cuda.empty_cache()
         if not args.no_side:
@@ -327,12 +356,17 @@ def main():
     ap.add_argument("--no-gemm", action="store_true")
     ap.add_argument("--no-side", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--profile-case", default="", choices=["", "c3ring", "c3fused"],
+                    help="run only a small single-kernel case (for ncu captures), not the benchmark")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.profile_case:
+        run_profile_case(args)
         return
     run_ours(args, rank, world, local_rank)
 

@@ -1,0 +1,104 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times (default options).
+
+Config 4 (51.6 GB resident) is checked on sampled (source, destination) segments that the oracle computes
+one by one, plus properties that hold at any size; config 3 (2 GiB of input) is small enough for the oracle
+to compute every output. Needs a GPU with ~60 GB free and ~8 GB of host memory."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as orc
+from paper_2608_00358_b200 import binding as hb
+from paper_2608_00358_b200 import synth
+from paper_2608_00358_b200 import workloads as wk
+
+pytestmark = pytest.mark.gpu
+
+
+def _free_gb():
+    free, _ = torch.cuda.mem_get_info()
+    return free / 2 ** 30
+
+
+def test_config4_full_size_sampled_segments_and_conservation():
+    if _free_gb() < 60:
+        pytest.skip("needs 60 GB of free device memory")
+    wl = wk.config4()                       # the plan bench.py times: default engine, budget and tiles
+    C, row = wl.meta["counts"], wl.meta["row_elems"]
+    R, rb = C.shape[0], row * 2
+    assert int(C.sum()) == 50396926 and wl.meta["payload_bytes"] == 25803226112
+    for _ in range(2):                      # a cached plan is re-executed without any reset
+        wl.dc.execute()
+    wl.dc.check()
+    SD, RD = orc.packed_displs(C)
+    # --- sampled segments: largest, smallest, and random ones; the oracle runs the same problem with every
+    #     other count set to zero and the true displacements
+    rng = np.random.default_rng(5)
+    pairs = {(int(s), int(d)) for s, d in zip(*np.where(C == C.max()))}
+    pairs = set(list(pairs)[:3]) | set(list({(int(s), int(d)) for s, d in zip(*np.where(C == 1))})[:5])
+    while len(pairs) < 24:
+        pairs.add((int(rng.integers(R)), int(rng.integers(R))))
+    Cs = np.zeros_like(C)
+    for s, d in pairs:
+        Cs[s, d] = C[s, d]
+    X = [np.empty(int(C[s].sum()) * rb, dtype=np.uint8) for s in range(R)]      # virtual: only sampled rows are touched
+    for s, d in pairs:
+        lo = int(SD[s, d])
+        X[s][lo * rb:(lo + int(C[s, d])) * rb] = synth.hashed_rows_np(s, lo, int(C[s, d]), row).reshape(-1).view(np.uint8)
+    Y = [np.empty(int(C[:, d].sum()) * rb, dtype=np.uint8) for d in range(R)]
+    orc.alltoallv(X, Y, Cs, SD, RD, rb)
+    for s, d in sorted(pairs):
+        lo, n = int(RD[d, s]) * rb, int(C[s, d]) * rb
+        got = wl.recv[d].view(torch.uint8)[lo:lo + n].cpu().numpy()
+        assert np.array_equal(got, Y[d][lo:lo + n]), "segment %d -> %d" % (s, d)
+    # --- properties at full size: every receive buffer is exactly full (packed), and for every destination
+    #     the sum of all received 16-bit words equals the sum of the words sent to it
+    for d in range(R):
+        assert wl.recv[d].numel() == int(C[:, d].sum()) * row
+    sd_t = torch.from_numpy(SD)
+    for d in range(0, R, 7):
+        want = 0
+        for s in range(R):
+            lo = int(sd_t[s, d]) * row
+            want += int(wl.send[s][lo:lo + int(C[s, d]) * row].to(torch.int64).sum())
+        assert int(wl.recv[d].to(torch.int64).sum()) == want, "destination %d" % d
+    del X, Y
+
+
+def test_config3_full_size_every_output():
+    if _free_gb() < 8:
+        pytest.skip("needs 8 GB of free device memory")
+    R, n = 16, 1 << 26
+    for algo in (hb.ALGO_RING, hb.ALGO_RING_FUSED):
+        wl = wk.config3(algo=algo)
+        for _ in range(2):
+            wl.dc.execute()
+        wl.dc.check()
+        if algo == hb.ALGO_RING:
+            X = [t.view(torch.int16).cpu().numpy().view(np.uint16) for t in wl.send]
+            rc = np.full(R, n // R)
+            want = orc.reducescatter(hb.BF16, X, rc)                 # FP64 definition, rounded once
+            bitwise = orc.reducescatter_ring_f32(hb.BF16, X, rc)     # the ring's FP32 adds in ring order
+        # (1) identical bits to the ring's own arithmetic (FP32 adds in ring order, one rounding)
+        # (2) against the FP64 definition: within 1 ulp, except where cancellation makes the FP32 accumulation
+        #     error itself larger than the result's bf16 ulp; there the bound of FP32 recursive summation must
+        #     hold: |g - o| <= ulp_bf16(g)/2 + (R-1) * 2^-24 * sum_q |x_q|
+        beyond = 0
+        for r in range(R):
+            got = wl.recv[r].view(torch.int16).cpu().numpy().view(np.uint16)
+            assert np.array_equal(got, bitwise[r]), "rank %d differs from the ring-ordered FP32 sums" % r
+            idx = np.nonzero(orc.ulp_distance(hb.BF16, got, want[r]) > 1)[0]
+            beyond += idx.size
+            if idx.size:
+                cols = idx + r * (n // R)
+                xs = np.stack([synth.from_bits(x[cols], hb.BF16) for x in X])
+                o = xs.sum(axis=0)
+                g = synth.from_bits(got[idx], hb.BF16)
+                half_ulp = np.maximum(np.abs(g), 2.0 ** -126) * 2.0 ** -8
+                bound = half_ulp + (R - 1) * 2.0 ** -24 * np.abs(xs).sum(axis=0)
+                assert np.all(np.abs(g - o) <= bound), "rank %d: outside the FP32 summation bound" % r
+        assert beyond <= 1e-3 * n, beyond
+        print("config 3 (%s): %d of %d outputs beyond 1 ulp of the FP64 sum, all within the FP32 summation bound"
+              % ("ring" if algo == hb.ALGO_RING else "ring fused", beyond, n))
+        del wl
+        torch.cuda.empty_cache()
