@@ -90,7 +90,7 @@ typedef struct {
     uint64_t tile_bytes;    /* work-item size, bytes of the widest operand (default: chosen from size and sm_budget) */
     uint64_t timeout_ns;    /* bound on every device-side wait (default 2e9) */
     uint32_t flags;         /* HCCL_FLAG_* */
-    int32_t chain_group;    /* chains scheduled together in chain-group-major order (default 8) */
+    int32_t chain_group;    /* chains scheduled together in chain-group-major order (default 16) */
     int32_t threads;        /* threads per block, multiple of 32 (default 512) */
     int32_t stages;         /* bulk engine: shared-memory stages of 32 KiB per block, 2..8 (default 6) */
     int32_t cluster;        /* register engine: launch blocks in clusters of this size (2, 4, 8) so that they sit on
@@ -145,6 +145,23 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
 hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_t* sdispls,
                                   const int64_t* recvcounts, const int64_t* rdispls, hccl_dtype_t dt,
                                   int64_t row_elems, const hccl_opts_t* opts, hccl_plan_t** out);
+
+/* Device-resident AllToAllv ("AllToAllvDynamic", Sec. IV-B.2): for exchanges whose per-peer sizes are
+ * produced on the device (a routing kernel) and must not travel through the host. The plan fixes only
+ * R, the row size and the CAPACITY of every buffer in rows (max_send_rows[s] for X_s, max_recv_rows[d] for
+ * Y_d); R <= 64. Before hccl_execute, hccl_plan_set_dynamic_metadata names the DEVICE array of R*R int64
+ * counts (counts[s*R+d] rows from s to d) that the kernel reads when it runs, and optionally two DEVICE
+ * arrays [d*R+s] that receive each destination's counts and displacements for the consumer of the result.
+ * Layout is packed on both sides (exclusive prefix sums, computed in the kernel with warp scans). The
+ * counts may change between executions of the same bound plan; combined with hccl_plan_set_trigger the
+ * collective can be enqueued before the counts exist and is released by the producer's signal
+ * (Sec. IV-B.3). If a count is negative, a source's rows exceed max_send_rows or a destination's rows
+ * exceed max_recv_rows, nothing is written and hccl_plan_status reports HCCL_ERR_BAD_DESCRIPTOR. */
+hccl_status_t hccl_plan_alltoallv_dynamic(int R, const int64_t* max_send_rows, const int64_t* max_recv_rows,
+                                          hccl_dtype_t dt, int64_t row_elems, const hccl_opts_t* opts,
+                                          hccl_plan_t** out);
+hccl_status_t hccl_plan_set_dynamic_metadata(hccl_plan_t*, const int64_t* dev_sendcounts,
+                                             int64_t* dev_recvcounts_out, int64_t* dev_rdispls_out);
 
 /* ------------------------------------------------------------------------
  * Work-packet builder: the paper's own vocabulary (Sec. III-B.2). A work packet is a set of
@@ -306,6 +323,11 @@ typedef struct {
     int64_t epoch;            /* executions enqueued since the last bind */
 } hccl_plan_info_t;
 hccl_status_t hccl_plan_info(const hccl_plan_t*, hccl_plan_info_t* out);
+
+/* Byte offsets of the regions inside a bound workspace, in this order: control block, dependency counters,
+ * signal slots, descriptors (64 B each), tiles (32 B each), wait lists (8 B per entry), FP32 scratch, total.
+ * For tools that inspect a workspace, and for tests that damage a table on purpose. */
+hccl_status_t hccl_plan_layout(const hccl_plan_t*, int64_t offsets[8]);
 
 /* Declared extent, in bytes, of rank r's send / receive buffer. */
 hccl_status_t hccl_plan_extents(const hccl_plan_t*, int rank, int64_t* send_bytes, int64_t* recv_bytes);

@@ -73,6 +73,8 @@ def _load() -> C.CDLL:
         "hccl_plan_reducescatter": [C.c_int, I64P, C.c_int64, C.c_int, C.c_int, C.POINTER(Opts), C.POINTER(P)],
         "hccl_plan_allgather": [C.c_int, I64P, C.c_int64, C.c_int, C.c_int, C.POINTER(Opts), C.POINTER(P)],
         "hccl_plan_alltoallv": [C.c_int, I64P, I64P, I64P, I64P, C.c_int, C.c_int64, C.POINTER(Opts), C.POINTER(P)],
+        "hccl_plan_alltoallv_dynamic": [C.c_int, I64P, I64P, C.c_int, C.c_int64, C.POINTER(Opts), C.POINTER(P)],
+        "hccl_plan_set_dynamic_metadata": [P, P, P, P],
         "hccl_graph_create": [C.c_int, I64P, I64P, C.c_int64, C.c_int32, C.POINTER(P)],
         "hccl_graph_add_subgraph": [P, C.c_int, C.POINTER(C.c_int32)],
         "hccl_graph_add_wqe": [P, C.c_int32, C.POINTER(Wqe), I64P],
@@ -87,6 +89,7 @@ def _load() -> C.CDLL:
         "hccl_plan_status": [P, C.POINTER(C.c_int), I64P],
         "hccl_plan_info": [P, C.POINTER(PlanInfo)],
         "hccl_plan_extents": [P, C.c_int, I64P, I64P],
+        "hccl_plan_layout": [P, I64P],
         "hccl_plan_check_hazards": [P, I64P],
         "hccl_plan_interpret_host": [P, C.POINTER(P), C.POINTER(P), P, C.POINTER(C.c_uint64), C.c_uint64],
     }
@@ -110,11 +113,12 @@ def _load() -> C.CDLL:
 _lib = _load()
 LIBRARY_PATH = _build.LIB
 EXPORTS = ["hccl_plan_allreduce", "hccl_plan_reducescatter", "hccl_plan_allgather", "hccl_plan_alltoallv",
+           "hccl_plan_alltoallv_dynamic", "hccl_plan_set_dynamic_metadata",
            "hccl_graph_create", "hccl_graph_add_subgraph", "hccl_graph_add_wqe", "hccl_graph_compile",
            "hccl_graph_destroy", "hccl_plan_workspace_bytes", "hccl_plan_bind", "hccl_execute", "hccl_execute_host",
            "hccl_execute_noalloc",
            "hccl_plan_set_user_signals", "hccl_plan_set_trigger", "hccl_plan_status", "hccl_plan_info",
-           "hccl_plan_extents", "hccl_plan_destroy", "hccl_status_string", "hccl_last_cuda_error", "hccl_version",
+           "hccl_plan_extents", "hccl_plan_layout", "hccl_plan_destroy", "hccl_status_string", "hccl_last_cuda_error", "hccl_version",
            "hccl_plan_check_hazards", "hccl_plan_interpret_host"]
 
 
@@ -178,6 +182,11 @@ class Plan:
         _chk(_lib.hccl_plan_extents(self._h, rank, C.byref(s), C.byref(r)), "hccl_plan_extents")
         return s.value, r.value
 
+    def layout(self) -> dict:
+        o = (C.c_int64 * 8)()
+        _chk(_lib.hccl_plan_layout(self._h, o), "hccl_plan_layout")
+        return dict(zip(["control", "counters", "signals", "descs", "tiles", "waits", "scratch", "total"], list(o)))
+
     def bind(self, dev_workspace: int, nbytes: int, stream: int = 0):
         _chk(_lib.hccl_plan_bind(self._h, C.c_void_p(dev_workspace), nbytes, C.c_void_p(stream)), "hccl_plan_bind")
 
@@ -197,6 +206,10 @@ class Plan:
         allocate device memory). Raises HcclError with the device-side verdict if it failed."""
         _chk(_lib.hccl_execute_noalloc(self._h, _ptr_array(sendbufs), _ptr_array(recvbufs), C.c_void_p(stream)),
              "hccl_execute_noalloc")
+
+    def set_dynamic_metadata(self, dev_sendcounts: int, dev_recvcounts_out: int = 0, dev_rdispls_out: int = 0):
+        _chk(_lib.hccl_plan_set_dynamic_metadata(self._h, C.c_void_p(dev_sendcounts), C.c_void_p(dev_recvcounts_out or None),
+                                                 C.c_void_p(dev_rdispls_out or None)), "hccl_plan_set_dynamic_metadata")
 
     def set_user_signals(self, dev_signals: int, n_slots: int):
         _chk(_lib.hccl_plan_set_user_signals(self._h, C.c_void_p(dev_signals), n_slots), "hccl_plan_set_user_signals")
@@ -252,6 +265,12 @@ def hccl_plan_alltoallv(R: int, sendcounts, sdispls=None, recvcounts=None, rdisp
     return _new_plan(_lib.hccl_plan_alltoallv(R, _i64(sendcounts), _i64(sdispls), _i64(recvcounts), _i64(rdispls), dt,
                                               row_elems, C.byref(make_opts(opts)), C.byref(h)), h,
                      "hccl_plan_alltoallv")
+
+
+def hccl_plan_alltoallv_dynamic(R: int, max_send_rows, max_recv_rows, dt: int = BF16, row_elems: int = 1, opts=None) -> Plan:
+    h = C.c_void_p()
+    return _new_plan(_lib.hccl_plan_alltoallv_dynamic(R, _i64(max_send_rows), _i64(max_recv_rows), dt, row_elems,
+                                                      C.byref(make_opts(opts)), C.byref(h)), h, "hccl_plan_alltoallv_dynamic")
 
 
 class Graph:

@@ -442,4 +442,46 @@ hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_
     return hccl_graph_compile(g.get(), &o, out);
 }
 
+hccl_status_t hccl_plan_alltoallv_dynamic(int R, const int64_t* max_send_rows, const int64_t* max_recv_rows, hccl_dtype_t dt,
+                                          int64_t row_elems, const hccl_opts_t* opts, hccl_plan_t** out) {
+    if (!out || !max_send_rows || !max_recv_rows || R < 1 || R > 64 || row_elems < 1) return HCCL_ERR_INVALID_ARG;
+    if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
+    const int64_t row_bytes = row_elems * elem_bytes(dt);
+    std::vector<int64_t> sext(R), rext(R);
+    for (int r = 0; r < R; ++r) {
+        if (max_send_rows[r] < 0 || max_recv_rows[r] < 0) return HCCL_ERR_INVALID_ARG;
+        if (max_send_rows[r] > (INT64_MAX / 4) / row_bytes || max_recv_rows[r] > (INT64_MAX / 4) / row_bytes) return HCCL_ERR_INVALID_ARG;
+        sext[r] = max_send_rows[r] * row_bytes;
+        rext[r] = max_recv_rows[r] * row_bytes;
+    }
+    hccl_opts_t o;
+    if (opts) o = *opts; else std::memset(&o, 0, sizeof(o));
+    o.engine = HCCL_ENGINE_LSU;  // the device-resident kernel moves bytes through registers
+    hccl_graph* graw = nullptr;
+    CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw));
+    GraphPtr g(graw);
+    g->compulsory_bytes = 0;  // not known before the counts exist
+    hccl_plan* p = nullptr;
+    CHECK(hccl_graph_compile(g.get(), &o, &p));
+    p->dynamic = true;
+    p->dyn_row_bytes = row_bytes;
+    p->dyn_max_send_rows.assign(max_send_rows, max_send_rows + R);
+    p->dyn_max_recv_rows.assign(max_recv_rows, max_recv_rows + R);
+    if (!opts || opts->tile_bytes == 0) p->opts.tile_bytes = (uint64_t)p->opts.threads * 128;  // one pass of all threads
+    p->opts.tile_bytes = std::max<uint64_t>(p->opts.tile_bytes, 512);
+    p->info.tile_bytes = (int64_t)p->opts.tile_bytes;
+    *out = p;
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_plan_set_dynamic_metadata(hccl_plan_t* p, const int64_t* dev_sendcounts, int64_t* dev_recvcounts_out,
+                                             int64_t* dev_rdispls_out) {
+    if (!p || !p->dynamic || !dev_sendcounts) return HCCL_ERR_INVALID_ARG;
+    if (((uintptr_t)dev_sendcounts | (uintptr_t)dev_recvcounts_out | (uintptr_t)dev_rdispls_out) % 8) return HCCL_ERR_ALIGNMENT;
+    p->dyn_counts = dev_sendcounts;
+    p->dyn_recvcounts_out = dev_recvcounts_out;
+    p->dyn_rdispls_out = dev_rdispls_out;
+    return HCCL_OK;
+}
+
 }  // extern "C"

@@ -85,7 +85,8 @@ __device__ __forceinline__ bool compare(unsigned long long v, int cmp, unsigned 
 }
 
 // Record a failure once per execution and tell everyone to stop.
-__device__ __noinline__ void fail(const ExecParams& p, uint32_t code, unsigned long long detail) {
+template <class P>
+__device__ __noinline__ void fail(const P& p, uint32_t code, unsigned long long detail) {
     if (atomicExch(&p.ctl->fail_epoch, p.epoch) != p.epoch) {  // first failure of this execution wins
         p.ctl->status = code;
         p.ctl->detail = detail;
@@ -93,7 +94,8 @@ __device__ __noinline__ void fail(const ExecParams& p, uint32_t code, unsigned l
     __threadfence();
     atomicExch(&p.ctl->abort, p.epoch);
 }
-__device__ __forceinline__ bool aborted(const ExecParams& p) { return ld_relaxed_u32(&p.ctl->abort) == p.epoch; }
+template <class P>
+__device__ __forceinline__ bool aborted(const P& p) { return ld_relaxed_u32(&p.ctl->abort) == p.epoch; }
 
 // Bounded wait until counters[sync] has received epoch * per_epoch bumps (wrap-safe compare).
 __device__ bool wait_counter(const ExecParams& p, uint32_t sync, uint32_t per_epoch, uint32_t tile) {
@@ -115,7 +117,8 @@ __device__ bool wait_counter(const ExecParams& p, uint32_t sync, uint32_t per_ep
     }
 }
 
-__device__ bool wait_signal(const ExecParams& p, const unsigned long long* addr, int cmp, unsigned long long want, uint32_t tile) {
+template <class P>
+__device__ bool wait_signal(const P& p, const unsigned long long* addr, int cmp, unsigned long long want, uint32_t tile) {
     if (compare(ld_acquire_u64(addr), cmp, want)) return true;
     const unsigned long long deadline = globaltimer_ns() + p.timeout_ns;
     uint32_t spins = 0;
@@ -542,7 +545,8 @@ __device__ __forceinline__ void publish_tile(const ExecParams& p, const Tile& t)
 }
 
 // Last block out: completion value for a device-triggered caller, epoch stamp, clean ticket.
-__device__ void leave(const ExecParams& p) {
+template <class P>
+__device__ void leave(const P& p) {
     __threadfence();
     const uint32_t prev = atomicAdd(&p.ctl->exits, 1);
     if (prev == p.nblocks - 1) {
@@ -1186,6 +1190,170 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
     }
 }
 
+
+// ====================================================================== device-resident AllToAllv
+// "AllToAllvDynamic" (paper Sec. IV-B.2): the per-peer row counts are produced on the device (by a routing
+// kernel) after the collective has been compiled and possibly already enqueued. The kernel reads the R x R
+// count matrix from device memory, derives packed send and receive displacements with warp-level prefix
+// sums, cuts every (source, destination) segment into equal-byte tiles, and moves them. Nothing about the
+// sizes goes through the host. Every count is validated against the capacities fixed at plan time before a
+// single byte is written.
+constexpr int DYN_MAX_RANKS = 64;
+
+struct DynParams {
+    const long long* counts;       // device, [R*R], counts[s*R+d] rows from s to d
+    long long* recvcounts_out;     // device, [R*R] indexed [d*R+s], or null
+    long long* rdispls_out;        // device, [R*R] indexed [d*R+s], or null
+    Control* ctl;
+    unsigned long long* user_signals;
+    uint32_t epoch, R, nblocks, pad0;
+    unsigned long long timeout_ns;
+    unsigned long long row_bytes, tile_bytes;
+    long long trig_wait_slot, trig_set_slot;
+    int trig_cmp, pad1;
+    unsigned long long trig_wait_value, trig_set_value;
+    long long max_send_rows[DYN_MAX_RANKS], max_recv_rows[DYN_MAX_RANKS];
+    const void* send[DYN_MAX_RANKS];
+    void* recv[DYN_MAX_RANKS];
+};
+
+__device__ __forceinline__ long long warp_inclusive_scan(long long v, uint32_t lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= (uint32_t)o) v += u;
+    }
+    return v;
+}
+
+__global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant__ DynParams q) {
+    extern __shared__ __align__(16) unsigned char dsm[];
+    const uint32_t R = q.R, RR = R * R;
+    long long* s_cnt = reinterpret_cast<long long*>(dsm);  // [RR] rows of segment (s,d)
+    long long* s_sd = s_cnt + RR;                          // [RR] first row of the segment in X_s
+    long long* s_rd = s_sd + RR;                           // [RR] first row of the segment in Y_d
+    uint32_t* s_tp = reinterpret_cast<uint32_t*>(s_rd + RR);  // [RR+1] exclusive prefix of tiles per segment
+    __shared__ int s_bad;
+    __shared__ unsigned long long s_bad_at;
+    __shared__ uint32_t s_ticket;
+    __shared__ int s_live;
+    const uint32_t tid = threadIdx.x, nth = blockDim.x, lane = tid & 31u, warp = tid >> 5, nwarps = nth >> 5;
+    if (tid == 0) {
+        s_bad = 0;
+        s_bad_at = 0;
+        bool live = true;
+        if (q.trig_wait_slot >= 0)
+            live = wait_signal(q, q.user_signals + q.trig_wait_slot, q.trig_cmp, q.trig_wait_value, 0xffffffffu);
+        s_live = live ? 1 : 0;
+    }
+    __syncthreads();
+    if (s_live) {
+        // ---- metadata from device memory (written by the producer before it released us)
+        for (uint32_t i = tid; i < RR; i += nth) {
+            const long long c = __ldcg(q.counts + i);
+            s_cnt[i] = c;
+            if (c < 0 || c > (1ll << 40)) {
+                s_bad = 1;
+                s_bad_at = i;
+            }
+        }
+        __syncthreads();
+        if (!s_bad) {
+            // send displacements: exclusive scan of each source's row of counts; one warp per source
+            for (uint32_t s = warp; s < R; s += nwarps) {
+                long long carry = 0;
+                for (uint32_t base = 0; base < R; base += 32) {
+                    const uint32_t d = base + lane;
+                    const long long v = d < R ? s_cnt[s * R + d] : 0;
+                    const long long inc = warp_inclusive_scan(v, lane);
+                    if (d < R) s_sd[s * R + d] = carry + inc - v;
+                    carry += __shfl_sync(0xffffffffu, inc, 31);
+                }
+                if (lane == 0 && carry > q.max_send_rows[s]) {
+                    s_bad = 1;
+                    s_bad_at = (unsigned long long)s * R;
+                }
+            }
+            // receive displacements: exclusive scan down each destination's column; one warp per destination
+            for (uint32_t d = warp; d < R; d += nwarps) {
+                long long carry = 0;
+                for (uint32_t base = 0; base < R; base += 32) {
+                    const uint32_t s = base + lane;
+                    const long long v = s < R ? s_cnt[s * R + d] : 0;
+                    const long long inc = warp_inclusive_scan(v, lane);
+                    if (s < R) s_rd[s * R + d] = carry + inc - v;
+                    carry += __shfl_sync(0xffffffffu, inc, 31);
+                }
+                if (lane == 0 && carry > q.max_recv_rows[d]) {
+                    s_bad = 1;
+                    s_bad_at = d;
+                }
+            }
+            // tiles per segment and their exclusive prefix over (s,d) in row-major order; warp 0
+            if (warp == 0) {
+                long long carry = 0;
+                for (uint32_t base = 0; base < RR; base += 32) {
+                    const uint32_t i = base + lane;
+                    const long long bytes = i < RR ? s_cnt[i] * (long long)q.row_bytes : 0;
+                    const long long v = (bytes + (long long)q.tile_bytes - 1) / (long long)q.tile_bytes;
+                    const long long inc = warp_inclusive_scan(v, lane);
+                    if (i < RR) s_tp[i] = (uint32_t)(carry + inc - v);
+                    carry += __shfl_sync(0xffffffffu, inc, 31);
+                }
+                if (lane == 0) {
+                    s_tp[RR] = (uint32_t)carry;
+                    if (carry > 0x7fffffffll) {
+                        s_bad = 1;
+                        s_bad_at = RR;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (s_bad) {
+            if (tid == 0) fail(q, HCCL_ERR_BAD_DESCRIPTOR, s_bad_at);
+        } else {
+            // what each receiver gets and where, for the kernels that consume the result
+            if (blockIdx.x == 0) {
+                for (uint32_t i = tid; i < RR; i += nth) {
+                    const uint32_t s = i / R, d = i % R;
+                    if (q.recvcounts_out) q.recvcounts_out[d * R + s] = s_cnt[i];
+                    if (q.rdispls_out) q.rdispls_out[d * R + s] = s_rd[i];
+                }
+            }
+            const uint32_t total = s_tp[RR];
+            uint32_t next = 0;
+            if (tid == 0) next = atomicAdd(&q.ctl->ticket, 1);
+            for (;;) {
+                if (tid == 0) {
+                    s_ticket = next;
+                    if (next < total) next = atomicAdd(&q.ctl->ticket, 1);  // one ahead
+                }
+                __syncthreads();
+                const uint32_t t = s_ticket;
+                if (t >= total) break;
+                // segment of tile t: the last i with s_tp[i] <= t (zero-length segments share a prefix value
+                // with their successor and are skipped by taking the last one)
+                uint32_t lo = 0, hi = RR;
+                while (hi - lo > 1) {
+                    const uint32_t mid = (lo + hi) >> 1;
+                    if (s_tp[mid] <= t) lo = mid; else hi = mid;
+                }
+                const uint32_t i = lo, s = i / R, d = i % R;
+                const unsigned long long off = (unsigned long long)(t - s_tp[i]) * q.tile_bytes;
+                const unsigned long long seg = (unsigned long long)s_cnt[i] * q.row_bytes;
+                const uint32_t len = (uint32_t)min((unsigned long long)q.tile_bytes, seg - off);
+                const char* src = (const char*)q.send[s] + (unsigned long long)s_sd[i] * q.row_bytes + off;
+                char* dst = (char*)q.recv[d] + (unsigned long long)s_rd[i] * q.row_bytes + off;
+                copy_tile_lsu<true>(dst, src, len, tid, nth);
+                __syncthreads();
+            }
+        }
+    }
+    __syncthreads();
+    if (tid == 0) leave(q);
+}
+
 }  // namespace hccl
 
 // ====================================================================== host side
@@ -1261,6 +1429,44 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     hccl_status_t st = check_buffers(p, sendbufs, recvbufs);
     if (st != HCCL_OK) return st;
     if ((p->trig_wait_slot >= 0 || p->trig_set_slot >= 0) && !p->user_signals) return HCCL_ERR_INVALID_ARG;
+    if (p->dynamic) {
+        if (!p->dyn_counts) return HCCL_ERR_INVALID_ARG;
+        static thread_local DynParams q;
+        const uint32_t epoch = p->epoch + 1;
+        q.counts = (const long long*)p->dyn_counts;
+        q.recvcounts_out = (long long*)p->dyn_recvcounts_out;
+        q.rdispls_out = (long long*)p->dyn_rdispls_out;
+        q.ctl = (Control*)((char*)p->workspace + p->layout.control);
+        q.user_signals = (unsigned long long*)p->user_signals;
+        q.epoch = epoch;
+        q.R = (uint32_t)p->R;
+        q.nblocks = (uint32_t)p->opts.sm_budget;
+        q.timeout_ns = p->opts.timeout_ns;
+        q.row_bytes = (unsigned long long)p->dyn_row_bytes;
+        q.tile_bytes = p->opts.tile_bytes;
+        q.trig_wait_slot = p->trig_wait_slot;
+        q.trig_set_slot = p->trig_set_slot;
+        q.trig_cmp = p->trig_cmp;
+        q.trig_wait_value = p->trig_wait_value + (uint64_t)epoch * p->trig_wait_per_epoch;
+        q.trig_set_value = p->trig_set_value + (uint64_t)epoch * p->trig_set_per_epoch;
+        for (int r = 0; r < p->R; ++r) {
+            q.max_send_rows[r] = p->dyn_max_send_rows[r];
+            q.max_recv_rows[r] = p->dyn_max_recv_rows[r];
+            q.send[r] = sendbufs[r];
+            q.recv[r] = recvbufs[r];
+        }
+        const size_t RR = (size_t)p->R * p->R;
+        const size_t smem = RR * 24 + (RR + 1) * 4 + 16;
+        static thread_local size_t dyn_smem_set = 0;
+        if (smem > 48 * 1024 && smem > dyn_smem_set) {
+            CUDA_TRY(cudaFuncSetAttribute(hccl_a2a_dynamic, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            dyn_smem_set = smem;
+        }
+        hccl_a2a_dynamic<<<p->opts.sm_budget, p->opts.threads, smem, (cudaStream_t)stream>>>(q);
+        CUDA_TRY(cudaGetLastError());
+        p->epoch = epoch;
+        return HCCL_OK;
+    }
     static thread_local ExecParams prm;  // 4 KB+: keep it off the stack
     char* ws = (char*)p->workspace;
     const Layout& L = p->layout;
@@ -1388,7 +1594,7 @@ extern "C" hccl_status_t hccl_execute_noalloc(hccl_plan_t* p, const void* const*
                  (unsigned long long)p->layout.total, HCCL_NOALLOC_WORKSPACE_BYTES);
         return HCCL_ERR_WORKSPACE;
     }
-    if (p->trig_wait_slot >= 0 || p->trig_set_slot >= 0) return HCCL_ERR_INVALID_ARG;  // triggers belong to bound plans
+    if (p->trig_wait_slot >= 0 || p->trig_set_slot >= 0 || p->dynamic) return HCCL_ERR_INVALID_ARG;  // triggers and device-resident plans belong to bound plans
     int dev = -1;
     CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return HCCL_ERR_INVALID_ARG;

@@ -78,7 +78,7 @@ void hccl::fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in) {
     if (o->engine == 0) o->engine = HCCL_ENGINE_LSU;
     if (o->chunk_bytes == 0) o->chunk_bytes = 2u << 20;
     if (o->timeout_ns == 0) o->timeout_ns = 2000000000ull;
-    if (o->chain_group <= 0) o->chain_group = 8;
+    if (o->chain_group <= 0) o->chain_group = 16;
     if (o->threads <= 0) o->threads = o->engine == HCCL_ENGINE_BULK ? 288 : 512;  // bulk: DMA warp + 8 compute warps; register: control warp + 15 workers
     o->threads = std::min(512, std::max(64, (o->threads + 31) / 32 * 32));  // one control warp + at least one worker warp
 }
@@ -453,6 +453,14 @@ hccl_status_t hccl_plan_info(const hccl_plan_t* p, hccl_plan_info_t* out) {
     if (!p || !out) return HCCL_ERR_INVALID_ARG;
     *out = p->info;
     out->epoch = p->epoch;
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_plan_layout(const hccl_plan_t* p, int64_t offsets[8]) {
+    if (!p || !offsets) return HCCL_ERR_INVALID_ARG;
+    const Layout& L = p->layout;
+    const uint64_t v[8] = {L.control, L.counters, L.signals, L.descs, L.tiles, L.waits, L.scratch, L.total};
+    for (int i = 0; i < 8; ++i) offsets[i] = (int64_t)v[i];
     return HCCL_OK;
 }
 

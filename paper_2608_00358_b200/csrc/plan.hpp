@@ -59,6 +59,13 @@ struct hccl_plan {
     int64_t trig_wait_slot = -1, trig_set_slot = -1;
     int32_t trig_cmp = 0;
     uint64_t trig_wait_value = 0, trig_wait_per_epoch = 0, trig_set_value = 0, trig_set_per_epoch = 0;
+    // device-resident AllToAllv (Sec. IV-B.2): sizes are read from device memory when the kernel runs
+    bool dynamic = false;
+    int64_t dyn_row_bytes = 0;
+    std::vector<int64_t> dyn_max_send_rows, dyn_max_recv_rows;
+    const void* dyn_counts = nullptr;
+    void* dyn_recvcounts_out = nullptr;
+    void* dyn_rdispls_out = nullptr;
     // binding
     void* workspace = nullptr;
     size_t workspace_bytes = 0;

@@ -1,0 +1,152 @@
+"""Device-resident and device-triggered AllToAllv: counts live in device memory, may change between
+executions of one bound plan, and a producer on another stream releases a pre-launched collective."""
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2608_00358_b200 import binding as hb
+from paper_2608_00358_b200 import synth
+
+SENT = 0x5A
+
+
+def test_dynamic_plan_validation():
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_alltoallv_dynamic(65, [1] * 65, [1] * 65, hb.BF16, 8)
+    assert e.value.status == hb.ERR_INVALID_ARG
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_alltoallv_dynamic(2, [1, -1], [1, 1], hb.BF16, 8)
+    assert e.value.status == hb.ERR_INVALID_ARG
+    p = hb.hccl_plan_alltoallv_dynamic(4, [10] * 4, [12] * 4, hb.FP16, 8)
+    assert p.extents(0) == (160, 192) and p.info().n_tiles == 0
+
+
+def _setup(R, row_elems, cap_rows, dt=hb.BF16, opts=None):
+    import torch
+    from paper_2608_00358_b200.runtime import DeviceCollective
+    rb = row_elems * hb.ELEM_BYTES[dt]
+    plan = hb.hccl_plan_alltoallv_dynamic(R, [cap_rows] * R, [cap_rows] * R, dt, row_elems, opts)
+    X = [synth.hashed_rows_np(s, 0, cap_rows, row_elems).reshape(-1).view(np.uint8) for s in range(R)]
+    send = [torch.from_numpy(x.copy()).cuda() for x in X]
+    recv = [torch.full((cap_rows * rb,), SENT, dtype=torch.uint8, device="cuda") for _ in range(R)]
+    counts = torch.zeros(R * R, dtype=torch.int64, device="cuda")
+    rc_out = torch.full((R * R,), -1, dtype=torch.int64, device="cuda")
+    rd_out = torch.full((R * R,), -1, dtype=torch.int64, device="cuda")
+    plan.set_dynamic_metadata(counts.data_ptr(), rc_out.data_ptr(), rd_out.data_ptr())
+    dc = DeviceCollective(plan)
+    dc.set_buffers([t.data_ptr() for t in send], [t.data_ptr() for t in recv])
+    return plan, dc, X, send, recv, counts, rc_out, rd_out, rb
+
+
+def _expect(X, C, rb, cap_rows):
+    R = C.shape[0]
+    SD, RD = orc.packed_displs(C)
+    Y = [np.full(cap_rows * rb, SENT, dtype=np.uint8) for _ in range(R)]
+    orc.alltoallv(X, Y, C, SD, RD, rb)
+    return Y, RD
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("R,row_elems,hi", [(2, 8, 5), (8, 128, 300), (8, 7, 50), (33, 64, 40), (64, 256, 24)])
+def test_dynamic_alltoallv_counts_change_between_executions(R, row_elems, hi):
+    import torch
+    cap = hi * R + 3
+    plan, dc, X, send, recv, counts, rc_out, rd_out, rb = _setup(R, row_elems, cap, opts=dict(sm_budget=24, tile_bytes=4096))
+    for seed in (1, 2, 3):
+        C = synth.uniform_counts(R, seed, hi=hi)
+        if seed == 2:
+            C[:, R // 2] = 0                       # a destination that receives nothing
+            C[0, :] = 0                            # a source that sends nothing
+        counts.copy_(torch.from_numpy(C.reshape(-1)))    # the "routing kernel": sizes written on the device
+        for t in recv:
+            t.fill_(SENT)
+        dc.execute()
+        dc.check()
+        want, RD = _expect(X, C, rb, cap)
+        for d in range(R):
+            assert np.array_equal(recv[d].cpu().numpy(), want[d]), (seed, d)
+        assert np.array_equal(rc_out.cpu().numpy().reshape(R, R), C.T)
+        assert np.array_equal(rd_out.cpu().numpy().reshape(R, R), RD)
+
+
+@pytest.mark.gpu
+def test_dynamic_alltoallv_rejects_counts_beyond_capacity_without_writing():
+    import torch
+    R, row_elems, cap = 4, 16, 20
+    plan, dc, X, send, recv, counts, rc_out, rd_out, rb = _setup(R, row_elems, cap)
+    for bad in ("overflow_recv", "negative"):
+        C = np.full((R, R), 2, dtype=np.int64)
+        if bad == "overflow_recv":
+            C[:, 1] = 6                        # 24 rows into a 20-row receive buffer
+        else:
+            C[2, 3] = -1
+        counts.copy_(torch.from_numpy(C.reshape(-1)))
+        dc.execute()
+        torch.cuda.synchronize()
+        st, _ = plan.status()
+        assert st == hb.ERR_BAD_DESCRIPTOR
+        for t in recv:
+            assert bool((t == SENT).all())
+    # the plan works again after being bound again, and the GPU is healthy
+    from paper_2608_00358_b200.runtime import DeviceCollective
+    dc2 = DeviceCollective(plan)
+    dc2.set_buffers([t.data_ptr() for t in send], [t.data_ptr() for t in recv])
+    C = np.full((R, R), 3, dtype=np.int64)
+    counts.copy_(torch.from_numpy(C.reshape(-1)))
+    dc2.execute()
+    dc2.check()
+    want, _ = _expect(X, C, rb, cap)
+    for d in range(R):
+        assert np.array_equal(recv[d].cpu().numpy(), want[d])
+
+
+@pytest.mark.gpu
+def test_device_triggered_dynamic_alltoallv_is_released_by_the_producer():
+    """The collective is enqueued first, on its own stream, and holds at its start gate. The producer stream
+    then writes the counts and raises the signal; when the collective is done it stores the completion value."""
+    import torch
+    R, row_elems, cap = 8, 64, 400
+    plan, dc, X, send, recv, counts, rc_out, rd_out, rb = _setup(R, row_elems, cap, opts=dict(sm_budget=8))
+    signals = torch.zeros(2, dtype=torch.int64, device="cuda")
+    plan.set_user_signals(signals.data_ptr(), 2)
+    # gate: slot 0 >= epoch; completion: slot 1 = 100 + epoch
+    plan.set_trigger(wait_slot=0, cmp=hb.CMP_GE, wait_value=0, wait_per_epoch=1, set_slot=1, set_value=100, set_per_epoch=1)
+    coll, prod = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for epoch in (1, 2):
+        C = synth.uniform_counts(R, 10 + epoch, hi=40)
+        host_counts = torch.from_numpy(C.reshape(-1)).pin_memory()
+        for t in recv:
+            t.fill_(SENT)
+        torch.cuda.synchronize()
+        dc.execute(coll)                                   # pre-launched: spins (bounded) on the gate
+        with torch.cuda.stream(prod):
+            counts.copy_(host_counts, non_blocking=True)   # stands in for the routing kernel's output
+            signals[0:1].fill_(epoch)                      # the producer's release
+        torch.cuda.synchronize()
+        st, _ = plan.status()
+        assert st == hb.OK
+        assert int(signals[1]) == 100 + epoch
+        want, _ = _expect(X, C, rb, cap)
+        for d in range(R):
+            assert np.array_equal(recv[d].cpu().numpy(), want[d]), (epoch, d)
+
+
+@pytest.mark.gpu
+def test_start_gate_that_never_opens_times_out_cleanly():
+    """A wait that cannot come true ends in HCCL_ERR_TIMEOUT after the plan's bound, the kernel returns
+    normally and the device stays usable."""
+    import torch
+    R, row_elems, cap = 2, 8, 8
+    plan, dc, X, send, recv, counts, rc_out, rd_out, rb = _setup(R, row_elems, cap, opts=dict(sm_budget=2, timeout_ns=200_000_000))
+    signals = torch.zeros(1, dtype=torch.int64, device="cuda")
+    plan.set_user_signals(signals.data_ptr(), 1)
+    plan.set_trigger(wait_slot=0, cmp=hb.CMP_EQ, wait_value=12345)
+    counts.fill_(1)
+    dc.execute()
+    torch.cuda.synchronize()
+    st, _ = plan.status()
+    assert st == hb.ERR_TIMEOUT
+    for t in recv:
+        assert bool((t == SENT).all())
+    assert float(torch.ones(4, device="cuda").sum()) == 4.0
