@@ -245,11 +245,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     wl.dc.check()
     total_ms = evs[0].elapsed_time(evs[-1])
     per_launch = np.array([evs[k].elapsed_time(evs[k + 1]) for k in range(args.steps)])
-    t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t.item())
-    value = world * info.schedule_bytes * args.steps / (total_ms_max * 1e-3) / 1e9
+    from paper_2608_00358_b200 import multi
+    value, total_ms_max = multi.replica_throughput_gbs(total_ms, info.schedule_bytes, args.steps, dist, "cuda")
 
     # ---- end to end through host buffers (rank-local; reported by rank 0)
     e2e = None

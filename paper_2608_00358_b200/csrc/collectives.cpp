@@ -149,16 +149,14 @@ hccl_status_t emit_ring(hccl_graph* g, int R, int dt, const std::vector<Chain>& 
     return HCCL_OK;
 }
 
-// Tile size in elements for a schedule whose widest operand has `widest` bytes per element. With
-// opts.tile_bytes unset the size follows the total work (about 8 tiles per block, 16..256 KiB) and is
-// rounded to whole passes of the block's threads for operation `op`.
-int64_t pick_tile_elems(int64_t weight_bytes, const hccl_opts_t& o, int widest, int op) {
+// Tile size in elements for a ring schedule: `level_elems` elements are worked on by one ring step of all
+// chains that run together, and a step should be about one tile per block (a chain advances one step per
+// tile, so few, large tiles keep the dependency chain short). With opts.tile_bytes set, that many bytes
+// of the widest operand.
+int64_t pick_tile_elems(int64_t level_elems, const hccl_opts_t& o, int widest, int op) {
     if (o.tile_bytes) return std::max<int64_t>(64, (int64_t)(o.tile_bytes / (uint64_t)widest));
-    uint64_t per = (uint64_t)weight_bytes / (8ull * (uint64_t)o.sm_budget);
-    uint64_t p2 = 1;
-    while (p2 * 2 <= per) p2 *= 2;
-    const uint64_t tb = std::min<uint64_t>(256u << 10, std::max<uint64_t>(16u << 10, p2));
-    return round_tile((int64_t)(tb / (uint64_t)widest), sweep_of(o, op));
+    const int64_t lo = op == HCCL_OP_REDUCE_N ? 1 << 10 : 4 << 10, hi = op == HCCL_OP_REDUCE_N ? 32 << 10 : 64 << 10;
+    return default_tile(level_elems, o.sm_budget, 1, lo, hi, sweep_of(o, op));
 }
 
 // Copy-only schedules: with the engine left to the library, the bulk copy unit moves the bytes
@@ -244,7 +242,9 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     const int64_t slot_elems = (int64_t)align_up((uint64_t)maxlen, 64);
     const int64_t scratch = need_scratch ? (int64_t)n_slots * slot_elems * 4 * (staged ? 2 : 1) : 0;
     const int64_t weight = count * 4 * (R - 1) + (int64_t)count * es * (R - 1);
-    const int64_t tile_elems = fused ? pick_tile_elems((int64_t)count * es * R, o, es * R / 4, HCCL_OP_REDUCE_N) : pick_tile_elems(weight, o, in_recv ? es : 4, HCCL_OP_REDUCE);
+    const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
+    (void)weight;
+    const int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, in_recv ? es : 4, HCCL_OP_REDUCE);
 
     hccl_graph* graw = nullptr;
     CHECK(hccl_graph_create(R, ext.data(), ext.data(), scratch, 0, &graw));
@@ -303,7 +303,8 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     const int n_slots = need_scratch ? (int)std::min<size_t>(chains.size(), slots_wanted) : 0;
     const int64_t slot_elems = (int64_t)align_up((uint64_t)maxlen, 64);
     const int64_t scratch = need_scratch ? (int64_t)n_slots * slot_elems * 4 * (staged ? 2 : 1) : 0;
-    const int64_t tile_elems = fused ? pick_tile_elems((int64_t)count * es * R, o, es * R / 4, HCCL_OP_REDUCE_N) : pick_tile_elems(count * 4 * (R - 1), o, 4, HCCL_OP_REDUCE);
+    const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
+    const int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, 4, HCCL_OP_REDUCE);
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), scratch, 0, &graw));
     GraphPtr g(graw);
     g->compulsory_bytes = compulsory;
@@ -331,7 +332,7 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw));
     GraphPtr g(graw);
     g->compulsory_bytes = offs[R] * es + (int64_t)R * offs[R] * es;
-    const int64_t tile = pick_tile_elems(offs[R] * es * R, o, 1, HCCL_OP_COPY);
+    const int64_t tile = o.tile_bytes ? (int64_t)o.tile_bytes : default_tile(offs[R] * es, o.sm_budget, 1, 16 << 10, 256 << 10, sweep_of(o, HCCL_OP_COPY));
     // one subgraph per chunk q: it first lands in its owner's receive buffer, then goes round (ring)
     // or is read by everyone directly (one-shot)
     std::vector<int32_t> sg(R);

@@ -39,7 +39,8 @@ struct ExecParams {
     unsigned long long timeout_ns;
     long long n_user_signals;
     long long trig_wait_slot, trig_set_slot;
-    int trig_cmp, pad0;
+    int trig_cmp;
+    int static_tickets;  // no dependencies and no more items than blocks: block b runs item b, no atomics
     unsigned long long trig_wait_value, trig_set_value;
     const void* send[HCCL_MAX_RANKS];
     void* recv[HCCL_MAX_RANKS];
@@ -639,7 +640,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     if (tid == 0) {
         if (p.trig_wait_slot >= 0)
             live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value, 0xffffffffu);
-        next = atomicAdd(&p.ctl->ticket, 1);
+        next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
     }
     uint32_t cur = 0;
@@ -653,7 +654,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 cur = next;
                 have = live && cur < p.n_tiles && !aborted(p);
                 if (have) {
-                    next = atomicAdd(&p.ctl->ticket, 1);
+                    next = p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
                     have = fetch_tile(p, cur, s_tile[0], s_desc[0]);
                     ready = have && deps_ready(p, s_tile[0]);
                 }
@@ -1119,12 +1120,12 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         bool live = true;
         if (p.trig_wait_slot >= 0)
             live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value, 0xffffffffu);
-        uint32_t next = atomicAdd(&p.ctl->ticket, 1);
+        uint32_t next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
         while (live && d.ok) {
             const uint32_t cur = next;
             if (cur >= p.n_tiles || aborted(p)) break;
-            next = atomicAdd(&p.ctl->ticket, 1);
+            next = p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
             if (!dma_item(p, d, cur)) break;
         }
         // wind down: finish what is in flight, release the compute warps, leave
@@ -1500,6 +1501,7 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     int blocks = p->opts.sm_budget;
     if ((uint32_t)blocks > prm.n_tiles) blocks = (int)std::max<uint32_t>(prm.n_tiles, 1u);
     prm.nblocks = (uint32_t)blocks;
+    prm.static_tickets = (prm.n_waits == 0 && prm.n_tiles <= (uint32_t)blocks) ? 1 : 0;
     if (p->opts.engine == HCCL_ENGINE_BULK) {
         const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : 6, 2), (int)bulk::MAX_STAGES);
         const size_t smem = (size_t)ns * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
@@ -1656,6 +1658,7 @@ extern "C" hccl_status_t hccl_execute_noalloc(hccl_plan_t* p, const void* const*
     prm.trig_wait_slot = -1;
     prm.trig_set_slot = -1;
     prm.trig_cmp = 0;
+    prm.static_tickets = 0;
     prm.trig_wait_value = prm.trig_set_value = 0;
     for (int r = 0; r < R; ++r) {
         prm.send[r] = sendbufs[r];

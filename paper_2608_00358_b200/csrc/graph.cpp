@@ -64,12 +64,6 @@ bool is_send(const hccl_wqe_t& w, int rank) {
     return a_local || b_local;
 }
 
-uint64_t pow2_floor(uint64_t x) {
-    uint64_t p = 1;
-    while (p * 2 <= x) p *= 2;
-    return p;
-}
-
 }  // namespace
 
 void hccl::fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in) {
@@ -302,13 +296,19 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
             if (w.op == HCCL_OP_REDUCE) need(w.b, w.dtype_b);
         }
     }
-    uint64_t tile_bytes = p->opts.tile_bytes;
-    if (tile_bytes == 0) {
-        uint64_t per = (uint64_t)weight / (8ull * (uint64_t)p->opts.sm_budget);
-        tile_bytes = std::min<uint64_t>(256u << 10, std::max<uint64_t>(16u << 10, pow2_floor(std::max<uint64_t>(per, 1))));
-    }
-    tile_bytes = std::max<uint64_t>(tile_bytes, 256);
+    // Default tile sizes: about two tiles per block for each kind of operation (latency-bound sizes want few,
+    // large tiles; big ones are capped), whole passes of the block's threads. opts.tile_bytes overrides.
+    int64_t units[3] = {0, 0, 0};  // COPY bytes, REDUCE elements, REDUCE_N elements of the whole packet
+    for (const Wqe& q : g->wqes)
+        if (is_data_op(q.w.op)) units[q.w.op] += q.w.count;
+    const int B = p->opts.sm_budget;
+    const bool fixed = p->opts.tile_bytes != 0;
+    const int64_t def_copy = default_tile(units[HCCL_OP_COPY], B, 2, 16 << 10, 256 << 10, sweep_of(p->opts, HCCL_OP_COPY));
+    const int64_t def_reduce = default_tile(units[HCCL_OP_REDUCE], B, 2, 4 << 10, 64 << 10, sweep_of(p->opts, HCCL_OP_REDUCE));
+    const int64_t def_reduce_n = default_tile(units[HCCL_OP_REDUCE_N], B, 2, 1 << 10, 32 << 10, sweep_of(p->opts, HCCL_OP_REDUCE_N));
+    const uint64_t tile_bytes = fixed ? std::max<uint64_t>(p->opts.tile_bytes, 256) : (uint64_t)def_copy;
     p->opts.tile_bytes = tile_bytes;
+    (void)weight;
 
     // ---- tiles per WQE
     std::vector<int64_t> tcount(n), ntiles(n);
@@ -321,11 +321,10 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         }
         int64_t tc = w.tile_count;
         if (tc <= 0) {
-            // default: tile_bytes of the widest operand (multi-input sums: four times that, spread over the
-            // sources), rounded to whole passes of the block's threads unless the caller fixed tile_bytes
-            const int64_t target = w.op == HCCL_OP_REDUCE_N ? (int64_t)(4 * tile_bytes / (uint64_t)(widest(w) * std::max<int>(w.nsrc, 1)))
-                                                             : (int64_t)(tile_bytes / (uint64_t)widest(w));
-            tc = opts_in && opts_in->tile_bytes ? std::max<int64_t>(target, 1) : round_tile(target, sweep_of(p->opts, w.op));
+            if (fixed)  // caller's tile_bytes, in bytes of the widest operand (all sources together for REDUCE_N)
+                tc = std::max<int64_t>(1, (int64_t)(tile_bytes / (uint64_t)(widest(w) * (w.op == HCCL_OP_REDUCE_N ? std::max<int>(w.nsrc, 1) : 1))));
+            else
+                tc = w.op == HCCL_OP_COPY ? def_copy : (w.op == HCCL_OP_REDUCE ? def_reduce : def_reduce_n);
         }
         tc = std::min<int64_t>(std::max<int64_t>(tc, 1), 0x7fffffff);
         tcount[i] = tc;

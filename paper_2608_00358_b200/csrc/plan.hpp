@@ -89,6 +89,18 @@ inline int64_t sweep_of(const hccl_opts_t& o, int op) {
     if (op == HCCL_OP_REDUCE) return workers * 32;            // 4 x 8 elements per thread
     return workers * 8;                                       // REDUCE_N: 8 elements per thread
 }
+// Default tile size, in the operation's count units, for work of `total_units` spread over `blocks` blocks:
+// about `per_block` tiles per block, a power of two between lo and hi, then whole passes of the threads.
+inline int64_t nearest_pow2(int64_t x) {
+    int64_t p = 1;
+    while (p * 2 <= x) p *= 2;
+    return (x - p > 2 * p - x) ? 2 * p : p;
+}
+inline int64_t round_tile(int64_t target, int64_t sweep);
+inline int64_t default_tile(int64_t total_units, int blocks, int per_block, int64_t lo, int64_t hi, int64_t sweep) {
+    const int64_t want = nearest_pow2(std::max<int64_t>(1, total_units / std::max(1, blocks * per_block)));
+    return round_tile(std::min(hi, std::max(lo, want)), sweep);
+}
 inline int64_t round_tile(int64_t target, int64_t sweep) {
     if (target >= sweep) return target / sweep * sweep;
     return std::max<int64_t>(64, (target + 63) / 64 * 64);
