@@ -669,8 +669,8 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         if (tid == 0) {
             const bool simple = have && ready && s_desc[b].op != HCCL_OP_WAIT && s_desc[b].op != HCCL_OP_SET;
             if (!simple && prev && (sig0 >= 0 || sig1 >= 0)) {
-                // item k may have to wait (perhaps for item k-1 itself): publish k-1 first
-                __threadfence();
+                // item k may have to wait (perhaps for item k-1 itself): publish k-1 first. The release is
+                // cumulative: it covers the workers' stores that the DONE barrier ordered before this thread.
                 if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
                 if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
                 sig0 = sig1 = -1;
@@ -683,7 +683,6 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         const int go = s_go[b];
         if (tid == 0) {
             if (sig0 >= 0 || sig1 >= 0) {  // publish item k-1 while the workers run item k
-                __threadfence();
                 if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
                 if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
             }
@@ -1179,8 +1178,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         }
         if (kind != PIECE_COPY && pi.last && (pi.signal[0] >= 0 || pi.signal[1] >= 0)) {
             asm volatile("bar.sync 1, %0;" ::"r"(cnth) : "memory");  // every compute warp has stored its share
-            if (ctid == 0) {
-                __threadfence();
+            if (ctid == 0) {  // release, cumulative over the stores the barrier ordered before this thread
                 if (pi.signal[0] >= 0) red_release_add_u32(p.counters + pi.signal[0], 1);
                 if (pi.signal[1] >= 0) red_release_add_u32(p.counters + pi.signal[1], 1);
             }
