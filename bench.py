@@ -168,6 +168,7 @@ def side_configs(quick: bool):
                     "schedule_bytes": int(i.schedule_bytes), "compulsory_bytes": int(i.compulsory_bytes),
                     "tiles": int(i.n_tiles), "chain_depth": int(i.chain_depth), "note": "L2-resident, latency-bound"}
         out[key]["schedule_gbs_back_to_back"] = i.schedule_bytes / out[key]["back_to_back_us"] / 1e3
+        out[key]["graph_replay_us"] = float(wk.time_graph_replay(wl) * 1e3)
 
     latency(wk.config1(), "1_allreduce_ring_r4_fp32_1Mi")
     latency(wk.config2(), "2_alltoallv_r8_bf16_dim128")

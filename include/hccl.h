@@ -92,7 +92,7 @@ typedef struct {
     uint32_t flags;         /* HCCL_FLAG_* */
     int32_t chain_group;    /* chains scheduled together in chain-group-major order (default 16) */
     int32_t threads;        /* threads per block, multiple of 32 (default 512) */
-    int32_t stages;         /* bulk engine: shared-memory stages of 32 KiB per block, 2..8 (default 6) */
+    int32_t stages;         /* bulk engine: shared-memory stages of 32 KiB per block, 2..6 (default 6) */
     int32_t cluster;        /* register engine: launch blocks in clusters of this size (2, 4, 8) so that they sit on
                                neighbouring SMs; 0/1 = no clusters. Ignored unless it divides the block count. */
     int32_t light;          /* register engine: nonzero = the 64-register build (several blocks per SM) */
@@ -305,8 +305,11 @@ hccl_status_t hccl_plan_set_trigger(hccl_plan_t*, int64_t wait_slot, int32_t cmp
                                     uint64_t wait_per_epoch, int64_t set_slot, uint64_t set_value,
                                     uint64_t set_per_epoch);
 
-/* After the stream has been synchronised: the device-side verdict of the LAST execution.
- * *device_status is HCCL_OK, HCCL_ERR_TIMEOUT or HCCL_ERR_BAD_DESCRIPTOR; *detail the tile index involved. */
+/* After the stream has been synchronised: the device-side verdict of the LAST execution. The device numbers
+ * its own executions (epoch = completed executions of the bound workspace + 1), so hccl_execute is a plain
+ * kernel launch that can be captured in a CUDA graph and replayed; replays count as executions.
+ * *device_status is HCCL_OK, HCCL_ERR_TIMEOUT or HCCL_ERR_BAD_DESCRIPTOR; *detail is the tile index
+ * involved or, on HCCL_OK, the number of executions completed since the plan was bound. */
 hccl_status_t hccl_plan_status(hccl_plan_t*, hccl_status_t* device_status, int64_t* detail);
 
 typedef struct {

@@ -35,16 +35,26 @@ struct ExecParams {
     char* scratch;
     unsigned long long* user_signals;
     uint32_t n_tiles, n_descs, n_syncs, n_waits;
-    uint32_t epoch, R, nblocks, n_signals;
+    uint32_t R, nblocks, n_signals, pad0;
     unsigned long long timeout_ns;
     long long n_user_signals;
     long long trig_wait_slot, trig_set_slot;
     int trig_cmp;
     int static_tickets;  // no dependencies and no more items than blocks: block b runs item b, no atomics
-    unsigned long long trig_wait_value, trig_set_value;
+    unsigned long long trig_wait_value, trig_wait_per_epoch, trig_set_value, trig_set_per_epoch;
     const void* send[HCCL_MAX_RANKS];
     void* recv[HCCL_MAX_RANKS];
 };
+
+// The execution number ("epoch") of the running launch. It lives on the device: every block derives it from
+// the control block (done_epoch of the previous execution + 1), so a launch captured in a CUDA graph finds
+// the right epoch on every replay. Kept in shared memory, written once per block at kernel entry.
+__shared__ uint32_t g_epoch;
+template <class P>
+__device__ __forceinline__ void init_epoch(const P& p) {
+    if (threadIdx.x == 0) g_epoch = *(volatile uint32_t*)&p.ctl->done_epoch + 1u;
+    __syncthreads();
+}
 
 // ------------------------------------------------------------------ device primitives
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
@@ -88,20 +98,20 @@ __device__ __forceinline__ bool compare(unsigned long long v, int cmp, unsigned 
 // Record a failure once per execution and tell everyone to stop.
 template <class P>
 __device__ __noinline__ void fail(const P& p, uint32_t code, unsigned long long detail) {
-    if (atomicExch(&p.ctl->fail_epoch, p.epoch) != p.epoch) {  // first failure of this execution wins
+    if (atomicExch(&p.ctl->fail_epoch, g_epoch) != g_epoch) {  // first failure of this execution wins
         p.ctl->status = code;
         p.ctl->detail = detail;
     }
     __threadfence();
-    atomicExch(&p.ctl->abort, p.epoch);
+    atomicExch(&p.ctl->abort, g_epoch);
 }
 template <class P>
-__device__ __forceinline__ bool aborted(const P& p) { return ld_relaxed_u32(&p.ctl->abort) == p.epoch; }
+__device__ __forceinline__ bool aborted(const P& p) { return ld_relaxed_u32(&p.ctl->abort) == g_epoch; }
 
 // Bounded wait until counters[sync] has received epoch * per_epoch bumps (wrap-safe compare).
 __device__ bool wait_counter(const ExecParams& p, uint32_t sync, uint32_t per_epoch, uint32_t tile) {
     const uint32_t* c = p.counters + sync;
-    const uint32_t target = p.epoch * per_epoch;
+    const uint32_t target = g_epoch * per_epoch;
     if ((int32_t)(ld_acquire_u32(c) - target) >= 0) return true;
     const unsigned long long deadline = globaltimer_ns() + p.timeout_ns;
     uint32_t spins = 0;
@@ -528,11 +538,11 @@ __device__ bool prepare_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d
     }
     if (d.op == HCCL_OP_WAIT) {
         const unsigned long long* addr = (d.kind_a == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + d.off_a;
-        if (!wait_signal(p, addr, d.cmp, d.value + (unsigned long long)p.epoch * d.value_per_epoch, cur)) return false;
+        if (!wait_signal(p, addr, d.cmp, d.value + (unsigned long long)g_epoch * d.value_per_epoch, cur)) return false;
     } else if (d.op == HCCL_OP_SET) {
         unsigned long long* addr = (d.kind_dst == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + d.off_dst;
         __threadfence();
-        st_release_u64(addr, d.value + (unsigned long long)p.epoch * d.value_per_epoch);
+        st_release_u64(addr, d.value + (unsigned long long)g_epoch * d.value_per_epoch);
     }
     return true;
 }
@@ -552,12 +562,12 @@ __device__ void leave(const P& p) {
     const uint32_t prev = atomicAdd(&p.ctl->exits, 1);
     if (prev == p.nblocks - 1) {
         __threadfence();
-        if (p.trig_set_slot >= 0 && !aborted(p)) st_release_u64(p.user_signals + p.trig_set_slot, p.trig_set_value);
+        if (p.trig_set_slot >= 0 && !aborted(p)) st_release_u64(p.user_signals + p.trig_set_slot, p.trig_set_value + (unsigned long long)g_epoch * p.trig_set_per_epoch);
         p.ctl->t_last_ns = globaltimer_ns();
         p.ctl->ticket = 0;
         p.ctl->exits = 0;
         __threadfence();
-        p.ctl->done_epoch = p.epoch;
+        p.ctl->done_epoch = g_epoch;
     }
 }
 
@@ -585,7 +595,7 @@ __device__ bool deps_ready(const ExecParams& p, const Tile& t) {
     for (uint32_t w = 0; w < t.wait_cnt; ++w) {
         const Wait x = p.waits[t.wait_off + w];
         if (x.sync >= p.n_syncs) return false;
-        if ((int32_t)(ld_acquire_u32(p.counters + x.sync) - p.epoch * x.per_epoch) < 0) return false;
+        if ((int32_t)(ld_acquire_u32(p.counters + x.sync) - g_epoch * x.per_epoch) < 0) return false;
     }
     return true;
 }
@@ -603,11 +613,11 @@ __device__ bool wait_deps(const ExecParams& p, uint32_t cur, const Tile& t, cons
     }
     if (d.op == HCCL_OP_WAIT) {
         const unsigned long long* addr = (d.kind_a == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + d.off_a;
-        if (!wait_signal(p, addr, d.cmp, d.value + (unsigned long long)p.epoch * d.value_per_epoch, cur)) return false;
+        if (!wait_signal(p, addr, d.cmp, d.value + (unsigned long long)g_epoch * d.value_per_epoch, cur)) return false;
     } else if (d.op == HCCL_OP_SET) {
         unsigned long long* addr = (d.kind_dst == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + d.off_dst;
         __threadfence();
-        st_release_u64(addr, d.value + (unsigned long long)p.epoch * d.value_per_epoch);
+        st_release_u64(addr, d.value + (unsigned long long)g_epoch * d.value_per_epoch);
     }
     return true;
 }
@@ -623,6 +633,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     __shared__ int s_go[2];
     const uint32_t tid = threadIdx.x, nth = blockDim.x;
     constexpr uint32_t FULL = 1, DONE = 3;  // barrier ids FULL+b, DONE+b
+    init_epoch(p);
     if (tid >= 32) {
         const uint32_t wtid = tid - 32, nwork = nth - 32;
         for (uint32_t k = 0;; ++k) {
@@ -639,7 +650,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     bool live = true, have = false, ready = false;
     if (tid == 0) {
         if (p.trig_wait_slot >= 0)
-            live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value, 0xffffffffu);
+            live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value + (unsigned long long)g_epoch * p.trig_wait_per_epoch, 0xffffffffu);
         next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
     }
@@ -718,7 +729,7 @@ __global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_c
 // is handed to the compute warps as a whole work item for the register path.
 namespace bulk {
 
-constexpr uint32_t MAX_STAGES = 8;
+constexpr uint32_t MAX_STAGES = 6;  // 6 x 32 KiB + bookkeeping fits the 227 KB a block may have
 constexpr uint32_t REGION = 16384;            // bytes per operand region of a stage
 constexpr uint32_t STAGE_BYTES = 2 * REGION;  // region A + region B; a COPY piece uses both as one buffer
 constexpr uint32_t PIECE_ELEMS = 4096;        // elements per REDUCE piece (fp32 fills a region exactly)
@@ -943,7 +954,7 @@ __device__ __forceinline__ void keep_lag(const ExecParams& p, Dma& d) {
 }
 
 __device__ bool wait_counter_draining(const ExecParams& p, Dma& d, uint32_t sync, uint32_t per_epoch, uint32_t tile) {
-    const uint32_t target = p.epoch * per_epoch;
+    const uint32_t target = g_epoch * per_epoch;
     if ((int32_t)(ld_acquire_u32(p.counters + sync) - target) >= 0) return true;
     drain(p, d);  // the item waited for may sit in this block's own pipeline
     if (!d.ok) return false;
@@ -995,14 +1006,14 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
             drain(p, d);
             if (!d.ok) return false;
             const unsigned long long* addr = (ds.kind_a == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + ds.off_a;
-            if (!wait_signal(p, addr, ds.cmp, ds.value + (unsigned long long)p.epoch * ds.value_per_epoch, cur)) return false;
+            if (!wait_signal(p, addr, ds.cmp, ds.value + (unsigned long long)g_epoch * ds.value_per_epoch, cur)) return false;
             publish_tile(p, t);
             return true;
         }
         case HCCL_OP_SET: {
             unsigned long long* addr = (ds.kind_dst == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + ds.off_dst;
             __threadfence();
-            st_release_u64(addr, ds.value + (unsigned long long)p.epoch * ds.value_per_epoch);
+            st_release_u64(addr, ds.value + (unsigned long long)g_epoch * ds.value_per_epoch);
             publish_tile(p, t);
             return true;
         }
@@ -1092,6 +1103,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
     const uint32_t tid = threadIdx.x;
     const uint32_t ncw = (blockDim.x >> 5) - 1;  // compute warps
     const uint32_t full = smem_u32(bars), empty = smem_u32(bars + ns);
+    init_epoch(p);
     if (tid == 0) {
         for (uint32_t s = 0; s < ns; ++s) {
             mbar_init(full + 8 * s, 1);
@@ -1118,7 +1130,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         d.ok = true;
         bool live = true;
         if (p.trig_wait_slot >= 0)
-            live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value, 0xffffffffu);
+            live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value + (unsigned long long)g_epoch * p.trig_wait_per_epoch, 0xffffffffu);
         uint32_t next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
         while (live && d.ok) {
@@ -1205,12 +1217,12 @@ struct DynParams {
     long long* rdispls_out;        // device, [R*R] indexed [d*R+s], or null
     Control* ctl;
     unsigned long long* user_signals;
-    uint32_t epoch, R, nblocks, pad0;
+    uint32_t R, nblocks;
     unsigned long long timeout_ns;
     unsigned long long row_bytes, tile_bytes;
     long long trig_wait_slot, trig_set_slot;
     int trig_cmp, pad1;
-    unsigned long long trig_wait_value, trig_set_value;
+    unsigned long long trig_wait_value, trig_wait_per_epoch, trig_set_value, trig_set_per_epoch;
     long long max_send_rows[DYN_MAX_RANKS], max_recv_rows[DYN_MAX_RANKS];
     const void* send[DYN_MAX_RANKS];
     void* recv[DYN_MAX_RANKS];
@@ -1237,12 +1249,13 @@ __global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant
     __shared__ uint32_t s_ticket;
     __shared__ int s_live;
     const uint32_t tid = threadIdx.x, nth = blockDim.x, lane = tid & 31u, warp = tid >> 5, nwarps = nth >> 5;
+    init_epoch(q);
     if (tid == 0) {
         s_bad = 0;
         s_bad_at = 0;
         bool live = true;
         if (q.trig_wait_slot >= 0)
-            live = wait_signal(q, q.user_signals + q.trig_wait_slot, q.trig_cmp, q.trig_wait_value, 0xffffffffu);
+            live = wait_signal(q, q.user_signals + q.trig_wait_slot, q.trig_cmp, q.trig_wait_value + (unsigned long long)g_epoch * q.trig_wait_per_epoch, 0xffffffffu);
         s_live = live ? 1 : 0;
     }
     __syncthreads();
@@ -1387,6 +1400,15 @@ hccl_status_t hccl_plan_bind(hccl_plan_t* p, void* dev_workspace, size_t bytes, 
     cudaStream_t s = (cudaStream_t)stream;
     CUDA_TRY(cudaMemcpyAsync(dev_workspace, img.data(), img.size(), cudaMemcpyHostToDevice, s));
     CUDA_TRY(cudaStreamSynchronize(s));
+    // opt-in shared memory sizes are set here, once, so that hccl_execute itself is only a launch
+    if (p->dynamic) {
+        const size_t RR = (size_t)p->R * p->R;
+        const size_t smem = RR * 24 + (RR + 1) * 4 + 16;
+        if (smem > 48 * 1024) CUDA_TRY(cudaFuncSetAttribute(hccl_a2a_dynamic, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(DYN_MAX_RANKS * DYN_MAX_RANKS * 24 + (DYN_MAX_RANKS * DYN_MAX_RANKS + 1) * 4 + 16)));
+    } else if (p->opts.engine == HCCL_ENGINE_BULK) {
+        const size_t smem = (size_t)bulk::MAX_STAGES * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
+        if (smem <= 227 * 1024) CUDA_TRY(cudaFuncSetAttribute(hccl_executor_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)std::min<size_t>(smem, 227 * 1024)));
+    }
     p->workspace = dev_workspace;
     p->workspace_bytes = bytes;
     p->epoch = 0;
@@ -1437,7 +1459,6 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
         q.rdispls_out = (long long*)p->dyn_rdispls_out;
         q.ctl = (Control*)((char*)p->workspace + p->layout.control);
         q.user_signals = (unsigned long long*)p->user_signals;
-        q.epoch = epoch;
         q.R = (uint32_t)p->R;
         q.nblocks = (uint32_t)p->opts.sm_budget;
         q.timeout_ns = p->opts.timeout_ns;
@@ -1446,8 +1467,10 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
         q.trig_wait_slot = p->trig_wait_slot;
         q.trig_set_slot = p->trig_set_slot;
         q.trig_cmp = p->trig_cmp;
-        q.trig_wait_value = p->trig_wait_value + (uint64_t)epoch * p->trig_wait_per_epoch;
-        q.trig_set_value = p->trig_set_value + (uint64_t)epoch * p->trig_set_per_epoch;
+        q.trig_wait_value = p->trig_wait_value;
+        q.trig_wait_per_epoch = p->trig_wait_per_epoch;
+        q.trig_set_value = p->trig_set_value;
+        q.trig_set_per_epoch = p->trig_set_per_epoch;
         for (int r = 0; r < p->R; ++r) {
             q.max_send_rows[r] = p->dyn_max_send_rows[r];
             q.max_recv_rows[r] = p->dyn_max_recv_rows[r];
@@ -1456,11 +1479,6 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
         }
         const size_t RR = (size_t)p->R * p->R;
         const size_t smem = RR * 24 + (RR + 1) * 4 + 16;
-        static thread_local size_t dyn_smem_set = 0;
-        if (smem > 48 * 1024 && smem > dyn_smem_set) {
-            CUDA_TRY(cudaFuncSetAttribute(hccl_a2a_dynamic, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            dyn_smem_set = smem;
-        }
         hccl_a2a_dynamic<<<p->opts.sm_budget, p->opts.threads, smem, (cudaStream_t)stream>>>(q);
         CUDA_TRY(cudaGetLastError());
         p->epoch = epoch;
@@ -1484,14 +1502,15 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     prm.n_signals = (uint32_t)p->n_signals;
     prm.R = (uint32_t)p->R;
     const uint32_t epoch = p->epoch + 1;
-    prm.epoch = epoch;
     prm.timeout_ns = p->opts.timeout_ns;
     prm.n_user_signals = p->n_user_signals;
     prm.trig_wait_slot = p->trig_wait_slot;
     prm.trig_set_slot = p->trig_set_slot;
     prm.trig_cmp = p->trig_cmp;
-    prm.trig_wait_value = p->trig_wait_value + (uint64_t)epoch * p->trig_wait_per_epoch;
-    prm.trig_set_value = p->trig_set_value + (uint64_t)epoch * p->trig_set_per_epoch;
+    prm.trig_wait_value = p->trig_wait_value;
+    prm.trig_wait_per_epoch = p->trig_wait_per_epoch;
+    prm.trig_set_value = p->trig_set_value;
+    prm.trig_set_per_epoch = p->trig_set_per_epoch;
     for (int r = 0; r < p->R; ++r) {
         prm.send[r] = sendbufs[r];
         prm.recv[r] = recvbufs[r];
@@ -1503,11 +1522,6 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     if (p->opts.engine == HCCL_ENGINE_BULK) {
         const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : 6, 2), (int)bulk::MAX_STAGES);
         const size_t smem = (size_t)ns * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
-        static thread_local size_t smem_set = 0;
-        if (smem > smem_set) {
-            CUDA_TRY(cudaFuncSetAttribute(hccl_executor_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            smem_set = smem;
-        }
         const int threads = std::max(64, p->opts.threads);
         hccl_executor_bulk<<<blocks, threads, smem, (cudaStream_t)stream>>>(prm, ns, (uint32_t)(p->opts.copy_by_warps != 0));
     } else {
@@ -1557,19 +1571,16 @@ hccl_status_t hccl_plan_status(hccl_plan_t* p, hccl_status_t* device_status, int
     if (!p->workspace) return HCCL_ERR_NOT_BOUND;
     Control c;
     CUDA_TRY(cudaMemcpy(&c, (char*)p->workspace + p->layout.control, sizeof(c), cudaMemcpyDeviceToHost));
-    if (p->epoch == 0) {
-        *device_status = HCCL_OK;
-        if (detail) *detail = 0;
-        return HCCL_OK;
-    }
-    if (c.fail_epoch == p->epoch) {
+    // The device numbers its own executions (so that graph replays count too): the last one failed if the
+    // failure stamp carries its number.
+    if (c.done_epoch != 0 && c.fail_epoch == c.done_epoch) {
         *device_status = (hccl_status_t)c.status;
         if (detail) *detail = (int64_t)c.detail;
         return HCCL_OK;
     }
-    if (c.done_epoch != p->epoch) return HCCL_ERR_BUSY;  // the last execution has not finished
+    if (c.exits != 0) return HCCL_ERR_BUSY;  // blocks of an execution are still leaving: synchronise first
     *device_status = HCCL_OK;
-    if (detail) *detail = 0;
+    if (detail) *detail = (int64_t)c.done_epoch;
     return HCCL_OK;
 }
 
@@ -1650,14 +1661,13 @@ extern "C" hccl_status_t hccl_execute_noalloc(hccl_plan_t* p, const void* const*
     prm.n_waits = (uint32_t)p->waits.size();
     prm.n_signals = (uint32_t)p->n_signals;
     prm.R = (uint32_t)R;
-    prm.epoch = 1;  // the tables were just reset, so every call is a first execution
     prm.timeout_ns = p->opts.timeout_ns;
     prm.n_user_signals = 0;
     prm.trig_wait_slot = -1;
     prm.trig_set_slot = -1;
     prm.trig_cmp = 0;
     prm.static_tickets = 0;
-    prm.trig_wait_value = prm.trig_set_value = 0;
+    prm.trig_wait_value = prm.trig_set_value = prm.trig_wait_per_epoch = prm.trig_set_per_epoch = 0;
     for (int r = 0; r < R; ++r) {
         prm.send[r] = sendbufs[r];
         prm.recv[r] = recvbufs[r];

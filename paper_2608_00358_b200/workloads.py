@@ -144,3 +144,25 @@ def time_each(wl: Workload, iters: int, warmup: int, flush: Optional[torch.Tenso
     s.synchronize()
     wl.dc.check()
     return np.array([a.elapsed_time(b) for a, b in ev])
+
+
+def time_graph_replay(wl: Workload, per_graph: int = 50, replays: int = 10) -> float:
+    """Mean milliseconds per execution when `per_graph` executions are captured in one CUDA graph and the
+    graph is replayed: what is left when the per-launch host cost is taken out."""
+    s = torch.cuda.Stream()
+    wl.dc.execute(s)
+    s.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        for _ in range(per_graph):
+            wl.dc.execute(s)
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    wl.dc.check()
+    return e0.elapsed_time(e1) / (replays * per_graph)
