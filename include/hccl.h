@@ -62,9 +62,13 @@ typedef enum { HCCL_FP32 = 0, HCCL_BF16 = 1, HCCL_FP16 = 2 } hccl_dtype_t; /* th
 typedef enum {
     HCCL_ALGO_RING = 0,      /* unidirectional ring, reduce-scatter then all-gather (Sec. III-B.2, Fig. 5) */
     HCCL_ALGO_ONESHOT = 1,   /* "all-to-all style": every rank reads every peer once (Sec. V-F, PE kernels) */
-    HCCL_ALGO_RING_FUSED = 2 /* the ring's sums in the ring's order, but each chunk's chain collapsed into
+    HCCL_ALGO_RING_FUSED = 2,/* the ring's sums in the ring's order, but each chunk's chain collapsed into
                                 one multi-input reduction (cf. NOOP-joined tree reductions, Sec. III-B.2).
                                 Reported as its own algorithm, never as "ring". */
+    HCCL_ALGO_RING_2LEVEL = 3 /* topology-aware two-level ring (Sec. V-D): ranks form racks of opts.rack_size; sums
+                                run round each rack's ring first, then round the ring of racks, and results
+                                are gathered across racks first, then inside each rack, so that only 1/rack_size
+                                of the data ever crosses between racks. AllReduce and AllGather. */
 } hccl_algo_t;
 
 /* Which data mover the executor uses for aligned bulk work. */
@@ -97,7 +101,8 @@ typedef struct {
                                neighbouring SMs; 0/1 = no clusters. Ignored unless it divides the block count. */
     int32_t light;          /* register engine: nonzero = the 64-register build (several blocks per SM) */
     int32_t copy_by_warps;  /* bulk engine: nonzero = COPY pieces are loaded by the bulk unit but stored by the compute warps */
-    int32_t reserved[1];
+    int32_t rack_size;      /* ranks per rack for HCCL_ALGO_RING_2LEVEL and for cross-rack byte accounting (default 16,
+                               the paper's rack, Sec. V-D) */
 } hccl_opts_t;
 
 typedef struct hccl_plan hccl_plan_t;   /* opaque, host-owned: a compiled, cacheable work packet (Sec. V-B) */
@@ -208,6 +213,7 @@ typedef struct {
  * into the same number of tiles; otherwise the whole of dep_wqe is waited for. The schedule's author is
  * responsible for the claim; hccl_plan_check_hazards verifies it tile by tile. */
 #define HCCL_DEP_ELEMENTWISE 32u
+#define HCCL_DEP_ELEMENTWISE2 64u /* the same claim for dep_wqe2 */
 
 /* Cache hints on data WQEs. READ_ONCE: no source byte of this WQE is read by any other WQE of the packet
  * (it is streamed through the L2 with an evict-first policy). */
@@ -324,6 +330,8 @@ typedef struct {
     int32_t R, sm_budget, threads, engine;
     int64_t tile_bytes;
     int64_t epoch;            /* executions enqueued since the last bind */
+    int64_t crossrack_bytes;  /* bytes that data WQEs move between ranks of different racks (racks of opts.rack_size):
+                                 what would cross the scale-out network with real ranks (Sec. II-A.3, V-D) */
 } hccl_plan_info_t;
 hccl_status_t hccl_plan_info(const hccl_plan_t*, hccl_plan_info_t* out);
 

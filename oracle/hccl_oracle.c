@@ -338,6 +338,39 @@ int oracle_allreduce_oneshot_f32(int R, int64_t n, int dt, const void *const *X,
     return 0;
 }
 
+/* Two-level ring order (Sec. V-D: topology-aware schedules that keep most exchanges inside a rack).
+ * R = G racks of L ranks; rank (g, l) = g*L + l. The buffer is cut into L chunks (offs1, L+1 entries) and
+ * every chunk j into G sub-chunks (offs2[j*(G+1) .. j*(G+1)+G], absolute element offsets). For sub-chunk
+ * (j, k): first every rack g sums its own L ranks round its ring, P_g = ((X_{g,j+1} + X_{g,j+2}) + ...) +
+ * X_{g,j} (local indices mod L); then the racks' partials are summed round the ring of racks,
+ * ((P_{k+1} + P_{k+2}) + ...) + P_k (rack indices mod G). Every add is FP32 (partials are never
+ * re-quantised), one rounding to the stored type at the end; all ranks receive the result. */
+int oracle_allreduce_ring2_f32(int G, int L, const int64_t *offs1, const int64_t *offs2, int dt,
+                               const void *const *X, void *const *Y) {
+    if (G < 1 || L < 1) return 1;
+    const int R = G * L;
+    (void)offs1;
+    for (int j = 0; j < L; ++j) {
+        for (int k = 0; k < G; ++k) {
+            const int64_t lo = offs2[j * (G + 1) + k], hi = offs2[j * (G + 1) + k + 1];
+            for (int64_t i = lo; i < hi; ++i) {
+                volatile float total = 0.0f;
+                for (int tg = 1; tg <= G; ++tg) {
+                    const int g = (k + tg) % G;
+                    volatile float part = (float)load_elem(X[g * L + (j + 1) % L], i, dt);
+                    for (int t = 2; t <= L; ++t) {
+                        volatile float x = (float)load_elem(X[g * L + (j + t) % L], i, dt);
+                        part = part + x;
+                    }
+                    if (tg == 1) total = part; else total = total + part;
+                }
+                for (int r = 0; r < R; ++r) store_elem(Y[r], i, dt, (double)total);
+            }
+        }
+    }
+    return 0;
+}
+
 /* Distance in units in the last place between two stored values of type dt,
  * measured on the monotone integer image of the bit patterns (sign-magnitude
  * mapped to an ordered integer; +0 and -0 coincide). Used by the tests'

@@ -154,6 +154,27 @@ def reducescatter_ring_f32(dt: int, X: list, recvcounts) -> list:
     return _ring(lib().oracle_reducescatter_ring_f32, dt, X, rc, lambda r: int(rc[r]))
 
 
+def two_level_offsets(n: int, G: int, L: int):
+    """Chunk j of L (floor split of n), each cut into G sub-chunks (floor split of the chunk)."""
+    offs1 = floor_chunk_offsets(n, L)
+    offs2 = np.zeros((L, G + 1), dtype=np.int64)
+    for j in range(L):
+        lo, hi = int(offs1[j]), int(offs1[j + 1])
+        offs2[j] = [lo + (k * (hi - lo)) // G for k in range(G + 1)]
+    return offs1, offs2
+
+
+def allreduce_ring2_f32(dt: int, X: list, G: int, L: int) -> list:
+    R, n = len(X), X[0].size
+    assert R == G * L
+    offs1, offs2 = two_level_offsets(n, G, L)
+    o1, p1 = _i64(offs1)
+    o2, p2 = _i64(offs2)
+    Y = [np.empty(n, dtype=np_dtype(dt)) for _ in range(R)]
+    _check(lib().oracle_allreduce_ring2_f32(G, L, p1, p2, dt, _ptrs(X), _ptrs(Y, True)), "ring2")
+    return Y
+
+
 def allreduce_oneshot_f32(dt: int, X: list) -> list:
     R, n = len(X), X[0].size
     Y = [np.empty(n, dtype=np_dtype(dt)) for _ in range(R)]

@@ -15,12 +15,12 @@ from . import _build
 OK, ERR_INVALID_ARG, ERR_DTYPE, ERR_COUNT_MISMATCH, ERR_OVERLAP, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_BUSY, \
     ERR_CUDA, ERR_TIMEOUT, ERR_BAD_DESCRIPTOR, ERR_NOT_BOUND, ERR_HAZARD = range(13)
 FP32, BF16, FP16 = 0, 1, 2
-ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED = 0, 1, 2
+ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED, ALGO_RING_2LEVEL = 0, 1, 2, 3
 ENGINE_AUTO, ENGINE_LSU, ENGINE_BULK = 0, 1, 2
 FLAG_LEVEL_MAJOR, FLAG_CHECK_HAZARDS, FLAG_STAGED_RING = 1, 2, 4
 OP_COPY, OP_REDUCE, OP_REDUCE_N, OP_WAIT, OP_SET, OP_NOOP = range(6)
 BUF_SEND, BUF_RECV, BUF_SCRATCH, BUF_SIGNAL, BUF_USER_SIGNAL = range(5)
-DEP_FENCE, DEP_SYNC, DEP_WQE_SYNC, DEP_RECV_SYNC, DEP_SEND_SYNC, DEP_ELEMENTWISE = 1, 2, 4, 8, 16, 32
+DEP_FENCE, DEP_SYNC, DEP_WQE_SYNC, DEP_RECV_SYNC, DEP_SEND_SYNC, DEP_ELEMENTWISE, DEP_ELEMENTWISE2 = 1, 2, 4, 8, 16, 32, 64
 CMP_EQ, CMP_NE, CMP_GE, CMP_GT, CMP_LE, CMP_LT = range(6)
 HINT_READ_ONCE = 1
 MAX_RANKS = 256
@@ -32,7 +32,7 @@ class Opts(C.Structure):
     _fields_ = [("sm_budget", C.c_int32), ("engine", C.c_int32), ("chunk_bytes", C.c_uint64),
                 ("tile_bytes", C.c_uint64), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
                 ("chain_group", C.c_int32), ("threads", C.c_int32), ("stages", C.c_int32), ("cluster", C.c_int32), ("light", C.c_int32),
-                ("copy_by_warps", C.c_int32), ("reserved", C.c_int32 * 1)]
+                ("copy_by_warps", C.c_int32), ("rack_size", C.c_int32)]
 
 
 class Ref(C.Structure):
@@ -52,7 +52,7 @@ class PlanInfo(C.Structure):
                 ("schedule_bytes", C.c_int64), ("compulsory_bytes", C.c_int64), ("scratch_bytes", C.c_int64),
                 ("send_bytes_total", C.c_int64), ("recv_bytes_total", C.c_int64), ("R", C.c_int32),
                 ("sm_budget", C.c_int32), ("threads", C.c_int32), ("engine", C.c_int32), ("tile_bytes", C.c_int64),
-                ("epoch", C.c_int64)]
+                ("epoch", C.c_int64), ("crossrack_bytes", C.c_int64)]
 
 
 class HcclError(RuntimeError):

@@ -185,6 +185,234 @@ std::vector<Chain> make_chains(int R, const std::vector<int64_t>& offs, bool sca
     return chains;
 }
 
+
+// ---------------------------------------------------------------- two-level (rack-aware) schedules
+// R = G racks of L ranks, rank (g, l) = g*L + l. One chain = one granule of one sub-chunk (j, k): chunk j of L,
+// cut again into G parts. Stages of a chain, each one WQE per participating rack:
+//   reduce inside every rack (L-1 steps, FP32 partial P_g in scratch), reduce across racks (G-1 steps,
+//   accumulator Q in scratch, the last step rounds into Y of rank (k, j)), gather across racks (G-1 hops
+//   between the ranks with local index j), gather inside every rack (L-1 hops). Only the middle two stages
+//   move bytes between racks, and they move 1/L of the data.
+struct Chain2 {
+    int j, k;
+    int64_t e0, len;
+};
+
+struct TwoLevel {
+    hccl_graph* g;
+    int G, L, dt, es;
+    int64_t n;            // elements per rank buffer (AllReduce) / total gathered elements (AllGather)
+    int64_t tile_elems;
+    hccl_opts_t o;
+    int rank(int rack, int local) const { return ((rack % G + G) % G) * L + ((local % L + L) % L); }
+};
+
+hccl_status_t add_dep_wqe(hccl_graph* g, int32_t sg, hccl_wqe_t& w, int64_t d1, int64_t d2, int64_t* id) {
+    w.dep_flags = 0;
+    w.dep_wqe = w.dep_wqe2 = -1;
+    if (d1 < 0) { d1 = d2; d2 = -1; }
+    if (d1 >= 0) {
+        w.dep_flags = HCCL_DEP_WQE_SYNC | HCCL_DEP_ELEMENTWISE;
+        w.dep_wqe = d1;
+        if (d2 >= 0) {
+            w.dep_wqe2 = d2;
+            w.dep_flags |= HCCL_DEP_ELEMENTWISE2;
+        }
+    }
+    return hccl_graph_add_wqe(g, sg, &w, id);
+}
+
+// Gather stages shared by AllReduce and AllGather: the data of a chain sits in Y of rank (k, j) at element
+// offset `yoff` (produced by WQE `origin`); it hops to the other racks' rank j, and inside every rack round
+// the local ring. `stage` selects which hop to emit (0 .. G-2 across racks, then G-1 .. G+L-3 inside racks).
+struct GatherState {
+    std::vector<int64_t> arrive;  // per rack: WQE that delivered the data to rank (rack, j)
+    std::vector<int64_t> last;    // per rack: last intra-rack hop emitted
+};
+
+hccl_status_t emit_gather_stage(const TwoLevel& T, int32_t sg, const Chain2& ch, int64_t yoff_elems, int stage, GatherState& st) {
+    const int G = T.G, es = T.es;
+    hccl_wqe_t w = blank();
+    w.op = HCCL_OP_COPY;
+    w.count = ch.len * es;
+    w.tile_count = T.tile_elems * es;
+    if (stage < G - 1) {
+        const int v = stage, src = T.rank(ch.k + v, ch.j), dst = T.rank(ch.k + v + 1, ch.j);
+        w.a = ref(HCCL_BUF_RECV, src, yoff_elems * es);
+        w.dst = ref(HCCL_BUF_RECV, dst, yoff_elems * es);
+        int64_t id;
+        CHECK(add_dep_wqe(T.g, sg, w, st.arrive[(ch.k + v) % G], -1, &id));
+        st.arrive[(ch.k + v + 1) % G] = id;
+        return HCCL_OK;
+    }
+    const int h = stage - (G - 1);
+    for (int rack = 0; rack < G; ++rack) {
+        const int src = T.rank(rack, ch.j + h), dst = T.rank(rack, ch.j + h + 1);
+        w.a = ref(HCCL_BUF_RECV, src, yoff_elems * es);
+        w.dst = ref(HCCL_BUF_RECV, dst, yoff_elems * es);
+        int64_t id;
+        CHECK(add_dep_wqe(T.g, sg, w, h == 0 ? st.arrive[rack] : st.last[rack], -1, &id));
+        st.last[rack] = id;
+    }
+    return HCCL_OK;
+}
+
+hccl_status_t emit_allreduce_2level(const TwoLevel& T, const std::vector<Chain2>& chains) {
+    const int G = T.G, L = T.L, dt = T.dt, es = T.es;
+    const int64_t Pbytes = T.n * 4;                 // one FP32 image of the buffer per rack, then the accumulator
+    auto P = [&](int rack, int64_t e) { return ref(HCCL_BUF_SCRATCH, 0, (int64_t)rack * Pbytes + e * 4); };
+    auto Q = [&](int64_t e) { return ref(HCCL_BUF_SCRATCH, 0, (int64_t)G * Pbytes + e * 4); };
+    const size_t nch = chains.size(), group = (size_t)T.o.chain_group;
+    std::vector<int32_t> sg(nch);
+    std::vector<std::vector<int64_t>> p_last(nch, std::vector<int64_t>(G, -1));  // last in-rack reduce per rack
+    std::vector<int64_t> q_last(nch, -1);
+    std::vector<GatherState> gs(nch);
+    for (size_t i = 0; i < nch; ++i) {
+        CHECK(hccl_graph_add_subgraph(T.g, T.rank(chains[i].k, chains[i].j), &sg[i]));
+        gs[i].arrive.assign(G, -1);
+        gs[i].last.assign(G, -1);
+    }
+    const int stages = (L - 1) + (G - 1) + (G - 1) + (L - 1);
+    for (size_t g0 = 0; g0 < nch; g0 += group) {
+        const size_t g1 = std::min(nch, g0 + group);
+        for (int stage = 0; stage < stages; ++stage) {
+            for (size_t i = g0; i < g1; ++i) {
+                const Chain2& ch = chains[i];
+                if (stage < L - 1) {
+                    // sums round each rack's ring: local rank (j+t+2) adds its own data to the rack's partial
+                    const int t = stage;
+                    for (int rack = 0; rack < G; ++rack) {
+                        const int l = (ch.j + t + 2) % L, r = T.rank(rack, l), pr = T.rank(rack, l - 1);
+                        hccl_wqe_t w = blank();
+                        w.op = HCCL_OP_REDUCE;
+                        w.count = ch.len;
+                        w.tile_count = T.tile_elems;
+                        w.dtype_dst = HCCL_FP32;
+                        w.dst = P(rack, ch.e0);
+                        w.dtype_b = dt;
+                        w.b = ref(HCCL_BUF_SEND, r, ch.e0 * es);
+                        if (t == 0) { w.dtype_a = dt; w.a = ref(HCCL_BUF_SEND, pr, ch.e0 * es); }
+                        else { w.dtype_a = HCCL_FP32; w.a = P(rack, ch.e0); }
+                        CHECK(add_dep_wqe(T.g, sg[i], w, p_last[i][rack], -1, &p_last[i][rack]));
+                    }
+                } else if (stage < (L - 1) + (G - 1)) {
+                    // sums round the ring of racks: rack (k+u+2) adds its partial
+                    const int u = stage - (L - 1);
+                    const int rk = (ch.k + u + 2) % G, prk = (rk + G - 1) % G;
+                    const bool first = u == 0, final = u == G - 2;
+                    hccl_wqe_t w = blank();
+                    w.op = HCCL_OP_REDUCE;
+                    w.count = ch.len;
+                    w.tile_count = T.tile_elems;
+                    w.dtype_a = w.dtype_b = HCCL_FP32;
+                    w.a = first ? P(prk, ch.e0) : Q(ch.e0);
+                    w.b = P(rk, ch.e0);
+                    if (final) { w.dtype_dst = dt; w.dst = ref(HCCL_BUF_RECV, T.rank(ch.k, ch.j), ch.e0 * es); }
+                    else { w.dtype_dst = HCCL_FP32; w.dst = Q(ch.e0); }
+                    int64_t id;
+                    CHECK(add_dep_wqe(T.g, sg[i], w, first ? p_last[i][prk] : q_last[i], p_last[i][rk], &id));
+                    q_last[i] = id;
+                    if (final) gs[i].arrive[ch.k] = id;
+                } else {
+                    CHECK(emit_gather_stage(T, sg[i], ch, ch.e0, stage - (L - 1) - (G - 1), gs[i]));
+                }
+            }
+        }
+    }
+    return HCCL_OK;
+}
+
+std::vector<Chain2> make_chains2(int G, int L, int64_t n, int64_t granule) {
+    std::vector<Chain2> out;
+    for (int j = 0; j < L; ++j) {
+        const int64_t lo = (int64_t)(((__int128)j * n) / L), hi = (int64_t)(((__int128)(j + 1) * n) / L);
+        for (int k = 0; k < G; ++k) {
+            const int64_t a = lo + (int64_t)(((__int128)k * (hi - lo)) / G), b = lo + (int64_t)(((__int128)(k + 1) * (hi - lo)) / G);
+            for (int64_t e = a; e < b; e += granule) out.push_back(Chain2{j, k, e, std::min(granule, b - e)});
+        }
+    }
+    return out;
+}
+
+hccl_status_t plan_allreduce_2level(int R, int64_t count, hccl_dtype_t dt, const hccl_opts_t& o, hccl_plan_t** out) {
+    const int L = o.rack_size, G = R / L, es = elem_bytes(dt);
+    std::vector<int64_t> ext(R, count * es);
+    const int64_t granule = std::max<int64_t>(1, (int64_t)(o.chunk_bytes / (uint64_t)es));
+    std::vector<Chain2> chains = make_chains2(G, L, count, granule);
+    int64_t maxlen = 0;
+    for (const Chain2& c : chains) maxlen = std::max(maxlen, c.len);
+    hccl_graph* graw = nullptr;
+    CHECK(hccl_graph_create(R, ext.data(), ext.data(), (int64_t)(G + 1) * count * 4, 0, &graw));
+    GraphPtr g(graw);
+    g->compulsory_bytes = 2ll * R * count * es;
+    TwoLevel T{g.get(), G, L, (int)dt, es, count, 0, o};
+    const int64_t level = std::min<int64_t>(count * G, (int64_t)o.chain_group * maxlen * G);
+    T.tile_elems = pick_tile_elems(level, o, 4, HCCL_OP_REDUCE);
+    CHECK(emit_allreduce_2level(T, chains));
+    return hccl_graph_compile(g.get(), &o, out);
+}
+
+
+// Two-level AllGather: rank (g, j)'s block first lands in its own receive buffer, then travels to the other
+// racks' rank j (the only hops between racks), and every rack passes it round its own ring.
+hccl_status_t plan_allgather_2level(int R, const std::vector<int64_t>& offs, hccl_dtype_t dt, const hccl_opts_t& o, hccl_plan_t** out) {
+    const int L = o.rack_size, G = R / L, es = elem_bytes(dt);
+    std::vector<int64_t> sext(R), rext(R, offs[R] * es);
+    for (int r = 0; r < R; ++r) sext[r] = (offs[r + 1] - offs[r]) * es;
+    hccl_graph* graw = nullptr;
+    CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw));
+    GraphPtr g(graw);
+    g->compulsory_bytes = offs[R] * es + (int64_t)R * offs[R] * es;
+    const int64_t granule = std::max<int64_t>(1, (int64_t)(o.chunk_bytes / (uint64_t)es));
+    struct Item { Chain2 ch; int64_t src_off; };
+    std::vector<Item> items;
+    for (int64_t k0 = 0;; ++k0) {  // granule-major, so that consecutive chains start on different ranks
+        bool any = false;
+        for (int q = 0; q < R; ++q) {
+            const int64_t lo = offs[q] + k0 * granule;
+            if (lo >= offs[q + 1]) continue;
+            any = true;
+            items.push_back(Item{Chain2{q % L, q / L, lo, std::min(granule, offs[q + 1] - lo)}, lo - offs[q]});
+        }
+        if (!any) break;
+    }
+    TwoLevel T{g.get(), G, L, (int)dt, es, offs[R], 0, o};
+    T.tile_elems = o.tile_bytes ? std::max<int64_t>(1, (int64_t)(o.tile_bytes / (uint64_t)es))
+                                : default_tile(std::min<int64_t>(offs[R], (int64_t)o.chain_group * granule) * G * es, o.sm_budget, 1, 16 << 10, 256 << 10,
+                                               sweep_of(o, HCCL_OP_COPY)) / es;
+    T.tile_elems = std::max<int64_t>(T.tile_elems, 1);
+    const size_t nch = items.size(), group = (size_t)o.chain_group;
+    std::vector<int32_t> sg(nch);
+    std::vector<GatherState> gs(nch);
+    for (size_t i = 0; i < nch; ++i) {
+        CHECK(hccl_graph_add_subgraph(g.get(), T.rank(items[i].ch.k, items[i].ch.j), &sg[i]));
+        gs[i].arrive.assign(G, -1);
+        gs[i].last.assign(G, -1);
+    }
+    const int stages = 1 + (G - 1) + (L - 1);
+    for (size_t g0 = 0; g0 < nch; g0 += group) {
+        const size_t g1 = std::min(nch, g0 + group);
+        for (int stage = 0; stage < stages; ++stage) {
+            for (size_t i = g0; i < g1; ++i) {
+                const Chain2& ch = items[i].ch;
+                if (stage == 0) {
+                    hccl_wqe_t w = blank();
+                    w.op = HCCL_OP_COPY;
+                    w.count = ch.len * es;
+                    w.tile_count = T.tile_elems * es;
+                    const int r = T.rank(ch.k, ch.j);
+                    w.a = ref(HCCL_BUF_SEND, r, items[i].src_off * es);
+                    w.dst = ref(HCCL_BUF_RECV, r, ch.e0 * es);
+                    CHECK(hccl_graph_add_wqe(g.get(), sg[i], &w, &gs[i].arrive[ch.k]));
+                } else {
+                    CHECK(emit_gather_stage(T, sg[i], ch, ch.e0, stage - 1, gs[i]));
+                }
+            }
+        }
+    }
+    return hccl_graph_compile(g.get(), &o, out);
+}
+
 }  // namespace
 
 extern "C" {
@@ -193,9 +421,15 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
                                   hccl_plan_t** out) {
     if (!out || R < 1 || R > HCCL_MAX_RANKS || count < 0) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
-    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_FUSED) return HCCL_ERR_INVALID_ARG;
+    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_RING_2LEVEL) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
     fill_default_opts(&o, opts);
+    if (algo == HCCL_ALGO_RING_2LEVEL) {
+        if (R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
+        // a single rack, or racks of one rank, is the flat ring
+        if (o.rack_size >= 2 && R / o.rack_size >= 2) return plan_allreduce_2level(R, count, dt, o, out);
+        algo = HCCL_ALGO_RING;
+    }
     const int es = elem_bytes(dt);
     std::vector<int64_t> ext(R, count * es);
     const int64_t compulsory = 2ll * R * count * es;
@@ -316,7 +550,7 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
                                   const hccl_opts_t* opts, hccl_plan_t** out) {
     if (!out || R < 1 || R > HCCL_MAX_RANKS || count < 0) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
-    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT) return HCCL_ERR_INVALID_ARG;
+    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_2LEVEL) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
     fill_copy_opts(&o, opts);
     const int es = elem_bytes(dt);
@@ -326,6 +560,11 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
         if (c < 0) return HCCL_ERR_INVALID_ARG;
         offs[r + 1] = offs[r] + c;
         sext[r] = c * es;
+    }
+    if (algo == HCCL_ALGO_RING_2LEVEL) {
+        if (R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
+        if (o.rack_size >= 2 && R / o.rack_size >= 2) return plan_allgather_2level(R, offs, dt, o, out);
+        algo = HCCL_ALGO_RING;
     }
     for (int r = 0; r < R; ++r) rext[r] = offs[R] * es;
     hccl_graph* graw = nullptr;

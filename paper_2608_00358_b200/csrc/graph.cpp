@@ -73,6 +73,7 @@ void hccl::fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in) {
     if (o->chunk_bytes == 0) o->chunk_bytes = 2u << 20;
     if (o->timeout_ns == 0) o->timeout_ns = 2000000000ull;
     if (o->chain_group <= 0) o->chain_group = 16;
+    if (o->rack_size <= 0) o->rack_size = 16;
     if (o->threads <= 0) o->threads = o->engine == HCCL_ENGINE_BULK ? 288 : 512;  // bulk: DMA warp + 8 compute warps; register: control warp + 15 workers
     o->threads = std::min(512, std::max(64, (o->threads + 31) / 32 * 32));  // one control warp + at least one worker warp
 }
@@ -225,7 +226,9 @@ hccl_status_t hccl_graph_add_wqe(hccl_graph_t* g, int32_t subgraph, const hccl_w
             push_unique(q.preds_elem, w.dep_wqe);
         else
             push_unique(q.preds_full, w.dep_wqe);
-        if (w.dep_wqe2 >= 0) push_unique(q.preds_full, w.dep_wqe2);
+        if (w.dep_wqe2 >= 0) {
+            if (w.dep_flags & HCCL_DEP_ELEMENTWISE2) push_unique(q.preds_elem, w.dep_wqe2); else push_unique(q.preds_full, w.dep_wqe2);
+        }
     }
     // a predecessor listed both ways is waited for entirely
     for (int64_t p : q.preds_full) {
@@ -280,9 +283,25 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         if (w.op == HCCL_OP_REDUCE_N) return std::max(elem_bytes(w.dtype_dst), elem_bytes(w.dtype_a));
         return 0;
     };
-    int64_t schedule = 0, weight = 0;
+    int64_t schedule = 0, weight = 0, crossrack = 0;
+    const int rack = std::max(1, p->opts.rack_size);
+    auto remote = [&](const hccl_ref_t& src, const hccl_ref_t& dst) {
+        const bool s_rank = src.kind == HCCL_BUF_SEND || src.kind == HCCL_BUF_RECV, d_rank = dst.kind == HCCL_BUF_RECV;
+        return s_rank && d_rank && src.rank / rack != dst.rank / rack;
+    };
     for (const Wqe& q : g->wqes) {
         const hccl_wqe_t& w = q.w;
+        if (w.op == HCCL_OP_COPY && remote(w.a, w.dst)) crossrack += w.count;
+        if (w.op == HCCL_OP_REDUCE) {
+            if (remote(w.a, w.dst)) crossrack += w.count * elem_bytes(w.dtype_a);
+            if (remote(w.b, w.dst)) crossrack += w.count * elem_bytes(w.dtype_b);
+        }
+        if (w.op == HCCL_OP_REDUCE_N)
+            for (int k = 0; k < w.nsrc; ++k) {
+                hccl_ref_t sr = w.a;
+                sr.rank = (w.a.rank + k) % g->R;
+                if (remote(sr, w.dst)) crossrack += w.count * elem_bytes(w.dtype_a);
+            }
         if (w.op == HCCL_OP_COPY) schedule += 2 * w.count;
         if (w.op == HCCL_OP_REDUCE) schedule += w.count * (elem_bytes(w.dtype_a) + elem_bytes(w.dtype_b) + elem_bytes(w.dtype_dst));
         if (w.op == HCCL_OP_REDUCE_N) schedule += w.count * ((int64_t)w.nsrc * elem_bytes(w.dtype_a) + elem_bytes(w.dtype_dst));
@@ -436,6 +455,7 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
     I.threads = p->opts.threads;
     I.engine = p->opts.engine;
     I.tile_bytes = (int64_t)tile_bytes;
+    I.crossrack_bytes = crossrack;
     *out = p;
     return HCCL_OK;
 }

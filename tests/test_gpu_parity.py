@@ -185,3 +185,31 @@ def test_overlapping_send_and_receive_is_rejected():
     with pytest.raises(hb.HcclError) as e:
         dc.execute()
     assert e.value.status == hb.ERR_OVERLAP
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("G,L,n", [(2, 2, 37), (4, 4, 40099), (4, 16, 100003), (3, 5, 257)])
+def test_two_level_allreduce(G, L, n, dt, engine):
+    R = G * L
+    X = synth.normal_ranks(R, n, dt, seed=G * 7 + L)
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING_2LEVEL, _with(dict(rack_size=L, tile_bytes=2048, chunk_bytes=8192, chain_group=4, sm_budget=32), engine))
+    Y = run_plan(p, X, iters=2)
+    bitwise, exact, want = orc.allreduce_ring2_f32(dt, X, G, L), orc.sum_f64(dt, X), orc.allreduce(dt, X)
+    for r in range(R):
+        got = Y[r].view(np_dtype(dt))
+        assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8)), "rank %d" % r
+        assert_reduction_close(dt, got, exact, want[r], X=X)      # 64 ranks in FP32: see the rule's docstring
+
+
+@pytest.mark.parametrize("G,L", [(2, 2), (4, 4), (8, 16)])
+def test_two_level_allgather(G, L, engine):
+    R = G * L
+    rng = np.random.default_rng(G * 100 + L)
+    cs = [int(c) for c in rng.integers(0, 3000, size=R)]
+    cs[1] = 0
+    X = [rng.integers(0, 65536, size=c, dtype=np.uint16) for c in cs]
+    p = hb.hccl_plan_allgather(R, cs, 0, hb.BF16, hb.ALGO_RING_2LEVEL, _with(dict(rack_size=L, tile_bytes=1024, chunk_bytes=2048, sm_budget=32), engine))
+    Y = run_plan(p, X, iters=2)
+    want = orc.allgatherv(X)
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np.uint16), want[r])

@@ -349,3 +349,40 @@ def test_config_count_draws():
     assert C.shape == (8, 8) and C.min() >= 0 and C.max() <= 4096
     Z = synth.zipf_counts(64, 0)
     assert Z.min() >= 1 and Z.max() == 32768
+
+
+# ------------------------------------------------------------- two-level ring order
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("G,L", [(2, 2), (2, 3), (4, 4), (3, 5), (1, 4), (4, 1)])
+def test_two_level_ring_order(G, L, dt):
+    R, n = G * L, 211
+    # exactly summable data: the order cannot matter, the result must be the plain sum on every rank
+    X = synth.small_int_ranks(R, n, dt, seed=G * 10 + L)
+    want = orc.allreduce(dt, X)
+    Y = orc.allreduce_ring2_f32(dt, X, G, L)
+    for r in range(R):
+        assert np.array_equal(Y[r], want[r])
+    # random data: within the acceptance rule of the FP64 definition
+    X = synth.normal_ranks(R, n, dt, seed=G * 100 + L)
+    Y, want, s = orc.allreduce_ring2_f32(dt, X, G, L), orc.allreduce(dt, X), orc.sum_f64(dt, X)
+    if dt == FP32:
+        assert np.all(np.abs(Y[0].astype(np.float64) - s) <= 1e-5 * np.abs(s) + 1e-6)
+    else:
+        assert orc.ulp_distance(dt, Y[0], want[0]).max() <= 1
+    # with a single rack, or racks of one rank, it is the flat ring
+    if G == 1:
+        assert np.array_equal(Y[0], orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, L))[0])
+
+
+def test_two_level_order_is_racks_first():
+    # G = 2 racks of L = 2, one element per sub-chunk; values make the FP32 result depend on the grouping.
+    big, one = np.float32(2.0 ** 24), np.float32(1.0)
+    # sub-chunk (j, k): racks' partials P_g = X_{g,j+1} + X_{g,j}, total = P_{k+1} + P_k
+    # element 0 is (j=0,k=0): P_0 = X[1] + X[0], P_1 = X[3] + X[2], total = P_1 + P_0
+    X = [np.full(4, v, dtype=np.float32) for v in (big, one, -big, one)]     # ranks (0,0) (0,1) (1,0) (1,1)
+    Y = orc.allreduce_ring2_f32(FP32, X, 2, 2)
+    # racks first: (1 + 2^24) -> 2^24 and (1 - 2^24) -> -2^24 + 1 exactly; total = 1
+    assert np.all(Y[0] == 1.0)
+    # the flat ring adds rank by rank and loses nothing different here? (X1 + X2) + X3 + X0 = ((1 - 2^24) + 1) + 2^24 = 2
+    assert orc.allreduce_ring_f32(FP32, X, [0, 1, 2, 3, 4])[0][0] == 2.0
+    assert orc.allreduce(FP32, X)[0][0] == 2.0

@@ -198,3 +198,58 @@ def test_all_zero_counts_is_an_empty_plan():
     p = hb.hccl_plan_alltoallv(3, np.zeros((3, 3), dtype=np.int64), None, None, None, hb.BF16, 128)
     assert p.info().n_tiles == 0 and p.info().schedule_bytes == 0
     assert interpret(p, [np.zeros(1, dtype=np.uint8)] * 3) is not None
+
+
+# ------------------------------------------------------------------ two-level (rack-aware) schedules
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("G,L,n", [(2, 2, 37), (2, 3, 1000), (4, 4, 4099), (3, 5, 257), (2, 2, 3), (2, 2, 0)])
+def test_two_level_allreduce_matches_oracle(G, L, n, dt):
+    R = G * L
+    X = synth.normal_ranks(R, n, dt, seed=G * 7 + L)
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING_2LEVEL, dict(SMALL, rack_size=L, chunk_bytes=512, chain_group=3))
+    assert p.check_hazards() == 0
+    bitwise = orc.allreduce_ring2_f32(dt, X, G, L)
+    exact, want = orc.sum_f64(dt, X), orc.allreduce(dt, X)
+    for seed in (0, 1, 2):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            got = Y[r].view(np_dtype(dt))
+            assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8))
+            assert_reduction_close(dt, got, exact, want[r])
+    # fewer dependent steps than the flat ring, and fewer bytes between racks
+    flat = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, dict(SMALL, rack_size=L)).info()
+    i = p.info()
+    if n >= R:
+        assert i.chain_depth == 2 * (L - 1) + 2 * (G - 1) < flat.chain_depth
+        assert i.crossrack_bytes < flat.crossrack_bytes
+
+
+def test_two_level_degenerates_to_the_flat_ring():
+    X = synth.normal_ranks(4, 100, hb.BF16, seed=1)
+    want = orc.allreduce_ring_f32(hb.BF16, X, orc.floor_chunk_offsets(100, 4))
+    for rack in (1, 4):
+        p = hb.hccl_plan_allreduce(4, 100, hb.BF16, hb.ALGO_RING_2LEVEL, dict(SMALL, rack_size=rack))
+        Y = interpret(p, X)
+        assert np.array_equal(Y[0].view(np.uint16), want[0])
+    with pytest.raises(hb.HcclError) as e:
+        hb.hccl_plan_allreduce(6, 100, hb.BF16, hb.ALGO_RING_2LEVEL, dict(rack_size=4))
+    assert e.value.status == hb.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("G,L", [(2, 2), (2, 3), (4, 4), (8, 16)])
+def test_two_level_allgather_matches_oracle(G, L):
+    R = G * L
+    rng = np.random.default_rng(G * 100 + L)
+    cs = [int(c) for c in rng.integers(0, 200, size=R)]
+    cs[0] = 0
+    X = [rng.integers(0, 65536, size=c, dtype=np.uint16) for c in cs]
+    p = hb.hccl_plan_allgather(R, cs, 0, hb.BF16, hb.ALGO_RING_2LEVEL, dict(SMALL, rack_size=L, tile_bytes=64, chunk_bytes=128, chain_group=3))
+    assert p.check_hazards() == 0
+    want = orc.allgatherv(X)
+    for seed in (0, 3):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            assert np.array_equal(Y[r].view(np.uint16), want[r])
+    flat = hb.hccl_plan_allgather(R, cs, 0, hb.BF16, hb.ALGO_RING, dict(SMALL, rack_size=L)).info()
+    assert p.info().chain_depth == 1 + (G - 1) + (L - 1) <= flat.chain_depth
+    assert p.info().crossrack_bytes < flat.crossrack_bytes
