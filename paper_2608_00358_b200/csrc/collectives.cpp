@@ -427,6 +427,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     if (algo == HCCL_ALGO_RING_2LEVEL) {
         if (R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
         // a single rack, or racks of one rank, is the flat ring
+        if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = 1 << 20;  // all chains together
         if (o.rack_size >= 2 && R / o.rack_size >= 2) return plan_allreduce_2level(R, count, dt, o, out);
         algo = HCCL_ALGO_RING;
     }
@@ -468,6 +469,9 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     std::vector<Chain> chains = make_chains(R, offs, false, granule);
     int64_t maxlen = 0;
     for (const Chain& ch : chains) maxlen = std::max(maxlen, ch.len);
+    // small buffers (all FP32 partials fit the L2 several times over): run every chain together, the
+    // dependency chain is then as short as the ring allows; large ones keep chain groups for L2 residency
+    if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
     const bool need_scratch = !in_recv && !fused && R > 2;
     const bool staged = (o.flags & HCCL_FLAG_STAGED_RING) != 0 && need_scratch;
     // level-major order runs every chain's step t before any step t+1, so no slot can be recycled
@@ -530,6 +534,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     std::vector<Chain> chains = make_chains(R, offs, true, granule);
     int64_t maxlen = 0;
     for (const Chain& ch : chains) maxlen = std::max(maxlen, ch.len);
+    if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
     const bool need_scratch = !fused && R > 2;
     const bool staged = (o.flags & HCCL_FLAG_STAGED_RING) != 0 && need_scratch;
     // level-major order runs every chain's step t before any step t+1, so no slot can be recycled
