@@ -174,8 +174,34 @@ def side_configs(quick: bool):
     latency(wk.config2(), "2_alltoallv_r8_bf16_dim128")
     for m in (4096, 65536, 262144, 1 << 20):
         for algo, nm in ((hb.ALGO_ONESHOT, "oneshot"), (hb.ALGO_RING, "ring")):
-            latency(wk.config5(m, algo), "5_allreduce_r8_bf16_%dB_%s" % (m, nm))
+            wl5 = wk.config5(m, algo)
+            key5 = "5_allreduce_r8_bf16_%dB_%s" % (m, nm)
+            latency(wl5, key5)
+            if algo == hb.ALGO_ONESHOT:
+                out[key5]["host_observed"] = wk.time_host_observed(wl5, 100 if quick else 300)
     torch.cuda.empty_cache()
+    # beyond the five configurations: schedules at rack scale (64 ranks = 4 racks of 16; 128 ranks = 8 racks)
+    def sched(name, plan, send, recv, iters):
+        wl = wk._bind(name, plan, send, recv, {})
+        ms = wk.time_back_to_back(wl, iters, 3)
+        i = wl.info
+        out[name] = {"ms": float(ms), "chain_depth": int(i.chain_depth), "tiles": int(i.n_tiles), "schedule_bytes": int(i.schedule_bytes),
+                     "compulsory_bytes": int(i.compulsory_bytes), "crossrack_bytes_racks_of_16": int(i.crossrack_bytes),
+                     "compulsory_gbs": i.compulsory_bytes / ms / 1e6}
+    for n in ((1 << 16, 1 << 22) if quick else (1 << 16, 1 << 22, 1 << 25)):
+        send = [torch.randn(n, device="cuda").to(torch.bfloat16) for _ in range(64)]
+        recv = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(64)]
+        for algo, nm in ((hb.ALGO_RING, "ring"), (hb.ALGO_RING_2LEVEL, "ring_2level"), (hb.ALGO_RING_FUSED, "ring_fused")):
+            sched("next_allreduce_r64_bf16_%d_%s" % (n, nm), hb.hccl_plan_allreduce(64, n, hb.BF16, algo, dict(rack_size=16)), send, recv, 20)
+        del send, recv
+        torch.cuda.empty_cache()
+    for n in ((1 << 12, 1 << 18) if quick else (1 << 12, 1 << 18, 1 << 21)):
+        send = [torch.randn(n, device="cuda").to(torch.bfloat16) for _ in range(128)]
+        recv = [torch.empty(n * 128, dtype=torch.bfloat16, device="cuda") for _ in range(128)]
+        for algo, nm in ((hb.ALGO_RING, "ring"), (hb.ALGO_RING_2LEVEL, "ring_2level"), (hb.ALGO_ONESHOT, "oneshot")):
+            sched("next_allgather_r128_bf16_%d_%s" % (n, nm), hb.hccl_plan_allgather(128, None, n, hb.BF16, algo, dict(rack_size=16)), send, recv, 10)
+        del send, recv
+        torch.cuda.empty_cache()
     for algo, nm in ((hb.ALGO_RING, "ring"), (hb.ALGO_RING_FUSED, "ring_fused")):
         wl = wk.config3(algo=algo)
         ms = wk.time_back_to_back(wl, 10 if quick else 50, 5)

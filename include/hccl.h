@@ -301,6 +301,26 @@ hccl_status_t hccl_execute_noalloc(hccl_plan_t*, const void* const* sendbufs, vo
 hccl_status_t hccl_execute_host(hccl_plan_t*, const void* const* host_send, void* const* host_recv,
                                 void* const* dev_send, void* const* dev_recv, void* stream);
 
+/* Resident, doorbell-fed execution (the express-doorbell idea of Sec. II-A.3 and the cached re-enqueue of
+ * Sec. V-B, without any launch per collective). hccl_server_start launches the register engine ONCE as a
+ * long-lived kernel bound to this plan and these buffers; afterwards hccl_server_ring is a single store
+ * into the doorbell record and costs no CUDA call, the resident blocks execute the plan once per ring, and
+ * hccl_server_wait spins (on the host) until the record says so. host_doorbell points to 64 bytes of
+ * pinned, MAPPED host memory owned by the caller (cudaHostAlloc with cudaHostAllocMapped, or torch pinned
+ * memory), 64-byte aligned; it must stay valid until the kernel has left. All blocks must be resident at
+ * once (sm_budget blocks of opts.threads threads; HCCL_ERR_INVALID_ARG otherwise). The kernel leaves by
+ * itself when no ring arrives for idle_timeout_ns (default 100 ms; then hccl_server_ring returns
+ * HCCL_ERR_TIMEOUT and the server can be started again), after hccl_server_stop, or after a failed
+ * execution (whose verdict hccl_server_ring / hccl_server_wait then return). While the server runs, use
+ * only these calls on the plan, and do not synchronise the whole device: the kernel occupies `stream` until
+ * it leaves. Rings are served in order; ring again only after the previous ring was waited for. */
+typedef struct { uint64_t request, completed, stop, exited, status, detail, pad[2]; } hccl_doorbell_t;
+hccl_status_t hccl_server_start(hccl_plan_t*, const void* const* sendbufs, void* const* recvbufs, void* host_doorbell,
+                                uint64_t idle_timeout_ns, void* stream);
+hccl_status_t hccl_server_ring(hccl_plan_t*);
+hccl_status_t hccl_server_wait(hccl_plan_t*, uint64_t timeout_ns);
+hccl_status_t hccl_server_stop(hccl_plan_t*);
+
 /* Device-triggered execution (Sec. IV-B.3): give the plan a caller-owned device array of uint64 that
  * HCCL_BUF_USER_SIGNAL refs index; hccl_plan_set_trigger makes every execution (a) hold all work until
  * user signal slot wait_slot satisfies cmp against wait_value + epoch*wait_per_epoch, and (b) store

@@ -84,6 +84,10 @@ def _load() -> C.CDLL:
         "hccl_execute": [P, C.POINTER(P), C.POINTER(P), P],
         "hccl_execute_host": [P, C.POINTER(P), C.POINTER(P), C.POINTER(P), C.POINTER(P), P],
         "hccl_execute_noalloc": [P, C.POINTER(P), C.POINTER(P), P],
+        "hccl_server_start": [P, C.POINTER(P), C.POINTER(P), P, C.c_uint64, P],
+        "hccl_server_ring": [P],
+        "hccl_server_wait": [P, C.c_uint64],
+        "hccl_server_stop": [P],
         "hccl_plan_set_user_signals": [P, P, C.c_int64],
         "hccl_plan_set_trigger": [P, C.c_int64, C.c_int32, C.c_uint64, C.c_uint64, C.c_int64, C.c_uint64, C.c_uint64],
         "hccl_plan_status": [P, C.POINTER(C.c_int), I64P],
@@ -116,7 +120,7 @@ EXPORTS = ["hccl_plan_allreduce", "hccl_plan_reducescatter", "hccl_plan_allgathe
            "hccl_plan_alltoallv_dynamic", "hccl_plan_set_dynamic_metadata",
            "hccl_graph_create", "hccl_graph_add_subgraph", "hccl_graph_add_wqe", "hccl_graph_compile",
            "hccl_graph_destroy", "hccl_plan_workspace_bytes", "hccl_plan_bind", "hccl_execute", "hccl_execute_host",
-           "hccl_execute_noalloc",
+           "hccl_execute_noalloc", "hccl_server_start", "hccl_server_ring", "hccl_server_wait", "hccl_server_stop",
            "hccl_plan_set_user_signals", "hccl_plan_set_trigger", "hccl_plan_status", "hccl_plan_info",
            "hccl_plan_extents", "hccl_plan_layout", "hccl_plan_destroy", "hccl_status_string", "hccl_last_cuda_error", "hccl_version",
            "hccl_plan_check_hazards", "hccl_plan_interpret_host"]
@@ -206,6 +210,20 @@ class Plan:
         allocate device memory). Raises HcclError with the device-side verdict if it failed."""
         _chk(_lib.hccl_execute_noalloc(self._h, _ptr_array(sendbufs), _ptr_array(recvbufs), C.c_void_p(stream)),
              "hccl_execute_noalloc")
+
+    def server_start(self, sendbufs: Sequence[int], recvbufs: Sequence[int], host_doorbell: int, idle_timeout_ns: int = 0,
+                     stream: int = 0):
+        _chk(_lib.hccl_server_start(self._h, _ptr_array(sendbufs), _ptr_array(recvbufs), C.c_void_p(host_doorbell),
+                                    idle_timeout_ns, C.c_void_p(stream)), "hccl_server_start")
+
+    def server_ring(self) -> int:
+        return _lib.hccl_server_ring(self._h)
+
+    def server_wait(self, timeout_ns: int = 0) -> int:
+        return _lib.hccl_server_wait(self._h, timeout_ns)
+
+    def server_stop(self):
+        _chk(_lib.hccl_server_stop(self._h), "hccl_server_stop")
 
     def set_dynamic_metadata(self, dev_sendcounts: int, dev_recvcounts_out: int = 0, dev_rdispls_out: int = 0):
         _chk(_lib.hccl_plan_set_dynamic_metadata(self._h, C.c_void_p(dev_sendcounts), C.c_void_p(dev_recvcounts_out or None),

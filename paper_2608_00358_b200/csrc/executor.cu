@@ -16,6 +16,9 @@
 #include <cuda_runtime.h>
 
 #include <cstdio>
+#include <atomic>
+#include <chrono>
+#include <cstddef>
 #include <cstring>
 #include <mutex>
 #include <type_traits>
@@ -1202,6 +1205,88 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
 }
 
 
+// ====================================================================== resident, doorbell-fed executor
+// The register engine as a long-lived kernel (paper Sec. II-A.3 "express doorbells": the work request's
+// write is the doorbell; Sec. V-B: re-enqueueing a cached work packet costs microseconds). The blocks stay
+// resident and execute the bound plan once per doorbell ring. The doorbell is a 64-byte record in pinned,
+// mapped HOST memory: the host rings by storing a larger request number, block 0 polls it, releases all
+// blocks through a device-side word, and reports completion (and a failure verdict) back into the record.
+// Every wait is bounded: the kernel leaves by itself after idle_ns without a ring, or when told to stop.
+struct Doorbell {                       // layout shared with hccl_doorbell_t in hccl.h
+    unsigned long long request;         // host -> device: number of executions asked for so far
+    unsigned long long completed;       // device -> host: executions finished
+    unsigned long long stop;            // host -> device: leave after the current execution
+    unsigned long long exited;          // device -> host: the kernel has left (1 = stop, 2 = idle, 3 = failure)
+    unsigned long long status, detail;  // device -> host: verdict of the last failed execution
+    unsigned long long pad[2];
+};
+
+__device__ __forceinline__ unsigned long long ld_sys_u64(const unsigned long long* p) {
+    unsigned long long v;
+    asm volatile("ld.relaxed.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_sys_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.release.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+__global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_constant__ ExecParams p, Doorbell* db,
+                                                                  const unsigned long long idle_ns, const uint32_t first_epoch) {
+    __shared__ uint32_t s_cmd;          // epoch to run, or 0 to leave
+    uint32_t epoch = first_epoch;       // the next execution's number
+    for (;;) {
+        if (threadIdx.x == 0) {
+            uint32_t cmd = 0;
+            if (blockIdx.x == 0) {
+                // the previous execution must have been left by every block before anything else happens
+                bool ok = true;
+                if (epoch != first_epoch) {
+                    const unsigned long long deadline = globaltimer_ns() + 2 * p.timeout_ns + 1000000000ull;
+                    while (ld_acquire_u32(&p.ctl->done_epoch) != epoch - 1) {
+                        if (globaltimer_ns() > deadline) { ok = false; break; }
+                        __nanosleep(50);
+                    }
+                    if (ok) {
+                        if (ld_acquire_u32(&p.ctl->fail_epoch) == epoch - 1) {
+                            st_sys_u64(&db->status, p.ctl->status);
+                            st_sys_u64(&db->detail, p.ctl->detail);
+                            ok = false;  // a failed execution leaves the counters inconsistent: stop serving
+                        }
+                        st_sys_u64(&db->completed, (unsigned long long)(epoch - first_epoch));
+                    }
+                }
+                unsigned long long why = ok ? 0 : 3;
+                if (ok) {
+                    const unsigned long long deadline = globaltimer_ns() + idle_ns;
+                    for (;;) {
+                        if (ld_sys_u64(&db->request) > (unsigned long long)(epoch - first_epoch)) { cmd = epoch; break; }
+                        if (ld_sys_u64(&db->stop) != 0) { why = 1; break; }
+                        if (globaltimer_ns() > deadline) { why = 2; break; }
+                        __nanosleep(100);
+                    }
+                }
+                if (cmd == 0) st_sys_u64(&db->exited, why);
+                // release the other blocks: server_go carries the epoch to run, or all ones to leave
+                asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&p.ctl->server_go), "r"(cmd ? cmd : 0xffffffffu) : "memory");
+            } else {
+                const unsigned long long deadline = globaltimer_ns() + idle_ns + 4 * p.timeout_ns + 4000000000ull;
+                for (;;) {
+                    const uint32_t go = ld_acquire_u32(&p.ctl->server_go);
+                    if (go == epoch) { cmd = epoch; break; }
+                    if (go == 0xffffffffu || globaltimer_ns() > deadline) break;
+                    __nanosleep(50);
+                }
+            }
+            s_cmd = cmd;
+        }
+        __syncthreads();
+        if (s_cmd == 0) break;
+        executor_lsu_body(p);           // one execution: tickets, dependencies, data, completion stamp
+        __syncthreads();
+        ++epoch;
+    }
+}
+
 // ====================================================================== device-resident AllToAllv
 // "AllToAllvDynamic" (paper Sec. IV-B.2): the per-peer row counts are produced on the device (by a routing
 // kernel) after the collective has been compiled and possibly already enqueued. The kernel reads the R x R
@@ -1581,6 +1666,111 @@ hccl_status_t hccl_plan_status(hccl_plan_t* p, hccl_status_t* device_status, int
     if (c.exits != 0) return HCCL_ERR_BUSY;  // blocks of an execution are still leaving: synchronise first
     *device_status = HCCL_OK;
     if (detail) *detail = (int64_t)c.done_epoch;
+    return HCCL_OK;
+}
+
+}  // extern "C"
+
+// ====================================================================== resident executor: host side
+extern "C" {
+
+hccl_status_t hccl_server_start(hccl_plan_t* p, const void* const* sendbufs, void* const* recvbufs, void* host_doorbell,
+                                uint64_t idle_timeout_ns, void* stream) {
+    if (!p || !sendbufs || !recvbufs || !host_doorbell) return HCCL_ERR_INVALID_ARG;
+    if (!p->workspace) return HCCL_ERR_NOT_BOUND;
+    if (p->dynamic || p->server_db) return HCCL_ERR_INVALID_ARG;
+    if (((uintptr_t)host_doorbell) % 64) return HCCL_ERR_ALIGNMENT;
+    hccl_status_t st = check_buffers(p, sendbufs, recvbufs);
+    if (st != HCCL_OK) return st;
+    void* dev_db = nullptr;
+    CUDA_TRY(cudaHostGetDevicePointer(&dev_db, host_doorbell, 0));  // fails unless the record is pinned, mapped memory
+    cudaStream_t s = (cudaStream_t)stream;
+    Control c;
+    CUDA_TRY(cudaStreamSynchronize(s));
+    CUDA_TRY(cudaMemcpy(&c, (char*)p->workspace + p->layout.control, sizeof(c), cudaMemcpyDeviceToHost));
+    CUDA_TRY(cudaMemsetAsync((char*)p->workspace + p->layout.control + offsetof(Control, server_go), 0, 4, s));
+    std::memset(host_doorbell, 0, sizeof(Doorbell));
+    static thread_local ExecParams prm;
+    char* ws = (char*)p->workspace;
+    const Layout& L = p->layout;
+    prm.descs = (const Desc*)(ws + L.descs);
+    prm.tiles = (const Tile*)(ws + L.tiles);
+    prm.waits = (const Wait*)(ws + L.waits);
+    prm.counters = (uint32_t*)(ws + L.counters);
+    prm.signals = (unsigned long long*)(ws + L.signals);
+    prm.ctl = (Control*)(ws + L.control);
+    prm.scratch = ws + L.scratch;
+    prm.user_signals = (unsigned long long*)p->user_signals;
+    prm.n_tiles = (uint32_t)p->tiles.size();
+    prm.n_descs = (uint32_t)p->descs.size();
+    prm.n_syncs = (uint32_t)p->sync_per_epoch.size();
+    prm.n_waits = (uint32_t)p->waits.size();
+    prm.n_signals = (uint32_t)p->n_signals;
+    prm.R = (uint32_t)p->R;
+    prm.timeout_ns = p->opts.timeout_ns;
+    prm.n_user_signals = p->n_user_signals;
+    prm.trig_wait_slot = p->trig_wait_slot;
+    prm.trig_set_slot = p->trig_set_slot;
+    prm.trig_cmp = p->trig_cmp;
+    prm.trig_wait_value = p->trig_wait_value;
+    prm.trig_wait_per_epoch = p->trig_wait_per_epoch;
+    prm.trig_set_value = p->trig_set_value;
+    prm.trig_set_per_epoch = p->trig_set_per_epoch;
+    for (int r = 0; r < p->R; ++r) {
+        prm.send[r] = sendbufs[r];
+        prm.recv[r] = recvbufs[r];
+    }
+    int blocks = p->opts.sm_budget;
+    if ((uint32_t)blocks > prm.n_tiles) blocks = (int)std::max<uint32_t>(prm.n_tiles, 1u);
+    prm.nblocks = (uint32_t)blocks;
+    prm.static_tickets = (prm.n_waits == 0 && prm.n_tiles <= (uint32_t)blocks) ? 1 : 0;
+    // every block must be resident at once (the blocks wait for each other between executions)
+    int dev = 0, sms = 0, per_sm = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, hccl_executor_resident, p->opts.threads, 0));
+    if (blocks > sms * per_sm) return HCCL_ERR_INVALID_ARG;
+    Doorbell* db = (Doorbell*)dev_db;
+    unsigned long long idle = idle_timeout_ns ? idle_timeout_ns : 100000000ull;
+    uint32_t first_epoch = c.done_epoch + 1;
+    void* args[] = {(void*)&prm, (void*)&db, (void*)&idle, (void*)&first_epoch};
+    CUDA_TRY(cudaLaunchCooperativeKernel((const void*)hccl_executor_resident, dim3((unsigned)blocks), dim3((unsigned)p->opts.threads), args, 0, s));
+    p->server_db = host_doorbell;
+    p->server_rings = 0;
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_server_ring(hccl_plan_t* p) {
+    if (!p || !p->server_db) return HCCL_ERR_INVALID_ARG;
+    volatile Doorbell* db = (volatile Doorbell*)p->server_db;
+    if (db->exited) return db->exited == 3 ? (hccl_status_t)db->status : HCCL_ERR_TIMEOUT;  // the kernel has left: start it again
+    std::atomic_thread_fence(std::memory_order_release);
+    db->request = ++p->server_rings;
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_server_wait(hccl_plan_t* p, uint64_t timeout_ns) {
+    if (!p || !p->server_db) return HCCL_ERR_INVALID_ARG;
+    volatile Doorbell* db = (volatile Doorbell*)p->server_db;
+    const auto t0 = std::chrono::steady_clock::now();
+    const uint64_t limit = timeout_ns ? timeout_ns : 5000000000ull;
+    for (;;) {
+        if (db->completed >= p->server_rings) break;
+        if (db->exited) break;
+        if ((uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count() > limit) return HCCL_ERR_TIMEOUT;
+    }
+    std::atomic_thread_fence(std::memory_order_acquire);
+    if (db->exited == 3) return (hccl_status_t)db->status;
+    if (db->completed < p->server_rings) return HCCL_ERR_TIMEOUT;  // left (idle or stopped) before serving this ring
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_server_stop(hccl_plan_t* p) {
+    if (!p || !p->server_db) return HCCL_ERR_INVALID_ARG;
+    volatile Doorbell* db = (volatile Doorbell*)p->server_db;
+    db->stop = 1;
+    p->epoch += p->server_rings;
+    p->server_db = nullptr;
     return HCCL_OK;
 }
 

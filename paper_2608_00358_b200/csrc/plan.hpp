@@ -66,6 +66,9 @@ struct hccl_plan {
     const void* dyn_counts = nullptr;
     void* dyn_recvcounts_out = nullptr;
     void* dyn_rdispls_out = nullptr;
+    // resident executor: the caller's doorbell record while a server kernel is running
+    void* server_db = nullptr;
+    uint64_t server_rings = 0;
     // binding
     void* workspace = nullptr;
     size_t workspace_bytes = 0;

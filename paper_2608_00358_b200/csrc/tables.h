@@ -47,6 +47,8 @@ struct Control {
     uint32_t done_epoch;  // epoch of the last completed execution
     uint64_t detail;      // tile index behind the failure
     uint64_t t_first_ns, t_last_ns;  // globaltimer at first claim / last exit of the last execution
+    uint32_t server_go;   // resident executor: epoch every block may now run, all ones = leave
+    uint32_t pad;
 };
 
 struct Layout {  // byte offsets inside the workspace

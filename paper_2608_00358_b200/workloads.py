@@ -166,3 +166,36 @@ def time_graph_replay(wl: Workload, per_graph: int = 50, replays: int = 10) -> f
     torch.cuda.synchronize()
     wl.dc.check()
     return e0.elapsed_time(e1) / (replays * per_graph)
+
+
+def time_host_observed(wl: Workload, iters: int = 200) -> dict:
+    """Wall-clock microseconds per collective as the host sees it, two ways: a launch followed by a stream
+    synchronisation, and a ring + wait on the resident executor (kernel launched once, no CUDA call per
+    collective). Register engine only."""
+    import time
+    s = torch.cuda.Stream()
+    for _ in range(10):
+        wl.dc.execute(s)
+    s.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(iters):
+        wl.dc.execute(s)
+        s.synchronize()
+    launch_us = (time.perf_counter() - t0) / iters * 1e6
+    bell = torch.zeros(8, dtype=torch.int64).pin_memory()
+    wl.plan.server_start([t.data_ptr() for t in wl.send], [t.data_ptr() for t in wl.recv], bell.data_ptr(), 200_000_000, s.cuda_stream)
+    try:
+        for _ in range(10):
+            wl.plan.server_ring()
+            wl.plan.server_wait(2_000_000_000)
+        t0 = time.perf_counter()
+        for _ in range(iters):
+            wl.plan.server_ring()
+            rc = wl.plan.server_wait(2_000_000_000)
+        ring_us = (time.perf_counter() - t0) / iters * 1e6
+    finally:
+        wl.plan.server_stop()
+        s.synchronize()
+    if rc != hb.OK:
+        raise hb.HcclError(rc, "hccl_server_wait")
+    return {"launch_and_sync_us": launch_us, "ring_and_wait_us": ring_us}
