@@ -159,6 +159,7 @@ def side_configs(quick: bool):
     from paper_2608_00358_b200 import workloads as wk
     out = {}
     it, warm = (200, 20) if quick else (1000, 100)
+    flush_buf = torch.zeros(256 << 20, dtype=torch.uint8, device="cuda")     # 2x the L2
 
     def latency(wl, key):
         ms = wk.time_each(wl, it, warm)
@@ -169,6 +170,9 @@ def side_configs(quick: bool):
                     "tiles": int(i.n_tiles), "chain_depth": int(i.chain_depth), "note": "L2-resident, latency-bound"}
         out[key]["schedule_gbs_back_to_back"] = i.schedule_bytes / out[key]["back_to_back_us"] / 1e3
         out[key]["graph_replay_us"] = float(wk.time_graph_replay(wl) * 1e3)
+        # cold variant: a buffer larger than the L2 is rewritten before every iteration
+        cold = wk.time_each(wl, 50, 5, flush=flush_buf)
+        out[key]["p50_us_cold_l2"] = float(np.percentile(cold, 50) * 1e3)
 
     latency(wk.config1(), "1_allreduce_ring_r4_fp32_1Mi")
     latency(wk.config2(), "2_alltoallv_r8_bf16_dim128")

@@ -102,3 +102,28 @@ def test_config3_full_size_every_output():
               % ("ring" if algo == hb.ALGO_RING else "ring fused", beyond, n))
         del wl
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("engine", [hb.ENGINE_LSU, hb.ENGINE_BULK], ids=["lsu", "bulk"])
+def test_single_segment_beyond_4_gib(engine):
+    """One (source, destination) segment of 5 GiB: tile offsets inside a descriptor exceed 32 bits."""
+    if _free_gb() < 24:
+        pytest.skip("needs 24 GB of free device memory")
+    rows = (5 << 30) // 512
+    C = np.array([[0, rows], [3, 0]], dtype=np.int64)
+    plan = hb.hccl_plan_alltoallv(2, C, None, None, None, hb.FP16, 256, dict(engine=engine))
+    send = [torch.empty(rows * 256, dtype=torch.int16, device="cuda"), torch.arange(3 * 256, dtype=torch.int16, device="cuda")]
+    synth.fill_hashed_rows_torch(send[0], 0, 256)
+    recv = [torch.zeros(3 * 256, dtype=torch.int16, device="cuda"), torch.zeros(rows * 256, dtype=torch.int16, device="cuda")]
+    wl = wk._bind("big_segment", plan, send, recv, {})
+    wl.dc.execute()
+    wl.dc.check()
+    assert torch.equal(recv[1], send[0]) and torch.equal(recv[0], send[1])
+    # the oracle on the rows around the 4 GiB boundary
+    lo = (4 << 30) // 512 - 2
+    X = [synth.hashed_rows_np(0, lo, 4, 256).reshape(-1).view(np.uint8), np.zeros(1, np.uint8)]
+    Y = [np.zeros(1, np.uint8), np.zeros(4 * 512, np.uint8)]
+    orc.alltoallv(X, Y, np.array([[0, 4], [0, 0]]), np.zeros((2, 2), np.int64), np.zeros((2, 2), np.int64), 512)
+    assert np.array_equal(recv[1][lo * 256:(lo + 4) * 256].cpu().numpy().view(np.uint8), Y[1])
+    del wl, send, recv
+    torch.cuda.empty_cache()
