@@ -226,7 +226,7 @@ def run_profile_case(args):
     from paper_2608_00358_b200 import binding as hb
     from paper_2608_00358_b200 import workloads as wk
     algo = {"c3ring": hb.ALGO_RING, "c3fused": hb.ALGO_RING_FUSED}[args.profile_case]
-    wl = wk.config3(algo=algo, n=1 << 23)
+    wl = wk.config3(algo=algo, n=args.profile_n)
     ms = wk.time_back_to_back(wl, args.steps, max(args.warmup, 3))
     i = wl.info
     print(json.dumps({"case": args.profile_case, "workload": wl.name, "ms": ms, "schedule_bytes": int(i.schedule_bytes),
@@ -384,6 +384,7 @@ def main():
     ap.add_argument("--no-gemm", action="store_true")
     ap.add_argument("--no-side", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--profile-n", type=int, default=1 << 23, help="elements per rank of the --profile-case")
     ap.add_argument("--profile-case", default="", choices=["", "c3ring", "c3fused"],
                     help="run only a small single-kernel case (for ncu captures), not the benchmark")
     args = ap.parse_args()

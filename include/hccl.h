@@ -96,11 +96,12 @@ typedef struct {
     uint32_t flags;         /* HCCL_FLAG_* */
     int32_t chain_group;    /* chains scheduled together in chain-group-major order (default 16) */
     int32_t threads;        /* threads per block, multiple of 32 (default 512) */
-    int32_t stages;         /* bulk engine: shared-memory stages of 32 KiB per block, 2..6 (default 6) */
+    int32_t stages;         /* bulk engine: shared-memory stages of 48 KiB per block, 2..4 (default 4) */
     int32_t cluster;        /* register engine: launch blocks in clusters of this size (2, 4, 8) so that they sit on
                                neighbouring SMs; 0/1 = no clusters. Ignored unless it divides the block count. */
     int32_t light;          /* register engine: nonzero = the 64-register build (several blocks per SM) */
-    int32_t copy_by_warps;  /* bulk engine: nonzero = COPY pieces are loaded by the bulk unit but stored by the compute warps */
+    int32_t copy_by_warps;  /* bulk engine: who stores COPY stages. 1 = the compute warps (a stage is free as soon as it is read;
+                               best per-block rate), 2 = the bulk unit, 0 = compute warps below 100 blocks, bulk unit otherwise */
     int32_t rack_size;      /* ranks per rack for HCCL_ALGO_RING_2LEVEL and for cross-rack byte accounting (default 16,
                                the paper's rack, Sec. V-D) */
 } hccl_opts_t;

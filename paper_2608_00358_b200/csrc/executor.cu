@@ -732,10 +732,11 @@ __global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_c
 // is handed to the compute warps as a whole work item for the register path.
 namespace bulk {
 
-constexpr uint32_t MAX_STAGES = 6;  // 6 x 32 KiB + bookkeeping fits the 227 KB a block may have
-constexpr uint32_t REGION = 16384;            // bytes per operand region of a stage
-constexpr uint32_t STAGE_BYTES = 2 * REGION;  // region A + region B; a COPY piece uses both as one buffer
-constexpr uint32_t PIECE_ELEMS = 4096;        // elements per REDUCE piece (fp32 fills a region exactly)
+constexpr uint32_t MAX_STAGES = 4;            // 4 x 48 KiB + bookkeeping fits the 227 KB a block may have
+constexpr uint32_t STAGE_BYTES = 49152;       // a COPY piece fills a stage; a REDUCE piece splits it into A and B
+// Elements per REDUCE piece: as many as fit a stage with both operands, in whole multiples of 512 elements
+// (6144 for fp32+fp32, 8192 for fp32+16-bit, 12288 for 16-bit+16-bit).
+__host__ __device__ constexpr uint32_t piece_elems(uint32_t ea, uint32_t eb) { return STAGE_BYTES / (ea + eb) / 512 * 512; }
 
 // PIECE_COPY: loaded and stored by the bulk unit. PIECE_COPYW: loaded by the bulk unit, stored by the compute
 // warps from shared memory (the stage is free as soon as the warps have read it, without waiting for a
@@ -751,7 +752,7 @@ struct alignas(16) PieceInfo {  // one per stage, in shared memory; written by t
     unsigned long long group;  // COPY: sequence number of the bulk store group that drains this stage
     int32_t signal[2];
     uint8_t dt_a, dt_b, dt_d, evict_first;
-    uint32_t pad;
+    uint32_t b_off;       // REDUCE: byte offset of operand B inside the stage
     Tile tile;            // PIECE_TILE: the work item and its descriptor for the register path
     Desc desc;
 };
@@ -1066,8 +1067,9 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
                 keep_lag(p, d);
                 return d.ok;
             }
-            for (uint32_t e0 = 0; e0 < t.count && d.ok; e0 += PIECE_ELEMS) {
-                const uint32_t ne = min(PIECE_ELEMS, t.count - e0);
+            const uint32_t pe = piece_elems(ea, eb);
+            for (uint32_t e0 = 0; e0 < t.count && d.ok; e0 += pe) {
+                const uint32_t ne = min(pe, t.count - e0);
                 const unsigned long long k = d.head;
                 if (!acquire_slot(p, d, k, cur)) return false;
                 const uint32_t slot = (uint32_t)(k % d.ns);
@@ -1080,9 +1082,10 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
                 pi.signal[0] = t.signal[0];
                 pi.signal[1] = t.signal[1];
                 pi.dt_a = ds.dt_a; pi.dt_b = ds.dt_b; pi.dt_d = ds.dt_dst;
+                pi.b_off = pe * ea;
                 mbar_arrive_expect_tx(d.full + 8 * slot, ne * (ea + eb));
                 bulk_load(d.stages + slot * STAGE_BYTES, a + (size_t)e0 * ea, ne * ea, d.full + 8 * slot, ds.kind_a == HCCL_BUF_SEND, d.pol);
-                bulk_load(d.stages + slot * STAGE_BYTES + REGION, b + (size_t)e0 * eb, ne * eb, d.full + 8 * slot, ds.kind_b == HCCL_BUF_SEND, d.pol);
+                bulk_load(d.stages + slot * STAGE_BYTES + pe * ea, b + (size_t)e0 * eb, ne * eb, d.full + 8 * slot, ds.kind_b == HCCL_BUF_SEND, d.pol);
                 d.head = k + 1;
                 keep_lag(p, d);
             }
@@ -1179,7 +1182,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         }
         if (kind == PIECE_REDUCE) {
             reduce_piece_dispatch(pi.dt_a, pi.dt_b, pi.dt_d, stages_ptr + (size_t)slot * STAGE_BYTES,
-                                  stages_ptr + (size_t)slot * STAGE_BYTES + REGION, pi.dst, pi.n, ctid, cnth);
+                                  stages_ptr + (size_t)slot * STAGE_BYTES + pi.b_off, pi.dst, pi.n, ctid, cnth);
         } else if (kind == PIECE_COPYW) {
             const uint4* src = reinterpret_cast<const uint4*>(stages_ptr + (size_t)slot * STAGE_BYTES);
             uint4* dst = reinterpret_cast<uint4*>(pi.dst);
@@ -1605,10 +1608,10 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     prm.nblocks = (uint32_t)blocks;
     prm.static_tickets = (prm.n_waits == 0 && prm.n_tiles <= (uint32_t)blocks) ? 1 : 0;
     if (p->opts.engine == HCCL_ENGINE_BULK) {
-        const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : 6, 2), (int)bulk::MAX_STAGES);
+        const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : (int)bulk::MAX_STAGES, 2), (int)bulk::MAX_STAGES);
         const size_t smem = (size_t)ns * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
         const int threads = std::max(64, p->opts.threads);
-        hccl_executor_bulk<<<blocks, threads, smem, (cudaStream_t)stream>>>(prm, ns, (uint32_t)(p->opts.copy_by_warps != 0));
+        hccl_executor_bulk<<<blocks, threads, smem, (cudaStream_t)stream>>>(prm, ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)));
     } else {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)blocks);

@@ -83,8 +83,8 @@ namespace hccl {
 // Tiles that are whole multiples of it leave no partly idle pass at the end of a tile.
 inline int64_t sweep_of(const hccl_opts_t& o, int op) {
     if (o.engine == HCCL_ENGINE_BULK) {
-        if (op == HCCL_OP_COPY) return 32768;                 // one stage
-        if (op == HCCL_OP_REDUCE) return 4096;                // one piece
+        if (op == HCCL_OP_COPY) return 49152;                 // one stage
+        if (op == HCCL_OP_REDUCE) return 24576;               // whole pieces for every operand mix (6144, 8192, 12288)
         return (int64_t)(o.threads - 32) * 8;                 // multi-input sums run on the compute warps
     }
     const int64_t workers = o.threads - 32;
