@@ -356,6 +356,14 @@ typedef struct {
 } hccl_plan_info_t;
 hccl_status_t hccl_plan_info(const hccl_plan_t*, hccl_plan_info_t* out);
 
+/* Tracing (the per-work-packet and per-subgraph counters of Sec. V-C, per work item here): give the plan a
+ * caller-owned DEVICE array of capacity_items x 4 uint64 and every later execution records, for work item i,
+ * [4i] = i | block << 32, [4i+1] = time it was claimed, [4i+2] = time its data movement was released (all
+ * dependencies met), [4i+3] = time its last byte was stored (bulk COPY: its last store issued); %globaltimer
+ * nanoseconds. Items beyond the capacity are not recorded. Pass capacity 0 to switch tracing off. The
+ * resident executor and hccl_execute_noalloc do not trace. */
+hccl_status_t hccl_plan_set_trace(hccl_plan_t*, void* dev_trace, int64_t capacity_items);
+
 /* Byte offsets of the regions inside a bound workspace, in this order: control block, dependency counters,
  * signal slots, descriptors (64 B each), tiles (32 B each), wait lists (8 B per entry), FP32 scratch, total.
  * For tools that inspect a workspace, and for tests that damage a table on purpose. */

@@ -89,6 +89,7 @@ def _load() -> C.CDLL:
         "hccl_server_wait": [P, C.c_uint64],
         "hccl_server_stop": [P],
         "hccl_plan_set_user_signals": [P, P, C.c_int64],
+        "hccl_plan_set_trace": [P, P, C.c_int64],
         "hccl_plan_set_trigger": [P, C.c_int64, C.c_int32, C.c_uint64, C.c_uint64, C.c_int64, C.c_uint64, C.c_uint64],
         "hccl_plan_status": [P, C.POINTER(C.c_int), I64P],
         "hccl_plan_info": [P, C.POINTER(PlanInfo)],
@@ -121,7 +122,7 @@ EXPORTS = ["hccl_plan_allreduce", "hccl_plan_reducescatter", "hccl_plan_allgathe
            "hccl_graph_create", "hccl_graph_add_subgraph", "hccl_graph_add_wqe", "hccl_graph_compile",
            "hccl_graph_destroy", "hccl_plan_workspace_bytes", "hccl_plan_bind", "hccl_execute", "hccl_execute_host",
            "hccl_execute_noalloc", "hccl_server_start", "hccl_server_ring", "hccl_server_wait", "hccl_server_stop",
-           "hccl_plan_set_user_signals", "hccl_plan_set_trigger", "hccl_plan_status", "hccl_plan_info",
+           "hccl_plan_set_user_signals", "hccl_plan_set_trace", "hccl_plan_set_trigger", "hccl_plan_status", "hccl_plan_info",
            "hccl_plan_extents", "hccl_plan_layout", "hccl_plan_destroy", "hccl_status_string", "hccl_last_cuda_error", "hccl_version",
            "hccl_plan_check_hazards", "hccl_plan_interpret_host"]
 
@@ -228,6 +229,9 @@ class Plan:
     def set_dynamic_metadata(self, dev_sendcounts: int, dev_recvcounts_out: int = 0, dev_rdispls_out: int = 0):
         _chk(_lib.hccl_plan_set_dynamic_metadata(self._h, C.c_void_p(dev_sendcounts), C.c_void_p(dev_recvcounts_out or None),
                                                  C.c_void_p(dev_rdispls_out or None)), "hccl_plan_set_dynamic_metadata")
+
+    def set_trace(self, dev_trace: int, capacity_items: int):
+        _chk(_lib.hccl_plan_set_trace(self._h, C.c_void_p(dev_trace or None), capacity_items), "hccl_plan_set_trace")
 
     def set_user_signals(self, dev_signals: int, n_slots: int):
         _chk(_lib.hccl_plan_set_user_signals(self._h, C.c_void_p(dev_signals), n_slots), "hccl_plan_set_user_signals")

@@ -37,6 +37,8 @@ struct ExecParams {
     Control* ctl;
     char* scratch;
     unsigned long long* user_signals;
+    unsigned long long* trace;  // optional: 4 words per work item (item | block << 32, claim, start, end in ns), or null
+    unsigned long long trace_cap;
     uint32_t n_tiles, n_descs, n_syncs, n_waits;
     uint32_t R, nblocks, n_signals, pad0;
     unsigned long long timeout_ns;
@@ -57,6 +59,11 @@ template <class P>
 __device__ __forceinline__ void init_epoch(const P& p) {
     if (threadIdx.x == 0) g_epoch = *(volatile uint32_t*)&p.ctl->done_epoch + 1u;
     __syncthreads();
+}
+
+// Per-item timestamps for the optional trace (counters per work packet and per subgraph, paper Sec. V-C).
+__device__ __forceinline__ void trace_put(unsigned long long* trace, unsigned long long cap, uint32_t item, int word, unsigned long long v) {
+    if (trace && item < cap) trace[(size_t)item * 4 + word] = v;
 }
 
 // ------------------------------------------------------------------ device primitives
@@ -581,6 +588,10 @@ __device__ __forceinline__ void named_sync(uint32_t id, uint32_t nthreads) {
 
 // Loads and checks the records of work item `cur`. No waiting here.
 __device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d) {
+    if (p.trace) {
+        trace_put(p.trace, p.trace_cap, cur, 0, (unsigned long long)cur | ((unsigned long long)blockIdx.x << 32));
+        trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
+    }
     t = p.tiles[cur];
     if (!tile_ok(p, t)) {
         fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
@@ -657,7 +668,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
     }
-    uint32_t cur = 0;
+    uint32_t cur = 0, prev_item = 0;
     for (uint32_t k = 0;; ++k) {
         const uint32_t b = k & 1;
         int32_t sig0 = -1, sig1 = -1;
@@ -680,6 +691,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
             }
         }
         if (k > 0) named_sync(DONE + (b ^ 1), nth);  // the workers have stored all of item k-1
+        if (tid == 0 && p.trace && k > 0) trace_put(p.trace, p.trace_cap, prev_item, 3, globaltimer_ns());
         if (tid == 0) {
             const bool simple = have && ready && s_desc[b].op != HCCL_OP_WAIT && s_desc[b].op != HCCL_OP_SET;
             if (!simple && prev && (sig0 >= 0 || sig1 >= 0)) {
@@ -695,6 +707,8 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         }
         named_sync(FULL + b, nth);  // workers start item k (or leave)
         const int go = s_go[b];
+        if (tid == 0 && p.trace && go) trace_put(p.trace, p.trace_cap, cur, 2, globaltimer_ns());
+        prev_item = cur;
         if (tid == 0) {
             if (sig0 >= 0 || sig1 >= 0) {  // publish item k-1 while the workers run item k
                 if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
@@ -922,6 +936,7 @@ __device__ void retire_one(const ExecParams& p, Dma& d) {
         if (d.ok) {
             bulk_store(pi.dst, d.stages + slot * STAGE_BYTES, pi.n, pi.evict_first != 0, d.pol);
             pi.group = d.groups++;
+            if (pi.last && p.trace) trace_put(p.trace, p.trace_cap, pi.tile_index, 3, globaltimer_ns());
             if (pi.last && (pi.signal[0] >= 0 || pi.signal[1] >= 0)) {
                 bulk_wait_all();  // the item's bytes are in global memory
                 fence_proxy_async();
@@ -984,6 +999,10 @@ __device__ void issue_simple(const ExecParams& p, Dma& d, uint32_t kind, uint32_
 
 // One work item through the DMA thread. Returns false when the block must stop.
 __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
+    if (p.trace) {
+        trace_put(p.trace, p.trace_cap, cur, 0, (unsigned long long)cur | ((unsigned long long)blockIdx.x << 32));
+        trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
+    }
     const Tile t = p.tiles[cur];
     if (!tile_ok(p, t)) {
         fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
@@ -1005,6 +1024,7 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
         waited = true;
     }
     if (waited) fence_proxy_async();  // what the acquired counters cover must be visible to the bulk unit too
+    if (p.trace) trace_put(p.trace, p.trace_cap, cur, 2, globaltimer_ns());
     switch (ds.op) {
         case HCCL_OP_WAIT: {
             drain(p, d);
@@ -1194,6 +1214,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         } else if (kind == PIECE_TILE) {
             run_tile_lsu(p, pi.desc, pi.tile, ctid, cnth);
         }
+        if (kind != PIECE_COPY && pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.tile_index, 3, globaltimer_ns());
         if (kind != PIECE_COPY && pi.last && (pi.signal[0] >= 0 || pi.signal[1] >= 0)) {
             asm volatile("bar.sync 1, %0;" ::"r"(cnth) : "memory");  // every compute warp has stored its share
             if (ctid == 0) {  // release, cumulative over the stores the barrier ordered before this thread
@@ -1583,6 +1604,8 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     prm.ctl = (Control*)(ws + L.control);
     prm.scratch = ws + L.scratch;
     prm.user_signals = (unsigned long long*)p->user_signals;
+    prm.trace = (unsigned long long*)p->trace;
+    prm.trace_cap = (unsigned long long)p->trace_cap;
     prm.n_tiles = (uint32_t)p->tiles.size();
     prm.n_descs = (uint32_t)p->descs.size();
     prm.n_syncs = (uint32_t)p->sync_per_epoch.size();
@@ -1704,6 +1727,8 @@ hccl_status_t hccl_server_start(hccl_plan_t* p, const void* const* sendbufs, voi
     prm.ctl = (Control*)(ws + L.control);
     prm.scratch = ws + L.scratch;
     prm.user_signals = (unsigned long long*)p->user_signals;
+    prm.trace = (unsigned long long*)p->trace;
+    prm.trace_cap = (unsigned long long)p->trace_cap;
     prm.n_tiles = (uint32_t)p->tiles.size();
     prm.n_descs = (uint32_t)p->descs.size();
     prm.n_syncs = (uint32_t)p->sync_per_epoch.size();
@@ -1848,6 +1873,8 @@ extern "C" hccl_status_t hccl_execute_noalloc(hccl_plan_t* p, const void* const*
     prm.ctl = (Control*)(ws + L.control);
     prm.scratch = ws + L.scratch;
     prm.user_signals = nullptr;
+    prm.trace = nullptr;
+    prm.trace_cap = 0;
     prm.n_tiles = (uint32_t)p->tiles.size();
     prm.n_descs = (uint32_t)p->descs.size();
     prm.n_syncs = (uint32_t)p->sync_per_epoch.size();

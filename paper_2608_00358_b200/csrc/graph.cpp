@@ -498,6 +498,14 @@ hccl_status_t hccl_plan_set_user_signals(hccl_plan_t* p, void* dev_signals, int6
     return HCCL_OK;
 }
 
+hccl_status_t hccl_plan_set_trace(hccl_plan_t* p, void* dev_trace, int64_t capacity_items) {
+    if (!p || capacity_items < 0 || (capacity_items > 0 && !dev_trace)) return HCCL_ERR_INVALID_ARG;
+    if (((uintptr_t)dev_trace) % 8) return HCCL_ERR_ALIGNMENT;
+    p->trace = capacity_items ? dev_trace : nullptr;
+    p->trace_cap = capacity_items;
+    return HCCL_OK;
+}
+
 hccl_status_t hccl_plan_set_trigger(hccl_plan_t* p, int64_t wait_slot, int32_t cmp, uint64_t wait_value,
                                     uint64_t wait_per_epoch, int64_t set_slot, uint64_t set_value, uint64_t set_per_epoch) {
     if (!p) return HCCL_ERR_INVALID_ARG;

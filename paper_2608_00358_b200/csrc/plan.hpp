@@ -66,6 +66,9 @@ struct hccl_plan {
     const void* dyn_counts = nullptr;
     void* dyn_recvcounts_out = nullptr;
     void* dyn_rdispls_out = nullptr;
+    // optional per-item timestamps
+    void* trace = nullptr;
+    int64_t trace_cap = 0;
     // resident executor: the caller's doorbell record while a server kernel is running
     void* server_db = nullptr;
     uint64_t server_rings = 0;

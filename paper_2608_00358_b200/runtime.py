@@ -66,3 +66,32 @@ class DeviceCollective:
         st, detail = self.plan.status()
         if st != hb.OK:
             raise hb.HcclError(st, "device status (tile %d)" % detail)
+
+
+def enable_trace(plan: hb.Plan, device="cuda") -> torch.Tensor:
+    """Allocates a trace array for every work item of `plan` and switches tracing on. Returns the tensor
+    ([n_tiles, 4] int64: item | block << 32, claimed, released, stored; nanoseconds of %globaltimer)."""
+    n = max(int(plan.info().n_tiles), 1)
+    t = torch.zeros((n, 4), dtype=torch.int64, device=device)
+    plan.set_trace(t.data_ptr(), n)
+    return t
+
+
+def chrome_trace(trace: torch.Tensor, name: str = "hccl") -> dict:
+    """Trace array -> Chrome trace-event JSON (one row per thread block, one slice per work item from the
+    moment its data movement was released to its last store, with the wait before it as a separate slice)."""
+    rows = trace.cpu().numpy()
+    rows = rows[rows[:, 1] != 0]
+    if rows.shape[0] == 0:
+        return {"traceEvents": []}
+    t0 = int(rows[:, 1].min())
+    ev = []
+    for item_block, claimed, released, stored in rows.tolist():
+        item, block = item_block & 0xFFFFFFFF, item_block >> 32
+        if released and released > claimed:
+            ev.append({"name": "wait", "cat": "dependency", "ph": "X", "pid": name, "tid": block,
+                       "ts": (claimed - t0) / 1e3, "dur": (released - claimed) / 1e3, "args": {"item": item}})
+        if stored and released:
+            ev.append({"name": "item %d" % item, "cat": "data", "ph": "X", "pid": name, "tid": block,
+                       "ts": (released - t0) / 1e3, "dur": max(stored - released, 0) / 1e3, "args": {"item": item}})
+    return {"traceEvents": ev, "displayTimeUnit": "ns"}
