@@ -213,3 +213,26 @@ def test_two_level_allgather(G, L, engine):
     want = orc.allgatherv(X)
     for r in range(R):
         assert np.array_equal(Y[r].view(np.uint16), want[r])
+
+
+def test_maximum_rank_count(engine):
+    """R = 256, the largest job size the paper mentions: pointer tables, rank arithmetic and ring rotation."""
+    R, n, dt = 256, 3001, hb.BF16
+    X = synth.small_int_ranks(R, n, dt, seed=256, span=1)          # exactly summable in bf16: unique result
+    want = orc.allreduce(dt, X)
+    for algo, extra in ((hb.ALGO_RING, {}), (hb.ALGO_ONESHOT, {}), (hb.ALGO_RING_2LEVEL, dict(rack_size=16))):
+        p = hb.hccl_plan_allreduce(R, n, dt, algo, _with(dict(sm_budget=64, **extra), engine))
+        Y = run_plan(p, X)
+        for r in (0, 1, 127, 255):
+            assert np.array_equal(Y[r].view(np.uint16), want[r]), (algo, r)
+    C = synth.uniform_counts(R, 3, hi=3)
+    SD, RD = orc.packed_displs(C)
+    rb = 16 * 2
+    Xa = [synth.hashed_rows_np(s, 0, int(C[s].sum()), 16).reshape(-1).view(np.uint8) for s in range(R)]
+    Xa = [x if x.size else np.zeros(16, np.uint8) for x in Xa]
+    p = hb.hccl_plan_alltoallv(R, C, None, None, None, hb.FP16, 16, _with(dict(sm_budget=64), engine))
+    Y = run_plan(p, Xa)
+    Yw = [np.full(p.extents(r)[1], 0xA5, dtype=np.uint8) for r in range(R)]
+    orc.alltoallv(Xa, Yw, C, SD, RD, rb)
+    for r in range(R):
+        assert np.array_equal(Y[r], Yw[r])
