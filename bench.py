@@ -254,7 +254,12 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             dist.barrier()
         torch.cuda.synchronize()
 
-    opts = dict(sm_budget=args.sm_budget) if args.sm_budget else None
+    opts = {}
+    if args.sm_budget:
+        opts["sm_budget"] = args.sm_budget
+    if args.engine:
+        opts["engine"] = {"lsu": 1, "bulk": 2}[args.engine]
+    opts = opts or None
     wl = wk.config4(opts, seed=0, cap=args.cap)
     info = wl.info
     payload = wl.meta["payload_bytes"]
@@ -377,6 +382,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cap", type=int, default=32768, help="clamp of the Zipf row counts (32768 = the named config)")
     ap.add_argument("--sm-budget", type=int, default=0)
+    ap.add_argument("--engine", default="", choices=["", "lsu", "bulk"], help="force an executor engine (default: the library's choice)")
     ap.add_argument("--oracle-dst", type=int, default=8, help="destination ranks in the CPU oracle's sample")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--quick", action="store_true")

@@ -28,6 +28,8 @@
  *    hccl_plan_status after the stream has been synchronised. After a
  *    device-side failure the plan must be bound again before reuse.
  *  - Only sum reductions exist (Sec. II-A.2). Element types: FP32, BF16, FP16.
+ *  - A plan or graph handle is not thread-safe: use one handle from one host thread at a time. Different
+ *    handles may be used from different threads.
  */
 #ifndef HCCL_B200_H
 #define HCCL_B200_H
