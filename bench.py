@@ -187,7 +187,6 @@ def side_configs(quick: bool):
     # and re-enqueueing a cached one; plus the device-resident AllToAllv, where the counts never visit the host
     import time as _time
     from paper_2608_00358_b200 import synth as _synth
-    from paper_2608_00358_b200.runtime import DeviceCollective as _DC
     host = {}
     for name, R, C, row, dt in (("alltoallv_r8", 8, _synth.uniform_counts(8, 0, 4096), 128, hb.BF16),
                                 ("alltoallv_r64_zipf", 64, _synth.zipf_counts(64, 0, 1.1, 32768), 256, hb.FP16)):

@@ -36,35 +36,6 @@ class Gemm:
         torch.matmul(self.a, self.b, out=self.c)
 
 
-def gemm_alone(gemm: Gemm, seconds: float = 3.0, discard: float = 1.0, batch: int = 10) -> dict:
-    """Sustained TFLOP/s of the GEMM with nothing else on the GPU; the first `discard` seconds are dropped."""
-    s = torch.cuda.Stream()
-    base = torch.cuda.Event(enable_timing=True)
-    evs = []
-    with torch.cuda.stream(s):
-        for _ in range(3):
-            gemm.run()
-        s.synchronize()
-        base.record(s)
-        t0 = time.time()
-        while time.time() - t0 < seconds:
-            for _ in range(batch):
-                gemm.run()
-            e = torch.cuda.Event(enable_timing=True)
-            e.record(s)
-            evs.append(e)
-            if len(evs) > 20:
-                evs[-20].synchronize()       # keep the queue bounded
-        s.synchronize()
-    ts = np.array([base.elapsed_time(e) for e in evs])     # ms at the end of each batch
-    keep = ts >= discard * 1e3
-    if keep.sum() < 3:
-        keep[:] = True
-    tk = ts[keep]
-    tf = gemm.flops * batch * (len(tk) - 1) / ((tk[-1] - tk[0]) * 1e-3) / 1e12
-    return dict(tflops=float(tf), batches=int(len(tk) - 1), seconds=float((tk[-1] - tk[0]) * 1e-3))
-
-
 def overlap(gemm: Gemm, wl: Optional[wk.Workload], seconds: float = 3.0, discard: float = 1.0, gemm_batch: int = 10) -> dict:
     """GEMM loop on one stream, collective loop on a high-priority stream; rates are computed only inside
     the window in which events show both loops running."""

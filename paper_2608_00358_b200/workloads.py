@@ -38,13 +38,6 @@ def _bind(name, plan, send, recv, meta=None, stream=None) -> Workload:
     return Workload(name, plan, dc, send, recv, meta or {})
 
 
-def packed_displs_np(C: np.ndarray):
-    """Row displacements of a packed layout (layout bookkeeping for buffer allocation, not the exchange)."""
-    sd = np.cumsum(C, axis=1) - C
-    rd = (np.cumsum(C, axis=0) - C).T.copy()
-    return sd, rd
-
-
 def config1(opts=None, seed=0) -> Workload:
     """AllReduce ring, R=4, 1 Mi fp32 per rank, uniform(-1,1)."""
     R, n = 4, 1 << 20

@@ -2,7 +2,6 @@
 import numpy as np
 import torch
 
-from paper_2608_00358_b200 import binding as hb
 from paper_2608_00358_b200.runtime import DeviceCollective
 
 GUARD = 256

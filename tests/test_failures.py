@@ -1,7 +1,6 @@
 """Failure detection without faulting a GPU: every failure is made on the host (an unsatisfiable WAIT, a
 damaged table entry, a workspace that is too small or misaligned) and must come back as a status code with
 the device healthy. Nothing here traps, hangs or reads out of bounds."""
-import numpy as np
 import pytest
 
 from paper_2608_00358_b200 import binding as hb

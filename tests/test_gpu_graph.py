@@ -4,7 +4,6 @@ stay consistent across replays (cached re-enqueue, paper Sec. V-B, taken one ste
 import numpy as np
 import pytest
 
-from helpers import np_dtype
 from oracle import oracle as orc
 from paper_2608_00358_b200 import binding as hb
 from paper_2608_00358_b200 import synth

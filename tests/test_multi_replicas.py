@@ -3,7 +3,6 @@ of the timed region, whole-job throughput = bytes of all replicas / slowest repl
 import os
 import socket
 
-import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
