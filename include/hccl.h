@@ -88,6 +88,9 @@ typedef enum {
                                     partial into this rank's staging slot, then REDUCE (A=A+B). Default fuses
                                     the pair into one REDUCE that reads the peer's buffer directly. */
 
+#define HCCL_FLAG_BIDIRECTIONAL 8u /* flat ring AllReduce / ReduceScatter: granules of a chunk alternate direction, even
+                                     ones travel r -> r+1, odd ones r -> r-1 (a bidirectional ring, Sec. III-B.2) */
+
 /* Options. A zero field means "default". */
 typedef struct {
     int32_t sm_budget;      /* thread blocks of the persistent executor = "message engines" (default 148) */

@@ -338,6 +338,27 @@ int oracle_allreduce_oneshot_f32(int R, int64_t n, int dt, const void *const *X,
     return 0;
 }
 
+/* Ring order with a direction per segment (bidirectional rings, Sec. III-B.2: half of the data travels
+ * r -> r+1, the other half r -> r-1). Segment s covers elements [seg_off[s], seg_off[s+1]) of chunk
+ * seg_chunk[s] and travels in direction seg_dir[s] (+1 or -1): its elements are summed as
+ * ((X_{c+d} + X_{c+2d}) + ...) + X_c (indices mod R), FP32 adds, one rounding; every rank gets the result. */
+int oracle_allreduce_ring_dir_f32(int R, int nseg, const int64_t *seg_off, const int64_t *seg_chunk,
+                                  const int64_t *seg_dir, int dt, const void *const *X, void *const *Y) {
+    if (R < 1 || nseg < 0) return 1;
+    for (int s = 0; s < nseg; ++s) {
+        const int c = (int)seg_chunk[s], d = seg_dir[s] >= 0 ? 1 : -1;
+        for (int64_t i = seg_off[s]; i < seg_off[s + 1]; ++i) {
+            volatile float acc = (float)load_elem(X[((c + d) % R + R) % R], i, dt);
+            for (int t = 2; t <= R; ++t) {
+                volatile float x = (float)load_elem(X[((c + d * t) % R + R) % R], i, dt);
+                acc = acc + x;
+            }
+            for (int r = 0; r < R; ++r) store_elem(Y[r], i, dt, (double)acc);
+        }
+    }
+    return 0;
+}
+
 /* Two-level ring order (Sec. V-D: topology-aware schedules that keep most exchanges inside a rack).
  * R = G racks of L ranks; rank (g, l) = g*L + l. The buffer is cut into L chunks (offs1, L+1 entries) and
  * every chunk j into G sub-chunks (offs2[j*(G+1) .. j*(G+1)+G], absolute element offsets). For sub-chunk

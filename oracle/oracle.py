@@ -154,6 +154,34 @@ def reducescatter_ring_f32(dt: int, X: list, recvcounts) -> list:
     return _ring(lib().oracle_reducescatter_ring_f32, dt, X, rc, lambda r: int(rc[r]))
 
 
+def bidirectional_segments(n: int, R: int, granule: int):
+    """Chunk c (floor split of n over R) cut into granules; granule k of a chunk travels forwards when k is
+    even and backwards when k is odd. Returns (seg_off [nseg+1], seg_chunk, seg_dir)."""
+    offs = floor_chunk_offsets(n, R)
+    off, chunk, direction = [], [], []
+    for c in range(R):
+        lo, hi = int(offs[c]), int(offs[c + 1])
+        k = 0
+        while lo < hi:
+            off.append(lo)
+            chunk.append(c)
+            direction.append(1 if k % 2 == 0 else -1)
+            lo = min(hi, lo + granule)
+            k += 1
+    off.append(n)
+    return np.array(off, dtype=np.int64), np.array(chunk, dtype=np.int64), np.array(direction, dtype=np.int64)
+
+
+def allreduce_ring_dir_f32(dt: int, X: list, seg_off, seg_chunk, seg_dir) -> list:
+    R, n = len(X), X[0].size
+    so, sop = _i64(seg_off)
+    sc, scp = _i64(seg_chunk)
+    sd, sdp = _i64(seg_dir)
+    Y = [np.empty(n, dtype=np_dtype(dt)) for _ in range(R)]
+    _check(lib().oracle_allreduce_ring_dir_f32(R, int(sc.size), sop, scp, sdp, dt, _ptrs(X), _ptrs(Y, True)), "ring_dir")
+    return Y
+
+
 def two_level_offsets(n: int, G: int, L: int):
     """Chunk j of L (floor split of n), each cut into G sub-chunks (floor split of the chunk)."""
     offs1 = floor_chunk_offsets(n, L)

@@ -33,6 +33,7 @@ struct Chain {
     int c;            // chunk index = rank the reduced chunk ends on
     int64_t e0, len;  // element range [e0, e0+len) in the send buffers
     int64_t out_off;  // element offset of e0 inside Y_c for a scatter (AllReduce: == e0)
+    int dir;          // +1: the chunk travels r -> r+1; -1: r -> r-1 (bidirectional rings)
 };
 
 #define CHECK(x)                         \
@@ -87,7 +88,8 @@ hccl_status_t emit_ring(hccl_graph* g, int R, int dt, const std::vector<Chain>& 
                     w.count = ch.len;
                 } else if (is_rs) {
                     const int t = step;
-                    const int r = (c + t + 2) % R, pr = (r + R - 1) % R;
+                    const int dir = ch.dir;
+                    const int r = (((c + dir * (t + 2)) % R) + R) % R, pr = (((r - dir) % R) + R) % R;
                     const bool first = t == 0, final = t == rs_steps - 1;
                     w.op = HCCL_OP_REDUCE;
                     w.count = ch.len;
@@ -132,7 +134,7 @@ hccl_status_t emit_ring(hccl_graph* g, int R, int dt, const std::vector<Chain>& 
                     }
                 } else {
                     const int u = fused ? step - 1 : step - rs_steps;
-                    const int dst_rank = (c + u + 1) % R, src_rank = (c + u) % R;
+                    const int dst_rank = (((c + ch.dir * (u + 1)) % R) + R) % R, src_rank = (((c + ch.dir * u) % R) + R) % R;
                     w.op = HCCL_OP_COPY;
                     w.tile_count = tile_elems * es;
                     w.count = ch.len * es;
@@ -178,7 +180,7 @@ void fill_copy_opts(hccl_opts_t* o, const hccl_opts_t* in) {
     fill_default_opts(o, &tmp);
 }
 
-std::vector<Chain> make_chains(int R, const std::vector<int64_t>& offs, bool scatter, int64_t granule_elems) {
+std::vector<Chain> make_chains(int R, const std::vector<int64_t>& offs, bool scatter, int64_t granule_elems, bool bidirectional) {
     // chunk c = [offs[c], offs[c+1]); cut into granules; granule-major order so that consecutive chains
     // belong to different chunks (different final ranks) and a chain group spans the ring evenly
     std::vector<Chain> chains;
@@ -189,7 +191,7 @@ std::vector<Chain> make_chains(int R, const std::vector<int64_t>& offs, bool sca
         for (int c = 0; c < R; ++c) {
             const int64_t lo = offs[c] + k * granule_elems, hi = std::min(offs[c + 1], lo + granule_elems);
             if (lo >= hi) continue;  // empty chunks and exhausted chunks are elided
-            chains.push_back(Chain{c, lo, hi - lo, scatter ? lo - offs[c] : lo});
+            chains.push_back(Chain{c, lo, hi - lo, scatter ? lo - offs[c] : lo, (bidirectional && (k & 1)) ? -1 : 1});
         }
     }
     return chains;
@@ -476,7 +478,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     std::vector<int64_t> offs(R + 1);
     for (int c = 0; c <= R; ++c) offs[c] = (int64_t)(((__int128)c * count) / R);
     const int64_t granule = std::max<int64_t>(1, (int64_t)(o.chunk_bytes / (uint64_t)es));
-    std::vector<Chain> chains = make_chains(R, offs, false, granule);
+    std::vector<Chain> chains = make_chains(R, offs, false, granule, (o.flags & HCCL_FLAG_BIDIRECTIONAL) != 0 && !fused);
     int64_t maxlen = 0;
     for (const Chain& ch : chains) maxlen = std::max(maxlen, ch.len);
     // small buffers (all FP32 partials fit the L2 several times over): run every chain together, the
@@ -541,7 +543,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     }
     const bool fused = algo == HCCL_ALGO_RING_FUSED;
     const int64_t granule = std::max<int64_t>(1, (int64_t)(o.chunk_bytes / (uint64_t)es));
-    std::vector<Chain> chains = make_chains(R, offs, true, granule);
+    std::vector<Chain> chains = make_chains(R, offs, true, granule, (o.flags & HCCL_FLAG_BIDIRECTIONAL) != 0 && !fused);
     int64_t maxlen = 0;
     for (const Chain& ch : chains) maxlen = std::max(maxlen, ch.len);
     if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);

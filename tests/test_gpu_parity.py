@@ -236,3 +236,16 @@ def test_maximum_rank_count(engine):
     orc.alltoallv(Xa, Yw, C, SD, RD, rb)
     for r in range(R):
         assert np.array_equal(Y[r], Yw[r])
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+def test_bidirectional_ring(dt, engine):
+    R, n, granule = 6, 100003, 2048
+    es = hb.ELEM_BYTES[dt]
+    X = synth.normal_ranks(R, n, dt, seed=66)
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, _with(dict(chunk_bytes=granule * es, tile_bytes=4096, sm_budget=32, flags=hb.FLAG_BIDIRECTIONAL), engine))
+    Y = run_plan(p, X, iters=2)
+    so, sc, sd = orc.bidirectional_segments(n, R, granule)
+    want = orc.allreduce_ring_dir_f32(dt, X, so, sc, sd)
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np_dtype(dt)).view(np.uint8), want[r].view(np.uint8)), "rank %d" % r

@@ -386,3 +386,44 @@ def test_two_level_order_is_racks_first():
     # the flat ring adds rank by rank and loses nothing different here? (X1 + X2) + X3 + X0 = ((1 - 2^24) + 1) + 2^24 = 2
     assert orc.allreduce_ring_f32(FP32, X, [0, 1, 2, 3, 4])[0][0] == 2.0
     assert orc.allreduce(FP32, X)[0][0] == 2.0
+
+
+# ------------------------------------------------------------- bidirectional ring order
+@pytest.mark.parametrize("dt", DTYPES)
+def test_bidirectional_ring_order(dt):
+    R, n, granule = 5, 403, 32
+    so, sc, sd = orc.bidirectional_segments(n, R, granule)
+    assert so[0] == 0 and so[-1] == n and np.all(np.diff(so) > 0) and set(sd) == {1, -1}
+    X = synth.small_int_ranks(R, n, dt, seed=8)               # exact: order cannot matter
+    Y = orc.allreduce_ring_dir_f32(dt, X, so, sc, sd)
+    assert np.array_equal(Y[0], orc.allreduce(dt, X)[0]) and np.array_equal(Y[R - 1], Y[0])
+    # all segments forwards = the unidirectional ring
+    X = synth.normal_ranks(R, n, dt, seed=9)
+    fwd = orc.allreduce_ring_dir_f32(dt, X, so, sc, np.ones_like(sd))
+    assert np.array_equal(fwd[0], orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))[0])
+    # backwards on ranks listed in reverse = forwards on the original list (a mirror image of the ring)
+    Xr = X[::-1]
+    scr = (R - 1 - sc)
+    # chunk ranges move with the mirror only if chunks are equal-sized; use one segment per equal chunk
+    n2 = 50 * R
+    X2 = synth.normal_ranks(R, n2, dt, seed=10)
+    so2, sc2, _ = orc.bidirectional_segments(n2, R, 10 ** 9)
+    back = orc.allreduce_ring_dir_f32(dt, X2, so2, sc2, -np.ones_like(sc2))
+    # element i of chunk c backwards: ((X_{c-1}+X_{c-2})+...)+X_c. Mirror ranks r -> R-1-r: chunk c' = R-1-c forwards
+    mirrored = [np.concatenate([x[(R - 1 - c) * 50:(R - c) * 50] for c in range(R)]) for x in X2[::-1]]
+    fwd2 = orc.allreduce_ring_f32(dt, mirrored, orc.floor_chunk_offsets(n2, R))
+    unmirror = np.concatenate([fwd2[0][(R - 1 - c) * 50:(R - c) * 50] for c in range(R)])
+    assert np.array_equal(back[0], unmirror)
+    del Xr, scr
+
+
+def test_bidirectional_order_example():
+    big, one = np.float32(2.0 ** 24), np.float32(1.0)
+    # R = 3, chunk 0, one element. forwards: (X1 + X2) + X0; backwards: (X2 + X1) + X0 -- same pair first, so use
+    # chunk 1: forwards (X2 + X0) + X1, backwards (X0 + X2) + X1: also the same pair. With R = 4, chunk 0:
+    # forwards ((X1 + X2) + X3) + X0, backwards ((X3 + X2) + X1) + X0.
+    X = [np.array([v], dtype=np.float32) for v in (one, big, one, -big)]       # X0..X3
+    so, sc = np.array([0, 1]), np.array([0])
+    f = orc.allreduce_ring_dir_f32(FP32, X, so, sc, np.array([1]))[0][0]      # ((2^24 + 1) - 2^24) + 1 = 0 + 1 = 1
+    b = orc.allreduce_ring_dir_f32(FP32, X, so, sc, np.array([-1]))[0][0]     # ((-2^24 + 1) + 2^24) + 1 = 1 + 1 = 2
+    assert f == 1.0 and b == 2.0

@@ -253,3 +253,26 @@ def test_two_level_allgather_matches_oracle(G, L):
     flat = hb.hccl_plan_allgather(R, cs, 0, hb.BF16, hb.ALGO_RING, dict(SMALL, rack_size=L)).info()
     assert p.info().chain_depth == 1 + (G - 1) + (L - 1) <= flat.chain_depth
     assert p.info().crossrack_bytes < flat.crossrack_bytes
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("R,n", [(4, 1000), (5, 4099), (8, 257)])
+def test_bidirectional_ring_matches_oracle(R, n, dt):
+    es = hb.ELEM_BYTES[dt]
+    granule = 64
+    X = synth.normal_ranks(R, n, dt, seed=R * 3 + n)
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, dict(SMALL, chunk_bytes=granule * es, flags=hb.FLAG_BIDIRECTIONAL))
+    assert p.check_hazards() == 0
+    so, sc, sd = orc.bidirectional_segments(n, R, granule)
+    want = orc.allreduce_ring_dir_f32(dt, X, so, sc, sd)
+    for seed in (0, 1):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            assert np.array_equal(Y[r].view(np_dtype(dt)).view(np.uint8), want[r].view(np.uint8))
+    # reduce-scatter: rank c keeps chunk c of the same sums
+    rs = hb.hccl_plan_reducescatter(R, None, n, dt, hb.ALGO_RING, dict(SMALL, chunk_bytes=granule * es, flags=hb.FLAG_BIDIRECTIONAL))
+    assert rs.check_hazards() == 0
+    offs = orc.floor_chunk_offsets(n, R)
+    Y = interpret(rs, X, 2)
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np_dtype(dt)).view(np.uint8), want[0][offs[r]:offs[r + 1]].view(np.uint8))
