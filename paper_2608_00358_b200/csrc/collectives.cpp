@@ -168,6 +168,12 @@ void fill_ring_opts(hccl_opts_t* o, const hccl_opts_t* in, int64_t input_bytes, 
     hccl_opts_t tmp;
     if (in) tmp = *in; else std::memset(&tmp, 0, sizeof(tmp));
     if (tmp.engine == HCCL_ENGINE_AUTO) tmp.engine = (!fused && input_bytes >= (256ll << 20)) ? HCCL_ENGINE_BULK : HCCL_ENGINE_LSU;
+    // large multi-input sums are pure streams of loads: two 64-register blocks per SM keep twice the loads in
+    // flight (measured 6.06 vs 5.78 TB/s at config 3's size)
+    if (fused && tmp.engine == HCCL_ENGINE_LSU && tmp.sm_budget == 0 && tmp.light == 0 && tmp.threads == 0 && input_bytes >= (256ll << 20)) {
+        tmp.light = 1;
+        tmp.sm_budget = 296;
+    }
     fill_default_opts(o, &tmp);
 }
 
