@@ -95,3 +95,55 @@ def chrome_trace(trace: torch.Tensor, name: str = "hccl") -> dict:
             ev.append({"name": "item %d" % item, "cat": "data", "ph": "X", "pid": name, "tid": block,
                        "ts": (released - t0) / 1e3, "dur": max(stored - released, 0) / 1e3, "args": {"item": item}})
     return {"traceEvents": ev, "displayTimeUnit": "ns"}
+
+
+class PlanCache:
+    """Work-packet cache (paper Sec. V-B): a collective that was compiled and bound once is found again by its
+    arguments and only re-enqueued, so neither generation nor upload is repeated. Keys are the planner's
+    arguments; AllToAllv keys include the count matrix."""
+
+    def __init__(self, device="cuda"):
+        self.device = device
+        self._entries = {}
+        self.hits = 0
+        self.misses = 0
+
+    @staticmethod
+    def _freeze(x):
+        if x is None:
+            return None
+        if isinstance(x, dict):
+            return tuple(sorted(x.items()))
+        if hasattr(x, "tobytes"):
+            return (getattr(x, "shape", None), x.tobytes())
+        if isinstance(x, (list, tuple)):
+            return tuple(PlanCache._freeze(v) for v in x)
+        return x
+
+    def _get(self, key, make):
+        ent = self._entries.get(key)
+        if ent is None:
+            self.misses += 1
+            ent = DeviceCollective(make(), device=self.device)
+            self._entries[key] = ent
+        else:
+            self.hits += 1
+        return ent
+
+    def allreduce(self, R, count, dt, algo=hb.ALGO_RING, opts=None) -> DeviceCollective:
+        return self._get(("allreduce", R, count, dt, algo, self._freeze(opts)), lambda: hb.hccl_plan_allreduce(R, count, dt, algo, opts))
+
+    def reducescatter(self, R, recvcounts, count, dt, algo=hb.ALGO_RING, opts=None) -> DeviceCollective:
+        return self._get(("reducescatter", R, self._freeze(recvcounts), count, dt, algo, self._freeze(opts)),
+                         lambda: hb.hccl_plan_reducescatter(R, recvcounts, count, dt, algo, opts))
+
+    def allgather(self, R, sendcounts, count, dt, algo=hb.ALGO_RING, opts=None) -> DeviceCollective:
+        return self._get(("allgather", R, self._freeze(sendcounts), count, dt, algo, self._freeze(opts)),
+                         lambda: hb.hccl_plan_allgather(R, sendcounts, count, dt, algo, opts))
+
+    def alltoallv(self, R, sendcounts, sdispls=None, rdispls=None, dt=hb.BF16, row_elems=1, opts=None) -> DeviceCollective:
+        key = ("alltoallv", R, self._freeze(sendcounts), self._freeze(sdispls), self._freeze(rdispls), dt, row_elems, self._freeze(opts))
+        return self._get(key, lambda: hb.hccl_plan_alltoallv(R, sendcounts, sdispls, None, rdispls, dt, row_elems, opts))
+
+    def __len__(self):
+        return len(self._entries)

@@ -249,3 +249,23 @@ def test_bidirectional_ring(dt, engine):
     want = orc.allreduce_ring_dir_f32(dt, X, so, sc, sd)
     for r in range(R):
         assert np.array_equal(Y[r].view(np_dtype(dt)).view(np.uint8), want[r].view(np.uint8)), "rank %d" % r
+
+
+def test_plan_cache_reuses_bound_plans():
+    import torch
+    from paper_2608_00358_b200.runtime import PlanCache
+    cache = PlanCache()
+    C = synth.uniform_counts(4, 1, hi=50)
+    a = cache.alltoallv(4, C, dt=hb.FP16, row_elems=32)
+    b = cache.alltoallv(4, C.copy(), dt=hb.FP16, row_elems=32)
+    c = cache.alltoallv(4, C + 1, dt=hb.FP16, row_elems=32)
+    assert a is b and a is not c and (cache.hits, cache.misses, len(cache)) == (1, 2, 2)
+    r1 = cache.allreduce(4, 1000, hb.BF16, hb.ALGO_ONESHOT, dict(sm_budget=8))
+    assert cache.allreduce(4, 1000, hb.BF16, hb.ALGO_ONESHOT, dict(sm_budget=8)) is r1
+    X = synth.normal_ranks(4, 1000, hb.BF16, seed=0)
+    send = [torch.from_numpy(x.view(np.int16)).cuda() for x in X]
+    recv = [torch.zeros(1000, dtype=torch.int16, device="cuda") for _ in range(4)]
+    r1.set_buffers([t.data_ptr() for t in send], [t.data_ptr() for t in recv])
+    r1.execute()
+    r1.check()
+    assert np.array_equal(recv[2].cpu().numpy().view(np.uint16), orc.allreduce_oneshot_f32(hb.BF16, X)[2])
