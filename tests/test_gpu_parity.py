@@ -269,3 +269,26 @@ def test_plan_cache_reuses_bound_plans():
     r1.execute()
     r1.check()
     assert np.array_equal(recv[2].cpu().numpy().view(np.uint16), orc.allreduce_oneshot_f32(hb.BF16, X)[2])
+
+
+@pytest.mark.parametrize("opts", [dict(engine=hb.ENGINE_BULK, stages=2), dict(engine=hb.ENGINE_BULK, stages=3, threads=64),
+                                  dict(engine=hb.ENGINE_BULK, threads=512, copy_by_warps=2), dict(engine=hb.ENGINE_LSU, threads=64),
+                                  dict(engine=hb.ENGINE_LSU, threads=96, cluster=2), dict(engine=hb.ENGINE_LSU, light=1, threads=512, cluster=4)],
+                         ids=["bulk2", "bulk3_64", "bulk512_tmastore", "lsu64", "lsu96_cluster2", "light512_cluster4"])
+def test_engine_geometry_variants(opts):
+    R, n, dt = 4, 300007, hb.BF16
+    X = synth.normal_ranks(R, n, dt, seed=12)
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, dict(opts, sm_budget=24))
+    Y = run_plan(p, X, iters=2)
+    want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np.uint16), want[r])
+    C = synth.uniform_counts(R, 5, hi=3000)
+    SD, RD = orc.packed_displs(C)
+    Xa = [synth.hashed_rows_np(s, 0, int(C[s].sum()), 64).reshape(-1).view(np.uint8) for s in range(R)]
+    pa = hb.hccl_plan_alltoallv(R, C, None, None, None, hb.FP16, 64, dict(opts, sm_budget=24))
+    Ya = run_plan(pa, Xa, iters=2)
+    Yw = [np.full(pa.extents(r)[1], 0xA5, dtype=np.uint8) for r in range(R)]
+    orc.alltoallv(Xa, Yw, C, SD, RD, 128)
+    for r in range(R):
+        assert np.array_equal(Ya[r], Yw[r])
