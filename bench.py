@@ -174,14 +174,36 @@ def side_configs(quick: bool):
         cold = wk.time_each(wl, 50, 5, flush=flush_buf)
         out[key]["p50_us_cold_l2"] = float(np.percentile(cold, 50) * 1e3)
 
-    latency(wk.config1(), "1_allreduce_ring_r4_fp32_1Mi")
-    latency(wk.config2(), "2_alltoallv_r8_bf16_dim128")
+    # the CPU oracle on the same inputs (one core, as it stands): a baseline, not a target
+    import time as _t
+    from oracle import oracle as orc
+
+    def oracle_time(key, fn):
+        t0 = _t.perf_counter()
+        fn()
+        out[key]["cpu_oracle_ms"] = (_t.perf_counter() - t0) * 1e3
+
+    w1 = wk.config1()
+    latency(w1, "1_allreduce_ring_r4_fp32_1Mi")
+    oracle_time("1_allreduce_ring_r4_fp32_1Mi", lambda: orc.allreduce(hb.FP32, w1.meta["host_inputs"]))
+    w2 = wk.config2()
+    latency(w2, "2_alltoallv_r8_bf16_dim128")
+
+    def _oracle_a2a():
+        C = w2.meta["counts"]
+        sd, rd = orc.packed_displs(C)
+        X = [x.view(np.uint8) for x in w2.meta["host_inputs"]]
+        Y = [np.empty(int(C[:, d].sum()) * 256, dtype=np.uint8) for d in range(8)]
+        orc.alltoallv(X, Y, C, sd, rd, 256)
+    oracle_time("2_alltoallv_r8_bf16_dim128", _oracle_a2a)
+    del w1, w2
     for m in (4096, 65536, 262144, 1 << 20):
         for algo, nm in ((hb.ALGO_ONESHOT, "oneshot"), (hb.ALGO_RING, "ring")):
             wl5 = wk.config5(m, algo)
             key5 = "5_allreduce_r8_bf16_%dB_%s" % (m, nm)
             latency(wl5, key5)
             if algo == hb.ALGO_ONESHOT:
+                oracle_time(key5, lambda: orc.allreduce(hb.BF16, wl5.meta["host_inputs"]))
                 out[key5]["host_observed"] = wk.time_host_observed(wl5, 100 if quick else 300)
     # host side of the compiled-communication model (Sec. V-B): generating the description, uploading it,
     # and re-enqueueing a cached one; plus the device-resident AllToAllv, where the counts never visit the host
