@@ -600,26 +600,27 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     std::vector<int32_t> sg(R);
     std::vector<int64_t> last(R, -1);
     for (int q = 0; q < R; ++q) CHECK(hccl_graph_add_subgraph(g.get(), q, &sg[q]));
-    const int steps = R;  // step 0: own copy; steps 1..R-1: hops
-    for (int u = 0; u < steps; ++u) {
-        for (int q = 0; q < R; ++q) {
-            const int64_t bytes = (offs[q + 1] - offs[q]) * es;
-            if (bytes == 0) continue;
-            hccl_wqe_t w = blank();
-            w.op = HCCL_OP_COPY;
-            w.count = bytes;
-            w.tile_count = tile;
-            const int dst_rank = (q + u) % R;
-            w.dst = ref(HCCL_BUF_RECV, dst_rank, offs[q] * es);
-            if (u == 0 || algo == HCCL_ALGO_ONESHOT) {
-                w.a = ref(HCCL_BUF_SEND, q, 0);
-            } else {
-                w.a = ref(HCCL_BUF_RECV, (q + u - 1) % R, offs[q] * es);
-                w.dep_flags = HCCL_DEP_WQE_SYNC | HCCL_DEP_ELEMENTWISE;
-                w.dep_wqe = last[q];
-            }
-            CHECK(hccl_graph_add_wqe(g.get(), sg[q], &w, &last[q]));
+    // Ring: step-major issue order (step 0: own copy; steps 1..R-1: hops). One-shot: chunk-major, so that
+    // the R reads of one chunk follow one another while it is still in the L2.
+    const bool oneshot = algo == HCCL_ALGO_ONESHOT;
+    for (int i = 0; i < R * R; ++i) {
+        const int u = oneshot ? i % R : i / R, q = oneshot ? i / R : i % R;
+        const int64_t bytes = (offs[q + 1] - offs[q]) * es;
+        if (bytes == 0) continue;
+        hccl_wqe_t w = blank();
+        w.op = HCCL_OP_COPY;
+        w.count = bytes;
+        w.tile_count = tile;
+        const int dst_rank = (q + u) % R;
+        w.dst = ref(HCCL_BUF_RECV, dst_rank, offs[q] * es);
+        if (u == 0 || oneshot) {
+            w.a = ref(HCCL_BUF_SEND, q, 0);
+        } else {
+            w.a = ref(HCCL_BUF_RECV, (q + u - 1) % R, offs[q] * es);
+            w.dep_flags = HCCL_DEP_WQE_SYNC | HCCL_DEP_ELEMENTWISE;
+            w.dep_wqe = last[q];
         }
+        CHECK(hccl_graph_add_wqe(g.get(), sg[q], &w, &last[q]));
     }
     return hccl_graph_compile(g.get(), &o, out);
 }
