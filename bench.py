@@ -198,7 +198,7 @@ def side_configs(quick: bool):
     oracle_time("2_alltoallv_r8_bf16_dim128", _oracle_a2a)
     del w1, w2
     for m in (4096, 65536, 262144, 1 << 20):
-        for algo, nm in ((hb.ALGO_ONESHOT, "oneshot"), (hb.ALGO_RING, "ring")):
+        for algo, nm in ((hb.ALGO_ONESHOT, "oneshot"), (hb.ALGO_RING, "ring"), (hb.ALGO_FANOUT, "fanout")):
             wl5 = wk.config5(m, algo)
             key5 = "5_allreduce_r8_bf16_%dB_%s" % (m, nm)
             latency(wl5, key5)
@@ -260,7 +260,7 @@ def side_configs(quick: bool):
     for n in ((1 << 12, 1 << 18) if quick else (1 << 12, 1 << 18, 1 << 21)):
         send = [torch.randn(n, device="cuda").to(torch.bfloat16) for _ in range(128)]
         recv = [torch.empty(n * 128, dtype=torch.bfloat16, device="cuda") for _ in range(128)]
-        for algo, nm in ((hb.ALGO_RING, "ring"), (hb.ALGO_RING_2LEVEL, "ring_2level"), (hb.ALGO_ONESHOT, "oneshot")):
+        for algo, nm in ((hb.ALGO_RING, "ring"), (hb.ALGO_RING_2LEVEL, "ring_2level"), (hb.ALGO_ONESHOT, "oneshot"), (hb.ALGO_FANOUT, "fanout")):
             sched("next_allgather_r128_bf16_%d_%s" % (n, nm), hb.hccl_plan_allgather(128, None, n, hb.BF16, algo, dict(rack_size=16)), send, recv, 10)
         del send, recv
         torch.cuda.empty_cache()

@@ -67,10 +67,15 @@ typedef enum {
     HCCL_ALGO_RING_FUSED = 2,/* the ring's sums in the ring's order, but each chunk's chain collapsed into
                                 one multi-input reduction (cf. NOOP-joined tree reductions, Sec. III-B.2).
                                 Reported as its own algorithm, never as "ring". */
-    HCCL_ALGO_RING_2LEVEL = 3 /* topology-aware two-level ring (Sec. V-D): ranks form racks of opts.rack_size; sums
+    HCCL_ALGO_RING_2LEVEL = 3,/* topology-aware two-level ring (Sec. V-D): ranks form racks of opts.rack_size; sums
                                 run round each rack's ring first, then round the ring of racks, and results
                                 are gathered across racks first, then inside each rack, so that only 1/rack_size
                                 of the data ever crosses between racks. AllReduce and AllGather. */
+    HCCL_ALGO_FANOUT = 4     /* one-shot with the destinations fused: each piece of the result is produced once
+                                (AllReduce: one sum over all ranks in rank order 0..R-1, the one-shot's order;
+                                AllGather: one read of the chunk) and written into all R receive buffers by the
+                                same work item. Possible only because the virtual ranks share one memory; not in
+                                the paper. Reported as its own algorithm, never as "one-shot". */
 } hccl_algo_t;
 
 /* Which data mover the executor uses for aligned bulk work. */
@@ -186,7 +191,11 @@ typedef enum {
     HCCL_OP_REDUCE = 1,   /* dst[i] = round(f32(a[i]) + f32(b[i])), count in ELEMENTS; dst may alias a or b
                              exactly (A=A+B, B=A+B) or be separate (S=A+B) */
     HCCL_OP_REDUCE_N = 2, /* dst[i] = round(((f32(a_0[i]) + f32(a_1[i])) + ...) + f32(a_{nsrc-1}[i])) where a_k is
-                             buffer a.kind of rank (a.rank + k) mod R at byte offset a.offset */
+                             buffer a.kind of rank (a.rank + k) mod R at byte offset a.offset.
+                             COPY and REDUCE_N may name several destinations (ndst > 1): the same bytes are then
+                             written at dst.offset into the receive buffer of every rank (dst.rank + k) mod R,
+                             k < ndst, from one read of the sources. The NMC of the paper has no such form (its ranks do
+                             not share a memory); here it plays the part a multicast in the switch plays. */
     HCCL_OP_WAIT = 3,     /* block until signal slot a.offset compares true against value (+ epoch*value_per_epoch) */
     HCCL_OP_SET = 4,      /* store value (+ epoch*value_per_epoch) to signal slot dst.offset */
     HCCL_OP_NOOP = 5      /* nothing; exists to carry dependencies */
@@ -238,6 +247,8 @@ typedef struct {
     int64_t dep_wqe2;                 /* optional second WQE_SYNC target, -1 if unused */
     int32_t cmp;                      /* WAIT: hccl_cmp_t */
     int32_t hints;                    /* data WQEs: HCCL_HINT_* */
+    int32_t ndst;                     /* COPY, REDUCE_N: number of destinations, 0 or 1 = one; > 1 needs dst.kind RECV */
+    int32_t reserved;                 /* 0 */
     int64_t tile_count;               /* tile size in units of count; 0 = derived from opts.tile_bytes */
     uint64_t value, value_per_epoch;  /* WAIT/SET: effective value = value + epoch*value_per_epoch, epoch = 1,2,.. per execute */
 } hccl_wqe_t;

@@ -15,7 +15,7 @@ from . import _build
 OK, ERR_INVALID_ARG, ERR_DTYPE, ERR_COUNT_MISMATCH, ERR_OVERLAP, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_BUSY, \
     ERR_CUDA, ERR_TIMEOUT, ERR_BAD_DESCRIPTOR, ERR_NOT_BOUND, ERR_HAZARD = range(13)
 FP32, BF16, FP16 = 0, 1, 2
-ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED, ALGO_RING_2LEVEL = 0, 1, 2, 3
+ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED, ALGO_RING_2LEVEL, ALGO_FANOUT = 0, 1, 2, 3, 4
 ENGINE_AUTO, ENGINE_LSU, ENGINE_BULK = 0, 1, 2
 FLAG_LEVEL_MAJOR, FLAG_CHECK_HAZARDS, FLAG_STAGED_RING, FLAG_BIDIRECTIONAL = 1, 2, 4, 8
 OP_COPY, OP_REDUCE, OP_REDUCE_N, OP_WAIT, OP_SET, OP_NOOP = range(6)
@@ -43,7 +43,7 @@ class Wqe(C.Structure):
     _fields_ = [("op", C.c_int32), ("dtype_dst", C.c_int32), ("dtype_a", C.c_int32), ("dtype_b", C.c_int32),
                 ("dst", Ref), ("a", Ref), ("b", Ref), ("count", C.c_int64), ("nsrc", C.c_int32),
                 ("dep_flags", C.c_uint32), ("dep_wqe", C.c_int64), ("dep_wqe2", C.c_int64), ("cmp", C.c_int32),
-                ("hints", C.c_int32), ("tile_count", C.c_int64), ("value", C.c_uint64),
+                ("hints", C.c_int32), ("ndst", C.c_int32), ("reserved", C.c_int32), ("tile_count", C.c_int64), ("value", C.c_uint64),
                 ("value_per_epoch", C.c_uint64)]
 
 
@@ -316,7 +316,7 @@ class Graph:
 
     def add_wqe(self, subgraph: int, op: int, dst=None, a=None, b=None, count: int = 0, dtypes=(FP32, FP32, FP32),
                 nsrc: int = 0, dep_flags: int = 0, dep_wqe: int = -1, dep_wqe2: int = -1, cmp: int = 0,
-                value: int = 0, value_per_epoch: int = 0, tile_count: int = 0, hints: int = 0) -> int:
+                value: int = 0, value_per_epoch: int = 0, tile_count: int = 0, hints: int = 0, ndst: int = 0) -> int:
         w = Wqe()
         w.op = op
         w.dtype_dst, w.dtype_a, w.dtype_b = dtypes
@@ -325,6 +325,7 @@ class Graph:
                 setattr(w, name, Ref(*r))
         w.count, w.nsrc, w.dep_flags, w.dep_wqe, w.dep_wqe2 = count, nsrc, dep_flags, dep_wqe, dep_wqe2
         w.cmp, w.value, w.value_per_epoch, w.tile_count, w.hints = cmp, value, value_per_epoch, tile_count, hints
+        w.ndst = ndst
         wid = C.c_int64()
         _chk(_lib.hccl_graph_add_wqe(self._h, subgraph, C.byref(w), C.byref(wid)), "hccl_graph_add_wqe")
         return wid.value

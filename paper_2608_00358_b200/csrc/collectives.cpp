@@ -439,9 +439,10 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
                                   hccl_plan_t** out) {
     if (!out || R < 1 || R > HCCL_MAX_RANKS || count < 0) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
-    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_RING_2LEVEL) return HCCL_ERR_INVALID_ARG;
+    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_RING_2LEVEL &&
+        algo != HCCL_ALGO_FANOUT) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
-    fill_ring_opts(&o, opts, (int64_t)R * count * elem_bytes(dt), algo == HCCL_ALGO_RING_FUSED || algo == HCCL_ALGO_ONESHOT || R == 1);
+    fill_ring_opts(&o, opts, (int64_t)R * count * elem_bytes(dt), algo == HCCL_ALGO_RING_FUSED || algo == HCCL_ALGO_ONESHOT || algo == HCCL_ALGO_FANOUT || R == 1);
     if (algo == HCCL_ALGO_RING_2LEVEL) {
         if (R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
         // a single rack, or racks of one rank, is the flat ring
@@ -453,6 +454,26 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     std::vector<int64_t> ext(R, count * es);
     const int64_t compulsory = 2ll * R * count * es;
 
+    if (R > 1 && algo == HCCL_ALGO_FANOUT) {
+        // one sum per element, in the one-shot's order, stored into every receive buffer by the work item that formed it
+        hccl_graph* graw = nullptr;
+        CHECK(hccl_graph_create(R, ext.data(), ext.data(), 0, 0, &graw));
+        GraphPtr g(graw);
+        g->compulsory_bytes = compulsory;
+        int32_t sg;
+        CHECK(hccl_graph_add_subgraph(g.get(), 0, &sg));
+        hccl_wqe_t w = blank();
+        w.op = HCCL_OP_REDUCE_N;
+        w.dtype_dst = w.dtype_a = dt;
+        w.count = count;
+        w.nsrc = R;
+        w.ndst = R;
+        w.hints = HCCL_HINT_READ_ONCE;
+        w.a = ref(HCCL_BUF_SEND, 0, 0);
+        w.dst = ref(HCCL_BUF_RECV, 0, 0);
+        CHECK(hccl_graph_add_wqe(g.get(), sg, &w, nullptr));
+        return hccl_graph_compile(g.get(), &o, out);
+    }
     if (R == 1 || algo == HCCL_ALGO_ONESHOT) {
         hccl_graph* graw = nullptr;
         CHECK(hccl_graph_create(R, ext.data(), ext.data(), 0, 0, &graw));
@@ -573,7 +594,7 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
                                   const hccl_opts_t* opts, hccl_plan_t** out) {
     if (!out || R < 1 || R > HCCL_MAX_RANKS || count < 0) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
-    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_2LEVEL) return HCCL_ERR_INVALID_ARG;
+    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_2LEVEL && algo != HCCL_ALGO_FANOUT) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
     fill_copy_opts(&o, opts);
     const int es = elem_bytes(dt);
@@ -600,27 +621,50 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     std::vector<int32_t> sg(R);
     std::vector<int64_t> last(R, -1);
     for (int q = 0; q < R; ++q) CHECK(hccl_graph_add_subgraph(g.get(), q, &sg[q]));
-    // Ring: step-major issue order (step 0: own copy; steps 1..R-1: hops). One-shot: chunk-major, so that
-    // the R reads of one chunk follow one another while it is still in the L2.
-    const bool oneshot = algo == HCCL_ALGO_ONESHOT;
-    for (int i = 0; i < R * R; ++i) {
-        const int u = oneshot ? i % R : i / R, q = oneshot ? i / R : i % R;
-        const int64_t bytes = (offs[q + 1] - offs[q]) * es;
-        if (bytes == 0) continue;
-        hccl_wqe_t w = blank();
-        w.op = HCCL_OP_COPY;
-        w.count = bytes;
-        w.tile_count = tile;
-        const int dst_rank = (q + u) % R;
-        w.dst = ref(HCCL_BUF_RECV, dst_rank, offs[q] * es);
-        if (u == 0 || oneshot) {
+    if (algo == HCCL_ALGO_FANOUT) {  // chunk q: one read, R writes
+        // a work item writes R times what it reads, so its tiles are small: a third of a stage at most
+        const int64_t ftile = o.tile_bytes ? (int64_t)o.tile_bytes : default_tile(offs[R] * es, o.sm_budget, 4, 8 << 10, 16 << 10, 64);
+        for (int q = 0; q < R; ++q) {
+            const int64_t bytes = (offs[q + 1] - offs[q]) * es;
+            if (bytes == 0) continue;
+            hccl_wqe_t w = blank();
+            w.op = HCCL_OP_COPY;
+            w.count = bytes;
+            w.tile_count = ftile;
+            w.ndst = R;
             w.a = ref(HCCL_BUF_SEND, q, 0);
-        } else {
-            w.a = ref(HCCL_BUF_RECV, (q + u - 1) % R, offs[q] * es);
-            w.dep_flags = HCCL_DEP_WQE_SYNC | HCCL_DEP_ELEMENTWISE;
-            w.dep_wqe = last[q];
+            w.dst = ref(HCCL_BUF_RECV, q, offs[q] * es);
+            CHECK(hccl_graph_add_wqe(g.get(), sg[q], &w, nullptr));
         }
-        CHECK(hccl_graph_add_wqe(g.get(), sg[q], &w, &last[q]));
+        return hccl_graph_compile(g.get(), &o, out);
+    }
+    // Issue order. One-shot: chunk-major (groups of one chunk), so that the R reads of a chunk follow one another
+    // while it is still in the L2. Ring: step-major over all chunks (step 0: own copy; steps 1..R-1: hops).
+    // Smaller ring groups would let a hop find the previous hop's bytes in the L2, but then every work item
+    // meets an unfinished predecessor; measured at R = 128 that costs more than the DRAM reads it saves.
+    const bool oneshot = algo == HCCL_ALGO_ONESHOT;
+    const int G = oneshot ? 1 : R;
+    for (int q0 = 0; q0 < R; q0 += G) {
+        for (int u = 0; u < R; ++u) {
+            for (int q = q0; q < std::min(R, q0 + G); ++q) {
+                const int64_t bytes = (offs[q + 1] - offs[q]) * es;
+                if (bytes == 0) continue;
+                hccl_wqe_t w = blank();
+                w.op = HCCL_OP_COPY;
+                w.count = bytes;
+                w.tile_count = tile;
+                const int dst_rank = (q + u) % R;
+                w.dst = ref(HCCL_BUF_RECV, dst_rank, offs[q] * es);
+                if (u == 0 || oneshot) {
+                    w.a = ref(HCCL_BUF_SEND, q, 0);
+                } else {
+                    w.a = ref(HCCL_BUF_RECV, (q + u - 1) % R, offs[q] * es);
+                    w.dep_flags = HCCL_DEP_WQE_SYNC | HCCL_DEP_ELEMENTWISE;
+                    w.dep_wqe = last[q];
+                }
+                CHECK(hccl_graph_add_wqe(g.get(), sg[q], &w, &last[q]));
+            }
+        }
     }
     return hccl_graph_compile(g.get(), &o, out);
 }

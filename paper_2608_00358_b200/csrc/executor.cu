@@ -295,6 +295,51 @@ __device__ void copy_tile_lsu(char* dst, const char* src, uint32_t n, const uint
     }
 }
 
+// COPY with several destinations: every byte is read once and stored into the receive buffer of each of the
+// nd ranks r0, r0+1, ... (mod R) at byte offset doff. Vector path when the source and all destinations
+// share their position inside a 16-byte word; otherwise one plain copy per destination.
+template <bool STREAM>
+__device__ void copy_tile_fanout(const ExecParams& p, const char* src, int r0, int nd, size_t doff, uint32_t n, const uint32_t tid, const uint32_t nth) {
+    const int R = (int)p.R;
+    auto dst = [&](int k) -> char* {
+        int r = r0 + k;
+        if (r >= R) r -= R;
+        return (char*)p.recv[r] + doff;
+    };
+    const uintptr_t sa = (uintptr_t)src;
+    bool vec = true;
+    for (int k = 0; k < nd; ++k) vec = vec && ((((uintptr_t)dst(k)) ^ sa) & 15u) == 0;
+    if (!vec) {
+        for (int k = 0; k < nd; ++k) copy_tile_lsu<false>(dst(k), src, n, tid, nth);
+        return;
+    }
+    uint32_t head = (uint32_t)((16u - (sa & 15u)) & 15u);
+    if (head > n) head = n;
+    const uint32_t nv = (n - head) >> 4, done = head + (nv << 4);
+    for (uint32_t i = tid; i < head + (n - done); i += nth) {
+        const uint32_t j = i < head ? i : done + (i - head);
+        const char b = __ldcg(src + j);
+        for (int k = 0; k < nd; ++k) dst(k)[j] = b;
+    }
+    const uint4* s = (const uint4*)(src + head);
+    constexpr int U = 4;
+    uint32_t base = 0;
+    for (; base + U * nth <= nv; base += U * nth) {
+        uint4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) v[u] = STREAM ? __ldcs(s + base + u * nth + tid) : __ldcg(s + base + u * nth + tid);
+        for (int k = 0; k < nd; ++k) {
+            uint4* d = (uint4*)(dst(k) + head) + base + tid;
+#pragma unroll
+            for (int u = 0; u < U; ++u) __stcs(d + u * nth, v[u]);
+        }
+    }
+    for (uint32_t i = base + tid; i < nv; i += nth) {
+        const uint4 v = STREAM ? __ldcs(s + i) : __ldcg(s + i);
+        for (int k = 0; k < nd; ++k) __stcs((uint4*)(dst(k) + head) + i, v);
+    }
+}
+
 // ------------------------------------------------------------------ REDUCE (S=A+B and in-place forms)
 template <int DA, int DB, int DD, bool STREAM_B>
 __device__ void reduce_tile_lsu(char* dst, const char* a, const char* b, uint32_t n, const uint32_t tid, const uint32_t nth) {
@@ -366,7 +411,16 @@ template <int DS, int DD>
 __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start, uint32_t n, const uint32_t tid, const uint32_t nth) {
     const int R = (int)p.R, nsrc = d.nsrc, r0 = d.rank_a;
     const size_t soff = (size_t)d.off_a + start * Elem<DS>::BYTES;
-    char* dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + start * Elem<DD>::BYTES;
+    // destinations: one, or the receive buffers of nd consecutive ranks at the same offset
+    const int nd = d.ndst > 1 ? d.ndst : 1, rd0 = d.rank_dst;
+    const size_t doff = (size_t)d.off_dst + start * Elem<DD>::BYTES;
+    char* const dst0 = buf_base(p, d.kind_dst, d.rank_dst) + doff;
+    auto dstp = [&](int j) -> char* {
+        if (j == 0) return dst0;
+        int r = rd0 + j;
+        if (r >= R) r -= R;
+        return (char*)p.recv[r] + doff;
+    };
     const bool from_send = d.kind_a == HCCL_BUF_SEND;
     auto src = [&](int k) -> const char* {
         int r = r0 + k;
@@ -374,14 +428,15 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
         return (const char*)(from_send ? p.send[r] : (const void*)p.recv[r]) + soff;
     };
     // same phase for every operand?
-    const uint32_t pd = (uint32_t)(((uintptr_t)dst / Elem<DD>::BYTES) & 7u);
+    const uint32_t pd = (uint32_t)(((uintptr_t)dst0 / Elem<DD>::BYTES) & 7u);
     bool vec = true;
     for (int k = 0; k < nsrc; ++k) vec = vec && ((uint32_t)(((uintptr_t)src(k) / Elem<DS>::BYTES) & 7u) == pd);
+    for (int j = 1; j < nd; ++j) vec = vec && ((uint32_t)(((uintptr_t)dstp(j) / Elem<DD>::BYTES) & 7u) == pd);
     if (!vec) {
         for (uint32_t i = tid; i < n; i += nth) {
             float acc = Elem<DS>::load(src(0), i);
             for (int k = 1; k < nsrc; ++k) acc = acc + Elem<DS>::load(src(k), i);
-            Elem<DD>::store(dst, i, acc);
+            for (int j = 0; j < nd; ++j) Elem<DD>::store(dstp(j), i, acc);
         }
         return;
     }
@@ -391,7 +446,7 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
     auto scalar = [&](uint32_t i) {
         float acc = Elem<DS>::load(src(0), i);
         for (int k = 1; k < nsrc; ++k) acc = acc + Elem<DS>::load(src(k), i);
-        Elem<DD>::store(dst, i, acc);
+        for (int j = 0; j < nd; ++j) Elem<DD>::store(dstp(j), i, acc);
     };
     if (tid < head) scalar(tid);
     for (uint32_t i = head + (nv << 3) + tid; i < n; i += nth) scalar(i);
@@ -453,7 +508,9 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
         else { group(std::integral_constant<int, 1>{}, T{}, 0, off, acc); k = 1; }
         for (; k + G <= nsrc; k += G) group(std::integral_constant<int, G>{}, F{}, k, off, acc);
         for (; k < nsrc; ++k) group(std::integral_constant<int, 1>{}, F{}, k, off, acc);
-        store8<DD, false>(dst + (size_t)head * Elem<DD>::BYTES + (size_t)i * 8 * Elem<DD>::BYTES, acc);
+        const size_t o = (size_t)head * Elem<DD>::BYTES + (size_t)i * 8 * Elem<DD>::BYTES;
+        store8<DD, false>(dst0 + o, acc);
+        for (int j = 1; j < nd; ++j) store8<DD, false>(dstp(j) + o, acc);
     }
 }
 
@@ -473,8 +530,13 @@ __device__ void reduce_n_dispatch(const ExecParams& p, const Desc& d, uint64_t s
 __device__ void run_tile_lsu(const ExecParams& p, const Desc& d, const Tile& t, const uint32_t tid, const uint32_t nth) {
     switch (d.op) {
         case HCCL_OP_COPY: {
-            char* dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + t.start;
             const char* src = buf_base(p, d.kind_a, d.rank_a) + d.off_a + t.start;
+            if (d.ndst > 1) {
+                if (d.kind_a == HCCL_BUF_SEND) copy_tile_fanout<true>(p, src, d.rank_dst, d.ndst, (size_t)d.off_dst + t.start, t.count, tid, nth);
+                else copy_tile_fanout<false>(p, src, d.rank_dst, d.ndst, (size_t)d.off_dst + t.start, t.count, tid, nth);
+                break;
+            }
+            char* dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + t.start;
             // send-to-receive copies (AllToAllv, AllGather's first hop) are read once and written once
             if (d.kind_a == HCCL_BUF_SEND) copy_tile_lsu<true>(dst, src, t.count, tid, nth); else copy_tile_lsu<false>(dst, src, t.count, tid, nth);
             break;
@@ -512,6 +574,7 @@ __device__ bool desc_ok(const ExecParams& p, const Desc& d) {
         if (d.op == HCCL_OP_REDUCE && (d.kind_b > HCCL_BUF_SCRATCH || d.rank_b >= p.R)) return false;
         if (d.op != HCCL_OP_COPY && (d.dt_dst > HCCL_FP16 || d.dt_a > HCCL_FP16 || (d.op == HCCL_OP_REDUCE && d.dt_b > HCCL_FP16))) return false;
         if (d.op == HCCL_OP_REDUCE_N && (d.nsrc < 1 || d.nsrc > p.R || d.kind_a > HCCL_BUF_RECV)) return false;
+        if (d.op != HCCL_OP_REDUCE && d.ndst > 1 && (d.ndst > p.R || d.kind_dst != HCCL_BUF_RECV)) return false;
     }
     if (d.op == HCCL_OP_WAIT) {
         if (d.kind_a == HCCL_BUF_SIGNAL) return (uint64_t)d.off_a < p.n_signals;
@@ -767,6 +830,8 @@ struct alignas(16) PieceInfo {  // one per stage, in shared memory; written by t
     int32_t signal[2];
     uint8_t dt_a, dt_b, dt_d, evict_first;
     uint32_t b_off;       // REDUCE: byte offset of operand B inside the stage
+    uint16_t ndst, rank_dst;   // COPY with several destinations: receive buffers of ranks rank_dst .. +ndst-1 (mod R)
+    unsigned long long dst_off;  // ... at this byte offset (dst is then the first of them)
     Tile tile;            // PIECE_TILE: the work item and its descriptor for the register path
     Desc desc;
 };
@@ -817,13 +882,17 @@ __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, u
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(smem_dst), "l"(gsrc), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void bulk_store(void* gdst, uint32_t smem_src, uint32_t bytes, bool hint, unsigned long long pol) {
+__device__ __forceinline__ void bulk_store_part(void* gdst, uint32_t smem_src, uint32_t bytes, bool hint, unsigned long long pol) {
     if (hint)
         asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
                      ::"l"(gdst), "r"(smem_src), "r"(bytes), "l"(pol) : "memory");
     else
         asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_store(void* gdst, uint32_t smem_src, uint32_t bytes, bool hint, unsigned long long pol) {
+    bulk_store_part(gdst, smem_src, bytes, hint, pol);
+    bulk_commit();
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Wait until at most `pending` of the most recent store groups are still reading shared memory.
@@ -934,7 +1003,16 @@ __device__ void retire_one(const ExecParams& p, Dma& d) {
     if (pi.kind == PIECE_COPY) {
         if (!mbar_wait(p, d.full + 8 * slot, parity, p.timeout_ns, pi.tile_index)) d.ok = false;
         if (d.ok) {
-            bulk_store(pi.dst, d.stages + slot * STAGE_BYTES, pi.n, pi.evict_first != 0, d.pol);
+            if (pi.ndst > 1) {  // one stage, several stores, one group
+                for (uint32_t k = 0; k < pi.ndst; ++k) {
+                    uint32_t r = pi.rank_dst + k;
+                    if (r >= p.R) r -= p.R;
+                    bulk_store_part((char*)p.recv[r] + pi.dst_off, d.stages + slot * STAGE_BYTES, pi.n, pi.evict_first != 0, d.pol);
+                }
+                bulk_commit();
+            } else {
+                bulk_store(pi.dst, d.stages + slot * STAGE_BYTES, pi.n, pi.evict_first != 0, d.pol);
+            }
             pi.group = d.groups++;
             if (pi.last && p.trace) trace_put(p.trace, p.trace_cap, pi.tile_index, 3, globaltimer_ns());
             if (pi.last && (pi.signal[0] >= 0 || pi.signal[1] >= 0)) {
@@ -1047,14 +1125,27 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
         case HCCL_OP_COPY: {
             char* dst = buf_base(p, ds.kind_dst, ds.rank_dst) + ds.off_dst + t.start;
             const char* src = buf_base(p, ds.kind_a, ds.rank_a) + ds.off_a + t.start;
-            if ((((uintptr_t)dst | (uintptr_t)src) & 15u) != 0 || t.count < 16) {
+            const uint32_t nd = ds.ndst > 1 ? ds.ndst : 1;
+            const unsigned long long doff = (unsigned long long)ds.off_dst + t.start;
+            auto dstk = [&](uint32_t k) -> char* {
+                uint32_t r = ds.rank_dst + k;
+                if (r >= p.R) r -= p.R;
+                return (char*)p.recv[r] + doff;
+            };
+            uintptr_t bits = (uintptr_t)dst | (uintptr_t)src;
+            for (uint32_t k = 1; k < nd; ++k) bits |= (uintptr_t)dstk(k);
+            if ((bits & 15u) != 0 || t.count < 16) {
                 issue_simple(p, d, PIECE_TILE, cur, &t, &ds);
                 keep_lag(p, d);
                 return d.ok;
             }
             const uint32_t body = t.count & ~15u, tailb = t.count - body;
             // the last few bytes (< 16) go through this thread; they belong to the item, so before its last piece
-            for (uint32_t i = 0; i < tailb; ++i) dst[body + i] = __ldcg(src + body + i);
+            for (uint32_t i = 0; i < tailb; ++i) {
+                const char b = __ldcg(src + body + i);
+                dst[body + i] = b;
+                for (uint32_t k = 1; k < nd; ++k) dstk(k)[body + i] = b;
+            }
             const bool stream = ds.kind_a == HCCL_BUF_SEND;
             for (uint32_t off = 0; off < body && d.ok; off += STAGE_BYTES) {
                 const uint32_t nb = min(STAGE_BYTES, body - off);
@@ -1067,6 +1158,9 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
                 pi.last = (off + nb == body) ? 1u : 0u;
                 pi.tile_index = cur;
                 pi.dst = dst + off;
+                pi.ndst = (uint16_t)nd;
+                pi.rank_dst = ds.rank_dst;
+                pi.dst_off = doff + off;
                 pi.signal[0] = t.signal[0];
                 pi.signal[1] = t.signal[1];
                 pi.evict_first = stream ? 1 : 0;
@@ -1208,6 +1302,32 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             uint4* dst = reinterpret_cast<uint4*>(pi.dst);
             const uint32_t nv = pi.n >> 4;
             const bool stream = pi.evict_first != 0;
+            if (pi.ndst > 1) {
+                const uint32_t nd = pi.ndst, r0 = pi.rank_dst;
+                const unsigned long long doff = pi.dst_off;
+                constexpr int U = 4;
+                uint32_t i = ctid;
+                for (; i + (U - 1) * cnth < nv; i += U * cnth) {
+                    uint4 v[U];
+#pragma unroll
+                    for (int u = 0; u < U; ++u) v[u] = src[i + u * cnth];
+                    for (uint32_t k = 0; k < nd; ++k) {
+                        uint32_t r = r0 + k;
+                        if (r >= p.R) r -= p.R;
+                        uint4* dk = reinterpret_cast<uint4*>((char*)p.recv[r] + doff) + i;
+#pragma unroll
+                        for (int u = 0; u < U; ++u) __stcs(dk + u * cnth, v[u]);
+                    }
+                }
+                for (; i < nv; i += cnth) {
+                    const uint4 v = src[i];
+                    for (uint32_t k = 0; k < nd; ++k) {
+                        uint32_t r = r0 + k;
+                        if (r >= p.R) r -= p.R;
+                        __stcs(reinterpret_cast<uint4*>((char*)p.recv[r] + doff) + i, v);
+                    }
+                }
+            } else
             for (uint32_t i = ctid; i < nv; i += cnth) {
                 if (stream) __stcs(dst + i, src[i]); else __stcg(dst + i, src[i]);
             }

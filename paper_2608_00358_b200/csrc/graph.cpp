@@ -45,19 +45,30 @@ void push_unique(std::vector<int64_t>& v, int64_t x) {
     if (std::find(v.begin(), v.end(), x) == v.end()) v.push_back(x);
 }
 
+int wqe_ndst(const hccl_wqe_t& w) { return (w.op == HCCL_OP_COPY || w.op == HCCL_OP_REDUCE_N) && w.ndst > 1 ? w.ndst : 1; }
+// Is `rank` one of the ranks whose receive buffer w writes? Is any other rank?
+bool writes_rank(const hccl_wqe_t& w, int rank, int R) {
+    if (w.dst.kind != HCCL_BUF_RECV) return false;
+    const int k = ((rank - w.dst.rank) % R + R) % R;
+    return k < wqe_ndst(w);
+}
+bool writes_other_rank(const hccl_wqe_t& w, int rank, int R) {
+    if (w.dst.kind != HCCL_BUF_RECV) return false;
+    return wqe_ndst(w) > 1 ? R > 1 : w.dst.rank != rank;
+}
+
 // Does WQE w, issued by a subgraph acting for `rank`, bring data into that rank from another one?
-bool is_receive(const hccl_wqe_t& w, int rank) {
-    if (!is_data_op(w.op) || w.dst.kind != HCCL_BUF_RECV || w.dst.rank != rank) return false;
+bool is_receive(const hccl_wqe_t& w, int rank, int R) {
+    if (!is_data_op(w.op) || !writes_rank(w, rank, R)) return false;
     if (w.op == HCCL_OP_REDUCE_N) return w.nsrc > 1 || w.a.rank != rank;
     bool a_remote = (w.a.kind == HCCL_BUF_SEND || w.a.kind == HCCL_BUF_RECV) && w.a.rank != rank;
     bool b_remote = w.op == HCCL_OP_REDUCE && (w.b.kind == HCCL_BUF_SEND || w.b.kind == HCCL_BUF_RECV) && w.b.rank != rank;
     return a_remote || b_remote;
 }
 // Does it read this rank's buffers on behalf of another rank (a "send": the buffer is busy until it completes)?
-bool is_send(const hccl_wqe_t& w, int rank) {
+bool is_send(const hccl_wqe_t& w, int rank, int R) {
     if (!is_data_op(w.op)) return false;
-    bool dst_remote = w.dst.kind == HCCL_BUF_RECV && w.dst.rank != rank;
-    if (!dst_remote) return false;
+    if (!writes_other_rank(w, rank, R)) return false;
     if (w.op == HCCL_OP_REDUCE_N) return true;
     bool a_local = (w.a.kind == HCCL_BUF_SEND || w.a.kind == HCCL_BUF_RECV) && w.a.rank == rank;
     bool b_local = w.op == HCCL_OP_REDUCE && (w.b.kind == HCCL_BUF_SEND || w.b.kind == HCCL_BUF_RECV) && w.b.rank == rank;
@@ -121,8 +132,14 @@ hccl_status_t hccl_graph_add_wqe(hccl_graph_t* g, int32_t subgraph, const hccl_w
         case HCCL_OP_COPY: {
             if (w.dst.kind != HCCL_BUF_RECV && w.dst.kind != HCCL_BUF_SCRATCH) return HCCL_ERR_INVALID_ARG;
             if (w.a.kind != HCCL_BUF_SEND && w.a.kind != HCCL_BUF_RECV && w.a.kind != HCCL_BUF_SCRATCH) return HCCL_ERR_INVALID_ARG;
-            if (!in_bounds(g, w.dst, w.count) || !in_bounds(g, w.a, w.count)) return HCCL_ERR_INVALID_ARG;
-            if (ranges_intersect(w.dst, w.count, w.a, w.count)) return HCCL_ERR_OVERLAP;
+            if (w.ndst < 0 || w.ndst > g->R || (w.ndst > 1 && w.dst.kind != HCCL_BUF_RECV)) return HCCL_ERR_INVALID_ARG;
+            if (!in_bounds(g, w.a, w.count)) return HCCL_ERR_INVALID_ARG;
+            for (int k = 0; k < wqe_ndst(w); ++k) {
+                hccl_ref_t d = w.dst;
+                if (k) d.rank = (w.dst.rank + k) % g->R;
+                if (!in_bounds(g, d, w.count)) return HCCL_ERR_INVALID_ARG;
+                if (ranges_intersect(d, w.count, w.a, w.count)) return HCCL_ERR_OVERLAP;
+            }
             break;
         }
         case HCCL_OP_REDUCE: {
@@ -151,16 +168,21 @@ hccl_status_t hccl_graph_add_wqe(hccl_graph_t* g, int32_t subgraph, const hccl_w
             if (!valid_dtype(w.dtype_dst) || !valid_dtype(w.dtype_a)) return HCCL_ERR_DTYPE;
             if (w.nsrc < 1 || w.nsrc > g->R) return HCCL_ERR_INVALID_ARG;
             if (w.dst.kind != HCCL_BUF_RECV && w.dst.kind != HCCL_BUF_SCRATCH) return HCCL_ERR_INVALID_ARG;
+            if (w.ndst < 0 || w.ndst > g->R || (w.ndst > 1 && w.dst.kind != HCCL_BUF_RECV)) return HCCL_ERR_INVALID_ARG;
             if (w.a.kind != HCCL_BUF_SEND && w.a.kind != HCCL_BUF_RECV) return HCCL_ERR_INVALID_ARG;
             const int64_t db = w.count * elem_bytes(w.dtype_dst), sb = w.count * elem_bytes(w.dtype_a);
-            if (!in_bounds(g, w.dst, db)) return HCCL_ERR_INVALID_ARG;
             if (w.dst.offset % elem_bytes(w.dtype_dst) || w.a.offset % elem_bytes(w.dtype_a)) return HCCL_ERR_ALIGNMENT;
             if (w.a.rank < 0 || w.a.rank >= g->R) return HCCL_ERR_INVALID_ARG;
-            for (int k = 0; k < w.nsrc; ++k) {
-                hccl_ref_t s = w.a;
-                s.rank = (w.a.rank + k) % g->R;
-                if (!in_bounds(g, s, sb)) return HCCL_ERR_INVALID_ARG;
-                if (ranges_intersect(w.dst, db, s, sb)) return HCCL_ERR_OVERLAP;
+            for (int j = 0; j < wqe_ndst(w); ++j) {
+                hccl_ref_t d = w.dst;
+                if (j) d.rank = (w.dst.rank + j) % g->R;
+                if (!in_bounds(g, d, db)) return HCCL_ERR_INVALID_ARG;
+                for (int k = 0; k < w.nsrc; ++k) {
+                    hccl_ref_t s = w.a;
+                    s.rank = (w.a.rank + k) % g->R;
+                    if (j == 0 && !in_bounds(g, s, sb)) return HCCL_ERR_INVALID_ARG;
+                    if (ranges_intersect(d, db, s, sb)) return HCCL_ERR_OVERLAP;
+                }
             }
             break;
         }
@@ -216,8 +238,8 @@ hccl_status_t hccl_graph_add_wqe(hccl_graph_t* g, int32_t subgraph, const hccl_w
         for (size_t i = from; i < sg.wqes.size(); ++i) {
             const hccl_wqe_t& p = g->wqes[sg.wqes[i]].w;
             bool hit = sg.wqes[i] == sg.last_sync;  // the barrier stands for everything older
-            if ((w.dep_flags & HCCL_DEP_RECV_SYNC) && is_receive(p, sg.rank)) hit = true;
-            if ((w.dep_flags & HCCL_DEP_SEND_SYNC) && is_send(p, sg.rank)) hit = true;
+            if ((w.dep_flags & HCCL_DEP_RECV_SYNC) && is_receive(p, sg.rank, g->R)) hit = true;
+            if ((w.dep_flags & HCCL_DEP_SEND_SYNC) && is_send(p, sg.rank, g->R)) hit = true;
             if (hit) push_unique(q.preds_full, sg.wqes[i]);
         }
     }
@@ -291,20 +313,28 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
     };
     for (const Wqe& q : g->wqes) {
         const hccl_wqe_t& w = q.w;
-        if (w.op == HCCL_OP_COPY && remote(w.a, w.dst)) crossrack += w.count;
+        const int nd = wqe_ndst(w);  // a byte counts as crossing once per destination in another rack
+        if (w.op == HCCL_OP_COPY)
+            for (int j = 0; j < nd; ++j) {
+                hccl_ref_t d = w.dst;
+                if (j) d.rank = (w.dst.rank + j) % g->R;
+                if (remote(w.a, d)) crossrack += w.count;
+            }
         if (w.op == HCCL_OP_REDUCE) {
             if (remote(w.a, w.dst)) crossrack += w.count * elem_bytes(w.dtype_a);
             if (remote(w.b, w.dst)) crossrack += w.count * elem_bytes(w.dtype_b);
         }
         if (w.op == HCCL_OP_REDUCE_N)
-            for (int k = 0; k < w.nsrc; ++k) {
-                hccl_ref_t sr = w.a;
-                sr.rank = (w.a.rank + k) % g->R;
-                if (remote(sr, w.dst)) crossrack += w.count * elem_bytes(w.dtype_a);
-            }
-        if (w.op == HCCL_OP_COPY) schedule += 2 * w.count;
+            for (int j = 0; j < nd; ++j)
+                for (int k = 0; k < w.nsrc; ++k) {
+                    hccl_ref_t sr = w.a, d = w.dst;
+                    sr.rank = (w.a.rank + k) % g->R;
+                    if (j) d.rank = (w.dst.rank + j) % g->R;
+                    if (remote(sr, d)) crossrack += w.count * elem_bytes(w.dtype_a);
+                }
+        if (w.op == HCCL_OP_COPY) schedule += (1 + (int64_t)nd) * w.count;
         if (w.op == HCCL_OP_REDUCE) schedule += w.count * (elem_bytes(w.dtype_a) + elem_bytes(w.dtype_b) + elem_bytes(w.dtype_dst));
-        if (w.op == HCCL_OP_REDUCE_N) schedule += w.count * ((int64_t)w.nsrc * elem_bytes(w.dtype_a) + elem_bytes(w.dtype_dst));
+        if (w.op == HCCL_OP_REDUCE_N) schedule += w.count * ((int64_t)w.nsrc * elem_bytes(w.dtype_a) + (int64_t)nd * elem_bytes(w.dtype_dst));
         weight += w.count * widest(w);
         if (w.op == HCCL_OP_REDUCE || w.op == HCCL_OP_REDUCE_N) {
             auto need = [&](const hccl_ref_t& r, int dt) {
@@ -389,7 +419,8 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         d.dt_dst = (uint8_t)w.dtype_dst; d.dt_a = (uint8_t)w.dtype_a; d.dt_b = (uint8_t)w.dtype_b;
         d.kind_dst = (uint8_t)w.dst.kind; d.kind_a = (uint8_t)w.a.kind; d.kind_b = (uint8_t)w.b.kind;
         d.cmp = (uint8_t)((w.op == HCCL_OP_WAIT) ? w.cmp : w.hints);  // data ops carry their cache hints here
-        d.rank_dst = (uint16_t)w.dst.rank; d.rank_a = (uint16_t)w.a.rank; d.rank_b = (uint16_t)w.b.rank;
+        d.rank_dst = (uint16_t)w.dst.rank; d.rank_a = (uint16_t)w.a.rank;
+        if (w.op == HCCL_OP_COPY || w.op == HCCL_OP_REDUCE_N) d.ndst = (uint16_t)wqe_ndst(w); else d.rank_b = (uint16_t)w.b.rank;
         d.nsrc = (uint16_t)w.nsrc;
         d.off_dst = w.dst.offset; d.off_a = w.a.offset; d.off_b = w.b.offset;
         d.count = w.count;

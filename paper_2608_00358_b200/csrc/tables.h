@@ -12,12 +12,23 @@ namespace hccl {
 struct alignas(16) Desc {  // 64 bytes
     uint8_t op, dt_dst, dt_a, dt_b;          // hccl_op_t, hccl_dtype_t x3
     uint8_t kind_dst, kind_a, kind_b, cmp;   // hccl_buf_t x3, hccl_cmp_t
-    uint16_t rank_dst, rank_a, rank_b, nsrc; // nsrc: REDUCE_N only
+    uint16_t rank_dst, rank_a;
+    union {
+        uint16_t rank_b;                     // REDUCE: rank of operand B
+        uint16_t ndst;                       // COPY, REDUCE_N: destinations written (0 and 1 both mean one);
+    };                                       // destination k is the receive buffer of rank (rank_dst + k) mod R
+    uint16_t nsrc;                           // REDUCE_N only
     int64_t off_dst, off_a, off_b;           // byte offsets (data) or slot index (signals)
     int64_t count;                           // bytes (COPY) or elements (REDUCE, REDUCE_N)
     uint64_t value, value_per_epoch;         // WAIT / SET operand
 };
 static_assert(sizeof(Desc) == 64, "Desc layout");
+
+// Number of destinations a data descriptor writes.
+#if defined(__CUDACC__)
+__host__ __device__
+#endif
+inline int ndst_of(const Desc& d) { return (d.op == 0 /*COPY*/ || d.op == 2 /*REDUCE_N*/) && d.ndst > 1 ? (int)d.ndst : 1; }
 
 struct alignas(16) Tile {  // 32 bytes
     uint32_t desc;      // index into descs

@@ -31,7 +31,8 @@ void tile_accesses(const hccl_plan* p, uint32_t ti, std::vector<Access>& out) {
     switch (d.op) {
         case HCCL_OP_COPY:
             add(d.kind_a, d.rank_a, d.off_a + (int64_t)t.start, t.count, false);
-            add(d.kind_dst, d.rank_dst, d.off_dst + (int64_t)t.start, t.count, true);
+            for (int j = 0; j < ndst_of(d); ++j)
+                add(d.kind_dst, (d.rank_dst + j) % p->R, d.off_dst + (int64_t)t.start, t.count, true);
             break;
         case HCCL_OP_REDUCE: {
             const int ea = elem_bytes(d.dt_a), eb = elem_bytes(d.dt_b), ed = elem_bytes(d.dt_dst);
@@ -44,7 +45,8 @@ void tile_accesses(const hccl_plan* p, uint32_t ti, std::vector<Access>& out) {
             const int ea = elem_bytes(d.dt_a), ed = elem_bytes(d.dt_dst);
             for (int k = 0; k < d.nsrc; ++k)
                 add(d.kind_a, (d.rank_a + k) % p->R, d.off_a + (int64_t)t.start * ea, (int64_t)t.count * ea, false);
-            add(d.kind_dst, d.rank_dst, d.off_dst + (int64_t)t.start * ed, (int64_t)t.count * ed, true);
+            for (int j = 0; j < ndst_of(d); ++j)
+                add(d.kind_dst, (d.rank_dst + j) % p->R, d.off_dst + (int64_t)t.start * ed, (int64_t)t.count * ed, true);
             break;
         }
         case HCCL_OP_WAIT:
@@ -209,7 +211,8 @@ hccl_status_t hccl_plan_interpret_host(const hccl_plan_t* p, const void* const* 
         const Desc& d = p->descs[t.desc];
         switch (d.op) {
             case HCCL_OP_COPY:
-                std::memmove(base(d.kind_dst, d.rank_dst) + d.off_dst + t.start, base(d.kind_a, d.rank_a) + d.off_a + t.start, t.count);
+                for (int j = 0; j < ndst_of(d); ++j)
+                    std::memmove(base(d.kind_dst, (d.rank_dst + j) % p->R) + d.off_dst + t.start, base(d.kind_a, d.rank_a) + d.off_a + t.start, t.count);
                 break;
             case HCCL_OP_REDUCE: {
                 const char* a = base(d.kind_a, d.rank_a) + d.off_a;
@@ -222,11 +225,10 @@ hccl_status_t hccl_plan_interpret_host(const hccl_plan_t* p, const void* const* 
                 break;
             }
             case HCCL_OP_REDUCE_N: {
-                char* o = base(d.kind_dst, d.rank_dst) + d.off_dst;
                 for (int64_t i = (int64_t)t.start; i < (int64_t)(t.start + t.count); ++i) {
                     volatile float s = load_f(base(d.kind_a, d.rank_a) + d.off_a, d.dt_a, i);
                     for (int k = 1; k < d.nsrc; ++k) s = s + load_f(base(d.kind_a, (d.rank_a + k) % p->R) + d.off_a, d.dt_a, i);
-                    store_f(o, d.dt_dst, i, s);
+                    for (int j = 0; j < ndst_of(d); ++j) store_f(base(d.kind_dst, (d.rank_dst + j) % p->R) + d.off_dst, d.dt_dst, i, s);
                 }
                 break;
             }

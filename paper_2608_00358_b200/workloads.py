@@ -93,13 +93,13 @@ def config4(opts=None, seed=0, cap: int = 32768, R: int = 64, row: int = 256) ->
 
 
 def config5(m_bytes: int, algo: int, opts=None, seed=0) -> Workload:
-    """AllReduce, R=8, bf16 messages of m_bytes per rank ~ N(0,1), one-shot or ring."""
+    """AllReduce, R=8, bf16 messages of m_bytes per rank ~ N(0,1), one-shot, ring or one of the fused forms."""
     R, n = 8, m_bytes // 2
     X = synth.normal_ranks(R, n, hb.BF16, seed=seed + m_bytes)
     send = [torch.from_numpy(x.view(np.int16)).cuda() for x in X]
     recv = [torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(R)]
     plan = hb.hccl_plan_allreduce(R, n, hb.BF16, algo, opts)
-    name = "allreduce_%s_r8_bf16_%dB" % ({hb.ALGO_RING: "ring", hb.ALGO_ONESHOT: "oneshot", hb.ALGO_RING_FUSED: "ringfused"}[algo], m_bytes)
+    name = "allreduce_%s_r8_bf16_%dB" % ({hb.ALGO_RING: "ring", hb.ALGO_ONESHOT: "oneshot", hb.ALGO_RING_FUSED: "ringfused", hb.ALGO_FANOUT: "fanout"}[algo], m_bytes)
     return _bind(name, plan, send, recv, dict(host_inputs=X, dt=hb.BF16, n=n, R=R))
 
 

@@ -28,7 +28,7 @@ def _check_allreduce(R, n, dt, algo, opts, X=None, iters=1, misalign=0):
     p = hb.hccl_plan_allreduce(R, n, dt, algo, opts)
     Y = run_plan(p, X, iters=iters, misalign=misalign)
     exact, want = orc.sum_f64(dt, X), orc.allreduce(dt, X)
-    bitwise = orc.allreduce_oneshot_f32(dt, X) if algo == hb.ALGO_ONESHOT else \
+    bitwise = orc.allreduce_oneshot_f32(dt, X) if algo in (hb.ALGO_ONESHOT, hb.ALGO_FANOUT) else \
         orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
     for r in range(R):
         got = Y[r].view(np_dtype(dt))
@@ -37,7 +37,7 @@ def _check_allreduce(R, n, dt, algo, opts, X=None, iters=1, misalign=0):
 
 
 @pytest.mark.parametrize("dt", DTYPES)
-@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED, hb.ALGO_FANOUT])
 @pytest.mark.parametrize("R,n", [(1, 5), (2, 9), (3, 2), (4, 257), (5, 1000), (8, 4099), (4, 0), (4, 3), (8, 100003)])
 def test_allreduce_small(R, n, dt, algo, engine):
     _check_allreduce(R, n, dt, algo, _with(dict(tile_bytes=1024, chunk_bytes=4096, chain_group=2, sm_budget=8), engine), iters=2)
@@ -56,6 +56,7 @@ def test_allreduce_misaligned_buffers(misalign, dt, engine):
         pytest.skip("buffers must be aligned to the element size")
     _check_allreduce(4, 10007, dt, hb.ALGO_RING, _with(dict(tile_bytes=4096, sm_budget=16), engine), misalign=misalign)
     _check_allreduce(4, 10007, dt, hb.ALGO_ONESHOT, _with(dict(tile_bytes=4096, sm_budget=16), engine), misalign=misalign)
+    _check_allreduce(4, 10007, dt, hb.ALGO_FANOUT, _with(dict(tile_bytes=4096, sm_budget=16), engine), misalign=misalign)
 
 
 def test_config1_allreduce_ring_r4_fp32(engine):
@@ -63,7 +64,7 @@ def test_config1_allreduce_ring_r4_fp32(engine):
     _check_allreduce(4, 1 << 20, hb.FP32, hb.ALGO_RING, _with(None, engine), X=X, iters=3)
 
 
-@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT])
 @pytest.mark.parametrize("m", [4096, 65536, 262144, 1 << 20])
 def test_config5_allreduce_r8_bf16(m, algo, engine):
     X = synth.normal_ranks(8, m // 2, hb.BF16, seed=m)
@@ -75,7 +76,7 @@ def test_closed_form_on_device(engine):
         for R in (2, 4, 8, 16):
             n = 3000
             X = [synth.to_bits(np.full(n, r + 1, dtype=np.float32), dt) for r in range(R)]
-            for algo in (hb.ALGO_RING, hb.ALGO_ONESHOT):
+            for algo in (hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT):
                 Y = run_plan(hb.hccl_plan_allreduce(R, n, dt, algo, _with(dict(tile_bytes=1024), engine)), X)
                 for r in range(R):
                     assert np.all(synth.from_bits(Y[r].view(np_dtype(dt)), dt) == R * (R + 1) / 2)
@@ -113,7 +114,7 @@ def test_config3_shape_reducescatter_r16_bf16_reduced_size(engine):
         assert np.array_equal(got, bitwise[r])
 
 
-@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT])
 @pytest.mark.parametrize("R,counts", [(1, [5]), (4, [3, 0, 1000, 17]), (8, None)])
 def test_allgather(R, counts, algo, engine):
     cs = counts if counts is not None else [32100] * R
@@ -220,11 +221,16 @@ def test_maximum_rank_count(engine):
     R, n, dt = 256, 3001, hb.BF16
     X = synth.small_int_ranks(R, n, dt, seed=256, span=1)          # exactly summable in bf16: unique result
     want = orc.allreduce(dt, X)
-    for algo, extra in ((hb.ALGO_RING, {}), (hb.ALGO_ONESHOT, {}), (hb.ALGO_RING_2LEVEL, dict(rack_size=16))):
+    for algo, extra in ((hb.ALGO_RING, {}), (hb.ALGO_ONESHOT, {}), (hb.ALGO_RING_2LEVEL, dict(rack_size=16)), (hb.ALGO_FANOUT, {})):
         p = hb.hccl_plan_allreduce(R, n, dt, algo, _with(dict(sm_budget=64, **extra), engine))
         Y = run_plan(p, X)
         for r in (0, 1, 127, 255):
             assert np.array_equal(Y[r].view(np.uint16), want[r]), (algo, r)
+    Xg = [x[:157] for x in X]                                          # AllGather, 256 destinations per work item
+    wantg = orc.allgatherv(Xg)[0]
+    Y = run_plan(hb.hccl_plan_allgather(R, None, 157, dt, hb.ALGO_FANOUT, _with(dict(sm_budget=64), engine)), Xg)
+    for r in (0, 1, 128, 255):
+        assert np.array_equal(Y[r].view(np.uint16), wantg), r
     C = synth.uniform_counts(R, 3, hi=3)
     SD, RD = orc.packed_displs(C)
     rb = 16 * 2

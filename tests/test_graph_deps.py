@@ -97,14 +97,27 @@ def g_signal_pair():
     return g, lambda X: [X[0], _sum(X[0], X[1])]
 
 
-CASES = {"fence": g_fence, "sync": g_sync, "wqe_sync": g_wqe_sync, "recv_sync": g_recv_sync,
+def g_fanout(with_dep=True):
+    # multi-destination forms: a copy into ranks 3, 0, 1 (wrapping), a dependent sum reading one of those
+    # copies, and a two-input sum written into ranks 0 and 1
+    g = hb.Graph(4, [NB] * 4, [2 * NB, 2 * NB, NB, NB])
+    sg = g.add_subgraph(3)
+    w0 = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 3, 0), a=(S, 3, 0), count=NB, ndst=3)
+    g.add_wqe(sg, hb.OP_REDUCE, dst=(Rv, 2, 0), a=(Rv, 1, 0), b=(S, 0, 0), count=N, dtypes=F3,
+              dep_flags=hb.DEP_WQE_SYNC if with_dep else 0, dep_wqe=w0)
+    g.add_wqe(sg, hb.OP_REDUCE_N, dst=(Rv, 0, NB), a=(S, 2, 0), count=N, nsrc=2, ndst=2, dtypes=F3)
+    return g, lambda X: [np.concatenate([X[3], _sum(X[2], X[3])]), np.concatenate([X[3], _sum(X[2], X[3])]),
+                         _sum(X[3], X[0]), X[3]]
+
+
+CASES = {"fanout": g_fanout, "fence": g_fence, "sync": g_sync, "wqe_sync": g_wqe_sync, "recv_sync": g_recv_sync,
          "send_sync": g_send_sync, "noop_join": g_noop_join}
 
 
 @pytest.mark.parametrize("name", sorted(CASES))
 def test_dependency_kind_on_host(name):
     g, want = CASES[name](True)
-    R = len(want(_x(3)))
+    R = len(want(_x(4)))
     X = _x(R, seed=1)
     p = g.compile(OPTS)
     assert p.check_hazards() == 0
@@ -115,6 +128,17 @@ def test_dependency_kind_on_host(name):
     # without the dependency the checker must object
     g2, _ = CASES[name](False)
     assert g2.compile(OPTS).check_hazards() > 0
+
+
+def test_fanout_destinations_are_bounds_checked_one_by_one():
+    g = hb.Graph(3, [NB] * 3, [NB, NB // 2, NB])
+    sg = g.add_subgraph(0)
+    with pytest.raises(hb.HcclError) as e:
+        g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, 0), a=(S, 0, 0), count=NB, ndst=3)   # rank 1's buffer is too short
+    assert e.value.status == hb.ERR_INVALID_ARG
+    assert g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 2, 0), a=(S, 0, 0), count=NB, ndst=2) == 0  # ranks 2 and 0
+    i = g.compile(OPTS).info()
+    assert i.schedule_bytes == 3 * NB   # one read, two writes
 
 
 def test_recv_sync_does_not_cover_local_copies():
@@ -153,6 +177,10 @@ def test_wqe_validation():
     bad(hb.ERR_ALIGNMENT, op=hb.OP_REDUCE, dst=(Rv, 0, 2), a=(S, 0, 0), b=(S, 1, 0), count=4, dtypes=F3)
     bad(hb.ERR_OVERLAP, op=hb.OP_REDUCE, dst=(Rv, 0, 4), a=(Rv, 0, 0), b=(S, 1, 0), count=4, dtypes=F3)   # shifted alias
     bad(hb.ERR_INVALID_ARG, op=hb.OP_REDUCE_N, dst=(Rv, 0, 0), a=(S, 0, 0), count=4, nsrc=3, dtypes=F3)
+    bad(hb.ERR_INVALID_ARG, op=hb.OP_COPY, dst=(Rv, 0, 0), a=(S, 1, 0), count=16, ndst=3)     # more destinations than ranks
+    bad(hb.ERR_INVALID_ARG, op=hb.OP_COPY, dst=(SC, 0, 0), a=(S, 1, 0), count=16, ndst=2)     # scratch has no ranks to fan out over
+    bad(hb.ERR_OVERLAP, op=hb.OP_COPY, dst=(Rv, 1, 0), a=(Rv, 0, 0), count=16, ndst=2)        # second destination is the source
+    bad(hb.ERR_INVALID_ARG, op=hb.OP_REDUCE_N, dst=(SC, 0, 0), a=(S, 0, 0), count=4, nsrc=2, ndst=2, dtypes=F3)
     bad(hb.ERR_INVALID_ARG, op=hb.OP_WAIT, a=(SIG, 0, 0), cmp=hb.CMP_GE)                      # no signal slots declared
     bad(hb.ERR_INVALID_ARG, op=hb.OP_NOOP, dep_flags=hb.DEP_WQE_SYNC, dep_wqe=5)             # dependency on the future
     ok = g.add_wqe(sg, hb.OP_REDUCE, dst=(Rv, 0, 0), a=(Rv, 0, 0), b=(S, 1, 0), count=N, dtypes=F3)   # A=A+B
@@ -167,7 +195,7 @@ def test_wqe_validation():
 def test_dependency_kind_on_gpu(name, budget, engine):
     from gpu_helpers import run_plan
     g, want = (g_signal_pair() if name == "signal_pair" else CASES[name](True))
-    R = len(want(_x(3)))
+    R = len(want(_x(4)))
     X = _x(R, seed=3)
     p = g.compile(dict(OPTS, sm_budget=budget, engine=engine))
     Y = run_plan(p, X, iters=5)

@@ -47,10 +47,13 @@ def test_config3_and_5_byte_accounting():
     for m in (4096, 1 << 20):
         assert hb.hccl_plan_allreduce(8, m // 2, hb.BF16, hb.ALGO_RING).info().schedule_bytes == 47 * m
         assert hb.hccl_plan_allreduce(8, m // 2, hb.BF16, hb.ALGO_ONESHOT).info().schedule_bytes == 72 * m
+        # destinations fused: every input read once, every output written once = the compulsory bytes
+        i = hb.hccl_plan_allreduce(8, m // 2, hb.BF16, hb.ALGO_FANOUT).info()
+        assert i.schedule_bytes == 16 * m == i.compulsory_bytes and i.chain_depth == 1
 
 
 @pytest.mark.parametrize("dt", DTYPES)
-@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED, hb.ALGO_FANOUT])
 @pytest.mark.parametrize("R,n", [(1, 5), (2, 9), (3, 2), (4, 257), (5, 1000), (8, 4099), (4, 0), (4, 3)])
 def test_allreduce_plans_match_oracle(R, n, dt, algo):
     X = synth.normal_ranks(R, n, dt, seed=R * 100 + n)
@@ -58,7 +61,7 @@ def test_allreduce_plans_match_oracle(R, n, dt, algo):
     assert p.check_hazards() == 0
     exact = orc.sum_f64(dt, X)
     want = orc.allreduce(dt, X)
-    if algo == hb.ALGO_ONESHOT:
+    if algo in (hb.ALGO_ONESHOT, hb.ALGO_FANOUT):  # the fused form sums in the one-shot's order
         bitwise = orc.allreduce_oneshot_f32(dt, X)
     else:
         bitwise = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
@@ -122,7 +125,7 @@ def test_reducescatter_rejects_bad_counts():
     assert e.value.status == hb.ERR_INVALID_ARG
 
 
-@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT])
 @pytest.mark.parametrize("R,counts", [(1, [5]), (4, [3, 0, 1000, 17]), (8, None)])
 def test_allgather_plans_match_oracle(R, counts, algo):
     dt = hb.BF16
