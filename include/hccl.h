@@ -131,7 +131,8 @@ typedef struct hccl_graph hccl_graph_t; /* opaque, host-owned: a work packet und
  * ((X_{c+1}+X_{c+2})+...)+X_c in FP32 and ends on rank c; all-gather step u copies it to rank c+u+1.
  * FP32 data keeps partials in the receive buffers; 16-bit data keeps FP32 partials in workspace
  * scratch and is rounded once, on the last reduce step. ONESHOT: R independent R-input sums in rank
- * order 0..R-1. Send and receive buffers: count elements each. */
+ * order 0..R-1. FANOUT: that sum formed once per element and stored into all R receive buffers (same
+ * bits as ONESHOT). RING_FUSED, RING_2LEVEL: see hccl_algo_t. Send and receive buffers: count elements each. */
 hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_algo_t algo,
                                   const hccl_opts_t* opts, hccl_plan_t** out);
 
@@ -145,7 +146,9 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
 
 /* AllGather(v): Y_r[o_q + j] = X_q[j] for all r, q; sendcounts[q] elements from rank q (NULL: count each).
  * algo RING copies hop by hop (rank r receives chunk (r-u-1) mod R from rank r-1 at step u);
- * ONESHOT has every rank read every peer directly. */
+ * ONESHOT has every rank read every peer directly (issued chunk by chunk, so a chunk's R reads follow one
+ * another); FANOUT reads each chunk once and writes it into all R receive buffers from the same work item;
+ * RING_2LEVEL gathers across racks first, then inside each rack. */
 hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t count, hccl_dtype_t dt,
                                   hccl_algo_t algo, const hccl_opts_t* opts, hccl_plan_t** out);
 
