@@ -355,20 +355,46 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             torch.cuda.synchronize()
             hp = ([h.data_ptr() for h in hs], [h.data_ptr() for h in hr])
             dp = ([d_.data_ptr() for d_ in wl.send], [d_.data_ptr() for d_ in wl.recv])
+            ksteps = args.e2e_steps
+            # (a) one stream: copy everything in, exchange, copy everything out
             wl.plan.execute_host(hp[0], hp[1], dp[0], dp[1], stream.cuda_stream)   # warm-up
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            ksteps = args.e2e_steps
             e0.record(stream)
             for _ in range(ksteps):
                 wl.plan.execute_host(hp[0], hp[1], dp[0], dp[1], stream.cuda_stream)
             e1.record(stream)
             torch.cuda.synchronize()
             wl.dc.check()
+            serial_ms = e0.elapsed_time(e1) / ksteps
+            # (b) pipelined by destination windows on three streams: both directions of the host link busy at once
+            pipe = hb.hccl_hostpipe_alltoallv_create(64, wl.meta["counts"], hb.FP16, 256, args.e2e_windows, opts)
+            pws = torch.empty(pipe.workspace_bytes() + 256, dtype=torch.uint8, device="cuda")
+            pipe.bind((pws.data_ptr() + 255) // 256 * 256, pipe.workspace_bytes(), stream.cuda_stream)
+            s_in, s_ex, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+            for h in hr:
+                h.zero_()
+            torch.cuda.synchronize()
+            pipe.execute(hp[0], hp[1], dp[0], dp[1], s_in.cuda_stream, s_ex.cuda_stream, s_out.cuda_stream)   # warm-up
+            torch.cuda.synchronize()
+            e0.record(s_in)
+            for _ in range(ksteps):
+                pipe.execute(hp[0], hp[1], dp[0], dp[1], s_in.cuda_stream, s_ex.cuda_stream, s_out.cuda_stream)
+            e1.record(s_out)
+            torch.cuda.synchronize()
+            pst, pdetail = pipe.status()
+            if pst != hb.OK:
+                raise hb.HcclError(pst, "hccl_hostpipe_status (detail %d)" % pdetail)
+            for d_ in (0, 31, 63):   # what came back to the host is what the device-resident run left on the device
+                if not torch.equal(hr[d_], wl.recv[d_].cpu()):
+                    raise RuntimeError("pipelined end-to-end result differs at destination %d" % d_)
             ms = e0.elapsed_time(e1) / ksteps
             e2e = {"value": info.schedule_bytes / ms / 1e6, "unit": UNIT, "h2d_bytes_per_step": int(payload),
                    "d2h_bytes_per_step": int(payload), "ms_per_step": ms, "steps": ksteps,
-                   "api": "hccl_execute_host (pinned host buffers -> device -> pinned host buffers)"}
+                   "api": "hccl_hostpipe_execute (pinned host buffers -> device -> pinned host buffers, %d destination windows on 3 streams)" % (len(pipe.windows()) - 1),
+                   "gpu_launches_per_step": len(pipe.windows()) - 1,
+                   "single_stream": {"value": info.schedule_bytes / serial_ms / 1e6, "ms_per_step": serial_ms, "api": "hccl_execute_host"}}
+            del pipe, pws
             del hs, hr
         else:
             e2e = {"value": None, "unit": UNIT, "skipped": "host memory too small to pin 2 x %.1f GB" % (payload / 1e9)}
@@ -443,6 +469,7 @@ def main():
     ap.add_argument("--engine", default="", choices=["", "lsu", "bulk"], help="force an executor engine (default: the library's choice)")
     ap.add_argument("--oracle-dst", type=int, default=8, help="destination ranks in the CPU oracle's sample")
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-windows", type=int, default=16, help="destination windows of the pipelined end-to-end path")
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-gemm", action="store_true")

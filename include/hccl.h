@@ -321,6 +321,37 @@ hccl_status_t hccl_execute_noalloc(hccl_plan_t*, const void* const* sendbufs, vo
 hccl_status_t hccl_execute_host(hccl_plan_t*, const void* const* host_send, void* const* host_recv,
                                 void* const* dev_send, void* const* dev_recv, void* stream);
 
+/* ------------------------------------------------------------------------
+ * AllToAllv through HOST buffers, pipelined by destination (the paper spreads an AllToAllv over several
+ * subgraphs to keep the links busy, Sec. IV-A; here the link is the host interface and the pieces are
+ * windows of destination ranks). The destinations are cut into n_windows contiguous groups of about equal
+ * received bytes. For window g: the rows bound for its destinations are copied host->device (with packed
+ * send displacements they are one contiguous slice of every send buffer), exchanged by a sub-plan that
+ * holds only those segments, and the window's receive buffers are copied device->host. The three steps
+ * run on three caller-supplied streams, ordered by events, so that copy-in of window g+1, exchange of g
+ * and copy-out of g-1 overlap and both directions of the host link are busy at once.
+ *   create    host only; sendcounts as in hccl_plan_alltoallv, packed displacements; n_windows is clamped
+ *             to [1, R]; windows that would receive nothing are merged into their neighbours.
+ *   bind      uploads every sub-plan's tables into the caller's workspace (workspace_bytes, 256-aligned)
+ *             and creates the ordering events (no device memory is allocated).
+ *   execute   asynchronous; everything has completed when stream_out has. host buffers should be pinned.
+ *             dev_send / dev_recv are the caller's staging buffers (full extents, as for hccl_execute).
+ *             A second execute may be enqueued at once: it starts after the first has finished.
+ *   status    after synchronising stream_out: the first device-side failure of any window, else HCCL_OK.
+ *   windows   first_dest[g] .. first_dest[g+1]-1 are window g's destinations (n_windows+1 entries).
+ * ------------------------------------------------------------------------ */
+typedef struct hccl_hostpipe hccl_hostpipe_t;
+hccl_status_t hccl_hostpipe_alltoallv_create(int R, const int64_t* sendcounts, hccl_dtype_t dt, int64_t row_elems,
+                                             int n_windows, const hccl_opts_t* opts, hccl_hostpipe_t** out);
+hccl_status_t hccl_hostpipe_windows(const hccl_hostpipe_t*, int32_t* n_windows, int32_t* first_dest /* [R+1] room */);
+hccl_status_t hccl_hostpipe_workspace_bytes(const hccl_hostpipe_t*, size_t* bytes);
+hccl_status_t hccl_hostpipe_bind(hccl_hostpipe_t*, void* dev_workspace, size_t bytes, void* stream);
+hccl_status_t hccl_hostpipe_execute(hccl_hostpipe_t*, const void* const* host_send, void* const* host_recv,
+                                    void* const* dev_send, void* const* dev_recv, void* stream_in, void* stream_exec,
+                                    void* stream_out);
+hccl_status_t hccl_hostpipe_status(hccl_hostpipe_t*, hccl_status_t* device_status, int64_t* detail);
+void hccl_hostpipe_destroy(hccl_hostpipe_t*);
+
 /* Resident, doorbell-fed execution (the express-doorbell idea of Sec. II-A.3 and the cached re-enqueue of
  * Sec. V-B, without any launch per collective). hccl_server_start launches the register engine ONCE as a
  * long-lived kernel bound to this plan and these buffers; afterwards hccl_server_ring is a single store

@@ -97,6 +97,12 @@ def _load() -> C.CDLL:
         "hccl_plan_layout": [P, I64P],
         "hccl_plan_check_hazards": [P, I64P],
         "hccl_plan_interpret_host": [P, C.POINTER(P), C.POINTER(P), P, C.POINTER(C.c_uint64), C.c_uint64],
+        "hccl_hostpipe_alltoallv_create": [C.c_int, I64P, C.c_int, C.c_int64, C.c_int, C.POINTER(Opts), C.POINTER(P)],
+        "hccl_hostpipe_windows": [P, C.POINTER(C.c_int32), C.POINTER(C.c_int32)],
+        "hccl_hostpipe_workspace_bytes": [P, C.POINTER(C.c_size_t)],
+        "hccl_hostpipe_bind": [P, P, C.c_size_t, P],
+        "hccl_hostpipe_execute": [P, C.POINTER(P), C.POINTER(P), C.POINTER(P), C.POINTER(P), P, P, P],
+        "hccl_hostpipe_status": [P, C.POINTER(C.c_int), I64P],
     }
     for name, args in sigs.items():
         fn = getattr(lib, name)
@@ -106,6 +112,8 @@ def _load() -> C.CDLL:
     lib.hccl_graph_destroy.restype = None
     lib.hccl_plan_destroy.argtypes = [P]
     lib.hccl_plan_destroy.restype = None
+    lib.hccl_hostpipe_destroy.argtypes = [P]
+    lib.hccl_hostpipe_destroy.restype = None
     lib.hccl_status_string.argtypes = [C.c_int]
     lib.hccl_status_string.restype = C.c_char_p
     lib.hccl_last_cuda_error.argtypes = []
@@ -124,7 +132,9 @@ EXPORTS = ["hccl_plan_allreduce", "hccl_plan_reducescatter", "hccl_plan_allgathe
            "hccl_execute_noalloc", "hccl_server_start", "hccl_server_ring", "hccl_server_wait", "hccl_server_stop",
            "hccl_plan_set_user_signals", "hccl_plan_set_trace", "hccl_plan_set_trigger", "hccl_plan_status", "hccl_plan_info",
            "hccl_plan_extents", "hccl_plan_layout", "hccl_plan_destroy", "hccl_status_string", "hccl_last_cuda_error", "hccl_version",
-           "hccl_plan_check_hazards", "hccl_plan_interpret_host"]
+           "hccl_plan_check_hazards", "hccl_plan_interpret_host",
+           "hccl_hostpipe_alltoallv_create", "hccl_hostpipe_windows", "hccl_hostpipe_workspace_bytes", "hccl_hostpipe_bind",
+           "hccl_hostpipe_execute", "hccl_hostpipe_status", "hccl_hostpipe_destroy"]
 
 
 def status_string(status: int) -> str:
@@ -293,6 +303,52 @@ def hccl_plan_alltoallv_dynamic(R: int, max_send_rows, max_recv_rows, dt: int = 
     h = C.c_void_p()
     return _new_plan(_lib.hccl_plan_alltoallv_dynamic(R, _i64(max_send_rows), _i64(max_recv_rows), dt, row_elems,
                                                       C.byref(make_opts(opts)), C.byref(h)), h, "hccl_plan_alltoallv_dynamic")
+
+
+class HostPipe:
+    """Owner of one hccl_hostpipe_t*: AllToAllv through host buffers, pipelined by destination windows."""
+
+    def __init__(self, handle: int):
+        self._h = C.c_void_p(handle)
+
+    def __del__(self):
+        self.destroy()
+
+    def destroy(self):
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.hccl_hostpipe_destroy(self._h)
+        self._h = None
+
+    def windows(self):
+        n = C.c_int32()
+        first = (C.c_int32 * (MAX_RANKS + 1))()
+        _chk(_lib.hccl_hostpipe_windows(self._h, C.byref(n), first), "hccl_hostpipe_windows")
+        return list(first[: n.value + 1])
+
+    def workspace_bytes(self) -> int:
+        n = C.c_size_t()
+        _chk(_lib.hccl_hostpipe_workspace_bytes(self._h, C.byref(n)), "hccl_hostpipe_workspace_bytes")
+        return n.value
+
+    def bind(self, dev_workspace: int, nbytes: int, stream: int = 0):
+        _chk(_lib.hccl_hostpipe_bind(self._h, C.c_void_p(dev_workspace), nbytes, C.c_void_p(stream)), "hccl_hostpipe_bind")
+
+    def execute(self, host_send, host_recv, dev_send, dev_recv, stream_in: int, stream_exec: int, stream_out: int):
+        _chk(_lib.hccl_hostpipe_execute(self._h, _ptr_array(host_send), _ptr_array(host_recv), _ptr_array(dev_send),
+                                        _ptr_array(dev_recv), C.c_void_p(stream_in), C.c_void_p(stream_exec),
+                                        C.c_void_p(stream_out)), "hccl_hostpipe_execute")
+
+    def status(self):
+        st, detail = C.c_int(), C.c_int64()
+        _chk(_lib.hccl_hostpipe_status(self._h, C.byref(st), C.byref(detail)), "hccl_hostpipe_status")
+        return st.value, detail.value
+
+
+def hccl_hostpipe_alltoallv_create(R: int, sendcounts, dt: int = BF16, row_elems: int = 1, n_windows: int = 8, opts=None) -> HostPipe:
+    h = C.c_void_p()
+    _chk(_lib.hccl_hostpipe_alltoallv_create(R, _i64(sendcounts), dt, row_elems, n_windows, C.byref(make_opts(opts)), C.byref(h)),
+         "hccl_hostpipe_alltoallv_create")
+    return HostPipe(h.value)
 
 
 class Graph:

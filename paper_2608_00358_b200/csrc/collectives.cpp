@@ -672,7 +672,18 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
 hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_t* sdispls, const int64_t* recvcounts,
                                   const int64_t* rdispls, hccl_dtype_t dt, int64_t row_elems, const hccl_opts_t* opts,
                                   hccl_plan_t** out) {
+    return hccl::plan_alltoallv_window(R, sendcounts, sdispls, recvcounts, rdispls, dt, row_elems, opts, 0, R, out);
+}
+
+}  // extern "C"
+
+// The AllToAllv planner restricted to the destinations [d_lo, d_hi): the same validation, displacements and
+// buffer extents as the whole exchange, but only the segments bound for those destinations become WQEs.
+hccl_status_t hccl::plan_alltoallv_window(int R, const int64_t* sendcounts, const int64_t* sdispls, const int64_t* recvcounts,
+                                          const int64_t* rdispls, hccl_dtype_t dt, int64_t row_elems, const hccl_opts_t* opts,
+                                          int d_lo, int d_hi, hccl_plan_t** out) {
     if (!out || !sendcounts || R < 1 || R > HCCL_MAX_RANKS || row_elems < 1) return HCCL_ERR_INVALID_ARG;
+    if (d_lo < 0 || d_hi > R || d_lo > d_hi) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
     hccl_opts_t o;
     fill_copy_opts(&o, opts);
@@ -731,14 +742,15 @@ hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_
     hccl_graph* graw = nullptr;
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw));
     GraphPtr g(graw);
-    g->compulsory_bytes = 2 * payload;
     // one subgraph per source rank; zero-length segments produce no WQE at all
+    int64_t moved = 0;
     for (int s = 0; s < R; ++s) {
         int32_t sg;
         CHECK(hccl_graph_add_subgraph(g.get(), s, &sg));
-        for (int d = 0; d < R; ++d) {
+        for (int d = d_lo; d < d_hi; ++d) {
             const int64_t c = sendcounts[(size_t)s * R + d];
             if (c == 0) continue;
+            moved += c * row_bytes;
             hccl_wqe_t w = blank();
             w.op = HCCL_OP_COPY;
             w.count = c * row_bytes;
@@ -747,8 +759,12 @@ hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_
             CHECK(hccl_graph_add_wqe(g.get(), sg, &w, nullptr));
         }
     }
+    g->compulsory_bytes = 2 * moved;
+    (void)payload;
     return hccl_graph_compile(g.get(), &o, out);
 }
+
+extern "C" {
 
 hccl_status_t hccl_plan_alltoallv_dynamic(int R, const int64_t* max_send_rows, const int64_t* max_recv_rows, hccl_dtype_t dt,
                                           int64_t row_elems, const hccl_opts_t* opts, hccl_plan_t** out) {

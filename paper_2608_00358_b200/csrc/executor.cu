@@ -1797,6 +1797,187 @@ hccl_status_t hccl_execute_host(hccl_plan_t* p, const void* const* host_send, vo
     return HCCL_OK;
 }
 
+// ---------------------------------------------------------------------- host pipeline (AllToAllv by destination windows)
+}  // extern "C"
+
+struct hccl_hostpipe {
+    int R = 0;
+    int64_t row_bytes = 0;
+    std::vector<int64_t> counts;          // [s*R+d] rows
+    std::vector<int64_t> sdispl;          // packed, rows
+    std::vector<int64_t> recv_rows;       // per destination
+    std::vector<int32_t> first_dest;      // n_windows + 1
+    std::vector<hccl_plan_t*> plans;      // one per window
+    std::vector<size_t> ws_off;           // each sub-plan's slice of the workspace
+    size_t ws_total = 0;
+    std::vector<cudaEvent_t> in_done, exec_done;
+    cudaEvent_t all_done = nullptr;
+    bool bound = false, ran = false;
+    ~hccl_hostpipe() {
+        for (hccl_plan_t* q : plans) hccl_plan_destroy(q);
+        for (cudaEvent_t e : in_done) cudaEventDestroy(e);
+        for (cudaEvent_t e : exec_done) cudaEventDestroy(e);
+        if (all_done) cudaEventDestroy(all_done);
+    }
+};
+
+extern "C" {
+
+hccl_status_t hccl_hostpipe_alltoallv_create(int R, const int64_t* sendcounts, hccl_dtype_t dt, int64_t row_elems, int n_windows,
+                                             const hccl_opts_t* opts, hccl_hostpipe_t** out) {
+    if (!out || !sendcounts || R < 1 || R > HCCL_MAX_RANKS || row_elems < 1 || n_windows < 1) return HCCL_ERR_INVALID_ARG;
+    if (dt != HCCL_FP32 && dt != HCCL_BF16 && dt != HCCL_FP16) return HCCL_ERR_DTYPE;
+    hccl_hostpipe* hp = new (std::nothrow) hccl_hostpipe();
+    if (!hp) return HCCL_ERR_INVALID_ARG;
+    hp->R = R;
+    hp->row_bytes = row_elems * (dt == HCCL_FP32 ? 4 : 2);
+    hp->counts.assign(sendcounts, sendcounts + (size_t)R * R);
+    hp->sdispl.assign((size_t)R * R, 0);
+    hp->recv_rows.assign(R, 0);
+    int64_t total = 0;
+    for (int s = 0; s < R; ++s) {
+        int64_t acc = 0;
+        for (int d = 0; d < R; ++d) {
+            const int64_t c = sendcounts[(size_t)s * R + d];
+            if (c < 0) {
+                delete hp;
+                return HCCL_ERR_INVALID_ARG;
+            }
+            hp->sdispl[(size_t)s * R + d] = acc;
+            acc += c;
+            hp->recv_rows[d] += c;
+            total += c;
+        }
+    }
+    // contiguous windows of destinations, each closed once it holds its share of the received rows
+    const int W = std::min(n_windows, R);
+    hp->first_dest.push_back(0);
+    int64_t acc = 0, in_window = 0;
+    for (int d = 0; d < R; ++d) {
+        acc += hp->recv_rows[d];
+        in_window += hp->recv_rows[d];
+        const int made = (int)hp->first_dest.size();  // windows closed so far + 1
+        if (made < W && acc * W >= total * made && in_window > 0 && d + 1 < R) {
+            hp->first_dest.push_back(d + 1);
+            in_window = 0;
+        }
+    }
+    hp->first_dest.push_back(R);
+    // a trailing window without rows joins the one before it
+    while (hp->first_dest.size() > 2) {
+        int64_t rows = 0;
+        for (int d = hp->first_dest[hp->first_dest.size() - 2]; d < R; ++d) rows += hp->recv_rows[d];
+        if (rows > 0) break;
+        hp->first_dest.erase(hp->first_dest.end() - 2);
+    }
+    const int nw = (int)hp->first_dest.size() - 1;
+    for (int g = 0; g < nw; ++g) {
+        hccl_plan_t* q = nullptr;
+        hccl_status_t st = hccl::plan_alltoallv_window(R, sendcounts, nullptr, nullptr, nullptr, dt, row_elems, opts,
+                                                       hp->first_dest[g], hp->first_dest[g + 1], &q);
+        if (st != HCCL_OK) {
+            delete hp;
+            return st;
+        }
+        hp->plans.push_back(q);
+        hp->ws_off.push_back(hp->ws_total);
+        hp->ws_total += (size_t)((q->layout.total + 255) / 256 * 256);
+    }
+    *out = hp;
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_hostpipe_windows(const hccl_hostpipe_t* hp, int32_t* n_windows, int32_t* first_dest) {
+    if (!hp || !n_windows) return HCCL_ERR_INVALID_ARG;
+    *n_windows = (int32_t)hp->plans.size();
+    if (first_dest)
+        for (size_t i = 0; i < hp->first_dest.size(); ++i) first_dest[i] = hp->first_dest[i];
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_hostpipe_workspace_bytes(const hccl_hostpipe_t* hp, size_t* bytes) {
+    if (!hp || !bytes) return HCCL_ERR_INVALID_ARG;
+    *bytes = hp->ws_total;
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_hostpipe_bind(hccl_hostpipe_t* hp, void* dev_workspace, size_t bytes, void* stream) {
+    if (!hp || !dev_workspace) return HCCL_ERR_INVALID_ARG;
+    if (((uintptr_t)dev_workspace) % 256) return HCCL_ERR_ALIGNMENT;
+    if (bytes < hp->ws_total) return HCCL_ERR_WORKSPACE;
+    for (size_t g = 0; g < hp->plans.size(); ++g) {
+        hccl_status_t st = hccl_plan_bind(hp->plans[g], (char*)dev_workspace + hp->ws_off[g], (size_t)hp->plans[g]->layout.total, stream);
+        if (st != HCCL_OK) return st;
+    }
+    if (!hp->all_done) {
+        hp->in_done.resize(hp->plans.size());
+        hp->exec_done.resize(hp->plans.size());
+        for (size_t g = 0; g < hp->plans.size(); ++g) {
+            CUDA_TRY(cudaEventCreateWithFlags(&hp->in_done[g], cudaEventDisableTiming));
+            CUDA_TRY(cudaEventCreateWithFlags(&hp->exec_done[g], cudaEventDisableTiming));
+        }
+        CUDA_TRY(cudaEventCreateWithFlags(&hp->all_done, cudaEventDisableTiming));
+    }
+    hp->bound = true;
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_hostpipe_execute(hccl_hostpipe_t* hp, const void* const* host_send, void* const* host_recv, void* const* dev_send,
+                                    void* const* dev_recv, void* stream_in, void* stream_exec, void* stream_out) {
+    if (!hp || !host_send || !host_recv || !dev_send || !dev_recv) return HCCL_ERR_INVALID_ARG;
+    if (!hp->bound) return HCCL_ERR_NOT_BOUND;
+    cudaStream_t si = (cudaStream_t)stream_in, sx = (cudaStream_t)stream_exec, so = (cudaStream_t)stream_out;
+    const int R = hp->R;
+    // the staging buffers are reused: nothing of this call starts before the previous call has finished
+    if (hp->ran) {
+        CUDA_TRY(cudaStreamWaitEvent(si, hp->all_done, 0));
+        CUDA_TRY(cudaStreamWaitEvent(sx, hp->all_done, 0));
+    }
+    for (size_t g = 0; g < hp->plans.size(); ++g) {
+        const int d0 = hp->first_dest[g], d1 = hp->first_dest[g + 1];
+        for (int s = 0; s < R; ++s) {  // rows of source s bound for destinations d0..d1-1: one contiguous slice
+            const int64_t lo = hp->sdispl[(size_t)s * R + d0];
+            const int64_t hi = d1 < R ? hp->sdispl[(size_t)s * R + d1] : hp->sdispl[(size_t)s * R + R - 1] + hp->counts[(size_t)s * R + R - 1];
+            if (hi > lo)
+                CUDA_TRY(cudaMemcpyAsync((char*)dev_send[s] + lo * hp->row_bytes, (const char*)host_send[s] + lo * hp->row_bytes,
+                                         (size_t)((hi - lo) * hp->row_bytes), cudaMemcpyHostToDevice, si));
+        }
+        CUDA_TRY(cudaEventRecord(hp->in_done[g], si));
+        CUDA_TRY(cudaStreamWaitEvent(sx, hp->in_done[g], 0));
+        hccl_status_t st = hccl_execute(hp->plans[g], (const void* const*)dev_send, dev_recv, stream_exec);
+        if (st != HCCL_OK) return st;
+        CUDA_TRY(cudaEventRecord(hp->exec_done[g], sx));
+        CUDA_TRY(cudaStreamWaitEvent(so, hp->exec_done[g], 0));
+        for (int d = d0; d < d1; ++d)
+            if (hp->recv_rows[d] > 0)
+                CUDA_TRY(cudaMemcpyAsync(host_recv[d], dev_recv[d], (size_t)(hp->recv_rows[d] * hp->row_bytes), cudaMemcpyDeviceToHost, so));
+    }
+    CUDA_TRY(cudaEventRecord(hp->all_done, so));
+    hp->ran = true;
+    return HCCL_OK;
+}
+
+hccl_status_t hccl_hostpipe_status(hccl_hostpipe_t* hp, hccl_status_t* device_status, int64_t* detail) {
+    if (!hp || !device_status) return HCCL_ERR_INVALID_ARG;
+    if (!hp->bound) return HCCL_ERR_NOT_BOUND;
+    *device_status = HCCL_OK;
+    for (hccl_plan_t* q : hp->plans) {
+        hccl_status_t ds = HCCL_OK;
+        int64_t dd = 0;
+        hccl_status_t st = hccl_plan_status(q, &ds, &dd);
+        if (st != HCCL_OK) return st;
+        if (ds != HCCL_OK) {
+            *device_status = ds;
+            if (detail) *detail = dd;
+            return HCCL_OK;
+        }
+    }
+    if (detail) *detail = 0;
+    return HCCL_OK;
+}
+
+void hccl_hostpipe_destroy(hccl_hostpipe_t* hp) { delete hp; }
+
 hccl_status_t hccl_plan_status(hccl_plan_t* p, hccl_status_t* device_status, int64_t* detail) {
     if (!p || !device_status) return HCCL_ERR_INVALID_ARG;
     if (!p->workspace) return HCCL_ERR_NOT_BOUND;

@@ -113,4 +113,7 @@ inline int64_t round_tile(int64_t target, int64_t sweep) {
 }
 hccl_status_t compile_graph(const hccl_graph* g, const hccl_opts_t* opts, hccl_plan** out);
 void fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in);
+hccl_status_t plan_alltoallv_window(int R, const int64_t* sendcounts, const int64_t* sdispls, const int64_t* recvcounts,
+                                    const int64_t* rdispls, hccl_dtype_t dt, int64_t row_elems, const hccl_opts_t* opts,
+                                    int d_lo, int d_hi, hccl_plan_t** out);
 }  // namespace hccl
