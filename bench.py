@@ -283,8 +283,16 @@ def run_profile_case(args):
     import torch
     from paper_2608_00358_b200 import binding as hb
     from paper_2608_00358_b200 import workloads as wk
-    algo = {"c3ring": hb.ALGO_RING, "c3fused": hb.ALGO_RING_FUSED}[args.profile_case]
-    wl = wk.config3(algo=algo, n=args.profile_n)
+    if args.profile_case in ("agfanout", "agoneshot"):
+        # AllGather R = 32, 1 Mi bf16 (2 MiB) per rank: 64 MiB read, 2 GiB written
+        R, n = 32, 1 << 20
+        algo = hb.ALGO_FANOUT if args.profile_case == "agfanout" else hb.ALGO_ONESHOT
+        send = [torch.randn(n, device="cuda").to(torch.bfloat16) for _ in range(R)]
+        recv = [torch.empty(n * R, dtype=torch.bfloat16, device="cuda") for _ in range(R)]
+        wl = wk._bind("allgather_r32_bf16_1Mi_" + args.profile_case[2:], hb.hccl_plan_allgather(R, None, n, hb.BF16, algo), send, recv, {})
+    else:
+        algo = {"c3ring": hb.ALGO_RING, "c3fused": hb.ALGO_RING_FUSED}[args.profile_case]
+        wl = wk.config3(algo=algo, n=args.profile_n)
     ms = wk.time_back_to_back(wl, args.steps, max(args.warmup, 3))
     i = wl.info
     print(json.dumps({"case": args.profile_case, "workload": wl.name, "ms": ms, "schedule_bytes": int(i.schedule_bytes),
@@ -476,7 +484,7 @@ def main():
     ap.add_argument("--no-side", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--profile-n", type=int, default=1 << 23, help="elements per rank of the --profile-case")
-    ap.add_argument("--profile-case", default="", choices=["", "c3ring", "c3fused"],
+    ap.add_argument("--profile-case", default="", choices=["", "c3ring", "c3fused", "agfanout", "agoneshot"],
                     help="run only a small single-kernel case (for ncu captures), not the benchmark")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
