@@ -1475,7 +1475,7 @@ __global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant
     uint32_t* s_tp = reinterpret_cast<uint32_t*>(s_rd + RR);  // [RR+1] exclusive prefix of tiles per segment
     __shared__ int s_bad;
     __shared__ unsigned long long s_bad_at;
-    __shared__ uint32_t s_ticket;
+    __shared__ uint32_t s_team_ticket[2];
     __shared__ int s_live;
     const uint32_t tid = threadIdx.x, nth = blockDim.x, lane = tid & 31u, warp = tid >> 5, nwarps = nth >> 5;
     init_epoch(q);
@@ -1563,31 +1563,37 @@ __global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant
                 }
             }
             const uint32_t total = s_tp[RR];
-            uint32_t next = 0;
-            if (tid == 0) next = atomicAdd(&q.ctl->ticket, 1);
-            for (;;) {
-                if (tid == 0) {
-                    s_ticket = next;
-                    if (next < total) next = atomicAdd(&q.ctl->ticket, 1);  // one ahead
+            // The block works as teams of 256 threads, each claiming and copying tiles on its own (named
+            // barrier per team), so that one team's gap between two tiles is covered by the other's copy.
+            const uint32_t team_size = nth >= 512 ? 256u : nth, n_teams = nth / team_size;
+            const uint32_t team = tid / team_size, ltid = tid - team * team_size;
+            if (team < n_teams) {
+                uint32_t next = 0;
+                if (ltid == 0) next = atomicAdd(&q.ctl->ticket, 1);
+                for (;;) {
+                    if (ltid == 0) {
+                        s_team_ticket[team] = next;
+                        if (next < total) next = atomicAdd(&q.ctl->ticket, 1);  // one ahead
+                    }
+                    named_sync(1 + team, team_size);
+                    const uint32_t t = s_team_ticket[team];
+                    if (t >= total) break;
+                    // segment of tile t: the last i with s_tp[i] <= t (zero-length segments share a prefix value
+                    // with their successor and are skipped by taking the last one)
+                    uint32_t lo = 0, hi = RR;
+                    while (hi - lo > 1) {
+                        const uint32_t mid = (lo + hi) >> 1;
+                        if (s_tp[mid] <= t) lo = mid; else hi = mid;
+                    }
+                    const uint32_t i = lo, s = i / R, d = i % R;
+                    const unsigned long long off = (unsigned long long)(t - s_tp[i]) * q.tile_bytes;
+                    const unsigned long long seg = (unsigned long long)s_cnt[i] * q.row_bytes;
+                    const uint32_t len = (uint32_t)min((unsigned long long)q.tile_bytes, seg - off);
+                    const char* src = (const char*)q.send[s] + (unsigned long long)s_sd[i] * q.row_bytes + off;
+                    char* dst = (char*)q.recv[d] + (unsigned long long)s_rd[i] * q.row_bytes + off;
+                    copy_tile_lsu<true>(dst, src, len, ltid, team_size);
+                    named_sync(1 + team, team_size);  // the ticket word is rewritten only after everyone has read it
                 }
-                __syncthreads();
-                const uint32_t t = s_ticket;
-                if (t >= total) break;
-                // segment of tile t: the last i with s_tp[i] <= t (zero-length segments share a prefix value
-                // with their successor and are skipped by taking the last one)
-                uint32_t lo = 0, hi = RR;
-                while (hi - lo > 1) {
-                    const uint32_t mid = (lo + hi) >> 1;
-                    if (s_tp[mid] <= t) lo = mid; else hi = mid;
-                }
-                const uint32_t i = lo, s = i / R, d = i % R;
-                const unsigned long long off = (unsigned long long)(t - s_tp[i]) * q.tile_bytes;
-                const unsigned long long seg = (unsigned long long)s_cnt[i] * q.row_bytes;
-                const uint32_t len = (uint32_t)min((unsigned long long)q.tile_bytes, seg - off);
-                const char* src = (const char*)q.send[s] + (unsigned long long)s_sd[i] * q.row_bytes + off;
-                char* dst = (char*)q.recv[d] + (unsigned long long)s_rd[i] * q.row_bytes + off;
-                copy_tile_lsu<true>(dst, src, len, tid, nth);
-                __syncthreads();
             }
         }
     }
