@@ -324,8 +324,8 @@ hccl_status_t hccl_execute_host(hccl_plan_t*, const void* const* host_send, void
 /* ------------------------------------------------------------------------
  * AllToAllv through HOST buffers, pipelined by destination (the paper spreads an AllToAllv over several
  * subgraphs to keep the links busy, Sec. IV-A; here the link is the host interface and the pieces are
- * windows of destination ranks). The destinations are cut into n_windows contiguous groups of about equal
- * received bytes. For window g: the rows bound for its destinations are copied host->device (with packed
+ * windows of destination ranks). The destinations are cut into n_windows contiguous groups by received
+ * bytes; the first and last few groups are smaller, since only their copy-in and copy-out overlap nothing. For window g: the rows bound for its destinations are copied host->device (with packed
  * send displacements they are one contiguous slice of every send buffer), exchanged by a sub-plan that
  * holds only those segments, and the window's receive buffers are copied device->host. The three steps
  * run on three caller-supplied streams, ordered by events, so that copy-in of window g+1, exchange of g
@@ -336,7 +336,10 @@ hccl_status_t hccl_execute_host(hccl_plan_t*, const void* const* host_send, void
  *             and creates the ordering events (no device memory is allocated).
  *   execute   asynchronous; everything has completed when stream_out has. host buffers should be pinned.
  *             dev_send / dev_recv are the caller's staging buffers (full extents, as for hccl_execute).
- *             A second execute may be enqueued at once: it starts after the first has finished.
+ *             A second execute may be enqueued at once, on the same three streams: its copies-in start when
+ *             the first call's last exchange has run, and its exchange of a window when the first call's
+ *             copy-out of that window has finished. The host buffers of a call must stay untouched until
+ *             stream_out has passed that call.
  *   status    after synchronising stream_out: the first device-side failure of any window, else HCCL_OK.
  *   windows   first_dest[g] .. first_dest[g+1]-1 are window g's destinations (n_windows+1 entries).
  * ------------------------------------------------------------------------ */

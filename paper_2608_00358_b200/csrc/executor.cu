@@ -1816,13 +1816,14 @@ struct hccl_hostpipe {
     std::vector<hccl_plan_t*> plans;      // one per window
     std::vector<size_t> ws_off;           // each sub-plan's slice of the workspace
     size_t ws_total = 0;
-    std::vector<cudaEvent_t> in_done, exec_done;
+    std::vector<cudaEvent_t> in_done, exec_done, out_done;
     cudaEvent_t all_done = nullptr;
     bool bound = false, ran = false;
     ~hccl_hostpipe() {
         for (hccl_plan_t* q : plans) hccl_plan_destroy(q);
         for (cudaEvent_t e : in_done) cudaEventDestroy(e);
         for (cudaEvent_t e : exec_done) cudaEventDestroy(e);
+        for (cudaEvent_t e : out_done) cudaEventDestroy(e);
         if (all_done) cudaEventDestroy(all_done);
     }
 };
@@ -1855,15 +1856,19 @@ hccl_status_t hccl_hostpipe_alltoallv_create(int R, const int64_t* sendcounts, h
             total += c;
         }
     }
-    // contiguous windows of destinations, each closed once it holds its share of the received rows
+    // Contiguous windows of destinations, each closed once the rows received so far reach its cumulative
+    // share. The shares taper towards both ends (weights 1, 2, 3, 4, 4, ..., 4, 3, 2, 1): the first copy-in
+    // and the last copy-out are the only steps nothing overlaps, so those windows are the small ones.
     const int W = std::min(n_windows, R);
+    std::vector<int64_t> cum(W + 1, 0);
+    for (int g = 0; g < W; ++g) cum[g + 1] = cum[g] + std::min(std::min(g + 1, W - g), 4);
     hp->first_dest.push_back(0);
     int64_t acc = 0, in_window = 0;
     for (int d = 0; d < R; ++d) {
         acc += hp->recv_rows[d];
         in_window += hp->recv_rows[d];
         const int made = (int)hp->first_dest.size();  // windows closed so far + 1
-        if (made < W && acc * W >= total * made && in_window > 0 && d + 1 < R) {
+        if (made < W && (__int128)acc * cum[W] >= (__int128)total * cum[made] && in_window > 0 && d + 1 < R) {
             hp->first_dest.push_back(d + 1);
             in_window = 0;
         }
@@ -1918,9 +1923,11 @@ hccl_status_t hccl_hostpipe_bind(hccl_hostpipe_t* hp, void* dev_workspace, size_
     if (!hp->all_done) {
         hp->in_done.resize(hp->plans.size());
         hp->exec_done.resize(hp->plans.size());
+        hp->out_done.resize(hp->plans.size());
         for (size_t g = 0; g < hp->plans.size(); ++g) {
             CUDA_TRY(cudaEventCreateWithFlags(&hp->in_done[g], cudaEventDisableTiming));
             CUDA_TRY(cudaEventCreateWithFlags(&hp->exec_done[g], cudaEventDisableTiming));
+            CUDA_TRY(cudaEventCreateWithFlags(&hp->out_done[g], cudaEventDisableTiming));
         }
         CUDA_TRY(cudaEventCreateWithFlags(&hp->all_done, cudaEventDisableTiming));
     }
@@ -1934,11 +1941,10 @@ hccl_status_t hccl_hostpipe_execute(hccl_hostpipe_t* hp, const void* const* host
     if (!hp->bound) return HCCL_ERR_NOT_BOUND;
     cudaStream_t si = (cudaStream_t)stream_in, sx = (cudaStream_t)stream_exec, so = (cudaStream_t)stream_out;
     const int R = hp->R;
-    // the staging buffers are reused: nothing of this call starts before the previous call has finished
-    if (hp->ran) {
-        CUDA_TRY(cudaStreamWaitEvent(si, hp->all_done, 0));
-        CUDA_TRY(cudaStreamWaitEvent(sx, hp->all_done, 0));
-    }
+    // The staging buffers are reused by the next call. Its copies-in may start once the previous call's last
+    // exchange has run (nothing reads the send staging after that), and its exchange of window g once the
+    // previous call's copy-out of window g has finished; so one call's drain overlaps the next one's fill.
+    if (hp->ran) CUDA_TRY(cudaStreamWaitEvent(si, hp->exec_done.back(), 0));
     for (size_t g = 0; g < hp->plans.size(); ++g) {
         const int d0 = hp->first_dest[g], d1 = hp->first_dest[g + 1];
         for (int s = 0; s < R; ++s) {  // rows of source s bound for destinations d0..d1-1: one contiguous slice
@@ -1950,6 +1956,7 @@ hccl_status_t hccl_hostpipe_execute(hccl_hostpipe_t* hp, const void* const* host
         }
         CUDA_TRY(cudaEventRecord(hp->in_done[g], si));
         CUDA_TRY(cudaStreamWaitEvent(sx, hp->in_done[g], 0));
+        if (hp->ran) CUDA_TRY(cudaStreamWaitEvent(sx, hp->out_done[g], 0));
         hccl_status_t st = hccl_execute(hp->plans[g], (const void* const*)dev_send, dev_recv, stream_exec);
         if (st != HCCL_OK) return st;
         CUDA_TRY(cudaEventRecord(hp->exec_done[g], sx));
@@ -1957,6 +1964,7 @@ hccl_status_t hccl_hostpipe_execute(hccl_hostpipe_t* hp, const void* const* host
         for (int d = d0; d < d1; ++d)
             if (hp->recv_rows[d] > 0)
                 CUDA_TRY(cudaMemcpyAsync(host_recv[d], dev_recv[d], (size_t)(hp->recv_rows[d] * hp->row_bytes), cudaMemcpyDeviceToHost, so));
+        CUDA_TRY(cudaEventRecord(hp->out_done[g], so));
     }
     CUDA_TRY(cudaEventRecord(hp->all_done, so));
     hp->ran = true;
