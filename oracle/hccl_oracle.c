@@ -338,6 +338,27 @@ int oracle_allreduce_oneshot_f32(int R, int64_t n, int dt, const void *const *X,
     return 0;
 }
 
+/* Binary-tree order (Sec. III-B.2 mentions tree-based NMC reductions as a user of multi-dependency joins):
+ * the R inputs are the leaves, in rank order; each level adds neighbours in pairs, (v_0 + v_1), (v_2 + v_3),
+ * ..., and an odd one out moves up unchanged; the levels repeat until one value is left. FP32 adds, one
+ * rounding to the stored type at the root; every rank receives the result. */
+int oracle_allreduce_tree_f32(int R, int64_t n, int dt, const void *const *X, void *const *Y) {
+    if (R < 1 || R > 4096) return 1;
+    volatile float v[4096];
+    for (int64_t i = 0; i < n; ++i) {
+        for (int q = 0; q < R; ++q) v[q] = (float)load_elem(X[q], i, dt);
+        int m = R;
+        while (m > 1) {
+            const int pairs = m / 2;
+            for (int j = 0; j < pairs; ++j) v[j] = v[2 * j] + v[2 * j + 1];
+            if (m & 1) v[pairs] = v[m - 1];
+            m = pairs + (m & 1);
+        }
+        for (int r = 0; r < R; ++r) store_elem(Y[r], i, dt, (double)v[0]);
+    }
+    return 0;
+}
+
 /* Ring order with a direction per segment (bidirectional rings, Sec. III-B.2: half of the data travels
  * r -> r+1, the other half r -> r-1). Segment s covers elements [seg_off[s], seg_off[s+1]) of chunk
  * seg_chunk[s] and travels in direction seg_dir[s] (+1 or -1): its elements are summed as

@@ -210,6 +210,13 @@ def allreduce_oneshot_f32(dt: int, X: list) -> list:
     return Y
 
 
+def allreduce_tree_f32(dt: int, X: list) -> list:
+    R, n = len(X), X[0].size
+    Y = [np.empty(n, dtype=np_dtype(dt)) for _ in range(R)]
+    _check(lib().oracle_allreduce_tree_f32(R, ctypes.c_int64(n), dt, _ptrs(X), _ptrs(Y, True)), "tree")
+    return Y
+
+
 def ulp_distance(dt: int, a: np.ndarray, b: np.ndarray) -> np.ndarray:
     assert a.size == b.size and a.dtype == b.dtype
     out = np.empty(a.size, dtype=np.int64)

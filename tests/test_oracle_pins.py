@@ -427,3 +427,48 @@ def test_bidirectional_order_example():
     f = orc.allreduce_ring_dir_f32(FP32, X, so, sc, np.array([1]))[0][0]      # ((2^24 + 1) - 2^24) + 1 = 0 + 1 = 1
     b = orc.allreduce_ring_dir_f32(FP32, X, so, sc, np.array([-1]))[0][0]     # ((-2^24 + 1) + 2^24) + 1 = 1 + 1 = 2
     assert f == 1.0 and b == 2.0
+
+
+# ----------------------------------------------------------------- binary-tree order
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("R", [1, 2, 3, 4, 5, 6, 7, 8, 13, 16, 64])
+def test_tree_order_built_from_the_pinned_two_input_sum(R, dt):
+    """The tree is pairs of neighbours, level by level, an odd one out moving up unchanged. Rebuilt here from
+    numpy float32 adds (a different implementation of the FP32 add than the oracle's C) and checked against
+    the closed form R(R+1)/2 on rank-constant inputs."""
+    n = 97
+    X = synth.normal_ranks(R, n, dt, seed=R * 7 + 1)
+    v = [synth.from_bits(x, dt).astype(np.float32) for x in X]
+    while len(v) > 1:
+        nxt = [v[2 * j] + v[2 * j + 1] for j in range(len(v) // 2)]   # numpy float32 add
+        if len(v) % 2:
+            nxt.append(v[-1])
+        v = nxt
+    want = orc.round_to(dt, v[0].astype(np.float64))
+    Y = orc.allreduce_tree_f32(dt, X)
+    for r in range(R):
+        assert np.array_equal(Y[r], want)
+    # within the acceptance rule of the FP64 definition
+    ref, s = orc.allreduce(dt, X)[0], orc.sum_f64(dt, X)
+    if dt == FP32:
+        assert np.all(np.abs(Y[0].astype(np.float64) - s) <= 1e-5 * np.abs(s) + 1e-6)
+    else:
+        assert orc.ulp_distance(dt, Y[0], ref).max() <= 1
+    # closed form, exact in every type for these R
+    if R in (1, 2, 4, 8, 16, 64):
+        Xc = [synth.to_bits(np.full(n, r + 1, dtype=np.float32), dt) for r in range(R)]
+        assert np.all(synth.from_bits(orc.allreduce_tree_f32(dt, Xc)[0], dt) == R * (R + 1) / 2)
+
+
+def test_tree_order_example():
+    # R = 5: ((x0 + x1) + (x2 + x3)) + x4. Values chosen so that other orders give other FP32 results.
+    big, one = np.float32(2.0 ** 24), np.float32(1.0)
+    X = [np.array([v], dtype=np.float32) for v in (big, one, one, -big, one)]
+    # (2^24 + 1) -> 2^24 ; (1 - 2^24) -> -2^24 + 1 exactly ; sum = 1 ; + 1 = 2
+    assert orc.allreduce_tree_f32(FP32, X)[3][0] == 2.0
+    # rank order 0..4: ((2^24 + 1) + 1) -> 2^24, - 2^24 = 0, + 1 = 1
+    assert orc.allreduce_oneshot_f32(FP32, X)[0][0] == 1.0
+    assert orc.allreduce(FP32, X)[0][0] == 3.0      # the FP64 definition keeps every 1
+    # swapping the two members of a pair changes nothing (FP32 addition commutes exactly)
+    Xs = [X[1], X[0], X[3], X[2], X[4]]
+    assert orc.allreduce_tree_f32(FP32, Xs)[0][0] == 2.0
