@@ -198,7 +198,7 @@ def side_configs(quick: bool):
     oracle_time("2_alltoallv_r8_bf16_dim128", _oracle_a2a)
     del w1, w2
     for m in (4096, 65536, 262144, 1 << 20):
-        for algo, nm in ((hb.ALGO_ONESHOT, "oneshot"), (hb.ALGO_RING, "ring"), (hb.ALGO_FANOUT, "fanout")):
+        for algo, nm in ((hb.ALGO_ONESHOT, "oneshot"), (hb.ALGO_RING, "ring"), (hb.ALGO_TREE, "tree"), (hb.ALGO_FANOUT, "fanout")):
             wl5 = wk.config5(m, algo)
             key5 = "5_allreduce_r8_bf16_%dB_%s" % (m, nm)
             latency(wl5, key5)
@@ -253,7 +253,7 @@ def side_configs(quick: bool):
     for n in ((1 << 16, 1 << 22) if quick else (1 << 16, 1 << 22, 1 << 25)):
         send = [torch.randn(n, device="cuda").to(torch.bfloat16) for _ in range(64)]
         recv = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(64)]
-        for algo, nm in ((hb.ALGO_RING, "ring"), (hb.ALGO_RING_2LEVEL, "ring_2level"), (hb.ALGO_RING_FUSED, "ring_fused"), (hb.ALGO_FANOUT, "fanout")):
+        for algo, nm in ((hb.ALGO_RING, "ring"), (hb.ALGO_RING_2LEVEL, "ring_2level"), (hb.ALGO_TREE, "tree"), (hb.ALGO_RING_FUSED, "ring_fused"), (hb.ALGO_FANOUT, "fanout")):
             sched("next_allreduce_r64_bf16_%d_%s" % (n, nm), hb.hccl_plan_allreduce(64, n, hb.BF16, algo, dict(rack_size=16)), send, recv, 20)
         del send, recv
         torch.cuda.empty_cache()

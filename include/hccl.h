@@ -71,11 +71,16 @@ typedef enum {
                                 run round each rack's ring first, then round the ring of racks, and results
                                 are gathered across racks first, then inside each rack, so that only 1/rack_size
                                 of the data ever crosses between racks. AllReduce and AllGather. */
-    HCCL_ALGO_FANOUT = 4     /* one-shot with the destinations fused: each piece of the result is produced once
+    HCCL_ALGO_FANOUT = 4,    /* one-shot with the destinations fused: each piece of the result is produced once
                                 (AllReduce: one sum over all ranks in rank order 0..R-1, the one-shot's order;
                                 AllGather: one read of the chunk) and written into all R receive buffers by the
                                 same work item. Possible only because the virtual ranks share one memory; not in
                                 the paper. Reported as its own algorithm, never as "one-shot". */
+    HCCL_ALGO_TREE = 5       /* AllReduce by a binary tree of two-input sums (tree-based NMC reduction, Sec.
+                                III-B.2): per granule of opts.chunk_bytes, neighbours in rank order are added in
+                                pairs level by level (an odd one out moves up unchanged), FP32 partials in scratch,
+                                one rounding at the root into rank 0's buffer, then a binomial tree of copies to
+                                every rank. Dependency depth 2*ceil(log2 R). */
 } hccl_algo_t;
 
 /* Which data mover the executor uses for aligned bulk work. */
@@ -132,7 +137,7 @@ typedef struct hccl_graph hccl_graph_t; /* opaque, host-owned: a work packet und
  * FP32 data keeps partials in the receive buffers; 16-bit data keeps FP32 partials in workspace
  * scratch and is rounded once, on the last reduce step. ONESHOT: R independent R-input sums in rank
  * order 0..R-1. FANOUT: that sum formed once per element and stored into all R receive buffers (same
- * bits as ONESHOT). RING_FUSED, RING_2LEVEL: see hccl_algo_t. Send and receive buffers: count elements each. */
+ * bits as ONESHOT). RING_FUSED, RING_2LEVEL, TREE: see hccl_algo_t. Send and receive buffers: count elements each. */
 hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_algo_t algo,
                                   const hccl_opts_t* opts, hccl_plan_t** out);
 

@@ -431,6 +431,126 @@ hccl_status_t plan_allgather_2level(int R, const std::vector<int64_t>& offs, hcc
     return hccl_graph_compile(g.get(), &o, out);
 }
 
+// Binary-tree AllReduce built from the two-input sum alone (Sec. III-B.2 names tree-based NMC reductions):
+// per granule, neighbours are added in pairs level by level (an odd one out moves up unchanged) with FP32
+// partials in scratch, the root is rounded into rank 0's receive buffer, and a binomial tree of copies
+// carries it to every rank. Depth 2*ceil(log2 R) instead of the ring's 2(R-1).
+hccl_status_t plan_allreduce_tree(int R, int64_t count, hccl_dtype_t dt, hccl_opts_t o, bool group_given, hccl_plan_t** out) {
+    const int es = elem_bytes(dt);
+    std::vector<int64_t> ext(R, count * es);
+    const int64_t granule = std::max<int64_t>(64, (int64_t)(o.chunk_bytes / (uint64_t)es) / 64 * 64);
+    const int64_t ng = count > 0 ? (count + granule - 1) / granule : 0;
+    if (!group_given && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<int64_t>(ng, 1);  // small: all granules together
+    const int64_t group = std::max<int64_t>(1, o.chain_group);
+    const int half = (R + 1) / 2;                                 // scratch slots one granule needs
+    const int64_t n_sets = std::min<int64_t>(std::max<int64_t>(ng, 1), 2 * group);  // recycled sets of slots
+    const int64_t slot_elems = (int64_t)align_up((uint64_t)std::min<int64_t>(granule, std::max<int64_t>(count, 1)), 64);
+    const int64_t scratch = R > 2 ? n_sets * half * slot_elems * 4 : 0;
+    const int64_t tile_elems = pick_tile_elems(std::min<int64_t>(std::max<int64_t>(count, 1), group * granule), o, 4, HCCL_OP_REDUCE);
+    hccl_graph* graw = nullptr;
+    CHECK(hccl_graph_create(R, ext.data(), ext.data(), scratch, 0, &graw));
+    GraphPtr g(graw);
+    g->compulsory_bytes = 2ll * R * count * es;
+
+    struct Node {
+        hccl_ref_t ref;
+        int dt;
+        int leaf;       // leftmost leaf (rank) under this node
+        int64_t made;   // WQE that produced it, -1 for a raw input
+    };
+    std::vector<std::vector<Node>> nodes((size_t)ng);
+    std::vector<int32_t> sg((size_t)ng);
+    std::vector<int64_t> root((size_t)ng, -1);
+    std::vector<std::vector<int64_t>> have((size_t)ng, std::vector<int64_t>(R, -1));  // producer of Y_r's copy of the granule
+    int K = 0;
+    while ((1 << K) < R) ++K;
+    for (int64_t i = 0; i < ng; ++i) {
+        CHECK(hccl_graph_add_subgraph(g.get(), 0, &sg[i]));
+        const int64_t e0 = i * granule;
+        for (int r = 0; r < R; ++r) nodes[i].push_back(Node{ref(HCCL_BUF_SEND, r, e0 * es), dt, r, -1});
+    }
+    for (int64_t g0 = 0; g0 < ng; g0 += group) {
+        const int64_t g1 = std::min(ng, g0 + group);
+        // ---- up: K levels of pairwise sums
+        for (int level = 0; level < K; ++level) {
+            for (int64_t i = g0; i < g1; ++i) {
+                const int64_t e0 = i * granule, len = std::min(granule, count - e0);
+                std::vector<Node>& v = nodes[i];
+                if (v.size() < 2) continue;
+                std::vector<Node> next;
+                for (size_t j = 0; j + 1 < v.size(); j += 2) {
+                    const Node &a = v[j], &b = v[j + 1];
+                    const bool final = v.size() == 2;
+                    hccl_wqe_t w = blank();
+                    w.op = HCCL_OP_REDUCE;
+                    w.count = len;
+                    w.tile_count = tile_elems;
+                    w.a = a.ref; w.dtype_a = a.dt;
+                    w.b = b.ref; w.dtype_b = b.dt;
+                    Node res;
+                    res.leaf = a.leaf;
+                    if (final) {
+                        res.ref = ref(HCCL_BUF_RECV, 0, e0 * es);
+                        res.dt = dt;
+                    } else {
+                        res.ref = ref(HCCL_BUF_SCRATCH, 0, (((i % n_sets) * half) + a.leaf / 2) * slot_elems * 4);
+                        res.dt = HCCL_FP32;
+                    }
+                    w.dst = res.ref; w.dtype_dst = res.dt;
+                    // dependencies: the producers of both operands, tile by tile; a fresh scratch slot of a
+                    // recycled set also waits for the set's previous user to have finished with it
+                    int64_t d1 = a.made, d2 = b.made;
+                    if (!final && a.made < 0 && i >= n_sets && root[i - n_sets] >= 0) d1 = root[i - n_sets];
+                    if (d1 < 0) { d1 = d2; d2 = -1; }
+                    if (d1 >= 0) {
+                        w.dep_flags = HCCL_DEP_WQE_SYNC | HCCL_DEP_ELEMENTWISE;
+                        w.dep_wqe = d1;
+                        if (d2 >= 0) {
+                            w.dep_flags |= HCCL_DEP_ELEMENTWISE2;
+                            w.dep_wqe2 = d2;
+                        }
+                    }
+                    CHECK(hccl_graph_add_wqe(g.get(), sg[i], &w, &res.made));
+                    if (final) root[i] = res.made;
+                    next.push_back(res);
+                }
+                if (v.size() & 1) next.push_back(v.back());
+                v.swap(next);
+            }
+        }
+        // ---- R == 1: the "sum" is a copy
+        for (int64_t i = g0; i < g1 && R == 1; ++i) {
+            const int64_t e0 = i * granule, len = std::min(granule, count - e0);
+            hccl_wqe_t w = blank();
+            w.op = HCCL_OP_COPY;
+            w.count = len * es;
+            w.tile_count = tile_elems * es;
+            w.a = ref(HCCL_BUF_SEND, 0, e0 * es);
+            w.dst = ref(HCCL_BUF_RECV, 0, e0 * es);
+            CHECK(hccl_graph_add_wqe(g.get(), sg[i], &w, &root[i]));
+        }
+        // ---- down: binomial tree of copies from rank 0
+        for (int64_t i = g0; i < g1; ++i) have[i][0] = root[i];
+        for (int k = K - 1; k >= 0; --k) {
+            for (int64_t i = g0; i < g1; ++i) {
+                const int64_t e0 = i * granule, len = std::min(granule, count - e0);
+                for (int r = 0; r + (1 << k) < R; r += 1 << (k + 1)) {
+                    hccl_wqe_t w = blank();
+                    w.op = HCCL_OP_COPY;
+                    w.count = len * es;
+                    w.tile_count = tile_elems * es;
+                    w.a = ref(HCCL_BUF_RECV, r, e0 * es);
+                    w.dst = ref(HCCL_BUF_RECV, r + (1 << k), e0 * es);
+                    w.dep_flags = HCCL_DEP_WQE_SYNC | HCCL_DEP_ELEMENTWISE;
+                    w.dep_wqe = have[i][r];
+                    CHECK(hccl_graph_add_wqe(g.get(), sg[i], &w, &have[i][r + (1 << k)]));
+                }
+            }
+        }
+    }
+    return hccl_graph_compile(g.get(), &o, out);
+}
+
 }  // namespace
 
 extern "C" {
@@ -440,7 +560,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     if (!out || R < 1 || R > HCCL_MAX_RANKS || count < 0) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
     if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_RING_2LEVEL &&
-        algo != HCCL_ALGO_FANOUT) return HCCL_ERR_INVALID_ARG;
+        algo != HCCL_ALGO_FANOUT && algo != HCCL_ALGO_TREE) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
     fill_ring_opts(&o, opts, (int64_t)R * count * elem_bytes(dt), algo == HCCL_ALGO_RING_FUSED || algo == HCCL_ALGO_ONESHOT || algo == HCCL_ALGO_FANOUT || R == 1);
     if (algo == HCCL_ALGO_RING_2LEVEL) {
@@ -450,6 +570,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
         if (o.rack_size >= 2 && R / o.rack_size >= 2) return plan_allreduce_2level(R, count, dt, o, out);
         algo = HCCL_ALGO_RING;
     }
+    if (algo == HCCL_ALGO_TREE) return plan_allreduce_tree(R, count, dt, o, opts && opts->chain_group != 0, out);
     const int es = elem_bytes(dt);
     std::vector<int64_t> ext(R, count * es);
     const int64_t compulsory = 2ll * R * count * es;

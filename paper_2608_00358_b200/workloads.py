@@ -99,7 +99,7 @@ def config5(m_bytes: int, algo: int, opts=None, seed=0) -> Workload:
     send = [torch.from_numpy(x.view(np.int16)).cuda() for x in X]
     recv = [torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(R)]
     plan = hb.hccl_plan_allreduce(R, n, hb.BF16, algo, opts)
-    name = "allreduce_%s_r8_bf16_%dB" % ({hb.ALGO_RING: "ring", hb.ALGO_ONESHOT: "oneshot", hb.ALGO_RING_FUSED: "ringfused", hb.ALGO_FANOUT: "fanout"}[algo], m_bytes)
+    name = "allreduce_%s_r8_bf16_%dB" % ({hb.ALGO_RING: "ring", hb.ALGO_ONESHOT: "oneshot", hb.ALGO_RING_FUSED: "ringfused", hb.ALGO_FANOUT: "fanout", hb.ALGO_TREE: "tree"}[algo], m_bytes)
     return _bind(name, plan, send, recv, dict(host_inputs=X, dt=hb.BF16, n=n, R=R))
 
 

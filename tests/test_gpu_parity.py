@@ -29,6 +29,7 @@ def _check_allreduce(R, n, dt, algo, opts, X=None, iters=1, misalign=0):
     Y = run_plan(p, X, iters=iters, misalign=misalign)
     exact, want = orc.sum_f64(dt, X), orc.allreduce(dt, X)
     bitwise = orc.allreduce_oneshot_f32(dt, X) if algo in (hb.ALGO_ONESHOT, hb.ALGO_FANOUT) else \
+        orc.allreduce_tree_f32(dt, X) if algo == hb.ALGO_TREE else \
         orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
     for r in range(R):
         got = Y[r].view(np_dtype(dt))
@@ -37,7 +38,7 @@ def _check_allreduce(R, n, dt, algo, opts, X=None, iters=1, misalign=0):
 
 
 @pytest.mark.parametrize("dt", DTYPES)
-@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED, hb.ALGO_FANOUT])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED, hb.ALGO_FANOUT, hb.ALGO_TREE])
 @pytest.mark.parametrize("R,n", [(1, 5), (2, 9), (3, 2), (4, 257), (5, 1000), (8, 4099), (4, 0), (4, 3), (8, 100003)])
 def test_allreduce_small(R, n, dt, algo, engine):
     _check_allreduce(R, n, dt, algo, _with(dict(tile_bytes=1024, chunk_bytes=4096, chain_group=2, sm_budget=8), engine), iters=2)
@@ -57,6 +58,7 @@ def test_allreduce_misaligned_buffers(misalign, dt, engine):
     _check_allreduce(4, 10007, dt, hb.ALGO_RING, _with(dict(tile_bytes=4096, sm_budget=16), engine), misalign=misalign)
     _check_allreduce(4, 10007, dt, hb.ALGO_ONESHOT, _with(dict(tile_bytes=4096, sm_budget=16), engine), misalign=misalign)
     _check_allreduce(4, 10007, dt, hb.ALGO_FANOUT, _with(dict(tile_bytes=4096, sm_budget=16), engine), misalign=misalign)
+    _check_allreduce(5, 10007, dt, hb.ALGO_TREE, _with(dict(tile_bytes=4096, chunk_bytes=8192, chain_group=1, sm_budget=16), engine), misalign=misalign)
 
 
 def test_config1_allreduce_ring_r4_fp32(engine):
@@ -64,7 +66,7 @@ def test_config1_allreduce_ring_r4_fp32(engine):
     _check_allreduce(4, 1 << 20, hb.FP32, hb.ALGO_RING, _with(None, engine), X=X, iters=3)
 
 
-@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT, hb.ALGO_TREE])
 @pytest.mark.parametrize("m", [4096, 65536, 262144, 1 << 20])
 def test_config5_allreduce_r8_bf16(m, algo, engine):
     X = synth.normal_ranks(8, m // 2, hb.BF16, seed=m)
@@ -76,7 +78,7 @@ def test_closed_form_on_device(engine):
         for R in (2, 4, 8, 16):
             n = 3000
             X = [synth.to_bits(np.full(n, r + 1, dtype=np.float32), dt) for r in range(R)]
-            for algo in (hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT):
+            for algo in (hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT, hb.ALGO_TREE):
                 Y = run_plan(hb.hccl_plan_allreduce(R, n, dt, algo, _with(dict(tile_bytes=1024), engine)), X)
                 for r in range(R):
                     assert np.all(synth.from_bits(Y[r].view(np_dtype(dt)), dt) == R * (R + 1) / 2)
@@ -221,7 +223,7 @@ def test_maximum_rank_count(engine):
     R, n, dt = 256, 3001, hb.BF16
     X = synth.small_int_ranks(R, n, dt, seed=256, span=1)          # exactly summable in bf16: unique result
     want = orc.allreduce(dt, X)
-    for algo, extra in ((hb.ALGO_RING, {}), (hb.ALGO_ONESHOT, {}), (hb.ALGO_RING_2LEVEL, dict(rack_size=16)), (hb.ALGO_FANOUT, {})):
+    for algo, extra in ((hb.ALGO_RING, {}), (hb.ALGO_ONESHOT, {}), (hb.ALGO_RING_2LEVEL, dict(rack_size=16)), (hb.ALGO_FANOUT, {}), (hb.ALGO_TREE, {})):
         p = hb.hccl_plan_allreduce(R, n, dt, algo, _with(dict(sm_budget=64, **extra), engine))
         Y = run_plan(p, X)
         for r in (0, 1, 127, 255):

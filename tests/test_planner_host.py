@@ -50,11 +50,15 @@ def test_config3_and_5_byte_accounting():
         # destinations fused: every input read once, every output written once = the compulsory bytes
         i = hb.hccl_plan_allreduce(8, m // 2, hb.BF16, hb.ALGO_FANOUT).info()
         assert i.schedule_bytes == 16 * m == i.compulsory_bytes and i.chain_depth == 1
+        # binary tree: 3 levels of sums + 3 levels of copies; per output position 4 x (2+2+4) + 2 x (4+4+4) +
+        # (4+4+2) reduce bytes and 7 x (2+2) copy bytes = 94 bytes (the ring's figure), at depth 6 instead of 14
+        i = hb.hccl_plan_allreduce(8, m // 2, hb.BF16, hb.ALGO_TREE).info()
+        assert i.chain_depth == 6 and i.n_wqe % 14 == 0 and i.schedule_bytes == 47 * m
 
 
 @pytest.mark.parametrize("dt", DTYPES)
-@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED, hb.ALGO_FANOUT])
-@pytest.mark.parametrize("R,n", [(1, 5), (2, 9), (3, 2), (4, 257), (5, 1000), (8, 4099), (4, 0), (4, 3)])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED, hb.ALGO_FANOUT, hb.ALGO_TREE])
+@pytest.mark.parametrize("R,n", [(1, 5), (2, 9), (3, 2), (4, 257), (5, 1000), (8, 4099), (4, 0), (4, 3), (7, 9001), (13, 700)])
 def test_allreduce_plans_match_oracle(R, n, dt, algo):
     X = synth.normal_ranks(R, n, dt, seed=R * 100 + n)
     p = hb.hccl_plan_allreduce(R, n, dt, algo, SMALL)
@@ -63,6 +67,8 @@ def test_allreduce_plans_match_oracle(R, n, dt, algo):
     want = orc.allreduce(dt, X)
     if algo in (hb.ALGO_ONESHOT, hb.ALGO_FANOUT):  # the fused form sums in the one-shot's order
         bitwise = orc.allreduce_oneshot_f32(dt, X)
+    elif algo == hb.ALGO_TREE:
+        bitwise = orc.allreduce_tree_f32(dt, X)
     else:
         bitwise = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
     for seed in (0, 1, 2):
