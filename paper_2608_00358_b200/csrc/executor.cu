@@ -629,17 +629,19 @@ __device__ __forceinline__ void publish_tile(const ExecParams& p, const Tile& t)
 }
 
 // Last block out: completion value for a device-triggered caller, epoch stamp, clean ticket.
+// `lean`: nobody reads the control block or the results before this launch has ended (no completion value to
+// publish, not the resident executor), so the end of the kernel orders everything and the fences are left out.
 template <class P>
-__device__ void leave(const P& p) {
-    __threadfence();
+__device__ void leave(const P& p, bool lean = false) {
+    if (!lean) __threadfence();
     const uint32_t prev = atomicAdd(&p.ctl->exits, 1);
     if (prev == p.nblocks - 1) {
-        __threadfence();
+        if (!lean) __threadfence();
         if (p.trig_set_slot >= 0 && !aborted(p)) st_release_u64(p.user_signals + p.trig_set_slot, p.trig_set_value + (unsigned long long)g_epoch * p.trig_set_per_epoch);
         p.ctl->t_last_ns = globaltimer_ns();
         p.ctl->ticket = 0;
         p.ctl->exits = 0;
-        __threadfence();
+        if (!lean) __threadfence();
         p.ctl->done_epoch = g_epoch;
     }
 }
@@ -650,12 +652,12 @@ __device__ __forceinline__ void named_sync(uint32_t id, uint32_t nthreads) {
 }
 
 // Loads and checks the records of work item `cur`. No waiting here.
-__device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d) {
+__device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d, const Tile* preloaded = nullptr) {
     if (p.trace) {
         trace_put(p.trace, p.trace_cap, cur, 0, (unsigned long long)cur | ((unsigned long long)blockIdx.x << 32));
         trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
     }
-    t = p.tiles[cur];
+    t = preloaded ? *preloaded : p.tiles[cur];
     if (!tile_ok(p, t)) {
         fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
         return false;
@@ -704,13 +706,32 @@ __device__ bool wait_deps(const ExecParams& p, uint32_t cur, const Tile& t, cons
 // and publishes an item's completion while the workers are already on the next one. Two shared-memory
 // buffers hold the current and the next item; named barriers FULL[b] (item in buffer b may start) and
 // DONE[b] (workers have stored all of it) pair the two sides.
+template <bool RESIDENT>
 __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     __shared__ Tile s_tile[2];
     __shared__ Desc s_desc[2];
     __shared__ int s_go[2];
     const uint32_t tid = threadIdx.x, nth = blockDim.x;
     constexpr uint32_t FULL = 1, DONE = 3;  // barrier ids FULL+b, DONE+b
-    init_epoch(p);
+    // Entry. The execution number, the abort word, the first ticket and (with static tickets) the first item's
+    // tile record do not depend on one another: thread 0 issues all of these loads before it uses any of
+    // them, so a small collective pays one trip to memory here instead of four in a row.
+    uint32_t next = 0, abort0 = 0;
+    Tile pre;
+    bool pre_ok = false;
+    const bool gated = p.trig_wait_slot >= 0;
+    if (tid == 0) {
+        if (!gated) {
+            next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+            if (next < p.n_tiles) {
+                pre = p.tiles[next];
+                pre_ok = true;
+            }
+        }
+        abort0 = *(volatile uint32_t*)&p.ctl->abort;
+        g_epoch = *(volatile uint32_t*)&p.ctl->done_epoch + 1u;
+    }
+    __syncthreads();
     if (tid >= 32) {
         const uint32_t wtid = tid - 32, nwork = nth - 32;
         for (uint32_t k = 0;; ++k) {
@@ -723,12 +744,12 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         return;
     }
     // ---- control warp; every lane executes the barriers, lane 0 does the rest
-    uint32_t next = 0;
     bool live = true, have = false, ready = false;
     if (tid == 0) {
-        if (p.trig_wait_slot >= 0)
+        if (gated) {
             live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value + (unsigned long long)g_epoch * p.trig_wait_per_epoch, 0xffffffffu);
-        next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+            next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+        }
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
     }
     uint32_t cur = 0, prev_item = 0;
@@ -740,10 +761,10 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
             // item k: its records were fetched during item k-1 (or are fetched now for the first one)
             if (k == 0) {
                 cur = next;
-                have = live && cur < p.n_tiles && !aborted(p);
+                have = live && cur < p.n_tiles && !(gated ? aborted(p) : abort0 == g_epoch);
                 if (have) {
                     next = p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
-                    have = fetch_tile(p, cur, s_tile[0], s_desc[0]);
+                    have = fetch_tile(p, cur, s_tile[0], s_desc[0], pre_ok ? &pre : nullptr);
                     ready = have && deps_ready(p, s_tile[0]);
                 }
             }
@@ -790,13 +811,13 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         }
         if (!go) break;
     }
-    if (tid == 0) leave(p);
+    if (tid == 0) leave(p, !RESIDENT && p.trig_set_slot < 0);
 }
 
-__global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p) { executor_lsu_body(p); }
+__global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p) { executor_lsu_body<false>(p); }
 // Same program compiled to at most 64 registers per thread: two 512-thread blocks (or four of 256) fit one
 // SM, and a block of 256 threads leaves three quarters of the register file to whatever else runs there.
-__global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p) { executor_lsu_body(p); }
+__global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p) { executor_lsu_body<false>(p); }
 
 // ====================================================================== bulk (TMA) engine
 // The same dispatch and dependency protocol, but the data mover is the bulk asynchronous copy unit:
@@ -1076,12 +1097,12 @@ __device__ void issue_simple(const ExecParams& p, Dma& d, uint32_t kind, uint32_
 }
 
 // One work item through the DMA thread. Returns false when the block must stop.
-__device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur) {
+__device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const Tile* preloaded = nullptr) {
     if (p.trace) {
         trace_put(p.trace, p.trace_cap, cur, 0, (unsigned long long)cur | ((unsigned long long)blockIdx.x << 32));
         trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
     }
-    const Tile t = p.tiles[cur];
+    const Tile t = preloaded ? *preloaded : p.tiles[cur];
     if (!tile_ok(p, t)) {
         fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
         return false;
@@ -1223,7 +1244,22 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
     const uint32_t tid = threadIdx.x;
     const uint32_t ncw = (blockDim.x >> 5) - 1;  // compute warps
     const uint32_t full = smem_u32(bars), empty = smem_u32(bars + ns);
-    init_epoch(p);
+    // entry: first ticket, its tile record, the abort word and the execution number are loaded together
+    uint32_t next0 = 0, abort0 = 0;
+    Tile pre;
+    bool pre_ok = false;
+    const bool gated = p.trig_wait_slot >= 0;
+    if (tid == 0) {
+        if (!gated) {
+            next0 = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+            if (next0 < p.n_tiles) {
+                pre = p.tiles[next0];
+                pre_ok = true;
+            }
+        }
+        abort0 = *(volatile uint32_t*)&p.ctl->abort;
+        g_epoch = *(volatile uint32_t*)&p.ctl->done_epoch + 1u;
+    }
     if (tid == 0) {
         for (uint32_t s = 0; s < ns; ++s) {
             mbar_init(full + 8 * s, 1);
@@ -1249,15 +1285,19 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         d.pol = policy_evict_first();
         d.ok = true;
         bool live = true;
-        if (p.trig_wait_slot >= 0)
+        uint32_t next = next0;
+        if (gated) {
             live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value + (unsigned long long)g_epoch * p.trig_wait_per_epoch, 0xffffffffu);
-        uint32_t next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+            next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+        }
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
+        bool first = true;
         while (live && d.ok) {
             const uint32_t cur = next;
-            if (cur >= p.n_tiles || aborted(p)) break;
+            if (cur >= p.n_tiles || (first && !gated ? abort0 == g_epoch : aborted(p))) break;
             next = p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
-            if (!dma_item(p, d, cur)) break;
+            if (!dma_item(p, d, cur, first && pre_ok ? &pre : nullptr)) break;
+            first = false;
         }
         // wind down: finish what is in flight, release the compute warps, leave
         if (d.ok && !aborted(p)) drain(p, d);
@@ -1278,7 +1318,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         }
         bulk_wait_all();
         // the compute warps must be out of the stages before the block's verdict is given
-        leave(p);
+        leave(p, p.trig_set_slot < 0);
         return;
     }
 
@@ -1425,7 +1465,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_co
         }
         __syncthreads();
         if (s_cmd == 0) break;
-        executor_lsu_body(p);           // one execution: tickets, dependencies, data, completion stamp
+        executor_lsu_body<true>(p);     // one execution: tickets, dependencies, data, completion stamp
         __syncthreads();
         ++epoch;
     }
