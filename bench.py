@@ -402,6 +402,31 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                    "api": "hccl_hostpipe_execute (pinned host buffers -> device -> pinned host buffers, %d destination windows on 3 streams)" % (len(pipe.windows()) - 1),
                    "gpu_launches_per_step": len(pipe.windows()) - 1,
                    "single_stream": {"value": info.schedule_bytes / serial_ms / 1e6, "ms_per_step": serial_ms, "api": "hccl_execute_host"}}
+            # the host link by itself, with the same pinned buffers: each direction alone, then both at once
+            def _link(h2d, d2h, reps=2):
+                torch.cuda.synchronize()
+                a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a0.record(stream)
+                s_in.wait_event(a0)
+                s_out.wait_event(a0)
+                nb = 0
+                for _ in range(reps):
+                    for k in range(16):
+                        if h2d:
+                            with torch.cuda.stream(s_in):
+                                wl.send[k].copy_(hs[k], non_blocking=True)
+                            nb += hs[k].numel() * 2
+                        if d2h:
+                            with torch.cuda.stream(s_out):
+                                hr[k].copy_(wl.recv[k], non_blocking=True)
+                stream.wait_stream(s_in)
+                stream.wait_stream(s_out)
+                a1.record(stream)
+                torch.cuda.synchronize()
+                one_way = nb if h2d else reps * sum(hr[k].numel() * 2 for k in range(16))
+                return one_way / a0.elapsed_time(a1) / 1e6
+            e2e["host_link_gbs"] = {"h2d_alone": _link(True, False), "d2h_alone": _link(False, True), "h2d_while_d2h_runs": _link(True, True),
+                                    "note": "plain pinned copies of 16 of the 64 rank buffers; the pipelined path needs both directions at once"}
             del pipe, pws
             del hs, hr
         else:
