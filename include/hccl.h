@@ -83,7 +83,10 @@ typedef enum {
                                 every rank. Dependency depth 2*ceil(log2 R). */
 } hccl_algo_t;
 
-/* Which data mover the executor uses for aligned bulk work. */
+/* Which data mover the executor uses for aligned bulk work. AUTO: the planner decides: the bulk engine for
+ * copies that do not wait on one another (AllToAllv, one-shot and fan-out AllGather) and for reductions with
+ * 256 MiB of input or more; the register engine for hop-by-hop copies, smaller reductions and all
+ * multi-input sums. Graphs compiled directly (hccl_graph_compile) default to the register engine. */
 typedef enum {
     HCCL_ENGINE_AUTO = 0,
     HCCL_ENGINE_LSU = 1,  /* 128-bit vector loads/stores through registers */
