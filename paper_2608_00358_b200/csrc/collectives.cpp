@@ -155,9 +155,20 @@ hccl_status_t emit_ring(hccl_graph* g, int R, int dt, const std::vector<Chain>& 
 // chains that run together, and a step should be about one tile per block (a chain advances one step per
 // tile, so few, large tiles keep the dependency chain short). With opts.tile_bytes set, that many bytes
 // of the widest operand.
-int64_t pick_tile_elems(int64_t level_elems, const hccl_opts_t& o, int widest, int op) {
+int64_t pick_tile_elems(int64_t level_elems, const hccl_opts_t& o, int widest, int op, int64_t chain_len = 0) {
     if (o.tile_bytes) return std::max<int64_t>(64, (int64_t)(o.tile_bytes / (uint64_t)widest));
     const int64_t lo = op == HCCL_OP_REDUCE_N ? 1 << 10 : 4 << 10, hi = op == HCCL_OP_REDUCE_N ? 32 << 10 : 64 << 10;
+    if (chain_len > 0 && op == HCCL_OP_REDUCE && o.engine == HCCL_ENGINE_LSU) {
+        // Register engine (the bulk engine prefers tiles that are whole stages). Chains of one length: cut each into the same number of tiles so that a step of all chains is a whole
+        // number of rounds of the blocks (one round if the tiles stay under the cap). Block b then tends to meet
+        // tile b of every step, i.e. its own earlier work, instead of waiting for another block's.
+        const int64_t chains = std::max<int64_t>(1, level_elems / chain_len);
+        for (int64_t rounds = 1; rounds <= 64; ++rounds) {
+            const int64_t per_chain = std::max<int64_t>(1, (int64_t)o.sm_budget * rounds / chains);
+            const int64_t tile = ((chain_len + per_chain - 1) / per_chain + 63) / 64 * 64;
+            if (tile <= hi) return std::max<int64_t>(tile, std::min<int64_t>(lo, (chain_len + 63) / 64 * 64));
+        }
+    }
     return default_tile(level_elems, o.sm_budget, 1, lo, hi, sweep_of(o, op));
 }
 
@@ -642,7 +653,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     const int64_t weight = count * 4 * (R - 1) + (int64_t)count * es * (R - 1);
     const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
     (void)weight;
-    const int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, in_recv ? es : 4, HCCL_OP_REDUCE);
+    const int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, in_recv ? es : 4, HCCL_OP_REDUCE, maxlen);
 
     hccl_graph* graw = nullptr;
     CHECK(hccl_graph_create(R, ext.data(), ext.data(), scratch, 0, &graw));
@@ -703,7 +714,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     const int64_t slot_elems = (int64_t)align_up((uint64_t)maxlen, 64);
     const int64_t scratch = need_scratch ? (int64_t)n_slots * slot_elems * 4 * (staged ? 2 : 1) : 0;
     const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
-    const int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, 4, HCCL_OP_REDUCE);
+    const int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, 4, HCCL_OP_REDUCE, maxlen);
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), scratch, 0, &graw));
     GraphPtr g(graw);
     g->compulsory_bytes = compulsory;
