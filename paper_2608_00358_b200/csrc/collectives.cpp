@@ -654,6 +654,12 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
     (void)weight;
     const int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, in_recv ? es : 4, HCCL_OP_REDUCE, maxlen);
+    if (!fused && o.engine == HCCL_ENGINE_LSU && (!opts || opts->sm_budget == 0) && maxlen > 0) {
+        // a step that is a little short of one round of the blocks: launch exactly that many blocks, so that
+        // block b keeps meeting tile b of every step (measured 54 vs 58 us at R = 8, 1 MiB per rank)
+        const int64_t per_step = std::max<int64_t>(1, level / maxlen) * ((maxlen + tile_elems - 1) / tile_elems);
+        if (per_step < o.sm_budget && per_step * 4 >= (int64_t)o.sm_budget * 3) o.sm_budget = (int32_t)per_step;
+    }
 
     hccl_graph* graw = nullptr;
     CHECK(hccl_graph_create(R, ext.data(), ext.data(), scratch, 0, &graw));
