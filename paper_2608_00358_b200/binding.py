@@ -18,6 +18,7 @@ FP32, BF16, FP16 = 0, 1, 2
 ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED, ALGO_RING_2LEVEL, ALGO_FANOUT, ALGO_TREE = 0, 1, 2, 3, 4, 5
 ENGINE_AUTO, ENGINE_LSU, ENGINE_BULK = 0, 1, 2
 FLAG_LEVEL_MAJOR, FLAG_CHECK_HAZARDS, FLAG_STAGED_RING, FLAG_BIDIRECTIONAL = 1, 2, 4, 8
+FLAG_STATIC_CHAINS, FLAG_DYNAMIC_TICKETS = 16, 32
 OP_COPY, OP_REDUCE, OP_REDUCE_N, OP_WAIT, OP_SET, OP_NOOP = range(6)
 BUF_SEND, BUF_RECV, BUF_SCRATCH, BUF_SIGNAL, BUF_USER_SIGNAL = range(5)
 DEP_FENCE, DEP_SYNC, DEP_WQE_SYNC, DEP_RECV_SYNC, DEP_SEND_SYNC, DEP_ELEMENTWISE, DEP_ELEMENTWISE2 = 1, 2, 4, 8, 16, 32, 64

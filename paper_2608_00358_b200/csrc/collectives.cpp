@@ -643,6 +643,8 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     // small buffers (all FP32 partials fit the L2 several times over): run every chain together, the
     // dependency chain is then as short as the ring allows; large ones keep chain groups for L2 residency
     if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
+    // ... and each chain of tiles can then stay inside one block (no slot is recycled, so nothing links the chains)
+    if (count * 4 <= (32ll << 20) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const bool need_scratch = !in_recv && !fused && R > 2;
     const bool staged = (o.flags & HCCL_FLAG_STAGED_RING) != 0 && need_scratch;
     // level-major order runs every chain's step t before any step t+1, so no slot can be recycled
@@ -712,6 +714,8 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     int64_t maxlen = 0;
     for (const Chain& ch : chains) maxlen = std::max(maxlen, ch.len);
     if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
+    // ... and each chain of tiles can then stay inside one block (no slot is recycled, so nothing links the chains)
+    if (count * 4 <= (32ll << 20) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const bool need_scratch = !fused && R > 2;
     const bool staged = (o.flags & HCCL_FLAG_STAGED_RING) != 0 && need_scratch;
     // level-major order runs every chain's step t before any step t+1, so no slot can be recycled
@@ -792,6 +796,9 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     // meets an unfinished predecessor; measured at R = 128 that costs more than the DRAM reads it saves.
     const bool oneshot = algo == HCCL_ALGO_ONESHOT;
     const int G = oneshot ? 1 : R;
+    // hop-by-hop copies: a block can walk a tile through all its hops by itself (each hop then reads what the
+    // same SM has just written)
+    if (!oneshot && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     for (int q0 = 0; q0 < R; q0 += G) {
         for (int u = 0; u < R; ++u) {
             for (int q = q0; q < std::min(R, q0 + G); ++q) {

@@ -46,6 +46,8 @@ struct ExecParams {
     long long trig_wait_slot, trig_set_slot;
     int trig_cmp;
     int static_tickets;  // no dependencies and no more items than blocks: block b runs item b, no atomics
+    uint32_t chain_len, n_chains;  // static chains (chain_len > 0): items [c*chain_len, (c+1)*chain_len) are chain c; block b
+                                   // runs its share of the chains one after the other, each in order, without counters
     unsigned long long trig_wait_value, trig_wait_per_epoch, trig_set_value, trig_set_per_epoch;
     const void* send[HCCL_MAX_RANKS];
     void* recv[HCCL_MAX_RANKS];
@@ -706,6 +708,27 @@ __device__ bool wait_deps(const ExecParams& p, uint32_t cur, const Tile& t, cons
 // and publishes an item's completion while the workers are already on the next one. Two shared-memory
 // buffers hold the current and the next item; named barriers FULL[b] (item in buffer b may start) and
 // DONE[b] (workers have stored all of it) pair the two sides.
+// Static chains: the items of block b (an even share of the chains, contiguous).
+__device__ __forceinline__ void chain_range(const ExecParams& p, uint32_t& first_item, uint32_t& end_item) {
+    const uint32_t B = p.nblocks, q = p.n_chains / B, rem = p.n_chains % B, b = blockIdx.x;
+    const uint32_t c0 = b * q + min(b, rem), c1 = c0 + q + (b < rem ? 1u : 0u);
+    first_item = c0 * p.chain_len;
+    end_item = c1 * p.chain_len;
+}
+// The first item of a block, and the one after `cur`.
+__device__ __forceinline__ uint32_t first_item(const ExecParams& p, uint32_t& range_end) {
+    if (p.chain_len) {
+        uint32_t f;
+        chain_range(p, f, range_end);
+        return f < range_end ? f : p.n_tiles;
+    }
+    return p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+}
+__device__ __forceinline__ uint32_t next_item(const ExecParams& p, uint32_t cur, uint32_t range_end) {
+    if (p.chain_len) return cur + 1 < range_end ? cur + 1 : p.n_tiles;
+    return p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
+}
+
 template <bool RESIDENT>
 __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     __shared__ Tile s_tile[2];
@@ -716,13 +739,13 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     // Entry. The execution number, the abort word, the first ticket and (with static tickets) the first item's
     // tile record do not depend on one another: thread 0 issues all of these loads before it uses any of
     // them, so a small collective pays one trip to memory here instead of four in a row.
-    uint32_t next = 0, abort0 = 0;
+    uint32_t next = 0, abort0 = 0, range_end = 0;
     Tile pre;
     bool pre_ok = false;
     const bool gated = p.trig_wait_slot >= 0;
     if (tid == 0) {
         if (!gated) {
-            next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+            next = first_item(p, range_end);
             if (next < p.n_tiles) {
                 pre = p.tiles[next];
                 pre_ok = true;
@@ -748,7 +771,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     if (tid == 0) {
         if (gated) {
             live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value + (unsigned long long)g_epoch * p.trig_wait_per_epoch, 0xffffffffu);
-            next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+            next = first_item(p, range_end);
         }
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
     }
@@ -763,7 +786,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 cur = next;
                 have = live && cur < p.n_tiles && !(gated ? aborted(p) : abort0 == g_epoch);
                 if (have) {
-                    next = p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
+                    next = next_item(p, cur, range_end);
                     have = fetch_tile(p, cur, s_tile[0], s_desc[0], pre_ok ? &pre : nullptr);
                     ready = have && deps_ready(p, s_tile[0]);
                 }
@@ -803,7 +826,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 cur = next;
                 have = cur < p.n_tiles && !aborted(p);
                 if (have) {
-                    next = atomicAdd(&p.ctl->ticket, 1);
+                    next = next_item(p, cur, range_end);
                     have = fetch_tile(p, cur, s_tile[b ^ 1], s_desc[b ^ 1]);
                     ready = have && deps_ready(p, s_tile[b ^ 1]);
                 }
@@ -1692,6 +1715,18 @@ hccl_status_t hccl_plan_bind(hccl_plan_t* p, void* dev_workspace, size_t bytes, 
     return HCCL_OK;
 }
 
+// How the blocks find their work: tickets, one item per block, or static chains.
+static int set_dispatch(const hccl_plan_t* p, ExecParams& prm) {
+    int blocks = p->opts.sm_budget;
+    if ((uint32_t)blocks > prm.n_tiles) blocks = (int)std::max<uint32_t>(prm.n_tiles, 1u);
+    prm.chain_len = p->chain_len;
+    prm.n_chains = p->n_chains;
+    if (p->chain_len) blocks = (int)std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)blocks, p->n_chains));
+    prm.nblocks = (uint32_t)blocks;
+    prm.static_tickets = (!p->chain_len && prm.n_waits == 0 && prm.n_tiles <= (uint32_t)blocks) ? 1 : 0;
+    return blocks;
+}
+
 static hccl_status_t check_buffers(hccl_plan_t* p, const void* const* sendbufs, void* const* recvbufs) {
     const int R = p->R;
     bool same = (int)p->checked_send.size() == R;
@@ -1792,10 +1827,7 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
         prm.send[r] = sendbufs[r];
         prm.recv[r] = recvbufs[r];
     }
-    int blocks = p->opts.sm_budget;
-    if ((uint32_t)blocks > prm.n_tiles) blocks = (int)std::max<uint32_t>(prm.n_tiles, 1u);
-    prm.nblocks = (uint32_t)blocks;
-    prm.static_tickets = (prm.n_waits == 0 && prm.n_tiles <= (uint32_t)blocks) ? 1 : 0;
+    const int blocks = set_dispatch(p, prm);
     if (p->opts.engine == HCCL_ENGINE_BULK) {
         const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : (int)bulk::MAX_STAGES, 2), (int)bulk::MAX_STAGES);
         const size_t smem = (size_t)ns * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
@@ -2103,10 +2135,7 @@ hccl_status_t hccl_server_start(hccl_plan_t* p, const void* const* sendbufs, voi
         prm.send[r] = sendbufs[r];
         prm.recv[r] = recvbufs[r];
     }
-    int blocks = p->opts.sm_budget;
-    if ((uint32_t)blocks > prm.n_tiles) blocks = (int)std::max<uint32_t>(prm.n_tiles, 1u);
-    prm.nblocks = (uint32_t)blocks;
-    prm.static_tickets = (prm.n_waits == 0 && prm.n_tiles <= (uint32_t)blocks) ? 1 : 0;
+    const int blocks = set_dispatch(p, prm);
     // every block must be resident at once (the blocks wait for each other between executions)
     int dev = 0, sms = 0, per_sm = 0;
     CUDA_TRY(cudaGetDevice(&dev));
@@ -2241,15 +2270,12 @@ extern "C" hccl_status_t hccl_execute_noalloc(hccl_plan_t* p, const void* const*
     prm.trig_wait_slot = -1;
     prm.trig_set_slot = -1;
     prm.trig_cmp = 0;
-    prm.static_tickets = 0;
     prm.trig_wait_value = prm.trig_set_value = prm.trig_wait_per_epoch = prm.trig_set_per_epoch = 0;
     for (int r = 0; r < R; ++r) {
         prm.send[r] = sendbufs[r];
         prm.recv[r] = recvbufs[r];
     }
-    int blocks = p->opts.sm_budget;
-    if ((uint32_t)blocks > prm.n_tiles) blocks = (int)std::max<uint32_t>(prm.n_tiles, 1u);
-    prm.nblocks = (uint32_t)blocks;
+    const int blocks = set_dispatch(p, prm);
     hccl_executor_lsu<<<blocks, p->opts.threads, 0, st>>>(prm);
     CUDA_TRY(cudaGetLastError());
     // This call owns the shared array until its kernel is done, so it waits here and hands back the

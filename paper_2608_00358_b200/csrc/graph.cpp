@@ -391,6 +391,38 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         for (int64_t i : pf[j]) need_desc[i] = 1;
         for (int64_t i : pe[j]) need_tile[i] = 1;
     }
+    // ---- static chains: the packet is a set of independent chains of equal length, linked tile by tile
+    std::vector<int64_t> chain_pred(n, -1), chain_succ(n, -1);
+    std::vector<int64_t> depth(n, 1);
+    int64_t max_depth = n ? 1 : 0;
+    for (size_t i = 0; i < n; ++i) {
+        for (int64_t q : pf[i]) depth[i] = std::max(depth[i], depth[q] + 1);
+        for (int64_t q : pe[i]) depth[i] = std::max(depth[i], depth[q] + 1);
+        max_depth = std::max(max_depth, depth[i]);
+    }
+    bool chains = (p->opts.flags & HCCL_FLAG_STATIC_CHAINS) != 0 && p->opts.engine == HCCL_ENGINE_LSU && n > 0 && max_depth > 1;
+    for (size_t j = 0; j < n && chains; ++j) {
+        const int op = g->wqes[j].w.op;
+        if (!pf[j].empty() || pe[j].size() > 1 || op == HCCL_OP_WAIT || op == HCCL_OP_SET) chains = false;
+        if (chains && pe[j].size() == 1) {
+            const int64_t i = pe[j][0];
+            if (chain_succ[i] >= 0) chains = false;
+            chain_succ[i] = (int64_t)j;
+            chain_pred[j] = i;
+        }
+    }
+    std::vector<int64_t> heads;
+    for (size_t i = 0; i < n && chains; ++i) {
+        if (chain_pred[i] >= 0) continue;
+        int64_t len = 0;
+        for (int64_t w = (int64_t)i; w >= 0; w = chain_succ[w]) ++len;
+        if (len != max_depth) chains = false;  // equal lengths: a block finds its tiles by arithmetic
+        heads.push_back((int64_t)i);
+    }
+    if (chains) {
+        for (size_t j = 0; j < n; ++j) pe[j].clear();  // the order inside a block replaces every counter
+        std::fill(need_tile.begin(), need_tile.end(), 0);
+    }
     std::vector<int64_t> desc_sync(n, -1), tile_sync0(n, -1);
     for (size_t i = 0; i < n; ++i) {
         if (need_desc[i]) {
@@ -409,8 +441,6 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
 
     // ---- descriptors, tiles, waits
     p->descs.resize(n);
-    std::vector<int64_t> depth(n, 1);
-    int64_t max_depth = n ? 1 : 0;
     for (size_t i = 0; i < n; ++i) {
         const hccl_wqe_t& w = g->wqes[i].w;
         Desc d;
@@ -426,9 +456,7 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         d.count = w.count;
         d.value = w.value; d.value_per_epoch = w.value_per_epoch;
         p->descs[i] = d;
-        for (int64_t q : pf[i]) depth[i] = std::max(depth[i], depth[q] + 1);
-        for (int64_t q : pe[i]) depth[i] = std::max(depth[i], depth[q] + 1);
-        max_depth = std::max(max_depth, depth[i]);
+        if (chains) continue;  // tiles are laid out chain by chain below
 
         if (pf[i].size() + pe[i].size() > 0xffff) {
             delete p;
@@ -454,6 +482,36 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
             delete p;
             return HCCL_ERR_INVALID_ARG;
         }
+    }
+
+    if (chains) {
+        // chain c = tile k of every WQE of one WQE chain, in order; chains are numbered WQE chain by WQE chain
+        uint64_t n_chains = 0;
+        for (int64_t h : heads) n_chains += (uint64_t)ntiles[h];
+        if (n_chains * (uint64_t)max_depth > 0x7ffffff0ull) {
+            delete p;
+            return HCCL_ERR_INVALID_ARG;
+        }
+        p->tiles.reserve((size_t)(n_chains * (uint64_t)max_depth));
+        for (int64_t h : heads) {
+            for (int64_t k = 0; k < ntiles[h]; ++k) {
+                for (int64_t w = h; w >= 0; w = chain_succ[w]) {
+                    const hccl_wqe_t& q = g->wqes[w].w;
+                    Tile t;
+                    std::memset(&t, 0, sizeof(t));
+                    t.desc = (uint32_t)w;
+                    if (tcount[w] > 0) {
+                        t.start = (uint64_t)(k * tcount[w]);
+                        t.count = (uint32_t)std::min<int64_t>(tcount[w], q.count - k * tcount[w]);
+                    }
+                    t.signal[0] = t.signal[1] = -1;
+                    p->tiles.push_back(t);
+                }
+            }
+        }
+        p->chain_len = (uint32_t)max_depth;
+        p->n_chains = (uint32_t)n_chains;
+        p->opts.sm_budget = (int32_t)std::max<uint64_t>(1, std::min<uint64_t>((uint64_t)p->opts.sm_budget, n_chains));
     }
 
     // ---- workspace layout

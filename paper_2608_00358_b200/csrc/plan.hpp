@@ -51,6 +51,8 @@ struct hccl_plan {
     std::vector<hccl::Wait> waits;
     std::vector<uint32_t> sync_per_epoch;  // bumps each sync object receives per execution
     hccl::Layout layout{};
+    // static chains (HCCL_FLAG_STATIC_CHAINS): tiles [c*chain_len, (c+1)*chain_len) form chain c, run in order by one block
+    uint32_t chain_len = 0, n_chains = 0;
     int buf_align = 1;                     // alignment every send/receive pointer must have (largest element read or written)
     hccl_plan_info_t info{};
     // device-triggered execution (Sec. IV-B.3)

@@ -166,6 +166,11 @@ hccl_status_t hccl_plan_check_hazards(const hccl_plan_t* p, int64_t* n_violation
                     }
                 }
             }
+            // static chains: a tile runs after its predecessor in the chain, in the same block
+            if (p->chain_len > 0 && x % p->chain_len != 0 && x - 1 >= floor && mark[x - 1] != v) {
+                mark[x - 1] = v;
+                stack.push_back(x - 1);
+            }
         }
         for (uint32_t u : partners[v])
             if (mark[u] != v) ++bad;
@@ -187,7 +192,12 @@ hccl_status_t hccl_plan_interpret_host(const hccl_plan_t* p, const void* const* 
         if (kind == HCCL_BUF_RECV) return (char*)host_recv[rank];
         return (char*)host_scratch;
     };
+    std::vector<char> done(nt, 0);
     auto ready = [&](const Tile& t) {
+        if (p->chain_len > 0) {  // static chains: strictly in order inside a chain
+            const size_t i = (size_t)(&t - p->tiles.data());
+            if (i % p->chain_len != 0 && !done[i - 1]) return false;
+        }
         for (uint32_t w = 0; w < t.wait_cnt; ++w) {
             const Wait& x = p->waits[t.wait_off + w];
             if (counters[x.sync] < x.per_epoch) return false;
@@ -240,6 +250,7 @@ hccl_status_t hccl_plan_interpret_host(const hccl_plan_t* p, const void* const* 
         }
         for (int k = 0; k < 2; ++k)
             if (t.signal[k] >= 0) ++counters[t.signal[k]];
+        done[(size_t)(&t - p->tiles.data())] = 1;
     };
     if (seed == 0) {
         for (size_t i = 0; i < nt; ++i) {

@@ -300,3 +300,26 @@ def test_engine_geometry_variants(opts):
     orc.alltoallv(Xa, Yw, C, SD, RD, 128)
     for r in range(R):
         assert np.array_equal(Ya[r], Yw[r])
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("flags", [0, hb.FLAG_DYNAMIC_TICKETS], ids=["chains", "tickets"])
+@pytest.mark.parametrize("budget", [1, 3, 148])
+def test_static_chains_and_tickets_same_bits(budget, flags, dt):
+    """Small rings run each chain of tiles inside one block (no device counters); with DYNAMIC_TICKETS the same
+    schedule runs through tickets and counters. Both must give the schedule-ordered oracle's bits."""
+    R, n = 6, 50021
+    opts = dict(tile_bytes=4096, chunk_bytes=32768, sm_budget=budget, flags=flags)
+    for algo in (hb.ALGO_RING, hb.ALGO_RING_FUSED):
+        p = hb.hccl_plan_allreduce(R, n, dt, algo, opts)
+        assert (p.info().n_syncs == 0) == (flags == 0)
+        _check_allreduce(R, n, dt, algo, opts, iters=3)
+    X = synth.normal_ranks(R, n, dt, seed=5)
+    rc = np.diff(orc.floor_chunk_offsets(n, R))
+    Y = run_plan(hb.hccl_plan_reducescatter(R, None, n, dt, hb.ALGO_RING, opts), X, iters=2)
+    for r, w in enumerate(orc.reducescatter_ring_f32(dt, X, rc)):
+        assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
+    Xg = [x[:7001] for x in X]
+    Y = run_plan(hb.hccl_plan_allgather(R, None, 7001, dt, hb.ALGO_RING, opts), Xg, iters=2, misalign=2 if dt != hb.FP32 else 4)
+    for r, w in enumerate(orc.allgatherv(Xg)):
+        assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))

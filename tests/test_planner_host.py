@@ -285,3 +285,72 @@ def test_bidirectional_ring_matches_oracle(R, n, dt):
     Y = interpret(rs, X, 2)
     for r in range(R):
         assert np.array_equal(Y[r].view(np_dtype(dt)).view(np.uint8), want[0][offs[r]:offs[r + 1]].view(np.uint8))
+
+
+# ----------------------------------------------------------------- static chains (a chain of tiles stays in one block)
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_RING_FUSED])
+def test_static_chains_and_tickets_give_the_same_bits(algo, dt):
+    R, n = 5, 20011
+    X = synth.normal_ranks(R, n, dt, seed=77)
+    want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    base = dict(tile_bytes=2048, chunk_bytes=8192, sm_budget=6)
+    for flags, chained in ((0, True), (hb.FLAG_DYNAMIC_TICKETS, False)):
+        p = hb.hccl_plan_allreduce(R, n, dt, algo, dict(base, flags=flags))
+        i = p.info()
+        assert (i.n_syncs == 0) == chained      # no device counter is left when the chains are static
+        assert p.check_hazards() == 0
+        for seed in (0, 3, 4):
+            Y = interpret(p, X, seed)
+            for r in range(R):
+                assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8))
+    # ReduceScatter and the hop-by-hop AllGather take the same route
+    rc = np.diff(orc.floor_chunk_offsets(n, R))
+    p = hb.hccl_plan_reducescatter(R, None, n, dt, hb.ALGO_RING, base)
+    assert p.info().n_syncs == 0 and p.check_hazards() == 0
+    Y = interpret(p, X, 5)
+    for r, w in enumerate(orc.reducescatter_ring_f32(dt, X, rc)):
+        assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
+    p = hb.hccl_plan_allgather(R, None, 777, dt, hb.ALGO_RING, base)
+    assert p.info().n_syncs == 0 and p.check_hazards() == 0
+    Xg = [x[:777] for x in X]
+    for r, w in enumerate(orc.allgatherv(Xg)):
+        assert np.array_equal(interpret(p, Xg, 6)[r].view(np.uint8), w.view(np.uint8))
+
+
+def test_static_chains_need_independent_linear_chains():
+    NB = 4096
+    S, Rv = hb.BUF_SEND, hb.BUF_RECV
+    opts = dict(tile_bytes=1024, sm_budget=4, flags=hb.FLAG_STATIC_CHAINS)
+    E = hb.DEP_WQE_SYNC | hb.DEP_ELEMENTWISE
+    # two chains of two copies each: eligible
+    g = hb.Graph(2, [NB, NB], [2 * NB, 2 * NB])
+    sg = g.add_subgraph(0)
+    a = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, 0), a=(S, 0, 0), count=NB)
+    b = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, 0), a=(S, 1, 0), count=NB)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, NB), a=(Rv, 0, 0), count=NB, dep_flags=E, dep_wqe=a)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, NB), a=(Rv, 1, 0), count=NB, dep_flags=E, dep_wqe=b)
+    p = g.compile(opts)
+    assert p.info().n_syncs == 0 and p.info().n_tiles == 16 and p.check_hazards() == 0
+    rng = np.random.default_rng(0)
+    X = [rng.integers(0, 256, NB, dtype=np.uint8) for _ in range(2)]
+    for seed in range(6):
+        Y = interpret(p, X, seed)
+        assert np.array_equal(Y[0], np.concatenate([X[0], X[1]])) and np.array_equal(Y[1], np.concatenate([X[1], X[0]]))
+    # a WQE with two successors is not a chain: the compiler keeps the counters
+    g = hb.Graph(2, [NB, NB], [2 * NB, 2 * NB])
+    sg = g.add_subgraph(0)
+    a = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, 0), a=(S, 0, 0), count=NB)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, 0), a=(Rv, 0, 0), count=NB, dep_flags=E, dep_wqe=a)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, NB), a=(Rv, 0, 0), count=NB, dep_flags=E, dep_wqe=a)
+    p = g.compile(opts)
+    assert p.info().n_syncs > 0 and p.check_hazards() == 0
+    # chains that touch the same bytes without a link between them: static or not, the checker objects
+    g = hb.Graph(2, [NB, NB], [2 * NB, 2 * NB])
+    sg = g.add_subgraph(0)
+    a = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, 0), a=(S, 0, 0), count=NB)
+    b = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, 0), a=(S, 1, 0), count=NB)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, NB), a=(Rv, 0, 0), count=NB, dep_flags=E, dep_wqe=a)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, NB), a=(Rv, 1, NB), count=NB, dep_flags=E, dep_wqe=b)   # reads the other chain's output
+    p = g.compile(opts)
+    assert p.info().n_syncs == 0 and p.check_hazards() > 0
