@@ -1727,6 +1727,43 @@ static int set_dispatch(const hccl_plan_t* p, ExecParams& prm) {
     return blocks;
 }
 
+// Kernel parameters of a bound plan: table addresses inside its workspace, sizes, trigger, rank buffers, and
+// how the blocks find their work. Returns the number of blocks to launch.
+static int fill_params(const hccl_plan_t* p, ExecParams& prm, const void* const* sendbufs, void* const* recvbufs) {
+    char* ws = (char*)p->workspace;
+    const Layout& L = p->layout;
+    prm.descs = (const Desc*)(ws + L.descs);
+    prm.tiles = (const Tile*)(ws + L.tiles);
+    prm.waits = (const Wait*)(ws + L.waits);
+    prm.counters = (uint32_t*)(ws + L.counters);
+    prm.signals = (unsigned long long*)(ws + L.signals);
+    prm.ctl = (Control*)(ws + L.control);
+    prm.scratch = ws + L.scratch;
+    prm.user_signals = (unsigned long long*)p->user_signals;
+    prm.trace = (unsigned long long*)p->trace;
+    prm.trace_cap = (unsigned long long)p->trace_cap;
+    prm.n_tiles = (uint32_t)p->tiles.size();
+    prm.n_descs = (uint32_t)p->descs.size();
+    prm.n_syncs = (uint32_t)p->sync_per_epoch.size();
+    prm.n_waits = (uint32_t)p->waits.size();
+    prm.n_signals = (uint32_t)p->n_signals;
+    prm.R = (uint32_t)p->R;
+    prm.timeout_ns = p->opts.timeout_ns;
+    prm.n_user_signals = p->n_user_signals;
+    prm.trig_wait_slot = p->trig_wait_slot;
+    prm.trig_set_slot = p->trig_set_slot;
+    prm.trig_cmp = p->trig_cmp;
+    prm.trig_wait_value = p->trig_wait_value;
+    prm.trig_wait_per_epoch = p->trig_wait_per_epoch;
+    prm.trig_set_value = p->trig_set_value;
+    prm.trig_set_per_epoch = p->trig_set_per_epoch;
+    for (int r = 0; r < p->R; ++r) {
+        prm.send[r] = sendbufs[r];
+        prm.recv[r] = recvbufs[r];
+    }
+    return set_dispatch(p, prm);
+}
+
 static hccl_status_t check_buffers(hccl_plan_t* p, const void* const* sendbufs, void* const* recvbufs) {
     const int R = p->R;
     bool same = (int)p->checked_send.size() == R;
@@ -1795,39 +1832,8 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
         return HCCL_OK;
     }
     static thread_local ExecParams prm;  // 4 KB+: keep it off the stack
-    char* ws = (char*)p->workspace;
-    const Layout& L = p->layout;
-    prm.descs = (const Desc*)(ws + L.descs);
-    prm.tiles = (const Tile*)(ws + L.tiles);
-    prm.waits = (const Wait*)(ws + L.waits);
-    prm.counters = (uint32_t*)(ws + L.counters);
-    prm.signals = (unsigned long long*)(ws + L.signals);
-    prm.ctl = (Control*)(ws + L.control);
-    prm.scratch = ws + L.scratch;
-    prm.user_signals = (unsigned long long*)p->user_signals;
-    prm.trace = (unsigned long long*)p->trace;
-    prm.trace_cap = (unsigned long long)p->trace_cap;
-    prm.n_tiles = (uint32_t)p->tiles.size();
-    prm.n_descs = (uint32_t)p->descs.size();
-    prm.n_syncs = (uint32_t)p->sync_per_epoch.size();
-    prm.n_waits = (uint32_t)p->waits.size();
-    prm.n_signals = (uint32_t)p->n_signals;
-    prm.R = (uint32_t)p->R;
     const uint32_t epoch = p->epoch + 1;
-    prm.timeout_ns = p->opts.timeout_ns;
-    prm.n_user_signals = p->n_user_signals;
-    prm.trig_wait_slot = p->trig_wait_slot;
-    prm.trig_set_slot = p->trig_set_slot;
-    prm.trig_cmp = p->trig_cmp;
-    prm.trig_wait_value = p->trig_wait_value;
-    prm.trig_wait_per_epoch = p->trig_wait_per_epoch;
-    prm.trig_set_value = p->trig_set_value;
-    prm.trig_set_per_epoch = p->trig_set_per_epoch;
-    for (int r = 0; r < p->R; ++r) {
-        prm.send[r] = sendbufs[r];
-        prm.recv[r] = recvbufs[r];
-    }
-    const int blocks = set_dispatch(p, prm);
+    const int blocks = fill_params(p, prm, sendbufs, recvbufs);
     if (p->opts.engine == HCCL_ENGINE_BULK) {
         const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : (int)bulk::MAX_STAGES, 2), (int)bulk::MAX_STAGES);
         const size_t smem = (size_t)ns * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
@@ -2104,38 +2110,7 @@ hccl_status_t hccl_server_start(hccl_plan_t* p, const void* const* sendbufs, voi
     CUDA_TRY(cudaMemsetAsync((char*)p->workspace + p->layout.control + offsetof(Control, server_go), 0, 4, s));
     std::memset(host_doorbell, 0, sizeof(Doorbell));
     static thread_local ExecParams prm;
-    char* ws = (char*)p->workspace;
-    const Layout& L = p->layout;
-    prm.descs = (const Desc*)(ws + L.descs);
-    prm.tiles = (const Tile*)(ws + L.tiles);
-    prm.waits = (const Wait*)(ws + L.waits);
-    prm.counters = (uint32_t*)(ws + L.counters);
-    prm.signals = (unsigned long long*)(ws + L.signals);
-    prm.ctl = (Control*)(ws + L.control);
-    prm.scratch = ws + L.scratch;
-    prm.user_signals = (unsigned long long*)p->user_signals;
-    prm.trace = (unsigned long long*)p->trace;
-    prm.trace_cap = (unsigned long long)p->trace_cap;
-    prm.n_tiles = (uint32_t)p->tiles.size();
-    prm.n_descs = (uint32_t)p->descs.size();
-    prm.n_syncs = (uint32_t)p->sync_per_epoch.size();
-    prm.n_waits = (uint32_t)p->waits.size();
-    prm.n_signals = (uint32_t)p->n_signals;
-    prm.R = (uint32_t)p->R;
-    prm.timeout_ns = p->opts.timeout_ns;
-    prm.n_user_signals = p->n_user_signals;
-    prm.trig_wait_slot = p->trig_wait_slot;
-    prm.trig_set_slot = p->trig_set_slot;
-    prm.trig_cmp = p->trig_cmp;
-    prm.trig_wait_value = p->trig_wait_value;
-    prm.trig_wait_per_epoch = p->trig_wait_per_epoch;
-    prm.trig_set_value = p->trig_set_value;
-    prm.trig_set_per_epoch = p->trig_set_per_epoch;
-    for (int r = 0; r < p->R; ++r) {
-        prm.send[r] = sendbufs[r];
-        prm.recv[r] = recvbufs[r];
-    }
-    const int blocks = set_dispatch(p, prm);
+    const int blocks = fill_params(p, prm, sendbufs, recvbufs);
     // every block must be resident at once (the blocks wait for each other between executions)
     int dev = 0, sms = 0, per_sm = 0;
     CUDA_TRY(cudaGetDevice(&dev));
