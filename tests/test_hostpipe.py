@@ -50,6 +50,14 @@ def test_create_rejects_bad_arguments():
         hb.hccl_hostpipe_alltoallv_create(3, C, hb.FP16, 4, 2)
     z = hb.hccl_hostpipe_alltoallv_create(3, np.zeros((3, 3), dtype=np.int64), hb.FP16, 4, 3)
     assert z.windows() == [0, 3]
+    # nothing runs, and no verdict exists, before the pipeline has a workspace
+    with pytest.raises(hb.HcclError) as e:
+        z.status()
+    assert e.value.status == hb.ERR_NOT_BOUND
+    with pytest.raises(hb.HcclError) as e:
+        z.execute([0] * 3, [0] * 3, [0] * 3, [0] * 3, 0, 0, 0)
+    assert e.value.status == hb.ERR_NOT_BOUND
+    assert z.workspace_bytes() % 256 == 0 and z.workspace_bytes() > 0
 
 
 @pytest.mark.gpu
