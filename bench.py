@@ -472,6 +472,18 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             line["interference"] = {"gemm": "bf16 8192^3 (cuBLAS via torch.matmul), back to back", "collective": wl.name,
                                     "protocol": "both loops kept 3 batches deep; rates taken inside the window where both run", "sweep": sweep}
             del gemm
+            if not args.quick:
+                # the same at budget 4 against a 16384^3 GEMM (55 waves of tiles instead of 14: losing one SM
+                # slot costs a smaller share of a wave)
+                torch.cuda.empty_cache()
+                gemm = interference.Gemm(16384)
+                plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(sm_budget=4))
+                w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
+                r = interference.measure(w2, seconds=2.5, gemm=gemm)
+                line["interference"]["gemm_16384_budget_4"] = {
+                    "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
+                    "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
+                del w2, plan, gemm
         dyn64 = None
         if not args.no_side:
             # device-resident AllToAllv at the benchmark's size: the same counts, read from device memory by the kernel

@@ -115,10 +115,11 @@ def main():
     ap.add_argument("--cap", type=int, default=32768)
     ap.add_argument("--seconds", type=float, default=3.0)
     ap.add_argument("--engine", type=int, default=0)
+    ap.add_argument("--gemm-n", type=int, default=8192, help="the GEMM is n x n x n, bf16")
     ap.add_argument("--opts", default="", help="extra plan options, e.g. threads=256,light=1,cluster=2")
     args = ap.parse_args()
     extra = {k: int(v) for k, v in (kv.split("=") for kv in args.opts.split(",") if kv)}
-    gemm = Gemm()
+    gemm = Gemm(args.gemm_n)
     base = wk.config4(dict(sm_budget=148, engine=args.engine), cap=args.cap)
     for b in [int(x) for x in args.budgets.split(",")]:
         plan = wk.hb.hccl_plan_alltoallv(base.meta["R"], base.meta["counts"], None, None, None, wk.hb.FP16,
@@ -126,6 +127,7 @@ def main():
         wl = wk._bind(base.name, plan, base.send, base.recv, base.meta)
         res = measure(wl, args.seconds, gemm)
         res["opts"] = extra
+        res["gemm_n"] = args.gemm_n
         print(json.dumps(res), flush=True)
 
 
