@@ -155,8 +155,10 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
 /* ReduceScatter(sum): rank r ends with Y_r[j] = round(sum_q X_q[o_r + j]), j < recvcounts[r],
  * o_r = sum of recvcounts below r. count = elements in every send buffer; recvcounts == NULL means
  * the floor split of count over R ranks; otherwise sum(recvcounts) must equal count
- * (HCCL_ERR_COUNT_MISMATCH). Ring only: each shard is cut into granules of opts->chunk_bytes and each
- * granule is an independent chain of R-1 reductions with FP32 partials in scratch. */
+ * (HCCL_ERR_COUNT_MISMATCH). RING: each shard is cut into granules of opts->chunk_bytes and each
+ * granule is an independent chain of R-1 reductions with FP32 partials in scratch. RING_FUSED: the same sums
+ * in the same order as one multi-input sum per granule. ONESHOT: every rank sums its shard over all ranks
+ * itself, in rank order 0..R-1. */
 hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t count, hccl_dtype_t dt,
                                       hccl_algo_t algo, const hccl_opts_t* opts, hccl_plan_t** out);
 

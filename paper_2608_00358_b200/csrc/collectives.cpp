@@ -675,9 +675,9 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
                                       const hccl_opts_t* opts, hccl_plan_t** out) {
     if (!out || R < 1 || R > HCCL_MAX_RANKS || count < 0) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
-    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_RING_FUSED) return HCCL_ERR_INVALID_ARG;
+    if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_ONESHOT) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
-    fill_ring_opts(&o, opts, (int64_t)R * count * elem_bytes(dt), algo == HCCL_ALGO_RING_FUSED || R == 1);
+    fill_ring_opts(&o, opts, (int64_t)R * count * elem_bytes(dt), algo != HCCL_ALGO_RING || R == 1);
     const int es = elem_bytes(dt);
     std::vector<int64_t> offs(R + 1, 0);
     if (recvcounts) {
@@ -706,6 +706,27 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
         w.a = ref(HCCL_BUF_SEND, 0, 0);
         w.dst = ref(HCCL_BUF_RECV, 0, 0);
         CHECK(hccl_graph_add_wqe(g.get(), sg, &w, nullptr));
+        return hccl_graph_compile(g.get(), &o, out);
+    }
+    if (algo == HCCL_ALGO_ONESHOT) {
+        // rank r sums its own shard over all ranks itself, in rank order 0..R-1 (the one-shot AllReduce's order)
+        CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw));
+        GraphPtr g(graw);
+        g->compulsory_bytes = compulsory;
+        for (int r = 0; r < R; ++r) {
+            int32_t sg;
+            CHECK(hccl_graph_add_subgraph(g.get(), r, &sg));
+            if (offs[r + 1] == offs[r]) continue;
+            hccl_wqe_t w = blank();
+            w.op = HCCL_OP_REDUCE_N;
+            w.hints = HCCL_HINT_READ_ONCE;
+            w.dtype_dst = w.dtype_a = dt;
+            w.count = offs[r + 1] - offs[r];
+            w.nsrc = R;
+            w.a = ref(HCCL_BUF_SEND, 0, offs[r] * es);
+            w.dst = ref(HCCL_BUF_RECV, r, 0);
+            CHECK(hccl_graph_add_wqe(g.get(), sg, &w, nullptr));
+        }
         return hccl_graph_compile(g.get(), &o, out);
     }
     const bool fused = algo == HCCL_ALGO_RING_FUSED;

@@ -101,6 +101,18 @@ def test_reducescatter_small(R, counts, dt, algo, engine):
         assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8))
 
 
+@pytest.mark.parametrize("dt", DTYPES)
+def test_reducescatter_oneshot(dt, engine):
+    R, counts = 5, [0, 7001, 1000, 1, 30000]
+    n = sum(counts)
+    offs = np.concatenate([[0], np.cumsum(counts)])
+    X = synth.normal_ranks(R, n, dt, seed=11, std=0.02)
+    Y = run_plan(hb.hccl_plan_reducescatter(R, counts, n, dt, hb.ALGO_ONESHOT, _with(dict(tile_bytes=4096, sm_budget=16), engine)), X, iters=2)
+    whole = orc.allreduce_oneshot_f32(dt, X)[0]
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np_dtype(dt)), whole[offs[r]:offs[r + 1]])
+
+
 def test_config3_shape_reducescatter_r16_bf16_reduced_size(engine):
     # config 3 at 1/16 of its size (4 Mi elements per rank, 2 MiB granules -> still several granules per shard? no:
     # shards of 256 Ki elements = 512 KiB, so use 128 KiB granules to keep 4 granules per shard)

@@ -116,6 +116,23 @@ def test_reducescatter_plans_match_oracle(R, counts, dt, algo):
             assert np.array_equal(got.view(np.uint8), bitwise[r].view(np.uint8))
 
 
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("R,counts", [(2, [3, 4]), (4, None), (5, [0, 7, 1000, 1, 300]), (3, [0, 0, 11])])
+def test_reducescatter_oneshot_is_the_oneshot_allreduce_cut_into_shards(R, counts, dt):
+    n = 4099 if counts is None else sum(counts)
+    offs = orc.floor_chunk_offsets(n, R) if counts is None else np.concatenate([[0], np.cumsum(counts)])
+    X = synth.normal_ranks(R, n, dt, seed=R + n, std=0.02)
+    p = hb.hccl_plan_reducescatter(R, counts, n, dt, hb.ALGO_ONESHOT, SMALL)
+    assert p.check_hazards() == 0 and p.info().chain_depth <= 1
+    whole = orc.allreduce_oneshot_f32(dt, X)[0]
+    exact, want = orc.sum_f64(dt, X), orc.reducescatter(dt, X, np.diff(offs))
+    Y = interpret(p, X, 3)
+    for r in range(R):
+        got = Y[r].view(np_dtype(dt))
+        assert np.array_equal(got, whole[offs[r]:offs[r + 1]])
+        assert_reduction_close(dt, got, exact[offs[r]:offs[r + 1]], want[r])
+
+
 def test_reducescatter_rejects_bad_counts():
     with pytest.raises(hb.HcclError) as e:
         hb.hccl_plan_reducescatter(4, [1, 2, 3, 4], 11, hb.BF16)
