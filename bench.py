@@ -272,6 +272,14 @@ def side_configs(quick: bool):
             "ms": float(ms), "schedule_bytes": int(i.schedule_bytes), "compulsory_bytes": int(i.compulsory_bytes),
             "schedule_gbs": i.schedule_bytes / ms / 1e6, "compulsory_gbs": i.compulsory_bytes / ms / 1e6,
             "tiles": int(i.n_tiles), "inputs": "2 GiB, larger than L2"}
+        if algo == hb.ALGO_RING and not quick:
+            # the oracle's ReduceScatter on the same 16 x 64 Mi bf16 inputs, single thread, host memory
+            Xh = [t.view(torch.int16).cpu().numpy().view(np.uint16) for t in wl.send]
+            rc = np.full(16, Xh[0].size // 16, dtype=np.int64)
+            t0 = _t.perf_counter()
+            orc.reducescatter(hb.BF16, Xh, rc)
+            out["3_reducescatter_r16_bf16_64Mi_" + nm]["cpu_oracle_ms"] = (_t.perf_counter() - t0) * 1e3
+            del Xh
         del wl
         torch.cuda.empty_cache()
     return out
