@@ -291,7 +291,10 @@ def run_profile_case(args):
     import torch
     from paper_2608_00358_b200 import binding as hb
     from paper_2608_00358_b200 import workloads as wk
-    if args.profile_case in ("agfanout", "agoneshot"):
+    if args.profile_case in ("c1chains", "c1tickets"):
+        # config 1 (AllReduce ring R = 4, 1 Mi fp32 per rank): static chains vs tickets and device counters
+        wl = wk.config1(dict(flags=0 if args.profile_case == "c1chains" else hb.FLAG_DYNAMIC_TICKETS))
+    elif args.profile_case in ("agfanout", "agoneshot"):
         # AllGather R = 32, 1 Mi bf16 (2 MiB) per rank: 64 MiB read, 2 GiB written
         R, n = 32, 1 << 20
         algo = hb.ALGO_FANOUT if args.profile_case == "agfanout" else hb.ALGO_ONESHOT
@@ -542,7 +545,7 @@ def main():
     ap.add_argument("--no-side", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--profile-n", type=int, default=1 << 23, help="elements per rank of the --profile-case")
-    ap.add_argument("--profile-case", default="", choices=["", "c3ring", "c3fused", "agfanout", "agoneshot"],
+    ap.add_argument("--profile-case", default="", choices=["", "c3ring", "c3fused", "agfanout", "agoneshot", "c1chains", "c1tickets"],
                     help="run only a small single-kernel case (for ncu captures), not the benchmark")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
