@@ -26,6 +26,14 @@
 
 #include "plan.hpp"
 
+// The file can be compiled whole (HCCL_PART undefined or 0) or in four slices that are linked together, so
+// that the build compiles its kernels in parallel: 1 = hccl_executor_lsu, 2 = hccl_executor_lsu_light,
+// 3 = hccl_executor_bulk, 4 = the resident and device-resident kernels and all host code.
+#ifndef HCCL_PART
+#define HCCL_PART 0
+#endif
+#define HCCL_IN_PART(n) (HCCL_PART == 0 || HCCL_PART == (n))
+
 namespace hccl {
 
 struct ExecParams {
@@ -56,7 +64,7 @@ struct ExecParams {
 // The execution number ("epoch") of the running launch. It lives on the device: every block derives it from
 // the control block (done_epoch of the previous execution + 1), so a launch captured in a CUDA graph finds
 // the right epoch on every replay. Kept in shared memory, written once per block at kernel entry.
-__shared__ uint32_t g_epoch;
+static __shared__ uint32_t g_epoch;
 template <class P>
 __device__ __forceinline__ void init_epoch(const P& p) {
     if (threadIdx.x == 0) g_epoch = *(volatile uint32_t*)&p.ctl->done_epoch + 1u;
@@ -121,7 +129,7 @@ template <class P>
 __device__ __forceinline__ bool aborted(const P& p) { return ld_relaxed_u32(&p.ctl->abort) == g_epoch; }
 
 // Bounded wait until counters[sync] has received epoch * per_epoch bumps (wrap-safe compare).
-__device__ bool wait_counter(const ExecParams& p, uint32_t sync, uint32_t per_epoch, uint32_t tile) {
+static __device__ bool wait_counter(const ExecParams& p, uint32_t sync, uint32_t per_epoch, uint32_t tile) {
     const uint32_t* c = p.counters + sync;
     const uint32_t target = g_epoch * per_epoch;
     if ((int32_t)(ld_acquire_u32(c) - target) >= 0) return true;
@@ -516,7 +524,7 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
     }
 }
 
-__device__ void reduce_n_dispatch(const ExecParams& p, const Desc& d, uint64_t start, uint32_t n, uint32_t tid, uint32_t nth) {
+static __device__ void reduce_n_dispatch(const ExecParams& p, const Desc& d, uint64_t start, uint32_t n, uint32_t tid, uint32_t nth) {
 #define RN(S, D) reduce_n_tile<S, D>(p, d, start, n, tid, nth)
     if (d.dt_a == HCCL_FP32) {
         if (d.dt_dst == HCCL_FP32) RN(HCCL_FP32, HCCL_FP32); else if (d.dt_dst == HCCL_BF16) RN(HCCL_FP32, HCCL_BF16); else RN(HCCL_FP32, HCCL_FP16);
@@ -529,7 +537,7 @@ __device__ void reduce_n_dispatch(const ExecParams& p, const Desc& d, uint64_t s
 }
 
 // ------------------------------------------------------------------ one work item, all threads
-__device__ void run_tile_lsu(const ExecParams& p, const Desc& d, const Tile& t, const uint32_t tid, const uint32_t nth) {
+static __device__ void run_tile_lsu(const ExecParams& p, const Desc& d, const Tile& t, const uint32_t tid, const uint32_t nth) {
     switch (d.op) {
         case HCCL_OP_COPY: {
             const char* src = buf_base(p, d.kind_a, d.rank_a) + d.off_a + t.start;
@@ -560,14 +568,14 @@ __device__ void run_tile_lsu(const ExecParams& p, const Desc& d, const Tile& t, 
 }
 
 // Checks on a table entry before it is used; a failing entry is reported, never dereferenced.
-__device__ bool tile_ok(const ExecParams& p, const Tile& t) {
+static __device__ bool tile_ok(const ExecParams& p, const Tile& t) {
     if (t.desc >= p.n_descs) return false;
     if ((uint64_t)t.wait_off + t.wait_cnt > p.n_waits) return false;
     for (int k = 0; k < 2; ++k)
         if (t.signal[k] >= (int32_t)p.n_syncs) return false;
     return true;
 }
-__device__ bool desc_ok(const ExecParams& p, const Desc& d) {
+static __device__ bool desc_ok(const ExecParams& p, const Desc& d) {
     if (d.op > HCCL_OP_NOOP) return false;
     if (d.op == HCCL_OP_COPY || d.op == HCCL_OP_REDUCE || d.op == HCCL_OP_REDUCE_N) {
         if (d.kind_dst != HCCL_BUF_RECV && d.kind_dst != HCCL_BUF_SCRATCH) return false;
@@ -587,37 +595,6 @@ __device__ bool desc_ok(const ExecParams& p, const Desc& d) {
         if (d.kind_dst == HCCL_BUF_SIGNAL) return (uint64_t)d.off_dst < p.n_signals;
         if (d.kind_dst == HCCL_BUF_USER_SIGNAL) return d.off_dst >= 0 && d.off_dst < p.n_user_signals;
         return false;
-    }
-    return true;
-}
-
-// Thread 0: everything that precedes the data movement of work item `cur`. Returns false to stop.
-__device__ bool prepare_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d) {
-    t = p.tiles[cur];
-    if (!tile_ok(p, t)) {
-        fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
-        return false;
-    }
-    d = p.descs[t.desc];
-    if (!desc_ok(p, d)) {
-        fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
-        return false;
-    }
-    for (uint32_t w = 0; w < t.wait_cnt; ++w) {
-        const Wait x = p.waits[t.wait_off + w];
-        if (x.sync >= p.n_syncs) {
-            fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
-            return false;
-        }
-        if (!wait_counter(p, x.sync, x.per_epoch, cur)) return false;
-    }
-    if (d.op == HCCL_OP_WAIT) {
-        const unsigned long long* addr = (d.kind_a == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + d.off_a;
-        if (!wait_signal(p, addr, d.cmp, d.value + (unsigned long long)g_epoch * d.value_per_epoch, cur)) return false;
-    } else if (d.op == HCCL_OP_SET) {
-        unsigned long long* addr = (d.kind_dst == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + d.off_dst;
-        __threadfence();
-        st_release_u64(addr, d.value + (unsigned long long)g_epoch * d.value_per_epoch);
     }
     return true;
 }
@@ -654,7 +631,7 @@ __device__ __forceinline__ void named_sync(uint32_t id, uint32_t nthreads) {
 }
 
 // Loads and checks the records of work item `cur`. No waiting here.
-__device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d, const Tile* preloaded = nullptr) {
+static __device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d, const Tile* preloaded = nullptr) {
     if (p.trace) {
         trace_put(p.trace, p.trace_cap, cur, 0, (unsigned long long)cur | ((unsigned long long)blockIdx.x << 32));
         trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
@@ -672,7 +649,7 @@ __device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, Desc& d, 
     return true;
 }
 // One non-blocking look at every dependency counter of the item.
-__device__ bool deps_ready(const ExecParams& p, const Tile& t) {
+static __device__ bool deps_ready(const ExecParams& p, const Tile& t) {
     for (uint32_t w = 0; w < t.wait_cnt; ++w) {
         const Wait x = p.waits[t.wait_off + w];
         if (x.sync >= p.n_syncs) return false;
@@ -681,7 +658,7 @@ __device__ bool deps_ready(const ExecParams& p, const Tile& t) {
     return true;
 }
 // Blocking (bounded) part: dependency counters, then a WAIT's condition; a SET is performed here.
-__device__ bool wait_deps(const ExecParams& p, uint32_t cur, const Tile& t, const Desc& d, bool counters_done) {
+static __device__ bool wait_deps(const ExecParams& p, uint32_t cur, const Tile& t, const Desc& d, bool counters_done) {
     if (!counters_done) {
         for (uint32_t w = 0; w < t.wait_cnt; ++w) {
             const Wait x = p.waits[t.wait_off + w];
@@ -837,10 +814,18 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     if (tid == 0) leave(p, !RESIDENT && p.trig_set_slot < 0);
 }
 
+#if HCCL_IN_PART(1)
 __global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p) { executor_lsu_body<false>(p); }
+#else
+__global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p);
+#endif
 // Same program compiled to at most 64 registers per thread: two 512-thread blocks (or four of 256) fit one
 // SM, and a block of 256 threads leaves three quarters of the register file to whatever else runs there.
+#if HCCL_IN_PART(2)
 __global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p) { executor_lsu_body<false>(p); }
+#else
+__global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p);
+#endif
 
 // ====================================================================== bulk (TMA) engine
 // The same dispatch and dependency protocol, but the data mover is the bulk asynchronous copy unit:
@@ -898,7 +883,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait on an mbarrier phase; gives up when the execution is aborted or the time budget runs out.
-__device__ bool mbar_wait(const ExecParams& p, uint32_t bar, uint32_t parity, unsigned long long budget_ns, uint32_t detail) {
+static __device__ bool mbar_wait(const ExecParams& p, uint32_t bar, uint32_t parity, unsigned long long budget_ns, uint32_t detail) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long deadline = globaltimer_ns() + budget_ns;
     uint32_t spins = 0;
@@ -1016,7 +1001,7 @@ __device__ __forceinline__ void reduce_piece(const char* sa, const char* sb, cha
         stg4<DD>(gdst + (size_t)u * 4 * Elem<DD>::BYTES, a);
     }
 }
-__device__ void reduce_piece_dispatch(int da, int db, int dd, const char* sa, const char* sb, char* g, uint32_t n, uint32_t ctid, uint32_t cnth) {
+static __device__ void reduce_piece_dispatch(int da, int db, int dd, const char* sa, const char* sb, char* g, uint32_t n, uint32_t ctid, uint32_t cnth) {
 #define RP(A, B, D) reduce_piece<A, B, D>(sa, sb, g, n, ctid, cnth)
 #define RP_D(A, B) do { if (dd == HCCL_FP32) RP(A, B, HCCL_FP32); else if (dd == HCCL_BF16) RP(A, B, HCCL_BF16); else RP(A, B, HCCL_FP16); } while (0)
 #define RP_B(A) do { if (db == HCCL_FP32) RP_D(A, HCCL_FP32); else if (db == HCCL_BF16) RP_D(A, HCCL_BF16); else RP_D(A, HCCL_FP16); } while (0)
@@ -1040,7 +1025,7 @@ struct Dma {
 
 // Retire the oldest outstanding piece. A COPY piece is drained to global memory here; REDUCE and TILE
 // pieces are finished by the compute warps on their own.
-__device__ void retire_one(const ExecParams& p, Dma& d) {
+static __device__ void retire_one(const ExecParams& p, Dma& d) {
     const unsigned long long j = d.tail;
     const uint32_t slot = (uint32_t)(j % d.ns), parity = (uint32_t)((j / d.ns) & 1);
     PieceInfo& pi = d.info[slot];
@@ -1070,12 +1055,12 @@ __device__ void retire_one(const ExecParams& p, Dma& d) {
     }
     d.tail = j + 1;
 }
-__device__ void drain(const ExecParams& p, Dma& d) {
+static __device__ void drain(const ExecParams& p, Dma& d) {
     while (d.tail < d.head) retire_one(p, d);
 }
 // Make stage (k mod ns) reusable for piece k: its previous piece (k - ns) must be retired, passed by every
 // compute warp, and, if it was a COPY, fully read out of shared memory by its store.
-__device__ bool acquire_slot(const ExecParams& p, Dma& d, unsigned long long k, uint32_t detail) {
+static __device__ bool acquire_slot(const ExecParams& p, Dma& d, unsigned long long k, uint32_t detail) {
     if (k < d.ns) return d.ok;
     const unsigned long long j = k - d.ns;
     while (d.tail <= j) retire_one(p, d);
@@ -1094,7 +1079,7 @@ __device__ __forceinline__ void keep_lag(const ExecParams& p, Dma& d) {
     while (d.ok && d.head - d.tail > d.lag) retire_one(p, d);
 }
 
-__device__ bool wait_counter_draining(const ExecParams& p, Dma& d, uint32_t sync, uint32_t per_epoch, uint32_t tile) {
+static __device__ bool wait_counter_draining(const ExecParams& p, Dma& d, uint32_t sync, uint32_t per_epoch, uint32_t tile) {
     const uint32_t target = g_epoch * per_epoch;
     if ((int32_t)(ld_acquire_u32(p.counters + sync) - target) >= 0) return true;
     drain(p, d);  // the item waited for may sit in this block's own pipeline
@@ -1102,7 +1087,7 @@ __device__ bool wait_counter_draining(const ExecParams& p, Dma& d, uint32_t sync
     return wait_counter(p, sync, per_epoch, tile);
 }
 
-__device__ void issue_simple(const ExecParams& p, Dma& d, uint32_t kind, uint32_t cur, const Tile* t, const Desc* ds) {
+static __device__ void issue_simple(const ExecParams& p, Dma& d, uint32_t kind, uint32_t cur, const Tile* t, const Desc* ds) {
     const unsigned long long k = d.head;
     if (!acquire_slot(p, d, k, cur)) return;
     const uint32_t slot = (uint32_t)(k % d.ns);
@@ -1120,7 +1105,7 @@ __device__ void issue_simple(const ExecParams& p, Dma& d, uint32_t kind, uint32_
 }
 
 // One work item through the DMA thread. Returns false when the block must stop.
-__device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const Tile* preloaded = nullptr) {
+static __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const Tile* preloaded = nullptr) {
     if (p.trace) {
         trace_put(p.trace, p.trace_cap, cur, 0, (unsigned long long)cur | ((unsigned long long)blockIdx.x << 32));
         trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
@@ -1258,6 +1243,9 @@ __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const Tile* 
 
 }  // namespace bulk
 
+#if !HCCL_IN_PART(3)
+__global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t copy_by_warps);
+#else
 __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t copy_by_warps) {
     using namespace bulk;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -1410,8 +1398,9 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         if ((tid & 31u) == 0) mbar_arrive(empty + 8 * slot);
     }
 }
+#endif  // part 3
 
-
+#if HCCL_IN_PART(4)
 // ====================================================================== resident, doorbell-fed executor
 // The register engine as a long-lived kernel (paper Sec. II-A.3 "express doorbells": the work request's
 // write is the doorbell; Sec. V-B: re-enqueueing a cached work packet costs microseconds). The blocks stay
@@ -1664,8 +1653,10 @@ __global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant
     if (tid == 0) leave(q);
 }
 
+#endif  // part 4: kernels
 }  // namespace hccl
 
+#if HCCL_IN_PART(4)
 // ====================================================================== host side
 using namespace hccl;
 
@@ -2262,3 +2253,4 @@ extern "C" hccl_status_t hccl_execute_noalloc(hccl_plan_t* p, const void* const*
     if (c.done_epoch != 1) return HCCL_ERR_BUSY;
     return HCCL_OK;
 }
+#endif  // part 4
