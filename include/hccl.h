@@ -424,6 +424,8 @@ typedef struct {
     int64_t epoch;            /* executions enqueued since the last bind */
     int64_t crossrack_bytes;  /* bytes that data WQEs move between ranks of different racks (racks of opts.rack_size):
                                  what would cross the scale-out network with real ranks (Sec. II-A.3, V-D) */
+    int64_t static_chains;    /* 0: tiles are handed out by ticket; otherwise the number of chains of tiles that run
+                                 inside one block each (HCCL_FLAG_STATIC_CHAINS), chain_depth tiles per chain */
 } hccl_plan_info_t;
 hccl_status_t hccl_plan_info(const hccl_plan_t*, hccl_plan_info_t* out);
 

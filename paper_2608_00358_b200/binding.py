@@ -53,7 +53,7 @@ class PlanInfo(C.Structure):
                 ("schedule_bytes", C.c_int64), ("compulsory_bytes", C.c_int64), ("scratch_bytes", C.c_int64),
                 ("send_bytes_total", C.c_int64), ("recv_bytes_total", C.c_int64), ("R", C.c_int32),
                 ("sm_budget", C.c_int32), ("threads", C.c_int32), ("engine", C.c_int32), ("tile_bytes", C.c_int64),
-                ("epoch", C.c_int64), ("crossrack_bytes", C.c_int64)]
+                ("epoch", C.c_int64), ("crossrack_bytes", C.c_int64), ("static_chains", C.c_int64)]
 
 
 class HcclError(RuntimeError):

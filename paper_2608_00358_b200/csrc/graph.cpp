@@ -545,6 +545,7 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
     I.engine = p->opts.engine;
     I.tile_bytes = (int64_t)tile_bytes;
     I.crossrack_bytes = crossrack;
+    I.static_chains = (int64_t)p->n_chains;
     *out = p;
     return HCCL_OK;
 }

@@ -315,7 +315,7 @@ def test_static_chains_and_tickets_give_the_same_bits(algo, dt):
     for flags, chained in ((0, True), (hb.FLAG_DYNAMIC_TICKETS, False)):
         p = hb.hccl_plan_allreduce(R, n, dt, algo, dict(base, flags=flags))
         i = p.info()
-        assert (i.n_syncs == 0) == chained      # no device counter is left when the chains are static
+        assert (i.n_syncs == 0) == chained and (i.static_chains > 0) == chained   # no device counter is left when the chains are static
         assert p.check_hazards() == 0
         for seed in (0, 3, 4):
             Y = interpret(p, X, seed)
