@@ -167,7 +167,8 @@ def side_configs(quick: bool):
         out[key] = {"p50_us": float(np.percentile(ms, 50) * 1e3), "p99_us": float(np.percentile(ms, 99) * 1e3),
                     "back_to_back_us": float(wk.time_back_to_back(wl, it, warm) * 1e3),
                     "schedule_bytes": int(i.schedule_bytes), "compulsory_bytes": int(i.compulsory_bytes),
-                    "tiles": int(i.n_tiles), "chain_depth": int(i.chain_depth), "note": "L2-resident, latency-bound"}
+                    "tiles": int(i.n_tiles), "chain_depth": int(i.chain_depth), "blocks": int(i.sm_budget),
+                    "dispatch": "static chains" if i.static_chains else "tickets", "note": "L2-resident, latency-bound"}
         out[key]["schedule_gbs_back_to_back"] = i.schedule_bytes / out[key]["back_to_back_us"] / 1e3
         out[key]["graph_replay_us"] = float(wk.time_graph_replay(wl) * 1e3)
         # cold variant: a buffer larger than the L2 is rewritten before every iteration
@@ -247,7 +248,8 @@ def side_configs(quick: bool):
         wl = wk._bind(name, plan, send, recv, {})
         ms = wk.time_back_to_back(wl, iters, 3)
         i = wl.info
-        out[name] = {"ms": float(ms), "chain_depth": int(i.chain_depth), "tiles": int(i.n_tiles), "schedule_bytes": int(i.schedule_bytes),
+        out[name] = {"ms": float(ms), "chain_depth": int(i.chain_depth), "tiles": int(i.n_tiles), "dispatch": "static chains" if i.static_chains else "tickets",
+                     "schedule_bytes": int(i.schedule_bytes),
                      "compulsory_bytes": int(i.compulsory_bytes), "crossrack_bytes_racks_of_16": int(i.crossrack_bytes),
                      "compulsory_gbs": i.compulsory_bytes / ms / 1e6}
     for n in ((1 << 16, 1 << 22) if quick else (1 << 16, 1 << 22, 1 << 25)):
