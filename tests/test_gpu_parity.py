@@ -335,3 +335,11 @@ def test_static_chains_and_tickets_same_bits(budget, flags, dt):
     Y = run_plan(hb.hccl_plan_allgather(R, None, 7001, dt, hb.ALGO_RING, opts), Xg, iters=2, misalign=2 if dt != hb.FP32 else 4)
     for r, w in enumerate(orc.allgatherv(Xg)):
         assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("R", [2, 3, 5])
+def test_static_chains_on_degenerate_sizes(R, dt):
+    for n in (1, R - 1, R, 257, 5000):
+        for budget in (1, 148):
+            _check_allreduce(R, n, dt, hb.ALGO_RING, dict(chunk_bytes=512, sm_budget=budget), iters=2)

@@ -371,3 +371,21 @@ def test_static_chains_need_independent_linear_chains():
     g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, NB), a=(Rv, 1, NB), count=NB, dep_flags=E, dep_wqe=b)   # reads the other chain's output
     p = g.compile(opts)
     assert p.info().n_syncs == 0 and p.check_hazards() > 0
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("R", [2, 3, 4, 5, 8])
+def test_static_chains_on_degenerate_sizes(R, dt):
+    """Default options (the planner asks for static chains by itself): empty chunks, one-element chunks, sizes
+    around the rank count, several granules per chunk."""
+    for n in (0, 1, 2, R - 1, R, R + 1, 17, 255, 257, 5000):
+        X = synth.normal_ranks(R, n, dt, seed=R * 31 + n)
+        want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+        p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, dict(chunk_bytes=512, sm_budget=3))
+        assert p.check_hazards() == 0
+        if n >= R:
+            assert p.info().static_chains > 0
+        for seed in (0, 2):
+            Y = interpret(p, X, seed)
+            for r in range(R):
+                assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8)), (n, r)
