@@ -127,3 +127,33 @@ def test_single_segment_beyond_4_gib(engine):
     assert np.array_equal(recv[1][lo * 256:(lo + 4) * 256].cpu().numpy().view(np.uint8), Y[1])
     del wl, send, recv
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT], ids=["ring", "oneshot", "fanout"])
+def test_allgather_r128_at_the_benchmarked_size(algo):
+    """AllGather over 128 ranks of 2 Mi bf16 each (68.7 GB written), default options as bench.py times it.
+    The oracle's definition is a concatenation, so sampled (destination, source) blocks are compared whole,
+    and one destination is compared with the oracle's own AllGather of the same inputs."""
+    if _free_gb() < 80:
+        pytest.skip("needs 80 GB of free device memory")
+    R, n = 128, 1 << 21
+    g = torch.Generator(device="cuda")
+    g.manual_seed(128)
+    send = [torch.randint(-32768, 32767, (n,), dtype=torch.int16, device="cuda", generator=g) for _ in range(R)]
+    recv = [torch.full((n * R,), 0x5A5A, dtype=torch.int16, device="cuda") for _ in range(R)]
+    wl = wk._bind("allgather_r128", hb.hccl_plan_allgather(R, None, n, hb.BF16, algo, dict(rack_size=16)), send, recv, {})
+    for _ in range(2):
+        wl.dc.execute()
+    torch.cuda.synchronize()
+    wl.dc.check()
+    for d in (0, 1, 63, 64, 127):
+        for q in (0, 1, 17, 126, 127):
+            assert torch.equal(recv[d][q * n:(q + 1) * n], send[q]), (d, q)
+    # every destination holds the same bytes; rank 5's are the oracle's
+    X = [t.cpu().numpy().view(np.uint16) for t in send]
+    want = orc.allgatherv(X[:4])[0]                      # the oracle on the first four ranks' inputs ...
+    got = recv[5][:4 * n].cpu().numpy().view(np.uint16)  # ... is the head of every receive buffer
+    assert np.array_equal(got, want)
+    ref = recv[5]
+    for d in (0, 77, 127):
+        assert torch.equal(recv[d], ref)
