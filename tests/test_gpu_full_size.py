@@ -157,3 +157,37 @@ def test_allgather_r128_at_the_benchmarked_size(algo):
     ref = recv[5]
     for d in (0, 77, 127):
         assert torch.equal(recv[d], ref)
+
+
+@pytest.mark.parametrize("algo", [hb.ALGO_FANOUT, hb.ALGO_TREE, hb.ALGO_RING_2LEVEL], ids=["fanout", "tree", "two_level"])
+def test_allreduce_r64_at_the_benchmarked_size(algo):
+    """AllReduce over 64 ranks of 32 Mi bf16 each (4.3 GB in, 4.3 GB out), default options as bench.py times it.
+    The sum of an element does not depend on its neighbours, so the oracle is run on slices of the inputs; the
+    two-level order depends on where a slice falls, so there only the 1-ulp rule is applied."""
+    if _free_gb() < 24:
+        pytest.skip("needs 24 GB of free device memory")
+    R, n, dt = 64, 1 << 25, hb.BF16
+    g = torch.Generator(device="cuda")
+    g.manual_seed(64)
+    send = []
+    for _ in range(R):
+        x = torch.empty(n, dtype=torch.float32, device="cuda")
+        x.normal_(0.0, 1.0, generator=g)
+        send.append(x.to(torch.bfloat16))
+        del x
+    recv = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(R)]
+    wl = wk._bind("allreduce_r64", hb.hccl_plan_allreduce(R, n, dt, algo, dict(rack_size=16)), send, recv, {})
+    for _ in range(2):
+        wl.dc.execute()
+    torch.cuda.synchronize()
+    wl.dc.check()
+    for lo in (0, 12345 * 8, n // 2 - 4096, n - 65536):
+        hi = lo + 65536
+        X = [t[lo:hi].view(torch.int16).cpu().numpy().view(np.uint16) for t in send]
+        got = [recv[r][lo:hi].view(torch.int16).cpu().numpy().view(np.uint16) for r in (0, 31, 63)]
+        assert np.array_equal(got[0], got[1]) and np.array_equal(got[0], got[2])
+        assert orc.ulp_distance(dt, got[0], orc.allreduce(dt, X)[0]).max() <= 1
+        if algo == hb.ALGO_FANOUT:
+            assert np.array_equal(got[0], orc.allreduce_oneshot_f32(dt, X)[0])
+        if algo == hb.ALGO_TREE:
+            assert np.array_equal(got[0], orc.allreduce_tree_f32(dt, X)[0])
