@@ -7,11 +7,12 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libhccl_b200.so")
-SOURCES = ["graph.cpp", "collectives.cpp", "verify.cpp", "executor.cu"]
-# executor.cu is compiled in slices (one kernel each, see HCCL_PART in the file) so that they build in parallel;
-# a slice does not use every helper of the file, hence no "declared but never referenced" diagnostics for them
-PARTS = {"executor.cu": [1, 2, 3, 4]}
-HEADERS = ["plan.hpp", "tables.h", os.path.join("..", "..", "include", "hccl.h")]
+# one translation unit per kernel, so that they compile in parallel (each takes about a minute)
+SOURCES = ["graph.cpp", "collectives.cpp", "verify.cpp", "executor.cu", "kernel_lsu.cu", "kernel_lsu_light.cu", "kernel_bulk.cu",
+           "kernel_resident.cu"]
+HEADERS = ["plan.hpp", "tables.h", "device.cuh", "bulk.cuh", "bulk_layout.h", "kernels.cuh", os.path.join("..", "..", "include", "hccl.h")]
+# a kernel's unit does not use every helper of the shared headers: no "declared but never referenced" remarks for them
+QUIET = ["-diag-suppress", "177"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 
@@ -31,12 +32,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     jobs = []
     for src in SOURCES:
-        base = os.path.splitext(src)[0]
-        for part in PARTS.get(src, [None]):
-            obj = os.path.join(CSRC, base + ("" if part is None else "_%d" % part) + ".o")
-            cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ([] if part is None else ["-DHCCL_PART=%d" % part, "-diag-suppress", "177"]) + \
-                ["-x", "cu", "-c", os.path.join(CSRC, src), "-o", obj]
-            jobs.append((cmd, obj))
+        obj = os.path.join(CSRC, os.path.splitext(src)[0] + ".o")
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + (QUIET if src.endswith(".cu") else []) + \
+            ["-x", "cu", "-c", os.path.join(CSRC, src), "-o", obj]
+        jobs.append((cmd, obj))
     procs = [(subprocess.Popen(cmd), cmd) for cmd, _ in jobs]
     failed = [cmd for pr, cmd in procs if pr.wait() != 0]
     if failed:

@@ -1,0 +1,38 @@
+// Shared-memory layout of the bulk engine, needed by the kernel and by the host code that sizes its launch.
+#pragma once
+#include <stdint.h>
+
+#include "tables.h"
+
+namespace hccl {
+namespace bulk {
+
+constexpr uint32_t MAX_STAGES = 4;            // 4 x 48 KiB + bookkeeping fits the 227 KB a block may have
+constexpr uint32_t STAGE_BYTES = 49152;       // a COPY piece fills a stage; a REDUCE piece splits it into A and B
+// Elements per REDUCE piece: as many as fit a stage with both operands, in whole multiples of 512 elements
+// (6144 for fp32+fp32, 8192 for fp32+16-bit, 12288 for 16-bit+16-bit).
+__host__ __device__ constexpr uint32_t piece_elems(uint32_t ea, uint32_t eb) { return STAGE_BYTES / (ea + eb) / 512 * 512; }
+
+// PIECE_COPY: loaded and stored by the bulk unit. PIECE_COPYW: loaded by the bulk unit, stored by the compute
+// warps from shared memory (the stage is free as soon as the warps have read it, without waiting for a
+// bulk store to drain, so more of the stage ring is loads in flight).
+enum : uint32_t { PIECE_COPY = 0, PIECE_REDUCE = 1, PIECE_TILE = 2, PIECE_EXIT = 3, PIECE_COPYW = 4 };
+
+struct alignas(16) PieceInfo {  // one per stage, in shared memory; written by the DMA thread
+    uint32_t kind;
+    uint32_t n;           // REDUCE: elements; COPY: bytes
+    uint32_t last;        // last piece of its work item: publish the item's completion after it
+    uint32_t tile_index;
+    char* dst;            // global destination of this piece
+    unsigned long long group;  // COPY: sequence number of the bulk store group that drains this stage
+    int32_t signal[2];
+    uint8_t dt_a, dt_b, dt_d, evict_first;
+    uint32_t b_off;       // REDUCE: byte offset of operand B inside the stage
+    uint16_t ndst, rank_dst;   // COPY with several destinations: receive buffers of ranks rank_dst .. +ndst-1 (mod R)
+    unsigned long long dst_off;  // ... at this byte offset (dst is then the first of them)
+    Tile tile;            // PIECE_TILE: the work item and its descriptor for the register path
+    Desc desc;
+};
+
+}  // namespace bulk
+}  // namespace hccl

@@ -1,0 +1,44 @@
+// Declarations of the library's kernels and of the parameter records only some of them take. Each kernel is
+// defined in a translation unit of its own (kernel_*.cu) so that they compile in parallel; the host code
+// (executor.cu) launches them through these declarations.
+#pragma once
+#include "device.cuh"
+
+namespace hccl {
+
+struct Doorbell {                       // layout shared with hccl_doorbell_t in hccl.h
+    unsigned long long request;         // host -> device: number of executions asked for so far
+    unsigned long long completed;       // device -> host: executions finished
+    unsigned long long stop;            // host -> device: leave after the current execution
+    unsigned long long exited;          // device -> host: the kernel has left (1 = stop, 2 = idle, 3 = failure)
+    unsigned long long status, detail;  // device -> host: verdict of the last failed execution
+    unsigned long long pad[2];
+};
+
+constexpr int DYN_MAX_RANKS = 64;
+
+struct DynParams {
+    const long long* counts;       // device, [R*R], counts[s*R+d] rows from s to d
+    long long* recvcounts_out;     // device, [R*R] indexed [d*R+s], or null
+    long long* rdispls_out;        // device, [R*R] indexed [d*R+s], or null
+    Control* ctl;
+    unsigned long long* user_signals;
+    uint32_t R, nblocks;
+    unsigned long long timeout_ns;
+    unsigned long long row_bytes, tile_bytes;
+    long long trig_wait_slot, trig_set_slot;
+    int trig_cmp, pad1;
+    unsigned long long trig_wait_value, trig_wait_per_epoch, trig_set_value, trig_set_per_epoch;
+    long long max_send_rows[DYN_MAX_RANKS], max_recv_rows[DYN_MAX_RANKS];
+    const void* send[DYN_MAX_RANKS];
+    void* recv[DYN_MAX_RANKS];
+};
+
+__global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p);
+__global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p);
+__global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t copy_by_warps);
+__global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_constant__ ExecParams p, Doorbell* db,
+                                                                  const unsigned long long idle_ns, const uint32_t first_epoch);
+__global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant__ DynParams q);
+
+}  // namespace hccl
