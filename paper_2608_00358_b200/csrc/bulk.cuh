@@ -1,3 +1,5 @@
+// The bulk (TMA) engine's device code: mbarrier and cp.async.bulk wrappers, the per-piece FP32 add from shared
+// memory, and the DMA thread that claims items, resolves dependencies and drives the stage ring.
 #pragma once
 #include "bulk_layout.h"
 #include "device.cuh"
