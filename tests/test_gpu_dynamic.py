@@ -150,3 +150,74 @@ def test_start_gate_that_never_opens_times_out_cleanly():
     for t in recv:
         assert bool((t == SENT).all())
     assert float(torch.ones(4, device="cuda").sum()) == 4.0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("kind", ["ring_chains", "ring_tickets", "alltoallv_bulk"])
+def test_device_triggered_static_plans(kind):
+    """The start gate and the completion value on statically planned collectives: the register engine with static
+    chains and with tickets, and the bulk engine. The collective is enqueued first and holds (bounded) at its
+    gate on a few SMs; a fill on another stream releases it."""
+    import torch
+    from gpu_helpers import SENTINEL
+    from oracle import oracle as orc
+    R = 4
+    if kind == "alltoallv_bulk":
+        C = synth.uniform_counts(R, 3, hi=50)
+        X = [synth.hashed_rows_np(s, 0, max(int(C[s].sum()), 1), 32).reshape(-1).view(np.uint8) for s in range(R)]
+        plan = hb.hccl_plan_alltoallv(R, C, None, None, None, hb.FP16, 32, dict(sm_budget=8, engine=hb.ENGINE_BULK))
+        want = [np.full(int(C[:, d].sum()) * 64, 0, dtype=np.uint8) for d in range(R)]
+        SD, RD = orc.packed_displs(C)
+        orc.alltoallv(X, want, C, SD, RD, 64)
+    else:
+        n = 30011
+        X = synth.normal_ranks(R, n, hb.BF16, seed=9)
+        flags = 0 if kind == "ring_chains" else hb.FLAG_DYNAMIC_TICKETS
+        plan = hb.hccl_plan_allreduce(R, n, hb.BF16, hb.ALGO_RING, dict(sm_budget=8, tile_bytes=4096, chunk_bytes=16384, flags=flags))
+        assert (plan.info().static_chains > 0) == (kind == "ring_chains")
+        want = [w.view(np.uint8) for w in orc.allreduce_ring_f32(hb.BF16, X, orc.floor_chunk_offsets(n, R))]
+    send = [torch.from_numpy(x.view(np.uint8).copy()).cuda() for x in X]
+    recv = [torch.full((max(plan.extents(r)[1], 16),), SENTINEL, dtype=torch.uint8, device="cuda") for r in range(R)]
+    from paper_2608_00358_b200.runtime import DeviceCollective
+    dc = DeviceCollective(plan)
+    dc.set_buffers([t.data_ptr() for t in send], [t.data_ptr() for t in recv], keep=(send, recv))
+    signals = torch.zeros(2, dtype=torch.int64, device="cuda")
+    plan.set_user_signals(signals.data_ptr(), 2)
+    plan.set_trigger(wait_slot=0, cmp=hb.CMP_GE, wait_value=0, wait_per_epoch=1, set_slot=1, set_value=500, set_per_epoch=1)
+    coll, prod = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for epoch in (1, 2):
+        for t in recv:
+            t.fill_(SENTINEL)
+        torch.cuda.synchronize()
+        dc.execute(coll)
+        with torch.cuda.stream(prod):
+            signals[0:1].fill_(epoch)
+        torch.cuda.synchronize()
+        assert plan.status()[0] == hb.OK
+        assert int(signals[1]) == 500 + epoch
+        for r in range(R):
+            assert np.array_equal(recv[r].cpu().numpy()[:want[r].size], want[r]), (kind, epoch, r)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("engine", [hb.ENGINE_LSU, hb.ENGINE_BULK], ids=["lsu", "bulk"])
+def test_static_plan_gate_that_never_opens_times_out_cleanly(engine):
+    import torch
+    R, n = 2, 4096
+    X = synth.normal_ranks(R, n, hb.FP32, seed=1)
+    plan = hb.hccl_plan_allreduce(R, n, hb.FP32, hb.ALGO_RING, dict(sm_budget=2, timeout_ns=200_000_000, engine=engine))
+    send = [torch.from_numpy(x).cuda() for x in X]
+    recv = [torch.full((n,), 7.0, dtype=torch.float32, device="cuda") for _ in range(R)]
+    from paper_2608_00358_b200.runtime import DeviceCollective
+    dc = DeviceCollective(plan)
+    dc.set_buffers([t.data_ptr() for t in send], [t.data_ptr() for t in recv], keep=(send, recv))
+    signals = torch.zeros(1, dtype=torch.int64, device="cuda")
+    plan.set_user_signals(signals.data_ptr(), 1)
+    plan.set_trigger(wait_slot=0, cmp=hb.CMP_EQ, wait_value=12345)
+    dc.execute()
+    torch.cuda.synchronize()
+    assert plan.status()[0] == hb.ERR_TIMEOUT
+    for t in recv:
+        assert bool((t == 7.0).all())
+    assert float(torch.ones(4, device="cuda").sum()) == 4.0
