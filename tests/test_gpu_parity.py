@@ -343,3 +343,27 @@ def test_static_chains_on_degenerate_sizes(R, dt):
     for n in (1, R - 1, R, 257, 5000):
         for budget in (1, 148):
             _check_allreduce(R, n, dt, hb.ALGO_RING, dict(chunk_bytes=512, sm_budget=budget), iters=2)
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("flags", [hb.FLAG_LEVEL_MAJOR, hb.FLAG_STAGED_RING, hb.FLAG_STAGED_RING | hb.FLAG_DYNAMIC_TICKETS,
+                                   hb.FLAG_LEVEL_MAJOR | hb.FLAG_BIDIRECTIONAL], ids=["level_major", "staged", "staged_tickets", "level_major_bidir"])
+def test_ring_order_flags_on_device(flags, dt, engine):
+    """Issue-order and staging variants of the ring move the same values through the same sums: identical bits."""
+    R, n, granule = 5, 30011, 1024
+    es = hb.ELEM_BYTES[dt]
+    X = synth.normal_ranks(R, n, dt, seed=flags + 3)
+    opts = _with(dict(tile_bytes=2048, chunk_bytes=granule * es, chain_group=2, sm_budget=24, flags=flags), engine)
+    Y = run_plan(hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, opts), X, iters=2)
+    if flags & hb.FLAG_BIDIRECTIONAL:
+        so, sc, sd = orc.bidirectional_segments(n, R, granule)
+        want = orc.allreduce_ring_dir_f32(dt, X, so, sc, sd)
+    else:
+        want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8)), r
+    rc = np.diff(orc.floor_chunk_offsets(n, R))
+    if not flags & hb.FLAG_BIDIRECTIONAL:
+        Y = run_plan(hb.hccl_plan_reducescatter(R, None, n, dt, hb.ALGO_RING, opts), X)
+        for r, w in enumerate(orc.reducescatter_ring_f32(dt, X, rc)):
+            assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
