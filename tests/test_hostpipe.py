@@ -94,3 +94,28 @@ def test_pipelined_alltoallv_matches_oracle(R, windows, engine):
             assert np.all(got[rb[d]:] == 0xA5), "bytes past the receive extent of rank %d were written" % d
     for d in range(R):   # staging buffers: nothing beyond the extents
         assert bool((dev_recv[d][rb[d]:] == 0xA5).all())
+
+
+@pytest.mark.gpu
+def test_execute_host_single_stream():
+    """hccl_execute_host: host buffers in, one stream (copy in, execute, copy out), host buffers out."""
+    import torch
+    R, n, dt = 4, 5001, hb.BF16
+    X = synth.normal_ranks(R, n, dt, seed=4)
+    plan = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, dict(sm_budget=8))
+    ws = torch.empty(plan.workspace_bytes() + 256, dtype=torch.uint8, device="cuda")
+    s = torch.cuda.Stream()
+    plan.bind((ws.data_ptr() + 255) // 256 * 256, plan.workspace_bytes(), s.cuda_stream)
+    hs = [torch.from_numpy(x.view(np.int16).copy()).pin_memory() for x in X]
+    hr = [torch.full((n + 8,), 0x5A5A, dtype=torch.int16).pin_memory() for _ in range(R)]
+    ds = [torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(R)]
+    dr = [torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(R)]
+    for _ in range(2):
+        plan.execute_host([t.data_ptr() for t in hs], [t.data_ptr() for t in hr], [t.data_ptr() for t in ds],
+                          [t.data_ptr() for t in dr], s.cuda_stream)
+    s.synchronize()
+    assert plan.status()[0] == hb.OK
+    want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    for r in range(R):
+        got = hr[r].numpy().view(np.uint16)
+        assert np.array_equal(got[:n], want[r]) and np.all(got[n:] == 0x5A5A)
