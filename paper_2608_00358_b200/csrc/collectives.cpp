@@ -788,7 +788,10 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw));
     GraphPtr g(graw);
     g->compulsory_bytes = offs[R] * es + (int64_t)R * offs[R] * es;
-    const int64_t tile = o.tile_bytes ? (int64_t)o.tile_bytes : default_tile(offs[R] * es, o.sm_budget, 1, 16 << 10, 256 << 10, sweep_of(o, HCCL_OP_COPY));
+    // hop-by-hop copies on the register engine: at most three passes of the block's threads per tile (180 KiB),
+    // which keeps what a block has just written (and reads next) inside the L2 (12.5 vs 14.0 ms at R = 128, 4 MiB)
+    const int64_t tile_cap = (algo == HCCL_ALGO_RING && o.engine == HCCL_ENGINE_LSU) ? 3 * sweep_of(o, HCCL_OP_COPY) : (256 << 10);
+    const int64_t tile = o.tile_bytes ? (int64_t)o.tile_bytes : default_tile(offs[R] * es, o.sm_budget, 1, 16 << 10, tile_cap, sweep_of(o, HCCL_OP_COPY));
     // one subgraph per chunk q: it first lands in its owner's receive buffer, then goes round (ring)
     // or is read by everyone directly (one-shot)
     std::vector<int32_t> sg(R);
