@@ -104,12 +104,14 @@ typedef enum {
 #define HCCL_FLAG_BIDIRECTIONAL 8u /* flat ring AllReduce / ReduceScatter: granules of a chunk alternate direction, even
                                      ones travel r -> r+1, odd ones r -> r-1 (a bidirectional ring, Sec. III-B.2) */
 
-#define HCCL_FLAG_STATIC_CHAINS 16u /* if every dependency of the packet is a tile-by-tile link to one predecessor and
-                                      every WQE has at most one such successor (the packet is a set of independent
-                                      chains, like a small ring), run each chain of tiles inside ONE block, in order:
-                                      a barrier of that block then stands where a device counter and a poll across
-                                      SMs would. Register engine only; ignored when the packet has another shape.
-                                      The ring planners ask for it themselves for small buffers. */
+#define HCCL_FLAG_STATIC_CHAINS 16u /* if every dependency of the packet is a tile-by-tile link (HCCL_DEP_ELEMENTWISE
+                                      between WQEs cut into the same number of tiles) and the groups of WQEs linked
+                                      that way are equally long (the chains of a small ring; the copies of one
+                                      chunk in a hop-by-hop AllGather; a granule's tree of sums), run tile k of a
+                                      whole group inside ONE block, in issue order: a barrier of that block then
+                                      stands where a device counter and a poll across SMs would. Register engine
+                                      only; ignored when the packet has another shape. The planners ask for it
+                                      themselves where it pays. */
 #define HCCL_FLAG_DYNAMIC_TICKETS 32u /* keep the planners from asking for HCCL_FLAG_STATIC_CHAINS */
 
 /* Options. A zero field means "default". */

@@ -384,7 +384,11 @@ hccl_status_t plan_allreduce_2level(int R, int64_t count, hccl_dtype_t dt, const
 
 // Two-level AllGather: rank (g, j)'s block first lands in its own receive buffer, then travels to the other
 // racks' rank j (the only hops between racks), and every rack passes it round its own ring.
-hccl_status_t plan_allgather_2level(int R, const std::vector<int64_t>& offs, hccl_dtype_t dt, const hccl_opts_t& o, hccl_plan_t** out) {
+hccl_status_t plan_allgather_2level(int R, const std::vector<int64_t>& offs, hccl_dtype_t dt, const hccl_opts_t& o_in, hccl_plan_t** out) {
+    hccl_opts_t o = o_in;
+    // all copies of one chunk (its trip round the racks and then round every rack) form one group of linked WQEs:
+    // a block can walk a tile through all of them by itself
+    if (!(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const int L = o.rack_size, G = R / L, es = elem_bytes(dt);
     std::vector<int64_t> sext(R), rext(R, offs[R] * es);
     for (int r = 0; r < R; ++r) sext[r] = (offs[r + 1] - offs[r]) * es;
@@ -407,8 +411,8 @@ hccl_status_t plan_allgather_2level(int R, const std::vector<int64_t>& offs, hcc
     }
     TwoLevel T{g.get(), G, L, (int)dt, es, offs[R], 0, o};
     T.tile_elems = o.tile_bytes ? std::max<int64_t>(1, (int64_t)(o.tile_bytes / (uint64_t)es))
-                                : default_tile(std::min<int64_t>(offs[R], (int64_t)o.chain_group * granule) * G * es, o.sm_budget, 1, 16 << 10, 256 << 10,
-                                               sweep_of(o, HCCL_OP_COPY)) / es;
+                                : default_tile(std::min<int64_t>(offs[R], (int64_t)o.chain_group * granule) * G * es, o.sm_budget, 1, 16 << 10,
+                                               o.engine == HCCL_ENGINE_LSU ? 3 * sweep_of(o, HCCL_OP_COPY) : (256 << 10), sweep_of(o, HCCL_OP_COPY)) / es;
     T.tile_elems = std::max<int64_t>(T.tile_elems, 1);
     const size_t nch = items.size(), group = (size_t)o.chain_group;
     std::vector<int32_t> sg(nch);
@@ -419,6 +423,35 @@ hccl_status_t plan_allgather_2level(int R, const std::vector<int64_t>& offs, hcc
         gs[i].last.assign(G, -1);
     }
     const int stages = 1 + (G - 1) + (L - 1);
+    if (o.flags & HCCL_FLAG_STATIC_CHAINS) {
+        // One block will run an item's copies in this order: own copy, the hops round the racks, then rack by
+        // rack the hops round that rack, so that every hop reads what the hop just before it wrote.
+        for (size_t i = 0; i < nch; ++i) {
+            const Chain2& ch = items[i].ch;
+            hccl_wqe_t w = blank();
+            w.op = HCCL_OP_COPY;
+            w.count = ch.len * es;
+            w.tile_count = T.tile_elems * es;
+            const int r0 = T.rank(ch.k, ch.j);
+            w.a = ref(HCCL_BUF_SEND, r0, items[i].src_off * es);
+            w.dst = ref(HCCL_BUF_RECV, r0, ch.e0 * es);
+            CHECK(hccl_graph_add_wqe(g.get(), sg[i], &w, &gs[i].arrive[ch.k]));
+            for (int stage = 0; stage < G - 1; ++stage) CHECK(emit_gather_stage(T, sg[i], ch, ch.e0, stage, gs[i]));
+            for (int rack = 0; rack < G; ++rack) {
+                int64_t prev = gs[i].arrive[rack];
+                for (int h = 0; h < L - 1; ++h) {
+                    hccl_wqe_t c = blank();
+                    c.op = HCCL_OP_COPY;
+                    c.count = ch.len * es;
+                    c.tile_count = T.tile_elems * es;
+                    c.a = ref(HCCL_BUF_RECV, T.rank(rack, ch.j + h), ch.e0 * es);
+                    c.dst = ref(HCCL_BUF_RECV, T.rank(rack, ch.j + h + 1), ch.e0 * es);
+                    CHECK(add_dep_wqe(g.get(), sg[i], c, prev, -1, &prev));
+                }
+            }
+        }
+        return hccl_graph_compile(g.get(), &o, out);
+    }
     for (size_t g0 = 0; g0 < nch; g0 += group) {
         const size_t g1 = std::min(nch, g0 + group);
         for (int stage = 0; stage < stages; ++stage) {
@@ -453,6 +486,10 @@ hccl_status_t plan_allreduce_tree(int R, int64_t count, hccl_dtype_t dt, hccl_op
     const int64_t ng = count > 0 ? (count + granule - 1) / granule : 0;
     if (!group_given && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<int64_t>(ng, 1);  // small: all granules together
     const int64_t group = std::max<int64_t>(1, o.chain_group);
+    // From about 1 MiB per rank a block does better walking one tile through the whole tree by itself (no
+    // hand-over between SMs, 2(R-1) items in a row) than the blocks do sharing the tree's 2 log2 R levels;
+    // below that the levels' parallelism wins (measured at R = 8: 28.7 vs 43.0 us at 1 MiB, 28.7 vs 25.1 at 256 KiB).
+    if (count * es >= (1ll << 20) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const int half = (R + 1) / 2;                                 // scratch slots one granule needs
     const int64_t n_sets = std::min<int64_t>(std::max<int64_t>(ng, 1), 2 * group);  // recycled sets of slots
     const int64_t slot_elems = (int64_t)align_up((uint64_t)std::min<int64_t>(granule, std::max<int64_t>(count, 1)), 64);

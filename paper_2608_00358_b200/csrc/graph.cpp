@@ -392,7 +392,6 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         for (int64_t i : pe[j]) need_tile[i] = 1;
     }
     // ---- static chains: the packet is a set of independent chains of equal length, linked tile by tile
-    std::vector<int64_t> chain_pred(n, -1), chain_succ(n, -1);
     std::vector<int64_t> depth(n, 1);
     int64_t max_depth = n ? 1 : 0;
     for (size_t i = 0; i < n; ++i) {
@@ -401,23 +400,38 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         max_depth = std::max(max_depth, depth[i]);
     }
     bool chains = (p->opts.flags & HCCL_FLAG_STATIC_CHAINS) != 0 && p->opts.engine == HCCL_ENGINE_LSU && n > 0 && max_depth > 1;
+    // Every dependency must be a tile-by-tile link; WQEs linked (directly or not) form a group that one block runs
+    // in issue order, which already has every predecessor before its successors. A ring's chain is such a
+    // group; so is a chunk that forks into several racks. Groups must be equally long, so that a block finds
+    // its tiles by arithmetic.
+    std::vector<int64_t> group_of(n);
+    for (size_t j = 0; j < n; ++j) group_of[j] = (int64_t)j;
+    auto root = [&](int64_t x) {
+        while (group_of[x] != x) x = group_of[x] = group_of[group_of[x]];
+        return x;
+    };
     for (size_t j = 0; j < n && chains; ++j) {
         const int op = g->wqes[j].w.op;
-        if (!pf[j].empty() || pe[j].size() > 1 || op == HCCL_OP_WAIT || op == HCCL_OP_SET) chains = false;
-        if (chains && pe[j].size() == 1) {
-            const int64_t i = pe[j][0];
-            if (chain_succ[i] >= 0) chains = false;
-            chain_succ[i] = (int64_t)j;
-            chain_pred[j] = i;
-        }
+        if (!pf[j].empty() || op == HCCL_OP_WAIT || op == HCCL_OP_SET) chains = false;
+        for (int64_t i : pe[j]) group_of[root((int64_t)j)] = root(i);   // roots keep the smallest id: i < j
     }
-    std::vector<int64_t> heads;
-    for (size_t i = 0; i < n && chains; ++i) {
-        if (chain_pred[i] >= 0) continue;
-        int64_t len = 0;
-        for (int64_t w = (int64_t)i; w >= 0; w = chain_succ[w]) ++len;
-        if (len != max_depth) chains = false;  // equal lengths: a block finds its tiles by arithmetic
-        heads.push_back((int64_t)i);
+    std::vector<std::vector<int64_t>> groups;   // in order of their first WQE
+    if (chains) {
+        std::vector<int64_t> index_of(n, -1);
+        for (size_t j = 0; j < n; ++j) {
+            const int64_t r = root((int64_t)j);
+            if (index_of[r] < 0) {
+                index_of[r] = (int64_t)groups.size();
+                groups.emplace_back();
+            }
+            groups[index_of[r]].push_back((int64_t)j);
+        }
+        for (const auto& grp : groups) {
+            if (grp.size() != groups[0].size()) chains = false;
+            for (int64_t w : grp)
+                if (ntiles[w] != ntiles[grp[0]]) chains = false;
+        }
+        if (groups.empty() || groups[0].size() < 2) chains = false;
     }
     if (chains) {
         for (size_t j = 0; j < n; ++j) pe[j].clear();  // the order inside a block replaces every counter
@@ -485,17 +499,18 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
     }
 
     if (chains) {
-        // chain c = tile k of every WQE of one WQE chain, in order; chains are numbered WQE chain by WQE chain
+        // chain c = tile k of every WQE of one group, in issue order; chains are numbered group by group
+        const uint64_t group_len = groups[0].size();
         uint64_t n_chains = 0;
-        for (int64_t h : heads) n_chains += (uint64_t)ntiles[h];
-        if (n_chains * (uint64_t)max_depth > 0x7ffffff0ull) {
+        for (const auto& grp : groups) n_chains += (uint64_t)ntiles[grp[0]];
+        if (n_chains * group_len > 0x7ffffff0ull) {
             delete p;
             return HCCL_ERR_INVALID_ARG;
         }
-        p->tiles.reserve((size_t)(n_chains * (uint64_t)max_depth));
-        for (int64_t h : heads) {
-            for (int64_t k = 0; k < ntiles[h]; ++k) {
-                for (int64_t w = h; w >= 0; w = chain_succ[w]) {
+        p->tiles.reserve((size_t)(n_chains * group_len));
+        for (const auto& grp : groups) {
+            for (int64_t k = 0; k < ntiles[grp[0]]; ++k) {
+                for (int64_t w : grp) {
                     const hccl_wqe_t& q = g->wqes[w].w;
                     Tile t;
                     std::memset(&t, 0, sizeof(t));
@@ -509,7 +524,7 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
                 }
             }
         }
-        p->chain_len = (uint32_t)max_depth;
+        p->chain_len = (uint32_t)group_len;
         p->n_chains = (uint32_t)n_chains;
         p->opts.sm_budget = (int32_t)std::max<uint64_t>(1, std::min<uint64_t>((uint64_t)p->opts.sm_budget, n_chains));
     }

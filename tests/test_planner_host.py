@@ -335,7 +335,7 @@ def test_static_chains_and_tickets_give_the_same_bits(algo, dt):
         assert np.array_equal(interpret(p, Xg, 6)[r].view(np.uint8), w.view(np.uint8))
 
 
-def test_static_chains_need_independent_linear_chains():
+def test_static_chains_need_independent_groups_of_equal_length():
     NB = 4096
     S, Rv = hb.BUF_SEND, hb.BUF_RECV
     opts = dict(tile_bytes=1024, sm_budget=4, flags=hb.FLAG_STATIC_CHAINS)
@@ -354,14 +354,32 @@ def test_static_chains_need_independent_linear_chains():
     for seed in range(6):
         Y = interpret(p, X, seed)
         assert np.array_equal(Y[0], np.concatenate([X[0], X[1]])) and np.array_equal(Y[1], np.concatenate([X[1], X[0]]))
-    # a WQE with two successors is not a chain: the compiler keeps the counters
+    # a WQE with two successors (a fork) still makes one group: the block runs its three WQEs in issue order
     g = hb.Graph(2, [NB, NB], [2 * NB, 2 * NB])
     sg = g.add_subgraph(0)
     a = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, 0), a=(S, 0, 0), count=NB)
     g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, 0), a=(Rv, 0, 0), count=NB, dep_flags=E, dep_wqe=a)
     g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, NB), a=(Rv, 0, 0), count=NB, dep_flags=E, dep_wqe=a)
     p = g.compile(opts)
-    assert p.info().n_syncs > 0 and p.check_hazards() == 0
+    assert p.info().static_chains == 4 and p.info().n_syncs == 0 and p.check_hazards() == 0
+    for seed in range(4):
+        Y = interpret(p, X, seed)
+        assert np.array_equal(Y[0][:NB], X[0]) and np.array_equal(Y[1], np.concatenate([X[0], X[0]]))
+    # groups of different lengths (a chain of two and a single WQE): the compiler keeps tickets and counters
+    g = hb.Graph(2, [NB, NB], [2 * NB, 2 * NB])
+    sg = g.add_subgraph(0)
+    a = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, 0), a=(S, 0, 0), count=NB)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, 0), a=(Rv, 0, 0), count=NB, dep_flags=E, dep_wqe=a)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, NB), a=(S, 1, 0), count=NB)
+    p = g.compile(opts)
+    assert p.info().static_chains == 0 and p.info().n_syncs > 0 and p.check_hazards() == 0
+    # a dependency on a whole WQE (not tile by tile) also keeps them
+    g = hb.Graph(2, [NB, NB], [2 * NB, 2 * NB])
+    sg = g.add_subgraph(0)
+    a = g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 0, 0), a=(S, 0, 0), count=NB)
+    g.add_wqe(sg, hb.OP_COPY, dst=(Rv, 1, 0), a=(Rv, 0, 0), count=NB, dep_flags=hb.DEP_WQE_SYNC, dep_wqe=a)
+    p = g.compile(opts)
+    assert p.info().static_chains == 0 and p.info().n_syncs > 0
     # chains that touch the same bytes without a link between them: static or not, the checker objects
     g = hb.Graph(2, [NB, NB], [2 * NB, 2 * NB])
     sg = g.add_subgraph(0)
