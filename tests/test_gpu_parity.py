@@ -367,3 +367,19 @@ def test_ring_order_flags_on_device(flags, dt, engine):
         Y = run_plan(hb.hccl_plan_reducescatter(R, None, n, dt, hb.ALGO_RING, opts), X)
         for r, w in enumerate(orc.reducescatter_ring_f32(dt, X, rc)):
             assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("flags", [hb.FLAG_STATIC_CHAINS, hb.FLAG_DYNAMIC_TICKETS], ids=["groups", "tickets"])
+def test_tree_and_two_level_allgather_as_groups(flags, dt):
+    R, n = 8, 40009
+    opts = dict(tile_bytes=2048, chunk_bytes=16384, chain_group=64, sm_budget=12, rack_size=4, flags=flags)
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_TREE, opts)
+    assert (p.info().static_chains > 0) == (flags == hb.FLAG_STATIC_CHAINS)
+    _check_allreduce(R, n, dt, hb.ALGO_TREE, opts, iters=2)
+    X = synth.normal_ranks(R, 5003, dt, seed=2)
+    p = hb.hccl_plan_allgather(R, None, 5003, dt, hb.ALGO_RING_2LEVEL, opts)
+    assert (p.info().static_chains > 0) == (flags == hb.FLAG_STATIC_CHAINS)
+    Y = run_plan(p, X, iters=2)
+    for r, w in enumerate(orc.allgatherv(X)):
+        assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))

@@ -407,3 +407,36 @@ def test_static_chains_on_degenerate_sizes(R, dt):
             Y = interpret(p, X, seed)
             for r in range(R):
                 assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8)), (n, r)
+
+
+@pytest.mark.parametrize("dt", DTYPES)
+@pytest.mark.parametrize("R,n", [(2, 600), (5, 3001), (8, 4099), (13, 700)])
+def test_tree_as_groups_inside_one_block(R, n, dt):
+    """The tree's sums have two predecessors each, so a granule's WQEs form one group (not a chain); with
+    HCCL_FLAG_STATIC_CHAINS a block runs tile k of the whole group in issue order. Same bits as with tickets."""
+    X = synth.normal_ranks(R, n, dt, seed=R + n)
+    want = orc.allreduce_tree_f32(dt, X)
+    for flags, grouped in ((hb.FLAG_STATIC_CHAINS, True), (0, False)):
+        p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_TREE, dict(tile_bytes=512, chunk_bytes=2048, chain_group=64, sm_budget=5, flags=flags))
+        i = p.info()
+        assert (i.static_chains > 0) == grouped and p.check_hazards() == 0
+        for seed in (0, 7):
+            Y = interpret(p, X, seed)
+            for r in range(R):
+                assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8)), (flags, r)
+
+
+def test_two_level_allgather_runs_as_groups_by_default():
+    p = hb.hccl_plan_allgather(8, None, 500, hb.BF16, hb.ALGO_RING_2LEVEL, dict(rack_size=4, tile_bytes=256))
+    i = p.info()
+    assert i.static_chains > 0 and i.n_syncs == 0 and p.check_hazards() == 0
+    q = hb.hccl_plan_allgather(8, None, 500, hb.BF16, hb.ALGO_RING_2LEVEL, dict(rack_size=4, tile_bytes=256, flags=hb.FLAG_DYNAMIC_TICKETS))
+    assert q.info().static_chains == 0 and q.info().n_syncs > 0 and q.check_hazards() == 0
+    assert q.info().crossrack_bytes == i.crossrack_bytes and q.info().schedule_bytes == i.schedule_bytes
+    rng = np.random.default_rng(1)
+    X = [rng.integers(0, 65536, size=500, dtype=np.uint16) for _ in range(8)]
+    want = orc.allgatherv(X)
+    for plan in (p, q):
+        Y = interpret(plan, X, 3)
+        for r in range(8):
+            assert np.array_equal(Y[r].view(np.uint16), want[r])
