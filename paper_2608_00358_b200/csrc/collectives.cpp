@@ -610,7 +610,14 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_RING_2LEVEL &&
         algo != HCCL_ALGO_FANOUT && algo != HCCL_ALGO_TREE) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
-    fill_ring_opts(&o, opts, (int64_t)R * count * elem_bytes(dt), algo == HCCL_ALGO_RING_FUSED || algo == HCCL_ALGO_ONESHOT || algo == HCCL_ALGO_FANOUT || R == 1);
+    // An FP32 ring keeps its partials in the receive buffers (no scratch slot is ever shared between chains), so
+    // its chains can stay inside one block at any size; that needs the register engine (measured ahead of the
+    // bulk engine with tickets: 0.50 vs 0.57 ms at R = 4 x 64 Mi, 0.63 vs 0.69 ms at R = 16 x 16 Mi).
+    const bool fp32_ring = dt == HCCL_FP32 && algo == HCCL_ALGO_RING && R > 1;
+    hccl_opts_t pre;
+    if (opts) pre = *opts; else std::memset(&pre, 0, sizeof(pre));
+    if (fp32_ring && pre.engine == HCCL_ENGINE_AUTO) pre.engine = HCCL_ENGINE_LSU;
+    fill_ring_opts(&o, &pre, (int64_t)R * count * elem_bytes(dt), algo == HCCL_ALGO_RING_FUSED || algo == HCCL_ALGO_ONESHOT || algo == HCCL_ALGO_FANOUT || R == 1);
     if (algo == HCCL_ALGO_RING_2LEVEL) {
         if (R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
         // a single rack, or racks of one rank, is the flat ring
@@ -681,7 +688,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     // dependency chain is then as short as the ring allows; large ones keep chain groups for L2 residency
     if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
     // ... and each chain of tiles can then stay inside one block (no slot is recycled, so nothing links the chains)
-    if (count * 4 <= (32ll << 20) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
+    if ((count * 4 <= (32ll << 20) || in_recv) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const bool need_scratch = !in_recv && !fused && R > 2;
     const bool staged = (o.flags & HCCL_FLAG_STAGED_RING) != 0 && need_scratch;
     // level-major order runs every chain's step t before any step t+1, so no slot can be recycled
@@ -692,7 +699,11 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     const int64_t weight = count * 4 * (R - 1) + (int64_t)count * es * (R - 1);
     const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
     (void)weight;
-    const int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, in_recv ? es : 4, HCCL_OP_REDUCE, maxlen);
+    int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, in_recv ? es : 4, HCCL_OP_REDUCE, maxlen);
+    // large FP32 rings as static chains: two passes of the block's threads per tile keep a block's current
+    // partial (written by one step, read by the next) in the L2
+    if (in_recv && o.engine == HCCL_ENGINE_LSU && !o.tile_bytes && count * 4 > (32ll << 20) && (o.flags & HCCL_FLAG_STATIC_CHAINS))
+        tile_elems = 2 * sweep_of(o, HCCL_OP_REDUCE);
     if (!fused && o.engine == HCCL_ENGINE_LSU && (!opts || opts->sm_budget == 0) && maxlen > 0) {
         // a step that is a little short of one round of the blocks: launch exactly that many blocks, so that
         // block b keeps meeting tile b of every step (measured 54 vs 58 us at R = 8, 1 MiB per rank)

@@ -191,3 +191,25 @@ def test_allreduce_r64_at_the_benchmarked_size(algo):
             assert np.array_equal(got[0], orc.allreduce_oneshot_f32(dt, X)[0])
         if algo == hb.ALGO_TREE:
             assert np.array_equal(got[0], orc.allreduce_tree_f32(dt, X)[0])
+
+
+def test_large_fp32_ring_allreduce_as_static_chains():
+    """FP32 rings keep their partials in the receive buffers, so they run as static chains at any size
+    (default options, as a caller gets them): R = 4, 16 Mi elements per rank, every output against the oracle."""
+    R, n = 4, 1 << 24
+    X = synth.uniform_ranks(R, n, hb.FP32, seed=24)
+    send = [torch.from_numpy(x).cuda() for x in X]
+    recv = [torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(R)]
+    plan = hb.hccl_plan_allreduce(R, n, hb.FP32, hb.ALGO_RING)
+    i = plan.info()
+    assert i.static_chains > 0 and i.n_syncs == 0 and i.engine == hb.ENGINE_LSU
+    wl = wk._bind("allreduce_r4_fp32_16Mi", plan, send, recv, {})
+    for _ in range(2):
+        wl.dc.execute()
+    wl.dc.check()
+    want = orc.allreduce_ring_f32(hb.FP32, X, orc.floor_chunk_offsets(n, R))
+    exact = orc.sum_f64(hb.FP32, X)
+    for r in range(R):
+        got = recv[r].cpu().numpy()
+        assert np.array_equal(got.view(np.uint32), want[r].view(np.uint32)), r
+    assert np.all(np.abs(got.astype(np.float64) - exact) <= 1e-5 * np.abs(exact) + 1e-6)
