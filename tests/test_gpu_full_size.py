@@ -159,7 +159,7 @@ def test_allgather_r128_at_the_benchmarked_size(algo):
         assert torch.equal(recv[d], ref)
 
 
-@pytest.mark.parametrize("algo", [hb.ALGO_FANOUT, hb.ALGO_TREE, hb.ALGO_RING_2LEVEL], ids=["fanout", "tree", "two_level"])
+@pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_FANOUT, hb.ALGO_TREE, hb.ALGO_RING_2LEVEL], ids=["ring", "fanout", "tree", "two_level"])
 def test_allreduce_r64_at_the_benchmarked_size(algo):
     """AllReduce over 64 ranks of 32 Mi bf16 each (4.3 GB in, 4.3 GB out), default options as bench.py times it.
     The sum of an element does not depend on its neighbours, so the oracle is run on slices of the inputs; the
@@ -191,6 +191,14 @@ def test_allreduce_r64_at_the_benchmarked_size(algo):
             assert np.array_equal(got[0], orc.allreduce_oneshot_f32(dt, X)[0])
         if algo == hb.ALGO_TREE:
             assert np.array_equal(got[0], orc.allreduce_tree_f32(dt, X)[0])
+        if algo == hb.ALGO_RING:
+            # an element of chunk c is summed starting at rank c + 1 and going round the ring: cut the slice at
+            # the chunk boundaries and give every piece its chunk
+            offs = orc.floor_chunk_offsets(n, R)
+            cuts = sorted({lo, hi} | {int(o) for o in offs if lo < o < hi})
+            chunk = [int(np.searchsorted(offs, a, side="right")) - 1 for a in cuts[:-1]]
+            ring = orc.allreduce_ring_dir_f32(dt, X, [a - lo for a in cuts], chunk, [1] * len(chunk))
+            assert np.array_equal(got[0], ring[0])
 
 
 def test_large_fp32_ring_allreduce_as_static_chains():
