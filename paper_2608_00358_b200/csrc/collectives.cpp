@@ -693,7 +693,9 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     // dependency chain is then as short as the ring allows; large ones keep chain groups for L2 residency
     if ((!opts || opts->chain_group == 0) && (count * 4 <= (32ll << 20) || own_slots)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
     // ... and each chain of tiles can then stay inside one block (no slot is recycled, so nothing links the chains)
-    if ((count * 4 <= (32ll << 20) || in_recv || own_slots) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
+    // (the fused form has no partials at all: its one sum per granule is followed by copies that hop from the
+    // bytes the same block has just written)
+    if ((count * 4 <= (32ll << 20) || in_recv || own_slots || fused) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const bool need_scratch = !in_recv && !fused && R > 2;
     const bool staged = (o.flags & HCCL_FLAG_STAGED_RING) != 0 && need_scratch;
     // level-major order runs every chain's step t before any step t+1, so no slot can be recycled
