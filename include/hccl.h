@@ -81,6 +81,10 @@ typedef enum {
                                 pairs level by level (an odd one out moves up unchanged), FP32 partials in scratch,
                                 one rounding at the root into rank 0's buffer, then a binomial tree of copies to
                                 every rank. Dependency depth 2*ceil(log2 R). */
+    HCCL_ALGO_AUTO = 6       /* AllReduce only: the planner picks between the paper's two forms by size (the
+                                algorithm, and with it the cost of generating the packet, changes with the size,
+                                Sec. V-B): ONESHOT while R times the bytes per rank is at most 32 MiB (every rank
+                                reads R buffers: the work grows with R squared), RING beyond. */
 } hccl_algo_t;
 
 /* Which data mover the executor uses for aligned bulk work. AUTO: the planner decides: the bulk engine for

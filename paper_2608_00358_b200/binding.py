@@ -15,7 +15,7 @@ from . import _build
 OK, ERR_INVALID_ARG, ERR_DTYPE, ERR_COUNT_MISMATCH, ERR_OVERLAP, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_BUSY, \
     ERR_CUDA, ERR_TIMEOUT, ERR_BAD_DESCRIPTOR, ERR_NOT_BOUND, ERR_HAZARD = range(13)
 FP32, BF16, FP16 = 0, 1, 2
-ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED, ALGO_RING_2LEVEL, ALGO_FANOUT, ALGO_TREE = 0, 1, 2, 3, 4, 5
+ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED, ALGO_RING_2LEVEL, ALGO_FANOUT, ALGO_TREE, ALGO_AUTO = 0, 1, 2, 3, 4, 5, 6
 ENGINE_AUTO, ENGINE_LSU, ENGINE_BULK = 0, 1, 2
 FLAG_LEVEL_MAJOR, FLAG_CHECK_HAZARDS, FLAG_STAGED_RING, FLAG_BIDIRECTIONAL = 1, 2, 4, 8
 FLAG_STATIC_CHAINS, FLAG_DYNAMIC_TICKETS = 16, 32

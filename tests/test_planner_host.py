@@ -440,3 +440,14 @@ def test_two_level_allgather_runs_as_groups_by_default():
         Y = interpret(plan, X, 3)
         for r in range(8):
             assert np.array_equal(Y[r].view(np.uint16), want[r])
+
+
+def test_allreduce_auto_picks_by_size():
+    small = hb.hccl_plan_allreduce(8, 1 << 19, hb.BF16, hb.ALGO_AUTO).info()       # 8 x 1 MiB: one-shot
+    assert small.chain_depth == 1 and small.schedule_bytes == hb.hccl_plan_allreduce(8, 1 << 19, hb.BF16, hb.ALGO_ONESHOT).info().schedule_bytes
+    large = hb.hccl_plan_allreduce(8, 1 << 23, hb.BF16, hb.ALGO_AUTO).info()       # 8 x 16 MiB: ring
+    assert large.chain_depth == 14 and large.schedule_bytes == hb.hccl_plan_allreduce(8, 1 << 23, hb.BF16, hb.ALGO_RING).info().schedule_bytes
+    assert hb.hccl_plan_allreduce(64, 1 << 19, hb.BF16, hb.ALGO_AUTO).info().chain_depth == 126   # 64 x 1 MiB: ring
+    for fn in (hb.hccl_plan_reducescatter, hb.hccl_plan_allgather):
+        with pytest.raises(hb.HcclError):
+            fn(4, None, 1024, hb.BF16, hb.ALGO_AUTO)
