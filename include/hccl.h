@@ -76,7 +76,7 @@ typedef enum {
                                 AllGather: one read of the chunk) and written into all R receive buffers by the
                                 same work item. Possible only because the virtual ranks share one memory; not in
                                 the paper. Reported as its own algorithm, never as "one-shot". */
-    HCCL_ALGO_TREE = 5       /* AllReduce by a binary tree of two-input sums (tree-based NMC reduction, Sec.
+    HCCL_ALGO_TREE = 5,      /* AllReduce by a binary tree of two-input sums (tree-based NMC reduction, Sec.
                                 III-B.2): per granule of opts.chunk_bytes, neighbours in rank order are added in
                                 pairs level by level (an odd one out moves up unchanged), FP32 partials in scratch,
                                 one rounding at the root into rank 0's buffer, then a binomial tree of copies to
