@@ -1,0 +1,77 @@
+"""Seeded random configurations of the AllReduce / AllGather planners and executor options against the
+schedule-ordered oracles: rank counts, sizes, element types, algorithms, engines, block counts, dispatch modes."""
+import numpy as np
+import pytest
+
+from gpu_helpers import run_plan
+from helpers import np_dtype
+from oracle import oracle as orc
+from paper_2608_00358_b200 import binding as hb
+from paper_2608_00358_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _options(rng):
+    o = dict(sm_budget=int(rng.choice([1, 2, 5, 16, 148])), engine=int(rng.choice([0, hb.ENGINE_LSU, hb.ENGINE_BULK])))
+    if rng.random() < 0.5:
+        o["tile_bytes"] = int(rng.choice([256, 1024, 4096, 49152]))
+    if rng.random() < 0.5:
+        o["chunk_bytes"] = int(rng.choice([512, 4096, 65536]))
+    if rng.random() < 0.3:
+        o["chain_group"] = int(rng.choice([1, 2, 7]))
+    if rng.random() < 0.3:
+        o["flags"] = int(rng.choice([hb.FLAG_DYNAMIC_TICKETS, hb.FLAG_STATIC_CHAINS, hb.FLAG_LEVEL_MAJOR]))
+    if o["engine"] != hb.ENGINE_BULK and rng.random() < 0.2:
+        o.update(light=1, threads=int(rng.choice([128, 256, 512])))
+    return o
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_allreduce(seed):
+    rng = np.random.default_rng(1000 + seed)
+    R = int(rng.integers(2, 13))
+    n = int(rng.choice([1, R - 1, R, R + 1, 255, 4097, int(rng.integers(1, 60000))]))
+    dt = int(rng.choice([hb.FP32, hb.BF16, hb.FP16]))
+    algos = [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_RING_FUSED, hb.ALGO_TREE, hb.ALGO_FANOUT, hb.ALGO_AUTO]
+    o = _options(rng)
+    racks = [L for L in (2, 3, 4) if R % L == 0 and R // L >= 2]
+    if racks:
+        algos.append(hb.ALGO_RING_2LEVEL)
+        o["rack_size"] = int(rng.choice(racks))
+    algo = int(rng.choice(algos))
+    X = synth.normal_ranks(R, n, dt, seed=seed)
+    p = hb.hccl_plan_allreduce(R, n, dt, algo, o)
+    Y = run_plan(p, X, iters=2, misalign=int(rng.choice([0, 0, 4, 8])) if dt == hb.FP32 else int(rng.choice([0, 0, 2, 6])))
+    if algo in (hb.ALGO_ONESHOT, hb.ALGO_FANOUT, hb.ALGO_AUTO):
+        want = orc.allreduce_oneshot_f32(dt, X)
+    elif algo == hb.ALGO_TREE:
+        want = orc.allreduce_tree_f32(dt, X)
+    elif algo == hb.ALGO_RING_2LEVEL:
+        L = o["rack_size"]
+        want = orc.allreduce_ring2_f32(dt, X, R // L, L)
+    else:
+        want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8)), (seed, R, n, dt, algo, o, r)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_allgather(seed):
+    rng = np.random.default_rng(2000 + seed)
+    R = int(rng.integers(1, 13))
+    counts = [int(c) for c in rng.integers(0, 3000, size=R)]
+    dt = int(rng.choice([hb.FP32, hb.BF16]))
+    algos = [hb.ALGO_RING, hb.ALGO_ONESHOT, hb.ALGO_FANOUT]
+    o = _options(rng)
+    racks = [L for L in (2, 3, 4) if R % L == 0 and R // L >= 2]
+    if racks:
+        algos.append(hb.ALGO_RING_2LEVEL)
+        o["rack_size"] = int(rng.choice(racks))
+    algo = int(rng.choice(algos))
+    X = [rng.integers(0, 2 ** 16, size=c * (2 if dt == hb.FP32 else 1), dtype=np.uint16) for c in counts]
+    p = hb.hccl_plan_allgather(R, counts, 0, dt, algo, o)
+    Y = run_plan(p, [x if x.size else np.zeros(8, np.uint16) for x in X], iters=2)
+    want = np.concatenate(X) if sum(counts) else np.zeros(0, np.uint16)
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np.uint16), want), (seed, R, counts, algo, o, r)
