@@ -75,3 +75,28 @@ def test_random_allgather(seed):
     want = np.concatenate(X) if sum(counts) else np.zeros(0, np.uint16)
     for r in range(R):
         assert np.array_equal(Y[r].view(np.uint16), want), (seed, R, counts, algo, o, r)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_reducescatter(seed):
+    rng = np.random.default_rng(3000 + seed)
+    R = int(rng.integers(1, 13))
+    counts = [int(c) for c in rng.integers(0, 5000, size=R)]
+    if rng.random() < 0.3:
+        counts[int(rng.integers(0, R))] = 0
+    n = sum(counts)
+    dt = int(rng.choice([hb.FP32, hb.BF16, hb.FP16]))
+    algo = int(rng.choice([hb.ALGO_RING, hb.ALGO_RING_FUSED, hb.ALGO_ONESHOT]))
+    o = _options(rng)
+    X = synth.normal_ranks(R, max(n, 1), dt, seed=seed)
+    X = [x[:n] if n else x[:0] for x in X]
+    p = hb.hccl_plan_reducescatter(R, counts, n, dt, algo, o)
+    Y = run_plan(p, [x if x.size else np.zeros(8, np_dtype(dt)) for x in X], iters=2)
+    offs = np.concatenate([[0], np.cumsum(counts)])
+    if algo == hb.ALGO_ONESHOT:
+        whole = orc.allreduce_oneshot_f32(dt, X)[0] if n else np.zeros(0, np_dtype(dt))
+        want = [whole[offs[r]:offs[r + 1]] for r in range(R)]
+    else:
+        want = orc.reducescatter_ring_f32(dt, X, np.array(counts, dtype=np.int64))
+    for r in range(R):
+        assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8)), (seed, R, counts, dt, algo, o, r)
