@@ -120,13 +120,18 @@ typedef enum {
 
 /* Options. A zero field means "default". */
 typedef struct {
-    int32_t sm_budget;      /* thread blocks of the persistent executor = "message engines" (default 148) */
+    int32_t sm_budget;      /* thread blocks of the persistent executor = "message engines" (default 148). An upper
+                               bound: a plan never launches more blocks than it has work items or static chains,
+                               and a ring planner left to the default may launch exactly one block per tile of a
+                               ring step. hccl_plan_info reports the number used. */
     int32_t engine;         /* hccl_engine_t */
     uint64_t chunk_bytes;   /* ring pipelining granule inside a shard/chunk, in bytes of the data type (default 2 MiB) */
     uint64_t tile_bytes;    /* work-item size, bytes of the widest operand (default: chosen from size and sm_budget) */
     uint64_t timeout_ns;    /* bound on every device-side wait (default 2e9) */
     uint32_t flags;         /* HCCL_FLAG_* */
-    int32_t chain_group;    /* chains scheduled together in chain-group-major order (default 16) */
+    int32_t chain_group;    /* chains scheduled together in chain-group-major order; FP32 scratch slots are recycled
+                               every two groups. Default: all chains together (a slot per chain, no recycling) while
+                               the FP32 partials take at most 32 MiB (AllReduce rings: 128 MiB), else 16 */
     int32_t threads;        /* threads per block, multiple of 32 (default 512) */
     int32_t stages;         /* bulk engine: shared-memory stages of 48 KiB per block, 2..4 (default 4) */
     int32_t cluster;        /* register engine: launch blocks in clusters of this size (2, 4, 8) so that they sit on
