@@ -451,3 +451,29 @@ def test_allreduce_auto_picks_by_size():
     for fn in (hb.hccl_plan_reducescatter, hb.hccl_plan_allgather):
         with pytest.raises(hb.HcclError):
             fn(4, None, 1024, hb.BF16, hb.ALGO_AUTO)
+
+
+def test_header_is_plain_c_and_links_against_the_library(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 and a C program must link and run against the
+    library (host-only calls: no GPU needed)."""
+    import os
+    import subprocess
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "use_hccl.c"
+    src.write_text(
+        '#include <stdio.h>\n#include "hccl.h"\n'
+        "int main(void) {\n"
+        "    hccl_plan_t* p = NULL;\n"
+        "    hccl_plan_info_t info;\n"
+        "    if (hccl_plan_allreduce(4, 1 << 20, HCCL_FP32, HCCL_ALGO_RING, NULL, &p) != HCCL_OK) return 1;\n"
+        "    if (hccl_plan_info(p, &info) != HCCL_OK) return 2;\n"
+        '    printf("%lld %lld %s\\n", (long long)info.n_wqe, (long long)info.schedule_bytes, hccl_status_string(HCCL_ERR_TIMEOUT));\n'
+        "    hccl_plan_destroy(p);\n"
+        "    return hccl_plan_allreduce(0, 1, HCCL_FP32, HCCL_ALGO_RING, NULL, &p) == HCCL_ERR_INVALID_ARG ? 0 : 3;\n"
+        "}\n")
+    exe = tmp_path / "use_hccl"
+    libdir = os.path.dirname(hb.LIBRARY_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(root, "include"), str(src),
+                           "-o", str(exe), "-L", libdir, "-l:" + os.path.basename(hb.LIBRARY_PATH), "-Wl,-rpath," + libdir])
+    out = subprocess.check_output([str(exe)]).decode().split()
+    assert out[0] == "24" and out[1] == str(60 << 20) and "timed" in " ".join(out[2:])
