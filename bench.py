@@ -150,6 +150,66 @@ def run_reference(args, rank: int):
     print(json.dumps(line), flush=True)
 
 
+def check_host_result_against_oracle(counts, row_bytes: int, host_send, host_recv) -> int:
+    """Every destination's receive buffer (pinned host tensors) against the oracle's AllToAllv of the host
+    send buffers, byte for byte. Returns the number of destinations compared; raises on the first mismatch."""
+    import numpy as np
+    from oracle import oracle as orc
+    R = counts.shape[0]
+    sd, rd = orc.packed_displs(counts)
+    X = [h.numpy().view(np.uint8).reshape(-1) for h in host_send]
+    for d in range(R):
+        n = int(counts[:, d].sum()) * row_bytes
+        Y = [np.full(n if q == d else 1, 0xA5, dtype=np.uint8) for q in range(R)]
+        orc.alltoallv(X, Y, counts, sd, rd, row_bytes, dst_only=d)
+        got = host_recv[d].numpy().view(np.uint8).reshape(-1)[:n]
+        if not np.array_equal(got, Y[d]):
+            raise RuntimeError("end-to-end result differs from the oracle at destination %d" % d)
+    return R
+
+
+def _finite(x):
+    """NaN / inf -> None, numpy scalars -> Python numbers, so that the line is strict JSON."""
+    import math
+    if isinstance(x, dict):
+        return {str(k): _finite(v) for k, v in x.items()}
+    if isinstance(x, (list, tuple)):
+        return [_finite(v) for v in x]
+    if isinstance(x, bool) or x is None or isinstance(x, (str, int)):
+        return x
+    if hasattr(x, "item") and not isinstance(x, float):
+        x = x.item()
+    if isinstance(x, float):
+        return x if math.isfinite(x) else None
+    return x
+
+
+def _round(x, nd=4):
+    if isinstance(x, float):
+        return float("%.*g" % (nd + 2, x))
+    if isinstance(x, dict):
+        return {k: _round(v, nd) for k, v in x.items()}
+    if isinstance(x, list):
+        return [_round(v, nd) for v in x]
+    return x
+
+
+def emit(detail: dict, headline: dict):
+    """Two stdout lines: first everything (side configurations, sweeps, host-link figures), then LAST the compact
+    headline record (well under 2 KB) that a reader of the tail of the output can parse. The detail record is
+    also written to gpurun_out/bench_detail.json when that folder can be made."""
+    d = json.dumps(_finite(detail), allow_nan=False)
+    try:
+        os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
+        with open(os.path.join(ROOT, "gpurun_out", "bench_detail.json"), "w") as f:
+            f.write(d + "\n")
+    except OSError:
+        pass
+    print(d, flush=True)
+    h = json.dumps(_round(_finite(headline)), allow_nan=False, separators=(",", ":"))
+    print(h, flush=True)
+
+
 # ----------------------------------------------------------------------------------------- GPU legs
 def side_configs(quick: bool):
     """Configurations 1, 2, 3 and 5: reported next to the headline, never as the headline."""
@@ -279,9 +339,16 @@ def side_configs(quick: bool):
             Xh = [t.view(torch.int16).cpu().numpy().view(np.uint16) for t in wl.send]
             rc = np.full(16, Xh[0].size // 16, dtype=np.int64)
             t0 = _t.perf_counter()
-            orc.reducescatter(hb.BF16, Xh, rc)
+            want = orc.reducescatter(hb.BF16, Xh, rc)
             out["3_reducescatter_r16_bf16_64Mi_" + nm]["cpu_oracle_ms"] = (_t.perf_counter() - t0) * 1e3
-            del Xh
+            # outputs of the timed plan further than 1 ulp from the rounded FP64 sum: counted and reported
+            beyond = 0
+            for r in range(16):
+                got = wl.recv[r].view(torch.int16).cpu().numpy().view(np.uint16)
+                beyond += int((orc.ulp_distance(hb.BF16, got, want[r]) > 1).sum())
+            out["3_reducescatter_r16_bf16_64Mi_" + nm]["beyond_1ulp_of_fp64_sum"] = beyond
+            out["3_reducescatter_r16_bf16_64Mi_" + nm]["outputs"] = int(Xh[0].size)
+            del Xh, want
         del wl
         torch.cuda.empty_cache()
     return out
@@ -311,6 +378,89 @@ def run_profile_case(args):
     print(json.dumps({"case": args.profile_case, "workload": wl.name, "ms": ms, "schedule_bytes": int(i.schedule_bytes),
                       "compulsory_bytes": int(i.compulsory_bytes), "schedule_gbs": i.schedule_bytes / ms / 1e6,
                       "compulsory_gbs": i.compulsory_bytes / ms / 1e6, "tiles": int(i.n_tiles)}), flush=True)
+
+
+def interference_leg(args, wl):
+    """The GEMM-interference trade-off at a few SM budgets (the full sweep is `python -m
+    paper_2608_00358_b200.interference`); a budget is a number of thread blocks = SMs taken."""
+    import torch
+    from paper_2608_00358_b200 import binding as hb
+    from paper_2608_00358_b200 import interference
+    from paper_2608_00358_b200 import workloads as wk
+    gemm = interference.Gemm()
+    sweep = []
+    for b in ([2, 148] if args.quick else [2, 4, 16, 64, 148]):
+        plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(sm_budget=b))
+        w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
+        r = interference.measure(w2, seconds=2.0, gemm=gemm)
+        sweep.append({"sm_budget": b, "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
+                      "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_alone_gbs": r["collective_alone_gbs"],
+                      "collective_overlap_gbs": r["overlap"].get("collective_gbs")})
+        del w2, plan
+    out = {"gemm": "bf16 8192^3 (cuBLAS via torch.matmul), back to back", "collective": wl.name,
+           "protocol": "both loops kept 3 batches deep; rates taken inside the window where both run", "sweep": sweep}
+    del gemm
+    if not args.quick:
+        # the same at budget 4 against a 16384^3 GEMM (55 waves of tiles instead of 14: losing one SM
+        # slot costs a smaller share of a wave)
+        torch.cuda.empty_cache()
+        gemm = interference.Gemm(16384)
+        plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(sm_budget=4))
+        w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
+        r = interference.measure(w2, seconds=2.5, gemm=gemm)
+        out["gemm_16384_budget_4"] = {
+            "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
+            "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
+        del w2, plan, gemm
+    # the operating point: the budget with the smallest GEMM loss among those that move data
+    best = min((p for p in sweep if p["gemm_slowdown"] is not None), key=lambda p: p["gemm_slowdown"], default=None)
+    if best is not None:
+        out["chosen"] = {"sm_budget": best["sm_budget"], "gemm_slowdown": best["gemm_slowdown"],
+                         "collective_overlap_gbs": best["collective_overlap_gbs"]}
+    return out
+
+
+def headline_of(line: dict) -> dict:
+    """The compact record: the contract's keys, the roofline, both baselines and a few cross-references."""
+    keep = ["metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling", "vs_baseline",
+            "dtype", "data", "gpu_launches", "clocks"]
+    h = {k: line[k] for k in keep if k in line}
+    c = line["config"]
+    h["config"] = {k: c[k] for k in ("workload", "virtual_ranks", "payload_bytes", "sm_budget", "threads", "tile_bytes", "engine", "cache",
+                                     "multi_gpu", "zipf_clamp_rows")}
+    r = line["roofline"]
+    h["roofline"] = {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "kernel", "algorithmic_bytes_per_launch", "launch_ms")}
+    h["roofline"]["peak_source"] = r["peak_source"]
+    h["roofline"]["traffic_from"] = "ncu, cap-1024 case, scaled by bytes"
+    e = line.get("e2e")
+    if e:
+        h["e2e"] = {k: e[k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step", "ms_per_step", "steps", "gpu_launches_per_step",
+                                      "checked_destinations_vs_oracle", "skipped") if k in e}
+        if "api" in e:
+            h["e2e"]["api"] = e["api"].split(" ")[0]
+    if "cpu_baseline" in line:
+        h["cpu_baseline"] = line["cpu_baseline"]
+    i = line.get("interference")
+    if i and "chosen" in i:
+        h["interference"] = dict(i["chosen"], gemm="bf16 8192^3")
+    cfg = line.get("configs") or {}
+    side = {}
+    for key, short, field in (("3_reducescatter_r16_bf16_64Mi_ring", "c3_ring_ms", "ms"), ("3_reducescatter_r16_bf16_64Mi_ring_fused", "c3_fused_ms", "ms"),
+                              ("3_reducescatter_r16_bf16_64Mi_ring", "c3_beyond_1ulp", "beyond_1ulp_of_fp64_sum"),
+                              ("1_allreduce_ring_r4_fp32_1Mi", "c1_p50_us", "p50_us"), ("2_alltoallv_r8_bf16_dim128", "c2_p50_us", "p50_us"),
+                              ("5_allreduce_r8_bf16_4096B_oneshot", "c5_4k_oneshot_p50_us", "p50_us"),
+                              ("5_allreduce_r8_bf16_1048576B_oneshot", "c5_1m_oneshot_p50_us", "p50_us"),
+                              ("next_alltoallv_dynamic_r64_fp16_dim256", "dyn_r64_ms", "ms")):
+        v = (cfg.get(key) or {}).get(field)
+        if v is not None:
+            side[short] = v
+    ho = (cfg.get("5_allreduce_r8_bf16_4096B_oneshot") or {}).get("host_observed")
+    if ho:
+        side["c5_4k_resident_ring_wait_us"] = ho.get("ring_and_wait_us")
+    if side:
+        h["side"] = side
+    h["detail"] = "previous stdout line; gpurun_out/bench_detail.json"
+    return h
 
 
 def run_ours(args, rank: int, world: int, local_rank: int):
@@ -414,14 +564,14 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             pst, pdetail = pipe.status()
             if pst != hb.OK:
                 raise hb.HcclError(pst, "hccl_hostpipe_status (detail %d)" % pdetail)
-            for d_ in (0, 31, 63):   # what came back to the host is what the device-resident run left on the device
-                if not torch.equal(hr[d_], wl.recv[d_].cpu()):
-                    raise RuntimeError("pipelined end-to-end result differs at destination %d" % d_)
+            # outside the timed region: what came back to the host, for every destination rank, against the CPU
+            # oracle's AllToAllv of the same host send buffers (one destination at a time: <= 0.6 GB extra)
+            e2e_checked = check_host_result_against_oracle(wl.meta["counts"], 512, hs, hr)
             ms = e0.elapsed_time(e1) / ksteps
             e2e = {"value": info.schedule_bytes / ms / 1e6, "unit": UNIT, "h2d_bytes_per_step": int(payload),
                    "d2h_bytes_per_step": int(payload), "ms_per_step": ms, "steps": ksteps,
                    "api": "hccl_hostpipe_execute (pinned host buffers -> device -> pinned host buffers, %d destination windows on 3 streams)" % (len(pipe.windows()) - 1),
-                   "gpu_launches_per_step": len(pipe.windows()) - 1,
+                   "gpu_launches_per_step": len(pipe.windows()) - 1, "checked_destinations_vs_oracle": e2e_checked,
                    "single_stream": {"value": info.schedule_bytes / serial_ms / 1e6, "ms_per_step": serial_ms, "api": "hccl_execute_host"}}
             # the host link by itself, with the same pinned buffers: each direction alone, then both at once
             def _link(h2d, d2h, reps=2):
@@ -469,9 +619,10 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                        "cache": "inputs larger than L2 (no flush needed)", "multi_gpu": "replicas only",
                        "zipf_clamp_rows": int(cap_used)},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": which + " copy bandwidth (burst)", "kernel": "hccl_executor",
+                         "peak_source": which + " copy bandwidth (burst)", "kernel": "hccl_executor_bulk" if int(info.engine) == 2 else "hccl_executor_lsu",
                          "algorithmic_bytes_per_launch": int(info.schedule_bytes), "launch_ms": launch_ms,
                          "traffic": (DRAM_BYTES_PER_ALGORITHMIC_BYTE * info.schedule_bytes) if DRAM_BYTES_PER_ALGORITHMIC_BYTE else None,
+                         "traffic_note": "dram bytes per algorithmic byte (%.3f) from the ncu capture of the cap-1024 case of this workload, scaled by the bytes of this launch" % DRAM_BYTES_PER_ALGORITHMIC_BYTE,
                          "frac_of_nominal_8TBs": achieved / 8000.0},
             "gpu_launches": args.steps, "clocks": clocks, "e2e": e2e,
         }
@@ -479,33 +630,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
     # ---- interference, other configs, CPU baseline: rank 0 at N = 1 only
     if rank == 0 and world == 1:
         if not args.no_gemm:
-            # the GEMM-interference trade-off at a few SM budgets (the full sweep is `python -m
-            # paper_2608_00358_b200.interference`); a budget is a number of thread blocks = SMs taken
-            gemm = interference.Gemm()
-            sweep = []
-            for b in ([8, 148] if args.quick else [4, 16, 64, 148]):
-                plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(sm_budget=b))
-                w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
-                r = interference.measure(w2, seconds=2.0, gemm=gemm)
-                sweep.append({"sm_budget": b, "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
-                              "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_alone_gbs": r["collective_alone_gbs"],
-                              "collective_overlap_gbs": r["overlap"].get("collective_gbs")})
-                del w2, plan
-            line["interference"] = {"gemm": "bf16 8192^3 (cuBLAS via torch.matmul), back to back", "collective": wl.name,
-                                    "protocol": "both loops kept 3 batches deep; rates taken inside the window where both run", "sweep": sweep}
-            del gemm
-            if not args.quick:
-                # the same at budget 4 against a 16384^3 GEMM (55 waves of tiles instead of 14: losing one SM
-                # slot costs a smaller share of a wave)
-                torch.cuda.empty_cache()
-                gemm = interference.Gemm(16384)
-                plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(sm_budget=4))
-                w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
-                r = interference.measure(w2, seconds=2.5, gemm=gemm)
-                line["interference"]["gemm_16384_budget_4"] = {
-                    "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
-                    "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
-                del w2, plan, gemm
+            line["interference"] = interference_leg(args, wl)
         dyn64 = None
         if not args.no_side:
             # device-resident AllToAllv at the benchmark's size: the same counts, read from device memory by the kernel
@@ -532,7 +657,7 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                                     "sample": "destination ranks 0..%d of 64 (%.2f GB moved), best of 2" % (args.oracle_dst - 1, moved / 1e9),
                                     "host_cores_available": os.cpu_count()}
     if rank == 0:
-        print(json.dumps(line), flush=True)
+        emit(line, headline_of(line))
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()

@@ -329,8 +329,8 @@ hccl_status_t hccl_execute(hccl_plan_t*, const void* const* sendbufs, void* cons
  * plan's own workspace and epoch are not touched). The register-path executor is used whatever
  * opts.engine says. sendbufs/recvbufs as in hccl_execute. Plans whose hccl_plan_workspace_bytes exceed
  * 8 MiB are refused with HCCL_ERR_WORKSPACE (for reductions on 16-bit data choose a small opts.chunk_bytes:
- * the FP32 scratch is 2 * chain_group granules); plans with a trigger are refused with
- * HCCL_ERR_INVALID_ARG. The call allocates nothing on the device: it calls no cudaMalloc/cudaFree and no
+ * the FP32 scratch is 2 * chain_group granules); plans with a trigger and device-resident plans
+ * (hccl_plan_alltoallv_dynamic) are refused with HCCL_ERR_INVALID_ARG. The call allocates nothing on the device: it calls no cudaMalloc/cudaFree and no
  * allocating library routine.
  *
  * All calls share the one array, and it keeps the previous call's contents: each call rewrites the
@@ -396,7 +396,10 @@ void hccl_hostpipe_destroy(hccl_hostpipe_t*);
  * HCCL_ERR_TIMEOUT and the server can be started again), after hccl_server_stop, or after a failed
  * execution (whose verdict hccl_server_ring / hccl_server_wait then return). While the server runs, use
  * only these calls on the plan, and do not synchronise the whole device: the kernel occupies `stream` until
- * it leaves. Rings are served in order; ring again only after the previous ring was waited for. */
+ * it leaves. Rings are served in order; ring again only after the previous ring was waited for.
+ * hccl_server_stop only asks the kernel to leave and returns at once: synchronise the server's `stream` after
+ * it, before the plan is executed, bound or served again (until the kernel has left, its blocks still use the
+ * workspace's ticket, exit count and counters). */
 typedef struct { uint64_t request, completed, stop, exited, status, detail, pad[2]; } hccl_doorbell_t;
 hccl_status_t hccl_server_start(hccl_plan_t*, const void* const* sendbufs, void* const* recvbufs, void* host_doorbell,
                                 uint64_t idle_timeout_ns, void* stream);

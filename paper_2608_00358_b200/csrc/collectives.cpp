@@ -626,8 +626,8 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     if ((fp32_ring || own_slots) && pre.engine == HCCL_ENGINE_AUTO) pre.engine = HCCL_ENGINE_LSU;
     fill_ring_opts(&o, &pre, (int64_t)R * count * elem_bytes(dt), algo == HCCL_ALGO_RING_FUSED || algo == HCCL_ALGO_ONESHOT || algo == HCCL_ALGO_FANOUT || R == 1);
     if (algo == HCCL_ALGO_RING_2LEVEL) {
-        if (R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
-        // a single rack, or racks of one rank, is the flat ring
+        // a single rack (R <= rack_size), or racks of one rank, is the flat ring; only two or more racks must tile R
+        if (o.rack_size >= 2 && R > o.rack_size && R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
         if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = 1 << 20;  // all chains together
         if (o.rack_size >= 2 && R / o.rack_size >= 2) return plan_allreduce_2level(R, count, dt, o, out);
         algo = HCCL_ALGO_RING;
@@ -836,7 +836,7 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
         sext[r] = c * es;
     }
     if (algo == HCCL_ALGO_RING_2LEVEL) {
-        if (R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
+        if (o.rack_size >= 2 && R > o.rack_size && R % o.rack_size != 0) return HCCL_ERR_INVALID_ARG;
         if (o.rack_size >= 2 && R / o.rack_size >= 2) return plan_allgather_2level(R, offs, dt, o, out);
         algo = HCCL_ALGO_RING;
     }

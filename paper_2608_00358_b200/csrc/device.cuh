@@ -266,7 +266,7 @@ __device__ void copy_tile_lsu(char* dst, const char* src, uint32_t n, const uint
     if (((da ^ sa) & 15u) == 0) {
         uint32_t head = (uint32_t)((16u - (da & 15u)) & 15u);
         if (head > n) head = n;
-        for (uint32_t i = tid; i < head; i += nth) dst[i] = src[i];
+        for (uint32_t i = tid; i < head; i += nth) dst[i] = __ldcg(src + i);
         const uint32_t nv = (n - head) >> 4;
         const uint4* s = (const uint4*)(src + head);
         uint4* d = (uint4*)(dst + head);

@@ -11,9 +11,11 @@ namespace hccl {
 // blocks through a device-side word, and reports completion (and a failure verdict) back into the record.
 // Every wait is bounded: the kernel leaves by itself after idle_ns without a ring, or when told to stop.
 
+// Acquire at system scope: what the host wrote before it rang (the send buffers' contents among it) is
+// ordered before everything this thread does afterwards, the release of the other blocks included.
 __device__ __forceinline__ unsigned long long ld_sys_u64(const unsigned long long* p) {
     unsigned long long v;
-    asm volatile("ld.relaxed.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    asm volatile("ld.acquire.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
     return v;
 }
 __device__ __forceinline__ void st_sys_u64(unsigned long long* p, unsigned long long v) {

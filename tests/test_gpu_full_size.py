@@ -1,7 +1,7 @@
 """Parity at the full benchmark sizes, in the launch configuration bench.py times (default options).
 
-Config 4 (51.6 GB resident) is checked on sampled (source, destination) segments that the oracle computes
-one by one, plus properties that hold at any size; config 3 (2 GiB of input) is small enough for the oracle
+Config 4 (51.6 GB resident) is checked on every byte of every destination, one destination at a time (the
+oracle's per-destination mode), and on sampled segments with host-regenerated rows; config 3 (2 GiB of input) is small enough for the oracle
 to compute every output. Needs a GPU with ~60 GB free and ~8 GB of host memory."""
 import numpy as np
 import pytest
@@ -20,7 +20,7 @@ def _free_gb():
     return free / 2 ** 30
 
 
-def test_config4_full_size_sampled_segments_and_conservation():
+def test_config4_full_size_every_destination():
     if _free_gb() < 60:
         pytest.skip("needs 60 GB of free device memory")
     wl = wk.config4()                       # the plan bench.py times: default engine, budget and tiles
@@ -51,18 +51,29 @@ def test_config4_full_size_sampled_segments_and_conservation():
         lo, n = int(RD[d, s]) * rb, int(C[s, d]) * rb
         got = wl.recv[d].view(torch.uint8)[lo:lo + n].cpu().numpy()
         assert np.array_equal(got, Y[d][lo:lo + n]), "segment %d -> %d" % (s, d)
-    # --- properties at full size: every receive buffer is exactly full (packed), and for every destination
-    #     the sum of all received 16-bit words equals the sum of the words sent to it
-    for d in range(R):
-        assert wl.recv[d].numel() == int(C[:, d].sum()) * row
-    sd_t = torch.from_numpy(SD)
-    for d in range(0, R, 7):
-        want = 0
-        for s in range(R):
-            lo = int(sd_t[s, d]) * row
-            want += int(wl.send[s][lo:lo + int(C[s, d]) * row].to(torch.int64).sum())
-        assert int(wl.recv[d].to(torch.int64).sum()) == want, "destination %d" % d
     del X, Y
+    # --- every destination, every byte: for destination d the oracle gets, per source, exactly the rows bound
+    #     for d (copied from the device send buffers, whose contents are the seeded generator's: the sampled
+    #     segments above were regenerated on the host), the true counts and receive displacements, and a
+    #     sentinel-filled receive buffer of d's full size; the result must equal the device's receive buffer.
+    #     Send displacements into these per-destination slices are zero; the true ones are exercised above.
+    SD0 = np.zeros_like(SD)
+    one = np.zeros(1, dtype=np.uint8)
+    for d in range(R):
+        assert wl.recv[d].numel() == int(C[:, d].sum()) * row          # packed: the buffer is exactly full
+        Xd = []
+        for s in range(R):
+            lo, cnt = int(SD[s, d]) * row, int(C[s, d]) * row
+            Xd.append(wl.send[s][lo:lo + cnt].cpu().numpy().view(np.uint8) if cnt else one)
+        s0 = (7 * d + 3) % R                                           # one slice per destination: the host generator's rows
+        k0 = min(int(C[s0, d]), 512)
+        assert np.array_equal(Xd[s0][:k0 * rb], synth.hashed_rows_np(s0, int(SD[s0, d]), k0, row).reshape(-1).view(np.uint8))
+        nd = int(C[:, d].sum()) * rb
+        Yd =[np.full(nd if q == d else 1, 0xA5, dtype=np.uint8) for q in range(R)]
+        orc.alltoallv(Xd, Yd, C, SD0, RD, rb, dst_only=d)
+        got = wl.recv[d].cpu().numpy().view(np.uint8)
+        assert np.array_equal(got, Yd[d]), "destination %d" % d
+        del Xd, Yd, got
 
 
 def test_config3_full_size_every_output():
@@ -79,10 +90,13 @@ def test_config3_full_size_every_output():
             rc = np.full(R, n // R)
             want = orc.reducescatter(hb.BF16, X, rc)                 # FP64 definition, rounded once
             bitwise = orc.reducescatter_ring_f32(hb.BF16, X, rc)     # the ring's FP32 adds in ring order
-        # (1) identical bits to the ring's own arithmetic (FP32 adds in ring order, one rounding)
-        # (2) against the FP64 definition: within 1 ulp, except where cancellation makes the FP32 accumulation
-        #     error itself larger than the result's bf16 ulp; there the bound of FP32 recursive summation must
-        #     hold: |g - o| <= ulp_bf16(g)/2 + (R-1) * 2^-24 * sum_q |x_q|
+        # (1) identical bits to the ring's own arithmetic (FP32 adds in ring order, one rounding): the primary check
+        # (2) against the FP64 definition: outputs further than 1 ulp from the rounded FP64 sum are counted and
+        #     reported, not excused. The method adds in FP32 (Sec. II-A.2), so where 16 inputs cancel to a result
+        #     whose bf16 ulp is smaller than the FP32 accumulation error the literal 1-ulp rule cannot hold; at
+        #     this size and seed that is 1 output of 67 108 864. The cap below is absolute and leaves room for
+        #     a different seed of the device generator, no more; each such output must satisfy the bound of
+        #     FP32 recursive summation, |g - o| <= ulp_bf16(g)/2 + (R-1) * 2^-24 * sum_q |x_q|
         beyond = 0
         for r in range(R):
             got = wl.recv[r].view(torch.int16).cpu().numpy().view(np.uint16)
@@ -97,7 +111,7 @@ def test_config3_full_size_every_output():
                 half_ulp = np.maximum(np.abs(g), 2.0 ** -126) * 2.0 ** -8
                 bound = half_ulp + (R - 1) * 2.0 ** -24 * np.abs(xs).sum(axis=0)
                 assert np.all(np.abs(g - o) <= bound), "rank %d: outside the FP32 summation bound" % r
-        assert beyond <= 1e-3 * n, beyond
+        assert beyond <= 4, "outputs beyond 1 ulp of the FP64 sum: %d of %d" % (beyond, n)
         print("config 3 (%s): %d of %d outputs beyond 1 ulp of the FP64 sum, all within the FP32 summation bound"
               % ("ring" if algo == hb.ALGO_RING else "ring fused", beyond, n))
         del wl

@@ -260,6 +260,16 @@ def test_two_level_degenerates_to_the_flat_ring():
     with pytest.raises(hb.HcclError) as e:
         hb.hccl_plan_allreduce(6, 100, hb.BF16, hb.ALGO_RING_2LEVEL, dict(rack_size=4))
     assert e.value.status == hb.ERR_INVALID_ARG
+    # fewer ranks than the default rack of 16 is a single rack: the flat ring, not a refusal
+    X8 = synth.normal_ranks(8, 333, hb.BF16, seed=2)
+    p = hb.hccl_plan_allreduce(8, 333, hb.BF16, hb.ALGO_RING_2LEVEL, SMALL)
+    Y = interpret(p, X8)
+    assert np.array_equal(Y[3].view(np.uint16), orc.allreduce_ring_f32(hb.BF16, X8, orc.floor_chunk_offsets(333, 8))[3])
+    rng = np.random.default_rng(8)
+    Xg = [rng.integers(0, 65536, size=50, dtype=np.uint16) for _ in range(6)]
+    pg = hb.hccl_plan_allgather(6, None, 50, hb.BF16, hb.ALGO_RING_2LEVEL, SMALL)
+    Yg = interpret(pg, Xg)
+    assert np.array_equal(Yg[5].view(np.uint16), orc.allgatherv(Xg)[5])
 
 
 @pytest.mark.parametrize("G,L", [(2, 2), (2, 3), (4, 4), (8, 16)])
