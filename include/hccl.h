@@ -117,6 +117,8 @@ typedef enum {
                                       only; ignored when the packet has another shape. The planners ask for it
                                       themselves where it pays. */
 #define HCCL_FLAG_DYNAMIC_TICKETS 32u /* keep the planners from asking for HCCL_FLAG_STATIC_CHAINS */
+#define HCCL_FLAG_DEVICE_TABLES 64u /* hccl_plan_alltoallv_dynamic: build descriptors and tiles on the device and run
+                                      them on the ordinary executor (always so beyond 64 ranks) */
 
 /* Options. A zero field means "default". */
 typedef struct {
@@ -197,14 +199,19 @@ hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_
 /* Device-resident AllToAllv ("AllToAllvDynamic", Sec. IV-B.2): for exchanges whose per-peer sizes are
  * produced on the device (a routing kernel) and must not travel through the host. The plan fixes only
  * R, the row size and the CAPACITY of every buffer in rows (max_send_rows[s] for X_s, max_recv_rows[d] for
- * Y_d); R <= 64. Before hccl_execute, hccl_plan_set_dynamic_metadata names the DEVICE array of R*R int64
+ * Y_d); R <= HCCL_MAX_RANKS. Up to 64 ranks one kernel holds the whole count matrix in shared memory and
+ * moves the rows itself. Beyond 64 ranks, or with HCCL_FLAG_DEVICE_TABLES, an execution is two launches: a small
+ * kernel (one block per source rank) writes the R*R descriptors and their tiles into the bound workspace
+ * -- the work requests are patched on the device, as the paper puts it -- and the ordinary executor
+ * (opts.engine, default the bulk engine) runs them; the workspace is sized for the capacities. Before hccl_execute, hccl_plan_set_dynamic_metadata names the DEVICE array of R*R int64
  * counts (counts[s*R+d] rows from s to d) that the kernel reads when it runs, and optionally two DEVICE
  * arrays [d*R+s] that receive each destination's counts and displacements for the consumer of the result.
  * Layout is packed on both sides (exclusive prefix sums, computed in the kernel with warp scans). The
  * counts may change between executions of the same bound plan; combined with hccl_plan_set_trigger the
  * collective can be enqueued before the counts exist and is released by the producer's signal
  * (Sec. IV-B.3). If a count is negative, a source's rows exceed max_send_rows or a destination's rows
- * exceed max_recv_rows, nothing is written and hccl_plan_status reports HCCL_ERR_BAD_DESCRIPTOR. */
+ * exceed max_recv_rows, no byte of a receive buffer is written and hccl_plan_status reports
+ * HCCL_ERR_BAD_DESCRIPTOR (the two optional output arrays are then unspecified). */
 hccl_status_t hccl_plan_alltoallv_dynamic(int R, const int64_t* max_send_rows, const int64_t* max_recv_rows,
                                           hccl_dtype_t dt, int64_t row_elems, const hccl_opts_t* opts,
                                           hccl_plan_t** out);
@@ -265,6 +272,11 @@ typedef struct {
 /* Cache hints on data WQEs. READ_ONCE: no source byte of this WQE is read by any other WQE of the packet
  * (it is streamed through the L2 with an evict-first policy). */
 #define HCCL_HINT_READ_ONCE 1
+/* LAST_READ_A (REDUCE whose operand A is in scratch): after this WQE nothing reads A's bytes again before they are
+ * rewritten, so the executor may tell the L2 to drop those lines instead of writing them back to memory (the
+ * cache-partition idea of Sec. II-A.3: temporary communication buffers should not cost the application).
+ * Honoured by the bulk engine; a hint only. */
+#define HCCL_HINT_LAST_READ_A 2
 
 typedef enum { HCCL_CMP_EQ = 0, HCCL_CMP_NE = 1, HCCL_CMP_GE = 2, HCCL_CMP_GT = 3, HCCL_CMP_LE = 4, HCCL_CMP_LT = 5 } hccl_cmp_t;
 

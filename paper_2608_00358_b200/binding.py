@@ -18,12 +18,12 @@ FP32, BF16, FP16 = 0, 1, 2
 ALGO_RING, ALGO_ONESHOT, ALGO_RING_FUSED, ALGO_RING_2LEVEL, ALGO_FANOUT, ALGO_TREE, ALGO_AUTO = 0, 1, 2, 3, 4, 5, 6
 ENGINE_AUTO, ENGINE_LSU, ENGINE_BULK = 0, 1, 2
 FLAG_LEVEL_MAJOR, FLAG_CHECK_HAZARDS, FLAG_STAGED_RING, FLAG_BIDIRECTIONAL = 1, 2, 4, 8
-FLAG_STATIC_CHAINS, FLAG_DYNAMIC_TICKETS = 16, 32
+FLAG_STATIC_CHAINS, FLAG_DYNAMIC_TICKETS, FLAG_DEVICE_TABLES = 16, 32, 64
 OP_COPY, OP_REDUCE, OP_REDUCE_N, OP_WAIT, OP_SET, OP_NOOP = range(6)
 BUF_SEND, BUF_RECV, BUF_SCRATCH, BUF_SIGNAL, BUF_USER_SIGNAL = range(5)
 DEP_FENCE, DEP_SYNC, DEP_WQE_SYNC, DEP_RECV_SYNC, DEP_SEND_SYNC, DEP_ELEMENTWISE, DEP_ELEMENTWISE2 = 1, 2, 4, 8, 16, 32, 64
 CMP_EQ, CMP_NE, CMP_GE, CMP_GT, CMP_LE, CMP_LT = range(6)
-HINT_READ_ONCE = 1
+HINT_READ_ONCE, HINT_LAST_READ_A = 1, 2
 MAX_RANKS = 256
 NOALLOC_WORKSPACE_BYTES = 8 << 20
 ELEM_BYTES = {FP32: 4, BF16: 2, FP16: 2}

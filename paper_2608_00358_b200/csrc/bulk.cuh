@@ -55,6 +55,15 @@ __device__ __forceinline__ unsigned long long policy_evict_first() {
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
     return pol;
 }
+// Partials that a later ring step reads back should outlive the streamed inputs in the L2.
+__device__ __forceinline__ unsigned long long policy_evict_last() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// The data at [p, p + 128) will not be read again before it is rewritten: the L2 may drop the line instead of
+// writing it back (p 128-byte aligned).
+__device__ __forceinline__ void discard_line(const void* p) { asm volatile("discard.global.L2 [%0], 128;" ::"l"(p) : "memory"); }
 __device__ __forceinline__ void bulk_load(uint32_t smem_dst, const void* gsrc, uint32_t bytes, uint32_t bar, bool hint, unsigned long long pol) {
     if (hint)
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
@@ -109,10 +118,14 @@ __device__ __forceinline__ void lds4(const char* p, float (&f)[4]) {
         }
     }
 }
-template <int DT>
-__device__ __forceinline__ void stg4(char* p, const float (&f)[4]) {
+// KEEP: the store carries an L2 cache-hint policy (FP32 partials only: they are what a next step reads back)
+template <int DT, bool KEEP = false>
+__device__ __forceinline__ void stg4(char* p, const float (&f)[4], unsigned long long pol = 0) {
     if constexpr (DT == HCCL_FP32) {
-        __stcg(reinterpret_cast<float4*>(p), make_float4(f[0], f[1], f[2], f[3]));
+        if constexpr (KEEP)
+            asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(p), "f"(f[0]), "f"(f[1]), "f"(f[2]), "f"(f[3]), "l"(pol) : "memory");
+        else
+            __stcg(reinterpret_cast<float4*>(p), make_float4(f[0], f[1], f[2], f[3]));
     } else {
         uint2 v;
         if constexpr (DT == HCCL_BF16) {
@@ -125,8 +138,8 @@ __device__ __forceinline__ void stg4(char* p, const float (&f)[4]) {
         __stcg(reinterpret_cast<uint2*>(p), v);
     }
 }
-template <int DA, int DB, int DD>
-__device__ __forceinline__ void reduce_piece(const char* sa, const char* sb, char* gdst, uint32_t n, uint32_t ctid, uint32_t cnth) {
+template <int DA, int DB, int DD, bool KEEP = false>
+__device__ __forceinline__ void reduce_piece(const char* sa, const char* sb, char* gdst, uint32_t n, uint32_t ctid, uint32_t cnth, unsigned long long pol = 0) {
     const uint32_t units = n >> 2;
     constexpr int U = 2;
     uint32_t u = ctid;
@@ -141,7 +154,7 @@ __device__ __forceinline__ void reduce_piece(const char* sa, const char* sb, cha
         for (int k = 0; k < U; ++k) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) a[k][e] = a[k][e] + b[k][e];
-            stg4<DD>(gdst + (size_t)(u + k * cnth) * 4 * Elem<DD>::BYTES, a[k]);
+            stg4<DD, KEEP>(gdst + (size_t)(u + k * cnth) * 4 * Elem<DD>::BYTES, a[k], pol);
         }
     }
     for (; u < units; u += cnth) {
@@ -150,12 +163,14 @@ __device__ __forceinline__ void reduce_piece(const char* sa, const char* sb, cha
         lds4<DB>(sb + (size_t)u * 4 * Elem<DB>::BYTES, b);
 #pragma unroll
         for (int e = 0; e < 4; ++e) a[e] = a[e] + b[e];
-        stg4<DD>(gdst + (size_t)u * 4 * Elem<DD>::BYTES, a);
+        stg4<DD, KEEP>(gdst + (size_t)u * 4 * Elem<DD>::BYTES, a, pol);
     }
 }
-static __device__ void reduce_piece_dispatch(int da, int db, int dd, const char* sa, const char* sb, char* g, uint32_t n, uint32_t ctid, uint32_t cnth) {
+static __device__ void reduce_piece_dispatch(int da, int db, int dd, const char* sa, const char* sb, char* g, uint32_t n, uint32_t ctid, uint32_t cnth,
+                                             bool keep, unsigned long long pol) {
 #define RP(A, B, D) reduce_piece<A, B, D>(sa, sb, g, n, ctid, cnth)
-#define RP_D(A, B) do { if (dd == HCCL_FP32) RP(A, B, HCCL_FP32); else if (dd == HCCL_BF16) RP(A, B, HCCL_BF16); else RP(A, B, HCCL_FP16); } while (0)
+#define RP_D(A, B) do { if (dd == HCCL_FP32) { if (keep) reduce_piece<A, B, HCCL_FP32, true>(sa, sb, g, n, ctid, cnth, pol); else RP(A, B, HCCL_FP32); } \
+                        else if (dd == HCCL_BF16) RP(A, B, HCCL_BF16); else RP(A, B, HCCL_FP16); } while (0)
 #define RP_B(A) do { if (db == HCCL_FP32) RP_D(A, HCCL_FP32); else if (db == HCCL_BF16) RP_D(A, HCCL_BF16); else RP_D(A, HCCL_FP16); } while (0)
     if (da == HCCL_FP32) RP_B(HCCL_FP32); else if (da == HCCL_BF16) RP_B(HCCL_BF16); else RP_B(HCCL_FP16);
 #undef RP_B
@@ -170,7 +185,8 @@ struct Dma {
     char* stages_ptr;
     PieceInfo* info;
     unsigned long long head, tail, groups;
-    unsigned long long pol;
+    unsigned long long pol;       // evict-first: streamed send data
+    unsigned long long pol_keep;  // evict-last: FP32 partials in scratch
     bool ok;
     bool copy_by_warps;
 };
@@ -263,6 +279,7 @@ static __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const
         trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
     }
     const Tile t = preloaded ? *preloaded : p.tiles[cur];
+    if (t.flags & TILE_FLAG_END) return false;  // behind the last item of a device-built table: no more work, no failure
     if (!tile_ok(p, t)) {
         fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
         return false;
@@ -378,8 +395,14 @@ static __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const
                 pi.signal[1] = t.signal[1];
                 pi.dt_a = ds.dt_a; pi.dt_b = ds.dt_b; pi.dt_d = ds.dt_dst;
                 pi.b_off = pe * ea;
+                // FP32 partials in scratch: kept in the L2 in preference to the streamed inputs (loads and stores carry
+                // an evict-last policy); after the step that reads a partial for the last time its lines are discarded
+                pi.keep_dst = (ds.kind_dst == HCCL_BUF_SCRATCH && ds.dt_dst == HCCL_FP32) ? 1 : 0;
+                pi.discard_src = (ds.cmp & HCCL_HINT_LAST_READ_A) && ds.kind_a == HCCL_BUF_SCRATCH ? a + (size_t)e0 * ea : nullptr;
+                pi.discard_bytes = ne * ea;
                 mbar_arrive_expect_tx(d.full + 8 * slot, ne * (ea + eb));
-                bulk_load(d.stages + slot * STAGE_BYTES, a + (size_t)e0 * ea, ne * ea, d.full + 8 * slot, ds.kind_a == HCCL_BUF_SEND, d.pol);
+                const bool a_keep = ds.kind_a == HCCL_BUF_SCRATCH;
+                bulk_load(d.stages + slot * STAGE_BYTES, a + (size_t)e0 * ea, ne * ea, d.full + 8 * slot, ds.kind_a == HCCL_BUF_SEND || a_keep, a_keep ? d.pol_keep : d.pol);
                 bulk_load(d.stages + slot * STAGE_BYTES + pe * ea, b + (size_t)e0 * eb, ne * eb, d.full + 8 * slot, ds.kind_b == HCCL_BUF_SEND, d.pol);
                 d.head = k + 1;
                 keep_lag(p, d);

@@ -28,6 +28,9 @@ struct alignas(16) PieceInfo {  // one per stage, in shared memory; written by t
     int32_t signal[2];
     uint8_t dt_a, dt_b, dt_d, evict_first;
     uint32_t b_off;       // REDUCE: byte offset of operand B inside the stage
+    uint32_t keep_dst;    // REDUCE: the result is an FP32 partial in scratch, stored with an evict-last L2 policy
+    uint32_t discard_bytes;   // REDUCE: ... and this many bytes from discard_src (operand A's global address, or null)
+    const char* discard_src;  //         were read for the last time: their L2 lines may be dropped
     uint16_t ndst, rank_dst;   // COPY with several destinations: receive buffers of ranks rank_dst .. +ndst-1 (mod R)
     unsigned long long dst_off;  // ... at this byte offset (dst is then the first of them)
     Tile tile;            // PIECE_TILE: the work item and its descriptor for the register path

@@ -104,6 +104,7 @@ hccl_status_t emit_ring(hccl_graph* g, int R, int dt, const std::vector<Chain>& 
                         w.a = first ? ref(HCCL_BUF_SEND, pr, ch.e0 * es) : ref(HCCL_BUF_SCRATCH, 0, slot);
                         w.dtype_dst = final ? dt : HCCL_FP32;
                         w.dst = final ? ref(HCCL_BUF_RECV, c, ch.out_off * es) : ref(HCCL_BUF_SCRATCH, 0, slot);
+                        if (final && !first && !staged) w.hints |= HCCL_HINT_LAST_READ_A;  // the chain's partial is dead after this step
                         if (first && !final && i >= (size_t)n_slots && last_reduce[i - n_slots] >= 0) {
                             // the slot is recycled: its previous user must have read it for the last time
                             w.dep_flags |= HCCL_DEP_WQE_SYNC;
@@ -1004,7 +1005,7 @@ extern "C" {
 
 hccl_status_t hccl_plan_alltoallv_dynamic(int R, const int64_t* max_send_rows, const int64_t* max_recv_rows, hccl_dtype_t dt,
                                           int64_t row_elems, const hccl_opts_t* opts, hccl_plan_t** out) {
-    if (!out || !max_send_rows || !max_recv_rows || R < 1 || R > 64 || row_elems < 1) return HCCL_ERR_INVALID_ARG;
+    if (!out || !max_send_rows || !max_recv_rows || R < 1 || R > HCCL_MAX_RANKS || row_elems < 1) return HCCL_ERR_INVALID_ARG;
     if (!valid_dtype(dt)) return HCCL_ERR_DTYPE;
     const int64_t row_bytes = row_elems * elem_bytes(dt);
     std::vector<int64_t> sext(R), rext(R);
@@ -1016,6 +1017,51 @@ hccl_status_t hccl_plan_alltoallv_dynamic(int R, const int64_t* max_send_rows, c
     }
     hccl_opts_t o;
     if (opts) o = *opts; else std::memset(&o, 0, sizeof(o));
+    const bool device_tables = R > 64 || (o.flags & HCCL_FLAG_DEVICE_TABLES) != 0;
+    if (device_tables) {
+        // Descriptors and tiles are written on the device at execute time and run by the ordinary executor: the
+        // plan holds empty tables of the largest size the capacities allow. A source of capacity b bytes yields
+        // at most b / tile + R tiles (every destination may end in one partial tile).
+        hccl_opts_t oc;
+        fill_copy_opts(&oc, &o);
+        hccl_graph* graw2 = nullptr;
+        CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw2));
+        GraphPtr g2(graw2);
+        g2->compulsory_bytes = 0;
+        hccl_plan* p = nullptr;
+        CHECK(hccl_graph_compile(g2.get(), &oc, &p));
+        int64_t total = 0;
+        for (int r = 0; r < R; ++r) total += sext[r];
+        const uint64_t tile = (opts && opts->tile_bytes) ? std::max<uint64_t>(opts->tile_bytes / 16 * 16, 512)
+                                                         : (uint64_t)default_tile(total, p->opts.sm_budget, 2, 16 << 10, 256 << 10, sweep_of(p->opts, HCCL_OP_COPY));
+        uint64_t max_tiles = (uint64_t)R * (uint64_t)R;
+        for (int r = 0; r < R; ++r) max_tiles += (uint64_t)sext[r] / tile;
+        const uint32_t end_tiles = 2u * (uint32_t)std::max(p->opts.sm_budget, 148) + 2u;
+        if (max_tiles + end_tiles > 0x7ffffff0ull) {
+            delete p;
+            return HCCL_ERR_INVALID_ARG;
+        }
+        p->descs.assign((size_t)R * R, Desc{});
+        Tile endt;
+        std::memset(&endt, 0, sizeof(endt));
+        endt.signal[0] = endt.signal[1] = -1;
+        endt.flags = TILE_FLAG_END;
+        p->tiles.assign((size_t)(max_tiles + end_tiles), endt);   // until the device has written real ones
+        compute_layout(p);
+        p->dynamic = true;
+        p->dyn_device_tables = true;
+        p->dyn_end_tiles = end_tiles;
+        p->dyn_row_bytes = row_bytes;
+        p->dyn_max_send_rows.assign(max_send_rows, max_send_rows + R);
+        p->dyn_max_recv_rows.assign(max_recv_rows, max_recv_rows + R);
+        p->opts.tile_bytes = tile;
+        p->buf_align = elem_bytes(dt);
+        p->info.tile_bytes = (int64_t)tile;
+        p->info.n_wqe = (int64_t)R * R;
+        p->info.n_tiles = (int64_t)p->tiles.size();
+        *out = p;
+        return HCCL_OK;
+    }
     o.engine = HCCL_ENGINE_LSU;  // the device-resident kernel moves bytes through registers
     hccl_graph* graw = nullptr;
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), 0, 0, &graw));

@@ -633,6 +633,7 @@ static __device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, De
         trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
     }
     t = preloaded ? *preloaded : p.tiles[cur];
+    if (t.flags & TILE_FLAG_END) return false;  // behind the last item of a device-built table: no more work, no failure
     if (!tile_ok(p, t)) {
         fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
         return false;

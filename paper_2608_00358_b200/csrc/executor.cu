@@ -37,7 +37,7 @@ hccl_status_t hccl_plan_bind(hccl_plan_t* p, void* dev_workspace, size_t bytes, 
     CUDA_TRY(cudaMemcpyAsync(dev_workspace, img.data(), img.size(), cudaMemcpyHostToDevice, s));
     CUDA_TRY(cudaStreamSynchronize(s));
     // opt-in shared memory sizes are set here, once, so that hccl_execute itself is only a launch
-    if (p->dynamic) {
+    if (p->dynamic && !p->dyn_device_tables) {
         const size_t RR = (size_t)p->R * p->R;
         const size_t smem = RR * 24 + (RR + 1) * 4 + 16;
         if (smem > 48 * 1024) CUDA_TRY(cudaFuncSetAttribute(hccl_a2a_dynamic, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(DYN_MAX_RANKS * DYN_MAX_RANKS * 24 + (DYN_MAX_RANKS * DYN_MAX_RANKS + 1) * 4 + 16)));
@@ -135,6 +135,53 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     hccl_status_t st = check_buffers(p, sendbufs, recvbufs);
     if (st != HCCL_OK) return st;
     if ((p->trig_wait_slot >= 0 || p->trig_set_slot >= 0) && !p->user_signals) return HCCL_ERR_INVALID_ARG;
+    if (p->dynamic && p->dyn_device_tables) {
+        // two launches: the table builder (one block per source rank), then the ordinary executor on what it wrote.
+        // The builder holds the start gate; the executor behind it is ordered by the stream.
+        if (!p->dyn_counts) return HCCL_ERR_INVALID_ARG;
+        static thread_local PatchParams q;
+        static thread_local ExecParams prm;
+        char* ws = (char*)p->workspace;
+        q.counts = (const long long*)p->dyn_counts;
+        q.recvcounts_out = (long long*)p->dyn_recvcounts_out;
+        q.rdispls_out = (long long*)p->dyn_rdispls_out;
+        q.ctl = (Control*)(ws + p->layout.control);
+        q.user_signals = (unsigned long long*)p->user_signals;
+        q.descs = (Desc*)(ws + p->layout.descs);
+        q.tiles = (Tile*)(ws + p->layout.tiles);
+        q.R = (uint32_t)p->R;
+        q.tile_cap = (uint32_t)p->tiles.size();
+        q.end_tiles = p->dyn_end_tiles;
+        q.timeout_ns = p->opts.timeout_ns;
+        q.row_bytes = (unsigned long long)p->dyn_row_bytes;
+        q.tile_bytes = p->opts.tile_bytes;
+        q.trig_wait_slot = p->trig_wait_slot;
+        q.trig_cmp = p->trig_cmp;
+        q.trig_wait_value = p->trig_wait_value;
+        q.trig_wait_per_epoch = p->trig_wait_per_epoch;
+        for (int r = 0; r < p->R; ++r) {
+            q.max_send_rows[r] = p->dyn_max_send_rows[r];
+            q.max_recv_rows[r] = p->dyn_max_recv_rows[r];
+        }
+        hccl_a2a_patch<<<p->R, 256, 0, (cudaStream_t)stream>>>(q);
+        CUDA_TRY(cudaGetLastError());
+        const int blocks = fill_params(p, prm, sendbufs, recvbufs);
+        prm.trig_wait_slot = -1;   // the builder has waited already
+        prm.static_tickets = 0;    // how many items are real is known only on the device: tickets and END markers
+        if (p->opts.engine == HCCL_ENGINE_BULK) {
+            const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : (int)bulk::MAX_STAGES, 2), (int)bulk::MAX_STAGES);
+            const size_t smem = (size_t)ns * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
+            hccl_executor_bulk<<<blocks, std::max(64, p->opts.threads), smem, (cudaStream_t)stream>>>(
+                prm, ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)));
+        } else if (p->opts.light) {
+            hccl_executor_lsu_light<<<blocks, p->opts.threads, 0, (cudaStream_t)stream>>>(prm);
+        } else {
+            hccl_executor_lsu<<<blocks, p->opts.threads, 0, (cudaStream_t)stream>>>(prm);
+        }
+        CUDA_TRY(cudaGetLastError());
+        p->epoch += 1;
+        return HCCL_OK;
+    }
     if (p->dynamic) {
         if (!p->dyn_counts) return HCCL_ERR_INVALID_ARG;
         static thread_local DynParams q;

@@ -529,17 +529,7 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         p->opts.sm_budget = (int32_t)std::max<uint64_t>(1, std::min<uint64_t>((uint64_t)p->opts.sm_budget, n_chains));
     }
 
-    // ---- workspace layout
-    Layout& L = p->layout;
-    uint64_t o = 0;
-    L.control = o; o = align_up(o + sizeof(Control), 256);
-    L.counters = o; o = align_up(o + 4ull * std::max<size_t>(p->sync_per_epoch.size(), 1), 256);
-    L.signals = o; o = align_up(o + 8ull * std::max<int32_t>(p->n_signals, 1), 256);
-    L.descs = o; o = align_up(o + sizeof(Desc) * std::max<size_t>(p->descs.size(), 1), 256);
-    L.tiles = o; o = align_up(o + sizeof(Tile) * std::max<size_t>(p->tiles.size(), 1), 256);
-    L.waits = o; o = align_up(o + sizeof(Wait) * std::max<size_t>(p->waits.size(), 1), 256);
-    L.scratch = o; o = align_up(o + (uint64_t)p->scratch_bytes, 256);
-    L.total = o;
+    compute_layout(p);
 
     hccl_plan_info_t& I = p->info;
     std::memset(&I, 0, sizeof(I));
@@ -563,6 +553,19 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
     I.static_chains = (int64_t)p->n_chains;
     *out = p;
     return HCCL_OK;
+}
+
+void hccl::compute_layout(hccl_plan* p) {
+    Layout& L = p->layout;
+    uint64_t o = 0;
+    L.control = o; o = align_up(o + sizeof(Control), 256);
+    L.counters = o; o = align_up(o + 4ull * std::max<size_t>(p->sync_per_epoch.size(), 1), 256);
+    L.signals = o; o = align_up(o + 8ull * std::max<int32_t>(p->n_signals, 1), 256);
+    L.descs = o; o = align_up(o + sizeof(Desc) * std::max<size_t>(p->descs.size(), 1), 256);
+    L.tiles = o; o = align_up(o + sizeof(Tile) * std::max<size_t>(p->tiles.size(), 1), 256);
+    L.waits = o; o = align_up(o + sizeof(Wait) * std::max<size_t>(p->waits.size(), 1), 256);
+    L.scratch = o; o = align_up(o + (uint64_t)p->scratch_bytes, 256);
+    L.total = o;
 }
 
 extern "C" {

@@ -52,6 +52,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         d.info = info;
         d.head = d.tail = d.groups = 0;
         d.pol = policy_evict_first();
+        d.pol_keep = policy_evict_last();
         d.ok = true;
         bool live = true;
         uint32_t next = next0;
@@ -93,6 +94,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
 
     // ------------------------------------------------------------ compute warps
     const uint32_t ctid = tid - 32, cnth = ncw * 32;
+    const unsigned long long pol_keep = policy_evict_last();
     for (unsigned long long k = 0;; ++k) {
         const uint32_t slot = (uint32_t)(k % ns), parity = (uint32_t)((k / ns) & 1);
         if (!mbar_wait(p, full + 8 * slot, parity, 2 * p.timeout_ns + 1000000000ull, 0xfffffffdu)) break;
@@ -105,7 +107,13 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         }
         if (kind == PIECE_REDUCE) {
             reduce_piece_dispatch(pi.dt_a, pi.dt_b, pi.dt_d, stages_ptr + (size_t)slot * STAGE_BYTES,
-                                  stages_ptr + (size_t)slot * STAGE_BYTES + pi.b_off, pi.dst, pi.n, ctid, cnth);
+                                  stages_ptr + (size_t)slot * STAGE_BYTES + pi.b_off, pi.dst, pi.n, ctid, cnth, pi.keep_dst != 0, pol_keep);
+            if (pi.discard_src) {
+                // whole 128-byte lines inside the piece; issued before the item is published, so the slot's next
+                // writer is ordered after them
+                const uintptr_t lo = ((uintptr_t)pi.discard_src + 127u) & ~(uintptr_t)127u, hi = ((uintptr_t)pi.discard_src + pi.discard_bytes) & ~(uintptr_t)127u;
+                for (uintptr_t a = lo + (uintptr_t)ctid * 128u; a < hi; a += (uintptr_t)cnth * 128u) discard_line((const void*)a);
+            }
         } else if (kind == PIECE_COPYW) {
             const uint4* src = reinterpret_cast<const uint4*>(stages_ptr + (size_t)slot * STAGE_BYTES);
             uint4* dst = reinterpret_cast<uint4*>(pi.dst);

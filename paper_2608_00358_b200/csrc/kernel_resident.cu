@@ -232,4 +232,132 @@ __global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant
     if (tid == 0) leave(q);
 }
 
+
+// ====================================================================== device-side table builder (any R up to 256)
+// The R x R count matrix does not fit shared memory beyond 64 ranks, and no block needs all of it: block s
+// builds the tables of source rank s only. It reads rows 0..s of the counts (coalesced, from the L2): from the
+// rows above its own it takes, per destination d, the rows that earlier sources send to d (= its receive
+// displacement in Y_d) and the number of tiles those sources produce (= the index of its own first tile); its
+// own row gives the send displacements and the tiles per segment, both by block-wide exclusive scans built from
+// warp shuffles. No block waits for another one. Every block validates what it reads; the block of the last
+// source also holds every destination's total and checks it against the receive capacities. A rejected matrix
+// raises the abort word, so the executor launched behind this kernel moves nothing.
+
+// Exclusive scan over the 256 threads of the block (one value per thread); *total = the sum. `s_w` holds 8 words.
+__device__ __forceinline__ long long block_exclusive_scan(long long v, long long* s_w, long long* total) {
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const long long inc = warp_inclusive_scan(v, lane);
+    if (lane == 31) s_w[warp] = inc;
+    __syncthreads();
+    long long before = 0, all = 0;
+#pragma unroll
+    for (uint32_t w = 0; w < 8; ++w) {
+        const long long x = s_w[w];
+        if (w < warp) before += x;
+        all += x;
+    }
+    __syncthreads();
+    *total = all;
+    return before + inc - v;
+}
+
+__global__ void __launch_bounds__(256, 1) hccl_a2a_patch(const __grid_constant__ PatchParams q) {
+    __shared__ long long s_w[8];
+    __shared__ uint32_t s_tp[HCCL_MAX_RANKS + 1];   // exclusive prefix of this source's tiles per destination
+    __shared__ long long s_bytes[HCCL_MAX_RANKS];   // bytes of segment (s, d)
+    __shared__ int s_bad, s_live;
+    const uint32_t R = q.R, s = blockIdx.x, d = threadIdx.x;
+    init_epoch(q);
+    if (d == 0) {
+        s_bad = 0;
+        bool live = true;
+        if (q.trig_wait_slot >= 0)
+            live = wait_signal(q, q.user_signals + q.trig_wait_slot, q.trig_cmp, q.trig_wait_value + (unsigned long long)g_epoch * q.trig_wait_per_epoch, 0xffffffffu);
+        s_live = live ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_live) return;   // the wait gave up (recorded by wait_signal) or the execution was aborted
+    const long long T = (long long)q.tile_bytes, rb = (long long)q.row_bytes;
+    // rows above this source's own: receive displacement of column d and tiles produced so far
+    long long col = 0, tiles_before = 0, own = 0;
+    bool bad = false;
+    if (d < R) {
+        for (uint32_t r = 0; r <= s; ++r) {
+            const long long c = __ldcg(q.counts + (size_t)r * R + d);
+            if (c < 0 || c > (1ll << 40)) { bad = true; break; }
+            if (r < s) {
+                col += c;
+                tiles_before += (c * rb + T - 1) / T;
+            } else {
+                own = c;
+            }
+        }
+    }
+    if (bad) s_bad = 1;
+    long long row_total, base_tiles, row_tiles;
+    const long long sd = block_exclusive_scan(own, s_w, &row_total);           // send displacement, rows
+    (void)block_exclusive_scan(tiles_before, s_w, &base_tiles);                // index of this source's first tile
+    const long long my_tiles = (own * rb + T - 1) / T;
+    const long long tp = block_exclusive_scan(my_tiles, s_w, &row_tiles);      // first tile of segment (s, d) within the row
+    if (d == 0 && row_total > q.max_send_rows[s]) s_bad = 1;
+    if (s == R - 1 && d < R && col + own > q.max_recv_rows[d]) s_bad = 1;
+    if (d < R) {
+        s_tp[d] = (uint32_t)tp;
+        s_bytes[d] = own * rb;
+    }
+    if (d == 0) s_tp[R] = (uint32_t)row_tiles;
+    __syncthreads();
+    const long long cap = (long long)q.tile_cap - (long long)q.end_tiles;   // real items must leave room for the END markers
+    if (s_bad || base_tiles + row_tiles > cap) {
+        if (d == 0) fail(q, HCCL_ERR_BAD_DESCRIPTOR, (unsigned long long)s * R);
+        return;
+    }
+    if (d < R) {
+        Desc ds;
+        memset(&ds, 0, sizeof(ds));
+        ds.op = HCCL_OP_COPY;
+        ds.kind_dst = HCCL_BUF_RECV;
+        ds.kind_a = HCCL_BUF_SEND;
+        ds.cmp = HCCL_HINT_READ_ONCE;
+        ds.rank_dst = (uint16_t)d;
+        ds.rank_a = (uint16_t)s;
+        ds.off_dst = col * rb;
+        ds.off_a = sd * rb;
+        ds.count = own * rb;
+        q.descs[(size_t)s * R + d] = ds;
+        if (q.recvcounts_out) q.recvcounts_out[(size_t)d * R + s] = own;
+        if (q.rdispls_out) q.rdispls_out[(size_t)d * R + s] = col;
+    }
+    // this source's tiles, spread over the block: tile j of the row belongs to the last destination whose prefix
+    // is <= j (destinations with nothing to send share a prefix value with their successor and are skipped)
+    for (uint32_t j = d; j < (uint32_t)row_tiles; j += blockDim.x) {
+        uint32_t lo = 0, hi = R;
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (s_tp[mid] <= j) lo = mid; else hi = mid;
+        }
+        const unsigned long long start = (unsigned long long)(j - s_tp[lo]) * (unsigned long long)T;
+        Tile t;
+        t.desc = s * R + lo;
+        t.count = (uint32_t)min((unsigned long long)T, (unsigned long long)s_bytes[lo] - start);
+        t.start = start;
+        t.signal[0] = t.signal[1] = -1;
+        t.wait_off = 0;
+        t.wait_cnt = 0;
+        t.flags = TILE_FLAG_NONE;
+        q.tiles[(size_t)base_tiles + j] = t;
+    }
+    if (s == R - 1) {
+        // behind the last item: END markers for every block's current and look-ahead claim
+        const size_t n = (size_t)(base_tiles + row_tiles);
+        for (uint32_t j = d; j < q.end_tiles; j += blockDim.x) {
+            Tile t;
+            memset(&t, 0, sizeof(t));
+            t.signal[0] = t.signal[1] = -1;
+            t.flags = TILE_FLAG_END;
+            q.tiles[n + j] = t;
+        }
+    }
+}
+
 }  // namespace hccl

@@ -34,6 +34,28 @@ struct DynParams {
     void* recv[DYN_MAX_RANKS];
 };
 
+// Device-side table builder of the device-resident AllToAllv for any rank count (Sec. IV-B.2: the work requests
+// are patched on the device): one block per source rank writes that source's R descriptors and their tiles
+// into the bound workspace, where the ordinary executor, launched right behind it, finds them.
+struct PatchParams {
+    const long long* counts;       // device, [R*R], counts[s*R+d] rows from s to d
+    long long* recvcounts_out;     // device, [R*R] indexed [d*R+s], or null
+    long long* rdispls_out;        // device, [R*R] indexed [d*R+s], or null
+    Control* ctl;
+    unsigned long long* user_signals;
+    Desc* descs;                   // [R*R] in the workspace, descriptor s*R+d = segment (s, d)
+    Tile* tiles;                   // [tile_cap] in the workspace
+    uint32_t R, tile_cap;          // tile_cap includes room for end_tiles END markers
+    uint32_t end_tiles, pad0;
+    unsigned long long timeout_ns;
+    unsigned long long row_bytes, tile_bytes;
+    long long trig_wait_slot;
+    int trig_cmp, pad1;
+    unsigned long long trig_wait_value, trig_wait_per_epoch;
+    long long max_send_rows[HCCL_MAX_RANKS], max_recv_rows[HCCL_MAX_RANKS];
+};
+
+__global__ void __launch_bounds__(256, 1) hccl_a2a_patch(const __grid_constant__ PatchParams q);
 __global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p);
 __global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p);
 __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t copy_by_warps);

@@ -63,6 +63,8 @@ struct hccl_plan {
     uint64_t trig_wait_value = 0, trig_wait_per_epoch = 0, trig_set_value = 0, trig_set_per_epoch = 0;
     // device-resident AllToAllv (Sec. IV-B.2): sizes are read from device memory when the kernel runs
     bool dynamic = false;
+    bool dyn_device_tables = false;        // descriptors and tiles are written by a kernel at execute time
+    uint32_t dyn_end_tiles = 0;            // END markers kept behind the last real tile
     int64_t dyn_row_bytes = 0;
     std::vector<int64_t> dyn_max_send_rows, dyn_max_recv_rows;
     const void* dyn_counts = nullptr;
@@ -114,6 +116,7 @@ inline int64_t round_tile(int64_t target, int64_t sweep) {
     return std::max<int64_t>(64, (target + 63) / 64 * 64);
 }
 hccl_status_t compile_graph(const hccl_graph* g, const hccl_opts_t* opts, hccl_plan** out);
+void compute_layout(hccl_plan* p);  // workspace offsets from the sizes of the plan's tables
 void fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in);
 hccl_status_t plan_alltoallv_window(int R, const int64_t* sendcounts, const int64_t* sdispls, const int64_t* recvcounts,
                                     const int64_t* rdispls, hccl_dtype_t dt, int64_t row_elems, const hccl_opts_t* opts,

@@ -66,6 +66,9 @@ struct Layout {  // byte offsets inside the workspace
     uint64_t control, counters, signals, descs, tiles, waits, scratch, total;
 };
 
-enum : uint16_t { TILE_FLAG_NONE = 0 };
+// TILE_FLAG_END: written by the device-side table builder of the device-resident AllToAllv behind the last real work
+// item of an execution; a block that claims such an item has no more work (the number of items is then known
+// only on the device).
+enum : uint16_t { TILE_FLAG_NONE = 0, TILE_FLAG_END = 1 };
 
 }  // namespace hccl

@@ -12,8 +12,17 @@ SENT = 0x5A
 
 def test_dynamic_plan_validation():
     with pytest.raises(hb.HcclError) as e:
-        hb.hccl_plan_alltoallv_dynamic(65, [1] * 65, [1] * 65, hb.BF16, 8)
+        hb.hccl_plan_alltoallv_dynamic(257, [1] * 257, [1] * 257, hb.BF16, 8)
     assert e.value.status == hb.ERR_INVALID_ARG
+    # beyond 64 ranks (or on request) the tables are built on the device: the plan holds room for the largest
+    # table the capacities allow (rows * row bytes / tile per source, plus one partial tile per pair, plus the
+    # END markers) and names the ordinary executor
+    big = hb.hccl_plan_alltoallv_dynamic(65, [100] * 65, [100] * 65, hb.BF16, 8, dict(tile_bytes=512))
+    i = big.info()
+    assert i.n_wqe == 65 * 65 and i.engine == hb.ENGINE_BULK and i.tile_bytes == 512
+    assert i.n_tiles == 65 * (100 * 16 // 512) + 65 * 65 + 2 * 148 + 2
+    same = hb.hccl_plan_alltoallv_dynamic(4, [10] * 4, [12] * 4, hb.FP16, 8, dict(flags=hb.FLAG_DEVICE_TABLES, engine=hb.ENGINE_LSU))
+    assert same.info().n_wqe == 16 and same.info().engine == hb.ENGINE_LSU and same.extents(0) == (160, 192)
     with pytest.raises(hb.HcclError) as e:
         hb.hccl_plan_alltoallv_dynamic(2, [1, -1], [1, 1], hb.BF16, 8)
     assert e.value.status == hb.ERR_INVALID_ARG
@@ -67,6 +76,120 @@ def test_dynamic_alltoallv_counts_change_between_executions(R, row_elems, hi):
             assert np.array_equal(recv[d].cpu().numpy(), want[d]), (seed, d)
         assert np.array_equal(rc_out.cpu().numpy().reshape(R, R), C.T)
         assert np.array_equal(rd_out.cpu().numpy().reshape(R, R), RD)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("R,row_elems,hi,opts", [
+    (8, 16, 50, dict(flags=hb.FLAG_DEVICE_TABLES, engine=hb.ENGINE_LSU, sm_budget=24, tile_bytes=2048)),
+    (8, 128, 300, dict(flags=hb.FLAG_DEVICE_TABLES, sm_budget=24, tile_bytes=4096)),
+    (8, 7, 50, dict(flags=hb.FLAG_DEVICE_TABLES, sm_budget=16, tile_bytes=1024)),          # rows of 14 bytes: unaligned segments
+    (64, 64, 24, dict(flags=hb.FLAG_DEVICE_TABLES, tile_bytes=4096)),
+    (65, 32, 12, dict(sm_budget=32, tile_bytes=2048)),
+    (128, 32, 12, dict(tile_bytes=4096)),
+    (128, 64, 10, dict(engine=hb.ENGINE_LSU, sm_budget=64, tile_bytes=8192)),
+    (256, 16, 6, None),
+], ids=["r8_lsu", "r8_bulk", "r8_rows_of_14_bytes", "r64", "r65", "r128_bulk", "r128_lsu", "r256_defaults"])
+def test_dynamic_alltoallv_tables_built_on_the_device(R, row_elems, hi, opts):
+    """Beyond 64 ranks (and, with HCCL_FLAG_DEVICE_TABLES, below) a kernel writes descriptors and tiles into the
+    workspace from the counts in device memory and the ordinary executor runs them. Counts change between
+    executions of one bound plan, including a shrinking table (stale tiles behind the END markers)."""
+    import torch
+    cap = hi * R + 3
+    plan, dc, X, send, recv, counts, rc_out, rd_out, rb = _setup(R, row_elems, cap, opts=opts)
+    assert plan.info().n_wqe == R * R
+    for seed in (1, 2, 3, 4):
+        C = synth.uniform_counts(R, seed, hi=hi)
+        if seed == 2:
+            C[:, R // 2] = 0                       # a destination that receives nothing
+            C[0, :] = 0                            # a source that sends nothing
+            C[R - 1, :] = 0                        # ... the last one too (it writes the END markers)
+        if seed == 3:
+            C[:] = 0
+            C[1, 0] = cap                          # one segment fills a whole send and a whole receive buffer
+        if seed == 4:
+            C[:] = 0                               # nothing at all
+        counts.copy_(torch.from_numpy(C.reshape(-1)))
+        for t in recv:
+            t.fill_(SENT)
+        rc_out.fill_(-1)
+        rd_out.fill_(-1)
+        dc.execute()
+        dc.check()
+        want, RD = _expect(X, C, rb, cap)
+        for d in range(R):
+            assert np.array_equal(recv[d].cpu().numpy(), want[d]), (seed, d)
+        assert np.array_equal(rc_out.cpu().numpy().reshape(R, R), C.T)
+        assert np.array_equal(rd_out.cpu().numpy().reshape(R, R), RD)
+    for s_ in range(R):
+        assert np.array_equal(send[s_].cpu().numpy(), X[s_])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("R", [8, 128])
+def test_device_built_tables_reject_counts_beyond_capacity_without_writing(R):
+    import torch
+    row_elems, cap = 16, 3 * R
+    opts = dict(flags=hb.FLAG_DEVICE_TABLES, tile_bytes=1024)
+    plan, dc, X, send, recv, counts, rc_out, rd_out, rb = _setup(R, row_elems, cap, opts=opts)
+    for bad in ("overflow_recv", "overflow_send", "negative", "overflow_recv_last_source"):
+        C = np.full((R, R), 2, dtype=np.int64)
+        if bad == "overflow_recv":
+            C[: R // 2 + 1, 1] = 7                 # more than 3R rows into destination 1
+        elif bad == "overflow_send":
+            C[R // 2, :] = 4                       # source R/2 would send 4R rows
+        elif bad == "negative":
+            C[R - 2, 3] = -1
+        else:
+            C[R - 1, :] = 1
+            C[R - 1, 0] = R + 3                    # only the last source's row tips destination 0 over (3R + 1 rows)
+        counts.copy_(torch.from_numpy(C.reshape(-1)))
+        dc.execute()
+        torch.cuda.synchronize()
+        st, _ = plan.status()
+        assert st == hb.ERR_BAD_DESCRIPTOR, bad
+        for t in recv:
+            assert bool((t == SENT).all()), bad
+        assert float(torch.ones(4, device="cuda").sum()) == 4.0
+        # a good matrix straight afterwards, on the same bound plan
+        C = synth.uniform_counts(R, 5, hi=2)
+        counts.copy_(torch.from_numpy(C.reshape(-1)))
+        dc.execute()
+        dc.check()
+        want, _ = _expect(X, C, rb, cap)
+        for d in range(R):
+            assert np.array_equal(recv[d].cpu().numpy(), want[d]), (bad, d)
+        for t in recv:
+            t.fill_(SENT)
+
+
+@pytest.mark.gpu
+def test_device_triggered_alltoallv_over_128_ranks():
+    """Pre-launched on its own stream, held at the start gate by the table builder, released by a producer
+    that writes the counts first; the completion value is stored by the executor behind the builder."""
+    import torch
+    R, row_elems, cap = 128, 32, 700
+    plan, dc, X, send, recv, counts, rc_out, rd_out, rb = _setup(R, row_elems, cap, opts=dict(sm_budget=16))
+    signals = torch.zeros(2, dtype=torch.int64, device="cuda")
+    plan.set_user_signals(signals.data_ptr(), 2)
+    plan.set_trigger(wait_slot=0, cmp=hb.CMP_GE, wait_value=0, wait_per_epoch=1, set_slot=1, set_value=100, set_per_epoch=1)
+    coll, prod = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for epoch in (1, 2):
+        C = synth.uniform_counts(R, 20 + epoch, hi=5)
+        host_counts = torch.from_numpy(C.reshape(-1)).pin_memory()
+        for t in recv:
+            t.fill_(SENT)
+        torch.cuda.synchronize()
+        dc.execute(coll)
+        with torch.cuda.stream(prod):
+            counts.copy_(host_counts, non_blocking=True)
+            signals[0:1].fill_(epoch)
+        torch.cuda.synchronize()
+        assert plan.status()[0] == hb.OK
+        assert int(signals[1]) == 100 + epoch
+        want, _ = _expect(X, C, rb, cap)
+        for d in range(R):
+            assert np.array_equal(recv[d].cpu().numpy(), want[d]), (epoch, d)
 
 
 @pytest.mark.gpu
