@@ -134,7 +134,8 @@ typedef struct {
     int32_t chain_group;    /* chains scheduled together in chain-group-major order; FP32 scratch slots are recycled
                                every two groups. Default: all chains together (a slot per chain, no recycling) while
                                the FP32 partials take at most 32 MiB (AllReduce rings: 128 MiB), else 16 */
-    int32_t threads;        /* threads per block, multiple of 32 (default 512) */
+    int32_t threads;        /* threads per block, multiple of 32. Register engine: one control warp + workers (default 512,
+                               at least 64). Bulk engine: DMA warp + control warp + compute warps (default 320, at least 96) */
     int32_t stages;         /* bulk engine: shared-memory stages of 48 KiB per block, 2..4 (default 4) */
     int32_t cluster;        /* register engine: launch blocks in clusters of this size (2, 4, 8) so that they sit on
                                neighbouring SMs; 0/1 = no clusters. Ignored unless it divides the block count. */
@@ -143,6 +144,9 @@ typedef struct {
                                best per-block rate), 2 = the bulk unit, 0 = compute warps below 100 blocks, bulk unit otherwise */
     int32_t rack_size;      /* ranks per rack for HCCL_ALGO_RING_2LEVEL and for cross-rack byte accounting (default 16,
                                the paper's rack, Sec. V-D) */
+    int32_t stage_kib;      /* bulk engine: KiB per shared-memory stage, a multiple of 12 in [12, 96] (default 48); with
+                               opts.stages left at 0 the number of stages keeps 192 KiB in flight (at most 8 stages) */
+    int32_t reserved0;      /* 0 */
 } hccl_opts_t;
 
 typedef struct hccl_plan hccl_plan_t;   /* opaque, host-owned: a compiled, cacheable work packet (Sec. V-B) */

@@ -180,11 +180,14 @@ static __device__ void reduce_piece_dispatch(int da, int db, int dd, const char*
 
 // State of the DMA thread.
 struct Dma {
-    uint32_t ns, lag;
+    uint32_t ns, lag, sb;  // stages, store lag, bytes per stage
     uint32_t stages, full, empty;  // shared-memory addresses
     char* stages_ptr;
     PieceInfo* info;
     unsigned long long head, tail, groups;
+    // stage and mbarrier phase parity of piece `head` and of piece `tail`, stepped along with the counters (a 64-bit
+    // division per piece on the one issuing thread would cost more than the issue itself)
+    uint32_t head_slot, head_par, tail_slot, tail_par;
     unsigned long long pol;       // evict-first: streamed send data
     unsigned long long pol_keep;  // evict-last: FP32 partials in scratch
     bool ok;
@@ -195,7 +198,7 @@ struct Dma {
 // pieces are finished by the compute warps on their own.
 static __device__ void retire_one(const ExecParams& p, Dma& d) {
     const unsigned long long j = d.tail;
-    const uint32_t slot = (uint32_t)(j % d.ns), parity = (uint32_t)((j / d.ns) & 1);
+    const uint32_t slot = d.tail_slot, parity = d.tail_par;
     PieceInfo& pi = d.info[slot];
     if (pi.kind == PIECE_COPY) {
         if (!mbar_wait(p, d.full + 8 * slot, parity, p.timeout_ns, pi.tile_index)) d.ok = false;
@@ -204,11 +207,11 @@ static __device__ void retire_one(const ExecParams& p, Dma& d) {
                 for (uint32_t k = 0; k < pi.ndst; ++k) {
                     uint32_t r = pi.rank_dst + k;
                     if (r >= p.R) r -= p.R;
-                    bulk_store_part((char*)p.recv[r] + pi.dst_off, d.stages + slot * STAGE_BYTES, pi.n, pi.evict_first != 0, d.pol);
+                    bulk_store_part((char*)p.recv[r] + pi.dst_off, d.stages + slot * d.sb, pi.n, pi.evict_first != 0, d.pol);
                 }
                 bulk_commit();
             } else {
-                bulk_store(pi.dst, d.stages + slot * STAGE_BYTES, pi.n, pi.evict_first != 0, d.pol);
+                bulk_store(pi.dst, d.stages + slot * d.sb, pi.n, pi.evict_first != 0, d.pol);
             }
             pi.group = d.groups++;
             if (pi.last && p.trace) trace_put(p.trace, p.trace_cap, pi.tile_index, 3, globaltimer_ns());
@@ -222,6 +225,18 @@ static __device__ void retire_one(const ExecParams& p, Dma& d) {
         }
     }
     d.tail = j + 1;
+    if (++d.tail_slot == d.ns) {
+        d.tail_slot = 0;
+        d.tail_par ^= 1u;
+    }
+}
+// The piece just written into stage head_slot has been issued.
+__device__ __forceinline__ void advance_head(Dma& d) {
+    d.head += 1;
+    if (++d.head_slot == d.ns) {
+        d.head_slot = 0;
+        d.head_par ^= 1u;
+    }
 }
 static __device__ void drain(const ExecParams& p, Dma& d) {
     while (d.tail < d.head) retire_one(p, d);
@@ -233,7 +248,7 @@ static __device__ bool acquire_slot(const ExecParams& p, Dma& d, unsigned long l
     const unsigned long long j = k - d.ns;
     while (d.tail <= j) retire_one(p, d);
     if (!d.ok) return false;
-    const uint32_t slot = (uint32_t)(j % d.ns), parity = (uint32_t)((j / d.ns) & 1);
+    const uint32_t slot = d.head_slot, parity = d.head_par ^ 1u;   // k is d.head; piece k - ns used the same stage one phase earlier
     if (!mbar_wait(p, d.empty + 8 * slot, parity, 2 * p.timeout_ns + 1000000000ull, detail)) {
         d.ok = false;
         return false;
@@ -247,18 +262,10 @@ __device__ __forceinline__ void keep_lag(const ExecParams& p, Dma& d) {
     while (d.ok && d.head - d.tail > d.lag) retire_one(p, d);
 }
 
-static __device__ bool wait_counter_draining(const ExecParams& p, Dma& d, uint32_t sync, uint32_t per_epoch, uint32_t tile) {
-    const uint32_t target = g_epoch * per_epoch;
-    if ((int32_t)(ld_acquire_u32(p.counters + sync) - target) >= 0) return true;
-    drain(p, d);  // the item waited for may sit in this block's own pipeline
-    if (!d.ok) return false;
-    return wait_counter(p, sync, per_epoch, tile);
-}
-
 static __device__ void issue_simple(const ExecParams& p, Dma& d, uint32_t kind, uint32_t cur, const Tile* t, const Desc* ds) {
     const unsigned long long k = d.head;
     if (!acquire_slot(p, d, k, cur)) return;
-    const uint32_t slot = (uint32_t)(k % d.ns);
+    const uint32_t slot = d.head_slot;
     PieceInfo& pi = d.info[slot];
     pi.kind = kind;
     pi.n = 0;
@@ -269,57 +276,77 @@ static __device__ void issue_simple(const ExecParams& p, Dma& d, uint32_t kind, 
     if (t) pi.tile = *t;
     if (ds) pi.desc = *ds;
     mbar_arrive(d.full + 8 * slot);  // no bytes expected: the phase completes at once
-    d.head = k + 1;
+    advance_head(d);
 }
 
-// One work item through the DMA thread. Returns false when the block must stop.
-static __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const Tile* preloaded = nullptr) {
+// ---- hand-over from the control thread to the DMA thread
+// The control thread (first lane of the block's second warp) claims items, fetches their records, waits for their
+// dependencies and performs WAIT / SET / NOOP items itself; items that move data are passed on through a small
+// ring in shared memory. The three or four dependent trips to the L2 that start an item thus overlap with the
+// DMA thread's piece issue instead of stalling it.
+constexpr uint32_t QUEUE = 2;                  // prepared items the control thread may be ahead by
+enum : uint32_t { Q_ITEM = 0, Q_STOP = 1 };
+struct alignas(16) Prepared {
+    Tile t;
+    Desc ds;
+    uint32_t item, kind, waited, pad;
+};
+
+// One item on the control thread. Returns 0: stop (no more work, failure or abort), 1: done here (no data to
+// move), 2: a data item, its records in t / ds, its dependencies met.
+static __device__ int control_item(const ExecParams& p, uint32_t cur, const Tile* preloaded, Tile& t, Desc& ds) {
     if (p.trace) {
         trace_put(p.trace, p.trace_cap, cur, 0, (unsigned long long)cur | ((unsigned long long)blockIdx.x << 32));
         trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
     }
-    const Tile t = preloaded ? *preloaded : p.tiles[cur];
-    if (t.flags & TILE_FLAG_END) return false;  // behind the last item of a device-built table: no more work, no failure
+    t = preloaded ? *preloaded : p.tiles[cur];
+    if (t.flags & TILE_FLAG_END) return 0;  // behind the last item of a device-built table: no more work, no failure
     if (!tile_ok(p, t)) {
         fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
-        return false;
+        return 0;
     }
-    const Desc ds = p.descs[t.desc];
+    ds = p.descs[t.desc];
     if (!desc_ok(p, ds)) {
         fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
-        return false;
+        return 0;
     }
-    bool waited = false;
     for (uint32_t w = 0; w < t.wait_cnt; ++w) {
         const Wait x = p.waits[t.wait_off + w];
         if (x.sync >= p.n_syncs) {
             fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
-            return false;
+            return 0;
         }
-        if (!wait_counter_draining(p, d, x.sync, x.per_epoch, cur)) return false;
-        waited = true;
+        // an item of this block's own pipeline may be what is waited for: the DMA thread retires (and so publishes)
+        // what it has in flight whenever it has nothing to issue
+        if (!wait_counter(p, x.sync, x.per_epoch, cur)) return 0;
     }
-    if (waited) fence_proxy_async();  // what the acquired counters cover must be visible to the bulk unit too
     if (p.trace) trace_put(p.trace, p.trace_cap, cur, 2, globaltimer_ns());
     switch (ds.op) {
         case HCCL_OP_WAIT: {
-            drain(p, d);
-            if (!d.ok) return false;
             const unsigned long long* addr = (ds.kind_a == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + ds.off_a;
-            if (!wait_signal(p, addr, ds.cmp, ds.value + (unsigned long long)g_epoch * ds.value_per_epoch, cur)) return false;
+            if (!wait_signal(p, addr, ds.cmp, ds.value + (unsigned long long)g_epoch * ds.value_per_epoch, cur)) return 0;
             publish_tile(p, t);
-            return true;
+            return 1;
         }
         case HCCL_OP_SET: {
             unsigned long long* addr = (ds.kind_dst == HCCL_BUF_SIGNAL ? p.signals : p.user_signals) + ds.off_dst;
             __threadfence();
             st_release_u64(addr, ds.value + (unsigned long long)g_epoch * ds.value_per_epoch);
             publish_tile(p, t);
-            return true;
+            return 1;
         }
         case HCCL_OP_NOOP:
             publish_tile(p, t);
-            return true;
+            return 1;
+        default:
+            return 2;
+    }
+}
+
+// One data item through the DMA thread (records and dependencies were dealt with by the control thread).
+// Returns false when the block must stop.
+static __device__ bool dma_issue(const ExecParams& p, Dma& d, uint32_t cur, const Tile& t, const Desc& ds) {
+    switch (ds.op) {
         case HCCL_OP_COPY: {
             char* dst = buf_base(p, ds.kind_dst, ds.rank_dst) + ds.off_dst + t.start;
             const char* src = buf_base(p, ds.kind_a, ds.rank_a) + ds.off_a + t.start;
@@ -345,11 +372,11 @@ static __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const
                 for (uint32_t k = 1; k < nd; ++k) dstk(k)[body + i] = b;
             }
             const bool stream = ds.kind_a == HCCL_BUF_SEND;
-            for (uint32_t off = 0; off < body && d.ok; off += STAGE_BYTES) {
-                const uint32_t nb = min(STAGE_BYTES, body - off);
+            for (uint32_t off = 0; off < body && d.ok; off += d.sb) {
+                const uint32_t nb = min(d.sb, body - off);
                 const unsigned long long k = d.head;
                 if (!acquire_slot(p, d, k, cur)) return false;
-                const uint32_t slot = (uint32_t)(k % d.ns);
+                const uint32_t slot = d.head_slot;
                 PieceInfo& pi = d.info[slot];
                 pi.kind = d.copy_by_warps ? PIECE_COPYW : PIECE_COPY;
                 pi.n = nb;
@@ -363,8 +390,8 @@ static __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const
                 pi.signal[1] = t.signal[1];
                 pi.evict_first = stream ? 1 : 0;
                 mbar_arrive_expect_tx(d.full + 8 * slot, nb);
-                bulk_load(d.stages + slot * STAGE_BYTES, src + off, nb, d.full + 8 * slot, stream, d.pol);
-                d.head = k + 1;
+                bulk_load(d.stages + slot * d.sb, src + off, nb, d.full + 8 * slot, stream, d.pol);
+                advance_head(d);
                 keep_lag(p, d);
             }
             return d.ok;
@@ -379,12 +406,12 @@ static __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const
                 keep_lag(p, d);
                 return d.ok;
             }
-            const uint32_t pe = piece_elems(ea, eb);
+            const uint32_t pe = piece_elems(d.sb, ea, eb);
             for (uint32_t e0 = 0; e0 < t.count && d.ok; e0 += pe) {
                 const uint32_t ne = min(pe, t.count - e0);
                 const unsigned long long k = d.head;
                 if (!acquire_slot(p, d, k, cur)) return false;
-                const uint32_t slot = (uint32_t)(k % d.ns);
+                const uint32_t slot = d.head_slot;
                 PieceInfo& pi = d.info[slot];
                 pi.kind = PIECE_REDUCE;
                 pi.n = ne;
@@ -402,9 +429,9 @@ static __device__ bool dma_item(const ExecParams& p, Dma& d, uint32_t cur, const
                 pi.discard_bytes = ne * ea;
                 mbar_arrive_expect_tx(d.full + 8 * slot, ne * (ea + eb));
                 const bool a_keep = ds.kind_a == HCCL_BUF_SCRATCH;
-                bulk_load(d.stages + slot * STAGE_BYTES, a + (size_t)e0 * ea, ne * ea, d.full + 8 * slot, ds.kind_a == HCCL_BUF_SEND || a_keep, a_keep ? d.pol_keep : d.pol);
-                bulk_load(d.stages + slot * STAGE_BYTES + pe * ea, b + (size_t)e0 * eb, ne * eb, d.full + 8 * slot, ds.kind_b == HCCL_BUF_SEND, d.pol);
-                d.head = k + 1;
+                bulk_load(d.stages + slot * d.sb, a + (size_t)e0 * ea, ne * ea, d.full + 8 * slot, ds.kind_a == HCCL_BUF_SEND || a_keep, a_keep ? d.pol_keep : d.pol);
+                bulk_load(d.stages + slot * d.sb + pe * ea, b + (size_t)e0 * eb, ne * eb, d.full + 8 * slot, ds.kind_b == HCCL_BUF_SEND, d.pol);
+                advance_head(d);
                 keep_lag(p, d);
             }
             return d.ok;

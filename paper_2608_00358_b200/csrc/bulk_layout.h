@@ -7,16 +7,24 @@
 namespace hccl {
 namespace bulk {
 
-constexpr uint32_t MAX_STAGES = 4;            // 4 x 48 KiB + bookkeeping fits the 227 KB a block may have
-constexpr uint32_t STAGE_BYTES = 49152;       // a COPY piece fills a stage; a REDUCE piece splits it into A and B
+constexpr uint32_t MAX_STAGES = 8;
+constexpr uint32_t STAGE_BYTES = 49152;       // default stage: a COPY piece fills a stage; a REDUCE piece splits it into A and B;
+                                              // 4 x 48 KiB + bookkeeping fits the 227 KB a block may have
+constexpr uint32_t MIN_STAGE_BYTES = 12288, MAX_STAGE_BYTES = 98304;  // opts.stage_kib, a multiple of 12 KiB in this range
 // Elements per REDUCE piece: as many as fit a stage with both operands, in whole multiples of 512 elements
-// (6144 for fp32+fp32, 8192 for fp32+16-bit, 12288 for 16-bit+16-bit).
-__host__ __device__ constexpr uint32_t piece_elems(uint32_t ea, uint32_t eb) { return STAGE_BYTES / (ea + eb) / 512 * 512; }
+// (48 KiB stages: 6144 for fp32+fp32, 8192 for fp32+16-bit, 12288 for 16-bit+16-bit).
+__host__ __device__ constexpr uint32_t piece_elems(uint32_t stage_bytes, uint32_t ea, uint32_t eb) { return stage_bytes / (ea + eb) / 512 * 512; }
+// Stages and stage size of a launch from the options (0 = default), and the dynamic shared memory they need.
+struct StageConfig { uint32_t ns, stage_bytes; size_t smem; };
+constexpr size_t MAX_DYNAMIC_SMEM = 227 * 1024 - 1024;   // a block may have 227 KB; the kernel's static shared memory comes out of it too
 
 // PIECE_COPY: loaded and stored by the bulk unit. PIECE_COPYW: loaded by the bulk unit, stored by the compute
 // warps from shared memory (the stage is free as soon as the warps have read it, without waiting for a
 // bulk store to drain, so more of the stage ring is loads in flight).
 enum : uint32_t { PIECE_COPY = 0, PIECE_REDUCE = 1, PIECE_TILE = 2, PIECE_EXIT = 3, PIECE_COPYW = 4 };
+
+struct alignas(16) PieceInfo;
+StageConfig stage_config(int stages_opt, int stage_kib_opt);
 
 struct alignas(16) PieceInfo {  // one per stage, in shared memory; written by the DMA thread
     uint32_t kind;
@@ -36,6 +44,19 @@ struct alignas(16) PieceInfo {  // one per stage, in shared memory; written by t
     Tile tile;            // PIECE_TILE: the work item and its descriptor for the register path
     Desc desc;
 };
+
+inline StageConfig stage_config(int stages_opt, int stage_kib_opt) {
+    uint32_t sb = stage_kib_opt > 0 ? (uint32_t)stage_kib_opt * 1024u : STAGE_BYTES;
+    sb = sb / 12288u * 12288u;
+    if (sb < MIN_STAGE_BYTES) sb = MIN_STAGE_BYTES;
+    if (sb > MAX_STAGE_BYTES) sb = MAX_STAGE_BYTES;
+    const size_t per = (size_t)sb + sizeof(PieceInfo) + 16, room = MAX_DYNAMIC_SMEM - 128;
+    uint32_t ns = stages_opt > 0 ? (uint32_t)stages_opt : (uint32_t)(4u * STAGE_BYTES / sb);   // default: the same bytes in flight
+    if (ns < 2) ns = 2;
+    if (ns > MAX_STAGES) ns = MAX_STAGES;
+    while (ns > 2 && ns * per > room) --ns;
+    return StageConfig{ns, sb, ns * per + 128};
+}
 
 }  // namespace bulk
 }  // namespace hccl

@@ -42,8 +42,7 @@ hccl_status_t hccl_plan_bind(hccl_plan_t* p, void* dev_workspace, size_t bytes, 
         const size_t smem = RR * 24 + (RR + 1) * 4 + 16;
         if (smem > 48 * 1024) CUDA_TRY(cudaFuncSetAttribute(hccl_a2a_dynamic, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(DYN_MAX_RANKS * DYN_MAX_RANKS * 24 + (DYN_MAX_RANKS * DYN_MAX_RANKS + 1) * 4 + 16)));
     } else if (p->opts.engine == HCCL_ENGINE_BULK) {
-        const size_t smem = (size_t)bulk::MAX_STAGES * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
-        if (smem <= 227 * 1024) CUDA_TRY(cudaFuncSetAttribute(hccl_executor_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)std::min<size_t>(smem, 227 * 1024)));
+        CUDA_TRY(cudaFuncSetAttribute(hccl_executor_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk::MAX_DYNAMIC_SMEM));
     }
     p->workspace = dev_workspace;
     p->workspace_bytes = bytes;
@@ -169,10 +168,9 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
         prm.trig_wait_slot = -1;   // the builder has waited already
         prm.static_tickets = 0;    // how many items are real is known only on the device: tickets and END markers
         if (p->opts.engine == HCCL_ENGINE_BULK) {
-            const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : (int)bulk::MAX_STAGES, 2), (int)bulk::MAX_STAGES);
-            const size_t smem = (size_t)ns * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
-            hccl_executor_bulk<<<blocks, std::max(64, p->opts.threads), smem, (cudaStream_t)stream>>>(
-                prm, ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)));
+            const bulk::StageConfig sc = bulk::stage_config(p->opts.stages, p->opts.stage_kib);
+            hccl_executor_bulk<<<blocks, std::max(96, p->opts.threads), sc.smem, (cudaStream_t)stream>>>(
+                prm, sc.ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)), sc.stage_bytes);
         } else if (p->opts.light) {
             hccl_executor_lsu_light<<<blocks, p->opts.threads, 0, (cudaStream_t)stream>>>(prm);
         } else {
@@ -220,10 +218,10 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     const uint32_t epoch = p->epoch + 1;
     const int blocks = fill_params(p, prm, sendbufs, recvbufs);
     if (p->opts.engine == HCCL_ENGINE_BULK) {
-        const uint32_t ns = (uint32_t)std::min<int>(std::max<int>(p->opts.stages > 0 ? p->opts.stages : (int)bulk::MAX_STAGES, 2), (int)bulk::MAX_STAGES);
-        const size_t smem = (size_t)ns * (bulk::STAGE_BYTES + sizeof(bulk::PieceInfo) + 16) + 128;
-        const int threads = std::max(64, p->opts.threads);
-        hccl_executor_bulk<<<blocks, threads, smem, (cudaStream_t)stream>>>(prm, ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)));
+        const bulk::StageConfig sc = bulk::stage_config(p->opts.stages, p->opts.stage_kib);
+        const int threads = std::max(96, p->opts.threads);
+        hccl_executor_bulk<<<blocks, threads, sc.smem, (cudaStream_t)stream>>>(prm, sc.ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)),
+                                                                              sc.stage_bytes);
     } else {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)blocks);

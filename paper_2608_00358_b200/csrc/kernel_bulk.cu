@@ -4,21 +4,25 @@
 
 namespace hccl {
 
-__global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t copy_by_warps) {
+__global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t copy_by_warps,
+                                                              const uint32_t stage_bytes) {
     using namespace bulk;
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ Prepared s_queue[QUEUE];
+    __shared__ __align__(8) unsigned long long s_qbar[2 * QUEUE + 1];  // q_full[QUEUE], q_empty[QUEUE], control thread has left
     char* stages_ptr = reinterpret_cast<char*>(smem_raw);
-    PieceInfo* info = reinterpret_cast<PieceInfo*>(stages_ptr + (size_t)ns * STAGE_BYTES);
+    PieceInfo* info = reinterpret_cast<PieceInfo*>(stages_ptr + (size_t)ns * stage_bytes);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(info + ns);  // full[ns], empty[ns]
     const uint32_t tid = threadIdx.x;
-    const uint32_t ncw = (blockDim.x >> 5) - 1;  // compute warps
+    const uint32_t ncw = (blockDim.x >> 5) - 2;  // compute warps: all but the DMA warp and the control warp
     const uint32_t full = smem_u32(bars), empty = smem_u32(bars + ns);
-    // entry: first ticket, its tile record, the abort word and the execution number are loaded together
+    const uint32_t q_full = smem_u32(s_qbar), q_empty = smem_u32(s_qbar + QUEUE), ctl_left = smem_u32(s_qbar + 2 * QUEUE);
+    // entry (control thread): first ticket, its tile record, the abort word and the execution number are loaded together
     uint32_t next0 = 0, abort0 = 0;
     Tile pre;
     bool pre_ok = false;
     const bool gated = p.trig_wait_slot >= 0;
-    if (tid == 0) {
+    if (tid == 32) {
         if (!gated) {
             next0 = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
             if (next0 < p.n_tiles) {
@@ -34,15 +38,71 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             mbar_init(full + 8 * s, 1);
             mbar_init(empty + 8 * s, ncw);
         }
+        for (uint32_t q = 0; q < 2 * QUEUE + 1; ++q) mbar_init(q_full + 8 * q, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
     __syncthreads();
+    const unsigned long long long_wait = 2 * p.timeout_ns + 1000000000ull;
+
+    if (tid >= 32 && tid < 64) {
+        // ------------------------------------------------------------ control thread
+        if (tid != 32) return;
+        bool live = true;
+        uint32_t cur = next0;
+        if (gated) {
+            live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value + (unsigned long long)g_epoch * p.trig_wait_per_epoch, 0xffffffffu);
+            cur = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
+        }
+        if (cur == 0) p.ctl->t_first_ns = globaltimer_ns();
+        uint32_t qs = 0, qpar = 0;      // ring position of the next hand-over, phase parity of its barriers
+        unsigned long long pushed = 0;
+        // hand one record to the DMA thread; false if the DMA thread no longer takes any (failure or abort)
+        auto push = [&](uint32_t kind, uint32_t item, const Tile* t, const Desc* ds) -> bool {
+            if (pushed >= QUEUE && !mbar_wait(p, q_empty + 8 * qs, qpar ^ 1u, long_wait, 0xfffffffbu)) return false;
+            Prepared& e = s_queue[qs];
+            e.kind = kind;
+            e.item = item;
+            if (t) {
+                e.t = *t;
+                e.ds = *ds;
+                e.waited = t->wait_cnt;
+            }
+            mbar_arrive(q_full + 8 * qs);  // release: the record is written
+            ++pushed;
+            if (++qs == QUEUE) {
+                qs = 0;
+                qpar ^= 1u;
+            }
+            return true;
+        };
+        bool first = true, consumer_alive = true;
+        while (live) {
+            if (cur >= p.n_tiles || (first && !gated ? abort0 == g_epoch : aborted(p))) break;
+            // the next ticket is claimed before this item's records are waited for: its latency hides behind them
+            const uint32_t next = p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
+            Tile t;
+            Desc ds;
+            const int what = control_item(p, cur, first && pre_ok ? &pre : nullptr, t, ds);
+            first = false;
+            if (what == 0) break;
+            if (what == 2 && !push(Q_ITEM, cur, &t, &ds)) {
+                consumer_alive = false;
+                break;
+            }
+            cur = next;
+        }
+        if (consumer_alive) push(Q_STOP, 0xffffffffu, nullptr, nullptr);
+        mbar_arrive(ctl_left);  // no ticket is claimed after this
+        return;
+    }
 
     if (tid < 32) {
-        if (tid != 0) return;  // one elected thread drives the DMA warp
+        // ------------------------------------------------------------ DMA thread
+        if (tid != 0) return;
         Dma d;
         d.ns = ns;
+        d.sb = stage_bytes;
         d.lag = copy_by_warps ? ns : (ns > 2 ? ns - 2 : 1);
         d.copy_by_warps = copy_by_warps != 0;
         d.stages = smem_u32(stages_ptr);
@@ -51,52 +111,85 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         d.empty = empty;
         d.info = info;
         d.head = d.tail = d.groups = 0;
+        d.head_slot = d.head_par = d.tail_slot = d.tail_par = 0;
         d.pol = policy_evict_first();
         d.pol_keep = policy_evict_last();
         d.ok = true;
-        bool live = true;
-        uint32_t next = next0;
-        if (gated) {
-            live = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value + (unsigned long long)g_epoch * p.trig_wait_per_epoch, 0xffffffffu);
-            next = p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
-        }
-        if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
-        bool first = true;
-        while (live && d.ok) {
-            const uint32_t cur = next;
-            if (cur >= p.n_tiles || (first && !gated ? abort0 == g_epoch : aborted(p))) break;
-            next = p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
-            if (!dma_item(p, d, cur, first && pre_ok ? &pre : nullptr)) break;
-            first = false;
+        uint32_t qs = 0, qpar = 0;
+        while (d.ok) {
+            // next prepared item; while there is none, what is in flight is retired (a COPY item is published when
+            // its last piece retires, and the control thread may be waiting for exactly that)
+            bool got = mbar_try_wait(q_full + 8 * qs, qpar);
+            if (!got) {
+                const unsigned long long deadline = globaltimer_ns() + long_wait;
+                uint32_t spins = 0;
+                while (!(got = mbar_try_wait(q_full + 8 * qs, qpar))) {
+                    if (d.tail < d.head) {
+                        retire_one(p, d);
+                        if (!d.ok) break;
+                        continue;
+                    }
+                    if ((++spins & 31u) == 0) {
+                        if (aborted(p)) break;
+                        if (globaltimer_ns() > deadline) {
+                            fail(p, HCCL_ERR_TIMEOUT, 0xfffffffau);
+                            break;
+                        }
+                    }
+                }
+            }
+            if (!got) break;
+            const Prepared& e = s_queue[qs];
+            if (e.kind == Q_STOP) break;
+            const uint32_t cur = e.item;
+            const Tile t = e.t;
+            const Desc ds = e.ds;
+            const bool waited = e.waited != 0;
+            mbar_arrive(q_empty + 8 * qs);  // the record is in registers: its place may be refilled
+            if (++qs == QUEUE) {
+                qs = 0;
+                qpar ^= 1u;
+            }
+            if (waited) fence_proxy_async();  // what the control thread's acquired counters cover must be visible to the bulk unit too
+            if (!dma_issue(p, d, cur, t, ds)) break;
         }
         // wind down: finish what is in flight, release the compute warps, leave
         if (d.ok && !aborted(p)) drain(p, d);
         if (d.ok && !aborted(p)) {
             const unsigned long long kx = d.head;
+            const uint32_t xslot = d.head_slot, xpar = d.head_par;
             issue_simple(p, d, PIECE_EXIT, 0xffffffffu, nullptr, nullptr);
             // every compute warp has passed the exit piece = all of this block's results are stored
-            if (d.ok && d.head == kx + 1)
-                mbar_wait(p, empty + 8 * (uint32_t)(kx % ns), (uint32_t)((kx / ns) & 1), 2 * p.timeout_ns + 1000000000ull, 0xfffffffcu);
+            if (d.ok && d.head == kx + 1) mbar_wait(p, empty + 8 * xslot, xpar, long_wait, 0xfffffffcu);
         }
         if (!d.ok || aborted(p)) {
             // stop path: no load may still be writing into this block's shared memory when it exits
+            uint32_t slot = d.tail_slot, par = d.tail_par;
             for (unsigned long long j = d.tail; j < d.head; ++j) {
-                const uint32_t slot = (uint32_t)(j % ns);
                 if (info[slot].kind == PIECE_COPY || info[slot].kind == PIECE_REDUCE || info[slot].kind == PIECE_COPYW)
-                    mbar_wait(p, full + 8 * slot, (uint32_t)((j / ns) & 1), 1000000000ull, 0xfffffffeu);
+                    mbar_wait(p, full + 8 * slot, par, 1000000000ull, 0xfffffffeu);
+                if (++slot == ns) {
+                    slot = 0;
+                    par ^= 1u;
+                }
             }
         }
         bulk_wait_all();
-        // the compute warps must be out of the stages before the block's verdict is given
+        // the control thread must have claimed its last ticket before the block's verdict is given (the last block
+        // out resets the ticket); on the stop path it notices the abort within a few polls
+        {
+            const unsigned long long deadline = globaltimer_ns() + 2 * long_wait;
+            while (!mbar_try_wait(ctl_left, 0) && globaltimer_ns() < deadline) {
+            }
+        }
         leave(p, p.trig_set_slot < 0);
         return;
     }
 
     // ------------------------------------------------------------ compute warps
-    const uint32_t ctid = tid - 32, cnth = ncw * 32;
+    const uint32_t ctid = tid - 64, cnth = ncw * 32;
     const unsigned long long pol_keep = policy_evict_last();
-    for (unsigned long long k = 0;; ++k) {
-        const uint32_t slot = (uint32_t)(k % ns), parity = (uint32_t)((k / ns) & 1);
+    for (uint32_t slot = 0, parity = 0;;) {
         if (!mbar_wait(p, full + 8 * slot, parity, 2 * p.timeout_ns + 1000000000ull, 0xfffffffdu)) break;
         const PieceInfo& pi = info[slot];
         const uint32_t kind = pi.kind;
@@ -106,8 +199,8 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             break;
         }
         if (kind == PIECE_REDUCE) {
-            reduce_piece_dispatch(pi.dt_a, pi.dt_b, pi.dt_d, stages_ptr + (size_t)slot * STAGE_BYTES,
-                                  stages_ptr + (size_t)slot * STAGE_BYTES + pi.b_off, pi.dst, pi.n, ctid, cnth, pi.keep_dst != 0, pol_keep);
+            reduce_piece_dispatch(pi.dt_a, pi.dt_b, pi.dt_d, stages_ptr + (size_t)slot * stage_bytes,
+                                  stages_ptr + (size_t)slot * stage_bytes + pi.b_off, pi.dst, pi.n, ctid, cnth, pi.keep_dst != 0, pol_keep);
             if (pi.discard_src) {
                 // whole 128-byte lines inside the piece; issued before the item is published, so the slot's next
                 // writer is ordered after them
@@ -115,7 +208,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
                 for (uintptr_t a = lo + (uintptr_t)ctid * 128u; a < hi; a += (uintptr_t)cnth * 128u) discard_line((const void*)a);
             }
         } else if (kind == PIECE_COPYW) {
-            const uint4* src = reinterpret_cast<const uint4*>(stages_ptr + (size_t)slot * STAGE_BYTES);
+            const uint4* src = reinterpret_cast<const uint4*>(stages_ptr + (size_t)slot * stage_bytes);
             uint4* dst = reinterpret_cast<uint4*>(pi.dst);
             const uint32_t nv = pi.n >> 4;
             const bool stream = pi.evict_first != 0;
@@ -152,16 +245,28 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             run_tile_lsu(p, pi.desc, pi.tile, ctid, cnth);
         }
         if (kind != PIECE_COPY && pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.tile_index, 3, globaltimer_ns());
-        if (kind != PIECE_COPY && pi.last && (pi.signal[0] >= 0 || pi.signal[1] >= 0)) {
-            asm volatile("bar.sync 1, %0;" ::"r"(cnth) : "memory");  // every compute warp has stored its share
-            if (ctid == 0) {  // release, cumulative over the stores the barrier ordered before this thread
-                if (pi.signal[0] >= 0) red_release_add_u32(p.counters + pi.signal[0], 1);
-                if (pi.signal[1] >= 0) red_release_add_u32(p.counters + pi.signal[1], 1);
+        const int32_t sig0 = pi.signal[0], sig1 = pi.signal[1];
+        if (kind != PIECE_COPY && pi.last && (sig0 >= 0 || sig1 >= 0)) {
+            // The item's completion is published by the first compute warp once every compute warp has stored its
+            // share: the others only arrive at the stage's named barrier and go on to the next piece; the release
+            // is cumulative over the stores that the barrier ordered before the publishing thread. One barrier per
+            // stage, since a stage is recycled only after every warp, the publishing one included, has left it.
+            if (ctid < 32) {
+                asm volatile("bar.sync %0, %1;" ::"r"(1u + slot), "r"(cnth) : "memory");
+                if (ctid == 0) {
+                    if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
+                    if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
+                }
+            } else {
+                asm volatile("bar.arrive %0, %1;" ::"r"(1u + slot), "r"(cnth) : "memory");
             }
-            asm volatile("bar.sync 1, %0;" ::"r"(cnth) : "memory");  // the stage's info is read before it is recycled
         }
         __syncwarp();
         if ((tid & 31u) == 0) mbar_arrive(empty + 8 * slot);
+        if (++slot == ns) {
+            slot = 0;
+            parity ^= 1u;
+        }
     }
 }
 
