@@ -169,7 +169,7 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
         prm.static_tickets = 0;    // how many items are real is known only on the device: tickets and END markers
         if (p->opts.engine == HCCL_ENGINE_BULK) {
             const bulk::StageConfig sc = bulk::stage_config(p->opts.stages, p->opts.stage_kib);
-            hccl_executor_bulk<<<blocks, std::max(96, p->opts.threads), sc.smem, (cudaStream_t)stream>>>(
+            hccl_executor_bulk<<<blocks, std::max(128, p->opts.threads), sc.smem, (cudaStream_t)stream>>>(
                 prm, sc.ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)), sc.stage_bytes);
         } else if (p->opts.light) {
             hccl_executor_lsu_light<<<blocks, p->opts.threads, 0, (cudaStream_t)stream>>>(prm);
@@ -219,7 +219,7 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     const int blocks = fill_params(p, prm, sendbufs, recvbufs);
     if (p->opts.engine == HCCL_ENGINE_BULK) {
         const bulk::StageConfig sc = bulk::stage_config(p->opts.stages, p->opts.stage_kib);
-        const int threads = std::max(96, p->opts.threads);
+        const int threads = std::max(128, p->opts.threads);
         hccl_executor_bulk<<<blocks, threads, sc.smem, (cudaStream_t)stream>>>(prm, sc.ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)),
                                                                               sc.stage_bytes);
     } else {

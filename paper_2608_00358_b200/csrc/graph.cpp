@@ -85,8 +85,8 @@ void hccl::fill_default_opts(hccl_opts_t* o, const hccl_opts_t* in) {
     if (o->timeout_ns == 0) o->timeout_ns = 2000000000ull;
     if (o->chain_group <= 0) o->chain_group = 16;
     if (o->rack_size <= 0) o->rack_size = 16;
-    if (o->threads <= 0) o->threads = o->engine == HCCL_ENGINE_BULK ? 320 : 512;  // bulk: DMA warp + control warp + 8 compute warps; register: control warp + 15 workers
-    o->threads = std::min(512, std::max(o->engine == HCCL_ENGINE_BULK ? 96 : 64, (o->threads + 31) / 32 * 32));  // the service warps + at least one worker warp
+    if (o->threads <= 0) o->threads = o->engine == HCCL_ENGINE_BULK ? 352 : 512;  // bulk: DMA, control and publishing warps + 8 compute warps; register: control warp + 15 workers
+    o->threads = std::min(512, std::max(o->engine == HCCL_ENGINE_BULK ? 128 : 64, (o->threads + 31) / 32 * 32));  // the service warps + at least one worker warp
 }
 
 extern "C" {

@@ -14,7 +14,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
     PieceInfo* info = reinterpret_cast<PieceInfo*>(stages_ptr + (size_t)ns * stage_bytes);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(info + ns);  // full[ns], empty[ns]
     const uint32_t tid = threadIdx.x;
-    const uint32_t ncw = (blockDim.x >> 5) - 2;  // compute warps: all but the DMA warp and the control warp
+    const uint32_t ncw = (blockDim.x >> 5) - 3;  // compute warps: all but the DMA, control and publishing warps
     const uint32_t full = smem_u32(bars), empty = smem_u32(bars + ns);
     const uint32_t q_full = smem_u32(s_qbar), q_empty = smem_u32(s_qbar + QUEUE), ctl_left = smem_u32(s_qbar + 2 * QUEUE);
     // entry (control thread): first ticket, its tile record, the abort word and the execution number are loaded together
@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
     if (tid == 0) {
         for (uint32_t s = 0; s < ns; ++s) {
             mbar_init(full + 8 * s, 1);
-            mbar_init(empty + 8 * s, ncw);
+            mbar_init(empty + 8 * s, ncw + 1);   // every compute warp and the publishing warp
         }
         for (uint32_t q = 0; q < 2 * QUEUE + 1; ++q) mbar_init(q_full + 8 * q, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -186,8 +186,40 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
         return;
     }
 
+    const uint32_t cnth = ncw * 32;
+    if (tid >= 64 && tid < 96) {
+        // ------------------------------------------------------------ publishing warp
+        // Follows the pieces like a compute warp but moves no data: after the last piece of an item it waits at
+        // the stage's named barrier until every compute warp has stored its share, and its first lane publishes
+        // the item's completion. The release has to wait for those stores to be performed, a microsecond or
+        // two that no data-moving warp spends this way. The release is cumulative over the stores that the barrier
+        // ordered before the publishing thread. One barrier per stage: a stage is recycled only after every warp,
+        // this one included, has left it, so a barrier never sees two items at once.
+        for (uint32_t slot = 0, parity = 0;;) {
+            if (!mbar_wait(p, full + 8 * slot, parity, long_wait, 0xfffffff9u)) break;
+            const PieceInfo& pi = info[slot];
+            const uint32_t kind = pi.kind, last = pi.last;
+            const int32_t sig0 = pi.signal[0], sig1 = pi.signal[1];
+            if (kind != PIECE_EXIT && kind != PIECE_COPY && last && (sig0 >= 0 || sig1 >= 0)) {
+                asm volatile("bar.sync %0, %1;" ::"r"(1u + slot), "r"(cnth + 32u) : "memory");
+                if (tid == 64) {
+                    if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
+                    if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
+                }
+            }
+            __syncwarp();
+            if (tid == 64) mbar_arrive(empty + 8 * slot);
+            if (kind == PIECE_EXIT) break;
+            if (++slot == ns) {
+                slot = 0;
+                parity ^= 1u;
+            }
+        }
+        return;
+    }
+
     // ------------------------------------------------------------ compute warps
-    const uint32_t ctid = tid - 64, cnth = ncw * 32;
+    const uint32_t ctid = tid - 96;
     const unsigned long long pol_keep = policy_evict_last();
     for (uint32_t slot = 0, parity = 0;;) {
         if (!mbar_wait(p, full + 8 * slot, parity, 2 * p.timeout_ns + 1000000000ull, 0xfffffffdu)) break;
@@ -245,22 +277,9 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             run_tile_lsu(p, pi.desc, pi.tile, ctid, cnth);
         }
         if (kind != PIECE_COPY && pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.tile_index, 3, globaltimer_ns());
-        const int32_t sig0 = pi.signal[0], sig1 = pi.signal[1];
-        if (kind != PIECE_COPY && pi.last && (sig0 >= 0 || sig1 >= 0)) {
-            // The item's completion is published by the first compute warp once every compute warp has stored its
-            // share: the others only arrive at the stage's named barrier and go on to the next piece; the release
-            // is cumulative over the stores that the barrier ordered before the publishing thread. One barrier per
-            // stage, since a stage is recycled only after every warp, the publishing one included, has left it.
-            if (ctid < 32) {
-                asm volatile("bar.sync %0, %1;" ::"r"(1u + slot), "r"(cnth) : "memory");
-                if (ctid == 0) {
-                    if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
-                    if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
-                }
-            } else {
-                asm volatile("bar.arrive %0, %1;" ::"r"(1u + slot), "r"(cnth) : "memory");
-            }
-        }
+        // the publishing warp waits at the stage's barrier for every compute warp's stores of an item's last piece
+        if (kind != PIECE_COPY && pi.last && (pi.signal[0] >= 0 || pi.signal[1] >= 0))
+            asm volatile("bar.arrive %0, %1;" ::"r"(1u + slot), "r"(cnth + 32u) : "memory");
         __syncwarp();
         if ((tid & 31u) == 0) mbar_arrive(empty + 8 * slot);
         if (++slot == ns) {

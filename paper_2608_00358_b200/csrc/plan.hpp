@@ -92,7 +92,7 @@ inline int64_t sweep_of(const hccl_opts_t& o, int op) {
     if (o.engine == HCCL_ENGINE_BULK) {
         if (op == HCCL_OP_COPY) return 49152;                 // one stage
         if (op == HCCL_OP_REDUCE) return 24576;               // whole pieces for every operand mix (6144, 8192, 12288)
-        return (int64_t)(o.threads - 64) * 8;                 // multi-input sums run on the compute warps
+        return (int64_t)(o.threads - 96) * 8;                 // multi-input sums run on the compute warps
     }
     const int64_t workers = o.threads - 32;
     if (op == HCCL_OP_COPY) return workers * 128;             // 8 x 16 bytes per thread
