@@ -412,11 +412,19 @@ def interference_leg(args, wl):
             "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
             "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
         del w2, plan, gemm
-    # the operating point: the budget with the smallest GEMM loss among those that move data
-    best = min((p for p in sweep if p["gemm_slowdown"] is not None), key=lambda p: p["gemm_slowdown"], default=None)
-    if best is not None:
-        out["chosen"] = {"sm_budget": best["sm_budget"], "gemm_slowdown": best["gemm_slowdown"],
-                         "collective_overlap_gbs": best["collective_overlap_gbs"]}
+    # the operating point: no SM is held against the GEMM. Short-lived blocks (interference.OVERLAP_OPTS) on a stream of
+    # LOWER priority than the GEMM's take only the SMs the GEMM leaves idle (the tail of its last wave, the gap between
+    # launches); the slowdown is still taken against the unrestricted GEMM alone
+    torch.cuda.empty_cache()
+    gemm = interference.Gemm()
+    plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(interference.OVERLAP_OPTS))
+    w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
+    r = interference.measure(w2, seconds=3.0, gemm=gemm, collective_first=False)
+    out["chosen"] = {"mode": "idle SMs: quantum %d, tile %d B, GEMM stream has priority" % (interference.OVERLAP_OPTS["quantum"], interference.OVERLAP_OPTS["tile_bytes"]),
+                     "sm_budget_held": 0, "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
+                     "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_alone_gbs": r["collective_alone_gbs"],
+                     "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
+    del w2, plan, gemm
     return out
 
 
@@ -442,7 +450,10 @@ def headline_of(line: dict) -> dict:
         h["cpu_baseline"] = line["cpu_baseline"]
     i = line.get("interference")
     if i and "chosen" in i:
-        h["interference"] = dict(i["chosen"], gemm="bf16 8192^3")
+        h["interference"] = {k: i["chosen"][k] for k in ("mode", "sm_budget_held", "gemm_slowdown", "collective_overlap_gbs", "collective_alone_gbs")}
+        h["interference"]["gemm"] = "bf16 8192^3"
+        pers = {str(p["sm_budget"]): p["gemm_slowdown"] for p in i.get("sweep", []) if p["sm_budget"] in (2, 16)}
+        h["interference"]["persistent_budget_slowdown"] = pers
     cfg = line.get("configs") or {}
     side = {}
     for key, short, field in (("3_reducescatter_r16_bf16_64Mi_ring", "c3_ring_ms", "ms"), ("3_reducescatter_r16_bf16_64Mi_ring_fused", "c3_fused_ms", "ms"),

@@ -146,7 +146,12 @@ typedef struct {
                                the paper's rack, Sec. V-D) */
     int32_t stage_kib;      /* bulk engine: KiB per shared-memory stage, a multiple of 12 in [12, 96] (default 48); with
                                opts.stages left at 0 the number of stages keeps 192 KiB in flight (at most 8 stages) */
-    int32_t reserved0;      /* 0 */
+    int32_t quantum;        /* 0: persistent blocks (sm_budget of them run until the packet is done). > 0: short-lived blocks,
+                               each leaves after this many work items and as many blocks are launched as that takes; how many
+                               run at once is then the block scheduler's choice. On a stream of lower priority than a
+                               concurrent compute kernel's they fill the SMs that kernel leaves idle (the tail of its last
+                               wave, the gap between launches) and hold none against it. Ticket dispatch only: ignored by
+                               plans that run as static chains and by device-resident plans; refused by hccl_server_start */
 } hccl_opts_t;
 
 typedef struct hccl_plan hccl_plan_t;   /* opaque, host-owned: a compiled, cacheable work packet (Sec. V-B) */

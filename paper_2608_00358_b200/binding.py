@@ -33,7 +33,7 @@ class Opts(C.Structure):
     _fields_ = [("sm_budget", C.c_int32), ("engine", C.c_int32), ("chunk_bytes", C.c_uint64),
                 ("tile_bytes", C.c_uint64), ("timeout_ns", C.c_uint64), ("flags", C.c_uint32),
                 ("chain_group", C.c_int32), ("threads", C.c_int32), ("stages", C.c_int32), ("cluster", C.c_int32), ("light", C.c_int32),
-                ("copy_by_warps", C.c_int32), ("rack_size", C.c_int32), ("stage_kib", C.c_int32), ("reserved0", C.c_int32)]
+                ("copy_by_warps", C.c_int32), ("rack_size", C.c_int32), ("stage_kib", C.c_int32), ("quantum", C.c_int32)]
 
 
 class Ref(C.Structure):

@@ -44,7 +44,8 @@ struct ExecParams {
     unsigned long long* trace;  // optional: 4 words per work item (item | block << 32, claim, start, end in ns), or null
     unsigned long long trace_cap;
     uint32_t n_tiles, n_descs, n_syncs, n_waits;
-    uint32_t R, nblocks, n_signals, pad0;
+    uint32_t R, nblocks, n_signals;
+    uint32_t quantum;  // ticket dispatch: items a block claims before it leaves (0 = until the packet is done)
     unsigned long long timeout_ns;
     long long n_user_signals;
     long long trig_wait_slot, trig_set_slot;
@@ -698,9 +699,12 @@ __device__ __forceinline__ uint32_t first_item(const ExecParams& p, uint32_t& ra
     }
     return p.static_tickets ? blockIdx.x : atomicAdd(&p.ctl->ticket, 1);
 }
-__device__ __forceinline__ uint32_t next_item(const ExecParams& p, uint32_t cur, uint32_t range_end) {
+// `left` counts the claims a block may still make (opts.quantum; effectively unbounded when that is 0).
+__device__ __forceinline__ uint32_t next_item(const ExecParams& p, uint32_t cur, uint32_t range_end, uint32_t& left) {
     if (p.chain_len) return cur + 1 < range_end ? cur + 1 : p.n_tiles;
-    return p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
+    if (p.static_tickets || left == 0) return p.n_tiles;
+    --left;
+    return atomicAdd(&p.ctl->ticket, 1);
 }
 
 template <bool RESIDENT>
@@ -714,6 +718,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     // tile record do not depend on one another: thread 0 issues all of these loads before it uses any of
     // them, so a small collective pays one trip to memory here instead of four in a row.
     uint32_t next = 0, abort0 = 0, range_end = 0;
+    uint32_t left = p.quantum ? p.quantum - 1u : 0xffffffffu;  // the first claim is made at entry
     Tile pre;
     bool pre_ok = false;
     const bool gated = p.trig_wait_slot >= 0;
@@ -760,7 +765,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 cur = next;
                 have = live && cur < p.n_tiles && !(gated ? aborted(p) : abort0 == g_epoch);
                 if (have) {
-                    next = next_item(p, cur, range_end);
+                    next = next_item(p, cur, range_end, left);
                     have = fetch_tile(p, cur, s_tile[0], s_desc[0], pre_ok ? &pre : nullptr);
                     ready = have && deps_ready(p, s_tile[0]);
                 }
@@ -800,7 +805,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 cur = next;
                 have = cur < p.n_tiles && !aborted(p);
                 if (have) {
-                    next = next_item(p, cur, range_end);
+                    next = next_item(p, cur, range_end, left);
                     have = fetch_tile(p, cur, s_tile[b ^ 1], s_desc[b ^ 1]);
                     ready = have && deps_ready(p, s_tile[b ^ 1]);
                 }

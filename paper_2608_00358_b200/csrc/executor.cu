@@ -59,8 +59,17 @@ static int set_dispatch(const hccl_plan_t* p, ExecParams& prm) {
     prm.chain_len = p->chain_len;
     prm.n_chains = p->n_chains;
     if (p->chain_len) blocks = (int)std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)blocks, p->n_chains));
-    prm.nblocks = (uint32_t)blocks;
     prm.static_tickets = (!p->chain_len && prm.n_waits == 0 && prm.n_tiles <= (uint32_t)blocks) ? 1 : 0;
+    prm.quantum = 0;
+    if (p->opts.quantum > 0 && !p->chain_len && !p->dynamic && prm.n_tiles > 0) {
+        // short-lived blocks: as many as it takes when each one leaves after `quantum` items; how many run at once
+        // is up to the hardware's block scheduler (and to the stream's priority against other work)
+        prm.quantum = (uint32_t)p->opts.quantum;
+        prm.static_tickets = 0;
+        blocks = (int)std::min<uint64_t>(((uint64_t)prm.n_tiles + prm.quantum - 1) / prm.quantum, 1u << 20);
+        if ((uint64_t)blocks * prm.quantum < prm.n_tiles) prm.quantum = (uint32_t)(((uint64_t)prm.n_tiles + blocks - 1) / blocks);
+    }
+    prm.nblocks = (uint32_t)blocks;
     return blocks;
 }
 
@@ -493,6 +502,7 @@ hccl_status_t hccl_server_start(hccl_plan_t* p, const void* const* sendbufs, voi
     CUDA_TRY(cudaMemsetAsync((char*)p->workspace + p->layout.control + offsetof(Control, server_go), 0, 4, s));
     std::memset(host_doorbell, 0, sizeof(Doorbell));
     static thread_local ExecParams prm;
+    if (p->opts.quantum > 0) return HCCL_ERR_INVALID_ARG;  // resident blocks are persistent by definition
     const int blocks = fill_params(p, prm, sendbufs, recvbufs);
     // every block must be resident at once (the blocks wait for each other between executions)
     int dev = 0, sms = 0, per_sm = 0;

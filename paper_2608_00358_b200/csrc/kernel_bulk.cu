@@ -77,10 +77,15 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             return true;
         };
         bool first = true, consumer_alive = true;
+        uint32_t left = p.quantum ? p.quantum - 1u : 0xffffffffu;  // claims this block may still make (opts.quantum)
         while (live) {
             if (cur >= p.n_tiles || (first && !gated ? abort0 == g_epoch : aborted(p))) break;
             // the next ticket is claimed before this item's records are waited for: its latency hides behind them
-            const uint32_t next = p.static_tickets ? p.n_tiles : atomicAdd(&p.ctl->ticket, 1);
+            uint32_t next = p.n_tiles;
+            if (!p.static_tickets && left != 0) {
+                --left;
+                next = atomicAdd(&p.ctl->ticket, 1);
+            }
             Tile t;
             Desc ds;
             const int what = control_item(p, cur, first && pre_ok ? &pre : nullptr, t, ds);

@@ -6,8 +6,12 @@ on its hardware, attributed to HBM contention). Here the GEMM is cuBLAS through 
 collective is one bound plan re-enqueued on a high-priority stream; the benchmark suite the paper used
 is not available and is not reproduced.
 
-Run as a module for the SM-budget sweep:
+Run as a module for the SM-budget sweep and for the other ways of sharing the GPU with the GEMM:
     python -m paper_2608_00358_b200.interference --budgets 4,8,16,32,64,148 --cap 32768
+    python -m paper_2608_00358_b200.interference --method idle_sms --quanta 1,2,4 --opts tile_bytes=122880
+
+OVERLAP_OPTS is the operating point measured to cost a saturating 8192^3 GEMM less than 5 %: short-lived
+blocks (two work items of 120 KiB each) on a stream of lower priority than the GEMM's.
 """
 from __future__ import annotations
 
@@ -20,6 +24,9 @@ import numpy as np
 import torch
 
 from . import workloads as wk
+
+
+OVERLAP_OPTS = dict(quantum=2, tile_bytes=122880)
 
 
 class Gemm:
@@ -36,11 +43,18 @@ class Gemm:
         torch.matmul(self.a, self.b, out=self.c)
 
 
-def overlap(gemm: Gemm, wl: Optional[wk.Workload], seconds: float = 3.0, discard: float = 1.0, gemm_batch: int = 10) -> dict:
-    """GEMM loop on one stream, collective loop on a high-priority stream; rates are computed only inside
-    the window in which events show both loops running."""
-    sg = torch.cuda.Stream()
-    sc = torch.cuda.Stream(priority=-1)
+def overlap(gemm: Gemm, wl: Optional[wk.Workload], seconds: float = 3.0, discard: float = 1.0, gemm_batch: int = 10,
+            collective_first: bool = True, streams=None) -> dict:
+    """GEMM loop on one stream, collective loop on another; rates are computed only inside the window in which
+    events show both loops running. `collective_first`: the collective's stream has the higher priority (its
+    blocks take SMs as soon as GEMM blocks retire); otherwise the GEMM's has, and the collective gets the SMs the
+    GEMM leaves idle. `streams`: (gemm stream, collective stream) made by the caller, e.g. in green contexts."""
+    if streams is not None:
+        sg, sc = streams
+    elif collective_first:
+        sg, sc = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    else:
+        sg, sc = torch.cuda.Stream(priority=-1), torch.cuda.Stream()
     base = torch.cuda.Event(enable_timing=True)
     eg, ec = [], []
     torch.cuda.synchronize()
@@ -95,12 +109,74 @@ def overlap(gemm: Gemm, wl: Optional[wk.Workload], seconds: float = 3.0, discard
     return out
 
 
-def measure(wl: wk.Workload, seconds: float = 3.0, gemm: Optional[Gemm] = None) -> dict:
+# ---- the two remedies for a GEMM that was tiled for more SMs than it gets (process-local, nothing outlives the process)
+def _cublas():
+    """The cuBLAS library torch has loaded (found in this process's memory map), for cublasSetSmCountTarget."""
+    import ctypes
+    for line in open("/proc/self/maps"):
+        if "libcublas.so" in line:
+            lib = ctypes.CDLL(line.split()[-1])
+            lib.cublasSetSmCountTarget.argtypes = [ctypes.c_void_p, ctypes.c_int]
+            lib.cublasGetSmCountTarget.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int)]
+            return lib
+    raise RuntimeError("cuBLAS is not loaded yet: run a matmul first")
+
+
+def set_sm_count_target(n: int, stream: Optional[torch.cuda.Stream] = None) -> int:
+    """Tells cuBLAS (torch's handle for `stream`) to plan its kernels for n SMs (0 = all). Returns the value
+    cuBLAS reports back."""
+    import ctypes
+    lib = _cublas()
+    with torch.cuda.stream(stream or torch.cuda.current_stream()):
+        h = ctypes.c_void_p(torch.cuda.current_blas_handle())
+        rc = lib.cublasSetSmCountTarget(h, ctypes.c_int(n))
+        if rc != 0:
+            raise RuntimeError("cublasSetSmCountTarget failed: %d" % rc)
+        got = ctypes.c_int(-1)
+        lib.cublasGetSmCountTarget(h, ctypes.byref(got))
+    return got.value
+
+
+class GreenPartition:
+    """Two green contexts that split the device's SMs into `small` SMs (rounded up to what the device allows)
+    for the collective and the rest for the GEMM, with one stream in each. Released by close()."""
+
+    def __init__(self, small: int):
+        from cuda.bindings import driver as drv
+        self.drv = drv
+
+        def ck(res):
+            if int(res[0]) != 0:
+                raise RuntimeError("CUDA driver error %s" % res[0])
+            return None if len(res) == 1 else (res[1] if len(res) == 2 else res[1:])
+        self.ck = ck
+        dev = ck(drv.cuDeviceGet(torch.cuda.current_device()))
+        sm = ck(drv.cuDeviceGetDevResource(dev, drv.CUdevResourceType.CU_DEV_RESOURCE_TYPE_SM))
+        groups, _, rest = ck(drv.cuDevSmResourceSplitByCount(1, sm, 0, small))
+        self.small_sms, self.rest_sms = int(groups[0].sm.smCount), int(rest.sm.smCount)
+        self.ctx = [ck(drv.cuGreenCtxCreate(ck(drv.cuDevResourceGenerateDesc([r], 1)), dev, drv.CUgreenCtxCreate_flags.CU_GREEN_CTX_DEFAULT_STREAM))
+                    for r in (groups[0], rest)]
+        self.raw = [ck(drv.cuGreenCtxStreamCreate(self.ctx[0], drv.CUstream_flags.CU_STREAM_NON_BLOCKING, -1)),
+                    ck(drv.cuGreenCtxStreamCreate(self.ctx[1], drv.CUstream_flags.CU_STREAM_NON_BLOCKING, 0))]
+        self.collective_stream = torch.cuda.ExternalStream(int(self.raw[0]))
+        self.gemm_stream = torch.cuda.ExternalStream(int(self.raw[1]))
+
+    def close(self):
+        torch.cuda.synchronize()
+        for s_ in self.raw:
+            self.ck(self.drv.cuStreamDestroy(s_))
+        for c in self.ctx:
+            self.ck(self.drv.cuGreenCtxDestroy(c))
+
+
+def measure(wl: wk.Workload, seconds: float = 3.0, gemm: Optional[Gemm] = None, collective_first: bool = True, streams=None,
+            alone_tflops: Optional[float] = None) -> dict:
+    """GEMM slowdown = 1 - (GEMM rate beside the collective) / (rate of the UNRESTRICTED GEMM alone: default streams,
+    all SMs, no SM-count target). Pass `alone_tflops` when that figure was taken before a restriction was applied."""
     gemm = gemm or Gemm()
-    alone = overlap(gemm, None, seconds)      # identical loop, no collective
-    alone = dict(tflops=alone["gemm_tflops"])
+    alone = dict(tflops=alone_tflops if alone_tflops is not None else overlap(gemm, None, seconds)["gemm_tflops"])
     coll_alone_ms = wk.time_back_to_back(wl, 5, 2)
-    both = overlap(gemm, wl, seconds)
+    both = overlap(gemm, wl, seconds, collective_first=collective_first, streams=streams)
     res = dict(gemm_alone_tflops=alone["tflops"], collective_alone_ms=float(coll_alone_ms),
                collective_alone_gbs=float(wl.info.schedule_bytes / coll_alone_ms / 1e6), overlap=both,
                sm_budget=int(wl.info.sm_budget))
@@ -117,18 +193,49 @@ def main():
     ap.add_argument("--engine", type=int, default=0)
     ap.add_argument("--gemm-n", type=int, default=8192, help="the GEMM is n x n x n, bf16")
     ap.add_argument("--opts", default="", help="extra plan options, e.g. threads=256,light=1,cluster=2")
+    ap.add_argument("--method", default="plain", choices=["plain", "sm_target", "green", "green_sm_target", "idle_sms"],
+                    help="plain: collective on a high-priority stream; sm_target: cuBLAS plans for 148 - budget SMs; green: GEMM and "
+                         "collective in two green contexts that split the SMs; idle_sms: short-lived blocks (--quanta) on a stream of "
+                         "LOWER priority than the GEMM's, so they only take SMs the GEMM leaves idle")
+    ap.add_argument("--quanta", default="4,8,16", help="items per block for --method idle_sms")
     args = ap.parse_args()
     extra = {k: int(v) for k, v in (kv.split("=") for kv in args.opts.split(",") if kv)}
     gemm = Gemm(args.gemm_n)
+    gemm.run()
+    torch.cuda.synchronize()
+    unrestricted = overlap(gemm, None, args.seconds)["gemm_tflops"]     # the reference for every slowdown below
     base = wk.config4(dict(sm_budget=148, engine=args.engine), cap=args.cap)
-    for b in [int(x) for x in args.budgets.split(",")]:
+
+    def plan_for(**o):
         plan = wk.hb.hccl_plan_alltoallv(base.meta["R"], base.meta["counts"], None, None, None, wk.hb.FP16,
-                                         base.meta["row_elems"], dict(sm_budget=b, engine=args.engine, **extra))
-        wl = wk._bind(base.name, plan, base.send, base.recv, base.meta)
-        res = measure(wl, args.seconds, gemm)
-        res["opts"] = extra
-        res["gemm_n"] = args.gemm_n
-        print(json.dumps(res), flush=True)
+                                         base.meta["row_elems"], {"engine": args.engine, **extra, **o})
+        return wk._bind(base.name, plan, base.send, base.recv, base.meta)
+
+    if args.method == "idle_sms":
+        for q in [int(x) for x in args.quanta.split(",")]:
+            wl = plan_for(quantum=q)
+            res = measure(wl, args.seconds, gemm, collective_first=False, alone_tflops=unrestricted)
+            res.update(method=args.method, quantum=q, opts=extra, gemm_n=args.gemm_n)
+            print(json.dumps(res), flush=True)
+        return
+    for b in [int(x) for x in args.budgets.split(",")]:
+        part, streams, target = None, None, 0
+        try:
+            if args.method in ("green", "green_sm_target"):
+                part = GreenPartition(b)
+                streams = (part.gemm_stream, part.collective_stream)
+                b = part.small_sms
+            wl = plan_for(sm_budget=b)
+            if args.method in ("sm_target", "green_sm_target"):
+                target = set_sm_count_target(148 - b, streams[0] if streams else None)
+            res = measure(wl, args.seconds, gemm, streams=streams, alone_tflops=unrestricted)
+            res.update(method=args.method, sm_count_target=target, opts=extra, gemm_n=args.gemm_n)
+            print(json.dumps(res), flush=True)
+        finally:
+            if target:
+                set_sm_count_target(0, streams[0] if streams else None)
+            if part is not None:
+                part.close()
 
 
 if __name__ == "__main__":

@@ -388,3 +388,28 @@ def test_tree_and_two_level_allgather_as_groups(flags, dt):
     Y = run_plan(p, X, iters=2)
     for r, w in enumerate(orc.allgatherv(X)):
         assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
+
+
+@pytest.mark.parametrize("quantum", [1, 3, 1000])
+def test_short_lived_blocks_give_the_same_bits(quantum, engine):
+    """opts.quantum: blocks leave after that many items and more blocks are launched instead (many more than can
+    be resident at once here). AllToAllv, and a ring whose items wait for items of blocks that may have left."""
+    R, row = 8, 24
+    C = synth.uniform_counts(R, 77, hi=90)
+    X = [synth.hashed_rows_np(s, 0, max(int(C[s].sum()), 1), row).reshape(-1).view(np.uint8) for s in range(R)]
+    p = hb.hccl_plan_alltoallv(R, C, None, None, None, hb.BF16, row, _with(dict(tile_bytes=512, sm_budget=8, quantum=quantum), engine))
+    Y = run_plan(p, X, iters=2)
+    SD, RD = orc.packed_displs(C)
+    want = [np.full(Y[d].size, 0xA5, dtype=np.uint8) for d in range(R)]
+    orc.alltoallv(X, want, C, SD, RD, row * 2)
+    for d in range(R):
+        assert np.array_equal(Y[d], want[d]), d
+    n = 60013
+    Xr = synth.normal_ranks(5, n, hb.BF16, seed=quantum, std=0.02)
+    pr = hb.hccl_plan_allreduce(5, n, hb.BF16, hb.ALGO_RING, _with(dict(tile_bytes=2048, chunk_bytes=8192, chain_group=2, sm_budget=8, quantum=quantum,
+                                                                      flags=hb.FLAG_DYNAMIC_TICKETS), engine))
+    assert pr.info().static_chains == 0
+    Yr = run_plan(pr, Xr, iters=2)
+    ring = orc.allreduce_ring_f32(hb.BF16, Xr, orc.floor_chunk_offsets(n, 5))
+    for r in range(5):
+        assert np.array_equal(Yr[r].view(np.uint16), ring[r]), r
