@@ -360,6 +360,19 @@ def run_profile_case(args):
     import torch
     from paper_2608_00358_b200 import binding as hb
     from paper_2608_00358_b200 import workloads as wk
+    if args.profile_case == "latency":
+        # the small, latency-bound configurations: one JSON line each (see workloads.latency_breakdown)
+        cases = [("1 allreduce ring r4 fp32 1Mi", lambda: wk.config1()), ("2 alltoallv r8 bf16 dim128", lambda: wk.config2())]
+        for m in (4096, 65536, 262144, 1 << 20):
+            cases.append(("5 allreduce r8 bf16 %d B one-shot" % m, lambda m=m: wk.config5(m, hb.ALGO_ONESHOT)))
+            cases.append(("5 allreduce r8 bf16 %d B ring" % m, lambda m=m: wk.config5(m, hb.ALGO_RING)))
+        for name, make in cases:
+            wl = make()
+            print(json.dumps(_round(_finite(dict(case=name, **wk.latency_breakdown(wl))), 2)), flush=True)
+            del wl
+        wl = wk.config5(4096, hb.ALGO_ONESHOT)
+        print(json.dumps(_round(_finite(dict(case="5 allreduce r8 bf16 4096 B one-shot, as the host sees it", **wk.time_host_observed(wl, 300))), 2)), flush=True)
+        return
     if args.profile_case in ("c1chains", "c1tickets"):
         # config 1 (AllReduce ring R = 4, 1 Mi fp32 per rank): static chains vs tickets and device counters
         wl = wk.config1(dict(flags=0 if args.profile_case == "c1chains" else hb.FLAG_DYNAMIC_TICKETS))
@@ -372,7 +385,7 @@ def run_profile_case(args):
         wl = wk._bind("allgather_r32_bf16_1Mi_" + args.profile_case[2:], hb.hccl_plan_allgather(R, None, n, hb.BF16, algo), send, recv, {})
     else:
         algo = {"c3ring": hb.ALGO_RING, "c3fused": hb.ALGO_RING_FUSED}[args.profile_case]
-        wl = wk.config3(algo=algo, n=args.profile_n)
+        wl = wk.config3(dict(chain_group=args.profile_chain_group) if args.profile_chain_group else None, algo=algo, n=args.profile_n)
     ms = wk.time_back_to_back(wl, args.steps, max(args.warmup, 3))
     i = wl.info
     print(json.dumps({"case": args.profile_case, "workload": wl.name, "ms": ms, "schedule_bytes": int(i.schedule_bytes),
@@ -461,7 +474,8 @@ def headline_of(line: dict) -> dict:
                               ("1_allreduce_ring_r4_fp32_1Mi", "c1_p50_us", "p50_us"), ("2_alltoallv_r8_bf16_dim128", "c2_p50_us", "p50_us"),
                               ("5_allreduce_r8_bf16_4096B_oneshot", "c5_4k_oneshot_p50_us", "p50_us"),
                               ("5_allreduce_r8_bf16_1048576B_oneshot", "c5_1m_oneshot_p50_us", "p50_us"),
-                              ("next_alltoallv_dynamic_r64_fp16_dim256", "dyn_r64_ms", "ms")):
+                              ("next_alltoallv_dynamic_r64_fp16_dim256", "dyn_r64_ms", "ms"),
+                              ("next_alltoallv_dynamic_r64_fp16_dim256", "dyn_r64_device_tables_ms", "device_tables_ms")):
         v = (cfg.get(key) or {}).get(field)
         if v is not None:
             side[short] = v
@@ -654,6 +668,15 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             dyn64 = {"ms": float(msd), "gbs": info.schedule_bytes / msd / 1e6, "statically_planned_ms": total_ms_max / args.steps,
                      "note": "counts read from device memory at run time; same payload as the benchmark step"}
             del wd, dyn
+            # the same with descriptors and tiles built on the device and run by the ordinary (bulk) executor: the form
+            # that serves any rank count
+            dyn = hb.hccl_plan_alltoallv_dynamic(64, Cd.sum(axis=1), Cd.sum(axis=0), hb.FP16, 256, dict(flags=hb.FLAG_DEVICE_TABLES))
+            dyn.set_dynamic_metadata(counts_dev.data_ptr())
+            wd = wk._bind("alltoallv_dynamic_r64_device_tables", dyn, wl.send, wl.recv, {})
+            msd = wk.time_back_to_back(wd, 5, 2)
+            dyn64["device_tables_ms"] = float(msd)
+            dyn64["device_tables_gbs"] = info.schedule_bytes / msd / 1e6
+            del wd, dyn
         del wl
         torch.cuda.empty_cache()
         if not args.no_side:
@@ -692,7 +715,8 @@ def main():
     ap.add_argument("--no-side", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--profile-n", type=int, default=1 << 23, help="elements per rank of the --profile-case")
-    ap.add_argument("--profile-case", default="", choices=["", "c3ring", "c3fused", "agfanout", "agoneshot", "c1chains", "c1tickets"],
+    ap.add_argument("--profile-chain-group", type=int, default=0, help="opts.chain_group of the c3ring / c3fused --profile-case (0 = default)")
+    ap.add_argument("--profile-case", default="", choices=["", "c3ring", "c3fused", "agfanout", "agoneshot", "c1chains", "c1tickets", "latency"],
                     help="run only a small single-kernel case (for ncu captures), not the benchmark")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

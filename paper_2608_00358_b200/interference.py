@@ -11,7 +11,7 @@ Run as a module for the SM-budget sweep and for the other ways of sharing the GP
     python -m paper_2608_00358_b200.interference --method idle_sms --quanta 1,2,4 --opts tile_bytes=122880
 
 OVERLAP_OPTS is the operating point measured to cost a saturating 8192^3 GEMM less than 5 %: short-lived
-blocks (two work items of 120 KiB each) on a stream of lower priority than the GEMM's.
+blocks (one work item of 120 KiB each) on a stream of lower priority than the GEMM's.
 """
 from __future__ import annotations
 
@@ -26,7 +26,7 @@ import torch
 from . import workloads as wk
 
 
-OVERLAP_OPTS = dict(quantum=2, tile_bytes=122880)
+OVERLAP_OPTS = dict(quantum=1, tile_bytes=122880)
 
 
 class Gemm:

@@ -192,3 +192,42 @@ def time_host_observed(wl: Workload, iters: int = 200) -> dict:
     if rc != hb.OK:
         raise hb.HcclError(rc, "hccl_server_wait")
     return {"launch_and_sync_us": launch_us, "ring_and_wait_us": ring_us}
+
+
+def latency_breakdown(wl: Workload, iters: int = 1000, warmup: int = 100, traced_runs: int = 20) -> dict:
+    """Where the microseconds of one execution go (the nesting T(engine) within T(control core) within T(event) that
+    the paper uses to attribute its overheads, Sec. V-C): event-pair p50, back-to-back and graph-replay time per
+    execution without tracing; then, from the per-item trace and the control block of the fastest of
+    `traced_runs` traced executions, the span from the first claim to the last block's exit, its parts, and
+    what is left of the event-pair time outside the kernel's own span (launch, kernel start, event records)."""
+    from .runtime import enable_trace
+    ms = time_each(wl, iters, warmup)
+    out = {"p50_event_us": float(np.percentile(ms, 50) * 1e3), "back_to_back_us": float(time_back_to_back(wl, iters, warmup) * 1e3),
+           "graph_replay_us": float(time_graph_replay(wl) * 1e3)}
+    tr = enable_trace(wl.plan)
+    base = wl.dc._ws_ptr - wl.dc.workspace.data_ptr()
+    best = None
+    for _ in range(traced_runs):
+        tr.zero_()
+        torch.cuda.synchronize()
+        wl.dc.execute()
+        torch.cuda.synchronize()
+        rows = tr.cpu().numpy()
+        rows = rows[rows[:, 1] != 0]
+        ctl = wl.dc.workspace[base:base + 48].cpu().numpy().view(np.uint64)   # control block: [5] = last exit (ns)
+        claimed, released, stored, blk = rows[:, 1], rows[:, 2], rows[:, 3], rows[:, 0] >> 32
+        first = int(claimed.min())
+        depth = max(int((blk == b).sum()) for b in np.unique(blk))
+        d = {"in_kernel_span_us": (int(ctl[5]) - first) / 1e3,
+             "first_item_records_and_dependencies_us": (int(released[np.argmin(claimed)]) - first) / 1e3,
+             "first_claim_to_last_store_us": (int(stored.max()) - first) / 1e3,
+             "last_store_to_last_exit_us": (int(ctl[5]) - int(stored.max())) / 1e3,
+             "item_data_movement_median_us": float(np.median(stored - released)) / 1e3,
+             "items": int(rows.shape[0]), "blocks": int(np.unique(blk).size), "items_in_a_row_per_block": depth}
+        d["per_item_in_a_row_us"] = d["first_claim_to_last_store_us"] / depth
+        if best is None or d["in_kernel_span_us"] < best["in_kernel_span_us"]:
+            best = d
+    wl.plan.set_trace(0, 0)
+    out.update(best)
+    out["outside_the_kernel_span_us"] = out["p50_event_us"] - out["in_kernel_span_us"]
+    return out
