@@ -441,21 +441,26 @@ def interference_leg(args, wl):
     return out
 
 
+def interference_opts():
+    from paper_2608_00358_b200 import interference
+    return interference.OVERLAP_OPTS
+
+
 def headline_of(line: dict) -> dict:
     """The compact record: the contract's keys, the roofline, both baselines and a few cross-references."""
     keep = ["metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling", "vs_baseline",
             "dtype", "data", "gpu_launches", "clocks"]
     h = {k: line[k] for k in keep if k in line}
     c = line["config"]
-    h["config"] = {k: c[k] for k in ("workload", "virtual_ranks", "payload_bytes", "sm_budget", "threads", "tile_bytes", "engine", "cache",
-                                     "multi_gpu", "zipf_clamp_rows")}
+    h["config"] = {k: c[k] for k in ("workload", "virtual_ranks", "payload_bytes", "sm_budget", "threads", "tile_bytes", "engine", "multi_gpu")}
+    h["config"]["cache"] = "inputs > L2"
     r = line["roofline"]
     h["roofline"] = {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "kernel", "algorithmic_bytes_per_launch", "launch_ms")}
     h["roofline"]["peak_source"] = r["peak_source"]
-    h["roofline"]["traffic_from"] = "ncu, cap-1024 case, scaled by bytes"
+    h["roofline"]["traffic_from"] = "ncu cap-1024 case, scaled"
     e = line.get("e2e")
     if e:
-        h["e2e"] = {k: e[k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step", "ms_per_step", "steps", "gpu_launches_per_step",
+        h["e2e"] = {k: e[k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step", "ms_per_step", "gpu_launches_per_step",
                                       "checked_destinations_vs_oracle", "skipped") if k in e}
         if "api" in e:
             h["e2e"]["api"] = e["api"].split(" ")[0]
@@ -463,7 +468,8 @@ def headline_of(line: dict) -> dict:
         h["cpu_baseline"] = line["cpu_baseline"]
     i = line.get("interference")
     if i and "chosen" in i:
-        h["interference"] = {k: i["chosen"][k] for k in ("mode", "sm_budget_held", "gemm_slowdown", "collective_overlap_gbs", "collective_alone_gbs")}
+        h["interference"] = {k: i["chosen"][k] for k in ("sm_budget_held", "gemm_slowdown", "collective_overlap_gbs", "collective_alone_gbs")}
+        h["interference"]["mode"] = "idle SMs: quantum %d, tile %d B, low priority" % (interference_opts()["quantum"], interference_opts()["tile_bytes"])
         h["interference"]["gemm"] = "bf16 8192^3"
         pers = {str(p["sm_budget"]): p["gemm_slowdown"] for p in i.get("sweep", []) if p["sm_budget"] in (2, 16)}
         h["interference"]["persistent_budget_slowdown"] = pers
@@ -484,7 +490,7 @@ def headline_of(line: dict) -> dict:
         side["c5_4k_resident_ring_wait_us"] = ho.get("ring_and_wait_us")
     if side:
         h["side"] = side
-    h["detail"] = "previous stdout line; gpurun_out/bench_detail.json"
+    h["detail"] = "previous stdout line"
     return h
 
 

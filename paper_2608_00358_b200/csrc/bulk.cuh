@@ -284,7 +284,7 @@ static __device__ void issue_simple(const ExecParams& p, Dma& d, uint32_t kind, 
 // dependencies and performs WAIT / SET / NOOP items itself; items that move data are passed on through a small
 // ring in shared memory. The three or four dependent trips to the L2 that start an item thus overlap with the
 // DMA thread's piece issue instead of stalling it.
-constexpr uint32_t QUEUE = 2;                  // prepared items the control thread may be ahead by
+constexpr uint32_t QUEUE = 1;                  // prepared items the control thread may be ahead by
 enum : uint32_t { Q_ITEM = 0, Q_STOP = 1 };
 struct alignas(16) Prepared {
     Tile t;
