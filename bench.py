@@ -31,7 +31,7 @@ UNIT = "GB/s"
 # dram bytes (read + write) per algorithmic byte of the executor kernel on this workload, from the ncu
 # capture summarised under profiles/ (captured on a smaller cap of the same workload, traffic scales with
 # the bytes moved). None until measured.
-DRAM_BYTES_PER_ALGORITHMIC_BYTE = 0.977
+DRAM_BYTES_PER_ALGORITHMIC_BYTE = 0.979
 
 
 def peaks():

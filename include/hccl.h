@@ -144,7 +144,7 @@ typedef struct {
                                best per-block rate), 2 = the bulk unit, 0 = compute warps below 100 blocks, bulk unit otherwise */
     int32_t rack_size;      /* ranks per rack for HCCL_ALGO_RING_2LEVEL and for cross-rack byte accounting (default 16,
                                the paper's rack, Sec. V-D) */
-    int32_t stage_kib;      /* bulk engine: KiB per shared-memory stage, a multiple of 12 in [12, 96] (default 48); with
+    int32_t stage_kib;      /* bulk engine: KiB per shared-memory stage, 12 to 96 (default 48; multiples of 12 split evenly for every operand mix); with
                                opts.stages left at 0 the number of stages keeps 192 KiB in flight (at most 8 stages) */
     int32_t quantum;        /* 0: persistent blocks (sm_budget of them run until the packet is done). > 0: short-lived blocks,
                                each leaves after this many work items and as many blocks are launched as that takes; how many

@@ -10,7 +10,7 @@ namespace bulk {
 constexpr uint32_t MAX_STAGES = 8;
 constexpr uint32_t STAGE_BYTES = 49152;       // default stage: a COPY piece fills a stage; a REDUCE piece splits it into A and B;
                                               // 4 x 48 KiB + bookkeeping fits the 227 KB a block may have
-constexpr uint32_t MIN_STAGE_BYTES = 12288, MAX_STAGE_BYTES = 98304;  // opts.stage_kib, a multiple of 12 KiB in this range
+constexpr uint32_t MIN_STAGE_BYTES = 12288, MAX_STAGE_BYTES = 98304;  // opts.stage_kib lies in this range
 // Elements per REDUCE piece: as many as fit a stage with both operands, in whole multiples of 512 elements
 // (48 KiB stages: 6144 for fp32+fp32, 8192 for fp32+16-bit, 12288 for 16-bit+16-bit).
 __host__ __device__ constexpr uint32_t piece_elems(uint32_t stage_bytes, uint32_t ea, uint32_t eb) { return stage_bytes / (ea + eb) / 512 * 512; }
@@ -47,7 +47,7 @@ struct alignas(16) PieceInfo {  // one per stage, in shared memory; written by t
 
 inline StageConfig stage_config(int stages_opt, int stage_kib_opt) {
     uint32_t sb = stage_kib_opt > 0 ? (uint32_t)stage_kib_opt * 1024u : STAGE_BYTES;
-    sb = sb / 12288u * 12288u;
+    sb = sb / 1024u * 1024u;
     if (sb < MIN_STAGE_BYTES) sb = MIN_STAGE_BYTES;
     if (sb > MAX_STAGE_BYTES) sb = MAX_STAGE_BYTES;
     const size_t per = (size_t)sb + sizeof(PieceInfo) + 16, room = MAX_DYNAMIC_SMEM - 128;
