@@ -425,25 +425,25 @@ def interference_leg(args, wl):
             "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
             "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
         del w2, plan, gemm
-    # the operating point: no SM is held against the GEMM. Short-lived blocks (interference.OVERLAP_OPTS) on a stream of
-    # LOWER priority than the GEMM's take only the SMs the GEMM leaves idle (the tail of its last wave, the gap between
-    # launches); the slowdown is still taken against the unrestricted GEMM alone
+    # the operating point: no SM is held against the GEMM. (1) interference.OVERLAP_OPTS: sixteen persistent blocks of the
+    # register engine's 64-register build, 128 threads each, small enough to run on SMs that GEMM blocks occupy.
+    # (2) interference.IDLE_SM_OPTS: short-lived blocks on a stream of LOWER priority than the GEMM's, which take only
+    # the SMs the GEMM leaves idle. Slowdowns are still taken against the unrestricted GEMM alone.
     torch.cuda.empty_cache()
     gemm = interference.Gemm()
-    plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(interference.OVERLAP_OPTS))
-    w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
-    r = interference.measure(w2, seconds=3.0, gemm=gemm, collective_first=False)
-    out["chosen"] = {"mode": "idle SMs: quantum %d, tile %d B, GEMM stream has priority" % (interference.OVERLAP_OPTS["quantum"], interference.OVERLAP_OPTS["tile_bytes"]),
-                     "sm_budget_held": 0, "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
-                     "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_alone_gbs": r["collective_alone_gbs"],
-                     "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
-    del w2, plan, gemm
+
+    def point(opts, collective_first):
+        plan = hb.hccl_plan_alltoallv(64, wl.meta["counts"], None, None, None, hb.FP16, 256, dict(opts))
+        w2 = wk._bind(wl.name, plan, wl.send, wl.recv, wl.meta)
+        r = interference.measure(w2, seconds=3.0, gemm=gemm, collective_first=collective_first)
+        return {"opts": dict(opts), "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
+                "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_alone_gbs": r["collective_alone_gbs"],
+                "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
+    out["chosen"] = dict(point(interference.OVERLAP_OPTS, True), mode="16 co-resident blocks (register engine, 64 registers, 128 threads)",
+                         sm_budget=interference.OVERLAP_OPTS["sm_budget"])
+    out["idle_sms"] = dict(point(interference.IDLE_SM_OPTS, False), mode="short-lived blocks, GEMM stream has priority")
+    del gemm
     return out
-
-
-def interference_opts():
-    from paper_2608_00358_b200 import interference
-    return interference.OVERLAP_OPTS
 
 
 def headline_of(line: dict) -> dict:
@@ -468,9 +468,10 @@ def headline_of(line: dict) -> dict:
         h["cpu_baseline"] = line["cpu_baseline"]
     i = line.get("interference")
     if i and "chosen" in i:
-        h["interference"] = {k: i["chosen"][k] for k in ("sm_budget_held", "gemm_slowdown", "collective_overlap_gbs", "collective_alone_gbs")}
-        h["interference"]["mode"] = "idle SMs: quantum %d, tile %d B, low priority" % (interference_opts()["quantum"], interference_opts()["tile_bytes"])
+        h["interference"] = {k: i["chosen"][k] for k in ("mode", "sm_budget", "gemm_slowdown", "collective_overlap_gbs", "collective_alone_gbs")}
         h["interference"]["gemm"] = "bf16 8192^3"
+        if "idle_sms" in i:
+            h["interference"]["idle_sms_slowdown"] = i["idle_sms"]["gemm_slowdown"]
         pers = {str(p["sm_budget"]): p["gemm_slowdown"] for p in i.get("sweep", []) if p["sm_budget"] in (2, 16)}
         h["interference"]["persistent_budget_slowdown"] = pers
     cfg = line.get("configs") or {}

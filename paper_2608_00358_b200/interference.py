@@ -10,8 +10,10 @@ Run as a module for the SM-budget sweep and for the other ways of sharing the GP
     python -m paper_2608_00358_b200.interference --budgets 4,8,16,32,64,148 --cap 32768
     python -m paper_2608_00358_b200.interference --method idle_sms --quanta 1,2,4 --opts tile_bytes=122880
 
-OVERLAP_OPTS is the operating point measured to cost a saturating 8192^3 GEMM less than 5 %: short-lived
-blocks (one work item of 120 KiB each) on a stream of lower priority than the GEMM's.
+OVERLAP_OPTS is the operating point measured to cost a saturating 8192^3 GEMM less than 5 %: sixteen persistent
+blocks of the register engine's 64-register build with 128 threads each, which are small enough to run on SMs
+that GEMM blocks occupy (they hold no SM against the GEMM). IDLE_SM_OPTS is the other way of holding no SM:
+short-lived blocks (one work item of 120 KiB each) on a stream of lower priority than the GEMM's.
 """
 from __future__ import annotations
 
@@ -26,7 +28,8 @@ import torch
 from . import workloads as wk
 
 
-OVERLAP_OPTS = dict(quantum=1, tile_bytes=122880)
+OVERLAP_OPTS = dict(engine=1, light=1, threads=128, sm_budget=16)
+IDLE_SM_OPTS = dict(quantum=1, tile_bytes=122880)
 
 
 class Gemm:
@@ -198,6 +201,7 @@ def main():
                          "collective in two green contexts that split the SMs; idle_sms: short-lived blocks (--quanta) on a stream of "
                          "LOWER priority than the GEMM's, so they only take SMs the GEMM leaves idle")
     ap.add_argument("--quanta", default="4,8,16", help="items per block for --method idle_sms")
+    ap.add_argument("--gemm-first", action="store_true", help="--method plain with the GEMM's stream at the higher priority")
     args = ap.parse_args()
     extra = {k: int(v) for k, v in (kv.split("=") for kv in args.opts.split(",") if kv)}
     gemm = Gemm(args.gemm_n)
@@ -228,8 +232,8 @@ def main():
             wl = plan_for(sm_budget=b)
             if args.method in ("sm_target", "green_sm_target"):
                 target = set_sm_count_target(148 - b, streams[0] if streams else None)
-            res = measure(wl, args.seconds, gemm, streams=streams, alone_tflops=unrestricted)
-            res.update(method=args.method, sm_count_target=target, opts=extra, gemm_n=args.gemm_n)
+            res = measure(wl, args.seconds, gemm, streams=streams, alone_tflops=unrestricted, collective_first=not args.gemm_first)
+            res.update(method=args.method, sm_count_target=target, opts=extra, gemm_n=args.gemm_n, gemm_first=bool(args.gemm_first))
             print(json.dumps(res), flush=True)
         finally:
             if target:
