@@ -157,6 +157,13 @@ typedef struct {
                                plans that run as static chains and by device-resident plans; refused by hccl_server_start */
 } hccl_opts_t;
 
+/* Fills *o with the options measured to let a collective run beside a saturating compute kernel for less than 5 % of
+ * that kernel's rate (the overlap experiment of Sec. V-E; 8192^3 bf16 GEMM, AllToAllv of config 4: 3.4-4.3 % at
+ * 300 GB/s): 16 persistent blocks of the register engine's 64-register build with 128 threads each, which are small
+ * enough to share an SM with a block of the compute kernel and so hold no SM against it. Every other field is zeroed
+ * (defaults). The library's general defaults aim at a GPU of its own instead: one full-size block per SM. */
+void hccl_opts_for_overlap(hccl_opts_t* o);
+
 typedef struct hccl_plan hccl_plan_t;   /* opaque, host-owned: a compiled, cacheable work packet (Sec. V-B) */
 typedef struct hccl_graph hccl_graph_t; /* opaque, host-owned: a work packet under construction */
 

@@ -121,6 +121,8 @@ def _load() -> C.CDLL:
     lib.hccl_last_cuda_error.restype = C.c_char_p
     lib.hccl_version.argtypes = []
     lib.hccl_version.restype = C.c_int
+    lib.hccl_opts_for_overlap.argtypes = [C.POINTER(Opts)]
+    lib.hccl_opts_for_overlap.restype = None
     return lib
 
 
@@ -135,7 +137,7 @@ EXPORTS = ["hccl_plan_allreduce", "hccl_plan_reducescatter", "hccl_plan_allgathe
            "hccl_plan_extents", "hccl_plan_layout", "hccl_plan_destroy", "hccl_status_string", "hccl_last_cuda_error", "hccl_version",
            "hccl_plan_check_hazards", "hccl_plan_interpret_host",
            "hccl_hostpipe_alltoallv_create", "hccl_hostpipe_windows", "hccl_hostpipe_workspace_bytes", "hccl_hostpipe_bind",
-           "hccl_hostpipe_execute", "hccl_hostpipe_status", "hccl_hostpipe_destroy"]
+           "hccl_hostpipe_execute", "hccl_hostpipe_status", "hccl_hostpipe_destroy", "hccl_opts_for_overlap"]
 
 
 def status_string(status: int) -> str:
@@ -156,6 +158,13 @@ def _i64(a) -> Optional[C.Array]:
 
 def _ptr_array(ptrs: Sequence[int]):
     return (C.c_void_p * len(ptrs))(*[int(p) if p else None for p in ptrs])
+
+
+def hccl_opts_for_overlap() -> dict:
+    """The library's operating point for running beside a saturating compute kernel, as a dict of options."""
+    o = Opts()
+    _lib.hccl_opts_for_overlap(C.byref(o))
+    return {name: getattr(o, name) for name, _ in Opts._fields_ if getattr(o, name)}
 
 
 def make_opts(opts=None, **kw) -> Opts:

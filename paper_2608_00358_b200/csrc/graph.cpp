@@ -650,6 +650,15 @@ const char* hccl_status_string(hccl_status_t s) {
     return "unknown status";
 }
 
-int hccl_version(void) { return 100; }
+int hccl_version(void) { return 200; }
+
+void hccl_opts_for_overlap(hccl_opts_t* o) {
+    if (!o) return;
+    std::memset(o, 0, sizeof(*o));
+    o->engine = HCCL_ENGINE_LSU;
+    o->light = 1;
+    o->threads = 128;
+    o->sm_budget = 16;
+}
 
 }  // extern "C"

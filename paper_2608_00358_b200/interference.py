@@ -28,7 +28,7 @@ import torch
 from . import workloads as wk
 
 
-OVERLAP_OPTS = dict(engine=1, light=1, threads=128, sm_budget=16)
+OVERLAP_OPTS = wk.hb.hccl_opts_for_overlap()      # engine = register, light = 1, threads = 128, sm_budget = 16
 IDLE_SM_OPTS = dict(quantum=1, tile_bytes=122880)
 
 
