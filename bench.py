@@ -481,8 +481,7 @@ def headline_of(line: dict) -> dict:
                               ("1_allreduce_ring_r4_fp32_1Mi", "c1_p50_us", "p50_us"), ("2_alltoallv_r8_bf16_dim128", "c2_p50_us", "p50_us"),
                               ("5_allreduce_r8_bf16_4096B_oneshot", "c5_4k_oneshot_p50_us", "p50_us"),
                               ("5_allreduce_r8_bf16_1048576B_oneshot", "c5_1m_oneshot_p50_us", "p50_us"),
-                              ("next_alltoallv_dynamic_r64_fp16_dim256", "dyn_r64_ms", "ms"),
-                              ("next_alltoallv_dynamic_r64_fp16_dim256", "dyn_r64_device_tables_ms", "device_tables_ms")):
+                              ("next_alltoallv_dynamic_r64_fp16_dim256", "dyn_r64_ms", "ms")):
         v = (cfg.get(key) or {}).get(field)
         if v is not None:
             side[short] = v
@@ -673,16 +672,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
             wd = wk._bind("alltoallv_dynamic_r64", dyn, wl.send, wl.recv, {})
             msd = wk.time_back_to_back(wd, 5, 2)
             dyn64 = {"ms": float(msd), "gbs": info.schedule_bytes / msd / 1e6, "statically_planned_ms": total_ms_max / args.steps,
+                     "form": "tables built on the device + the ordinary executor" if int(dyn.info().n_wqe) else "one kernel",
                      "note": "counts read from device memory at run time; same payload as the benchmark step"}
-            del wd, dyn
-            # the same with descriptors and tiles built on the device and run by the ordinary (bulk) executor: the form
-            # that serves any rank count
-            dyn = hb.hccl_plan_alltoallv_dynamic(64, Cd.sum(axis=1), Cd.sum(axis=0), hb.FP16, 256, dict(flags=hb.FLAG_DEVICE_TABLES))
-            dyn.set_dynamic_metadata(counts_dev.data_ptr())
-            wd = wk._bind("alltoallv_dynamic_r64_device_tables", dyn, wl.send, wl.recv, {})
-            msd = wk.time_back_to_back(wd, 5, 2)
-            dyn64["device_tables_ms"] = float(msd)
-            dyn64["device_tables_gbs"] = info.schedule_bytes / msd / 1e6
             del wd, dyn
         del wl
         torch.cuda.empty_cache()

@@ -219,7 +219,7 @@ hccl_status_t hccl_plan_alltoallv(int R, const int64_t* sendcounts, const int64_
  * produced on the device (a routing kernel) and must not travel through the host. The plan fixes only
  * R, the row size and the CAPACITY of every buffer in rows (max_send_rows[s] for X_s, max_recv_rows[d] for
  * Y_d); R <= HCCL_MAX_RANKS. Up to 64 ranks one kernel holds the whole count matrix in shared memory and
- * moves the rows itself. Beyond 64 ranks, or with HCCL_FLAG_DEVICE_TABLES, an execution is two launches: a small
+ * moves the rows itself. Beyond 64 ranks, from 1 GiB of send capacity on, or with HCCL_FLAG_DEVICE_TABLES, an execution is two launches: a small
  * kernel (one block per source rank) writes the R*R descriptors and their tiles into the bound workspace
  * -- the work requests are patched on the device, as the paper puts it -- and the ordinary executor
  * (opts.engine, default the bulk engine) runs them; the workspace is sized for the capacities. Before hccl_execute, hccl_plan_set_dynamic_metadata names the DEVICE array of R*R int64
