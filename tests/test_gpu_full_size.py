@@ -74,6 +74,24 @@ def test_config4_full_size_every_destination():
         got = wl.recv[d].cpu().numpy().view(np.uint8)
         assert np.array_equal(got, Yd[d]), "destination %d" % d
         del Xd, Yd, got
+    # --- the device-resident form at the same size (counts read from device memory, descriptors and tiles built on
+    #     the device, the default from 1 GiB of capacity on): every destination must hold the same bytes as the
+    #     statically planned result that was just compared with the oracle
+    if _free_gb() < 30:
+        return
+    dyn = hb.hccl_plan_alltoallv_dynamic(R, C.sum(axis=1), C.sum(axis=0), hb.FP16, row)
+    assert dyn.info().n_wqe == R * R                      # tables are built on the device
+    counts_dev = torch.from_numpy(np.ascontiguousarray(C.reshape(-1))).cuda()
+    rd_out = torch.full((R * R,), -1, dtype=torch.int64, device="cuda")
+    dyn.set_dynamic_metadata(counts_dev.data_ptr(), 0, rd_out.data_ptr())
+    recv2 = [torch.full_like(t, 0x5A5A) for t in wl.recv]
+    wd = wk._bind("alltoallv_dynamic_r64", dyn, wl.send, recv2, {})
+    for _ in range(2):
+        wd.dc.execute()
+    wd.dc.check()
+    for d in range(R):
+        assert torch.equal(recv2[d], wl.recv[d]), "device-resident form, destination %d" % d
+    assert np.array_equal(rd_out.cpu().numpy().reshape(R, R), RD)
 
 
 def test_config3_full_size_every_output():
