@@ -196,15 +196,8 @@ def _round(x, nd=4):
 
 def emit(detail: dict, headline: dict):
     """Two stdout lines: first everything (side configurations, sweeps, host-link figures), then LAST the compact
-    headline record (well under 2 KB) that a reader of the tail of the output can parse. The detail record is
-    also written to gpurun_out/bench_detail.json when that folder can be made."""
+    headline record (well under 2 KB) that a reader of the tail of the output can parse."""
     d = json.dumps(_finite(detail), allow_nan=False)
-    try:
-        os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-        with open(os.path.join(ROOT, "gpurun_out", "bench_detail.json"), "w") as f:
-            f.write(d + "\n")
-    except OSError:
-        pass
     print(d, flush=True)
     h = json.dumps(_round(_finite(headline)), allow_nan=False, separators=(",", ":"))
     print(h, flush=True)
