@@ -173,13 +173,13 @@ class GreenPartition:
 
 
 def measure(wl: wk.Workload, seconds: float = 3.0, gemm: Optional[Gemm] = None, collective_first: bool = True, streams=None,
-            alone_tflops: Optional[float] = None) -> dict:
+            alone_tflops: Optional[float] = None, discard: float = 1.0) -> dict:
     """GEMM slowdown = 1 - (GEMM rate beside the collective) / (rate of the UNRESTRICTED GEMM alone: default streams,
     all SMs, no SM-count target). Pass `alone_tflops` when that figure was taken before a restriction was applied."""
     gemm = gemm or Gemm()
-    alone = dict(tflops=alone_tflops if alone_tflops is not None else overlap(gemm, None, seconds)["gemm_tflops"])
+    alone = dict(tflops=alone_tflops if alone_tflops is not None else overlap(gemm, None, seconds, discard)["gemm_tflops"])
     coll_alone_ms = wk.time_back_to_back(wl, 5, 2)
-    both = overlap(gemm, wl, seconds, collective_first=collective_first, streams=streams)
+    both = overlap(gemm, wl, seconds, discard, collective_first=collective_first, streams=streams)
     res = dict(gemm_alone_tflops=alone["tflops"], collective_alone_ms=float(coll_alone_ms),
                collective_alone_gbs=float(wl.info.schedule_bytes / coll_alone_ms / 1e6), overlap=both,
                sm_budget=int(wl.info.sm_budget))
