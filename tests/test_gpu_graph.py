@@ -64,3 +64,41 @@ def test_graph_replay_latency_is_reported():
     want = orc.allreduce_oneshot_f32(hb.BF16, X)
     for r in range(8):
         assert np.array_equal(wl.recv[r].cpu().numpy().view(np.uint16), want[r])
+
+
+def test_device_resident_alltoallv_over_128_ranks_replayed_from_a_cuda_graph():
+    """The device-resident AllToAllv with tables built on the device is two launches (table builder, executor); both
+    are captured, and every replay reads the counts that are in device memory at that moment."""
+    import torch
+    from paper_2608_00358_b200.runtime import DeviceCollective
+    R, row, hi = 128, 32, 6
+    cap, rb = hi * R + 1, row * 2
+    plan = hb.hccl_plan_alltoallv_dynamic(R, [cap] * R, [cap] * R, hb.BF16, row, dict(sm_budget=32, tile_bytes=2048))
+    X = [synth.hashed_rows_np(s, 0, cap, row).reshape(-1).view(np.uint8) for s in range(R)]
+    send = [torch.from_numpy(x.copy()).cuda() for x in X]
+    recv = [torch.full((cap * rb,), 0x5A, dtype=torch.uint8, device="cuda") for _ in range(R)]
+    counts = torch.zeros(R * R, dtype=torch.int64, device="cuda")
+    plan.set_dynamic_metadata(counts.data_ptr())
+    dc = DeviceCollective(plan)
+    dc.set_buffers([t.data_ptr() for t in send], [t.data_ptr() for t in recv])
+    s = torch.cuda.Stream()
+    dc.execute(s)                         # with all counts zero: nothing moves
+    s.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        dc.execute(s)
+    for it in range(3):
+        C = synth.uniform_counts(R, 40 + it, hi=hi)
+        counts.copy_(torch.from_numpy(C.reshape(-1)))
+        for t in recv:
+            t.fill_(0x5A)
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        st, done = plan.status()
+        assert st == hb.OK and done == 2 + it
+        SD, RD = orc.packed_displs(C)
+        want = [np.full(cap * rb, 0x5A, dtype=np.uint8) for _ in range(R)]
+        orc.alltoallv(X, want, C, SD, RD, rb)
+        for d in range(R):
+            assert np.array_equal(recv[d].cpu().numpy(), want[d]), (it, d)
