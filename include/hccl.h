@@ -136,7 +136,8 @@ typedef struct {
                                the FP32 partials take at most 32 MiB (AllReduce rings: 128 MiB), else 16 */
     int32_t threads;        /* threads per block, multiple of 32. Register engine: one control warp + workers (default 512,
                                at least 64). Bulk engine: DMA, control and publishing warps + compute warps (default 352, at least 128) */
-    int32_t stages;         /* bulk engine: shared-memory stages of 48 KiB per block, 2..4 (default 4) */
+    int32_t stages;         /* bulk engine: shared-memory stages per block, 2..8 (default: 4 of 48 KiB; copy-only plans on 100 blocks
+                               or more: 3, since the memory is then the limit and fewer bytes in flight per block serve it better) */
     int32_t cluster;        /* register engine: launch blocks in clusters of this size (2, 4, 8) so that they sit on
                                neighbouring SMs; 0/1 = no clusters. Ignored unless it divides the block count. */
     int32_t light;          /* register engine: nonzero = the 64-register build (several blocks per SM). With 64-128 threads such a
