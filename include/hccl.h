@@ -133,7 +133,8 @@ typedef struct {
     uint32_t flags;         /* HCCL_FLAG_* */
     int32_t chain_group;    /* chains scheduled together in chain-group-major order; FP32 scratch slots are recycled
                                every two groups. Default: all chains together (a slot per chain, no recycling) while
-                               the FP32 partials take at most 32 MiB (AllReduce rings: 128 MiB), else 16 */
+                               the FP32 partials take at most 32 MiB (AllReduce rings: 48 MiB), else as many as keep one
+                               group-step's partials at 64 MiB, half the L2 (16 for 2 MiB granules of 16-bit data) */
     int32_t threads;        /* threads per block, multiple of 32. Register engine: one control warp + workers (default 512,
                                at least 64). Bulk engine: DMA, control and publishing warps + compute warps (default 352, at least 128) */
     int32_t stages;         /* bulk engine: shared-memory stages per block, 2..8 (default: 4 of 48 KiB; copy-only plans on 100 blocks

@@ -201,6 +201,15 @@ void fill_copy_opts(hccl_opts_t* o, const hccl_opts_t* in) {
     if (o->engine == HCCL_ENGINE_BULK && o->stages == 0 && o->stage_kib == 0 && o->sm_budget >= 100) o->stages = 3;
 }
 
+// Chains per group for large rings: the FP32 partials of one group-step (chains x granule x 4 bytes) should fill
+// about half the L2 (64 MiB): fewer chains leave a step with too few tiles for the blocks, more push the partials
+// out of the L2 between two steps (R = 64 x 32 Mi bf16, granules of 512 Ki elements: 16 / 32 / 48 / 64 chains per
+// group 6.5 / 3.5 / 4.3 / 4.3 ms; config 3, granules of 1 Mi: 8 / 16 / 24 chains 1.20 / 0.87 / 1.33 ms).
+int32_t l2_chain_group(int64_t granule_elems, size_t n_chains) {
+    const int64_t g = (64ll << 20) / std::max<int64_t>(granule_elems * 4, 1);
+    return (int32_t)std::max<int64_t>(1, std::min<int64_t>(g, (int64_t)std::max<size_t>(n_chains, 1)));
+}
+
 std::vector<Chain> make_chains(int R, const std::vector<int64_t>& offs, bool scatter, int64_t granule_elems, bool bidirectional) {
     // chunk c = [offs[c], offs[c+1]); cut into granules; granule-major order so that consecutive chains
     // belong to different chunks (different final ranks) and a chain group spans the ring evenly
@@ -607,7 +616,7 @@ hccl_status_t plan_allreduce_tree(int R, int64_t count, hccl_dtype_t dt, hccl_op
 
 extern "C" {
 
-constexpr int64_t kOwnSlotBytes = 128ll << 20;
+constexpr int64_t kOwnSlotBytes = 48ll << 20;
 
 hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_algo_t algo, const hccl_opts_t* opts,
                                   hccl_plan_t** out) {
@@ -622,8 +631,10 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     // its chains can stay inside one block at any size; that needs the register engine (measured ahead of the
     // bulk engine with tickets: 0.50 vs 0.57 ms at R = 4 x 64 Mi, 0.63 vs 0.69 ms at R = 16 x 16 Mi).
     const bool fp32_ring = dt == HCCL_FP32 && algo == HCCL_ALGO_RING && R > 1;
-    // A 16-bit ring whose FP32 partials take at most 128 MiB gives every chain a scratch slot of its own (no
-    // recycling), so its chains are independent too (R = 64 x 4 Mi bf16: 0.58 vs 0.95 ms; x 32 Mi: 4.0 vs 4.4 ms).
+    // A 16-bit ring whose FP32 partials take at most 48 MiB gives every chain a scratch slot of its own (no
+    // recycling), so its chains are independent too and run as static chains on the register engine (R = 64 x 4 Mi
+    // bf16: 0.59 vs 1.50 ms on the bulk engine with tickets; x 8 Mi: 1.05 vs 1.61 ms). From 64 MiB of partials on the
+    // bulk engine with chain groups sized for the L2 is ahead (x 16 Mi: 1.81 vs 2.16 ms; x 32 Mi: 3.50 vs 4.01 ms).
     const bool own_slots = algo == HCCL_ALGO_RING && R > 1 && count * 4 <= kOwnSlotBytes && (!opts || opts->chain_group == 0);
     hccl_opts_t pre;
     if (opts) pre = *opts; else std::memset(&pre, 0, sizeof(pre));
@@ -698,6 +709,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     // small buffers (all FP32 partials fit the L2 several times over): run every chain together, the
     // dependency chain is then as short as the ring allows; large ones keep chain groups for L2 residency
     if ((!opts || opts->chain_group == 0) && (count * 4 <= (32ll << 20) || own_slots)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
+    else if (!opts || opts->chain_group == 0) o.chain_group = l2_chain_group(maxlen, chains.size());
     // ... and each chain of tiles can then stay inside one block (no slot is recycled, so nothing links the chains)
     // (the fused form has no partials at all: its one sum per granule is followed by copies that hop from the
     // bytes the same block has just written)
@@ -796,6 +808,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     int64_t maxlen = 0;
     for (const Chain& ch : chains) maxlen = std::max(maxlen, ch.len);
     if ((!opts || opts->chain_group == 0) && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
+    else if (!opts || opts->chain_group == 0) o.chain_group = l2_chain_group(maxlen, chains.size());
     // ... and each chain of tiles can then stay inside one block (no slot is recycled, so nothing links the chains)
     if (count * 4 <= (32ll << 20) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const bool need_scratch = !fused && R > 2;
