@@ -433,7 +433,11 @@ void hccl_hostpipe_destroy(hccl_hostpipe_t*);
  * hccl_server_stop only asks the kernel to leave and returns at once: synchronise the server's `stream` after
  * it, before the plan is executed, bound or served again (until the kernel has left, its blocks still use the
  * workspace's ticket, exit count and counters). */
-typedef struct { uint64_t request, completed, stop, exited, status, detail, pad[2]; } hccl_doorbell_t;
+typedef struct {
+    uint64_t request, completed, stop, exited, status, detail;
+    uint64_t t_seen_ns, t_done_ns; /* device clock (%globaltimer) when the kernel saw the last ring and when that execution's last
+                                      block had left: the part of a ring-to-wait round trip that is spent on the device */
+} hccl_doorbell_t;
 hccl_status_t hccl_server_start(hccl_plan_t*, const void* const* sendbufs, void* const* recvbufs, void* host_doorbell,
                                 uint64_t idle_timeout_ns, void* stream);
 hccl_status_t hccl_server_ring(hccl_plan_t*);

@@ -46,6 +46,11 @@ struct ExecParams {
     uint32_t n_tiles, n_descs, n_syncs, n_waits;
     uint32_t R, nblocks, n_signals;
     uint32_t quantum;  // ticket dispatch: items a block claims before it leaves (0 = until the packet is done)
+    // resident executor only: where the last block out of an execution reports it to the host (doorbell record), and the
+    // execution number that counts as the first one
+    unsigned long long* host_completed;
+    unsigned long long* host_t_done;
+    uint32_t first_epoch, pad2;
     unsigned long long timeout_ns;
     long long n_user_signals;
     long long trig_wait_slot, trig_set_slot;
@@ -607,8 +612,9 @@ __device__ __forceinline__ void publish_tile(const ExecParams& p, const Tile& t)
 // Last block out: completion value for a device-triggered caller, epoch stamp, clean ticket.
 // `lean`: nobody reads the control block or the results before this launch has ended (no completion value to
 // publish, not the resident executor), so the end of the kernel orders everything and the fences are left out.
+// Returns true in the block that was last.
 template <class P>
-__device__ void leave(const P& p, bool lean = false) {
+__device__ bool leave(const P& p, bool lean = false) {
     if (!lean) __threadfence();
     const uint32_t prev = atomicAdd(&p.ctl->exits, 1);
     if (prev == p.nblocks - 1) {
@@ -619,7 +625,9 @@ __device__ void leave(const P& p, bool lean = false) {
         p.ctl->exits = 0;
         if (!lean) __threadfence();
         p.ctl->done_epoch = g_epoch;
+        return true;
     }
+    return false;
 }
 
 // Named barriers of the register engine (id 0 is left to __syncthreads).
@@ -813,7 +821,15 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         }
         if (!go) break;
     }
-    if (tid == 0) leave(p, !RESIDENT && p.trig_set_slot < 0);
+    if (tid == 0) {
+        const bool last = leave(p, !RESIDENT && p.trig_set_slot < 0);
+        if (RESIDENT && last && p.host_completed && ld_relaxed_u32(&p.ctl->fail_epoch) != g_epoch) {
+            // the host learns of a successful execution from the block that ended it, not a poll later from block 0
+            // (a failed one is reported by block 0, verdict first)
+            asm volatile("st.relaxed.sys.global.u64 [%0], %1;" ::"l"(p.host_t_done), "l"(globaltimer_ns()) : "memory");
+            asm volatile("st.release.sys.global.u64 [%0], %1;" ::"l"(p.host_completed), "l"((unsigned long long)(g_epoch - p.first_epoch + 1u)) : "memory");
+        }
+    }
 }
 
 }  // namespace hccl

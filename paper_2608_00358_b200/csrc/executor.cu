@@ -58,6 +58,10 @@ static int set_dispatch(const hccl_plan_t* p, ExecParams& prm) {
     if ((uint32_t)blocks > prm.n_tiles) blocks = (int)std::max<uint32_t>(prm.n_tiles, 1u);
     prm.chain_len = p->chain_len;
     prm.n_chains = p->n_chains;
+    prm.host_completed = nullptr;
+    prm.host_t_done = nullptr;
+    prm.first_epoch = 0;
+    prm.pad2 = 0;
     if (p->chain_len) blocks = (int)std::max<uint32_t>(1u, std::min<uint32_t>((uint32_t)blocks, p->n_chains));
     prm.static_tickets = (!p->chain_len && prm.n_waits == 0 && prm.n_tiles <= (uint32_t)blocks) ? 1 : 0;
     prm.quantum = 0;
@@ -513,6 +517,9 @@ hccl_status_t hccl_server_start(hccl_plan_t* p, const void* const* sendbufs, voi
     Doorbell* db = (Doorbell*)dev_db;
     unsigned long long idle = idle_timeout_ns ? idle_timeout_ns : 100000000ull;
     uint32_t first_epoch = c.done_epoch + 1;
+    prm.host_completed = &db->completed;
+    prm.host_t_done = &db->t_done_ns;
+    prm.first_epoch = first_epoch;
     void* args[] = {(void*)&prm, (void*)&db, (void*)&idle, (void*)&first_epoch};
     CUDA_TRY(cudaLaunchCooperativeKernel((const void*)hccl_executor_resident, dim3((unsigned)blocks), dim3((unsigned)p->opts.threads), args, 0, s));
     p->server_db = host_doorbell;

@@ -21,6 +21,10 @@ __device__ __forceinline__ unsigned long long ld_sys_u64(const unsigned long lon
 __device__ __forceinline__ void st_sys_u64(unsigned long long* p, unsigned long long v) {
     asm volatile("st.release.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
+// No ordering of its own: made visible to the host by the next release store.
+__device__ __forceinline__ void st_sys_relaxed_u64(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.sys.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
 
 __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_constant__ ExecParams p, Doorbell* db,
                                                                   const unsigned long long idle_ns, const uint32_t first_epoch) {
@@ -38,20 +42,23 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_co
                         if (globaltimer_ns() > deadline) { ok = false; break; }
                         __nanosleep(50);
                     }
-                    if (ok) {
-                        if (ld_acquire_u32(&p.ctl->fail_epoch) == epoch - 1) {
-                            st_sys_u64(&db->status, p.ctl->status);
-                            st_sys_u64(&db->detail, p.ctl->detail);
-                            ok = false;  // a failed execution leaves the counters inconsistent: stop serving
-                        }
-                        st_sys_u64(&db->completed, (unsigned long long)(epoch - first_epoch));
+                    if (ok && ld_acquire_u32(&p.ctl->fail_epoch) == epoch - 1) {
+                        // the verdict first, then (below) the exit code that makes the host look at it; `completed` is
+                        // not advanced for a failed execution (a successful one was reported by its last block out)
+                        st_sys_relaxed_u64(&db->status, p.ctl->status);
+                        st_sys_relaxed_u64(&db->detail, p.ctl->detail);
+                        ok = false;  // a failed execution leaves the counters inconsistent: stop serving
                     }
                 }
-                unsigned long long why = ok ? 0 : 3;
+                unsigned long long why = ok ? 0 : 3, t_seen = 0;
                 if (ok) {
                     const unsigned long long deadline = globaltimer_ns() + idle_ns;
                     for (;;) {
-                        if (ld_sys_u64(&db->request) > (unsigned long long)(epoch - first_epoch)) { cmd = epoch; break; }
+                        if (ld_sys_u64(&db->request) > (unsigned long long)(epoch - first_epoch)) {
+                            cmd = epoch;
+                            t_seen = globaltimer_ns();
+                            break;
+                        }
                         if (ld_sys_u64(&db->stop) != 0) { why = 1; break; }
                         if (globaltimer_ns() > deadline) { why = 2; break; }
                         __nanosleep(100);
@@ -60,6 +67,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_co
                 if (cmd == 0) st_sys_u64(&db->exited, why);
                 // release the other blocks: server_go carries the epoch to run, or all ones to leave
                 asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&p.ctl->server_go), "r"(cmd ? cmd : 0xffffffffu) : "memory");
+                if (cmd) st_sys_relaxed_u64(&db->t_seen_ns, t_seen);  // off the path of the blocks that were just released
             } else {
                 const unsigned long long deadline = globaltimer_ns() + idle_ns + 4 * p.timeout_ns + 4000000000ull;
                 for (;;) {

@@ -12,7 +12,7 @@ struct Doorbell {                       // layout shared with hccl_doorbell_t in
     unsigned long long stop;            // host -> device: leave after the current execution
     unsigned long long exited;          // device -> host: the kernel has left (1 = stop, 2 = idle, 3 = failure)
     unsigned long long status, detail;  // device -> host: verdict of the last failed execution
-    unsigned long long pad[2];
+    unsigned long long t_seen_ns, t_done_ns;  // device -> host: device clock when the last ring was seen / when its execution was over
 };
 
 constexpr int DYN_MAX_RANKS = 64;

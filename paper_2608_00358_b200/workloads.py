@@ -186,12 +186,13 @@ def time_host_observed(wl: Workload, iters: int = 200) -> dict:
             wl.plan.server_ring()
             rc = wl.plan.server_wait(2_000_000_000)
         ring_us = (time.perf_counter() - t0) / iters * 1e6
+        on_device_us = (int(bell[7]) - int(bell[6])) / 1e3      # last execution: ring seen -> last block out, device clock
     finally:
         wl.plan.server_stop()
         s.synchronize()
     if rc != hb.OK:
         raise hb.HcclError(rc, "hccl_server_wait")
-    return {"launch_and_sync_us": launch_us, "ring_and_wait_us": ring_us}
+    return {"launch_and_sync_us": launch_us, "ring_and_wait_us": ring_us, "ring_seen_to_done_on_device_us": on_device_us}
 
 
 def latency_breakdown(wl: Workload, iters: int = 1000, warmup: int = 100, traced_runs: int = 20) -> dict:
