@@ -100,3 +100,31 @@ def test_server_refuses_more_blocks_than_fit():
     with pytest.raises(hb.HcclError) as e:
         plan.server_start([t.data_ptr() for t in send], [t.data_ptr() for t in recv], bell.data_ptr(), 50_000_000, 0)
     assert e.value.status == hb.ERR_INVALID_ARG
+
+
+def test_server_reports_a_failed_execution_and_leaves():
+    """A WAIT that nothing satisfies, bounded at 0.1 s: the ring is accepted, the wait returns the device's verdict
+    (never HCCL_OK), the completion count is not advanced, the kernel leaves by itself and the GPU stays usable."""
+    import torch
+    N = 1024
+    g = hb.Graph(2, [N * 4, N * 4], [N * 4, N * 4], n_signals=1)
+    a = g.add_subgraph(0)
+    g.add_wqe(a, hb.OP_COPY, dst=(hb.BUF_RECV, 0, 0), a=(hb.BUF_SEND, 0, 0), count=N * 4)
+    g.add_wqe(a, hb.OP_WAIT, a=(hb.BUF_SIGNAL, 0, 0), cmp=hb.CMP_GE, value=5, dep_flags=hb.DEP_FENCE)
+    g.add_wqe(a, hb.OP_COPY, dst=(hb.BUF_RECV, 1, 0), a=(hb.BUF_SEND, 1, 0), count=N * 4)
+    plan = g.compile(dict(engine=hb.ENGINE_LSU, sm_budget=2, timeout_ns=100_000_000))
+    X = [np.arange(N, dtype=np.float32) + r for r in range(2)]
+    send, recv, dc, bell = _setup(plan, X, 2, N * 4)
+    srv = torch.cuda.Stream()
+    plan.server_start([t.data_ptr() for t in send], [t.data_ptr() for t in recv], bell.data_ptr(), 500_000_000, srv.cuda_stream)
+    try:
+        assert plan.server_ring() == hb.OK
+        assert plan.server_wait(3_000_000_000) == hb.ERR_TIMEOUT
+        srv.synchronize()                           # the kernel has left after the failed execution
+        assert int(bell[3]) == 3 and int(bell[1]) == 0 and int(bell[4]) == hb.ERR_TIMEOUT
+        assert plan.server_ring() == hb.ERR_TIMEOUT     # the verdict again: nothing is served any more
+    finally:
+        plan.server_stop()
+        srv.synchronize()
+    assert bool((recv[1] == 0).all())              # what was fenced behind the WAIT never ran
+    assert float(torch.ones(8, device="cuda").sum()) == 8.0
