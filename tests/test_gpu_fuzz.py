@@ -24,6 +24,12 @@ def _options(rng):
         o["flags"] = int(rng.choice([hb.FLAG_DYNAMIC_TICKETS, hb.FLAG_STATIC_CHAINS, hb.FLAG_LEVEL_MAJOR]))
     if o["engine"] != hb.ENGINE_BULK and rng.random() < 0.2:
         o.update(light=1, threads=int(rng.choice([128, 256, 512])))
+    if o["engine"] != hb.ENGINE_LSU and rng.random() < 0.4:      # bulk engine (or the library's choice): stage ring and block shape
+        o.update(stage_kib=int(rng.choice([12, 20, 24, 36, 48, 96])), stages=int(rng.choice([0, 2, 3, 5, 8])))
+        if rng.random() < 0.5:
+            o["threads"] = int(rng.choice([128, 160, 224, 352, 512]))
+    if rng.random() < 0.2:
+        o["quantum"] = int(rng.choice([1, 2, 5]))               # short-lived blocks (ignored by plans that run as static chains)
     return o
 
 
