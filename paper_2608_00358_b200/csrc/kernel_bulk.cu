@@ -13,6 +13,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
     char* stages_ptr = reinterpret_cast<char*>(smem_raw);
     PieceInfo* info = reinterpret_cast<PieceInfo*>(stages_ptr + (size_t)ns * stage_bytes);
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(info + ns);  // full[ns], empty[ns]
+    __shared__ __align__(8) unsigned long long s_stored[MAX_STAGES];  // per stage: every compute warp has stored its share of an item's last piece
     const uint32_t tid = threadIdx.x;
     const uint32_t ncw = (blockDim.x >> 5) - 3;  // compute warps: all but the DMA, control and publishing warps
     const uint32_t full = smem_u32(bars), empty = smem_u32(bars + ns);
@@ -39,6 +40,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             mbar_init(empty + 8 * s, ncw + 1);   // every compute warp and the publishing warp
         }
         for (uint32_t q = 0; q < 2 * QUEUE + 1; ++q) mbar_init(q_full + 8 * q, 1);
+        for (uint32_t s = 0; s < ns; ++s) mbar_init(smem_u32(s_stored) + 8 * s, ncw);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
@@ -193,27 +195,28 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
 
     const uint32_t cnth = ncw * 32;
     if (tid >= 64 && tid < 96) {
-        // ------------------------------------------------------------ publishing warp
-        // Follows the pieces like a compute warp but moves no data: after the last piece of an item it waits at
-        // the stage's named barrier until every compute warp has stored its share, and its first lane publishes
-        // the item's completion. The release has to wait for those stores to be performed, a microsecond or
-        // two that no data-moving warp spends this way. The release is cumulative over the stores that the barrier
-        // ordered before the publishing thread. One barrier per stage: a stage is recycled only after every warp,
-        // this one included, has left it, so a barrier never sees two items at once.
+        // ------------------------------------------------------------ publishing thread
+        // Follows the pieces like a compute warp but moves no data: after the last piece of an item it waits (bounded)
+        // on the stage's `stored` barrier until every compute warp has stored its share, and publishes the item's
+        // completion. The release has to wait for those stores to be performed, a microsecond or two that no
+        // data-moving warp spends this way; it is cumulative over the stores that the barrier ordered before this
+        // thread. A stage is recycled only after every warp, this one included, has left it, so a `stored`
+        // barrier never sees two items at once.
+        if (tid != 64) return;
+        const uint32_t stored = smem_u32(s_stored);
+        uint32_t stored_parity = 0;  // bit s: phase parity of stage s's `stored` barrier (advances only when it is used)
         for (uint32_t slot = 0, parity = 0;;) {
             if (!mbar_wait(p, full + 8 * slot, parity, long_wait, 0xfffffff9u)) break;
             const PieceInfo& pi = info[slot];
             const uint32_t kind = pi.kind, last = pi.last;
             const int32_t sig0 = pi.signal[0], sig1 = pi.signal[1];
             if (kind != PIECE_EXIT && kind != PIECE_COPY && last && (sig0 >= 0 || sig1 >= 0)) {
-                asm volatile("bar.sync %0, %1;" ::"r"(1u + slot), "r"(cnth + 32u) : "memory");
-                if (tid == 64) {
-                    if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
-                    if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
-                }
+                if (!mbar_wait(p, stored + 8 * slot, (stored_parity >> slot) & 1u, long_wait, 0xfffffff8u)) break;
+                stored_parity ^= 1u << slot;
+                if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
+                if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
             }
-            __syncwarp();
-            if (tid == 64) mbar_arrive(empty + 8 * slot);
+            mbar_arrive(empty + 8 * slot);
             if (kind == PIECE_EXIT) break;
             if (++slot == ns) {
                 slot = 0;
@@ -282,11 +285,13 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
             run_tile_lsu(p, pi.desc, pi.tile, ctid, cnth);
         }
         if (kind != PIECE_COPY && pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.tile_index, 3, globaltimer_ns());
-        // the publishing warp waits at the stage's barrier for every compute warp's stores of an item's last piece
-        if (kind != PIECE_COPY && pi.last && (pi.signal[0] >= 0 || pi.signal[1] >= 0))
-            asm volatile("bar.arrive %0, %1;" ::"r"(1u + slot), "r"(cnth + 32u) : "memory");
+        // the publishing thread waits on the stage's `stored` barrier for every compute warp's stores of an item's last piece
+        const bool tell = kind != PIECE_COPY && pi.last && (pi.signal[0] >= 0 || pi.signal[1] >= 0);
         __syncwarp();
-        if ((tid & 31u) == 0) mbar_arrive(empty + 8 * slot);
+        if ((tid & 31u) == 0) {
+            if (tell) mbar_arrive(smem_u32(s_stored) + 8 * slot);
+            mbar_arrive(empty + 8 * slot);
+        }
         if (++slot == ns) {
             slot = 0;
             parity ^= 1u;
