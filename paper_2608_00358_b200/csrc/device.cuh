@@ -654,6 +654,42 @@ static __device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, De
     }
     return true;
 }
+// Static chains: a block's items are consecutive table entries known from the start, so the 32 lanes of the control
+// warp fetch the records of the next 32 of them at once (one trip to memory for the tiles, one for the
+// descriptors) instead of lane 0 paying both trips for every item. `lane`: every lane of the warp calls this.
+constexpr uint32_t WINDOW = 32;
+// Each lane also runs the checks on its own item, so that lane 0 later only copies the records (its work between two
+// items of a chain is on the chain's critical path, one instruction after the other).
+__device__ __forceinline__ void window_fill(const ExecParams& p, uint32_t first, uint32_t end, uint32_t lane, Tile* wt, Desc* wd, uint8_t* wok) {
+    const uint32_t idx = first + lane;
+    if (idx < end && idx < p.n_tiles) {
+        const Tile t = p.tiles[idx];
+        wt[lane] = t;
+        bool ok = false;
+        if (!(t.flags & TILE_FLAG_END) && tile_ok(p, t)) {
+            const Desc d = p.descs[t.desc];
+            wd[lane] = d;
+            ok = desc_ok(p, d);
+        }
+        wok[lane] = ok ? 1 : 0;
+    }
+    __syncwarp();
+}
+// An item whose records are in the window.
+static __device__ bool fetch_windowed(const ExecParams& p, uint32_t cur, Tile& t, Desc& d, const Tile& wt, const Desc& wd, uint8_t ok) {
+    if (p.trace) {
+        trace_put(p.trace, p.trace_cap, cur, 0, (unsigned long long)cur | ((unsigned long long)blockIdx.x << 32));
+        trace_put(p.trace, p.trace_cap, cur, 1, globaltimer_ns());
+    }
+    t = wt;
+    if (t.flags & TILE_FLAG_END) return false;
+    if (!ok) {
+        fail(p, HCCL_ERR_BAD_DESCRIPTOR, cur);
+        return false;
+    }
+    d = wd;
+    return true;
+}
 // One non-blocking look at every dependency counter of the item.
 static __device__ bool deps_ready(const ExecParams& p, const Tile& t) {
     for (uint32_t w = 0; w < t.wait_cnt; ++w) {
@@ -715,11 +751,16 @@ __device__ __forceinline__ uint32_t next_item(const ExecParams& p, uint32_t cur,
     return atomicAdd(&p.ctl->ticket, 1);
 }
 
-template <bool RESIDENT>
+template <bool RESIDENT, bool AHEAD>
 __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     __shared__ Tile s_tile[2];
     __shared__ Desc s_desc[2];
     __shared__ int s_go[2];
+    __shared__ Tile s_wtile[AHEAD ? WINDOW : 1];  // static chains: records of the items [win_base, win_base + WINDOW)
+    __shared__ Desc s_wdesc[AHEAD ? WINDOW : 1];
+    __shared__ uint8_t s_wok[AHEAD ? WINDOW : 1];   // the checks on them, done by the lane that fetched them
+    const bool window = AHEAD && p.chain_len != 0;
+    uint32_t win_base = 0, win_end = 0;  // win_end: end of the block's items
     const uint32_t tid = threadIdx.x, nth = blockDim.x;
     constexpr uint32_t FULL = 1, DONE = 3;  // barrier ids FULL+b, DONE+b
     // Entry. The execution number, the abort word, the first ticket and (with static tickets) the first item's
@@ -733,13 +774,17 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     if (tid == 0) {
         if (!gated) {
             next = first_item(p, range_end);
-            if (next < p.n_tiles) {
+            if (next < p.n_tiles && !window) {
                 pre = p.tiles[next];
                 pre_ok = true;
             }
         }
         abort0 = *(volatile uint32_t*)&p.ctl->abort;
         g_epoch = *(volatile uint32_t*)&p.ctl->done_epoch + 1u;
+    }
+    if (window && tid < 32) {  // the tables do not change: they may be read before a trigger has fired
+        chain_range(p, win_base, win_end);
+        window_fill(p, win_base, win_end, tid, s_wtile, s_wdesc, s_wok);
     }
     __syncthreads();
     if (tid >= 32) {
@@ -774,7 +819,9 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 have = live && cur < p.n_tiles && !(gated ? aborted(p) : abort0 == g_epoch);
                 if (have) {
                     next = next_item(p, cur, range_end, left);
-                    have = fetch_tile(p, cur, s_tile[0], s_desc[0], pre_ok ? &pre : nullptr);
+                    const uint32_t slot = cur - win_base;
+                    if (window && slot < WINDOW) have = fetch_windowed(p, cur, s_tile[0], s_desc[0], s_wtile[slot], s_wdesc[slot], s_wok[slot]);
+                    else have = fetch_tile(p, cur, s_tile[0], s_desc[0], pre_ok ? &pre : nullptr);
                     ready = have && deps_ready(p, s_tile[0]);
                 }
             }
@@ -795,7 +842,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 if (sig1 >= 0) red_release_add_u32(p.counters + sig1, 1);
                 sig0 = sig1 = -1;
             }
-            bool go = have && !aborted(p);
+            bool go = have;  // `have` carries the abort word as the look-ahead saw it; waits look at it again
             if (go && !simple) go = wait_deps(p, cur, s_tile[b], s_desc[b], ready);
             s_go[b] = go ? 1 : 0;
         }
@@ -803,6 +850,13 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         const int go = s_go[b];
         if (tid == 0 && p.trace && go) trace_put(p.trace, p.trace_cap, cur, 2, globaltimer_ns());
         prev_item = cur;
+        if (window && go) {  // every lane: the item after this one lies beyond the window
+            const uint32_t nx = __shfl_sync(0xffffffffu, next, 0);
+            if (nx < p.n_tiles && nx - win_base >= WINDOW) {
+                win_base = nx;
+                window_fill(p, win_base, win_end, tid, s_wtile, s_wdesc, s_wok);
+            }
+        }
         if (tid == 0) {
             if (sig0 >= 0 || sig1 >= 0) {  // publish item k-1 while the workers run item k
                 if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
@@ -811,12 +865,16 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
             if (go) {
                 // look ahead: claim, fetch and poll item k+1 behind the workers' back
                 cur = next;
-                have = cur < p.n_tiles && !aborted(p);
+                const uint32_t ab = ld_relaxed_u32(&p.ctl->abort);  // asked for first, looked at when the records are in
+                have = cur < p.n_tiles;
                 if (have) {
                     next = next_item(p, cur, range_end, left);
-                    have = fetch_tile(p, cur, s_tile[b ^ 1], s_desc[b ^ 1]);
+                    const uint32_t slot = cur - win_base;
+                    if (window && slot < WINDOW) have = fetch_windowed(p, cur, s_tile[b ^ 1], s_desc[b ^ 1], s_wtile[slot], s_wdesc[slot], s_wok[slot]);
+                    else have = fetch_tile(p, cur, s_tile[b ^ 1], s_desc[b ^ 1]);
                     ready = have && deps_ready(p, s_tile[b ^ 1]);
                 }
+                have = have && ab != g_epoch;
             }
         }
         if (!go) break;

@@ -3,6 +3,6 @@
 
 namespace hccl {
 
-__global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p) { executor_lsu_body<false>(p); }
+__global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constant__ ExecParams p) { executor_lsu_body<false, true>(p); }
 
 }  // namespace hccl

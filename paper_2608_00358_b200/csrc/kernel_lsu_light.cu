@@ -4,6 +4,6 @@
 
 namespace hccl {
 
-__global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p) { executor_lsu_body<false>(p); }
+__global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p) { executor_lsu_body<false, false>(p); }
 
 }  // namespace hccl

@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_co
         }
         __syncthreads();
         if (s_cmd == 0) break;
-        executor_lsu_body<true>(p);     // one execution: tickets, dependencies, data, completion stamp
+        executor_lsu_body<true, true>(p);    // one execution: tickets, dependencies, data, completion stamp
         __syncthreads();
         ++epoch;
     }
