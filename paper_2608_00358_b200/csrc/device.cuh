@@ -794,7 +794,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
             named_sync(FULL + b, nth);
             if (!s_go[b]) break;
             run_tile_lsu(p, s_desc[b], s_tile[b], wtid, nwork);
-            named_sync(DONE + b, nth);
+            if (!window) named_sync(DONE + b, nth);  // static chains: the next item's FULL barrier says it as well
         }
         return;
     }
@@ -808,6 +808,41 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         if (next == 0) p.ctl->t_first_ns = globaltimer_ns();
     }
     uint32_t cur = 0, prev_item = 0;
+    if (window) {
+        // Static chains: no item waits for anything but the item before it in this block, and none has anything to
+        // publish. One barrier per item then does: FULL[b] lets the workers start item k, and their arrival at
+        // it says that item k-1 is stored. The control warp fills the other buffer with item k+1 in the meantime.
+        const uint32_t end = min(win_end, p.n_tiles);
+        cur = win_base;  // every lane keeps the item numbers (the lanes refill the window together)
+        if (tid == 0) {
+            const bool h = live && cur < end && !(gated ? aborted(p) : abort0 == g_epoch);
+            s_go[0] = h && fetch_windowed(p, cur, s_tile[0], s_desc[0], s_wtile[0], s_wdesc[0], s_wok[0]);
+        }
+        for (uint32_t k = 0;; ++k) {
+            const uint32_t b = k & 1;
+            named_sync(FULL + b, nth);
+            const int go = s_go[b];
+            if (tid == 0 && p.trace) {
+                const unsigned long long now = globaltimer_ns();
+                if (k > 0) trace_put(p.trace, p.trace_cap, prev_item, 3, now);
+                if (go) trace_put(p.trace, p.trace_cap, cur, 2, now);
+            }
+            if (!go) break;
+            const uint32_t nx = cur + 1;
+            if (nx < end && nx - win_base >= WINDOW) {
+                win_base = nx;
+                window_fill(p, win_base, win_end, tid, s_wtile, s_wdesc, s_wok);
+            }
+            if (tid == 0) {
+                const uint32_t ab = ld_relaxed_u32(&p.ctl->abort);  // asked for first, looked at when the records are in
+                const uint32_t slot = nx < end ? nx - win_base : 0;
+                const bool h = nx < end && fetch_windowed(p, nx, s_tile[b ^ 1], s_desc[b ^ 1], s_wtile[slot], s_wdesc[slot], s_wok[slot]);
+                s_go[b ^ 1] = h && ab != g_epoch;
+            }
+            prev_item = cur;
+            cur = nx;
+        }
+    } else
     for (uint32_t k = 0;; ++k) {
         const uint32_t b = k & 1;
         int32_t sig0 = -1, sig1 = -1;
@@ -819,9 +854,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 have = live && cur < p.n_tiles && !(gated ? aborted(p) : abort0 == g_epoch);
                 if (have) {
                     next = next_item(p, cur, range_end, left);
-                    const uint32_t slot = cur - win_base;
-                    if (window && slot < WINDOW) have = fetch_windowed(p, cur, s_tile[0], s_desc[0], s_wtile[slot], s_wdesc[slot], s_wok[slot]);
-                    else have = fetch_tile(p, cur, s_tile[0], s_desc[0], pre_ok ? &pre : nullptr);
+                    have = fetch_tile(p, cur, s_tile[0], s_desc[0], pre_ok ? &pre : nullptr);
                     ready = have && deps_ready(p, s_tile[0]);
                 }
             }
@@ -850,13 +883,6 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         const int go = s_go[b];
         if (tid == 0 && p.trace && go) trace_put(p.trace, p.trace_cap, cur, 2, globaltimer_ns());
         prev_item = cur;
-        if (window && go) {  // every lane: the item after this one lies beyond the window
-            const uint32_t nx = __shfl_sync(0xffffffffu, next, 0);
-            if (nx < p.n_tiles && nx - win_base >= WINDOW) {
-                win_base = nx;
-                window_fill(p, win_base, win_end, tid, s_wtile, s_wdesc, s_wok);
-            }
-        }
         if (tid == 0) {
             if (sig0 >= 0 || sig1 >= 0) {  // publish item k-1 while the workers run item k
                 if (sig0 >= 0) red_release_add_u32(p.counters + sig0, 1);
@@ -869,9 +895,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
                 have = cur < p.n_tiles;
                 if (have) {
                     next = next_item(p, cur, range_end, left);
-                    const uint32_t slot = cur - win_base;
-                    if (window && slot < WINDOW) have = fetch_windowed(p, cur, s_tile[b ^ 1], s_desc[b ^ 1], s_wtile[slot], s_wdesc[slot], s_wok[slot]);
-                    else have = fetch_tile(p, cur, s_tile[b ^ 1], s_desc[b ^ 1]);
+                    have = fetch_tile(p, cur, s_tile[b ^ 1], s_desc[b ^ 1]);
                     ready = have && deps_ready(p, s_tile[b ^ 1]);
                 }
                 have = have && ab != g_epoch;
