@@ -342,6 +342,24 @@ def test_static_chains_and_tickets_same_bits(budget, flags, dt):
         assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
 
 
+@pytest.mark.parametrize("budget", [1, 2, 148])
+def test_static_chains_longer_than_the_control_warps_window(budget):
+    """Chains of 39 and 78 items: the control warp fetches the records of a block's items 32 at a time, so these
+    chains cross a refill in their middle, and with one or two blocks many chains follow each other in one block."""
+    R, dt = 40, hb.BF16
+    opts = dict(engine=hb.ENGINE_LSU, tile_bytes=1024, chunk_bytes=4096, sm_budget=budget)
+    Xg = synth.normal_ranks(R, 1531, dt, seed=77)
+    p = hb.hccl_plan_allgather(R, None, 1531, dt, hb.ALGO_RING, opts)
+    assert p.info().static_chains > 0 and p.info().n_syncs == 0
+    Y = run_plan(p, Xg, iters=2, misalign=2)
+    for r, w in enumerate(orc.allgatherv(Xg)):
+        assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
+    n = 40 * 97 + 13
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, opts)
+    assert p.info().static_chains > 0 and p.info().n_syncs == 0
+    _check_allreduce(R, n, dt, hb.ALGO_RING, opts, iters=2)
+
+
 @pytest.mark.parametrize("dt", DTYPES)
 @pytest.mark.parametrize("R", [2, 3, 5])
 def test_static_chains_on_degenerate_sizes(R, dt):
