@@ -419,7 +419,29 @@ __device__ void reduce_dispatch(int da, int db, int dd, char* dst, const char* a
 }
 
 // ------------------------------------------------------------------ REDUCE_N (multi-input sum, fixed order)
-template <int DS, int DD>
+// Barrier over `nthreads` threads that also ANDs a predicate over them.
+__device__ __forceinline__ bool named_sync_and(uint32_t id, uint32_t nthreads, bool pred) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred q, r;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred r, %2, %3, q;\n\tselp.u32 %0, 1, 0, r;\n\t}"
+        : "=r"(out) : "r"((uint32_t)pred), "r"(id), "r"(nthreads) : "memory");
+    return out != 0;
+}
+constexpr uint32_t BARRIER_WORKERS = 5;  // named barrier of the register engine's worker threads alone
+// Shared memory for the operand addresses of one REDUCE_N item (sources, then destinations): one array for all
+// element-type instantiations, and none in kernels that never ask for it.
+template <bool USED>
+__device__ __forceinline__ const char** operand_table() {
+    __shared__ const char* s_operands[USED ? 2 * HCCL_MAX_RANKS : 1];
+    return s_operands;
+}
+
+// TABLE (register engine, one block per SM): the operand addresses are put into shared memory first, one per
+// thread, and the alignment check is one AND over the block's worker threads. Without it every thread walks the
+// pointer arrays of the parameter block (constant cache) for every source and destination, one dependent lookup
+// after the other, again for every vector it handles. All `nth` threads must call this together (they meet at a
+// named barrier).
+template <int DS, int DD, bool TABLE>
 __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start, uint32_t n, const uint32_t tid, const uint32_t nth) {
     const int R = (int)p.R, nsrc = d.nsrc, r0 = d.rank_a;
     const size_t soff = (size_t)d.off_a + start * Elem<DS>::BYTES;
@@ -434,7 +456,7 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
         return (char*)p.recv[r] + doff;
     };
     const bool from_send = d.kind_a == HCCL_BUF_SEND;
-    auto src = [&](int k) -> const char* {
+    auto src_lookup = [&](int k) -> const char* {
         int r = r0 + k;
         if (r >= R) r -= R;
         return (const char*)(from_send ? p.send[r] : (const void*)p.recv[r]) + soff;
@@ -442,13 +464,37 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
     // same phase for every operand?
     const uint32_t pd = (uint32_t)(((uintptr_t)dst0 / Elem<DD>::BYTES) & 7u);
     bool vec = true;
-    for (int k = 0; k < nsrc; ++k) vec = vec && ((uint32_t)(((uintptr_t)src(k) / Elem<DS>::BYTES) & 7u) == pd);
-    for (int j = 1; j < nd; ++j) vec = vec && ((uint32_t)(((uintptr_t)dstp(j) / Elem<DD>::BYTES) & 7u) == pd);
+    const char** const s_src = TABLE ? operand_table<TABLE>() : nullptr;
+    char** const s_dst = TABLE ? (char**)(operand_table<TABLE>() + HCCL_MAX_RANKS) : nullptr;
+    if constexpr (TABLE) {
+        // one operand per warp and round: a constant-cache lookup is fast only when a warp's lanes ask for the same word
+        for (int k = (int)(tid >> 5); k < nsrc + nd; k += (int)(nth >> 5)) {
+            if (k < nsrc) {
+                const char* q = src_lookup(k);
+                if ((tid & 31u) == 0) s_src[k] = q;
+                vec = vec && ((uint32_t)(((uintptr_t)q / Elem<DS>::BYTES) & 7u) == pd);
+            } else {
+                char* q = dstp(k - nsrc);
+                if ((tid & 31u) == 0) s_dst[k - nsrc] = q;
+                vec = vec && ((uint32_t)(((uintptr_t)q / Elem<DD>::BYTES) & 7u) == pd);
+            }
+        }
+        vec = named_sync_and(BARRIER_WORKERS, nth, vec);
+    } else {
+        for (int k = 0; k < nsrc; ++k) vec = vec && ((uint32_t)(((uintptr_t)src_lookup(k) / Elem<DS>::BYTES) & 7u) == pd);
+        for (int j = 1; j < nd; ++j) vec = vec && ((uint32_t)(((uintptr_t)dstp(j) / Elem<DD>::BYTES) & 7u) == pd);
+    }
+    auto src = [&](int k) -> const char* {
+        if constexpr (TABLE) return s_src[k]; else return src_lookup(k);
+    };
+    auto dst = [&](int j) -> char* {
+        if constexpr (TABLE) return s_dst[j]; else return dstp(j);
+    };
     if (!vec) {
         for (uint32_t i = tid; i < n; i += nth) {
             float acc = Elem<DS>::load(src(0), i);
             for (int k = 1; k < nsrc; ++k) acc = acc + Elem<DS>::load(src(k), i);
-            for (int j = 0; j < nd; ++j) Elem<DD>::store(dstp(j), i, acc);
+            for (int j = 0; j < nd; ++j) Elem<DD>::store(dst(j), i, acc);
         }
         return;
     }
@@ -458,7 +504,7 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
     auto scalar = [&](uint32_t i) {
         float acc = Elem<DS>::load(src(0), i);
         for (int k = 1; k < nsrc; ++k) acc = acc + Elem<DS>::load(src(k), i);
-        for (int j = 0; j < nd; ++j) Elem<DD>::store(dstp(j), i, acc);
+        for (int j = 0; j < nd; ++j) Elem<DD>::store(dst(j), i, acc);
     };
     if (tid < head) scalar(tid);
     for (uint32_t i = head + (nv << 3) + tid; i < n; i += nth) scalar(i);
@@ -522,12 +568,13 @@ __device__ void reduce_n_tile(const ExecParams& p, const Desc& d, uint64_t start
         for (; k < nsrc; ++k) group(std::integral_constant<int, 1>{}, F{}, k, off, acc);
         const size_t o = (size_t)head * Elem<DD>::BYTES + (size_t)i * 8 * Elem<DD>::BYTES;
         store8<DD, false>(dst0 + o, acc);
-        for (int j = 1; j < nd; ++j) store8<DD, false>(dstp(j) + o, acc);
+        for (int j = 1; j < nd; ++j) store8<DD, false>(dst(j) + o, acc);
     }
 }
 
+template <bool TABLE>
 static __device__ void reduce_n_dispatch(const ExecParams& p, const Desc& d, uint64_t start, uint32_t n, uint32_t tid, uint32_t nth) {
-#define RN(S, D) reduce_n_tile<S, D>(p, d, start, n, tid, nth)
+#define RN(S, D) reduce_n_tile<S, D, TABLE>(p, d, start, n, tid, nth)
     if (d.dt_a == HCCL_FP32) {
         if (d.dt_dst == HCCL_FP32) RN(HCCL_FP32, HCCL_FP32); else if (d.dt_dst == HCCL_BF16) RN(HCCL_FP32, HCCL_BF16); else RN(HCCL_FP32, HCCL_FP16);
     } else if (d.dt_a == HCCL_BF16) {
@@ -539,6 +586,8 @@ static __device__ void reduce_n_dispatch(const ExecParams& p, const Desc& d, uin
 }
 
 // ------------------------------------------------------------------ one work item, all threads
+// TABLE: see reduce_n_tile (all `nth` threads call this together and may meet at the workers' named barrier).
+template <bool TABLE>
 static __device__ void run_tile_lsu(const ExecParams& p, const Desc& d, const Tile& t, const uint32_t tid, const uint32_t nth) {
     switch (d.op) {
         case HCCL_OP_COPY: {
@@ -562,7 +611,7 @@ static __device__ void run_tile_lsu(const ExecParams& p, const Desc& d, const Ti
             break;
         }
         case HCCL_OP_REDUCE_N:
-            reduce_n_dispatch(p, d, t.start, t.count, tid, nth);
+            reduce_n_dispatch<TABLE>(p, d, t.start, t.count, tid, nth);
             break;
         default:
             break;
@@ -793,7 +842,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
             const uint32_t b = k & 1;
             named_sync(FULL + b, nth);
             if (!s_go[b]) break;
-            run_tile_lsu(p, s_desc[b], s_tile[b], wtid, nwork);
+            run_tile_lsu<AHEAD>(p, s_desc[b], s_tile[b], wtid, nwork);
             if (!window) named_sync(DONE + b, nth);  // static chains: the next item's FULL barrier says it as well
         }
         return;

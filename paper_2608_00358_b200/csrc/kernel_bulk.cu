@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
                 if (stream) __stcs(dst + i, src[i]); else __stcg(dst + i, src[i]);
             }
         } else if (kind == PIECE_TILE) {
-            run_tile_lsu(p, pi.desc, pi.tile, ctid, cnth);
+            run_tile_lsu<false>(p, pi.desc, pi.tile, ctid, cnth);
         }
         if (kind != PIECE_COPY && pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.tile_index, 3, globaltimer_ns());
         // the publishing thread waits on the stage's `stored` barrier for every compute warp's stores of an item's last piece
