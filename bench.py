@@ -474,6 +474,8 @@ def headline_of(line: dict) -> dict:
                               ("1_allreduce_ring_r4_fp32_1Mi", "c1_p50_us", "p50_us"), ("2_alltoallv_r8_bf16_dim128", "c2_p50_us", "p50_us"),
                               ("5_allreduce_r8_bf16_4096B_oneshot", "c5_4k_oneshot_p50_us", "p50_us"),
                               ("5_allreduce_r8_bf16_1048576B_oneshot", "c5_1m_oneshot_p50_us", "p50_us"),
+                              ("5_allreduce_r8_bf16_4096B_ring", "c5_4k_ring_p50_us", "p50_us"),
+                              ("5_allreduce_r8_bf16_1048576B_ring", "c5_1m_ring_p50_us", "p50_us"),
                               ("next_alltoallv_dynamic_r64_fp16_dim256", "dyn_r64_ms", "ms")):
         v = (cfg.get(key) or {}).get(field)
         if v is not None:
