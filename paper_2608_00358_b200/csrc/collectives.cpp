@@ -376,8 +376,13 @@ std::vector<Chain2> make_chains2(int G, int L, int64_t n, int64_t granule) {
     return out;
 }
 
-hccl_status_t plan_allreduce_2level(int R, int64_t count, hccl_dtype_t dt, const hccl_opts_t& o, hccl_plan_t** out) {
+hccl_status_t plan_allreduce_2level(int R, int64_t count, hccl_dtype_t dt, const hccl_opts_t& o_in, hccl_plan_t** out) {
+    hccl_opts_t o = o_in;
     const int L = o.rack_size, G = R / L, es = elem_bytes(dt);
+    // Up to 256 KiB per rank a block does better walking one tile through all of a chunk's steps by itself than the
+    // blocks do handing it on through device counters (measured, bf16: R=64 in racks of 16 0.10-0.11 vs 0.16 ms, R=16
+    // in racks of 4 0.027-0.039 vs 0.042-0.049 ms; from 512 KiB on the other way round: 0.23 vs 0.20 ms at 1 MiB).
+    if (count * es <= (256ll << 10) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     std::vector<int64_t> ext(R, count * es);
     const int64_t granule = std::max<int64_t>(1, (int64_t)(o.chunk_bytes / (uint64_t)es));
     std::vector<Chain2> chains = make_chains2(G, L, count, granule);
@@ -499,10 +504,11 @@ hccl_status_t plan_allreduce_tree(int R, int64_t count, hccl_dtype_t dt, hccl_op
     const int64_t ng = count > 0 ? (count + granule - 1) / granule : 0;
     if (!group_given && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<int64_t>(ng, 1);  // small: all granules together
     const int64_t group = std::max<int64_t>(1, o.chain_group);
-    // From about 1 MiB per rank a block does better walking one tile through the whole tree by itself (no
-    // hand-over between SMs, 2(R-1) items in a row) than the blocks do sharing the tree's 2 log2 R levels;
-    // below that the levels' parallelism wins (measured at R = 8: 28.7 vs 43.0 us at 1 MiB, 28.7 vs 25.1 at 256 KiB).
-    if (count * es >= (1ll << 20) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
+    // From about 1 MiB per rank (256 KiB up to 8 ranks) a block does better walking one tile through the whole tree by
+    // itself (no hand-over between SMs, 2(R-1) items in a row) than the blocks do sharing the tree's 2 log2 R levels;
+    // below that the levels' parallelism wins (measured at R = 8, per execution from a CUDA graph: 20.1 vs 38.2 us at
+    // 1 MiB, 19.9 vs 22.5 at 256 KiB, 19.5 vs 18.5 at 64 KiB; at R = 64 and 128 KiB 0.148 vs 0.058 ms).
+    if (count * es >= (R <= 8 ? (256ll << 10) : (1ll << 20)) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const int half = (R + 1) / 2;                                 // scratch slots one granule needs
     const int64_t n_sets = std::min<int64_t>(std::max<int64_t>(ng, 1), 2 * group);  // recycled sets of slots
     const int64_t slot_elems = (int64_t)align_up((uint64_t)std::min<int64_t>(granule, std::max<int64_t>(count, 1)), 64);
