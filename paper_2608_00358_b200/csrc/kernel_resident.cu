@@ -53,15 +53,18 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_co
                 unsigned long long why = ok ? 0 : 3, t_seen = 0;
                 if (ok) {
                     const unsigned long long deadline = globaltimer_ns() + idle_ns;
-                    for (;;) {
+                    for (uint32_t polls = 0;; ++polls) {
+                        // every look at the doorbell is a trip over the host link: the stop word gets one look in eight
                         if (ld_sys_u64(&db->request) > (unsigned long long)(epoch - first_epoch)) {
                             cmd = epoch;
                             t_seen = globaltimer_ns();
                             break;
                         }
-                        if (ld_sys_u64(&db->stop) != 0) { why = 1; break; }
-                        if (globaltimer_ns() > deadline) { why = 2; break; }
-                        __nanosleep(100);
+                        if ((polls & 7u) == 7u) {
+                            if (ld_sys_u64(&db->stop) != 0) { why = 1; break; }
+                            if (globaltimer_ns() > deadline) { why = 2; break; }
+                        }
+                        __nanosleep(50);
                     }
                 }
                 if (cmd == 0) st_sys_u64(&db->exited, why);
@@ -74,7 +77,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_co
                     const uint32_t go = ld_acquire_u32(&p.ctl->server_go);
                     if (go == epoch) { cmd = epoch; break; }
                     if (go == 0xffffffffu || globaltimer_ns() > deadline) break;
-                    __nanosleep(50);
+                    __nanosleep(20);
                 }
             }
             s_cmd = cmd;
