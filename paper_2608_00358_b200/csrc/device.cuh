@@ -586,9 +586,43 @@ static __device__ void reduce_n_dispatch(const ExecParams& p, const Desc& d, uin
 }
 
 // ------------------------------------------------------------------ one work item, all threads
+// The operand addresses of a COPY (one destination) or REDUCE item. With static chains the control warp works them
+// out for 32 items at once, one lane per item, so that the worker threads do not each walk from buffer kind and rank
+// to a base address and on to the tile's offset before their first load (0.25 us of a chain step of 0.75 us).
+struct Resolved {
+    char* dst;
+    const char* a;
+    const char* b;
+};
+__device__ __forceinline__ bool resolve(const ExecParams& p, const Desc& d, const Tile& t, Resolved& r) {
+    if (d.op == HCCL_OP_COPY && d.ndst <= 1) {
+        r.a = buf_base(p, d.kind_a, d.rank_a) + d.off_a + t.start;
+        r.dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + t.start;
+        r.b = nullptr;
+        return true;
+    }
+    if (d.op == HCCL_OP_REDUCE) {
+        r.dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + t.start * (d.dt_dst == HCCL_FP32 ? 4 : 2);
+        r.a = buf_base(p, d.kind_a, d.rank_a) + d.off_a + t.start * (d.dt_a == HCCL_FP32 ? 4 : 2);
+        r.b = buf_base(p, d.kind_b, d.rank_b) + d.off_b + t.start * (d.dt_b == HCCL_FP32 ? 4 : 2);
+        return true;
+    }
+    return false;
+}
+
 // TABLE: see reduce_n_tile (all `nth` threads call this together and may meet at the workers' named barrier).
+// `r`: the item's operand addresses if they have been worked out already, else null.
 template <bool TABLE>
-static __device__ void run_tile_lsu(const ExecParams& p, const Desc& d, const Tile& t, const uint32_t tid, const uint32_t nth) {
+static __device__ void run_tile_lsu(const ExecParams& p, const Desc& d, const Tile& t, const uint32_t tid, const uint32_t nth, const Resolved* r = nullptr) {
+    if (TABLE && r) {  // only the builds that can afford the code (and ever pass addresses)
+        if (d.op == HCCL_OP_COPY) {
+            if (d.kind_a == HCCL_BUF_SEND) copy_tile_lsu<true>(r->dst, r->a, t.count, tid, nth); else copy_tile_lsu<false>(r->dst, r->a, t.count, tid, nth);
+        } else {
+            if (d.kind_b == HCCL_BUF_SEND) reduce_dispatch<true>(d.dt_a, d.dt_b, d.dt_dst, r->dst, r->a, r->b, t.count, tid, nth);
+            else reduce_dispatch<false>(d.dt_a, d.dt_b, d.dt_dst, r->dst, r->a, r->b, t.count, tid, nth);
+        }
+        return;
+    }
     switch (d.op) {
         case HCCL_OP_COPY: {
             const char* src = buf_base(p, d.kind_a, d.rank_a) + d.off_a + t.start;
@@ -709,18 +743,23 @@ static __device__ bool fetch_tile(const ExecParams& p, uint32_t cur, Tile& t, De
 constexpr uint32_t WINDOW = 32;
 // Each lane also runs the checks on its own item, so that lane 0 later only copies the records (its work between two
 // items of a chain is on the chain's critical path, one instruction after the other).
-__device__ __forceinline__ void window_fill(const ExecParams& p, uint32_t first, uint32_t end, uint32_t lane, Tile* wt, Desc* wd, uint8_t* wok) {
+// wok: 0 the item fails its checks, 1 it passes, 2 it passes and its operand addresses are in wr.
+__device__ __forceinline__ void window_fill(const ExecParams& p, uint32_t first, uint32_t end, uint32_t lane, Tile* wt, Desc* wd, Resolved* wr, uint8_t* wok) {
     const uint32_t idx = first + lane;
     if (idx < end && idx < p.n_tiles) {
         const Tile t = p.tiles[idx];
         wt[lane] = t;
-        bool ok = false;
+        uint8_t ok = 0;
         if (!(t.flags & TILE_FLAG_END) && tile_ok(p, t)) {
             const Desc d = p.descs[t.desc];
             wd[lane] = d;
-            ok = desc_ok(p, d);
+            if (desc_ok(p, d)) {
+                Resolved r;
+                ok = resolve(p, d, t, r) ? 2 : 1;
+                if (ok == 2) wr[lane] = r;
+            }
         }
-        wok[lane] = ok ? 1 : 0;
+        wok[lane] = ok;
     }
     __syncwarp();
 }
@@ -808,6 +847,8 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     __shared__ Tile s_wtile[AHEAD ? WINDOW : 1];  // static chains: records of the items [win_base, win_base + WINDOW)
     __shared__ Desc s_wdesc[AHEAD ? WINDOW : 1];
     __shared__ uint8_t s_wok[AHEAD ? WINDOW : 1];   // the checks on them, done by the lane that fetched them
+    __shared__ Resolved s_wres[AHEAD ? WINDOW : 1]; // and their operand addresses
+    __shared__ Resolved s_res[2];                   // of the items in s_tile / s_desc (valid where s_go says 2)
     const bool window = AHEAD && p.chain_len != 0;
     uint32_t win_base = 0, win_end = 0;  // win_end: end of the block's items
     const uint32_t tid = threadIdx.x, nth = blockDim.x;
@@ -833,7 +874,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
     }
     if (window && tid < 32) {  // the tables do not change: they may be read before a trigger has fired
         chain_range(p, win_base, win_end);
-        window_fill(p, win_base, win_end, tid, s_wtile, s_wdesc, s_wok);
+        window_fill(p, win_base, win_end, tid, s_wtile, s_wdesc, s_wres, s_wok);
     }
     __syncthreads();
     if (tid >= 32) {
@@ -842,7 +883,7 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
             const uint32_t b = k & 1;
             named_sync(FULL + b, nth);
             if (!s_go[b]) break;
-            run_tile_lsu<AHEAD>(p, s_desc[b], s_tile[b], wtid, nwork);
+            run_tile_lsu<AHEAD>(p, s_desc[b], s_tile[b], wtid, nwork, s_go[b] == 2 ? &s_res[b] : nullptr);
             if (!window) named_sync(DONE + b, nth);  // static chains: the next item's FULL barrier says it as well
         }
         return;
@@ -865,7 +906,9 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
         cur = win_base;  // every lane keeps the item numbers (the lanes refill the window together)
         if (tid == 0) {
             const bool h = live && cur < end && !(gated ? aborted(p) : abort0 == g_epoch);
-            s_go[0] = h && fetch_windowed(p, cur, s_tile[0], s_desc[0], s_wtile[0], s_wdesc[0], s_wok[0]);
+            const bool f = h && fetch_windowed(p, cur, s_tile[0], s_desc[0], s_wtile[0], s_wdesc[0], s_wok[0]);
+            if (f && s_wok[0] == 2) s_res[0] = s_wres[0];
+            s_go[0] = f ? s_wok[0] : 0;  // 1: run it; 2: run it, its operand addresses are in s_res
         }
         for (uint32_t k = 0;; ++k) {
             const uint32_t b = k & 1;
@@ -880,13 +923,14 @@ __device__ __forceinline__ void executor_lsu_body(const ExecParams& p) {
             const uint32_t nx = cur + 1;
             if (nx < end && nx - win_base >= WINDOW) {
                 win_base = nx;
-                window_fill(p, win_base, win_end, tid, s_wtile, s_wdesc, s_wok);
+                window_fill(p, win_base, win_end, tid, s_wtile, s_wdesc, s_wres, s_wok);
             }
             if (tid == 0) {
                 const uint32_t ab = ld_relaxed_u32(&p.ctl->abort);  // asked for first, looked at when the records are in
                 const uint32_t slot = nx < end ? nx - win_base : 0;
                 const bool h = nx < end && fetch_windowed(p, nx, s_tile[b ^ 1], s_desc[b ^ 1], s_wtile[slot], s_wdesc[slot], s_wok[slot]);
-                s_go[b ^ 1] = h && ab != g_epoch;
+                if (h && s_wok[slot] == 2) s_res[b ^ 1] = s_wres[slot];
+                s_go[b ^ 1] = (h && ab != g_epoch) ? s_wok[slot] : 0;
             }
             prev_item = cur;
             cur = nx;
