@@ -504,11 +504,12 @@ hccl_status_t plan_allreduce_tree(int R, int64_t count, hccl_dtype_t dt, hccl_op
     const int64_t ng = count > 0 ? (count + granule - 1) / granule : 0;
     if (!group_given && count * 4 <= (32ll << 20)) o.chain_group = (int32_t)std::max<int64_t>(ng, 1);  // small: all granules together
     const int64_t group = std::max<int64_t>(1, o.chain_group);
-    // From about 1 MiB per rank (256 KiB up to 8 ranks) a block does better walking one tile through the whole tree by
-    // itself (no hand-over between SMs, 2(R-1) items in a row) than the blocks do sharing the tree's 2 log2 R levels;
-    // below that the levels' parallelism wins (measured at R = 8, per execution from a CUDA graph: 20.1 vs 38.2 us at
-    // 1 MiB, 19.9 vs 22.5 at 256 KiB, 19.5 vs 18.5 at 64 KiB; at R = 64 and 128 KiB 0.148 vs 0.058 ms).
-    if (count * es >= (R <= 8 ? (256ll << 10) : (1ll << 20)) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
+    // From about 1 MiB per rank (any size up to 8 ranks) a block does better walking one tile through the whole tree by
+    // itself (no hand-over between SMs, 2(R-1) items in a row at about 0.7 us each) than the blocks do sharing the
+    // tree's 2 log2 R levels at about 2.5 us per hand-over through a device counter; below that the levels' parallelism
+    // wins (measured per execution from a CUDA graph at R = 8: 12.7 vs 15.3 us at 4 KiB, 18.0 vs 19.0 at 64 KiB, 18.1
+    // vs 22.7 at 256 KiB, 18.5 vs 38.1 at 1 MiB; at R = 64 and 128 KiB 0.148 vs 0.058 ms).
+    if ((R <= 8 || count * es >= (1ll << 20)) && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) o.flags |= HCCL_FLAG_STATIC_CHAINS;
     const int half = (R + 1) / 2;                                 // scratch slots one granule needs
     const int64_t n_sets = std::min<int64_t>(std::max<int64_t>(ng, 1), 2 * group);  // recycled sets of slots
     const int64_t slot_elems = (int64_t)align_up((uint64_t)std::min<int64_t>(granule, std::max<int64_t>(count, 1)), 64);

@@ -429,7 +429,7 @@ def test_tree_as_groups_inside_one_block(R, n, dt):
     HCCL_FLAG_STATIC_CHAINS a block runs tile k of the whole group in issue order. Same bits as with tickets."""
     X = synth.normal_ranks(R, n, dt, seed=R + n)
     want = orc.allreduce_tree_f32(dt, X)
-    for flags, grouped in ((hb.FLAG_STATIC_CHAINS, True), (0, False)):
+    for flags, grouped in ((hb.FLAG_STATIC_CHAINS, True), (hb.FLAG_DYNAMIC_TICKETS, False)):
         p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_TREE, dict(tile_bytes=512, chunk_bytes=2048, chain_group=64, sm_budget=5, flags=flags))
         i = p.info()
         assert (i.static_chains > 0) == grouped and p.check_hazards() == 0
