@@ -9,7 +9,7 @@ CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libhccl_b200.so")
 # one translation unit per kernel, so that they compile in parallel (each takes about a minute)
 SOURCES = ["graph.cpp", "collectives.cpp", "verify.cpp", "executor.cu", "kernel_lsu.cu", "kernel_lsu_light.cu", "kernel_bulk.cu",
-           "kernel_resident.cu"]
+           "kernel_resident.cu", "kernel_chain.cu"]
 HEADERS = ["plan.hpp", "tables.h", "device.cuh", "bulk.cuh", "bulk_layout.h", "kernels.cuh", os.path.join("..", "..", "include", "hccl.h")]
 # a kernel's unit does not use every helper of the shared headers: no "declared but never referenced" remarks for them
 QUIET = ["-diag-suppress", "177"]

@@ -43,6 +43,7 @@ hccl_status_t hccl_plan_bind(hccl_plan_t* p, void* dev_workspace, size_t bytes, 
         if (smem > 48 * 1024) CUDA_TRY(cudaFuncSetAttribute(hccl_a2a_dynamic, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(DYN_MAX_RANKS * DYN_MAX_RANKS * 24 + (DYN_MAX_RANKS * DYN_MAX_RANKS + 1) * 4 + 16)));
     } else if (p->opts.engine == HCCL_ENGINE_BULK) {
         CUDA_TRY(cudaFuncSetAttribute(hccl_executor_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk::MAX_DYNAMIC_SMEM));
+        if (p->chain_len) CUDA_TRY(cudaFuncSetAttribute(hccl_executor_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM_BYTES));
     }
     p->workspace = dev_workspace;
     p->workspace_bytes = bytes;
@@ -230,7 +231,12 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     static thread_local ExecParams prm;  // 4 KB+: keep it off the stack
     const uint32_t epoch = p->epoch + 1;
     const int blocks = fill_params(p, prm, sendbufs, recvbufs);
-    if (p->opts.engine == HCCL_ENGINE_BULK) {
+    if (p->opts.engine == HCCL_ENGINE_BULK && p->chain_len) {
+        // stages sized for the widest operand that arrives through them (B of every step, A of a chain's first)
+        bool wide = false;
+        for (const Desc& d : p->descs) wide = wide || (d.op == HCCL_OP_REDUCE && (d.dt_b == HCCL_FP32 || (d.kind_a == HCCL_BUF_SEND && d.dt_a == HCCL_FP32)));
+        hccl_executor_chain<<<blocks, CHAIN_THREADS, CHAIN_SMEM_BYTES, (cudaStream_t)stream>>>(prm, wide ? 3u : 6u, CHAIN_PIECE_ELEMS * (wide ? 4u : 2u));
+    } else if (p->opts.engine == HCCL_ENGINE_BULK) {
         const bulk::StageConfig sc = bulk::stage_config(p->opts.stages, p->opts.stage_kib);
         const int threads = std::max(128, p->opts.threads);
         hccl_executor_bulk<<<blocks, threads, sc.smem, (cudaStream_t)stream>>>(prm, sc.ns, (uint32_t)(p->opts.copy_by_warps == 1 || (p->opts.copy_by_warps == 0 && p->opts.sm_budget < 100)),

@@ -399,7 +399,12 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         for (int64_t q : pe[i]) depth[i] = std::max(depth[i], depth[q] + 1);
         max_depth = std::max(max_depth, depth[i]);
     }
-    bool chains = (p->opts.flags & HCCL_FLAG_STATIC_CHAINS) != 0 && p->opts.engine == HCCL_ENGINE_LSU && n > 0 && max_depth > 1;
+    // On the bulk engine static chains run in the forwarding kernel, which is built for chains of REDUCE items (anything
+    // else it runs item by item through its few compute warps): only packets made of REDUCE items go there.
+    bool chains = (p->opts.flags & HCCL_FLAG_STATIC_CHAINS) != 0 && n > 0 && max_depth > 1;
+    if (chains && p->opts.engine != HCCL_ENGINE_LSU)
+        for (size_t j = 0; j < n && chains; ++j)
+            if (g->wqes[j].w.op != HCCL_OP_REDUCE) chains = false;
     // Every dependency must be a tile-by-tile link; WQEs linked (directly or not) form a group that one block runs
     // in issue order, which already has every predecessor before its successors. A ring's chain is such a
     // group; so is a chunk that forks into several racks. Groups must be equally long, so that a block finds

@@ -1,0 +1,395 @@
+// Static chains on the bulk copy unit: a block walks a piece of 14336 elements through every step of its chain with the
+// running FP32 sums held in registers.
+//
+// A ring ReduceScatter (paper Sec. II-A.2: send, receive, compute WQEs, step after step) is, per chunk, a chain of
+// S = A + B items in which A of step t+1 is what step t stored. The other engines read that partial back from the
+// L2; per element and step that is 4 bytes stored, 4 read back and 2 (bf16) read from the own input through an SM's
+// port to the L2, which moves about 63 GB/s of stores and takes loads and stores in turn. Here every step still
+// stores its result where its descriptor says, but the thread that stored an element keeps it and adds the next
+// step's B to it: 4 bytes stored and 2 loaded per element and step. The B operands (send buffers, which no step
+// writes) are fetched ahead by cp.async.bulk into a ring of stages; stores are plain 16-byte stores from registers.
+//
+// Warp 0: lane 0 is the DMA thread; all 32 lanes fetch and check the records of a chain's steps together. Warps 1-7
+// are the compute warps. A chain whose steps are not all of the form above (another operation, an operand that is
+// not 16-byte aligned, B not in a send buffer, an A that is neither a send buffer nor the step before) runs item by
+// item through the register path, as the register engine's static chains do.
+#include "bulk.cuh"
+#include "kernels.cuh"
+
+namespace hccl {
+namespace chainfw {
+using namespace bulk;
+
+constexpr uint32_t CW = 7, CTH = CW * 32;    // compute warps, compute threads: 8 warps in all, so that a thread may have 255 registers
+                                             // (nine warps are given registers like twelve: 168, and the 32 running sums spill)
+constexpr int G = 16;                         // groups of 4 elements per compute thread and piece
+constexpr uint32_t PIECE = CTH * 4 * G;      // elements per piece: 64 per compute thread (one DMA issue per piece: the fewer the better)
+constexpr uint32_t MAX_NS = 6;               // stages: 6 of PIECE * 2 bytes (16-bit operands) or 3 of PIECE * 4 (FP32)
+constexpr uint32_t MAX_STEPS = 512;          // items per chain that fit the step table (2 R - 2 for R = 256: 510)
+
+enum : uint32_t { K_A = 0, K_B = 1, K_ITEM = 2, K_EXIT = 3 };
+struct alignas(16) Piece {
+    char* dst;                  // K_B: where this piece's sums go
+    const char* tail_src;       // K_A, K_B: the operand's last (n mod 8) elements, read with plain loads
+    const char* discard;        // K_B: FP32 partial that a non-forwarding engine would read here for the last time (or null)
+    uint32_t n;                 // elements in the piece
+    uint32_t item;              // work item: K_ITEM runs it whole; trace and failure reports
+    uint8_t kind, dt_src, dt_dst, keep;
+    uint8_t last, pad[3];       // last piece of its item (trace)
+};
+struct alignas(8) Step {        // one item of the current chain, tile offset applied
+    char* dst;
+    const char* a;
+    const char* b;
+    uint32_t n;
+    uint32_t item;
+    uint8_t dt_a, dt_b, dt_dst, flags;
+};
+enum : uint8_t { S_OK = 1, S_FAST = 2, S_KEEP = 4, S_DISCARD_A = 8 };
+
+template <int DS>
+__device__ __forceinline__ void take(const char* stage, uint32_t nv, uint32_t ctid, float (&S)[G][4]) {
+#pragma unroll
+    for (int k = 0; k < G; ++k) {
+        const uint32_t e = (k * CTH + ctid) * 4;
+        if (e < nv) lds4<DS>(stage + (size_t)e * Elem<DS>::BYTES, S[k]);
+    }
+}
+// The add and the store are separate steps (three variants by the operand's type, four by the destination's), not
+// twelve fused ones: with those inlined side by side the compiler ran out of its 255 registers.
+template <int DS>
+__device__ __forceinline__ void accumulate(const char* stage, uint32_t nv, uint32_t ctid, float (&S)[G][4]) {
+#pragma unroll
+    for (int h = 0; h < G; h += 8) {  // eight loads in flight at a time
+        float b[8][4];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t e = ((h + k) * CTH + ctid) * 4;
+            if (e < nv) lds4<DS>(stage + (size_t)e * Elem<DS>::BYTES, b[k]);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const uint32_t e = ((h + k) * CTH + ctid) * 4;
+            if (e < nv) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) S[h + k][j] = S[h + k][j] + b[k][j];
+            }
+        }
+    }
+}
+template <int DD, bool KEEP>
+__device__ __forceinline__ void store_all(char* dst, uint32_t nv, uint32_t ctid, const float (&S)[G][4], unsigned long long pol) {
+#pragma unroll
+    for (int k = 0; k < G; ++k) {
+        const uint32_t e = (k * CTH + ctid) * 4;
+        if (e < nv) stg4<DD, KEEP>(dst + (size_t)e * Elem<DD>::BYTES, S[k], pol);
+    }
+}
+__device__ __forceinline__ float load_elem(int dt, const char* p, uint32_t i) {
+    return dt == HCCL_FP32 ? Elem<HCCL_FP32>::load(p, i) : dt == HCCL_BF16 ? Elem<HCCL_BF16>::load(p, i) : Elem<HCCL_FP16>::load(p, i);
+}
+__device__ __forceinline__ void store_elem(int dt, char* p, uint32_t i, float v) {
+    if (dt == HCCL_FP32) Elem<HCCL_FP32>::store(p, i, v); else if (dt == HCCL_BF16) Elem<HCCL_BF16>::store(p, i, v); else Elem<HCCL_FP16>::store(p, i, v);
+}
+__device__ __forceinline__ uint32_t esize(int dt) { return dt == HCCL_FP32 ? 4u : 2u; }
+// The compute warps' bounded wait, inlined: across a call the 32 running sums of every thread would be written to local
+// memory and read back, once per piece (the L1 has little room left beside the stages, so from the L2).
+__device__ __forceinline__ bool wait_inline(const ExecParams& p, uint32_t bar, uint32_t parity, unsigned long long budget_ns, uint32_t detail) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long deadline = 0;
+    for (uint32_t spins = 1;; ++spins) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spins & 31u) == 0) {
+            if (aborted(p)) return false;
+            const unsigned long long now = globaltimer_ns();
+            if (deadline == 0) deadline = now + budget_ns;
+            if (now > deadline) {
+                fail(p, HCCL_ERR_TIMEOUT, detail);
+                return false;
+            }
+        }
+    }
+}
+// Bounded wait that does not look at the abort word (for loads that are in flight whatever happens to the execution).
+__device__ __forceinline__ void mbar_wait_quiet(uint32_t bar, uint32_t parity, unsigned long long budget_ns) {
+    if (mbar_try_wait(bar, parity)) return;
+    const unsigned long long deadline = globaltimer_ns() + budget_ns;
+    while (!mbar_try_wait(bar, parity) && globaltimer_ns() < deadline) {}
+}
+
+}  // namespace chainfw
+
+using namespace chainfw;
+
+__global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t stage_bytes) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ __align__(8) unsigned long long s_bar[2 * MAX_NS + 1];  // full, empty, and the compute warps' own barrier
+    __shared__ Piece s_info[MAX_NS];
+    __shared__ Step s_step[MAX_STEPS];
+    const uint32_t tid = threadIdx.x;
+    const uint32_t stages = smem_u32(smem), full = smem_u32(s_bar), empty = full + 8 * MAX_NS, cbar = empty + 8 * MAX_NS;
+    if (tid == 0) {
+        for (uint32_t s = 0; s < ns; ++s) {
+            mbar_init(full + 8 * s, 1);
+            mbar_init(empty + 8 * s, CW);
+        }
+        mbar_init(cbar, CW);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    init_epoch(p);  // ends with __syncthreads
+    const unsigned long long long_wait = 2 * p.timeout_ns + 1000000000ull;
+    const bool lean = p.trig_set_slot < 0;
+
+    if (tid >= 32) {
+        // ------------------------------------------------------------ compute warps
+        const uint32_t ctid = tid - 32, lane = tid & 31u;
+        const unsigned long long pol_keep = policy_evict_last();
+        float S[G][4];
+        float s_tail = 0.f;
+#pragma unroll
+        for (int k = 0; k < G; ++k)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) S[k][j] = 0.f;
+        uint32_t cpar = 0;  // phase parity of the compute warps' barrier
+        for (uint32_t slot = 0, parity = 0;;) {
+            if (!wait_inline(p, full + 8 * slot, parity, long_wait, 0xfffffff7u)) break;
+            const Piece pi = s_info[slot];
+            if (pi.kind == K_EXIT) {
+                if (!lean) __threadfence();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty + 8 * slot);  // tells the DMA thread that everything is stored
+                break;
+            }
+            const char* stage = (const char*)smem + (size_t)slot * stage_bytes;
+            const uint32_t nv = pi.n & ~7u, rem = pi.n - nv;
+            if (pi.kind == K_A) {
+                if (pi.dt_src == HCCL_FP32) take<HCCL_FP32>(stage, nv, ctid, S);
+                else if (pi.dt_src == HCCL_BF16) take<HCCL_BF16>(stage, nv, ctid, S);
+                else take<HCCL_FP16>(stage, nv, ctid, S);
+                if (ctid < rem) s_tail = load_elem(pi.dt_src, pi.tail_src, ctid);
+            } else if (pi.kind == K_B) {
+                if (pi.dt_src == HCCL_FP32) accumulate<HCCL_FP32>(stage, nv, ctid, S);
+                else if (pi.dt_src == HCCL_BF16) accumulate<HCCL_BF16>(stage, nv, ctid, S);
+                else accumulate<HCCL_FP16>(stage, nv, ctid, S);
+                if (pi.dt_dst == HCCL_FP32) {
+                    if (pi.keep) store_all<HCCL_FP32, true>(pi.dst, nv, ctid, S, pol_keep); else store_all<HCCL_FP32, false>(pi.dst, nv, ctid, S, pol_keep);
+                } else if (pi.dt_dst == HCCL_BF16) {
+                    store_all<HCCL_BF16, false>(pi.dst, nv, ctid, S, pol_keep);
+                } else {
+                    store_all<HCCL_FP16, false>(pi.dst, nv, ctid, S, pol_keep);
+                }
+                if (ctid < rem) {
+                    s_tail = s_tail + load_elem(pi.dt_src, pi.tail_src, ctid);
+                    store_elem(pi.dt_dst, pi.dst, nv + ctid, s_tail);
+                }
+                if (pi.discard) {
+                    // whole 128-byte lines inside the partial that a re-reading engine would have read here for the last time
+                    const uintptr_t lo = ((uintptr_t)pi.discard + 127u) & ~(uintptr_t)127u, hi = ((uintptr_t)pi.discard + (size_t)pi.n * 4) & ~(uintptr_t)127u;
+                    for (uintptr_t a = lo + (uintptr_t)ctid * 128u; a < hi; a += (uintptr_t)CTH * 128u) discard_line((const void*)a);
+                }
+                if (pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
+            } else {  // K_ITEM: the whole item through the register path; items of a chain follow each other in this block
+                // the item before must be stored by all compute threads. A bounded wait on an mbarrier, not a named barrier:
+                // a warp that has left an aborted execution would leave the others waiting at one for ever
+                __syncwarp();
+                if (lane == 0) mbar_arrive(cbar);
+                if (!wait_inline(p, cbar, cpar, long_wait, 0xfffffff3u)) break;
+                cpar ^= 1u;
+                const Tile t = p.tiles[pi.item];
+                run_tile_lsu<false>(p, p.descs[t.desc], t, ctid, CTH);
+                // nothing is forwarded out of an item that ran this way (and the sums need not survive the call)
+                s_tail = 0.f;
+#pragma unroll
+                for (int k = 0; k < G; ++k)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) S[k][j] = 0.f;
+                if (p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + 8 * slot);
+            if (++slot == ns) {
+                slot = 0;
+                parity ^= 1u;
+            }
+        }
+        return;
+    }
+
+    // ------------------------------------------------------------ warp 0: DMA thread (lane 0) and the step table (all lanes)
+    const uint32_t lane = tid;
+    const unsigned long long pol = policy_evict_first();
+    uint32_t first = 0, end = 0;
+    chain_range(p, first, end);
+    end = min(end, p.n_tiles);
+    bool ok = true;
+    if (lane == 0) {
+        if (p.trig_wait_slot >= 0)
+            ok = wait_signal(p, p.user_signals + p.trig_wait_slot, p.trig_cmp, p.trig_wait_value + (unsigned long long)g_epoch * p.trig_wait_per_epoch, 0xffffffffu);
+        if (ok && aborted(p)) ok = false;
+        if (first == 0 && first < end) p.ctl->t_first_ns = globaltimer_ns();
+    }
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    uint32_t slot = 0, parity = 0;    // next stage to fill and the phase parity of this use of it
+    unsigned long long issued = 0;
+    // lane 0: make stage `slot` free for a new piece
+    auto acquire = [&]() -> bool {
+        if (issued >= ns && !mbar_wait(p, empty + 8 * slot, parity ^ 1u, long_wait, 0xfffffff6u)) return false;
+        return true;
+    };
+    auto advance = [&]() {
+        ++issued;
+        if (++slot == ns) {
+            slot = 0;
+            parity ^= 1u;
+        }
+    };
+    const uint32_t L = p.chain_len;
+    for (uint32_t base = first; ok && base < end; base += L) {
+        // ---- the chain's steps: records fetched, checked and resolved by the warp's lanes
+        bool good = true, fast = L <= MAX_STEPS;  // a longer chain runs item by item
+        for (uint32_t t0 = 0; t0 < L && good; t0 += 32) {
+            const uint32_t t = t0 + lane;
+            bool g = true, f = true;
+            if (t < L) {
+                const uint32_t item = base + t;
+                Step st;
+                st.item = item;
+                st.flags = 0;
+                st.n = 0;
+                st.dst = nullptr; st.a = nullptr; st.b = nullptr;
+                st.dt_a = st.dt_b = st.dt_dst = 0;
+                const Tile tl = p.tiles[item];
+                g = tile_ok(p, tl) && !(tl.flags & TILE_FLAG_END);
+                if (g) {
+                    const Desc d = p.descs[tl.desc];
+                    g = desc_ok(p, d);
+                    if (g) {
+                        st.flags = S_OK;
+                        st.n = tl.count;
+                        st.dt_a = d.dt_a; st.dt_b = d.dt_b; st.dt_dst = d.dt_dst;
+                        f = d.op == HCCL_OP_REDUCE && d.kind_b == HCCL_BUF_SEND;
+                        if (f) {
+                            st.dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + tl.start * esize(d.dt_dst);
+                            st.a = buf_base(p, d.kind_a, d.rank_a) + d.off_a + tl.start * esize(d.dt_a);
+                            st.b = buf_base(p, d.kind_b, d.rank_b) + d.off_b + tl.start * esize(d.dt_b);
+                            f = (((uintptr_t)st.dst | (uintptr_t)st.a | (uintptr_t)st.b) & 15u) == 0;
+                            if (t == 0 && (d.kind_a != HCCL_BUF_SEND || PIECE * esize(d.dt_a) > stage_bytes)) f = false;
+                            if (PIECE * esize(d.dt_b) > stage_bytes) f = false;  // the launch sized the stages for 16-bit operands
+                            if (d.kind_dst == HCCL_BUF_SCRATCH && d.dt_dst == HCCL_FP32) st.flags |= S_KEEP;
+                            if ((d.cmp & HCCL_HINT_LAST_READ_A) && d.kind_a == HCCL_BUF_SCRATCH && d.dt_a == HCCL_FP32) st.flags |= S_DISCARD_A;
+                        }
+                    }
+                }
+                if (t < MAX_STEPS) s_step[t] = st;
+            }
+            good = __all_sync(0xffffffffu, g);
+            fast = fast && __all_sync(0xffffffffu, f);
+        }
+        __syncwarp();
+        if (good && fast) {
+            // every step after the first must take exactly what the step before stored, as FP32
+            for (uint32_t t0 = 1; t0 < L; t0 += 32) {
+                const uint32_t t = t0 + lane;
+                bool f = true;
+                if (t < L) f = s_step[t].a == s_step[t - 1].dst && s_step[t].dt_a == HCCL_FP32 && s_step[t - 1].dt_dst == HCCL_FP32 && s_step[t].n == s_step[t - 1].n;
+                fast = fast && __all_sync(0xffffffffu, f);
+            }
+        }
+        if (lane == 0) {
+            if (!good) {
+                fail(p, HCCL_ERR_BAD_DESCRIPTOR, base);
+                ok = false;
+            } else if (!fast) {
+                for (uint32_t t = 0; t < L && ok; ++t) {
+                    if (!acquire()) { ok = false; break; }
+                    Piece& pi = s_info[slot];
+                    pi.kind = K_ITEM;
+                    pi.item = base + t;
+                    pi.n = 0;
+                    if (p.trace) {
+                        trace_put(p.trace, p.trace_cap, base + t, 0, (unsigned long long)(base + t) | ((unsigned long long)blockIdx.x << 32));
+                        trace_put(p.trace, p.trace_cap, base + t, 1, globaltimer_ns());
+                        trace_put(p.trace, p.trace_cap, base + t, 2, globaltimer_ns());
+                    }
+                    mbar_arrive(full + 8 * slot);
+                    advance();
+                }
+            } else {
+                const uint32_t n = s_step[0].n;
+                for (uint32_t e0 = 0; e0 < n && ok; e0 += PIECE) {
+                    const uint32_t ne = min(PIECE, n - e0), nv = ne & ~7u;
+                    for (uint32_t t = 0; t < L && ok; ++t) {
+                        const Step& st = s_step[t];
+                        if (p.trace && e0 == 0) {
+                            trace_put(p.trace, p.trace_cap, st.item, 0, (unsigned long long)st.item | ((unsigned long long)blockIdx.x << 32));
+                            trace_put(p.trace, p.trace_cap, st.item, 1, globaltimer_ns());
+                            trace_put(p.trace, p.trace_cap, st.item, 2, globaltimer_ns());
+                        }
+                        if (t == 0) {  // the chain's first operand, from a send buffer
+                            if (!acquire()) { ok = false; break; }
+                            Piece& pa = s_info[slot];
+                            const uint32_t ea = esize(st.dt_a);
+                            pa.kind = K_A;
+                            pa.n = ne;
+                            pa.item = st.item;
+                            pa.dt_src = st.dt_a;
+                            pa.tail_src = st.a + (size_t)(e0 + nv) * ea;
+                            if (nv) {
+                                mbar_arrive_expect_tx(full + 8 * slot, nv * ea);
+                                bulk_load(stages + slot * stage_bytes, st.a + (size_t)e0 * ea, nv * ea, full + 8 * slot, true, pol);
+                            } else {
+                                mbar_arrive(full + 8 * slot);
+                            }
+                            advance();
+                        }
+                        if (!acquire()) { ok = false; break; }
+                        Piece& pb = s_info[slot];
+                        const uint32_t eb = esize(st.dt_b), ed = esize(st.dt_dst);
+                        pb.kind = K_B;
+                        pb.n = ne;
+                        pb.item = st.item;
+                        pb.dt_src = st.dt_b;
+                        pb.dt_dst = st.dt_dst;
+                        pb.keep = (st.flags & S_KEEP) ? 1 : 0;
+                        pb.last = (e0 + ne == n) ? 1 : 0;
+                        pb.dst = st.dst + (size_t)e0 * ed;
+                        pb.tail_src = st.b + (size_t)(e0 + nv) * eb;
+                        pb.discard = (t > 0 && (st.flags & S_DISCARD_A)) ? st.a + (size_t)e0 * 4 : nullptr;
+                        if (nv) {
+                            mbar_arrive_expect_tx(full + 8 * slot, nv * eb);
+                            bulk_load(stages + slot * stage_bytes, st.b + (size_t)e0 * eb, nv * eb, full + 8 * slot, true, pol);
+                        } else {
+                            mbar_arrive(full + 8 * slot);
+                        }
+                        advance();
+                    }
+                }
+            }
+            if (ok && aborted(p)) ok = false;
+        }
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+    }
+    if (lane != 0) return;
+    if (ok && acquire()) {
+        // the end marker; the compute warps answer on its `empty` barrier when all their stores are issued
+        s_info[slot].kind = K_EXIT;
+        mbar_arrive(full + 8 * slot);
+        mbar_wait(p, empty + 8 * slot, parity, long_wait, 0xfffffff5u);
+    } else {
+        // given up (a failure is on record, or the execution was aborted): the compute warps leave at their next bounded
+        // wait. Loads already issued still write into this block's stages: wait (bounded) for each of them to land.
+        const unsigned long long back = issued < ns ? issued : ns;
+        for (unsigned long long k = 0; k < back; ++k) {
+            if (slot == 0) {
+                slot = ns;
+                parity ^= 1u;
+            }
+            --slot;
+            mbar_wait_quiet(full + 8 * slot, parity, 2000000000ull);
+        }
+    }
+    leave(p, lean);
+}
+
+}  // namespace hccl

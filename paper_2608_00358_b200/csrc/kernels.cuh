@@ -60,6 +60,9 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_lsu(const __grid_constan
 __global__ void __launch_bounds__(512, 2) hccl_executor_lsu_light(const __grid_constant__ ExecParams p);
 __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t copy_by_warps,
                                                               const uint32_t stage_bytes);
+// static chains on the bulk copy unit: running sums forwarded from step to step in registers
+constexpr uint32_t CHAIN_SMEM_BYTES = 6 * 28672, CHAIN_PIECE_ELEMS = 14336, CHAIN_THREADS = 256;  // 6 stages of 16-bit pieces or 3 of FP32 pieces
+__global__ void __launch_bounds__(256, 1) hccl_executor_chain(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t stage_bytes);
 __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_constant__ ExecParams p, Doorbell* db,
                                                                   const unsigned long long idle_ns, const uint32_t first_epoch);
 __global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant__ DynParams q);
