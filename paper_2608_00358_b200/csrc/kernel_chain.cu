@@ -27,9 +27,9 @@ constexpr uint32_t PIECE = CTH * 4 * G;      // elements per piece: 64 per compu
 constexpr uint32_t MAX_NS = 6;               // stages: 6 of PIECE * 2 bytes (16-bit operands) or 3 of PIECE * 4 (FP32)
 constexpr uint32_t MAX_STEPS = 512;          // items per chain that fit the step table (2 R - 2 for R = 256: 510)
 
-enum : uint32_t { K_A = 0, K_B = 1, K_ITEM = 2, K_EXIT = 3 };
+enum : uint32_t { K_A = 0, K_B = 1, K_ITEM = 2, K_EXIT = 3, K_C = 4 };
 struct alignas(16) Piece {
-    char* dst;                  // K_B: where this piece's sums go
+    char* dst;                  // K_B: where this piece's sums go; K_C: where the held values are copied to
     const char* tail_src;       // K_A, K_B: the operand's last (n mod 8) elements, read with plain loads
     const char* discard;        // K_B: FP32 partial that a non-forwarding engine would read here for the last time (or null)
     uint32_t n;                 // elements in the piece
@@ -45,7 +45,7 @@ struct alignas(8) Step {        // one item of the current chain, tile offset ap
     uint32_t item;
     uint8_t dt_a, dt_b, dt_dst, flags;
 };
-enum : uint8_t { S_OK = 1, S_FAST = 2, S_KEEP = 4, S_DISCARD_A = 8 };
+enum : uint8_t { S_OK = 1, S_COPY = 2, S_KEEP = 4, S_DISCARD_A = 8 };
 
 template <int DS>
 __device__ __forceinline__ void take(const char* stage, uint32_t nv, uint32_t ctid, float (&S)[G][4]) {
@@ -189,6 +189,12 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                     for (uintptr_t a = lo + (uintptr_t)ctid * 128u; a < hi; a += (uintptr_t)CTH * 128u) discard_line((const void*)a);
                 }
                 if (pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
+            } else if (pi.kind == K_C) {
+                if (pi.dt_dst == HCCL_FP32) store_all<HCCL_FP32, false>(pi.dst, nv, ctid, S, pol_keep);
+                else if (pi.dt_dst == HCCL_BF16) store_all<HCCL_BF16, false>(pi.dst, nv, ctid, S, pol_keep);
+                else store_all<HCCL_FP16, false>(pi.dst, nv, ctid, S, pol_keep);
+                if (ctid < rem) store_elem(pi.dt_dst, pi.dst, nv + ctid, s_tail);
+                if (pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
             } else {  // K_ITEM: the whole item through the register path; items of a chain follow each other in this block
                 // the item before must be stored by all compute threads. A bounded wait on an mbarrier, not a named barrier:
                 // a warp that has left an aborted execution would leave the others waiting at one for ever
@@ -268,8 +274,18 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                         st.flags = S_OK;
                         st.n = tl.count;
                         st.dt_a = d.dt_a; st.dt_b = d.dt_b; st.dt_dst = d.dt_dst;
-                        f = d.op == HCCL_OP_REDUCE && d.kind_b == HCCL_BUF_SEND;
-                        if (f) {
+                        if (d.op == HCCL_OP_COPY) {
+                            // a copy of what the step before stored (a ring's AllGather hops): the block stores what it holds again
+                            f = t > 0 && d.ndst <= 1;
+                            st.flags |= S_COPY;
+                            st.dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + tl.start;
+                            st.a = buf_base(p, d.kind_a, d.rank_a) + d.off_a + tl.start;
+                            st.n = tl.count;  // bytes for now; elements once the type of the held values is known (below)
+                            f = f && (((uintptr_t)st.dst | (uintptr_t)st.a) & 15u) == 0;
+                        } else {
+                            f = d.op == HCCL_OP_REDUCE && d.kind_b == HCCL_BUF_SEND;
+                        }
+                        if (f && d.op == HCCL_OP_REDUCE) {
                             st.dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + tl.start * esize(d.dt_dst);
                             st.a = buf_base(p, d.kind_a, d.rank_a) + d.off_a + tl.start * esize(d.dt_a);
                             st.b = buf_base(p, d.kind_b, d.rank_b) + d.off_b + tl.start * esize(d.dt_b);
@@ -287,16 +303,22 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
             fast = fast && __all_sync(0xffffffffu, f);
         }
         __syncwarp();
-        if (good && fast) {
-            // every step after the first must take exactly what the step before stored, as FP32
-            for (uint32_t t0 = 1; t0 < L; t0 += 32) {
-                const uint32_t t = t0 + lane;
-                bool f = true;
-                if (t < L) f = s_step[t].a == s_step[t - 1].dst && s_step[t].dt_a == HCCL_FP32 && s_step[t - 1].dt_dst == HCCL_FP32 && s_step[t].n == s_step[t - 1].n;
-                fast = fast && __all_sync(0xffffffffu, f);
-            }
-        }
         if (lane == 0) {
+            if (good && fast) {
+                // every step after the first must take exactly what the step before stored: a sum takes an FP32 sum, a copy
+                // takes whatever the block holds (and learns its element type from the step before)
+                for (uint32_t t = 1; t < L && fast; ++t) {
+                    Step& st = s_step[t];
+                    const Step& pv = s_step[t - 1];
+                    if (st.a != pv.dst) fast = false;
+                    else if (st.flags & S_COPY) {
+                        st.dt_dst = pv.dt_dst;
+                        if (st.n != pv.n * esize(pv.dt_dst)) fast = false;
+                        st.n = pv.n;
+                    } else if ((pv.flags & S_COPY) || st.dt_a != HCCL_FP32 || pv.dt_dst != HCCL_FP32 || st.n != pv.n) fast = false;
+                }
+                if (s_step[0].flags & S_COPY) fast = false;
+            }
             if (!good) {
                 fail(p, HCCL_ERR_BAD_DESCRIPTOR, base);
                 ok = false;
@@ -342,6 +364,19 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                                 mbar_arrive(full + 8 * slot);
                             }
                             advance();
+                        }
+                        if (st.flags & S_COPY) {
+                            if (!acquire()) { ok = false; break; }
+                            Piece& pc = s_info[slot];
+                            pc.kind = K_C;
+                            pc.n = ne;
+                            pc.item = st.item;
+                            pc.dt_dst = st.dt_dst;
+                            pc.last = (e0 + ne == n) ? 1 : 0;
+                            pc.dst = st.dst + (size_t)e0 * esize(st.dt_dst);
+                            mbar_arrive(full + 8 * slot);
+                            advance();
+                            continue;
                         }
                         if (!acquire()) { ok = false; break; }
                         Piece& pb = s_info[slot];

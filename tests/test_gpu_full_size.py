@@ -235,14 +235,15 @@ def test_allreduce_r64_at_the_benchmarked_size(algo):
 
 def test_large_fp32_ring_allreduce_as_static_chains():
     """FP32 rings keep their partials in the receive buffers, so they run as static chains at any size
-    (default options, as a caller gets them): R = 4, 16 Mi elements per rank, every output against the oracle."""
+    (default options, as a caller gets them; at this size in the forwarding kernel of the bulk engine): R = 4,
+    16 Mi elements per rank, every output against the oracle."""
     R, n = 4, 1 << 24
     X = synth.uniform_ranks(R, n, hb.FP32, seed=24)
     send = [torch.from_numpy(x).cuda() for x in X]
     recv = [torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(R)]
     plan = hb.hccl_plan_allreduce(R, n, hb.FP32, hb.ALGO_RING)
     i = plan.info()
-    assert i.static_chains > 0 and i.n_syncs == 0 and i.engine == hb.ENGINE_LSU
+    assert i.static_chains > 0 and i.n_syncs == 0 and i.engine == hb.ENGINE_BULK
     wl = wk._bind("allreduce_r4_fp32_16Mi", plan, send, recv, {})
     for _ in range(2):
         wl.dc.execute()
