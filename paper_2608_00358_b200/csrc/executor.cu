@@ -233,8 +233,7 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     const int blocks = fill_params(p, prm, sendbufs, recvbufs);
     if (p->opts.engine == HCCL_ENGINE_BULK && p->chain_len) {
         // stages sized for the widest operand that arrives through them (B of every step, A of a chain's first)
-        bool wide = false;
-        for (const Desc& d : p->descs) wide = wide || (d.op == HCCL_OP_REDUCE && (d.dt_b == HCCL_FP32 || (d.kind_a == HCCL_BUF_SEND && d.dt_a == HCCL_FP32)));
+        const bool wide = p->chain_wide;
         hccl_executor_chain<<<blocks, CHAIN_THREADS, CHAIN_SMEM_BYTES, (cudaStream_t)stream>>>(prm, wide ? 3u : 6u, CHAIN_PIECE_ELEMS * (wide ? 4u : 2u));
     } else if (p->opts.engine == HCCL_ENGINE_BULK) {
         const bulk::StageConfig sc = bulk::stage_config(p->opts.stages, p->opts.stage_kib);

@@ -317,6 +317,41 @@ def test_bidirectional_ring_matches_oracle(R, n, dt):
         assert np.array_equal(Y[r].view(np_dtype(dt)).view(np.uint8), want[0][offs[r]:offs[r + 1]].view(np.uint8))
 
 
+# ----------------------------------------------------------------- rings for the forwarding kernel (bulk engine, static chains)
+@pytest.mark.parametrize("dt", DTYPES)
+def test_bulk_engine_rings_are_independent_chains_with_a_slot_each(dt):
+    """On the bulk engine a ring's chains get a scratch slot each (nothing is recycled, so nothing links them) and
+    the packet carries no device counter; the hazard checker and the random-order interpreter agree with the oracle."""
+    R, n = 5, 20011
+    X = synth.normal_ranks(R, n, dt, seed=78)
+    opts = dict(engine=hb.ENGINE_BULK, tile_bytes=2048, chunk_bytes=8192, sm_budget=6)
+    p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, opts)
+    i = p.info()
+    assert i.engine == hb.ENGINE_BULK and i.static_chains > 0 and i.n_syncs == 0 and p.check_hazards() == 0
+    want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    for seed in (0, 1):
+        Y = interpret(p, X, seed)
+        for r in range(R):
+            assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8))
+    p = hb.hccl_plan_reducescatter(R, None, n, dt, hb.ALGO_RING, opts)
+    assert p.info().static_chains > 0 and p.info().n_syncs == 0 and p.check_hazards() == 0
+    Y = interpret(p, X, 2)
+    for r, w in enumerate(orc.reducescatter_ring_f32(dt, X, np.diff(orc.floor_chunk_offsets(n, R)))):
+        assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
+    # what is not a set of simple REDUCE-then-COPY chains keeps tickets and counters on this engine
+    assert hb.hccl_plan_allgather(R, None, 777, dt, hb.ALGO_RING, opts).info().static_chains == 0
+    assert hb.hccl_plan_allreduce(8, 4099, dt, hb.ALGO_TREE, dict(opts, flags=hb.FLAG_STATIC_CHAINS)).info().static_chains == 0
+
+
+def test_engine_left_to_the_library_for_rings():
+    big = hb.hccl_plan_allreduce(8, 1 << 22, hb.BF16, hb.ALGO_RING).info()
+    assert big.engine == hb.ENGINE_BULK and big.static_chains >= 148 and big.n_syncs == 0
+    assert hb.hccl_plan_allreduce(8, 1 << 18, hb.BF16, hb.ALGO_RING).info().engine == hb.ENGINE_LSU
+    assert hb.hccl_plan_allreduce(64, 1 << 18, hb.BF16, hb.ALGO_RING).info().engine == hb.ENGINE_BULK
+    assert hb.hccl_plan_reducescatter(16, None, 1 << 26, hb.BF16, hb.ALGO_RING).info().static_chains > 0      # config 3
+    assert hb.hccl_plan_allreduce(8, 1 << 22, hb.BF16, hb.ALGO_RING, dict(flags=hb.FLAG_LEVEL_MAJOR)).info().engine == hb.ENGINE_LSU   # another issue order: as before
+
+
 # ----------------------------------------------------------------- static chains (a chain of tiles stays in one block)
 @pytest.mark.parametrize("dt", DTYPES)
 @pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_RING_FUSED])
