@@ -94,7 +94,8 @@ typedef enum {
 typedef enum {
     HCCL_ENGINE_AUTO = 0,
     HCCL_ENGINE_LSU = 1,  /* 128-bit vector loads/stores through registers */
-    HCCL_ENGINE_BULK = 2  /* cp.async.bulk (TMA) global->shared->global with mbarrier pipelining */
+    HCCL_ENGINE_BULK = 2  /* cp.async.bulk (TMA) global->shared->global with mbarrier pipelining; with static chains
+                             (ring reductions) the forwarding kernel, see HCCL_FLAG_STATIC_CHAINS */
 } hccl_engine_t;
 
 /* Ticket order of a reduction plan. */
@@ -113,9 +114,14 @@ typedef enum {
                                       that way are equally long (the chains of a small ring; the copies of one
                                       chunk in a hop-by-hop AllGather; a granule's tree of sums), run tile k of a
                                       whole group inside ONE block, in issue order: a barrier of that block then
-                                      stands where a device counter and a poll across SMs would. Register engine
-                                      only; ignored when the packet has another shape. The planners ask for it
-                                      themselves where it pays. */
+                                      stands where a device counter and a poll across SMs would. Ignored when the
+                                      packet has another shape. On the bulk engine only packets of simple chains
+                                      (one predecessor, one successor) of REDUCE items, optionally followed by
+                                      plain copies, run this way, in the forwarding kernel: a block walks a piece of
+                                      14336 elements through all steps of its chain with the running FP32 sums in
+                                      registers; every step's result is stored where its descriptor says, none is
+                                      read back. The planners ask for it themselves where it pays (rings with about
+                                      a chain of tiles per SM or more, each chain with a scratch slot of its own). */
 #define HCCL_FLAG_DYNAMIC_TICKETS 32u /* keep the planners from asking for HCCL_FLAG_STATIC_CHAINS */
 #define HCCL_FLAG_DEVICE_TABLES 64u /* hccl_plan_alltoallv_dynamic: build descriptors and tiles on the device and run
                                       them on the ordinary executor (always so beyond 64 ranks) */
