@@ -29,6 +29,8 @@ hccl_wqe_t blank() {
 }
 
 // One chain = one granule of one chunk travelling round the ring.
+constexpr int64_t kForwardPieceElems = 14336;  // elements the forwarding kernel moves per step and block (kernel_chain.cu)
+
 struct Chain {
     int c;            // chunk index = rank the reduced chunk ends on
     int64_t e0, len;  // element range [e0, e0+len) in the send buffers
@@ -177,9 +179,31 @@ int64_t pick_tile_elems(int64_t level_elems, const hccl_opts_t& o, int widest, i
 // running sums in registers, no partial read back). Measured against the register engine's static chains: AllReduce
 // bf16 R=8 0.66 at 8 MiB per rank, a tie at 4 MiB, 1.10 at 1 MiB; FP32 R=4 0.74 at 8 MiB, 1.07 at 4 MiB; bf16 R=64 0.85 at
 // 512 KiB, 1.44 at 128 KiB; ReduceScatter bf16 R=16 0.74 at 8 MiB, 0.95 at 2 MiB.
-bool ring_wants_forwarding(int R, int64_t count, bool fused, const hccl_opts_t& o) {
+// (Chunks that do not start on a multiple of 8 elements would make every operand miss the 16-byte alignment the bulk
+// copies need, and the kernel would run such chains item by item through its few compute warps: those stay where they were.)
+bool ring_wants_forwarding(int R, int64_t count, bool fused, const hccl_opts_t& o, const int64_t* recvcounts = nullptr) {
+    int64_t off = 0;
+    for (int c = 0; c < R; ++c) {
+        if (off % 8) return false;
+        off = recvcounts ? off + recvcounts[c] : (int64_t)(((__int128)(c + 1) * count) / R);
+    }
     if (o.chain_group != 0 || (o.flags & (HCCL_FLAG_DYNAMIC_TICKETS | HCCL_FLAG_LEVEL_MAJOR | HCCL_FLAG_STAGED_RING | HCCL_FLAG_BIDIRECTIONAL))) return false;
-    return !fused && R > 2 && count * 4 <= (1ll << 30) && (count >= (1ll << 21) || (R >= 32 && count >= (1ll << 18)));
+    return !fused && R > 2 && count * 4 <= (1ll << 30) && (count >= (1ll << 20) || (R >= 32 && count >= (1ll << 18)));
+}
+
+// Tile size for the forwarding kernel. A chain of tiles costs about the same however short its tiles are (a fixed cost
+// per step), and a block runs its chains one after the other: if one round of the blocks can take all chains, the
+// smallest tile that leaves no more chains than blocks; else whole pieces.
+int64_t forward_tile_elems(const std::vector<Chain>& chains, int blocks) {
+    int64_t total = 0;
+    for (const Chain& c : chains) total += c.len;
+    if (total > (int64_t)blocks * kForwardPieceElems || blocks <= 0) return kForwardPieceElems;
+    for (int64_t tile = std::max<int64_t>(256, (total / blocks + 7) / 8 * 8); tile < kForwardPieceElems; tile += 8) {
+        int64_t n = 0;
+        for (const Chain& c : chains) n += (c.len + tile - 1) / tile;
+        if (n <= blocks) return tile;
+    }
+    return kForwardPieceElems;
 }
 
 // Ring reductions: with the engine left to the library, large ones feed the adds from shared memory through
@@ -632,7 +656,6 @@ hccl_status_t plan_allreduce_tree(int R, int64_t count, hccl_dtype_t dt, hccl_op
 
 extern "C" {
 
-constexpr int64_t kForwardPieceElems = 14336;  // elements the forwarding kernel moves per step and block (kernel_chain.cu)
 constexpr int64_t kOwnSlotBytes = 48ll << 20;
 
 hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_algo_t algo, const hccl_opts_t* opts,
@@ -748,7 +771,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, in_recv ? es : 4, HCCL_OP_REDUCE, maxlen);
     // large FP32 rings as static chains: two passes of the block's threads per tile keep a block's current
     // partial (written by one step, read by the next) in the L2
-    if (forward && !o.tile_bytes) tile_elems = kForwardPieceElems;
+    if (forward && !o.tile_bytes) tile_elems = forward_tile_elems(chains, o.sm_budget);
     if (in_recv && o.engine == HCCL_ENGINE_LSU && !o.tile_bytes && count * 4 > (32ll << 20) && (o.flags & HCCL_FLAG_STATIC_CHAINS))
         tile_elems = 2 * sweep_of(o, HCCL_OP_REDUCE);
     if (!fused && o.engine == HCCL_ENGINE_LSU && (!opts || opts->sm_budget == 0) && maxlen > 0) {
@@ -773,7 +796,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_ONESHOT) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o, pre;
     if (opts) pre = *opts; else std::memset(&pre, 0, sizeof(pre));
-    if (algo == HCCL_ALGO_RING && pre.engine == HCCL_ENGINE_AUTO && ring_wants_forwarding(R, count, false, pre)) pre.engine = HCCL_ENGINE_BULK;
+    if (algo == HCCL_ALGO_RING && pre.engine == HCCL_ENGINE_AUTO && ring_wants_forwarding(R, count, false, pre, recvcounts)) pre.engine = HCCL_ENGINE_BULK;
     fill_ring_opts(&o, &pre, (int64_t)R * count * elem_bytes(dt), algo != HCCL_ALGO_RING || R == 1);
     const int es = elem_bytes(dt);
     std::vector<int64_t> offs(R + 1, 0);
@@ -849,7 +872,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     const int64_t scratch = need_scratch ? (int64_t)n_slots * slot_elems * 4 * (staged ? 2 : 1) : 0;
     const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
     int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, 4, HCCL_OP_REDUCE, maxlen);
-    if (forward && !o.tile_bytes) tile_elems = kForwardPieceElems;  // one piece of the forwarding kernel per tile: the most chains to share out
+    if (forward && !o.tile_bytes) tile_elems = forward_tile_elems(chains, o.sm_budget);
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), scratch, 0, &graw));
     GraphPtr g(graw);
     g->compulsory_bytes = compulsory;
