@@ -367,8 +367,8 @@ def run_profile_case(args):
         print(json.dumps(_round(_finite(dict(case="5 allreduce r8 bf16 4096 B one-shot, as the host sees it", **wk.time_host_observed(wl, 300))), 2)), flush=True)
         return
     if args.profile_case in ("c1chains", "c1tickets"):
-        # config 1 (AllReduce ring R = 4, 1 Mi fp32 per rank): static chains vs tickets and device counters
-        wl = wk.config1(dict(flags=0 if args.profile_case == "c1chains" else hb.FLAG_DYNAMIC_TICKETS))
+        # config 1 (AllReduce ring R = 4, 1 Mi fp32 per rank) on the register engine: static chains vs tickets and device counters
+        wl = wk.config1(dict(engine=hb.ENGINE_LSU, flags=0 if args.profile_case == "c1chains" else hb.FLAG_DYNAMIC_TICKETS))
     elif args.profile_case in ("agfanout", "agoneshot"):
         # AllGather R = 32, 1 Mi bf16 (2 MiB) per rank: 64 MiB read, 2 GiB written
         R, n = 32, 1 << 20
