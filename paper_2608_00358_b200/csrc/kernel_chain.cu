@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
         }
     };
     const uint32_t L = p.chain_len;
-    for (uint32_t base = first; ok && base < end; base += L) {
+    for (uint32_t base = first; ok && L > 0 && base < end; base += L) {
         // ---- the chain's steps: records fetched, checked and resolved by the warp's lanes
         bool good = true, fast = L <= MAX_STEPS;  // a longer chain runs item by item
         for (uint32_t t0 = 0; t0 < L && good; t0 += 32) {

@@ -276,10 +276,10 @@ def test_start_gate_that_never_opens_times_out_cleanly():
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("kind", ["ring_chains", "ring_tickets", "alltoallv_bulk"])
+@pytest.mark.parametrize("kind", ["ring_chains", "ring_tickets", "ring_forwarded", "alltoallv_bulk"])
 def test_device_triggered_static_plans(kind):
     """The start gate and the completion value on statically planned collectives: the register engine with static
-    chains and with tickets, and the bulk engine. The collective is enqueued first and holds (bounded) at its
+    chains and with tickets, the forwarding kernel, and the bulk engine. The collective is enqueued first and holds (bounded) at its
     gate on a few SMs; a fill on another stream releases it."""
     import torch
     from gpu_helpers import SENTINEL
@@ -295,9 +295,10 @@ def test_device_triggered_static_plans(kind):
     else:
         n = 30011
         X = synth.normal_ranks(R, n, hb.BF16, seed=9)
-        flags = 0 if kind == "ring_chains" else hb.FLAG_DYNAMIC_TICKETS
-        plan = hb.hccl_plan_allreduce(R, n, hb.BF16, hb.ALGO_RING, dict(sm_budget=8, tile_bytes=4096, chunk_bytes=16384, flags=flags))
-        assert (plan.info().static_chains > 0) == (kind == "ring_chains")
+        flags = hb.FLAG_DYNAMIC_TICKETS if kind == "ring_tickets" else 0
+        engine = hb.ENGINE_BULK if kind == "ring_forwarded" else hb.ENGINE_LSU
+        plan = hb.hccl_plan_allreduce(R, n, hb.BF16, hb.ALGO_RING, dict(sm_budget=8, tile_bytes=4096, chunk_bytes=16384, flags=flags, engine=engine))
+        assert (plan.info().static_chains > 0) == (kind != "ring_tickets") and plan.info().engine == engine
         want = [w.view(np.uint8) for w in orc.allreduce_ring_f32(hb.BF16, X, orc.floor_chunk_offsets(n, R))]
     send = [torch.from_numpy(x.view(np.uint8).copy()).cuda() for x in X]
     recv = [torch.full((max(plan.extents(r)[1], 16),), SENTINEL, dtype=torch.uint8, device="cuda") for r in range(R)]
@@ -324,12 +325,14 @@ def test_device_triggered_static_plans(kind):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("engine", [hb.ENGINE_LSU, hb.ENGINE_BULK], ids=["lsu", "bulk"])
-def test_static_plan_gate_that_never_opens_times_out_cleanly(engine):
+@pytest.mark.parametrize("engine,R,flags", [(hb.ENGINE_LSU, 2, 0), (hb.ENGINE_BULK, 2, hb.FLAG_DYNAMIC_TICKETS), (hb.ENGINE_BULK, 4, 0)],
+                         ids=["lsu", "bulk", "forwarding"])
+def test_static_plan_gate_that_never_opens_times_out_cleanly(engine, R, flags):
     import torch
-    R, n = 2, 4096
+    n = 4096
     X = synth.normal_ranks(R, n, hb.FP32, seed=1)
-    plan = hb.hccl_plan_allreduce(R, n, hb.FP32, hb.ALGO_RING, dict(sm_budget=2, timeout_ns=200_000_000, engine=engine))
+    plan = hb.hccl_plan_allreduce(R, n, hb.FP32, hb.ALGO_RING, dict(sm_budget=2, timeout_ns=200_000_000, engine=engine, flags=flags))
+    assert (plan.info().static_chains > 0) == (flags == 0)     # static chains on the bulk engine: the forwarding kernel
     send = [torch.from_numpy(x).cuda() for x in X]
     recv = [torch.full((n,), 7.0, dtype=torch.float32, device="cuda") for _ in range(R)]
     from paper_2608_00358_b200.runtime import DeviceCollective
