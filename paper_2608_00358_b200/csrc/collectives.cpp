@@ -71,7 +71,9 @@ hccl_status_t emit_ring(hccl_graph* g, int R, int dt, const std::vector<Chain>& 
             for (size_t i = g0; i < g1; ++i) {
                 const Chain& ch = chains[i];
                 const int c = ch.c;
-                const int64_t slot = (int64_t)(i % (size_t)std::max(n_slots, 1)) * slot_elems * 4;
+                // (AllReduce: the partial sits at the element phase, modulo 8, of the rank buffers' range it belongs to, so that
+                // all operands of a step reach a 16-byte boundary after the same number of elements; slots leave room for it)
+                const int64_t slot = (int64_t)(i % (size_t)std::max(n_slots, 1)) * slot_elems * 4 + (gather ? (ch.e0 % 8) * 4 : 0);
                 hccl_wqe_t w = blank();
                 w.tile_count = tile_elems;
                 if (last[i] >= 0) {
@@ -179,11 +181,13 @@ int64_t pick_tile_elems(int64_t level_elems, const hccl_opts_t& o, int widest, i
 // running sums in registers, no partial read back). Measured against the register engine's static chains: AllReduce
 // bf16 R=8 0.66 at 8 MiB per rank, a tie at 4 MiB, 1.10 at 1 MiB; FP32 R=4 0.74 at 8 MiB, 1.07 at 4 MiB; bf16 R=64 0.85 at
 // 512 KiB, 1.44 at 128 KiB; ReduceScatter bf16 R=16 0.74 at 8 MiB, 0.95 at 2 MiB.
-// (Chunks that do not start on a multiple of 8 elements would make every operand miss the 16-byte alignment the bulk
-// copies need, and the kernel would run such chains item by item through its few compute warps: those stay where they were.)
-bool ring_wants_forwarding(int R, int64_t count, bool fused, const hccl_opts_t& o, const int64_t* recvcounts = nullptr) {
+// (A ReduceScatter whose shards do not start on multiples of 8 elements stays where it was: a shard's place in the send
+// buffers and its place in the receive buffer then differ in their position inside a 16-byte word, and the kernel would
+// run such chains item by item through its few compute warps. An AllReduce has no such problem: the kernel starts
+// every piece with the few elements before the first 16-byte boundary, the same number for all operands.)
+bool ring_wants_forwarding(int R, int64_t count, bool fused, const hccl_opts_t& o, bool scatter = false, const int64_t* recvcounts = nullptr) {
     int64_t off = 0;
-    for (int c = 0; c < R; ++c) {
+    for (int c = 0; c < R && scatter; ++c) {
         if (off % 8) return false;
         off = recvcounts ? off + recvcounts[c] : (int64_t)(((__int128)(c + 1) * count) / R);
     }
@@ -763,7 +767,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     // level-major order runs every chain's step t before any step t+1, so no slot can be recycled
     const size_t slots_wanted = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? chains.size() : 2 * (size_t)o.chain_group;
     const int n_slots = need_scratch ? (int)std::min<size_t>(chains.size(), slots_wanted) : 0;
-    const int64_t slot_elems = (int64_t)align_up((uint64_t)maxlen, 64);
+    const int64_t slot_elems = (int64_t)align_up((uint64_t)maxlen + 8, 64);  // + 8: room for the phase shift (emit_ring)
     const int64_t scratch = need_scratch ? (int64_t)n_slots * slot_elems * 4 * (staged ? 2 : 1) : 0;
     const int64_t weight = count * 4 * (R - 1) + (int64_t)count * es * (R - 1);
     const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
@@ -796,7 +800,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_RING_FUSED && algo != HCCL_ALGO_ONESHOT) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o, pre;
     if (opts) pre = *opts; else std::memset(&pre, 0, sizeof(pre));
-    if (algo == HCCL_ALGO_RING && pre.engine == HCCL_ENGINE_AUTO && ring_wants_forwarding(R, count, false, pre, recvcounts)) pre.engine = HCCL_ENGINE_BULK;
+    if (algo == HCCL_ALGO_RING && pre.engine == HCCL_ENGINE_AUTO && ring_wants_forwarding(R, count, false, pre, true, recvcounts)) pre.engine = HCCL_ENGINE_BULK;
     fill_ring_opts(&o, &pre, (int64_t)R * count * elem_bytes(dt), algo != HCCL_ALGO_RING || R == 1);
     const int es = elem_bytes(dt);
     std::vector<int64_t> offs(R + 1, 0);

@@ -11,7 +11,7 @@
 //
 // Warp 0: lane 0 is the DMA thread; all 32 lanes fetch and check the records of a chain's steps together. Warps 1-7
 // are the compute warps. A chain whose steps are not all of the form above (another operation, an operand that is
-// not 16-byte aligned, B not in a send buffer, an A that is neither a send buffer nor the step before) runs item by
+// whose element phase modulo 8 differs from the others, B not in a send buffer, an A that is neither a send buffer nor the step before) runs item by
 // item through the register path, as the register engine's static chains do.
 #include "bulk.cuh"
 #include "kernels.cuh"
@@ -30,12 +30,13 @@ constexpr uint32_t MAX_STEPS = 512;          // items per chain that fit the ste
 enum : uint32_t { K_A = 0, K_B = 1, K_ITEM = 2, K_EXIT = 3, K_C = 4 };
 struct alignas(16) Piece {
     char* dst;                  // K_B: where this piece's sums go; K_C: where the held values are copied to
-    const char* tail_src;       // K_A, K_B: the operand's last (n mod 8) elements, read with plain loads
+    const char* src0;           // K_A, K_B: where the operand's piece starts; its first `head` and last ((n - head) mod 8)
+                                //           elements are read with plain loads, the rest arrives through the stage
     const char* discard;        // K_B: FP32 partial that a non-forwarding engine would read here for the last time (or null)
     uint32_t n;                 // elements in the piece
     uint32_t item;              // work item: K_ITEM runs it whole; trace and failure reports
     uint8_t kind, dt_src, dt_dst, keep;
-    uint8_t last, pad[3];       // last piece of its item (trace)
+    uint8_t last, head, pad[2]; // last piece of its item (trace); elements before the first 16-byte boundary (0..7)
 };
 struct alignas(8) Step {        // one item of the current chain, tile offset applied
     char* dst;
@@ -45,6 +46,10 @@ struct alignas(8) Step {        // one item of the current chain, tile offset ap
     uint32_t item;
     uint8_t dt_a, dt_b, dt_dst, flags;
 };
+// Element phase of an address: all operands of a chain must share it, so that one scalar head of (8 - phase) mod 8
+// elements brings all of them to a 16-byte boundary together.
+__device__ __forceinline__ uint32_t phase_of(const void* p, uint32_t es) { return (uint32_t)(((uintptr_t)p / es) & 7u); }
+__device__ __forceinline__ bool whole_elements(const void* p, uint32_t es) { return ((uintptr_t)p % es) == 0; }
 enum : uint8_t { S_OK = 1, S_COPY = 2, S_KEEP = 4, S_DISCARD_A = 8 };
 
 template <int DS>
@@ -146,7 +151,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
         const uint32_t ctid = tid - 32, lane = tid & 31u;
         const unsigned long long pol_keep = policy_evict_last();
         float S[G][4];
-        float s_tail = 0.f;
+        float s_tail = 0.f, s_head = 0.f;
 #pragma unroll
         for (int k = 0; k < G; ++k)
 #pragma unroll
@@ -162,26 +167,32 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                 break;
             }
             const char* stage = (const char*)smem + (size_t)slot * stage_bytes;
-            const uint32_t nv = pi.n & ~7u, rem = pi.n - nv;
+            const uint32_t head = pi.head, nv = (pi.n - head) & ~7u, rem = pi.n - head - nv;
+            char* const body = pi.dst + (size_t)head * esize(pi.dt_dst);  // K_B, K_C: where the 16-byte part of the piece goes
             if (pi.kind == K_A) {
                 if (pi.dt_src == HCCL_FP32) take<HCCL_FP32>(stage, nv, ctid, S);
                 else if (pi.dt_src == HCCL_BF16) take<HCCL_BF16>(stage, nv, ctid, S);
                 else take<HCCL_FP16>(stage, nv, ctid, S);
-                if (ctid < rem) s_tail = load_elem(pi.dt_src, pi.tail_src, ctid);
+                if (ctid < head) s_head = load_elem(pi.dt_src, pi.src0, ctid);
+                if (ctid < rem) s_tail = load_elem(pi.dt_src, pi.src0, head + nv + ctid);
             } else if (pi.kind == K_B) {
                 if (pi.dt_src == HCCL_FP32) accumulate<HCCL_FP32>(stage, nv, ctid, S);
                 else if (pi.dt_src == HCCL_BF16) accumulate<HCCL_BF16>(stage, nv, ctid, S);
                 else accumulate<HCCL_FP16>(stage, nv, ctid, S);
                 if (pi.dt_dst == HCCL_FP32) {
-                    if (pi.keep) store_all<HCCL_FP32, true>(pi.dst, nv, ctid, S, pol_keep); else store_all<HCCL_FP32, false>(pi.dst, nv, ctid, S, pol_keep);
+                    if (pi.keep) store_all<HCCL_FP32, true>(body, nv, ctid, S, pol_keep); else store_all<HCCL_FP32, false>(body, nv, ctid, S, pol_keep);
                 } else if (pi.dt_dst == HCCL_BF16) {
-                    store_all<HCCL_BF16, false>(pi.dst, nv, ctid, S, pol_keep);
+                    store_all<HCCL_BF16, false>(body, nv, ctid, S, pol_keep);
                 } else {
-                    store_all<HCCL_FP16, false>(pi.dst, nv, ctid, S, pol_keep);
+                    store_all<HCCL_FP16, false>(body, nv, ctid, S, pol_keep);
+                }
+                if (ctid < head) {
+                    s_head = s_head + load_elem(pi.dt_src, pi.src0, ctid);
+                    store_elem(pi.dt_dst, pi.dst, ctid, s_head);
                 }
                 if (ctid < rem) {
-                    s_tail = s_tail + load_elem(pi.dt_src, pi.tail_src, ctid);
-                    store_elem(pi.dt_dst, pi.dst, nv + ctid, s_tail);
+                    s_tail = s_tail + load_elem(pi.dt_src, pi.src0, head + nv + ctid);
+                    store_elem(pi.dt_dst, pi.dst, head + nv + ctid, s_tail);
                 }
                 if (pi.discard) {
                     // whole 128-byte lines inside the partial that a re-reading engine would have read here for the last time
@@ -190,10 +201,11 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                 }
                 if (pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
             } else if (pi.kind == K_C) {
-                if (pi.dt_dst == HCCL_FP32) store_all<HCCL_FP32, false>(pi.dst, nv, ctid, S, pol_keep);
-                else if (pi.dt_dst == HCCL_BF16) store_all<HCCL_BF16, false>(pi.dst, nv, ctid, S, pol_keep);
-                else store_all<HCCL_FP16, false>(pi.dst, nv, ctid, S, pol_keep);
-                if (ctid < rem) store_elem(pi.dt_dst, pi.dst, nv + ctid, s_tail);
+                if (pi.dt_dst == HCCL_FP32) store_all<HCCL_FP32, false>(body, nv, ctid, S, pol_keep);
+                else if (pi.dt_dst == HCCL_BF16) store_all<HCCL_BF16, false>(body, nv, ctid, S, pol_keep);
+                else store_all<HCCL_FP16, false>(body, nv, ctid, S, pol_keep);
+                if (ctid < head) store_elem(pi.dt_dst, pi.dst, ctid, s_head);
+                if (ctid < rem) store_elem(pi.dt_dst, pi.dst, head + nv + ctid, s_tail);
                 if (pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
             } else {  // K_ITEM: the whole item through the register path; items of a chain follow each other in this block
                 // the item before must be stored by all compute threads. A bounded wait on an mbarrier, not a named barrier:
@@ -205,7 +217,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                 const Tile t = p.tiles[pi.item];
                 run_tile_lsu<false>(p, p.descs[t.desc], t, ctid, CTH);
                 // nothing is forwarded out of an item that ran this way (and the sums need not survive the call)
-                s_tail = 0.f;
+                s_tail = s_head = 0.f;
 #pragma unroll
                 for (int k = 0; k < G; ++k)
 #pragma unroll
@@ -281,7 +293,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                             st.dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + tl.start;
                             st.a = buf_base(p, d.kind_a, d.rank_a) + d.off_a + tl.start;
                             st.n = tl.count;  // bytes for now; elements once the type of the held values is known (below)
-                            f = f && (((uintptr_t)st.dst | (uintptr_t)st.a) & 15u) == 0;
+                            // (its element size is known only from the step before: the phase is checked below)
                         } else {
                             f = d.op == HCCL_OP_REDUCE && d.kind_b == HCCL_BUF_SEND;
                         }
@@ -289,7 +301,9 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                             st.dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + tl.start * esize(d.dt_dst);
                             st.a = buf_base(p, d.kind_a, d.rank_a) + d.off_a + tl.start * esize(d.dt_a);
                             st.b = buf_base(p, d.kind_b, d.rank_b) + d.off_b + tl.start * esize(d.dt_b);
-                            f = (((uintptr_t)st.dst | (uintptr_t)st.a | (uintptr_t)st.b) & 15u) == 0;
+                            const uint32_t ph = phase_of(st.b, esize(d.dt_b));
+                            f = whole_elements(st.b, esize(d.dt_b)) && whole_elements(st.dst, esize(d.dt_dst)) && phase_of(st.dst, esize(d.dt_dst)) == ph &&
+                                (t > 0 || (whole_elements(st.a, esize(d.dt_a)) && phase_of(st.a, esize(d.dt_a)) == ph));
                             if (t == 0 && (d.kind_a != HCCL_BUF_SEND || PIECE * esize(d.dt_a) > stage_bytes)) f = false;
                             if (PIECE * esize(d.dt_b) > stage_bytes) f = false;  // the launch sized the stages for 16-bit operands
                             if (d.kind_dst == HCCL_BUF_SCRATCH && d.dt_dst == HCCL_FP32) st.flags |= S_KEEP;
@@ -315,6 +329,9 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                         st.dt_dst = pv.dt_dst;
                         if (st.n != pv.n * esize(pv.dt_dst)) fast = false;
                         st.n = pv.n;
+                        if (!whole_elements(st.dst, esize(st.dt_dst)) || phase_of(st.dst, esize(st.dt_dst)) != phase_of(pv.dst, esize(pv.dt_dst))) fast = false;
+                    } else if (phase_of(st.b, esize(st.dt_b)) != phase_of(pv.dst, esize(pv.dt_dst))) {
+                        fast = false;
                     } else if ((pv.flags & S_COPY) || st.dt_a != HCCL_FP32 || pv.dt_dst != HCCL_FP32 || st.n != pv.n) fast = false;
                 }
                 if (s_step[0].flags & S_COPY) fast = false;
@@ -339,8 +356,9 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                 }
             } else {
                 const uint32_t n = s_step[0].n;
+                const uint32_t h0 = (8u - phase_of(s_step[0].b, esize(s_step[0].dt_b))) & 7u;  // the same for every operand and piece of the chain
                 for (uint32_t e0 = 0; e0 < n && ok; e0 += PIECE) {
-                    const uint32_t ne = min(PIECE, n - e0), nv = ne & ~7u;
+                    const uint32_t ne = min(PIECE, n - e0), head = min(h0, ne), nv = (ne - head) & ~7u;
                     for (uint32_t t = 0; t < L && ok; ++t) {
                         const Step& st = s_step[t];
                         if (p.trace && e0 == 0) {
@@ -356,10 +374,11 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                             pa.n = ne;
                             pa.item = st.item;
                             pa.dt_src = st.dt_a;
-                            pa.tail_src = st.a + (size_t)(e0 + nv) * ea;
+                            pa.src0 = st.a + (size_t)e0 * ea;
+                            pa.head = (uint8_t)head;
                             if (nv) {
                                 mbar_arrive_expect_tx(full + 8 * slot, nv * ea);
-                                bulk_load(stages + slot * stage_bytes, st.a + (size_t)e0 * ea, nv * ea, full + 8 * slot, true, pol);
+                                bulk_load(stages + slot * stage_bytes, st.a + (size_t)(e0 + head) * ea, nv * ea, full + 8 * slot, true, pol);
                             } else {
                                 mbar_arrive(full + 8 * slot);
                             }
@@ -373,6 +392,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                             pc.item = st.item;
                             pc.dt_dst = st.dt_dst;
                             pc.last = (e0 + ne == n) ? 1 : 0;
+                            pc.head = (uint8_t)head;
                             pc.dst = st.dst + (size_t)e0 * esize(st.dt_dst);
                             mbar_arrive(full + 8 * slot);
                             advance();
@@ -389,11 +409,12 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                         pb.keep = (st.flags & S_KEEP) ? 1 : 0;
                         pb.last = (e0 + ne == n) ? 1 : 0;
                         pb.dst = st.dst + (size_t)e0 * ed;
-                        pb.tail_src = st.b + (size_t)(e0 + nv) * eb;
+                        pb.src0 = st.b + (size_t)e0 * eb;
+                        pb.head = (uint8_t)head;
                         pb.discard = (t > 0 && (st.flags & S_DISCARD_A)) ? st.a + (size_t)e0 * 4 : nullptr;
                         if (nv) {
                             mbar_arrive_expect_tx(full + 8 * slot, nv * eb);
-                            bulk_load(stages + slot * stage_bytes, st.b + (size_t)e0 * eb, nv * eb, full + 8 * slot, true, pol);
+                            bulk_load(stages + slot * stage_bytes, st.b + (size_t)(e0 + head) * eb, nv * eb, full + 8 * slot, true, pol);
                         } else {
                             mbar_arrive(full + 8 * slot);
                         }

@@ -48,6 +48,21 @@ def test_reducescatter_and_allreduce_rings_in_the_forwarding_kernel(budget, dt):
             assert_reduction_close(dt, got, exact, want[r], "rank %d" % r)
 
 
+def test_chunks_off_the_16_byte_boundary_are_forwarded_too():
+    """R = 3 and 6 with a power-of-two count: no chunk starts on a multiple of 8 elements. Every piece then begins with
+    the few elements before the first 16-byte boundary (the partials' scratch slots are shifted to the same phase), and
+    the library picks the kernel by itself."""
+    for R, n in ((3, 1 << 20), (6, (1 << 20) + 3)):
+        for dt in (hb.BF16, hb.FP32):
+            X = synth.normal_ranks(R, n, dt, seed=R + n)
+            p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING)
+            assert p.info().engine == hb.ENGINE_BULK and p.info().static_chains > 0 and p.check_hazards() == 0
+            Y = run_plan(p, X, iters=2)
+            ring = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+            for r in range(R):
+                assert np.array_equal(Y[r].view(np.uint8), ring[r].view(np.uint8)), (R, n, dt, r)
+
+
 def test_default_options_choose_the_forwarding_kernel_for_large_rings():
     """With about a chain of tiles per SM or more the planners pick it themselves; small rings stay on the register engine."""
     big = hb.hccl_plan_allreduce(8, 1 << 22, hb.BF16, hb.ALGO_RING).info()
