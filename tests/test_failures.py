@@ -62,12 +62,13 @@ def test_wait_that_never_comes_true_times_out(engine):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("engine", [hb.ENGINE_LSU, hb.ENGINE_BULK], ids=["lsu", "bulk"])
+@pytest.mark.parametrize("engine,flags", [(hb.ENGINE_LSU, 0), (hb.ENGINE_BULK, hb.FLAG_DYNAMIC_TICKETS), (hb.ENGINE_BULK, 0)], ids=["lsu", "bulk", "forwarding"])
 @pytest.mark.parametrize("damage", ["desc_index", "wait_range", "op_code", "rank"])
-def test_damaged_table_entry_is_reported_not_dereferenced(engine, damage):
+def test_damaged_table_entry_is_reported_not_dereferenced(engine, flags, damage):
     import torch
     from paper_2608_00358_b200.runtime import DeviceCollective
-    plan = hb.hccl_plan_allreduce(4, 4096, hb.FP32, hb.ALGO_RING, dict(engine=engine, sm_budget=4, tile_bytes=4096, timeout_ns=150_000_000))
+    plan = hb.hccl_plan_allreduce(4, 4096, hb.FP32, hb.ALGO_RING, dict(engine=engine, flags=flags, sm_budget=4, tile_bytes=4096, timeout_ns=150_000_000))
+    assert (plan.info().static_chains > 0) == (flags == 0)     # static chains on the bulk engine: the forwarding kernel
     send = [torch.randn(4096, device="cuda") for _ in range(4)]
     recv = [torch.zeros(4096, device="cuda") for _ in range(4)]
     dc = DeviceCollective(plan)
