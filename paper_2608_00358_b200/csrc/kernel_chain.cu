@@ -48,8 +48,9 @@ struct alignas(8) Step {        // one item of the current chain, tile offset ap
 };
 // Element phase of an address: all operands of a chain must share it, so that one scalar head of (8 - phase) mod 8
 // elements brings all of them to a 16-byte boundary together.
-__device__ __forceinline__ uint32_t phase_of(const void* p, uint32_t es) { return (uint32_t)(((uintptr_t)p / es) & 7u); }
-__device__ __forceinline__ bool whole_elements(const void* p, uint32_t es) { return ((uintptr_t)p % es) == 0; }
+// (es is 2 or 4: shifts and masks, no 64-bit division on the one thread that checks every step of every chain)
+__device__ __forceinline__ uint32_t phase_of(const void* p, uint32_t es) { return (uint32_t)(((uintptr_t)p >> (es == 4 ? 2 : 1)) & 7u); }
+__device__ __forceinline__ bool whole_elements(const void* p, uint32_t es) { return ((uintptr_t)p & (uintptr_t)(es - 1)) == 0; }
 enum : uint8_t { S_OK = 1, S_COPY = 2, S_KEEP = 4, S_DISCARD_A = 8 };
 
 template <int DS>
@@ -151,7 +152,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
         const uint32_t ctid = tid - 32, lane = tid & 31u;
         const unsigned long long pol_keep = policy_evict_last();
         float S[G][4];
-        float s_tail = 0.f, s_head = 0.f;
+        float s_tail = 0.f;  // this thread's scalar element of the piece, if it has one
 #pragma unroll
         for (int k = 0; k < G; ++k)
 #pragma unroll
@@ -167,14 +168,15 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                 break;
             }
             const char* stage = (const char*)smem + (size_t)slot * stage_bytes;
-            const uint32_t head = pi.head, nv = (pi.n - head) & ~7u, rem = pi.n - head - nv;
-            char* const body = pi.dst + (size_t)head * esize(pi.dt_dst);  // K_B, K_C: where the 16-byte part of the piece goes
+            // the piece: `head` scalar elements up to the first 16-byte boundary, nv elements in 16-byte groups, the rest scalar again;
+            // thread ctid < edge keeps scalar element number ei
+            const uint32_t head = pi.head, nv = (pi.n - head) & ~7u, edge = pi.n - nv, ei = ctid < head ? ctid : nv + ctid;
+            char* const body = pi.dst + (size_t)head * esize(pi.dt_dst);  // K_B, K_C: where the 16-byte groups go
             if (pi.kind == K_A) {
                 if (pi.dt_src == HCCL_FP32) take<HCCL_FP32>(stage, nv, ctid, S);
                 else if (pi.dt_src == HCCL_BF16) take<HCCL_BF16>(stage, nv, ctid, S);
                 else take<HCCL_FP16>(stage, nv, ctid, S);
-                if (ctid < head) s_head = load_elem(pi.dt_src, pi.src0, ctid);
-                if (ctid < rem) s_tail = load_elem(pi.dt_src, pi.src0, head + nv + ctid);
+                if (ctid < edge) s_tail = load_elem(pi.dt_src, pi.src0, ei);
             } else if (pi.kind == K_B) {
                 if (pi.dt_src == HCCL_FP32) accumulate<HCCL_FP32>(stage, nv, ctid, S);
                 else if (pi.dt_src == HCCL_BF16) accumulate<HCCL_BF16>(stage, nv, ctid, S);
@@ -186,13 +188,9 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                 } else {
                     store_all<HCCL_FP16, false>(body, nv, ctid, S, pol_keep);
                 }
-                if (ctid < head) {
-                    s_head = s_head + load_elem(pi.dt_src, pi.src0, ctid);
-                    store_elem(pi.dt_dst, pi.dst, ctid, s_head);
-                }
-                if (ctid < rem) {
-                    s_tail = s_tail + load_elem(pi.dt_src, pi.src0, head + nv + ctid);
-                    store_elem(pi.dt_dst, pi.dst, head + nv + ctid, s_tail);
+                if (ctid < edge) {
+                    s_tail = s_tail + load_elem(pi.dt_src, pi.src0, ei);
+                    store_elem(pi.dt_dst, pi.dst, ei, s_tail);
                 }
                 if (pi.discard) {
                     // whole 128-byte lines inside the partial that a re-reading engine would have read here for the last time
@@ -204,8 +202,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                 if (pi.dt_dst == HCCL_FP32) store_all<HCCL_FP32, false>(body, nv, ctid, S, pol_keep);
                 else if (pi.dt_dst == HCCL_BF16) store_all<HCCL_BF16, false>(body, nv, ctid, S, pol_keep);
                 else store_all<HCCL_FP16, false>(body, nv, ctid, S, pol_keep);
-                if (ctid < head) store_elem(pi.dt_dst, pi.dst, ctid, s_head);
-                if (ctid < rem) store_elem(pi.dt_dst, pi.dst, head + nv + ctid, s_tail);
+                if (ctid < edge) store_elem(pi.dt_dst, pi.dst, ei, s_tail);
                 if (pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
             } else {  // K_ITEM: the whole item through the register path; items of a chain follow each other in this block
                 // the item before must be stored by all compute threads. A bounded wait on an mbarrier, not a named barrier:
@@ -217,7 +214,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                 const Tile t = p.tiles[pi.item];
                 run_tile_lsu<false>(p, p.descs[t.desc], t, ctid, CTH);
                 // nothing is forwarded out of an item that ran this way (and the sums need not survive the call)
-                s_tail = s_head = 0.f;
+                s_tail = 0.f;
 #pragma unroll
                 for (int k = 0; k < G; ++k)
 #pragma unroll
@@ -317,25 +314,42 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
             fast = fast && __all_sync(0xffffffffu, f);
         }
         __syncwarp();
-        if (lane == 0) {
-            if (good && fast) {
-                // every step after the first must take exactly what the step before stored: a sum takes an FP32 sum, a copy
-                // takes whatever the block holds (and learns its element type from the step before)
-                for (uint32_t t = 1; t < L && fast; ++t) {
-                    Step& st = s_step[t];
-                    const Step& pv = s_step[t - 1];
-                    if (st.a != pv.dst) fast = false;
-                    else if (st.flags & S_COPY) {
-                        st.dt_dst = pv.dt_dst;
-                        if (st.n != pv.n * esize(pv.dt_dst)) fast = false;
-                        st.n = pv.n;
-                        if (!whole_elements(st.dst, esize(st.dt_dst)) || phase_of(st.dst, esize(st.dt_dst)) != phase_of(pv.dst, esize(pv.dt_dst))) fast = false;
-                    } else if (phase_of(st.b, esize(st.dt_b)) != phase_of(pv.dst, esize(pv.dt_dst))) {
-                        fast = false;
-                    } else if ((pv.flags & S_COPY) || st.dt_a != HCCL_FP32 || pv.dt_dst != HCCL_FP32 || st.n != pv.n) fast = false;
-                }
-                if (s_step[0].flags & S_COPY) fast = false;
+        if (good && fast) {
+            // Every step after the first must take exactly what the step before stored: sums first (each takes an FP32 sum),
+            // then copies of what the block holds, whose element type is that of the last sum's result. Checked by all lanes,
+            // a step each (the one thread that issues the pieces has no time for a walk over every step of every chain).
+            uint32_t first_copy = L;
+            for (uint32_t t0 = 0; t0 < L; t0 += 32) {
+                const uint32_t t = t0 + lane;
+                const uint32_t copies = __ballot_sync(0xffffffffu, t < L && (s_step[t].flags & S_COPY));
+                if (copies && first_copy == L) first_copy = t0 + (uint32_t)__ffs((int)copies) - 1u;
             }
+            if (first_copy == 0) fast = false;
+            const uint32_t held_dt = first_copy >= 1 && first_copy < L ? s_step[first_copy - 1].dt_dst : 0;  // type of what the copies move
+            const uint32_t held_n = first_copy >= 1 && first_copy < L ? s_step[first_copy - 1].n : 0;
+            __syncwarp();
+            for (uint32_t t0 = 0; t0 < L && fast; t0 += 32) {
+                const uint32_t t = t0 + lane;
+                bool f = true;
+                if (t >= 1 && t < L) {
+                    Step& st = s_step[t];
+                    const Step& pv = s_step[t - 1];  // only fields that no lane rewrites are read from it (dst; for a sum also dt_dst, n)
+                    f = st.a == pv.dst;
+                    if (t < first_copy) {
+                        f = f && !(st.flags & S_COPY) && st.dt_a == HCCL_FP32 && pv.dt_dst == HCCL_FP32 && st.n == pv.n &&
+                            phase_of(st.b, esize(st.dt_b)) == phase_of(pv.dst, 4);
+                    } else {
+                        f = f && (st.flags & S_COPY) && st.n == held_n * esize(held_dt) && whole_elements(st.dst, esize(held_dt)) &&
+                            phase_of(st.dst, esize(held_dt)) == phase_of(pv.dst, esize(held_dt));
+                        st.dt_dst = (uint8_t)held_dt;
+                        st.n = held_n;
+                    }
+                }
+                fast = __all_sync(0xffffffffu, f);
+            }
+            __syncwarp();
+        }
+        if (lane == 0) {
             if (!good) {
                 fail(p, HCCL_ERR_BAD_DESCRIPTOR, base);
                 ok = false;
