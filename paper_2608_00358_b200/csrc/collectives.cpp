@@ -866,7 +866,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     for (const Chain& ch : chains) maxlen = std::max(maxlen, ch.len);
     // Large rings on the bulk engine: every chain gets a scratch slot of its own (up to 1 GiB in all), so the chains are
     // independent and run in the forwarding kernel, which keeps a chain's running sums in registers and only stores
-    // the partials (config 3: 0.71 vs 0.86 ms through tickets with recycled slots whose partials are read back).
+    // the partials (config 3: 0.69 vs 0.86 ms through tickets with recycled slots whose partials are read back).
     const bool forward = !fused && R > 2 && o.engine == HCCL_ENGINE_BULK && (!opts || opts->chain_group == 0) && count * 4 <= (1ll << 30) &&
                          !(o.flags & (HCCL_FLAG_DYNAMIC_TICKETS | HCCL_FLAG_LEVEL_MAJOR | HCCL_FLAG_STAGED_RING | HCCL_FLAG_BIDIRECTIONAL));
     if ((!opts || opts->chain_group == 0) && (count * 4 <= (32ll << 20) || forward)) o.chain_group = (int32_t)std::max<size_t>(chains.size(), 1);
