@@ -195,23 +195,33 @@ bool ring_wants_forwarding(int R, int64_t count, bool fused, const hccl_opts_t& 
     return !fused && R > 2 && count * 4 <= (1ll << 30) && (count >= (1ll << 20) || (R >= 32 && count >= (1ll << 18)));
 }
 
-// Tile size for the forwarding kernel. A chain of tiles costs about the same however short its tiles are (a fixed cost
-// per step), and a block runs its chains one after the other: if one round of the blocks can take all chains, the
-// smallest tile that leaves no more chains than blocks; else whole pieces.
-int64_t forward_tile_elems(const std::vector<Chain>& chains, int blocks) {
-    int64_t total = 0;
-    for (const Chain& c : chains) total += c.len;
-    // plenty of pieces per block: two pieces per tile halve what a block pays between two chains (the records of the next
-    // chain's steps are fetched while little work is queued for the compute warps: AllReduce bf16 R=16 x 128 MiB 1.10 vs
-    // 1.20 ms); four and more leave too few chains to share out evenly
-    if (blocks > 0 && total >= 8 * (int64_t)blocks * kForwardPieceElems) return 2 * kForwardPieceElems;
-    if (total > (int64_t)blocks * kForwardPieceElems || blocks <= 0) return kForwardPieceElems;
-    for (int64_t tile = std::max<int64_t>(256, (total / blocks + 7) / 8 * 8); tile < kForwardPieceElems; tile += 8) {
+// Tile size for the forwarding kernel: the one with the shortest estimated makespan. A block runs its chains of tiles one
+// after the other; a chain of `steps` steps over a tile of t elements costs steps x (pieces(t) x 0.45 us + t x 0.05 ns)
+// plus about 4 us between two chains (fixed cost per piece and step, store time per element, and the fetch of the next
+// chain's records; fitted to measurements: config 3, AllReduce bf16 R=64 x 8 MiB, R=8 x 16 MiB, R=16 x 4 MiB), and the
+// blocks need ceil(chains / blocks) rounds. Candidates: every chain of the longest granule cut into k equal tiles.
+int64_t forward_tile_elems(const std::vector<Chain>& chains, int blocks, int steps) {
+    int64_t maxlen = 0;
+    for (const Chain& c : chains) maxlen = std::max(maxlen, c.len);
+    if (blocks <= 0 || maxlen <= 0) return kForwardPieceElems;
+    double best = 0;
+    int64_t best_tile = kForwardPieceElems;
+    const int64_t kmax = std::min<int64_t>(4096, std::max<int64_t>(1, maxlen / 256));
+    for (int64_t k = 1; k <= kmax; ++k) {
+        const int64_t tile = ((maxlen + k - 1) / k + 7) / 8 * 8;
         int64_t n = 0;
         for (const Chain& c : chains) n += (c.len + tile - 1) / tile;
-        if (n <= blocks) return tile;
+        const double pieces = (double)((tile + kForwardPieceElems - 1) / kForwardPieceElems);
+        const double rounds = (double)((n + blocks - 1) / blocks);
+        // (tiles of more than two pieces measured about 5 % slower per further piece than this sum: config 3 with 4 / 8 pieces
+        // per tile 0.72-0.75 / 0.83 ms against 0.69 with two)
+        const double cost = rounds * (steps * (pieces * 0.45 + (double)tile * 0.00005) + 4.0) * (1.0 + 0.05 * std::max(0.0, pieces - 2.0));
+        if (best == 0 || cost < best * 0.999) {  // ties go to the larger tile (k grows)
+            best = cost;
+            best_tile = tile;
+        }
     }
-    return kForwardPieceElems;
+    return best_tile;
 }
 
 // Ring reductions: with the engine left to the library, large ones feed the adds from shared memory through
@@ -781,7 +791,7 @@ hccl_status_t hccl_plan_allreduce(int R, int64_t count, hccl_dtype_t dt, hccl_al
     int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, in_recv ? es : 4, HCCL_OP_REDUCE, maxlen);
     // large FP32 rings as static chains: two passes of the block's threads per tile keep a block's current
     // partial (written by one step, read by the next) in the L2
-    if (forward && !o.tile_bytes) tile_elems = forward_tile_elems(chains, o.sm_budget);
+    if (forward && !o.tile_bytes) tile_elems = forward_tile_elems(chains, o.sm_budget, 2 * (R - 1));
     if (in_recv && o.engine == HCCL_ENGINE_LSU && !o.tile_bytes && count * 4 > (32ll << 20) && (o.flags & HCCL_FLAG_STATIC_CHAINS))
         tile_elems = 2 * sweep_of(o, HCCL_OP_REDUCE);
     if (!fused && o.engine == HCCL_ENGINE_LSU && (!opts || opts->sm_budget == 0) && maxlen > 0) {
@@ -882,7 +892,7 @@ hccl_status_t hccl_plan_reducescatter(int R, const int64_t* recvcounts, int64_t 
     const int64_t scratch = need_scratch ? (int64_t)n_slots * slot_elems * 4 * (staged ? 2 : 1) : 0;
     const int64_t level = (o.flags & HCCL_FLAG_LEVEL_MAJOR) ? count : std::min<int64_t>(count, (int64_t)o.chain_group * maxlen);
     int64_t tile_elems = fused ? pick_tile_elems(level, o, es * R, HCCL_OP_REDUCE_N) : pick_tile_elems(level, o, 4, HCCL_OP_REDUCE, maxlen);
-    if (forward && !o.tile_bytes) tile_elems = forward_tile_elems(chains, o.sm_budget);
+    if (forward && !o.tile_bytes) tile_elems = forward_tile_elems(chains, o.sm_budget, R - 1);
     CHECK(hccl_graph_create(R, sext.data(), rext.data(), scratch, 0, &graw));
     GraphPtr g(graw);
     g->compulsory_bytes = compulsory;
