@@ -9,10 +9,14 @@
 // step's B to it: 4 bytes stored and 2 loaded per element and step. The B operands (send buffers, which no step
 // writes) are fetched ahead by cp.async.bulk into a ring of stages; stores are plain 16-byte stores from registers.
 //
+// A ring AllReduce's AllGather hops (copies of what the step before stored) are stored from the same registers.
+//
 // Warp 0: lane 0 is the DMA thread; all 32 lanes fetch and check the records of a chain's steps together. Warps 1-7
-// are the compute warps. A chain whose steps are not all of the form above (another operation, an operand that is
-// whose element phase modulo 8 differs from the others, B not in a send buffer, an A that is neither a send buffer nor the step before) runs item by
-// item through the register path, as the register engine's static chains do.
+// are the compute warps. A piece may start off a 16-byte boundary if all operands of the chain do so by the same
+// number of elements: its first few and last few elements are read and stored with plain accesses by one thread each.
+// A chain whose steps are not all of the form above (another operation first, an operand at another position inside
+// a 16-byte word than the others, B not in a send buffer, an A that is neither a send buffer nor the step before)
+// runs item by item through the register path, as the register engine's static chains do.
 #include "bulk.cuh"
 #include "kernels.cuh"
 
@@ -21,7 +25,7 @@ namespace chainfw {
 using namespace bulk;
 
 constexpr uint32_t CW = 7, CTH = CW * 32;    // compute warps, compute threads: 8 warps in all, so that a thread may have 255 registers
-                                             // (nine warps are given registers like twelve: 168, and the 32 running sums spill)
+                                             // (nine warps are given registers like twelve: 168, and the running sums spill)
 constexpr int G = 16;                         // groups of 4 elements per compute thread and piece
 constexpr uint32_t PIECE = CTH * 4 * G;      // elements per piece: 64 per compute thread (one DMA issue per piece: the fewer the better)
 constexpr uint32_t MAX_NS = 6;               // stages: 6 of PIECE * 2 bytes (16-bit operands) or 3 of PIECE * 4 (FP32)
