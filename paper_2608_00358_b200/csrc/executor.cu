@@ -43,7 +43,10 @@ hccl_status_t hccl_plan_bind(hccl_plan_t* p, void* dev_workspace, size_t bytes, 
         if (smem > 48 * 1024) CUDA_TRY(cudaFuncSetAttribute(hccl_a2a_dynamic, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(DYN_MAX_RANKS * DYN_MAX_RANKS * 24 + (DYN_MAX_RANKS * DYN_MAX_RANKS + 1) * 4 + 16)));
     } else if (p->opts.engine == HCCL_ENGINE_BULK) {
         CUDA_TRY(cudaFuncSetAttribute(hccl_executor_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bulk::MAX_DYNAMIC_SMEM));
-        if (p->chain_len) CUDA_TRY(cudaFuncSetAttribute(hccl_executor_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM_BYTES));
+        if (p->chain_len) {
+            CUDA_TRY(cudaFuncSetAttribute(hccl_executor_chain, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM_BYTES));
+            CUDA_TRY(cudaFuncSetAttribute(hccl_executor_chain_sums, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM_BYTES));
+        }
     }
     p->workspace = dev_workspace;
     p->workspace_bytes = bytes;
@@ -234,7 +237,8 @@ hccl_status_t hccl_execute(hccl_plan_t* p, const void* const* sendbufs, void* co
     if (p->opts.engine == HCCL_ENGINE_BULK && p->chain_len) {
         // stages sized for the widest operand that arrives through them (B of every step, A of a chain's first)
         const bool wide = p->chain_wide;
-        hccl_executor_chain<<<blocks, CHAIN_THREADS, CHAIN_SMEM_BYTES, (cudaStream_t)stream>>>(prm, wide ? 3u : 6u, CHAIN_PIECE_ELEMS * (wide ? 4u : 2u));
+        if (p->chain_copies) hccl_executor_chain<<<blocks, CHAIN_THREADS, CHAIN_SMEM_BYTES, (cudaStream_t)stream>>>(prm, wide ? 3u : 6u, CHAIN_PIECE_ELEMS * (wide ? 4u : 2u));
+        else hccl_executor_chain_sums<<<blocks, CHAIN_THREADS, CHAIN_SMEM_BYTES, (cudaStream_t)stream>>>(prm, wide ? 3u : 6u, CHAIN_PIECE_ELEMS * (wide ? 4u : 2u));
     } else if (p->opts.engine == HCCL_ENGINE_BULK) {
         const bulk::StageConfig sc = bulk::stage_config(p->opts.stages, p->opts.stage_kib);
         const int threads = std::max(128, p->opts.threads);

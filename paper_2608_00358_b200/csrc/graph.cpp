@@ -582,7 +582,8 @@ void hccl::compute_layout(hccl_plan* p) {
     L.waits = o; o = align_up(o + sizeof(Wait) * std::max<size_t>(p->waits.size(), 1), 256);
     L.scratch = o; o = align_up(o + (uint64_t)p->scratch_bytes, 256);
     L.total = o;
-    p->chain_wide = false;
+    p->chain_wide = p->chain_copies = false;
+    for (const Desc& d : p->descs) p->chain_copies = p->chain_copies || d.op == HCCL_OP_COPY;
     for (const Desc& d : p->descs)
         if (d.op == HCCL_OP_REDUCE && (d.dt_b == HCCL_FP32 || (d.kind_a == HCCL_BUF_SEND && d.dt_a == HCCL_FP32))) p->chain_wide = true;
 }

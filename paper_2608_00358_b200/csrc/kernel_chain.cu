@@ -29,18 +29,22 @@ constexpr uint32_t CW = 7, CTH = CW * 32;    // compute warps, compute threads: 
 constexpr int G = 16;                         // groups of 4 elements per compute thread and piece
 constexpr uint32_t PIECE = CTH * 4 * G;      // elements per piece: 64 per compute thread (one DMA issue per piece: the fewer the better)
 constexpr uint32_t MAX_NS = 6;               // stages: 6 of PIECE * 2 bytes (16-bit operands) or 3 of PIECE * 4 (FP32)
+constexpr uint32_t MAX_CDST = 256;           // destinations of one K_C piece: a chain's copies are stored one after the other by one piece
 constexpr uint32_t MAX_STEPS = 512;          // items per chain that fit the step table (2 R - 2 for R = 256: 510)
 
-enum : uint32_t { K_A = 0, K_B = 1, K_ITEM = 2, K_EXIT = 3, K_C = 4 };
+enum : uint32_t { K_A = 0, K_B = 1, K_ITEM = 2, K_EXIT = 3, K_C = 4, K_CM = 5 };
+constexpr uint32_t CM_MIN16 = 6, CM_MIN32 = 12;  // from this many copies on (16-bit / FP32 values), a chain's copies go out as one K_CM piece
 struct alignas(16) Piece {
-    char* dst;                  // K_B: where this piece's sums go; K_C: where the held values are copied to
+    char* dst;                  // K_B: where this piece's sums go; K_C: where the held values are copied to (K_CM: the stage's
+                                //      destination list says where)
     const char* src0;           // K_A, K_B: where the operand's piece starts; its first `head` and last ((n - head) mod 8)
                                 //           elements are read with plain loads, the rest arrives through the stage
     const char* discard;        // K_B: FP32 partial that a non-forwarding engine would read here for the last time (or null)
     uint32_t n;                 // elements in the piece
     uint32_t item;              // work item: K_ITEM runs it whole; trace and failure reports
     uint8_t kind, dt_src, dt_dst, keep;
-    uint8_t last, head, pad[2]; // last piece of its item (trace); elements before the first 16-byte boundary (0..7)
+    uint8_t last, head;         // last piece of its item (trace); elements before the first 16-byte boundary (0..7)
+    uint16_t ndst;              // K_CM: destinations (consecutive items from `item` on)
 };
 struct alignas(8) Step {        // one item of the current chain, tile offset applied
     char* dst;
@@ -95,6 +99,29 @@ __device__ __forceinline__ void store_all(char* dst, uint32_t nv, uint32_t ctid,
         if (e < nv) stg4<DD, KEEP>(dst + (size_t)e * Elem<DD>::BYTES, S[k], pol);
     }
 }
+// The same values, rounded the same way, into shared memory (for the bulk copies of a chain's AllGather hops).
+template <int DD>
+__device__ __forceinline__ void stage_all(char* out, uint32_t nv, uint32_t ctid, const float (&S)[G][4]) {
+#pragma unroll
+    for (int k = 0; k < G; ++k) {
+        const uint32_t e = (k * CTH + ctid) * 4;
+        if (e < nv) {
+            if constexpr (DD == HCCL_FP32) {
+                *reinterpret_cast<float4*>(out + (size_t)e * 4) = make_float4(S[k][0], S[k][1], S[k][2], S[k][3]);
+            } else {
+                uint2 v;
+                if constexpr (DD == HCCL_BF16) {
+                    const __nv_bfloat162 a = __floats2bfloat162_rn(S[k][0], S[k][1]), b = __floats2bfloat162_rn(S[k][2], S[k][3]);
+                    v.x = *reinterpret_cast<const uint32_t*>(&a); v.y = *reinterpret_cast<const uint32_t*>(&b);
+                } else {
+                    const __half2 a = __floats2half2_rn(S[k][0], S[k][1]), b = __floats2half2_rn(S[k][2], S[k][3]);
+                    v.x = *reinterpret_cast<const uint32_t*>(&a); v.y = *reinterpret_cast<const uint32_t*>(&b);
+                }
+                *reinterpret_cast<uint2*>(out + (size_t)e * 2) = v;
+            }
+        }
+    }
+}
 __device__ __forceinline__ float load_elem(int dt, const char* p, uint32_t i) {
     return dt == HCCL_FP32 ? Elem<HCCL_FP32>::load(p, i) : dt == HCCL_BF16 ? Elem<HCCL_BF16>::load(p, i) : Elem<HCCL_FP16>::load(p, i);
 }
@@ -131,11 +158,16 @@ __device__ __forceinline__ void mbar_wait_quiet(uint32_t bar, uint32_t parity, u
 
 using namespace chainfw;
 
-__global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t stage_bytes) {
+// COPIES: the build that also forwards a chain's copies (ring AllReduce). A packet of sums alone (ring ReduceScatter)
+// runs in the build without that code: the compiler is at its register limit here, and the extra paths cost the sums'
+// loop 6 % (config 3: 0.73 against 0.69 ms).
+template <bool COPIES>
+__device__ __forceinline__ void executor_chain_body(const ExecParams& p, const uint32_t ns, const uint32_t stage_bytes) {
     extern __shared__ __align__(128) unsigned char smem[];
     __shared__ __align__(8) unsigned long long s_bar[2 * MAX_NS + 1];  // full, empty, and the compute warps' own barrier
     __shared__ Piece s_info[MAX_NS];
     __shared__ Step s_step[MAX_STEPS];
+    __shared__ char* s_cdst[MAX_NS][MAX_CDST];  // K_C: where the piece in each stage is copied to
     const uint32_t tid = threadIdx.x;
     const uint32_t stages = smem_u32(smem), full = smem_u32(s_bar), empty = full + 8 * MAX_NS, cbar = empty + 8 * MAX_NS;
     if (tid == 0) {
@@ -166,6 +198,10 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
             if (!wait_inline(p, full + 8 * slot, parity, long_wait, 0xfffffff7u)) break;
             const Piece pi = s_info[slot];
             if (pi.kind == K_EXIT) {
+                if (ctid == 0) {  // the bulk copies of the chains' last pieces must have arrived, not only have left the stages
+                    bulk_wait_all();
+                    fence_proxy_async();
+                }
                 if (!lean) __threadfence();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(empty + 8 * slot);  // tells the DMA thread that everything is stored
@@ -202,12 +238,46 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                     for (uintptr_t a = lo + (uintptr_t)ctid * 128u; a < hi; a += (uintptr_t)CTH * 128u) discard_line((const void*)a);
                 }
                 if (pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
-            } else if (pi.kind == K_C) {
+            } else if (COPIES && pi.kind == K_C) {
+                // a copy of what this block holds, stored from the registers (chains with few copies)
                 if (pi.dt_dst == HCCL_FP32) store_all<HCCL_FP32, false>(body, nv, ctid, S, pol_keep);
                 else if (pi.dt_dst == HCCL_BF16) store_all<HCCL_BF16, false>(body, nv, ctid, S, pol_keep);
                 else store_all<HCCL_FP16, false>(body, nv, ctid, S, pol_keep);
                 if (ctid < edge) store_elem(pi.dt_dst, pi.dst, ei, s_tail);
                 if (pi.last && p.trace && ctid == 0) trace_put(p.trace, p.trace_cap, pi.item, 3, globaltimer_ns());
+            } else if (COPIES && pi.kind == K_CM) {
+                // The chain's copies: the held values, rounded to the copies' type, go into this piece's stage (which no load
+                // uses) once; one thread then stores the stage to every destination with cp.async.bulk. One piece for all
+                // the copies of a long chain: between two pieces the compute warps wait, which costs as much as storing a copy
+                // (with few copies the trip through shared memory and the barrier cost more than that: FP32 R = 4 +13 %, R = 8 +5 %;
+                // bf16 R = 8 -6 %, R = 64 -8 %).
+                const uint32_t nd = pi.ndst, ed = esize(pi.dt_dst);
+                char* const out = (char*)smem + (size_t)slot * stage_bytes;
+                if (pi.dt_dst == HCCL_FP32) stage_all<HCCL_FP32>(out, nv, ctid, S);
+                else if (pi.dt_dst == HCCL_BF16) stage_all<HCCL_BF16>(out, nv, ctid, S);
+                else stage_all<HCCL_FP16>(out, nv, ctid, S);
+                if (ctid < edge)
+                    for (uint32_t j = 0; j < nd; ++j) store_elem(pi.dt_dst, s_cdst[slot][j], ei, s_tail);
+                // the copies end the chain: what follows is another chain's first operand, and the sums need not be kept
+                s_tail = 0.f;
+#pragma unroll
+                for (int k = 0; k < G; ++k)
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) S[k][jj] = 0.f;
+                fence_proxy_async();  // this thread's writes to the stage, before the bulk copies read it
+                __syncwarp();
+                if (lane == 0) mbar_arrive(cbar);
+                if (!wait_inline(p, cbar, cpar, long_wait, 0xfffffff2u)) break;
+                cpar ^= 1u;
+                if (ctid == 0) {
+                    if (nv) {
+                        for (uint32_t j = 0; j < nd; ++j) bulk_store_part(s_cdst[slot][j] + (size_t)head * ed, smem_u32(out), nv * ed, false, 0);
+                        bulk_commit();
+                        bulk_wait_read(0);  // the stage is read out: it may be given away (this warp's arrival below)
+                    }
+                    if (pi.last && p.trace)
+                        for (uint32_t j = 0; j < nd; ++j) trace_put(p.trace, p.trace_cap, pi.item + j, 3, globaltimer_ns());
+                }
             } else {  // K_ITEM: the whole item through the register path; items of a chain follow each other in this block
                 // the item before must be stored by all compute threads. A bounded wait on an mbarrier, not a named barrier:
                 // a warp that has left an aborted execution would leave the others waiting at one for ever
@@ -287,7 +357,7 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                         st.flags = S_OK;
                         st.n = tl.count;
                         st.dt_a = d.dt_a; st.dt_b = d.dt_b; st.dt_dst = d.dt_dst;
-                        if (d.op == HCCL_OP_COPY) {
+                        if (COPIES && d.op == HCCL_OP_COPY) {
                             // a copy of what the step before stored (a ring's AllGather hops): the block stores what it holds again
                             f = t > 0 && d.ndst <= 1;
                             st.flags |= S_COPY;
@@ -403,17 +473,35 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
                             advance();
                         }
                         if (st.flags & S_COPY) {
+                            // all copies from here on (nothing but copies follows a copy in a chain that got this far)
+                            const uint32_t m = min(L - t, MAX_CDST);
                             if (!acquire()) { ok = false; break; }
                             Piece& pc = s_info[slot];
-                            pc.kind = K_C;
                             pc.n = ne;
                             pc.item = st.item;
                             pc.dt_dst = st.dt_dst;
                             pc.last = (e0 + ne == n) ? 1 : 0;
                             pc.head = (uint8_t)head;
-                            pc.dst = st.dst + (size_t)e0 * esize(st.dt_dst);
+                            if (m < (st.dt_dst == HCCL_FP32 ? CM_MIN32 : CM_MIN16)) {  // one piece per copy, from the registers
+                                pc.kind = K_C;
+                                pc.dst = st.dst + (size_t)e0 * esize(st.dt_dst);
+                                mbar_arrive(full + 8 * slot);
+                                advance();
+                                continue;
+                            }
+                            pc.kind = K_CM;
+                            pc.ndst = (uint16_t)m;
+                            for (uint32_t j = 0; j < m; ++j) {
+                                s_cdst[slot][j] = s_step[t + j].dst + (size_t)e0 * esize(st.dt_dst);
+                                if (p.trace && e0 == 0 && j > 0) {
+                                    trace_put(p.trace, p.trace_cap, st.item + j, 0, (unsigned long long)(st.item + j) | ((unsigned long long)blockIdx.x << 32));
+                                    trace_put(p.trace, p.trace_cap, st.item + j, 1, globaltimer_ns());
+                                    trace_put(p.trace, p.trace_cap, st.item + j, 2, globaltimer_ns());
+                                }
+                            }
                             mbar_arrive(full + 8 * slot);
                             advance();
+                            t += m - 1;
                             continue;
                         }
                         if (!acquire()) { ok = false; break; }
@@ -464,6 +552,13 @@ __global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_
         }
     }
     leave(p, lean);
+}
+
+__global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t stage_bytes) {
+    executor_chain_body<true>(p, ns, stage_bytes);
+}
+__global__ void __launch_bounds__(32 + CTH, 1) hccl_executor_chain_sums(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t stage_bytes) {
+    executor_chain_body<false>(p, ns, stage_bytes);
 }
 
 }  // namespace hccl

@@ -63,6 +63,7 @@ __global__ void __launch_bounds__(512, 1) hccl_executor_bulk(const __grid_consta
 // static chains on the bulk copy unit: running sums forwarded from step to step in registers
 constexpr uint32_t CHAIN_SMEM_BYTES = 6 * 28672, CHAIN_PIECE_ELEMS = 14336, CHAIN_THREADS = 256;  // 6 stages of 16-bit pieces or 3 of FP32 pieces
 __global__ void __launch_bounds__(256, 1) hccl_executor_chain(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t stage_bytes);
+__global__ void __launch_bounds__(256, 1) hccl_executor_chain_sums(const __grid_constant__ ExecParams p, const uint32_t ns, const uint32_t stage_bytes);  // packets without copies
 __global__ void __launch_bounds__(512, 1) hccl_executor_resident(const __grid_constant__ ExecParams p, Doorbell* db,
                                                                   const unsigned long long idle_ns, const uint32_t first_epoch);
 __global__ void __launch_bounds__(512, 1) hccl_a2a_dynamic(const __grid_constant__ DynParams q);

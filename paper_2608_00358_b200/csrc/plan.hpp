@@ -53,6 +53,7 @@ struct hccl_plan {
     hccl::Layout layout{};
     // static chains (HCCL_FLAG_STATIC_CHAINS): tiles [c*chain_len, (c+1)*chain_len) form chain c, run in order by one block
     uint32_t chain_len = 0, n_chains = 0;
+    bool chain_copies = false;  // forwarding kernel: the packet has COPY items (the build that forwards them too)
     bool chain_wide = false;  // forwarding kernel: an FP32 operand arrives through the stages (3 stages of FP32 pieces instead of 6 of 16-bit ones)
     int buf_align = 1;                     // alignment every send/receive pointer must have (largest element read or written)
     hccl_plan_info_t info{};
