@@ -471,6 +471,8 @@ def headline_of(line: dict) -> dict:
     side = {}
     for key, short, field in (("3_reducescatter_r16_bf16_64Mi_ring", "c3_ring_ms", "ms"), ("3_reducescatter_r16_bf16_64Mi_ring_fused", "c3_fused_ms", "ms"),
                               ("3_reducescatter_r16_bf16_64Mi_ring", "c3_beyond_1ulp", "beyond_1ulp_of_fp64_sum"),
+                              ("3_reducescatter_r16_bf16_64Mi_ring", "c3_ring_compulsory_gbs", "compulsory_gbs"),
+                              ("3_reducescatter_r16_bf16_64Mi_ring_fused", "c3_fused_compulsory_gbs", "compulsory_gbs"),
                               ("1_allreduce_ring_r4_fp32_1Mi", "c1_p50_us", "p50_us"), ("2_alltoallv_r8_bf16_dim128", "c2_p50_us", "p50_us"),
                               ("5_allreduce_r8_bf16_4096B_oneshot", "c5_4k_oneshot_p50_us", "p50_us"),
                               ("5_allreduce_r8_bf16_1048576B_oneshot", "c5_1m_oneshot_p50_us", "p50_us"),
