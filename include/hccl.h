@@ -477,7 +477,7 @@ typedef struct {
     int64_t scratch_bytes;
     int64_t send_bytes_total, recv_bytes_total; /* declared extents */
     int32_t R, sm_budget, threads, engine;
-    int64_t tile_bytes;
+    int64_t tile_bytes;       /* the largest work item cut, in bytes of its widest operand */
     int64_t epoch;            /* executions enqueued since the last bind */
     int64_t crossrack_bytes;  /* bytes that data WQEs move between ranks of different racks (racks of opts.rack_size):
                                  what would cross the scale-out network with real ranks (Sec. II-A.3, V-D) */

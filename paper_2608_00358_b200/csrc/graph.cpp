@@ -564,7 +564,13 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
     I.sm_budget = p->opts.sm_budget;
     I.threads = p->opts.threads;
     I.engine = p->opts.engine;
-    I.tile_bytes = (int64_t)tile_bytes;
+    // the largest work item actually cut, in bytes of its widest operand (planners set tile sizes per WQE)
+    int64_t widest_tile = 0;
+    for (size_t i = 0; i < n; ++i) {
+        const hccl_wqe_t& w = g->wqes[i].w;
+        if (tcount[i] > 0) widest_tile = std::max<int64_t>(widest_tile, std::min<int64_t>(tcount[i], w.count) * widest(w) * (w.op == HCCL_OP_REDUCE_N ? std::max<int>(w.nsrc, 1) : 1));
+    }
+    I.tile_bytes = widest_tile > 0 ? widest_tile : (int64_t)tile_bytes;
     I.crossrack_bytes = crossrack;
     I.static_chains = (int64_t)p->n_chains;
     *out = p;
