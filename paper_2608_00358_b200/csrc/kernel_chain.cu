@@ -398,7 +398,7 @@ __device__ __forceinline__ void executor_chain_body(const ExecParams& p, const u
                 const uint32_t copies = __ballot_sync(0xffffffffu, t < L && (s_step[t].flags & S_COPY));
                 if (copies && first_copy == L) first_copy = t0 + (uint32_t)__ffs((int)copies) - 1u;
             }
-            if (first_copy == 0) fast = false;
+            if (first_copy == 0 || (first_copy < L && L - first_copy > MAX_CDST)) fast = false;  // (a K_CM piece takes all copies of a chain)
             const uint32_t held_dt = first_copy >= 1 && first_copy < L ? s_step[first_copy - 1].dt_dst : 0;  // type of what the copies move
             const uint32_t held_n = first_copy >= 1 && first_copy < L ? s_step[first_copy - 1].n : 0;
             __syncwarp();
@@ -482,7 +482,8 @@ __device__ __forceinline__ void executor_chain_body(const ExecParams& p, const u
                             pc.dt_dst = st.dt_dst;
                             pc.last = (e0 + ne == n) ? 1 : 0;
                             pc.head = (uint8_t)head;
-                            if (m < (st.dt_dst == HCCL_FP32 ? CM_MIN32 : CM_MIN16)) {  // one piece per copy, from the registers
+                            // one piece per copy, from the registers: few copies, or values wider than the stages were sized for
+                            if (m < (st.dt_dst == HCCL_FP32 ? CM_MIN32 : CM_MIN16) || PIECE * esize(st.dt_dst) > stage_bytes) {
                                 pc.kind = K_C;
                                 pc.dst = st.dst + (size_t)e0 * esize(st.dt_dst);
                                 mbar_arrive(full + 8 * slot);

@@ -120,3 +120,39 @@ def test_trace_of_a_forwarded_ring_is_complete():
     assert (rows[:, 1] != 0).all() and (rows[:, 3] >= rows[:, 1]).all()      # every item was claimed and finished
     assert ((rows[:, 0] & 0xffffffff) == np.arange(p.info().n_tiles)).all()
     p.set_trace(0, 0)
+
+
+def test_hand_built_chains_with_copies_wider_than_the_stages():
+    """A work packet built WQE by WQE: two chains of bf16 + bf16 -> FP32 (scratch) -> + bf16 -> FP32 (receive buffer of rank 0),
+    followed by 13 copies of that FP32 result round the ranks. The stages are sized for the 16-bit operands, so the FP32
+    copies must go out from the registers although there are enough of them for the staged form. Against numpy."""
+    import torch
+    from paper_2608_00358_b200.runtime import DeviceCollective
+    R, n = 14, 2 * 14336 + 1000                      # elements per chain: two whole pieces and a ragged third
+    es, T = 2, 20000                               # tiles of 20000 elements: a whole piece and a part of one
+    g = hb.Graph(R, [2 * n * es] * R, [2 * n * 4] * R, scratch_bytes=2 * n * 4)
+    dep = hb.DEP_WQE_SYNC | hb.DEP_ELEMENTWISE
+    for c in range(2):
+        sg = g.add_subgraph(c)
+        so, fo = c * n * es, c * n * 4
+        w = g.add_wqe(sg, hb.OP_REDUCE, dst=(hb.BUF_SCRATCH, 0, fo), a=(hb.BUF_SEND, 0, so), b=(hb.BUF_SEND, 1, so), count=n,
+                      dtypes=(hb.FP32, hb.BF16, hb.BF16), tile_count=T)
+        w = g.add_wqe(sg, hb.OP_REDUCE, dst=(hb.BUF_RECV, 0, fo), a=(hb.BUF_SCRATCH, 0, fo), b=(hb.BUF_SEND, 2, so), count=n,
+                      dtypes=(hb.FP32, hb.FP32, hb.BF16), dep_flags=dep, dep_wqe=w, tile_count=T)
+        for r in range(1, R):
+            w = g.add_wqe(sg, hb.OP_COPY, dst=(hb.BUF_RECV, r, fo), a=(hb.BUF_RECV, r - 1, fo), count=n * 4, dep_flags=dep, dep_wqe=w, tile_count=T * 4)
+    p = g.compile(dict(engine=hb.ENGINE_BULK, flags=hb.FLAG_STATIC_CHAINS, sm_budget=3))
+    assert p.info().static_chains > 0 and p.info().n_syncs == 0 and p.check_hazards() == 0
+    X = synth.normal_ranks(R, 2 * n, hb.BF16, seed=41)
+    send = [torch.from_numpy(x.view(np.int16)).cuda() for x in X]
+    recv = [torch.zeros(2 * n, dtype=torch.float32, device="cuda") for _ in range(R)]
+    dc = DeviceCollective(p)
+    dc.set_buffers([t.data_ptr() for t in send], [t.data_ptr() for t in recv])
+    for _ in range(2):
+        dc.execute()
+    torch.cuda.synchronize()
+    dc.check()
+    f = [(x.astype(np.uint32) << 16).view(np.float32) for x in X[:3]]
+    want = (f[0] + f[1]) + f[2]
+    for r in range(R):
+        assert np.array_equal(recv[r].cpu().numpy().view(np.uint32), want.view(np.uint32)), r
