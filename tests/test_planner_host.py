@@ -352,6 +352,20 @@ def test_engine_left_to_the_library_for_rings():
     assert hb.hccl_plan_allreduce(8, 1 << 22, hb.BF16, hb.ALGO_RING, dict(flags=hb.FLAG_LEVEL_MAJOR)).info().engine == hb.ENGINE_LSU   # another issue order: as before
 
 
+def test_forwarding_tiles_fill_the_blocks():
+    """Tile choice for the forwarding kernel: one round of the 148 blocks where the ring is small enough for that,
+    many chains of one or two pieces per tile where it is large; every chain has a scratch slot of its own."""
+    c1 = hb.hccl_plan_allreduce(4, 1 << 20, hb.FP32, hb.ALGO_RING).info()                    # config 1
+    assert c1.engine == hb.ENGINE_BULK and c1.static_chains == 148 and c1.n_tiles == 148 * 6 and c1.scratch_bytes == 0
+    c3 = hb.hccl_plan_reducescatter(16, None, 1 << 26, hb.BF16, hb.ALGO_RING).info()           # config 3
+    assert c3.engine == hb.ENGINE_BULK and c3.static_chains >= 8 * 148 and c3.n_tiles == c3.static_chains * 15
+    assert c3.tile_bytes <= 2 * 14336 * 4 and c3.scratch_bytes == (1 << 26) * 4                # at most two pieces per tile; a slot per chain
+    mid = hb.hccl_plan_allreduce(16, 1 << 21, hb.BF16, hb.ALGO_RING).info()
+    assert mid.engine == hb.ENGINE_BULK and 74 <= mid.static_chains <= 148                     # one round
+    few = hb.hccl_plan_allreduce(16, 1 << 21, hb.BF16, hb.ALGO_RING, dict(sm_budget=8)).info()
+    assert few.sm_budget == 8 and few.static_chains >= 8
+
+
 # ----------------------------------------------------------------- static chains (a chain of tiles stays in one block)
 @pytest.mark.parametrize("dt", DTYPES)
 @pytest.mark.parametrize("algo", [hb.ALGO_RING, hb.ALGO_RING_FUSED])
