@@ -142,7 +142,8 @@ typedef struct {
                                the FP32 partials take at most 32 MiB (AllReduce rings: 48 MiB), else as many as keep one
                                group-step's partials at 64 MiB, half the L2 (16 for 2 MiB granules of 16-bit data) */
     int32_t threads;        /* threads per block, multiple of 32. Register engine: one control warp + workers (default 512,
-                               at least 64). Bulk engine: DMA, control and publishing warps + compute warps (default 352, at least 128) */
+                               at least 64). Bulk engine: DMA, control and publishing warps + compute warps (default 352, at least 128);
+                               its forwarding kernel (static chains) always runs 256 threads and its own stages */
     int32_t stages;         /* bulk engine: shared-memory stages per block, 2..8 (default: 4 of 48 KiB; copy-only plans on 100 blocks
                                or more: 3, since the memory is then the limit and fewer bytes in flight per block serve it better) */
     int32_t cluster;        /* register engine: launch blocks in clusters of this size (2, 4, 8) so that they sit on
