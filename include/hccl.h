@@ -117,7 +117,7 @@ typedef enum {
                                       stands where a device counter and a poll across SMs would. Ignored when the
                                       packet has another shape. On the bulk engine only packets of simple chains
                                       (one predecessor, one successor) of REDUCE items, optionally followed by
-                                      plain copies, run this way, in the forwarding kernel: a block walks a piece of
+                                      plain copies, or of copies of one send-buffer range, run this way, in the forwarding kernel: a block walks a piece of
                                       14336 elements through all steps of its chain with the running FP32 sums in
                                       registers; every step's result is stored where its descriptor says, none is
                                       read back. The planners ask for it themselves where it pays (rings with about

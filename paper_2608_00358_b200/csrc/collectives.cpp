@@ -907,12 +907,22 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     if (algo != HCCL_ALGO_RING && algo != HCCL_ALGO_ONESHOT && algo != HCCL_ALGO_RING_2LEVEL && algo != HCCL_ALGO_FANOUT) return HCCL_ERR_INVALID_ARG;
     hccl_opts_t o;
     if ((algo == HCCL_ALGO_RING || algo == HCCL_ALGO_RING_2LEVEL) && (!opts || opts->engine == HCCL_ENGINE_AUTO)) {
-        // hop-by-hop copies wait on one another item by item: the register engine hands a finished item on
-        // sooner than the bulk engine can (which must drain its stores first); measured ahead or level at
-        // R = 128 from 8 KiB to 4 MiB per rank
+        // hop-by-hop copies wait on one another item by item: through tickets the register engine hands a finished item
+        // on sooner than the bulk engine can (which must drain its stores first). The flat ring's chains of copies run in
+        // the forwarding kernel of the bulk engine instead (a piece is loaded once and stored to every hop's destination:
+        // R = 128 x 8 KiB per rank 0.040 vs 0.109 ms on the register engine's static chains, x 512 KiB 1.51 vs 1.70 ms, x 4 MiB
+        // 11.6 vs 11.5 ms; R = 16 x 2 MiB 0.104 vs 0.153 ms), if every block starts on a 16-byte boundary of the receive buffers
+        // (else its chains would run item by item there).
+        const int es0 = elem_bytes(dt);
+        bool aligned = algo == HCCL_ALGO_RING && !(opts && (opts->flags & HCCL_FLAG_DYNAMIC_TICKETS));
+        int64_t off = 0;
+        for (int r = 0; r < R && aligned; ++r) {
+            if ((off * es0) % 16) aligned = false;
+            off += sendcounts ? sendcounts[r] : count;
+        }
         hccl_opts_t tmp;
         if (opts) tmp = *opts; else std::memset(&tmp, 0, sizeof(tmp));
-        tmp.engine = HCCL_ENGINE_LSU;
+        tmp.engine = aligned ? HCCL_ENGINE_BULK : HCCL_ENGINE_LSU;
         fill_default_opts(&o, &tmp);
     } else {
         fill_copy_opts(&o, opts);
@@ -938,7 +948,9 @@ hccl_status_t hccl_plan_allgather(int R, const int64_t* sendcounts, int64_t coun
     // hop-by-hop copies on the register engine: at most three passes of the block's threads per tile (180 KiB),
     // which keeps what a block has just written (and reads next) inside the L2 (12.5 vs 14.0 ms at R = 128, 4 MiB)
     const int64_t tile_cap = (algo == HCCL_ALGO_RING && o.engine == HCCL_ENGINE_LSU) ? 3 * sweep_of(o, HCCL_OP_COPY) : (256 << 10);
-    const int64_t tile = o.tile_bytes ? (int64_t)o.tile_bytes : default_tile(offs[R] * es, o.sm_budget, 1, 16 << 10, tile_cap, sweep_of(o, HCCL_OP_COPY));
+    int64_t tile = o.tile_bytes ? (int64_t)o.tile_bytes : default_tile(offs[R] * es, o.sm_budget, 1, 16 << 10, tile_cap, sweep_of(o, HCCL_OP_COPY));
+    // the forwarding kernel moves 28 KiB per piece: at most two pieces per tile (more chains to share out)
+    if (!o.tile_bytes && algo == HCCL_ALGO_RING && o.engine == HCCL_ENGINE_BULK && !(o.flags & HCCL_FLAG_DYNAMIC_TICKETS)) tile = std::min<int64_t>(tile, 2 * 28672);
     // one subgraph per chunk q: it first lands in its owner's receive buffer, then goes round (ring)
     // or is read by everyone directly (one-shot)
     std::vector<int32_t> sg(R);

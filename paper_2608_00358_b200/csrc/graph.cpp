@@ -399,15 +399,12 @@ hccl_status_t hccl::compile_graph(const hccl_graph* g, const hccl_opts_t* opts_i
         for (int64_t q : pe[i]) depth[i] = std::max(depth[i], depth[q] + 1);
         max_depth = std::max(max_depth, depth[i]);
     }
-    // On the bulk engine static chains run in the forwarding kernel, which is built for chains of REDUCE items followed by plain copies (anything
+    // On the bulk engine static chains run in the forwarding kernel, which is built for chains of REDUCE items followed by plain copies, and for chains of copies of one source (anything
     // else it runs item by item through its few compute warps): only packets made of such items go there.
     bool chains = (p->opts.flags & HCCL_FLAG_STATIC_CHAINS) != 0 && n > 0 && max_depth > 1;
     if (chains && p->opts.engine != HCCL_ENGINE_LSU) {
         // ... and only simple chains (a ring's): one predecessor, one successor
         std::vector<int> successors(n, 0);
-        bool any_reduce = false;  // chains of copies alone gain nothing there: they stay with the tickets
-        for (size_t j = 0; j < n; ++j) any_reduce = any_reduce || g->wqes[j].w.op == HCCL_OP_REDUCE;
-        if (!any_reduce) chains = false;
         for (size_t j = 0; j < n && chains; ++j) {
             const hccl_wqe_t& w = g->wqes[j].w;
             if (w.op != HCCL_OP_REDUCE && !(w.op == HCCL_OP_COPY && wqe_ndst(w) <= 1)) chains = false;

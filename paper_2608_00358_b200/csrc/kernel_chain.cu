@@ -32,7 +32,7 @@ constexpr uint32_t MAX_NS = 6;               // stages: 6 of PIECE * 2 bytes (16
 constexpr uint32_t MAX_CDST = 256;           // destinations of one K_C piece: a chain's copies are stored one after the other by one piece
 constexpr uint32_t MAX_STEPS = 512;          // items per chain that fit the step table (2 R - 2 for R = 256: 510)
 
-enum : uint32_t { K_A = 0, K_B = 1, K_ITEM = 2, K_EXIT = 3, K_C = 4, K_CM = 5 };
+enum : uint32_t { K_A = 0, K_B = 1, K_ITEM = 2, K_EXIT = 3, K_C = 4, K_CM = 5, K_RM = 6 };
 constexpr uint32_t CM_MIN16 = 6, CM_MIN32 = 12;  // from this many copies on (16-bit / FP32 values), a chain's copies go out as one K_CM piece
 struct alignas(16) Piece {
     char* dst;                  // K_B: where this piece's sums go; K_C: where the held values are copied to (K_CM: the stage's
@@ -278,6 +278,22 @@ __device__ __forceinline__ void executor_chain_body(const ExecParams& p, const u
                     if (pi.last && p.trace)
                         for (uint32_t j = 0; j < nd; ++j) trace_put(p.trace, p.trace_cap, pi.item + j, 3, globaltimer_ns());
                 }
+            } else if (COPIES && pi.kind == K_RM) {
+                // a piece of a chain of copies: the stage holds the source's bytes; one thread stores it to every destination
+                const uint32_t nd = pi.ndst, hb = pi.head, nvb = (pi.n - hb) & ~15u, eb = pi.n - nvb, bi = ctid < hb ? ctid : nvb + ctid;
+                if (ctid < eb) {
+                    const char v = __ldcg(pi.src0 + bi);
+                    for (uint32_t j = 0; j < nd; ++j) s_cdst[slot][j][bi] = v;
+                }
+                if (ctid == 0) {
+                    if (nvb) {
+                        for (uint32_t j = 0; j < nd; ++j) bulk_store_part(s_cdst[slot][j] + hb, smem_u32(stage), nvb, false, 0);
+                        bulk_commit();
+                        bulk_wait_read(0);
+                    }
+                    if (pi.last && p.trace)
+                        for (uint32_t j = 0; j < nd; ++j) trace_put(p.trace, p.trace_cap, pi.item + j, 3, globaltimer_ns());
+                }
             } else {  // K_ITEM: the whole item through the register path; items of a chain follow each other in this block
                 // the item before must be stored by all compute threads. A bounded wait on an mbarrier, not a named barrier:
                 // a warp that has left an aborted execution would leave the others waiting at one for ever
@@ -359,7 +375,8 @@ __device__ __forceinline__ void executor_chain_body(const ExecParams& p, const u
                         st.dt_a = d.dt_a; st.dt_b = d.dt_b; st.dt_dst = d.dt_dst;
                         if (COPIES && d.op == HCCL_OP_COPY) {
                             // a copy of what the step before stored (a ring's AllGather hops): the block stores what it holds again
-                            f = t > 0 && d.ndst <= 1;
+                            // ... or, at the head of a chain of copies alone, of a send buffer (a hop-by-hop AllGather): bytes, not values
+                            f = d.ndst <= 1 && (t > 0 || d.kind_a == HCCL_BUF_SEND);
                             st.flags |= S_COPY;
                             st.dst = buf_base(p, d.kind_dst, d.rank_dst) + d.off_dst + tl.start;
                             st.a = buf_base(p, d.kind_a, d.rank_a) + d.off_a + tl.start;
@@ -388,6 +405,7 @@ __device__ __forceinline__ void executor_chain_body(const ExecParams& p, const u
             fast = fast && __all_sync(0xffffffffu, f);
         }
         __syncwarp();
+        bool raw_chain = false;
         if (good && fast) {
             // Every step after the first must take exactly what the step before stored: sums first (each takes an FP32 sum),
             // then copies of what the block holds, whose element type is that of the last sum's result. Checked by all lanes,
@@ -398,14 +416,20 @@ __device__ __forceinline__ void executor_chain_body(const ExecParams& p, const u
                 const uint32_t copies = __ballot_sync(0xffffffffu, t < L && (s_step[t].flags & S_COPY));
                 if (copies && first_copy == L) first_copy = t0 + (uint32_t)__ffs((int)copies) - 1u;
             }
-            if (first_copy == 0 || (first_copy < L && L - first_copy > MAX_CDST)) fast = false;  // (a K_CM piece takes all copies of a chain)
+            if (first_copy < L && L - first_copy > MAX_CDST) fast = false;  // (one piece takes all copies of a chain)
+            const bool raw = first_copy == 0;  // copies alone: the bytes of the first source go to every destination
+            raw_chain = raw;
             const uint32_t held_dt = first_copy >= 1 && first_copy < L ? s_step[first_copy - 1].dt_dst : 0;  // type of what the copies move
             const uint32_t held_n = first_copy >= 1 && first_copy < L ? s_step[first_copy - 1].n : 0;
             __syncwarp();
             for (uint32_t t0 = 0; t0 < L && fast; t0 += 32) {
                 const uint32_t t = t0 + lane;
                 bool f = true;
-                if (t >= 1 && t < L) {
+                if (raw && t < L) {
+                    const Step& st = s_step[t];
+                    f = (st.flags & S_COPY) && (((uintptr_t)st.dst ^ (uintptr_t)s_step[0].a) & 15u) == 0 && st.n == s_step[0].n &&
+                        (t == 0 || st.a == s_step[t - 1].dst);
+                } else if (t >= 1 && t < L) {
                     Step& st = s_step[t];
                     const Step& pv = s_step[t - 1];  // only fields that no lane rewrites are read from it (dst; for a sum also dt_dst, n)
                     f = st.a == pv.dst;
@@ -440,6 +464,37 @@ __device__ __forceinline__ void executor_chain_body(const ExecParams& p, const u
                         trace_put(p.trace, p.trace_cap, base + t, 2, globaltimer_ns());
                     }
                     mbar_arrive(full + 8 * slot);
+                    advance();
+                }
+            } else if (raw_chain) {
+                // copies alone: a piece of the first source is loaded into a stage once and stored from there to the destination of
+                // every copy of the chain (bytes as they are; the few before the first and behind the last 16-byte word by plain accesses)
+                const uint32_t nb = s_step[0].n, hb0 = (16u - (uint32_t)((uintptr_t)s_step[0].a & 15u)) & 15u;
+                for (uint32_t e0 = 0; e0 < nb && ok; e0 += stage_bytes) {
+                    const uint32_t ne = min(stage_bytes, nb - e0), head = min(hb0, ne), nvb = (ne - head) & ~15u;
+                    if (!acquire()) { ok = false; break; }
+                    Piece& pr = s_info[slot];
+                    pr.kind = K_RM;
+                    pr.n = ne;
+                    pr.item = s_step[0].item;
+                    pr.head = (uint8_t)head;
+                    pr.last = (e0 + ne == nb) ? 1 : 0;
+                    pr.ndst = (uint16_t)L;
+                    pr.src0 = s_step[0].a + e0;
+                    for (uint32_t j = 0; j < L; ++j) {
+                        s_cdst[slot][j] = s_step[j].dst + e0;
+                        if (p.trace && e0 == 0) {
+                            trace_put(p.trace, p.trace_cap, s_step[j].item, 0, (unsigned long long)s_step[j].item | ((unsigned long long)blockIdx.x << 32));
+                            trace_put(p.trace, p.trace_cap, s_step[j].item, 1, globaltimer_ns());
+                            trace_put(p.trace, p.trace_cap, s_step[j].item, 2, globaltimer_ns());
+                        }
+                    }
+                    if (nvb) {
+                        mbar_arrive_expect_tx(full + 8 * slot, nvb);
+                        bulk_load(stages + slot * stage_bytes, s_step[0].a + e0 + head, nvb, full + 8 * slot, true, pol);
+                    } else {
+                        mbar_arrive(full + 8 * slot);
+                    }
                     advance();
                 }
             } else {

@@ -338,8 +338,13 @@ def test_bulk_engine_rings_are_independent_chains_with_a_slot_each(dt):
     Y = interpret(p, X, 2)
     for r, w in enumerate(orc.reducescatter_ring_f32(dt, X, np.diff(orc.floor_chunk_offsets(n, R)))):
         assert np.array_equal(Y[r].view(np.uint8), w.view(np.uint8))
-    # what is not a set of simple REDUCE-then-COPY chains keeps tickets and counters on this engine
-    assert hb.hccl_plan_allgather(R, None, 777, dt, hb.ALGO_RING, opts).info().static_chains == 0
+    # a hop-by-hop AllGather is a set of chains of copies of one source each: forwarded too
+    pg = hb.hccl_plan_allgather(R, None, 776, dt, hb.ALGO_RING, opts)
+    assert pg.info().static_chains > 0 and pg.info().n_syncs == 0 and pg.check_hazards() == 0
+    Xg = [x[:776] for x in X]
+    for r, w in enumerate(orc.allgatherv(Xg)):
+        assert np.array_equal(interpret(pg, Xg, 4)[r].view(np.uint8), w.view(np.uint8))
+    # what is not a set of simple chains keeps tickets and counters on this engine
     assert hb.hccl_plan_allreduce(8, 4099, dt, hb.ALGO_TREE, dict(opts, flags=hb.FLAG_STATIC_CHAINS)).info().static_chains == 0
 
 
