@@ -156,3 +156,28 @@ def test_hand_built_chains_with_copies_wider_than_the_stages():
     want = (f[0] + f[1]) + f[2]
     for r in range(R):
         assert np.array_equal(recv[r].cpu().numpy().view(np.uint32), want.view(np.uint32)), r
+
+
+def test_hop_by_hop_allgather_forwarded_as_bytes():
+    """A flat-ring AllGather is a set of chains of copies of one source each: a piece is loaded once and stored to every
+    hop's destination. Equal blocks, blocks of different (16-byte aligned) sizes, 256 ranks (256 copies per chain: the
+    most one piece can take), and a block size off the 16-byte grid (then the library keeps the register engine)."""
+    for dt in DTYPES:
+        es = hb.ELEM_BYTES[dt]
+        for R, counts in ((5, None), (7, [8 * (3 + 5 * r) for r in range(7)]), (6, [0, 64, 8, 0, 40000, 16])):
+            n = 30008 if counts is None else None
+            X = [synth.normal_ranks(1, (n if counts is None else max(counts[r], 1)), dt, seed=50 + r)[0][:(n if counts is None else counts[r])] for r in range(R)]
+            p = hb.hccl_plan_allgather(R, counts, n or 0, dt, hb.ALGO_RING)
+            assert p.info().engine == hb.ENGINE_BULK and p.info().static_chains > 0 and p.info().n_syncs == 0 and p.check_hazards() == 0
+            Y = run_plan(p, X, iters=2)
+            for r, w in enumerate(orc.allgatherv(X)):
+                assert np.array_equal(Y[r].view(np.uint8)[:w.view(np.uint8).size], w.view(np.uint8)), (dt, R, r)
+        assert hb.hccl_plan_allgather(4, None, 1001, dt, hb.ALGO_RING).info().engine == (hb.ENGINE_BULK if (1001 * es) % 16 == 0 else hb.ENGINE_LSU)
+    R, n = 256, 72
+    X = [synth.normal_ranks(1, n, hb.BF16, seed=r)[0] for r in range(R)]
+    p = hb.hccl_plan_allgather(R, None, n, hb.BF16, hb.ALGO_RING, dict(sm_budget=32))
+    assert p.info().engine == hb.ENGINE_BULK and p.info().static_chains > 0
+    Y = run_plan(p, X)
+    want = orc.allgatherv(X)
+    for r in (0, 1, 128, 255):
+        assert np.array_equal(Y[r].view(np.uint8)[:want[r].view(np.uint8).size], want[r].view(np.uint8)), r
