@@ -106,3 +106,46 @@ def test_random_reducescatter(seed):
         want = orc.reducescatter_ring_f32(dt, X, np.array(counts, dtype=np.int64))
     for r in range(R):
         assert np.array_equal(Y[r].view(np.uint8), want[r].view(np.uint8)), (seed, R, counts, dt, algo, o, r)
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_random_forwarded_rings(seed):
+    """Rings on the bulk engine with static chains (the forwarding kernel) at sizes of several pieces per chunk: random
+    rank counts, ragged counts, operand misalignment, tile sizes and block counts; ReduceScatter with uneven shards
+    (shards off the 16-byte grid run item by item inside the same kernel), AllReduce and AllGather with aligned blocks."""
+    rng = np.random.default_rng(4000 + seed)
+    R = int(rng.integers(2, 20))
+    dt = int(rng.choice([hb.FP32, hb.BF16, hb.FP16]))
+    o = dict(engine=hb.ENGINE_BULK, sm_budget=int(rng.choice([1, 3, 16, 148])))
+    if rng.random() < 0.6:
+        o["tile_bytes"] = int(rng.choice([4096, 28672, 57344, 100000, 262144]))
+    if rng.random() < 0.4:
+        o["chunk_bytes"] = int(rng.choice([4096, 65536, 1 << 20]))
+    mis = int(rng.choice([0, 0, 4, 8, 12])) if dt == hb.FP32 else int(rng.choice([0, 0, 2, 6, 10]))
+    kind = int(rng.integers(0, 3))
+    if kind == 0:
+        n = int(rng.integers(1, 600000))
+        X = synth.normal_ranks(R, n, dt, seed=seed)
+        p = hb.hccl_plan_allreduce(R, n, dt, hb.ALGO_RING, o)
+        want = orc.allreduce_ring_f32(dt, X, orc.floor_chunk_offsets(n, R))
+    elif kind == 1:
+        grid = int(rng.choice([1, 8]))
+        counts = [grid * int(c) for c in rng.integers(0, 60000 // grid, size=R)]
+        if rng.random() < 0.3:
+            counts[int(rng.integers(0, R))] = 0
+        n = max(sum(counts), 1)
+        X = [x[:sum(counts)] for x in synth.normal_ranks(R, n, dt, seed=seed)]
+        p = hb.hccl_plan_reducescatter(R, counts, sum(counts), dt, hb.ALGO_RING, o)
+        want = orc.reducescatter_ring_f32(dt, X, np.array(counts, dtype=np.int64))
+        X = [x if x.size else np.zeros(8, np_dtype(dt)) for x in X]
+    else:
+        counts = [8 * int(c) for c in rng.integers(0, 9000, size=R)]
+        X = [synth.normal_ranks(1, max(c, 1), dt, seed=seed * 31 + r)[0][:c] for r, c in enumerate(counts)]
+        p = hb.hccl_plan_allgather(R, counts, 0, dt, hb.ALGO_RING, o)
+        want = orc.allgatherv(X)
+        X = [x if x.size else np.zeros(8, np_dtype(dt)) for x in X]
+    assert p.info().engine == hb.ENGINE_BULK and p.check_hazards() == 0
+    Y = run_plan(p, X, iters=2, misalign=mis)
+    for r in range(R):
+        w = want[r].view(np.uint8)
+        assert np.array_equal(Y[r][:w.size], w), (seed, kind, R, dt, o, mis, r)
