@@ -262,7 +262,7 @@ typedef enum {
                              COPY and REDUCE_N may name several destinations (ndst > 1): the same bytes are then
                              written at dst.offset into the receive buffer of every rank (dst.rank + k) mod R,
                              k < ndst, from one read of the sources. The NMC of the paper has no such form (its ranks do
-                             not share a memory); here it plays the part a multicast in the switch plays. */
+                             not share a memory); here it plays the part of a one-to-many send replicated inside the switch. */
     HCCL_OP_WAIT = 3,     /* block until signal slot a.offset compares true against value (+ epoch*value_per_epoch) */
     HCCL_OP_SET = 4,      /* store value (+ epoch*value_per_epoch) to signal slot dst.offset */
     HCCL_OP_NOOP = 5      /* nothing; exists to carry dependencies */
