@@ -418,7 +418,7 @@ def interference_leg(args, wl):
             "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
             "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
         del w2, plan, gemm
-    # the operating point: no SM is held against the GEMM. (1) interference.OVERLAP_OPTS: sixteen persistent blocks of the
+    # the operating point: no SM is held against the GEMM. (1) interference.OVERLAP_OPTS: twelve persistent blocks of the
     # register engine's 64-register build, 128 threads each, small enough to run on SMs that GEMM blocks occupy.
     # (2) interference.IDLE_SM_OPTS: short-lived blocks on a stream of LOWER priority than the GEMM's, which take only
     # the SMs the GEMM leaves idle. Slowdowns are still taken against the unrestricted GEMM alone.
@@ -432,7 +432,7 @@ def interference_leg(args, wl):
         return {"opts": dict(opts), "gemm_slowdown": r.get("gemm_slowdown"), "gemm_alone_tflops": r["gemm_alone_tflops"],
                 "gemm_overlap_tflops": r["overlap"].get("gemm_tflops"), "collective_alone_gbs": r["collective_alone_gbs"],
                 "collective_overlap_gbs": r["overlap"].get("collective_gbs")}
-    out["chosen"] = dict(point(interference.OVERLAP_OPTS, True), mode="16 co-resident blocks (register engine, 64 registers, 128 threads)",
+    out["chosen"] = dict(point(interference.OVERLAP_OPTS, True), mode="%d co-resident blocks (register engine, 64 registers, 128 threads)" % interference.OVERLAP_OPTS["sm_budget"],
                          sm_budget=interference.OVERLAP_OPTS["sm_budget"])
     out["idle_sms"] = dict(point(interference.IDLE_SM_OPTS, False), mode="short-lived blocks, GEMM stream has priority")
     del gemm

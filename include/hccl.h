@@ -150,7 +150,7 @@ typedef struct {
                                neighbouring SMs; 0/1 = no clusters. Ignored unless it divides the block count. */
     int32_t light;          /* register engine: nonzero = the 64-register build (several blocks per SM). With 64-128 threads such a
                                block is small enough to be placed on an SM that a large compute kernel's block already occupies:
-                               16 of them moved 300 GB/s beside a saturating bf16 GEMM for 3.4-4.3 % of its rate, where two
+                               12 of them moved 230-240 GB/s beside a saturating bf16 GEMM for 1.9-4.6 % of its rate (16: 300 GB/s for 2.8-5.6 %), where two
                                full-size blocks (two SMs held) cost it 6 % */
     int32_t copy_by_warps;  /* bulk engine: who stores COPY stages. 1 = the compute warps (a stage is free as soon as it is read;
                                best per-block rate), 2 = the bulk unit, 0 = compute warps below 100 blocks, bulk unit otherwise */
@@ -167,8 +167,8 @@ typedef struct {
 } hccl_opts_t;
 
 /* Fills *o with the options measured to let a collective run beside a saturating compute kernel for less than 5 % of
- * that kernel's rate (the overlap experiment of Sec. V-E; 8192^3 bf16 GEMM, AllToAllv of config 4: 3.4-4.3 % at
- * 300 GB/s): 16 persistent blocks of the register engine's 64-register build with 128 threads each, which are small
+ * that kernel's rate (the overlap experiment of Sec. V-E; 8192^3 bf16 GEMM, AllToAllv of config 4: 1.9-4.6 % at
+ * 230-240 GB/s over a dozen runs): 12 persistent blocks of the register engine's 64-register build with 128 threads each, which are small
  * enough to share an SM with a block of the compute kernel and so hold no SM against it. Every other field is zeroed
  * (defaults). The library's general defaults aim at a GPU of its own instead: one full-size block per SM. */
 void hccl_opts_for_overlap(hccl_opts_t* o);

@@ -681,7 +681,7 @@ void hccl_opts_for_overlap(hccl_opts_t* o) {
     o->engine = HCCL_ENGINE_LSU;
     o->light = 1;
     o->threads = 128;
-    o->sm_budget = 16;
+    o->sm_budget = 12;
 }
 
 }  // extern "C"

@@ -10,7 +10,7 @@ Run as a module for the SM-budget sweep and for the other ways of sharing the GP
     python -m paper_2608_00358_b200.interference --budgets 4,8,16,32,64,148 --cap 32768
     python -m paper_2608_00358_b200.interference --method idle_sms --quanta 1,2,4 --opts tile_bytes=122880
 
-OVERLAP_OPTS is the operating point measured to cost a saturating 8192^3 GEMM less than 5 %: sixteen persistent
+OVERLAP_OPTS is the operating point measured to cost a saturating 8192^3 GEMM less than 5 % in every run: twelve persistent
 blocks of the register engine's 64-register build with 128 threads each, which are small enough to run on SMs
 that GEMM blocks occupy (they hold no SM against the GEMM). IDLE_SM_OPTS is the other way of holding no SM:
 short-lived blocks (one work item of 120 KiB each) on a stream of lower priority than the GEMM's.
@@ -28,7 +28,7 @@ import torch
 from . import workloads as wk
 
 
-OVERLAP_OPTS = wk.hb.hccl_opts_for_overlap()      # engine = register, light = 1, threads = 128, sm_budget = 16
+OVERLAP_OPTS = wk.hb.hccl_opts_for_overlap()      # engine = register, light = 1, threads = 128, sm_budget = 12
 IDLE_SM_OPTS = dict(quantum=1, tile_bytes=122880)
 
 
@@ -175,12 +175,17 @@ class GreenPartition:
 def measure(wl: wk.Workload, seconds: float = 3.0, gemm: Optional[Gemm] = None, collective_first: bool = True, streams=None,
             alone_tflops: Optional[float] = None, discard: float = 1.0) -> dict:
     """GEMM slowdown = 1 - (GEMM rate beside the collective) / (rate of the UNRESTRICTED GEMM alone: default streams,
-    all SMs, no SM-count target). Pass `alone_tflops` when that figure was taken before a restriction was applied."""
+    all SMs, no SM-count target). Pass `alone_tflops` when that figure was taken before a restriction was applied.
+    Otherwise the GEMM alone is timed before AND after the overlapped run and the two are averaged: a GEMM at the
+    power limit drifts by a few per cent over seconds, which is the size of the effect that is measured here."""
     gemm = gemm or Gemm()
-    alone = dict(tflops=alone_tflops if alone_tflops is not None else overlap(gemm, None, seconds, discard)["gemm_tflops"])
+    before = alone_tflops if alone_tflops is not None else overlap(gemm, None, seconds, discard)["gemm_tflops"]
     coll_alone_ms = wk.time_back_to_back(wl, 5, 2)
     both = overlap(gemm, wl, seconds, discard, collective_first=collective_first, streams=streams)
-    res = dict(gemm_alone_tflops=alone["tflops"], collective_alone_ms=float(coll_alone_ms),
+    after = alone_tflops if alone_tflops is not None else overlap(gemm, None, seconds, discard)["gemm_tflops"]
+    alone = dict(tflops=0.5 * (before + after))
+    res = dict(gemm_alone_tflops=alone["tflops"], gemm_alone_before_after=[float(before), float(after)],
+               collective_alone_ms=float(coll_alone_ms),
                collective_alone_gbs=float(wl.info.schedule_bytes / coll_alone_ms / 1e6), overlap=both,
                sm_budget=int(wl.info.sm_budget))
     if "gemm_tflops" in both:

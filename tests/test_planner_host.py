@@ -25,9 +25,9 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(lib, name), name
     assert set(hb.EXPORTS) == declared
     assert lib.hccl_version() >= 100
-    assert hb.hccl_opts_for_overlap() == dict(engine=hb.ENGINE_LSU, light=1, threads=128, sm_budget=16)
+    assert hb.hccl_opts_for_overlap() == dict(engine=hb.ENGINE_LSU, light=1, threads=128, sm_budget=12)
     i = hb.hccl_plan_alltoallv(4, np.full((4, 4), 100), None, None, None, hb.BF16, 64, hb.hccl_opts_for_overlap()).info()
-    assert (i.engine, i.threads, i.sm_budget) == (hb.ENGINE_LSU, 128, 16)
+    assert (i.engine, i.threads, i.sm_budget) == (hb.ENGINE_LSU, 128, 12)
 
 
 def test_config1_plan_shape():
