@@ -223,7 +223,7 @@ def main():
     if args.method == "idle_sms":
         for q in [int(x) for x in args.quanta.split(",")]:
             wl = plan_for(quantum=q)
-            res = measure(wl, args.seconds, gemm, collective_first=False, alone_tflops=unrestricted)
+            res = measure(wl, args.seconds, gemm, collective_first=False)   # GEMM alone timed before and after
             res.update(method=args.method, quantum=q, opts=extra, gemm_n=args.gemm_n)
             print(json.dumps(res), flush=True)
         return
@@ -237,7 +237,9 @@ def main():
             wl = plan_for(sm_budget=b)
             if args.method in ("sm_target", "green_sm_target"):
                 target = set_sm_count_target(148 - b, streams[0] if streams else None)
-            res = measure(wl, args.seconds, gemm, streams=streams, alone_tflops=unrestricted, collective_first=not args.gemm_first)
+            # (a restricted GEMM is compared with the unrestricted one timed at the start; otherwise alone = before and after)
+            res = measure(wl, args.seconds, gemm, streams=streams, alone_tflops=None if args.method == "plain" else unrestricted,
+                          collective_first=not args.gemm_first)
             res.update(method=args.method, sm_count_target=target, opts=extra, gemm_n=args.gemm_n, gemm_first=bool(args.gemm_first))
             print(json.dumps(res), flush=True)
         finally:
