@@ -149,3 +149,55 @@ def test_random_forwarded_rings(seed):
     for r in range(R):
         w = want[r].view(np.uint8)
         assert np.array_equal(Y[r][:w.size], w), (seed, kind, R, dt, o, mis, r)
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_alltoallv(seed):
+    """AllToAllv with random rank counts, row sizes (rows that are and are not multiples of 16 bytes), count matrices
+    (uniform, mostly empty, one heavy pair), packed layouts and explicit displacements with gaps, engines, tile and
+    stage geometry, block counts, short-lived blocks and buffer misalignment; bit-exact against the oracle, guard
+    bands and the gaps between segments untouched."""
+    rng = np.random.default_rng(5000 + seed)
+    R = int(rng.integers(1, 25))
+    dt = int(rng.choice([hb.FP32, hb.BF16, hb.FP16]))
+    row_elems = int(rng.choice([1, 3, 7, 8, 64, 128, 250, 256]))
+    rb = row_elems * hb.ELEM_BYTES[dt]
+    hi = int(rng.choice([3, 40, 400])) if rb * R < 8000 else int(rng.choice([3, 40]))
+    C = rng.integers(0, hi + 1, size=(R, R)).astype(np.int64)
+    shape = int(rng.integers(0, 3))
+    if shape == 1:
+        C *= (rng.random((R, R)) < 0.2)
+    elif shape == 2:
+        C[int(rng.integers(0, R)), int(rng.integers(0, R))] = 20 * hi
+    packed = bool(rng.random() < 0.5)
+    if packed:
+        SD, RD = orc.packed_displs(C)
+        send_rows = C.sum(axis=1)
+    else:
+        # send segments may overlap each other (the same rows sent to several peers); receive segments are disjoint, with gaps
+        send_rows = np.full(R, int(C.sum(axis=1).max()) + 2)
+        SD = rng.integers(0, int(send_rows[0]) - int(C.max()) + 1, size=(R, R))
+        RD = np.zeros((R, R), dtype=np.int64)
+        for d in range(R):
+            o = int(rng.integers(0, 3))
+            for s in rng.permutation(R):
+                RD[d, s] = o
+                o += int(C[s, d]) + int(rng.integers(0, 3))
+    X = [rng.integers(0, 256, size=max(int(send_rows[s]) * rb, 16), dtype=np.uint8) for s in range(R)]
+    o = dict(sm_budget=int(rng.choice([1, 2, 5, 16, 148])), engine=int(rng.choice([0, hb.ENGINE_LSU, hb.ENGINE_BULK])))
+    if rng.random() < 0.6:
+        o["tile_bytes"] = int(rng.choice([256, 1000, 4096, 49152, 245760]))
+    if o["engine"] != hb.ENGINE_LSU and rng.random() < 0.4:
+        o.update(stage_kib=int(rng.choice([12, 24, 48, 96])), stages=int(rng.choice([0, 2, 3, 8])), copy_by_warps=int(rng.choice([0, 1, 2])))
+    if o["engine"] != hb.ENGINE_BULK and rng.random() < 0.2:
+        o.update(light=1, threads=int(rng.choice([64, 128, 256])))
+    if rng.random() < 0.2:
+        o["quantum"] = int(rng.choice([1, 3]))
+    mis = int(rng.choice([0, 0, 1, 2, 4, 8]))
+    p = hb.hccl_plan_alltoallv(R, C, None if packed else SD, C.T.copy(), None if packed else RD, dt, row_elems, o)
+    assert p.check_hazards() == 0
+    Y = run_plan(p, X, iters=2, misalign=mis)
+    Yw = [np.full(p.extents(r)[1], 0xA5, dtype=np.uint8) for r in range(R)]
+    orc.alltoallv([x[:int(send_rows[s]) * rb] for s, x in enumerate(X)], Yw, C, SD, RD, rb)
+    for r in range(R):
+        assert np.array_equal(Y[r], Yw[r]), (seed, R, dt, row_elems, packed, o, mis, r)
