@@ -347,3 +347,44 @@ def test_static_plan_gate_that_never_opens_times_out_cleanly(engine, R, flags):
     for t in recv:
         assert bool((t == 7.0).all())
     assert float(torch.ones(4, device="cuda").sum()) == 4.0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(16))
+def test_random_device_resident_alltoallv(seed):
+    """Random rank counts on both sides of the 64-rank boundary (one kernel with the count matrix in shared memory up to
+    64 ranks, device-built tables beyond), row sizes, engines, tiles and block counts; counts redrawn for each of three
+    executions of one bound plan (dense, sparse, skewed onto one destination), always within the buffers' capacity."""
+    import torch
+    rng = np.random.default_rng(7000 + seed)
+    R = int(rng.choice([1, 2, 5, 17, 40, 63, 64, 65, 90, 130, 200]))
+    row_elems = int(rng.choice([4, 7, 16, 64, 128]))
+    hi = int(rng.integers(2, max(3, 2400 // R)))
+    cap = hi * R + int(rng.integers(0, 4))
+    o = dict(sm_budget=int(rng.choice([1, 8, 24, 148])), tile_bytes=int(rng.choice([512, 2048, 4096, 16384])))
+    if rng.random() < 0.5:
+        o["engine"] = int(rng.choice([hb.ENGINE_LSU, hb.ENGINE_BULK]))
+    if R <= 64 and rng.random() < 0.5:
+        o["flags"] = hb.FLAG_DEVICE_TABLES
+    plan, dc, X, send, recv, counts, rc_out, rd_out, rb = _setup(R, row_elems, cap, opts=o)
+    for it in range(3):
+        C = rng.integers(0, hi + 1, size=(R, R)).astype(np.int64)
+        if it == 1:
+            C *= (rng.random((R, R)) < 0.15)
+        if it == 2:
+            d = int(rng.integers(0, R))
+            C[:] = 0
+            C[:, d] = rng.integers(0, hi + 1, size=R)      # everything goes to one destination
+        assert C.sum(axis=0).max() <= cap and C.sum(axis=1).max() <= cap
+        counts.copy_(torch.from_numpy(C.reshape(-1)))
+        for t in recv:
+            t.fill_(SENT)
+        dc.execute()
+        dc.check()
+        want, RD = _expect(X, C, rb, cap)
+        for d in range(R):
+            assert np.array_equal(recv[d].cpu().numpy(), want[d]), (seed, it, R, row_elems, o, d)
+        assert np.array_equal(rc_out.cpu().numpy().reshape(R, R), C.T)
+        assert np.array_equal(rd_out.cpu().numpy().reshape(R, R), RD)
+    for s_ in range(R):
+        assert np.array_equal(send[s_].cpu().numpy(), X[s_])
