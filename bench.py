@@ -454,7 +454,7 @@ def headline_of(line: dict) -> dict:
     e = line.get("e2e")
     if e:
         h["e2e"] = {k: e[k] for k in ("value", "unit", "h2d_bytes_per_step", "d2h_bytes_per_step", "ms_per_step", "gpu_launches_per_step",
-                                      "checked_destinations_vs_oracle", "skipped") if k in e}
+                                      "checked_destinations_vs_oracle", "skipped", "ranks_measured") if k in e}
         if "api" in e:
             h["e2e"]["api"] = e["api"].split(" ")[0]
     if "cpu_baseline" in line:
@@ -626,6 +626,8 @@ def run_ours(args, rank: int, world: int, local_rank: int):
                 return one_way / a0.elapsed_time(a1) / 1e6
             e2e["host_link_gbs"] = {"h2d_alone": _link(True, False), "d2h_alone": _link(False, True), "h2d_while_d2h_runs": _link(True, True),
                                     "note": "plain pinned copies of 16 of the 64 rank buffers; the pipelined path needs both directions at once"}
+            if world > 1:   # the other ranks idle meanwhile: this is one replica's end-to-end rate, not the job's
+                e2e["ranks_measured"] = 1
             del pipe, pws
             del hs, hr
         else:
